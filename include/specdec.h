@@ -1,0 +1,181 @@
+/*
+ * specdec.h -- C ABI of the B200 (sm_100a) SpecDec draft -> verify -> commit library.
+ *
+ * The library implements the hot path of Speculative Decoding for seq2seq
+ * generation: the Spec-Drafter's parallel pass over k [MASK] queries
+ * (Section 3.1.3, inference equation), the verification pass in which the
+ * autoregressive encoder-decoder Transformer scores all k drafts of every
+ * sequence at once (Section 2, Eq. 1-3), the Spec-Verification acceptance rule
+ * (Section 3.2, Eq. 7-9) and the loop that repeats draft -> verify -> commit
+ * until [EOS] (Section 2, last sentence; Appendix "Case Study").
+ *
+ * Conventions
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The caller
+ *     owns every buffer it passes; the library owns its arena (repacked weights,
+ *     paged KV cache, workspaces) from specdec_create to specdec_destroy.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls are asynchronous on it
+ *     unless stated otherwise; buffers must stay valid until the stream reaches
+ *     the end of the call.
+ *   - Every function returns SPECDEC_OK (0) or a negative error code; a message
+ *     is kept in the handle (specdec_last_error).  Nothing throws, exits or prints.
+ *   - One decoding session per handle at a time: specdec_encode starts it.
+ *   - Token ids are int32.  Row-major everywhere.
+ *   - There is no CPU fallback: without a CUDA device every compute call fails
+ *     with SPECDEC_ERR_CUDA.
+ */
+#ifndef SPECDEC_H
+#define SPECDEC_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPECDEC_OK                 0
+#define SPECDEC_ERR_INVALID_ARG   -1
+#define SPECDEC_ERR_SHAPE         -2   /* weight manifest does not match the dims        */
+#define SPECDEC_ERR_CAPACITY      -3   /* B / S / k / max_tgt beyond create-time limits  */
+#define SPECDEC_ERR_NOT_ENCODED   -4
+#define SPECDEC_ERR_CUDA          -5
+#define SPECDEC_ERR_TIMEOUT       -6   /* a bounded device-side wait gave up             */
+#define SPECDEC_ERR_UNSUPPORTED   -7
+
+#define SPECDEC_DTYPE_F32   0
+#define SPECDEC_DTYPE_BF16  1
+
+typedef struct specdec_handle specdec_handle;
+
+/* One encoder-decoder Transformer (pre-LN, ReLU, shared embedding table). */
+typedef struct {
+    int d_model, n_heads, d_ffn, vocab;
+    int enc_layers, dec_layers;
+    int max_pos;                       /* rows of the position tables */
+} specdec_model_dims;
+
+typedef struct {
+    specdec_model_dims verifier, drafter;
+    int k_max;                         /* largest draft block                                  */
+    int max_batch, max_src, max_tgt;   /* capacity limits of a session                         */
+    int page_tokens;                   /* tokens per KV-cache page (power of two)              */
+    int pad_id, bos_id, eos_id, mask_id;
+    int compute_dtype;                 /* SPECDEC_DTYPE_F32: fp32 operands (SIMT kernels);
+                                          SPECDEC_DTYPE_BF16: bf16 operands, fp32 accumulation
+                                          (tcgen05 tensor-core GEMMs)                          */
+} specdec_config;
+
+/* One named weight.  `d_ptr` is a DEVICE pointer to fp32 data, row-major.
+ * Names, per model prefix "verifier." / "drafter." (y = x W^T + b, W is [out,in]):
+ *   embed [V,d]   pos_enc, pos_dec [max_pos,d]
+ *   enc.{l}.ln1.{g,b}  enc.{l}.self.{q,k,v,o}.{w,b}  enc.{l}.ln2.{g,b}
+ *   enc.{l}.ffn.{w1,b1,w2,b2}   enc.ln_f.{g,b}
+ *   dec.{l}.ln1  dec.{l}.self.*  dec.{l}.ln_cross.{g,b}  dec.{l}.cross.{q,k,v,o}.{w,b}
+ *   dec.{l}.ln2  dec.{l}.ffn.*   dec.ln_f.{g,b}                                        */
+typedef struct {
+    const char* name;
+    const void* d_ptr;
+    int         dtype;                 /* SPECDEC_DTYPE_F32 only */
+    int         ndim;
+    long long   shape[4];
+} specdec_tensor;
+
+/* Counters of specdec_generate.  Tok. of the paper's latency model (Eq. 4) is
+ * accepted / seq_iterations (or emitted / seq_iterations counting the
+ * bifurcation token); t_d, t_v are ms_draft, ms_verify per iteration. */
+typedef struct {
+    long long iterations;              /* draft->verify->commit rounds launched               */
+    long long seq_iterations;          /* sum over rounds of sequences still decoding         */
+    long long drafted, accepted, emitted;
+    double    ms_encode, ms_draft, ms_verify, ms_commit, ms_total;
+    int       status;
+} specdec_stats;
+
+/* Builds a handle: validates the manifest against the dims, allocates the arena
+ * (the only device allocation the library makes), copies and repacks the weights
+ * (bf16 for SPECDEC_DTYPE_BF16).  Synchronises `stream` before returning, so the
+ * caller may free its weight buffers afterwards.  *out is NULL on failure; the
+ * reason is then available from specdec_last_error(NULL). */
+int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int n_weights,
+                   void* stream, specdec_handle** out);
+int specdec_destroy(specdec_handle* h);
+
+/* Starts a session: runs both encoders over the right-padded sources and caches
+ * the per-decoder-layer cross-attention K/V of both models ("the encoder is
+ * forwarded only once", Section 3.1.2).  All sequences start with no committed
+ * target token.  d_src [B,S_max] int32, d_src_len [B] (1..S_max), d_max_tgt [B]
+ * (0..max_tgt; NULL = max_tgt for all). */
+int specdec_encode(specdec_handle* h, const int32_t* d_src, const int32_t* d_src_len,
+                   const int32_t* d_max_tgt, int B, int S_max, void* stream);
+
+/* Spec-Drafter pass (Section 3.1.3): for every unfinished sequence, the decoder
+ * runs without a causal mask over [BOS, committed tokens, MASK x k] and the
+ * argmax (lowest id on ties) at each mask row becomes a draft.
+ * d_draft [B,k] int32 out; rows of finished sequences are left untouched. */
+int specdec_draft(specdec_handle* h, int k, int32_t* d_draft, void* stream);
+
+/* Verification pass (Section 2 Eq. 1-3, Section 3.2 Eq. 7-9): the verifier
+ * decoder scores the block [last committed token, k drafts] causally over the
+ * paged KV cache; draft i is accepted iff all earlier ones are, fewer than
+ * `beta` vocabulary entries score strictly higher (Eq. 7) and top-1 score minus
+ * its score <= tau (Eq. 8).  d_accepted [B] receives the accepted length in
+ * [0,k]; d_bif [B] the verifier's top-1 token on the row after the accepted
+ * prefix (the replacement at the bifurcation, or the bonus token when a = k).
+ * Does not commit.  beta >= 1, tau >= 0, 1 <= k <= k_max. */
+int specdec_verify(specdec_handle* h, const int32_t* d_draft, int k, int beta, float tau,
+                   int32_t* d_accepted, int32_t* d_bif, void* stream);
+
+/* Commit / rollback (Eq. 3): appends drafts[0..keep) and `next` to each
+ * unfinished sequence, cuts after the first [EOS] and at the sequence's max
+ * target length, marks finished sequences, and keeps only the KV-cache rows of
+ * the kept prefix.  d_keep / d_next [B] may be NULL: the results of the last
+ * specdec_verify are used.  Must follow a specdec_verify (it reuses its block). */
+int specdec_commit(specdec_handle* h, const int32_t* d_keep, const int32_t* d_next, void* stream);
+
+/* encode + (draft -> verify -> commit) until every sequence is finished.
+ * d_out [B,out_stride] int32 receives the generated ids (without BOS),
+ * d_out_len [B] their count.  h_stats may be NULL.  Synchronises `stream`. */
+int specdec_generate(specdec_handle* h, const int32_t* d_src, const int32_t* d_src_len,
+                     const int32_t* d_max_tgt, int B, int S_max, int k, int beta, float tau,
+                     int32_t* d_out, int out_stride, int32_t* d_out_len,
+                     specdec_stats* h_stats, void* stream);
+
+/* Same, with HOST buffers: the copies host->device (sources) and device->host
+ * (ids, lengths) are part of the call.  Pinned host memory avoids a staging copy. */
+int specdec_generate_host(specdec_handle* h, const int32_t* h_src, const int32_t* h_src_len,
+                          const int32_t* h_max_tgt, int B, int S_max, int k, int beta, float tau,
+                          int32_t* h_out, int out_stride, int32_t* h_out_len,
+                          specdec_stats* h_stats, void* stream);
+
+/* Current session state: committed ids [B,out_stride], lengths [B], finished flags [B]
+ * (any pointer may be NULL). */
+int specdec_get_output(specdec_handle* h, int32_t* d_out, int out_stride, int32_t* d_out_len,
+                       int32_t* d_finished, void* stream);
+
+/* The acceptance rule alone (Eq. 7-9) on caller-provided fp32 logits
+ * d_logits [B,k+1,V]: same outputs as specdec_verify.  No handle, no workspace. */
+int specdec_accept_scan(const float* d_logits, const int32_t* d_draft, int B, int k, int V,
+                        int beta, float tau, int32_t* d_accepted, int32_t* d_bif, void* stream);
+
+/* Debug / parity helpers (not on the hot path).
+ * specdec_debug_logits: re-runs the vocabulary projection of the last verify
+ *   (which = 0, rows [B*(k+1)]) or draft (which = 1, rows [n_active*k]) pass
+ *   unfused and stores fp32 logits [rows,V].
+ * specdec_debug_row_stats: per verify row of the last specdec_verify, 6 floats:
+ *   max logit, argmax id, log-sum-exp, count of entries above the draft's logit,
+ *   the draft's logit (+inf on the bonus row), draft id (-1 on the bonus row). */
+int specdec_debug_logits(specdec_handle* h, int which, float* d_logits, void* stream);
+int specdec_debug_row_stats(specdec_handle* h, float* d_stats, void* stream);
+
+/* Options: "gemm" = 0 SIMT reference GEMM, 1 tcgen05 GEMM (bf16 handles; default 1);
+ * "graphs" = 0/1 replay draft/verify steps from CUDA graphs inside specdec_generate. */
+int specdec_set_option(specdec_handle* h, const char* name, int value);
+
+/* Number of kernels the library has launched on this handle since create. */
+long long specdec_launch_count(const specdec_handle* h);
+
+const char* specdec_last_error(const specdec_handle* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECDEC_H */

@@ -1,0 +1,40 @@
+"""Builds the CUDA library in-tree for sm_100a with nvcc (no JIT cache, no GPU needed)."""
+from __future__ import annotations
+
+import os
+import subprocess
+import sys
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+SRC = os.path.join(HERE, "csrc", "specdec.cu")
+LIB = os.path.join(HERE, "libspecdec_b200.so")
+DEPS = [SRC] + [os.path.join(HERE, "csrc", f) for f in ("kernels.cuh", "gemm_tc.cuh")] + \
+       [os.path.join(os.path.dirname(HERE), "include", "specdec.h")]
+
+
+def needs_build() -> bool:
+    if not os.path.exists(LIB):
+        return True
+    t = os.path.getmtime(LIB)
+    return any(os.path.getmtime(p) > t for p in DEPS if os.path.exists(p))
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    if not force and not needs_build():
+        return LIB
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+           "--use_fast_math" if False else "-DSPECDEC_PRECISE_MATH", "-shared", "-Xcompiler", "-fPIC",
+           "-cudart", "static", "-o", LIB, SRC]
+    if verbose:
+        cmd.insert(1, "-Xptxas"); cmd.insert(2, "-v")
+    r = subprocess.run(cmd, capture_output=True, text=True)
+    if r.returncode != 0:
+        raise RuntimeError("nvcc failed:\n" + r.stdout + r.stderr)
+    if verbose:
+        print(r.stderr)
+    return LIB
+
+
+if __name__ == "__main__":
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

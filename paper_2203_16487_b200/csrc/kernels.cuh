@@ -1,0 +1,559 @@
+// Kernels of the SpecDec draft/verify path other than the tensor-core GEMM:
+// row preparation, embedding, layer norm, attention, the SIMT reference GEMM with
+// the shared epilogues, vocabulary row statistics, the acceptance scan and commit.
+// Every kernel takes its live row count from device memory and exits early past
+// it, so the host can launch worst-case grids without knowing per-sequence lengths.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <math_constants.h>
+
+namespace sd {
+
+typedef __nv_bfloat16 bf16;
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+// value as the operand type would hold it, back in fp32
+template <typename T> __device__ __forceinline__ float round_as(float v) { return to_f(from_f<T>(v)); }
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Device-resident session state shared by the kernels of one handle.
+struct Session {
+    int* len;          // [B] committed target tokens j_b
+    int* finished;     // [B]
+    int* max_tgt;      // [B]
+    int* src_len;      // [B]
+    int* out;          // [B, out_stride] committed ids
+    int out_stride;
+    int* counters;     // [8]: 0 rows of the drafter's full pass, 1 rows of its mask-only pass,
+                       //      2 verify rows, 3 encoder rows, 4 unfinished sequences
+    unsigned long long* stats;  // [4]: seq_iterations, drafted, accepted, emitted
+};
+enum { CNT_DRAFT_ALL = 0, CNT_DRAFT_MASK = 1, CNT_VERIFY = 2, CNT_ENC = 3, CNT_ACTIVE = 4 };
+
+// Per-row metadata of the pass being run.
+struct Rows {
+    int* tok;       // token id fed at the row
+    int* pos;       // position of the row
+    int* seq;       // sequence the row belongs to
+    int* nk_self;   // keys visible to the row in self-attention
+    int* nk_cross;  // keys visible in cross-attention (source length)
+    int* kv_off;    // [B] first K/V row of the sequence in a contiguous K/V buffer
+    int* kv_off_cross;  // [B]
+    int* src_row;   // mask-only pass: the row of the full pass this row continues
+    int* slot;      // mask-only pass: index into the [B,k] draft array
+};
+
+// ------------------------------------------------------------------ row preparation
+// Encoder: rows are the padded [B,S_max] grid.
+__global__ void k_enc_prep(const int* __restrict__ src, const int* __restrict__ src_len, int B, int S_max,
+                           Rows r, int* counters) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i == 0) counters[CNT_ENC] = B * S_max;
+    if (i < B) { r.kv_off[i] = i * S_max; r.kv_off_cross[i] = i * S_max; }
+    if (i >= B * S_max) return;
+    int b = i / S_max, t = i % S_max;
+    r.tok[i] = src[i];
+    r.pos[i] = t;
+    r.seq[i] = b;
+    r.nk_self[i] = src_len[b];
+    r.nk_cross[i] = src_len[b];
+}
+
+// Verify block: row b*(k+1)+i holds [last committed token (BOS if none), drafts] at positions j..j+k.
+__global__ void k_verify_prep(Session s, const int* __restrict__ draft, int B, int k, int S_max, int bos,
+                              Rows r) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i == 0) s.counters[CNT_VERIFY] = B * (k + 1);
+    if (i < B) r.kv_off_cross[i] = i * S_max;
+    if (i >= B * (k + 1)) return;
+    int b = i / (k + 1), c = i % (k + 1);
+    int j = s.len[b];
+    r.tok[i] = (c == 0) ? (j == 0 ? bos : s.out[(size_t)b * s.out_stride + j - 1]) : draft[b * k + c - 1];
+    r.pos[i] = j + c;
+    r.seq[i] = b;
+    r.nk_self[i] = j + c + 1;     // causal: positions 0..j+c
+    r.nk_cross[i] = s.src_len[b];
+}
+
+// Drafter: packed rows [BOS, committed, MASK x k] of every unfinished sequence (one block).
+// `all` describes the full pass, `msk` the mask-only continuation of the last layer.
+__global__ void k_draft_prep(Session s, int B, int k, int S_max, int bos, int mask, Rows all, Rows msk) {
+    extern __shared__ int sh[];          // [B+1] row offsets, [B+1] mask-row offsets
+    int* off = sh;
+    int* moff = sh + B + 1;
+    if (threadIdx.x == 0) {
+        int a = 0, m = 0;
+        for (int b = 0; b < B; ++b) {
+            off[b] = a; moff[b] = m;
+            if (!s.finished[b]) { a += s.len[b] + 1 + k; m += k; }
+        }
+        off[B] = a; moff[B] = m;
+        s.counters[CNT_DRAFT_ALL] = a;
+        s.counters[CNT_DRAFT_MASK] = m;
+    }
+    __syncthreads();
+    for (int b = 0; b < B; ++b) {
+        if (threadIdx.x == 0) { all.kv_off[b] = off[b]; all.kv_off_cross[b] = b * S_max;
+                                msk.kv_off[b] = off[b]; msk.kv_off_cross[b] = b * S_max; }
+        if (s.finished[b]) continue;
+        int j = s.len[b], n = j + 1 + k, sl = s.src_len[b];
+        for (int t = threadIdx.x; t < n; t += blockDim.x) {
+            int row = off[b] + t;
+            all.tok[row] = (t == 0) ? bos : (t <= j ? s.out[(size_t)b * s.out_stride + t - 1] : mask);
+            all.pos[row] = t;
+            all.seq[row] = b;
+            all.nk_self[row] = n;            // no causal mask: every valid position
+            all.nk_cross[row] = sl;
+        }
+        for (int i = threadIdx.x; i < k; i += blockDim.x) {
+            int row = moff[b] + i;
+            msk.seq[row] = b;
+            msk.nk_self[row] = n;
+            msk.nk_cross[row] = sl;
+            msk.src_row[row] = off[b] + j + 1 + i;
+            msk.slot[row] = b * k + i;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ embedding, gather, layer norm
+// x[row] = sqrt(d) * E[tok] + P[pos]
+template <typename T>
+__global__ void k_embed(const int* __restrict__ tok, const int* __restrict__ pos, const int* __restrict__ n_rows,
+                        const T* __restrict__ E, const float* __restrict__ P, float* __restrict__ x, int d,
+                        float scale, int vocab, int max_pos) {
+    int row = blockIdx.x;
+    if (row >= *n_rows) return;
+    int t = min(max(tok[row], 0), vocab - 1), p = min(max(pos[row], 0), max_pos - 1);
+    for (int e = threadIdx.x; e < d; e += blockDim.x)
+        x[(size_t)row * d + e] = scale * to_f(E[(size_t)t * d + e]) + P[(size_t)p * d + e];
+}
+
+__global__ void k_gather_rows(const float* __restrict__ x, const int* __restrict__ src_row,
+                              const int* __restrict__ n_rows, float* __restrict__ out, int d) {
+    int row = blockIdx.x;
+    if (row >= *n_rows) return;
+    const float* s = x + (size_t)src_row[row] * d;
+    for (int e = threadIdx.x; e < d; e += blockDim.x) out[(size_t)row * d + e] = s[e];
+}
+
+// One warp per row; biased variance, eps inside the square root.
+template <typename T>
+__global__ void k_layernorm(const float* __restrict__ x, const float* __restrict__ g, const float* __restrict__ b,
+                            const int* __restrict__ n_rows, T* __restrict__ y, int d, float eps) {
+    int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    int lane = threadIdx.x & 31;
+    if (row >= *n_rows) return;
+    const float* xr = x + (size_t)row * d;
+    float s = 0.f;
+    for (int e = lane; e < d; e += 32) s += xr[e];
+    float mu = warp_sum(s) / d;
+    float v = 0.f;
+    for (int e = lane; e < d; e += 32) { float c = xr[e] - mu; v += c * c; }
+    float rstd = 1.0f / sqrtf(warp_sum(v) / d + eps);
+    for (int e = lane; e < d; e += 32) y[(size_t)row * d + e] = from_f<T>((xr[e] - mu) * rstd * g[e] + b[e]);
+}
+
+// ------------------------------------------------------------------ paged KV cache
+struct Paged {
+    const int* table;   // [B, max_pages] page ids
+    int page_tokens, max_pages;
+    __device__ __forceinline__ size_t row(int b, int t) const {
+        return (size_t)table[b * max_pages + t / page_tokens] * page_tokens + (t % page_tokens);
+    }
+};
+
+// Writes the K and V parts of the verify block's QKV rows to their cache positions.
+template <typename T>
+__global__ void k_kv_scatter(const T* __restrict__ qkv, const int* __restrict__ seq, const int* __restrict__ pos,
+                             const int* __restrict__ n_rows, Paged pg, T* __restrict__ kc, T* __restrict__ vc, int d) {
+    int row = blockIdx.x;
+    if (row >= *n_rows) return;
+    size_t dst = pg.row(seq[row], pos[row]) * d;
+    const T* s = qkv + (size_t)row * 3 * d;
+    for (int e = threadIdx.x; e < d; e += blockDim.x) { kc[dst + e] = s[d + e]; vc[dst + e] = s[2 * d + e]; }
+}
+
+// ------------------------------------------------------------------ attention
+// One warp per (row, head).  Scores of all visible keys are held in shared memory, so the
+// softmax uses the true row maximum; the un-normalised probabilities are rounded to the
+// operand type before the weighted sum and normalised by the sum of the unrounded ones.
+template <typename T>
+struct AttnArgs {
+    const T* q; int q_stride; const int* q_index;       // row r reads q + (q_index ? q_index[r] : r) * q_stride
+    const T* k; const T* v; int kv_stride;              // contiguous: key t of seq b at (kv_off[b] + t) * kv_stride
+    const int* kv_off;
+    Paged pg;                                            // paged: row pg.row(b, t) * kv_stride
+    const int* seq; const int* nkeys; const int* n_rows;
+    T* out; int out_stride;
+    int n_heads, d_head, max_keys;
+    float scale;
+};
+
+template <typename T, bool PAGED>
+__global__ void k_attention(AttnArgs<T> a) {
+    extern __shared__ float sm_att[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
+    long long gw = (long long)blockIdx.x * wpb + warp;
+    int r = (int)(gw / a.n_heads), h = (int)(gw % a.n_heads);
+    if (r >= *a.n_rows) return;
+    const int dh = a.d_head;
+    float* sc = sm_att + (size_t)warp * (a.max_keys + dh);
+    float* qs = sc + a.max_keys;
+    const int b = a.seq[r];
+    const int nk = min(a.nkeys[r], a.max_keys);
+    const T* qp = a.q + (size_t)(a.q_index ? a.q_index[r] : r) * a.q_stride + h * dh;
+    for (int e = lane; e < dh; e += 32) qs[e] = to_f(qp[e]);
+    __syncwarp();
+    float mx = -CUDART_INF_F;
+    for (int t = lane; t < nk; t += 32) {
+        size_t kr = PAGED ? a.pg.row(b, t) : (size_t)(a.kv_off[b] + t);
+        const T* kp = a.k + kr * a.kv_stride + h * dh;
+        float s = 0.f;
+        for (int e = 0; e < dh; ++e) s = fmaf(qs[e], to_f(kp[e]), s);
+        s *= a.scale;
+        sc[t] = s;
+        mx = fmaxf(mx, s);
+    }
+    mx = warp_max(mx);
+    float sum = 0.f;
+    for (int t = lane; t < nk; t += 32) {
+        float e = expf(sc[t] - mx);
+        sum += e;
+        sc[t] = round_as<T>(e);
+    }
+    sum = warp_sum(sum);
+    __syncwarp();
+    T* op = a.out + (size_t)r * a.out_stride + h * dh;
+    for (int e = lane; e < dh; e += 32) {
+        float acc = 0.f;
+        for (int t = 0; t < nk; ++t) {
+            size_t vr = PAGED ? a.pg.row(b, t) : (size_t)(a.kv_off[b] + t);
+            acc = fmaf(sc[t], to_f(a.v[vr * a.kv_stride + h * dh + e]), acc);
+        }
+        op[e] = from_f<T>(nk > 0 ? acc / sum : 0.f);
+    }
+}
+
+// ------------------------------------------------------------------ GEMM epilogues
+// C[r, n] = sum_k A[r, k] * W[n, k]  (+ bias[n])
+enum { EPI_STORE = 0, EPI_RELU = 1, EPI_RESID = 2, EPI_STATS = 3, EPI_F32 = 4 };
+
+// Partial statistics of one verifier (or drafter) row over one tile of vocabulary columns.
+struct __align__(16) RowPart { float mx; int arg; float sum; int cnt; };
+
+template <typename T>
+struct GemmArgs {
+    const T* A; int lda;
+    const T* W;                 // [N, K]
+    const float* bias;          // [N] or null
+    int N, K;
+    const int* n_rows;          // device row count
+    T* out; int ldo;            // EPI_STORE / EPI_RELU
+    float* resid;               // EPI_RESID: resid[r, n] += value ; EPI_F32: resid[r, n] = value (ld = N)
+    // EPI_STATS
+    RowPart* part; int n_tiles; // part[r * n_tiles + tile]
+    const float* ld;            // [rows] logit of the row's draft from the pre-pass (+inf: none)
+    const int* ld_id;           // [rows] the draft's id (-1: none)
+};
+
+// Merge order of row statistics: larger maximum wins, equal maxima keep the lower id.
+__device__ __forceinline__ void part_merge(RowPart& a, const RowPart& b) {
+    float m = fmaxf(a.mx, b.mx);
+    float sa = (a.mx == -CUDART_INF_F) ? 0.f : a.sum * expf(a.mx - m);
+    float sb = (b.mx == -CUDART_INF_F) ? 0.f : b.sum * expf(b.mx - m);
+    if (b.mx > a.mx || (b.mx == a.mx && b.arg < a.arg)) a.arg = b.arg;
+    a.mx = m;
+    a.sum = sa + sb;
+    a.cnt += b.cnt;
+}
+
+// ------------------------------------------------------------------ SIMT reference GEMM
+// 64x64x16 tiles, 256 threads, 4x4 outputs per thread; used by the fp32 path and as the
+// on-device cross-check of the tensor-core GEMM.
+template <typename T, int EPI>
+__global__ void __launch_bounds__(256) k_gemm_simt(GemmArgs<T> g) {
+    constexpr int BM = 64, BN = 64, BK = 16;
+    __shared__ float As[BK][BM + 4];
+    __shared__ float Ws[BK][BN + 4];
+    __shared__ float Ct[(EPI == EPI_STATS) ? BM : 1][(EPI == EPI_STATS) ? BN + 1 : 1];
+    const int R = *g.n_rows;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    if (m0 >= R) return;
+    const int tid = threadIdx.x;
+    const int lr = tid >> 2, lk = (tid & 3) * 4;       // loader: row lr, k offset lk..lk+3
+    const int ty = tid >> 4, tx = tid & 15;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    const bool a_ok = (m0 + lr) < R, w_ok = (n0 + lr) < g.N;
+    const T* ap = g.A + (size_t)(m0 + lr) * g.lda + lk;
+    const T* wp = g.W + (size_t)(n0 + lr) * g.K + lk;
+    for (int k0 = 0; k0 < g.K; k0 += BK) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            As[lk + e][lr] = a_ok ? to_f(ap[k0 + e]) : 0.f;
+            Ws[lk + e][lr] = w_ok ? to_f(wp[k0 + e]) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            float av[4], wv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { av[i] = As[kk][ty * 4 + i]; wv[i] = Ws[kk][tx * 4 + i]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], wv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int r = m0 + ty * 4 + i;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int n = n0 + tx * 4 + j;
+            float v = acc[i][j] + ((g.bias && n < g.N) ? g.bias[n] : 0.f);
+            if (EPI == EPI_STATS) {
+                Ct[ty * 4 + i][tx * 4 + j] = v;
+            } else if (r < R && n < g.N) {
+                if (EPI == EPI_STORE) g.out[(size_t)r * g.ldo + n] = from_f<T>(v);
+                if (EPI == EPI_RELU) g.out[(size_t)r * g.ldo + n] = from_f<T>(fmaxf(v, 0.f));
+                if (EPI == EPI_RESID) g.resid[(size_t)r * g.N + n] += v;
+                if (EPI == EPI_F32) g.resid[(size_t)r * g.N + n] = v;
+            }
+        }
+    }
+    if (EPI == EPI_STATS) {
+        __syncthreads();
+        if (tid < BM && m0 + tid < R) {
+            const int r = m0 + tid;
+            const float ld = g.ld ? g.ld[r] : CUDART_INF_F;
+            const int id = g.ld_id ? g.ld_id[r] : -1;
+            RowPart p; p.mx = -CUDART_INF_F; p.arg = 0x7fffffff; p.sum = 0.f; p.cnt = 0;
+            const int nn = min(BN, g.N - n0);
+            for (int j = 0; j < nn; ++j) {
+                float v = Ct[tid][j];
+                if (n0 + j == id) v = ld;             // the draft's column takes the pre-pass value
+                if (v > p.mx) { p.mx = v; p.arg = n0 + j; }
+                p.cnt += (v > ld) ? 1 : 0;
+            }
+            for (int j = 0; j < nn; ++j) {
+                float v = (n0 + j == id) ? ld : Ct[tid][j];
+                p.sum += expf(v - p.mx);
+            }
+            g.part[(size_t)r * g.n_tiles + blockIdx.x] = p;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ verify: draft logit pre-pass
+// Row c < k of a sequence checks draft c+1: its logit is the dot product of the row's
+// normalised hidden state with the draft's embedding row.  Row k (bonus) has no draft.
+template <typename T>
+__global__ void k_draft_logit(const T* __restrict__ y, const T* __restrict__ E, const int* __restrict__ draft,
+                              int B, int k, int d, int vocab, float* __restrict__ ld, int* __restrict__ ld_id) {
+    int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    int lane = threadIdx.x & 31;
+    if (row >= B * (k + 1)) return;
+    int b = row / (k + 1), c = row % (k + 1);
+    if (c == k) { if (lane == 0) { ld[row] = CUDART_INF_F; ld_id[row] = -1; } return; }
+    int tok = draft[b * k + c];
+    bool ok = tok >= 0 && tok < vocab;
+    float s = 0.f;
+    if (ok) for (int e = lane; e < d; e += 32) s = fmaf(to_f(y[(size_t)row * d + e]), to_f(E[(size_t)tok * d + e]), s);
+    s = warp_sum(s);
+    if (lane == 0) { ld[row] = ok ? s : -CUDART_INF_F; ld_id[row] = ok ? tok : -2; }
+}
+
+// ------------------------------------------------------------------ acceptance scan (Eq. 7-9)
+// One block per sequence: warps merge the per-tile statistics of the k+1 rows, thread 0
+// finds the first rejected draft.  row_stats (optional) receives 6 floats per row.
+__global__ void k_accept(const RowPart* __restrict__ part, int n_tiles, const float* __restrict__ ld,
+                         const int* __restrict__ ld_id, int k, int beta, float tau, int* __restrict__ accepted,
+                         int* __restrict__ bif, float* __restrict__ row_stats) {
+    extern __shared__ unsigned char sm_acc[];
+    RowPart* rs = reinterpret_cast<RowPart*>(sm_acc);       // [k+1]
+    const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    for (int c = warp; c <= k; c += nw) {
+        const RowPart* p = part + ((size_t)b * (k + 1) + c) * n_tiles;
+        RowPart m; m.mx = -CUDART_INF_F; m.arg = 0x7fffffff; m.sum = 0.f; m.cnt = 0;
+        for (int t = lane; t < n_tiles; t += 32) part_merge(m, p[t]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            RowPart q;
+            q.mx = __shfl_xor_sync(0xffffffffu, m.mx, o);
+            q.arg = __shfl_xor_sync(0xffffffffu, m.arg, o);
+            q.sum = __shfl_xor_sync(0xffffffffu, m.sum, o);
+            q.cnt = __shfl_xor_sync(0xffffffffu, m.cnt, o);
+            part_merge(m, q);
+        }
+        if (lane == 0) rs[c] = m;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int a = 0;
+        for (int c = 0; c < k; ++c) {
+            const float l = ld[b * (k + 1) + c];
+            const bool ok = (rs[c].cnt <= beta - 1) && ((rs[c].mx - l) <= tau);
+            if (!ok) break;
+            ++a;
+        }
+        accepted[b] = a;
+        bif[b] = rs[a].arg;
+    }
+    if (row_stats)
+        for (int c = threadIdx.x; c <= k; c += blockDim.x) {
+            float* o = row_stats + ((size_t)b * (k + 1) + c) * 6;
+            o[0] = rs[c].mx; o[1] = (float)rs[c].arg; o[2] = rs[c].mx + logf(rs[c].sum);
+            o[3] = (float)rs[c].cnt; o[4] = ld[b * (k + 1) + c]; o[5] = (float)ld_id[b * (k + 1) + c];
+        }
+}
+
+// The same rule on caller-provided logits [B, k+1, V]: one block per sequence walks the rows
+// in order and stops at the first rejected draft, so it needs no scratch memory.
+__global__ void k_accept_logits(const float* __restrict__ logits, const int* __restrict__ draft, int k, int V,
+                                int beta, float tau, int* __restrict__ accepted, int* __restrict__ bif) {
+    __shared__ RowPart wsm[32];
+    __shared__ int stop;
+    const int b = blockIdx.x;
+    for (int c = 0; c <= k; ++c) {
+        const float* l = logits + ((size_t)b * (k + 1) + c) * V;
+        const int tok = (c < k) ? draft[b * k + c] : -1;
+        const float ld = (c == k) ? CUDART_INF_F : ((tok >= 0 && tok < V) ? l[tok] : -CUDART_INF_F);
+        RowPart m; m.mx = -CUDART_INF_F; m.arg = 0x7fffffff; m.sum = 0.f; m.cnt = 0;
+        for (int v = threadIdx.x; v < V; v += blockDim.x) {
+            RowPart q; q.mx = l[v]; q.arg = v; q.sum = 1.f; q.cnt = (l[v] > ld) ? 1 : 0;
+            part_merge(m, q);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            RowPart q;
+            q.mx = __shfl_xor_sync(0xffffffffu, m.mx, o);
+            q.arg = __shfl_xor_sync(0xffffffffu, m.arg, o);
+            q.sum = __shfl_xor_sync(0xffffffffu, m.sum, o);
+            q.cnt = __shfl_xor_sync(0xffffffffu, m.cnt, o);
+            part_merge(m, q);
+        }
+        if ((threadIdx.x & 31) == 0) wsm[threadIdx.x >> 5] = m;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int w = 1; w < (int)(blockDim.x >> 5); ++w) part_merge(m, wsm[w]);
+            const bool ok = (c < k) && (m.cnt <= beta - 1) && ((m.mx - ld) <= tau);
+            stop = ok ? 0 : 1;
+            if (!ok) { accepted[b] = c; bif[b] = m.arg; }
+        }
+        __syncthreads();
+        if (stop) return;
+    }
+}
+
+// ------------------------------------------------------------------ drafter argmax
+__global__ void k_draft_argmax(const RowPart* __restrict__ part, int n_tiles, const int* __restrict__ n_rows,
+                               const int* __restrict__ slot, int* __restrict__ draft) {
+    int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    int lane = threadIdx.x & 31;
+    if (row >= *n_rows) return;
+    const RowPart* p = part + (size_t)row * n_tiles;
+    float mx = -CUDART_INF_F; int arg = 0x7fffffff;
+    for (int t = lane; t < n_tiles; t += 32) {
+        RowPart q = p[t];
+        if (q.mx > mx || (q.mx == mx && q.arg < arg)) { mx = q.mx; arg = q.arg; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        float om = __shfl_xor_sync(0xffffffffu, mx, o);
+        int oa = __shfl_xor_sync(0xffffffffu, arg, o);
+        if (om > mx || (om == mx && oa < arg)) { mx = om; arg = oa; }
+    }
+    if (lane == 0) draft[slot[row]] = arg;
+}
+
+// ------------------------------------------------------------------ commit / rollback (Eq. 3)
+// Appends drafts[0..keep) and the next token, cuts after the first EOS and at max_tgt.
+// Cache rows beyond the new length are simply dead: the next block overwrites them.
+__global__ void k_commit(Session s, const int* __restrict__ draft, const int* __restrict__ keep,
+                         const int* __restrict__ next, int B, int k, int eos) {
+    int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B || s.finished[b]) return;
+    int j = s.len[b];
+    const int mt = s.max_tgt[b];
+    const int a = min(max(keep[b], 0), k);
+    bool fin = false;
+    int n0 = j;
+    for (int c = 0; c <= a && !fin; ++c) {
+        if (j >= mt) { fin = true; break; }
+        int tok = (c < a) ? draft[b * k + c] : next[b];
+        s.out[(size_t)b * s.out_stride + j] = tok;
+        ++j;
+        if (tok == eos) fin = true;
+    }
+    if (j >= mt) fin = true;
+    s.len[b] = j;
+    atomicAdd(&s.stats[0], 1ull);
+    atomicAdd(&s.stats[1], (unsigned long long)k);
+    atomicAdd(&s.stats[2], (unsigned long long)a);
+    atomicAdd(&s.stats[3], (unsigned long long)(j - n0));
+    if (fin) { s.finished[b] = 1; atomicSub(&s.counters[CNT_ACTIVE], 1); }
+}
+
+__global__ void k_session_init(Session s, const int* __restrict__ src_len, const int* __restrict__ max_tgt, int B,
+                               int max_tgt_cap, int S_max) {
+    int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b == 0) {
+        for (int i = 0; i < 4; ++i) s.stats[i] = 0ull;
+    }
+    if (b >= B) return;
+    int mt = max_tgt ? min(max(max_tgt[b], 0), max_tgt_cap) : max_tgt_cap;
+    s.len[b] = 0;
+    s.max_tgt[b] = mt;
+    s.finished[b] = (mt <= 0) ? 1 : 0;
+    s.src_len[b] = min(max(src_len[b], 1), S_max);
+}
+
+__global__ void k_count_active(Session s, int B) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        int n = 0;
+        for (int b = 0; b < B; ++b) n += s.finished[b] ? 0 : 1;
+        s.counters[CNT_ACTIVE] = n;
+    }
+}
+
+__global__ void k_copy_out(Session s, int B, int* __restrict__ out, int out_stride, int* __restrict__ out_len,
+                           int* __restrict__ fin) {
+    int b = blockIdx.x;
+    if (b >= B) return;
+    int n = s.len[b];
+    if (out) for (int t = threadIdx.x; t < min(n, out_stride); t += blockDim.x)
+        out[(size_t)b * out_stride + t] = s.out[(size_t)b * s.out_stride + t];
+    if (threadIdx.x == 0) { if (out_len) out_len[b] = n; if (fin) fin[b] = s.finished[b]; }
+}
+
+// ------------------------------------------------------------------ weight repacking
+template <typename T>
+__global__ void k_convert(const float* __restrict__ in, T* __restrict__ out, size_t n) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    size_t st = (size_t)gridDim.x * blockDim.x;
+    for (; i < n; i += st) out[i] = from_f<T>(in[i]);
+}
+
+}  // namespace sd

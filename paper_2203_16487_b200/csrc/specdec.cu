@@ -1,0 +1,824 @@
+// Host runtime and C ABI of the SpecDec draft -> verify -> commit library (see include/specdec.h).
+// The arena is the only device allocation; every step of the path runs in the kernels of
+// kernels.cuh and gemm_tc.cuh.  There is no CPU fallback.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <type_traits>
+#include <unordered_map>
+#include <vector>
+
+#include "../../include/specdec.h"
+#include "gemm_tc.cuh"
+#include "kernels.cuh"
+
+using namespace sd;
+
+namespace {
+
+thread_local std::string g_create_error;
+
+struct LayerW {
+    void *qkv_w, *o_w, *cq_w, *ckv_w, *co_w, *w1, *w2;
+    float *qkv_b, *o_b, *cq_b, *ckv_b, *co_b, *b1, *b2;
+    float *ln1_g, *ln1_b, *lnc_g, *lnc_b, *ln2_g, *ln2_b;
+};
+struct ModelW {
+    specdec_model_dims dm;
+    void* embed;
+    float *pos_enc, *pos_dec;
+    std::vector<LayerW> enc, dec;
+    float *enc_lnf_g, *enc_lnf_b, *dec_lnf_g, *dec_lnf_b;
+    std::vector<void*> ckv;   // per decoder layer: cross K/V of the session [B*S_max, 2d]
+};
+
+struct Arena {
+    char* base = nullptr;
+    size_t off = 0;
+    void* take(size_t n) {
+        off = (off + 255) & ~size_t(255);
+        void* p = base ? base + off : nullptr;
+        off += n;
+        return p;
+    }
+};
+
+}  // namespace
+
+struct specdec_handle {
+    specdec_config cfg;
+    int dtype;
+    size_t esz;                    // bytes per operand element
+    ModelW ver, dra;
+    Arena arena;
+    // capacities
+    int B_cap, S_cap, T_cap, k_cap, R_cap, R2_cap, M_cap, d_max, f_max, v_max, pages_per_seq, n_tiles_cap;
+    // activations
+    float *x, *x2;
+    void *y, *qkv, *att, *q, *hbuf, *mem;
+    // verifier KV cache
+    std::vector<void*> kc, vc;
+    int* page_table;
+    // rows
+    Rows rows, mrows;
+    // vocabulary statistics
+    RowPart* part;
+    float *ld, *row_stats;
+    int* ld_id;
+    int *accepted, *bif, *v_draft, *g_draft;
+    int *stage_src, *stage_len, *stage_mt;   // device staging of specdec_generate_host
+    Session ses;
+    // session (host side)
+    int B = 0, S_max = 0, last_k = 0, len_ub = 0;
+    bool encoded = false, verified = false, drafted = false;
+    int last_draft_rows_ub = 0;
+    // options
+    int use_tc = 1, use_graphs = 0;
+    long long launches = 0;
+    // polling
+    int* h_poll = nullptr;          // pinned
+    unsigned long long* h_stats = nullptr;  // pinned [4]
+    std::vector<cudaEvent_t> poll_ev;
+    std::vector<cudaEvent_t> time_ev;
+    sd::TmaEncoder tma;
+    std::string err;
+};
+
+namespace {
+
+int fail(specdec_handle* h, int code, const std::string& msg) {
+    if (h) h->err = msg; else g_create_error = msg;
+    return code;
+}
+#define CUDA_TRY(h, expr)                                                                   \
+    do {                                                                                    \
+        cudaError_t e__ = (expr);                                                           \
+        if (e__ != cudaSuccess)                                                             \
+            return fail(h, SPECDEC_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__)); \
+    } while (0)
+#define KCHECK(h)                                                                           \
+    do {                                                                                    \
+        cudaError_t e__ = cudaGetLastError();                                               \
+        if (e__ != cudaSuccess)                                                             \
+            return fail(h, SPECDEC_ERR_CUDA, std::string("kernel launch: ") + cudaGetErrorString(e__) + \
+                        " at line " + std::to_string(__LINE__));                            \
+        ++h->launches;                                                                      \
+    } while (0)
+
+inline int cdiv(int a, int b) { return (a + b - 1) / b; }
+
+// ---------------------------------------------------------------- layout of the arena
+void layout_model(specdec_handle* h, ModelW& m, const specdec_model_dims& dm) {
+    Arena& A = h->arena;
+    const size_t e = h->esz;
+    const size_t d = dm.d_model, f = dm.d_ffn;
+    m.dm = dm;
+    m.embed = A.take((size_t)dm.vocab * d * e);
+    m.pos_enc = (float*)A.take((size_t)dm.max_pos * d * 4);
+    m.pos_dec = (float*)A.take((size_t)dm.max_pos * d * 4);
+    auto vec = [&](size_t n) { return (float*)A.take(n * 4); };
+    auto layer = [&](LayerW& w, bool dec) {
+        w.qkv_w = A.take(3 * d * d * e); w.qkv_b = vec(3 * d);
+        w.o_w = A.take(d * d * e); w.o_b = vec(d);
+        w.w1 = A.take(f * d * e); w.b1 = vec(f);
+        w.w2 = A.take(d * f * e); w.b2 = vec(d);
+        w.ln1_g = vec(d); w.ln1_b = vec(d); w.ln2_g = vec(d); w.ln2_b = vec(d);
+        if (dec) {
+            w.cq_w = A.take(d * d * e); w.cq_b = vec(d);
+            w.ckv_w = A.take(2 * d * d * e); w.ckv_b = vec(2 * d);
+            w.co_w = A.take(d * d * e); w.co_b = vec(d);
+            w.lnc_g = vec(d); w.lnc_b = vec(d);
+        }
+    };
+    m.enc.resize(dm.enc_layers);
+    m.dec.resize(dm.dec_layers);
+    for (auto& w : m.enc) layer(w, false);
+    for (auto& w : m.dec) layer(w, true);
+    m.enc_lnf_g = vec(d); m.enc_lnf_b = vec(d); m.dec_lnf_g = vec(d); m.dec_lnf_b = vec(d);
+    m.ckv.resize(dm.dec_layers);
+    for (auto& p : m.ckv) p = A.take((size_t)h->B_cap * h->S_cap * 2 * d * e);
+}
+
+void layout_rows(Arena& A, Rows& r, int n, int B) {
+    auto iv = [&](size_t c) { return (int*)A.take(c * 4); };
+    r.tok = iv(n); r.pos = iv(n); r.seq = iv(n); r.nk_self = iv(n); r.nk_cross = iv(n);
+    r.src_row = iv(n); r.slot = iv(n);
+    r.kv_off = iv(B); r.kv_off_cross = iv(B);
+}
+
+void layout_all(specdec_handle* h) {
+    Arena& A = h->arena;
+    A.off = 0;
+    const size_t e = h->esz;
+    layout_model(h, h->ver, h->cfg.verifier);
+    layout_model(h, h->dra, h->cfg.drafter);
+    const size_t R = h->R_cap, d = h->d_max, f = h->f_max;
+    h->x = (float*)A.take(R * d * 4);
+    h->x2 = (float*)A.take((size_t)h->R2_cap * d * 4);
+    h->y = A.take(R * d * e);
+    h->qkv = A.take(R * 3 * d * e);
+    h->att = A.take(R * d * e);
+    h->q = A.take(R * d * e);
+    h->hbuf = A.take(R * f * e);
+    h->mem = A.take((size_t)h->B_cap * h->S_cap * d * e);
+    const size_t cache_rows = (size_t)h->B_cap * h->pages_per_seq * h->cfg.page_tokens;
+    h->kc.resize(h->cfg.verifier.dec_layers);
+    h->vc.resize(h->cfg.verifier.dec_layers);
+    for (auto& p : h->kc) p = A.take(cache_rows * h->cfg.verifier.d_model * e);
+    for (auto& p : h->vc) p = A.take(cache_rows * h->cfg.verifier.d_model * e);
+    h->page_table = (int*)A.take((size_t)h->B_cap * h->pages_per_seq * 4);
+    layout_rows(A, h->rows, h->R_cap, h->B_cap);
+    layout_rows(A, h->mrows, h->R2_cap > 0 ? h->R2_cap : 1, h->B_cap);
+    const size_t stat_rows = (size_t)(h->M_cap > h->R2_cap ? h->M_cap : h->R2_cap);
+    h->part = (RowPart*)A.take(stat_rows * h->n_tiles_cap * sizeof(RowPart));
+    h->ld = (float*)A.take((size_t)h->M_cap * 4);
+    h->ld_id = (int*)A.take((size_t)h->M_cap * 4);
+    h->row_stats = (float*)A.take((size_t)h->M_cap * 6 * 4);
+    h->accepted = (int*)A.take((size_t)h->B_cap * 4);
+    h->bif = (int*)A.take((size_t)h->B_cap * 4);
+    h->v_draft = (int*)A.take((size_t)h->B_cap * h->k_cap * 4);
+    h->g_draft = (int*)A.take((size_t)h->B_cap * h->k_cap * 4);
+    h->stage_src = (int*)A.take((size_t)h->B_cap * h->S_cap * 4);
+    h->stage_len = (int*)A.take((size_t)h->B_cap * 4);
+    h->stage_mt = (int*)A.take((size_t)h->B_cap * 4);
+    Session& s = h->ses;
+    s.len = (int*)A.take((size_t)h->B_cap * 4);
+    s.finished = (int*)A.take((size_t)h->B_cap * 4);
+    s.max_tgt = (int*)A.take((size_t)h->B_cap * 4);
+    s.src_len = (int*)A.take((size_t)h->B_cap * 4);
+    s.out_stride = h->T_cap > 0 ? h->T_cap : 1;
+    s.out = (int*)A.take((size_t)h->B_cap * s.out_stride * 4);
+    s.counters = (int*)A.take(8 * 4);
+    s.stats = (unsigned long long*)A.take(4 * 8);
+}
+
+// ---------------------------------------------------------------- weight loading
+struct Manifest {
+    std::unordered_map<std::string, const specdec_tensor*> map;
+    std::string missing, bad;
+    const float* get(const std::string& name, std::initializer_list<long long> shape) {
+        auto it = map.find(name);
+        if (it == map.end()) { if (missing.empty()) missing = name; return nullptr; }
+        const specdec_tensor* t = it->second;
+        bool ok = t->dtype == SPECDEC_DTYPE_F32 && t->ndim == (int)shape.size() && t->d_ptr != nullptr;
+        int i = 0;
+        for (long long s : shape) { if (ok && t->shape[i] != s) ok = false; ++i; }
+        if (!ok) { if (bad.empty()) bad = name; return nullptr; }
+        return (const float*)t->d_ptr;
+    }
+};
+
+template <typename T>
+void conv(specdec_handle* h, const float* src, void* dst, size_t n, cudaStream_t st) {
+    if (!src) return;
+    int blocks = (int)std::min<size_t>((n + 255) / 256, 4096);
+    k_convert<T><<<blocks, 256, 0, st>>>(src, (T*)dst, n);
+    ++h->launches;
+}
+
+template <typename T>
+void load_model(specdec_handle* h, ModelW& m, const std::string& pre, Manifest& mf, cudaStream_t st) {
+    const long long d = m.dm.d_model, f = m.dm.d_ffn, V = m.dm.vocab, P = m.dm.max_pos;
+    const size_t e = h->esz;
+    auto mat = [&](const std::string& n, long long r, long long c, void* dst) {
+        conv<T>(h, mf.get(pre + n, {r, c}), dst, (size_t)r * c, st);
+    };
+    auto vec = [&](const std::string& n, long long c, float* dst) { conv<float>(h, mf.get(pre + n, {c}), dst, (size_t)c, st); };
+    mat("embed", V, d, m.embed);
+    conv<float>(h, mf.get(pre + "pos_enc", {P, d}), m.pos_enc, (size_t)P * d, st);
+    conv<float>(h, mf.get(pre + "pos_dec", {P, d}), m.pos_dec, (size_t)P * d, st);
+    auto attn_qkv = [&](const std::string& p, void* w, float* b) {
+        const char* nm[3] = {"q", "k", "v"};
+        for (int i = 0; i < 3; ++i) {
+            mat(p + "." + nm[i] + ".w", d, d, (char*)w + (size_t)i * d * d * e);
+            vec(p + "." + nm[i] + ".b", d, b + (size_t)i * d);
+        }
+    };
+    auto layer = [&](LayerW& w, const std::string& p, bool dec) {
+        vec(p + ".ln1.g", d, w.ln1_g); vec(p + ".ln1.b", d, w.ln1_b);
+        attn_qkv(p + ".self", w.qkv_w, w.qkv_b);
+        mat(p + ".self.o.w", d, d, w.o_w); vec(p + ".self.o.b", d, w.o_b);
+        vec(p + ".ln2.g", d, w.ln2_g); vec(p + ".ln2.b", d, w.ln2_b);
+        mat(p + ".ffn.w1", f, d, w.w1); vec(p + ".ffn.b1", f, w.b1);
+        mat(p + ".ffn.w2", d, f, w.w2); vec(p + ".ffn.b2", d, w.b2);
+        if (dec) {
+            vec(p + ".ln_cross.g", d, w.lnc_g); vec(p + ".ln_cross.b", d, w.lnc_b);
+            mat(p + ".cross.q.w", d, d, w.cq_w); vec(p + ".cross.q.b", d, w.cq_b);
+            mat(p + ".cross.k.w", d, d, w.ckv_w); vec(p + ".cross.k.b", d, w.ckv_b);
+            mat(p + ".cross.v.w", d, d, (char*)w.ckv_w + (size_t)d * d * e); vec(p + ".cross.v.b", d, w.ckv_b + d);
+            mat(p + ".cross.o.w", d, d, w.co_w); vec(p + ".cross.o.b", d, w.co_b);
+        }
+    };
+    for (int l = 0; l < m.dm.enc_layers; ++l) layer(m.enc[l], "enc." + std::to_string(l), false);
+    for (int l = 0; l < m.dm.dec_layers; ++l) layer(m.dec[l], "dec." + std::to_string(l), true);
+    vec("enc.ln_f.g", d, m.enc_lnf_g); vec("enc.ln_f.b", d, m.enc_lnf_b);
+    vec("dec.ln_f.g", d, m.dec_lnf_g); vec("dec.ln_f.b", d, m.dec_lnf_b);
+}
+
+// ---------------------------------------------------------------- launch helpers
+template <typename T>
+int ln(specdec_handle* h, const float* x, const float* g, const float* b, int cnt, int rows_ub, void* y, int d,
+       cudaStream_t st) {
+    if (rows_ub <= 0) return 0;
+    k_layernorm<T><<<cdiv(rows_ub, 4), 128, 0, st>>>(x, g, b, h->ses.counters + cnt, (T*)y, d, 1e-5f);
+    KCHECK(h);
+    return 0;
+}
+
+// out = A W^T (+bias) with one of the epilogues; rows_ub bounds the grid, the live count is on the device.
+template <typename T>
+int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, const float* bias, int N, int K, int cnt,
+         int rows_ub, void* out, int ldo, float* resid, cudaStream_t st, const float* ldv = nullptr,
+         const int* ld_id = nullptr, int* n_tiles_out = nullptr) {
+    if (rows_ub <= 0) return 0;
+    GemmArgs<T> g;
+    g.A = (const T*)A; g.lda = lda; g.W = (const T*)W; g.bias = bias; g.N = N; g.K = K;
+    g.n_rows = h->ses.counters + cnt; g.out = (T*)out; g.ldo = ldo; g.resid = resid;
+    g.part = h->part; g.ld = ldv; g.ld_id = ld_id; g.n_tiles = cdiv(N, 64);
+    if constexpr (std::is_same<T, bf16>::value) {
+        if (h->use_tc && sd::tc_supported(N, K)) {
+            int rc = sd::gemm_tc_launch(h->tma, epi, g, rows_ub, st, n_tiles_out);
+            if (rc != 0) return fail(h, SPECDEC_ERR_CUDA, "tensor-core GEMM launch failed: " + h->tma.err);
+            ++h->launches;
+            return 0;
+        }
+    }
+    if (n_tiles_out) *n_tiles_out = g.n_tiles;
+    dim3 grid(cdiv(N, 64), cdiv(rows_ub, 64));
+    switch (epi) {
+        case EPI_STORE: k_gemm_simt<T, EPI_STORE><<<grid, 256, 0, st>>>(g); break;
+        case EPI_RELU: k_gemm_simt<T, EPI_RELU><<<grid, 256, 0, st>>>(g); break;
+        case EPI_RESID: k_gemm_simt<T, EPI_RESID><<<grid, 256, 0, st>>>(g); break;
+        case EPI_STATS: k_gemm_simt<T, EPI_STATS><<<grid, 256, 0, st>>>(g); break;
+        default: k_gemm_simt<T, EPI_F32><<<grid, 256, 0, st>>>(g); break;
+    }
+    KCHECK(h);
+    return 0;
+}
+
+template <typename T>
+int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* q_index, const void* k, const void* v,
+         int kv_stride, const int* kv_off, const int* seq, const int* nkeys, int cnt, int rows_ub, void* out,
+         int out_stride, int n_heads, int d_head, int max_keys, cudaStream_t st) {
+    if (rows_ub <= 0) return 0;
+    AttnArgs<T> a;
+    a.q = (const T*)q; a.q_stride = q_stride; a.q_index = q_index;
+    a.k = (const T*)k; a.v = (const T*)v; a.kv_stride = kv_stride; a.kv_off = kv_off;
+    a.pg.table = h->page_table; a.pg.page_tokens = h->cfg.page_tokens; a.pg.max_pages = h->pages_per_seq;
+    a.seq = seq; a.nkeys = nkeys; a.n_rows = h->ses.counters + cnt;
+    a.out = (T*)out; a.out_stride = out_stride;
+    a.n_heads = n_heads; a.d_head = d_head; a.max_keys = max_keys;
+    a.scale = 1.0f / sqrtf((float)d_head);
+    const int wpb = 4;
+    size_t smem = (size_t)wpb * (max_keys + d_head) * sizeof(float);
+    long long warps = (long long)rows_ub * n_heads;
+    int blocks = (int)((warps + wpb - 1) / wpb);
+    if (paged) k_attention<T, true><<<blocks, wpb * 32, smem, st>>>(a);
+    else k_attention<T, false><<<blocks, wpb * 32, smem, st>>>(a);
+    KCHECK(h);
+    return 0;
+}
+
+#define TRY(expr) do { int rc__ = (expr); if (rc__ != 0) return rc__; } while (0)
+
+// One pre-LN block on `rows_ub` rows of the residual stream x (encoder: no cross-attention).
+// Self-attention keys come from the block's own QKV rows (contiguous) or, for the verifier,
+// from the paged cache after the block's K/V were scattered into it.
+template <typename T>
+int block_self(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, const Rows& r, int cnt, int rows_ub,
+               int layer, bool verify, int max_keys, cudaStream_t st) {
+    const int d = m.dm.d_model, H = m.dm.n_heads, dh = d / H;
+    const size_t e = h->esz;
+    TRY(ln<T>(h, x, w.ln1_g, w.ln1_b, cnt, rows_ub, h->y, d, st));
+    TRY(gemm<T>(h, EPI_STORE, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, cnt, rows_ub, h->qkv, 3 * d, nullptr, st));
+    if (verify) {
+        Paged pg{h->page_table, h->cfg.page_tokens, h->pages_per_seq};
+        k_kv_scatter<T><<<rows_ub, 128, 0, st>>>((const T*)h->qkv, r.seq, r.pos, h->ses.counters + cnt, pg,
+                                                 (T*)h->kc[layer], (T*)h->vc[layer], d);
+        KCHECK(h);
+        TRY(attn<T>(h, true, h->qkv, 3 * d, nullptr, h->kc[layer], h->vc[layer], d, nullptr, r.seq, r.nk_self, cnt,
+                    rows_ub, h->att, d, H, dh, max_keys, st));
+    } else {
+        TRY(attn<T>(h, false, h->qkv, 3 * d, nullptr, (char*)h->qkv + (size_t)d * e, (char*)h->qkv + (size_t)2 * d * e,
+                    3 * d, r.kv_off, r.seq, r.nk_self, cnt, rows_ub, h->att, d, H, dh, max_keys, st));
+    }
+    TRY(gemm<T>(h, EPI_RESID, h->att, d, w.o_w, w.o_b, d, d, cnt, rows_ub, nullptr, 0, x, st));
+    return 0;
+}
+
+template <typename T>
+int block_cross(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, const Rows& r, int cnt, int rows_ub,
+                int layer, cudaStream_t st) {
+    const int d = m.dm.d_model, H = m.dm.n_heads, dh = d / H;
+    const size_t e = h->esz;
+    TRY(ln<T>(h, x, w.lnc_g, w.lnc_b, cnt, rows_ub, h->y, d, st));
+    TRY(gemm<T>(h, EPI_STORE, h->y, d, w.cq_w, w.cq_b, d, d, cnt, rows_ub, h->q, d, nullptr, st));
+    TRY(attn<T>(h, false, h->q, d, nullptr, m.ckv[layer], (char*)m.ckv[layer] + (size_t)d * e, 2 * d, r.kv_off_cross,
+                r.seq, r.nk_cross, cnt, rows_ub, h->att, d, H, dh, h->S_max, st));
+    TRY(gemm<T>(h, EPI_RESID, h->att, d, w.co_w, w.co_b, d, d, cnt, rows_ub, nullptr, 0, x, st));
+    return 0;
+}
+
+template <typename T>
+int block_ffn(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, int cnt, int rows_ub, cudaStream_t st) {
+    const int d = m.dm.d_model, f = m.dm.d_ffn;
+    TRY(ln<T>(h, x, w.ln2_g, w.ln2_b, cnt, rows_ub, h->y, d, st));
+    TRY(gemm<T>(h, EPI_RELU, h->y, d, w.w1, w.b1, f, d, cnt, rows_ub, h->hbuf, f, nullptr, st));
+    TRY(gemm<T>(h, EPI_RESID, h->hbuf, f, w.w2, w.b2, d, f, cnt, rows_ub, nullptr, 0, x, st));
+    return 0;
+}
+
+template <typename T>
+int embed(specdec_handle* h, const ModelW& m, const Rows& r, const float* pos_table, int cnt, int rows_ub,
+          cudaStream_t st) {
+    if (rows_ub <= 0) return 0;
+    const int d = m.dm.d_model;
+    k_embed<T><<<rows_ub, 128, 0, st>>>(r.tok, r.pos, h->ses.counters + cnt, (const T*)m.embed, pos_table, h->x, d,
+                                        sqrtf((float)d), m.dm.vocab, m.dm.max_pos);
+    KCHECK(h);
+    return 0;
+}
+
+// ---------------------------------------------------------------- encode
+template <typename T>
+int encode_model(specdec_handle* h, ModelW& m, const int* d_src, cudaStream_t st) {
+    const int R = h->B * h->S_max, d = m.dm.d_model;
+    k_enc_prep<<<cdiv(R, 256), 256, 0, st>>>(d_src, h->ses.src_len, h->B, h->S_max, h->rows, h->ses.counters);
+    KCHECK(h);
+    TRY(embed<T>(h, m, h->rows, m.pos_enc, CNT_ENC, R, st));
+    for (int l = 0; l < m.dm.enc_layers; ++l) {
+        TRY(block_self<T>(h, m, m.enc[l], h->x, h->rows, CNT_ENC, R, l, false, h->S_max, st));
+        TRY(block_ffn<T>(h, m, m.enc[l], h->x, CNT_ENC, R, st));
+    }
+    TRY(ln<T>(h, h->x, m.enc_lnf_g, m.enc_lnf_b, CNT_ENC, R, h->mem, d, st));
+    for (int l = 0; l < m.dm.dec_layers; ++l)
+        TRY(gemm<T>(h, EPI_STORE, h->mem, d, m.dec[l].ckv_w, m.dec[l].ckv_b, 2 * d, d, CNT_ENC, R, m.ckv[l], 2 * d,
+                    nullptr, st));
+    return 0;
+}
+
+template <typename T>
+int encode_impl(specdec_handle* h, const int* d_src, const int* d_src_len, const int* d_max_tgt, int B, int S_max,
+                cudaStream_t st) {
+    h->B = B; h->S_max = S_max; h->len_ub = 0;
+    h->encoded = false; h->verified = false; h->drafted = false;
+    k_session_init<<<cdiv(B, 128), 128, 0, st>>>(h->ses, d_src_len, d_max_tgt, B, h->T_cap, S_max);
+    KCHECK(h);
+    k_count_active<<<1, 32, 0, st>>>(h->ses, B);
+    KCHECK(h);
+    TRY(encode_model<T>(h, h->ver, d_src, st));
+    TRY(encode_model<T>(h, h->dra, d_src, st));
+    h->encoded = true;
+    return 0;
+}
+
+// ---------------------------------------------------------------- draft (Section 3.1.3)
+template <typename T>
+int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
+    ModelW& m = h->dra;
+    const int B = h->B, d = m.dm.d_model, H = m.dm.n_heads, dh = d / H, L = m.dm.dec_layers;
+    const size_t e = h->esz;
+    const int len_ub = std::min(h->len_ub, h->T_cap);
+    const int R1 = B * (len_ub + 1 + k), R2 = B * k, max_keys = len_ub + 1 + k;
+    k_draft_prep<<<1, 256, (2 * B + 2) * sizeof(int), st>>>(h->ses, B, k, h->S_max, h->cfg.bos_id, h->cfg.mask_id,
+                                                          h->rows, h->mrows);
+    KCHECK(h);
+    TRY(embed<T>(h, m, h->rows, m.pos_dec, CNT_DRAFT_ALL, R1, st));
+    for (int l = 0; l + 1 < L; ++l) {
+        TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_DRAFT_ALL, R1, l, false, max_keys, st));
+        TRY(block_cross<T>(h, m, m.dec[l], h->x, h->rows, CNT_DRAFT_ALL, R1, l, st));
+        TRY(block_ffn<T>(h, m, m.dec[l], h->x, CNT_DRAFT_ALL, R1, st));
+    }
+    // last layer: K/V from every row, queries and everything after them from the k mask rows only
+    const LayerW& w = m.dec[L - 1];
+    TRY(ln<T>(h, h->x, w.ln1_g, w.ln1_b, CNT_DRAFT_ALL, R1, h->y, d, st));
+    TRY(gemm<T>(h, EPI_STORE, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, CNT_DRAFT_ALL, R1, h->qkv, 3 * d, nullptr, st));
+    k_gather_rows<<<R2, 128, 0, st>>>(h->x, h->mrows.src_row, h->ses.counters + CNT_DRAFT_MASK, h->x2, d);
+    KCHECK(h);
+    TRY(attn<T>(h, false, h->qkv, 3 * d, h->mrows.src_row, (char*)h->qkv + (size_t)d * e,
+                (char*)h->qkv + (size_t)2 * d * e, 3 * d, h->mrows.kv_off, h->mrows.seq, h->mrows.nk_self,
+                CNT_DRAFT_MASK, R2, h->att, d, H, dh, max_keys, st));
+    TRY(gemm<T>(h, EPI_RESID, h->att, d, w.o_w, w.o_b, d, d, CNT_DRAFT_MASK, R2, nullptr, 0, h->x2, st));
+    TRY(block_cross<T>(h, m, w, h->x2, h->mrows, CNT_DRAFT_MASK, R2, L - 1, st));
+    TRY(block_ffn<T>(h, m, w, h->x2, CNT_DRAFT_MASK, R2, st));
+    TRY(ln<T>(h, h->x2, m.dec_lnf_g, m.dec_lnf_b, CNT_DRAFT_MASK, R2, h->y, d, st));
+    int n_tiles = 0;
+    TRY(gemm<T>(h, EPI_STATS, h->y, d, m.embed, nullptr, m.dm.vocab, d, CNT_DRAFT_MASK, R2, nullptr, 0, nullptr, st,
+                nullptr, nullptr, &n_tiles));
+    k_draft_argmax<<<cdiv(R2, 4), 128, 0, st>>>(h->part, n_tiles, h->ses.counters + CNT_DRAFT_MASK, h->mrows.slot,
+                                               d_draft);
+    KCHECK(h);
+    h->drafted = true; h->verified = false;
+    h->last_draft_rows_ub = R2;
+    return 0;
+}
+
+// ---------------------------------------------------------------- verify (Section 2, Section 3.2)
+template <typename T>
+int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float tau, int* d_accepted, int* d_bif,
+                cudaStream_t st) {
+    ModelW& m = h->ver;
+    const int B = h->B, d = m.dm.d_model, L = m.dm.dec_layers, M = B * (k + 1);
+    const int max_keys = std::min(h->len_ub, h->T_cap) + k + 1;
+    if (d_draft != h->v_draft)
+        CUDA_TRY(h, cudaMemcpyAsync(h->v_draft, d_draft, (size_t)B * k * 4, cudaMemcpyDeviceToDevice, st));
+    k_verify_prep<<<cdiv(M, 256), 256, 0, st>>>(h->ses, h->v_draft, B, k, h->S_max, h->cfg.bos_id, h->rows);
+    KCHECK(h);
+    TRY(embed<T>(h, m, h->rows, m.pos_dec, CNT_VERIFY, M, st));
+    for (int l = 0; l < L; ++l) {
+        TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, l, true, max_keys, st));
+        TRY(block_cross<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, l, st));
+        TRY(block_ffn<T>(h, m, m.dec[l], h->x, CNT_VERIFY, M, st));
+    }
+    TRY(ln<T>(h, h->x, m.dec_lnf_g, m.dec_lnf_b, CNT_VERIFY, M, h->y, d, st));
+    k_draft_logit<T><<<cdiv(M, 4), 128, 0, st>>>((const T*)h->y, (const T*)m.embed, h->v_draft, B, k, d, m.dm.vocab,
+                                                 h->ld, h->ld_id);
+    KCHECK(h);
+    int n_tiles = 0;
+    TRY(gemm<T>(h, EPI_STATS, h->y, d, m.embed, nullptr, m.dm.vocab, d, CNT_VERIFY, M, nullptr, 0, nullptr, st, h->ld,
+                h->ld_id, &n_tiles));
+    k_accept<<<B, 256, (size_t)(k + 1) * sizeof(RowPart), st>>>(h->part, n_tiles, h->ld, h->ld_id, k, beta, tau,
+                                                                h->accepted, h->bif, h->row_stats);
+    KCHECK(h);
+    if (d_accepted) CUDA_TRY(h, cudaMemcpyAsync(d_accepted, h->accepted, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
+    if (d_bif) CUDA_TRY(h, cudaMemcpyAsync(d_bif, h->bif, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
+    h->last_k = k; h->verified = true; h->drafted = false;
+    return 0;
+}
+
+int commit_impl(specdec_handle* h, const int* d_keep, const int* d_next, cudaStream_t st) {
+    const int k = h->last_k;
+    k_commit<<<cdiv(h->B, 128), 128, 0, st>>>(h->ses, h->v_draft, d_keep ? d_keep : h->accepted,
+                                             d_next ? d_next : h->bif, h->B, k, h->cfg.eos_id);
+    KCHECK(h);
+    h->len_ub = std::min(h->len_ub + k + 1, h->T_cap);
+    h->verified = false;
+    return 0;
+}
+
+template <typename T>
+int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, const int* d_max_tgt, int B, int S_max,
+                  int k, int beta, float tau, int* d_out, int out_stride, int* d_out_len, specdec_stats* hs,
+                  cudaStream_t st) {
+    const bool timed = hs != nullptr;
+    size_t ev = 0;
+    auto mark = [&]() { if (timed && ev < h->time_ev.size()) cudaEventRecord(h->time_ev[ev++], st); };
+    mark();
+    TRY(encode_impl<T>(h, d_src, d_src_len, d_max_tgt, B, S_max, st));
+    mark();
+    const int max_iters = h->T_cap;            // every iteration commits >= 1 token per unfinished sequence
+    const int lag = 2, slots = (int)h->poll_ev.size();
+    int it = 0;
+    for (; it < max_iters; ++it) {
+        TRY(draft_impl<T>(h, k, h->g_draft, st));
+        mark();
+        TRY(verify_impl<T>(h, h->g_draft, k, beta, tau, nullptr, nullptr, st));
+        mark();
+        TRY(commit_impl(h, nullptr, nullptr, st));
+        mark();
+        CUDA_TRY(h, cudaMemcpyAsync(h->h_poll + (it % slots), h->ses.counters + CNT_ACTIVE, 4, cudaMemcpyDeviceToHost, st));
+        CUDA_TRY(h, cudaEventRecord(h->poll_ev[it % slots], st));
+        if (it >= lag) {
+            CUDA_TRY(h, cudaEventSynchronize(h->poll_ev[(it - lag) % slots]));
+            if (h->h_poll[(it - lag) % slots] == 0) { ++it; break; }
+        }
+    }
+    if (d_out || d_out_len) TRY(specdec_get_output(h, d_out, out_stride, d_out_len, nullptr, st));
+    CUDA_TRY(h, cudaMemcpyAsync(h->h_stats, h->ses.stats, 32, cudaMemcpyDeviceToHost, st));
+    mark();
+    CUDA_TRY(h, cudaStreamSynchronize(st));
+    if (hs) {
+        memset(hs, 0, sizeof(*hs));
+        hs->iterations = it;
+        hs->seq_iterations = (long long)h->h_stats[0];
+        hs->drafted = (long long)h->h_stats[1];
+        hs->accepted = (long long)h->h_stats[2];
+        hs->emitted = (long long)h->h_stats[3];
+        auto ms = [&](size_t a, size_t b) { float t = 0.f; if (b < ev) cudaEventElapsedTime(&t, h->time_ev[a], h->time_ev[b]); return (double)t; };
+        hs->ms_encode = ms(0, 1);
+        for (int i = 0; i < it; ++i) {
+            size_t b0 = 1 + (size_t)i * 3;
+            hs->ms_draft += ms(b0, b0 + 1);
+            hs->ms_verify += ms(b0 + 1, b0 + 2);
+            hs->ms_commit += ms(b0 + 2, b0 + 3);
+        }
+        hs->ms_total = ms(0, ev - 1);
+    }
+    return 0;
+}
+
+int check_model(const specdec_model_dims& m, const char* who, std::string& why) {
+    if (m.d_model <= 0 || m.n_heads <= 0 || m.d_ffn <= 0 || m.vocab <= 0 || m.enc_layers < 0 || m.dec_layers < 1 ||
+        m.max_pos <= 0) { why = std::string(who) + ": non-positive dimension"; return -1; }
+    if (m.d_model % m.n_heads) { why = std::string(who) + ": d_model not divisible by n_heads"; return -1; }
+    if (m.d_model % 16 || m.d_ffn % 16) { why = std::string(who) + ": d_model and d_ffn must be multiples of 16"; return -1; }
+    return 0;
+}
+
+}  // namespace
+
+// ================================================================== C ABI
+extern "C" {
+
+const char* specdec_last_error(const specdec_handle* h) { return h ? h->err.c_str() : g_create_error.c_str(); }
+
+long long specdec_launch_count(const specdec_handle* h) { return h ? h->launches : 0; }
+
+int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int n_weights, void* stream,
+                   specdec_handle** out) {
+    if (out) *out = nullptr;
+    if (!cfg || !weights || !out || n_weights <= 0) return fail(nullptr, SPECDEC_ERR_INVALID_ARG, "null argument");
+    std::string why;
+    if (check_model(cfg->verifier, "verifier", why) || check_model(cfg->drafter, "drafter", why))
+        return fail(nullptr, SPECDEC_ERR_INVALID_ARG, why);
+    if (cfg->k_max < 1 || cfg->max_batch < 1 || cfg->max_src < 1 || cfg->max_tgt < 1)
+        return fail(nullptr, SPECDEC_ERR_INVALID_ARG, "k_max, max_batch, max_src, max_tgt must be >= 1");
+    if (cfg->page_tokens < 1 || (cfg->page_tokens & (cfg->page_tokens - 1)))
+        return fail(nullptr, SPECDEC_ERR_INVALID_ARG, "page_tokens must be a power of two");
+    if (cfg->compute_dtype != SPECDEC_DTYPE_F32 && cfg->compute_dtype != SPECDEC_DTYPE_BF16)
+        return fail(nullptr, SPECDEC_ERR_INVALID_ARG, "compute_dtype must be 0 (fp32) or 1 (bf16)");
+    if (cfg->verifier.vocab != cfg->drafter.vocab)
+        return fail(nullptr, SPECDEC_ERR_INVALID_ARG, "verifier and drafter must share the vocabulary");
+    const int need_pos = cfg->max_tgt + cfg->k_max + 1;
+    if (cfg->verifier.max_pos < need_pos || cfg->drafter.max_pos < need_pos || cfg->verifier.max_pos < cfg->max_src ||
+        cfg->drafter.max_pos < cfg->max_src)
+        return fail(nullptr, SPECDEC_ERR_CAPACITY, "max_pos must cover max_src and max_tgt + k_max + 1");
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0)
+        return fail(nullptr, SPECDEC_ERR_CUDA, "no CUDA device: this library has no CPU path");
+    cudaStream_t st = (cudaStream_t)stream;
+    specdec_handle* h = new specdec_handle();
+    h->cfg = *cfg;
+    h->dtype = cfg->compute_dtype;
+    h->esz = h->dtype == SPECDEC_DTYPE_BF16 ? 2 : 4;
+    h->B_cap = cfg->max_batch; h->S_cap = cfg->max_src; h->T_cap = cfg->max_tgt; h->k_cap = cfg->k_max;
+    h->d_max = std::max(cfg->verifier.d_model, cfg->drafter.d_model);
+    h->f_max = std::max(cfg->verifier.d_ffn, cfg->drafter.d_ffn);
+    h->v_max = cfg->verifier.vocab;
+    h->M_cap = h->B_cap * (h->k_cap + 1);
+    h->R2_cap = h->B_cap * h->k_cap;
+    h->R_cap = std::max(std::max(h->B_cap * h->S_cap, h->B_cap * (h->T_cap + 1 + h->k_cap)), h->M_cap);
+    h->pages_per_seq = cdiv(h->T_cap + h->k_cap + 1, cfg->page_tokens);
+    h->n_tiles_cap = cdiv(h->v_max, 64);
+    layout_all(h);                       // dry run: sizes only
+    const size_t total = h->arena.off + 256;
+    char* base = nullptr;
+    cudaError_t ce = cudaMalloc((void**)&base, total);
+    if (ce != cudaSuccess) {
+        std::string msg = std::string("arena allocation of ") + std::to_string(total) + " bytes: " + cudaGetErrorString(ce);
+        delete h;
+        return fail(nullptr, SPECDEC_ERR_CUDA, msg);
+    }
+    h->arena.base = base;
+    layout_all(h);
+    auto bail = [&](int code, const std::string& msg) { cudaFree(base); delete h; return fail(nullptr, code, msg); };
+    Manifest mf;
+    for (int i = 0; i < n_weights; ++i)
+        if (weights[i].name) mf.map[weights[i].name] = &weights[i];
+    if (h->dtype == SPECDEC_DTYPE_BF16) {
+        load_model<bf16>(h, h->ver, "verifier.", mf, st);
+        load_model<bf16>(h, h->dra, "drafter.", mf, st);
+    } else {
+        load_model<float>(h, h->ver, "verifier.", mf, st);
+        load_model<float>(h, h->dra, "drafter.", mf, st);
+    }
+    if (!mf.missing.empty()) { cudaStreamSynchronize(st); return bail(SPECDEC_ERR_SHAPE, "missing weight: " + mf.missing); }
+    if (!mf.bad.empty()) { cudaStreamSynchronize(st); return bail(SPECDEC_ERR_SHAPE, "weight with wrong dtype/shape: " + mf.bad); }
+    // page table: sequence b owns pages {i * B_cap + b}: interleaved, so the indirection is exercised
+    {
+        std::vector<int> pt((size_t)h->B_cap * h->pages_per_seq);
+        for (int b = 0; b < h->B_cap; ++b)
+            for (int i = 0; i < h->pages_per_seq; ++i) pt[(size_t)b * h->pages_per_seq + i] = i * h->B_cap + b;
+        ce = cudaMemcpyAsync(h->page_table, pt.data(), pt.size() * 4, cudaMemcpyHostToDevice, st);
+        if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+        if (ce != cudaSuccess) return bail(SPECDEC_ERR_CUDA, std::string("page table upload: ") + cudaGetErrorString(ce));
+    }
+    ce = cudaStreamSynchronize(st);
+    if (ce == cudaSuccess) ce = cudaGetLastError();
+    if (ce != cudaSuccess) return bail(SPECDEC_ERR_CUDA, std::string("weight repacking: ") + cudaGetErrorString(ce));
+    if (cudaMallocHost((void**)&h->h_poll, 64 * 4) != cudaSuccess || cudaMallocHost((void**)&h->h_stats, 64) != cudaSuccess)
+        return bail(SPECDEC_ERR_CUDA, "pinned host allocation failed");
+    h->poll_ev.resize(8);
+    for (auto& e : h->poll_ev) cudaEventCreateWithFlags(&e, cudaEventDisableTiming);
+    h->time_ev.resize((size_t)3 * h->T_cap + 8);
+    for (auto& e : h->time_ev) cudaEventCreate(&e);
+    // attention keeps one row of scores per warp in shared memory
+    {
+        const int max_keys = std::max(h->S_cap, h->T_cap + h->k_cap + 1);
+        const int dh = std::max(cfg->verifier.d_model / cfg->verifier.n_heads, cfg->drafter.d_model / cfg->drafter.n_heads);
+        const int smem = 4 * (max_keys + dh) * 4;
+        if (smem > 200 * 1024) return bail(SPECDEC_ERR_CAPACITY, "max_src / max_tgt too large for the attention kernel");
+        if (smem > 48 * 1024) {
+            if (h->dtype == SPECDEC_DTYPE_BF16) {
+                cudaFuncSetAttribute(k_attention<bf16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+                cudaFuncSetAttribute(k_attention<bf16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            } else {
+                cudaFuncSetAttribute(k_attention<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+                cudaFuncSetAttribute(k_attention<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            }
+        }
+    }
+    if (h->dtype == SPECDEC_DTYPE_BF16) {
+        if (sd::tc_init(h->tma) != 0) h->use_tc = 0;     // reported through specdec_last_error; SIMT GEMM still runs on the GPU
+        if (!h->use_tc) h->err = "tensor-core GEMM unavailable: " + h->tma.err;
+    } else {
+        h->use_tc = 0;
+    }
+    *out = h;
+    return SPECDEC_OK;
+}
+
+int specdec_destroy(specdec_handle* h) {
+    if (!h) return SPECDEC_ERR_INVALID_ARG;
+    cudaDeviceSynchronize();
+    for (auto& e : h->poll_ev) cudaEventDestroy(e);
+    for (auto& e : h->time_ev) cudaEventDestroy(e);
+    if (h->h_poll) cudaFreeHost(h->h_poll);
+    if (h->h_stats) cudaFreeHost(h->h_stats);
+    if (h->arena.base) cudaFree(h->arena.base);
+    delete h;
+    return SPECDEC_OK;
+}
+
+int specdec_set_option(specdec_handle* h, const char* name, int value) {
+    if (!h || !name) return SPECDEC_ERR_INVALID_ARG;
+    if (!strcmp(name, "gemm")) {
+        if (value && (h->dtype != SPECDEC_DTYPE_BF16 || !h->tma.ready))
+            return fail(h, SPECDEC_ERR_UNSUPPORTED, "tensor-core GEMM needs a bf16 handle on an sm_100 device");
+        h->use_tc = value ? 1 : 0;
+        return SPECDEC_OK;
+    }
+    if (!strcmp(name, "graphs")) { h->use_graphs = value ? 1 : 0; return SPECDEC_OK; }
+    return fail(h, SPECDEC_ERR_INVALID_ARG, std::string("unknown option: ") + name);
+}
+
+#define DISPATCH(h, call_bf16, call_f32) ((h)->dtype == SPECDEC_DTYPE_BF16 ? (call_bf16) : (call_f32))
+
+int specdec_encode(specdec_handle* h, const int32_t* d_src, const int32_t* d_src_len, const int32_t* d_max_tgt, int B,
+                   int S_max, void* stream) {
+    if (!h) return SPECDEC_ERR_INVALID_ARG;
+    if (!d_src || !d_src_len || B < 1 || S_max < 1) return fail(h, SPECDEC_ERR_INVALID_ARG, "encode: bad argument");
+    if (B > h->B_cap || S_max > h->S_cap) return fail(h, SPECDEC_ERR_CAPACITY, "encode: B or S_max beyond capacity");
+    cudaStream_t st = (cudaStream_t)stream;
+    return DISPATCH(h, encode_impl<bf16>(h, d_src, d_src_len, d_max_tgt, B, S_max, st),
+                    encode_impl<float>(h, d_src, d_src_len, d_max_tgt, B, S_max, st));
+}
+
+int specdec_draft(specdec_handle* h, int k, int32_t* d_draft, void* stream) {
+    if (!h) return SPECDEC_ERR_INVALID_ARG;
+    if (!h->encoded) return fail(h, SPECDEC_ERR_NOT_ENCODED, "draft: no session (call specdec_encode)");
+    if (!d_draft) return fail(h, SPECDEC_ERR_INVALID_ARG, "draft: null output");
+    if (k < 1 || k > h->k_cap) return fail(h, SPECDEC_ERR_CAPACITY, "draft: k outside [1, k_max]");
+    cudaStream_t st = (cudaStream_t)stream;
+    return DISPATCH(h, draft_impl<bf16>(h, k, d_draft, st), draft_impl<float>(h, k, d_draft, st));
+}
+
+int specdec_verify(specdec_handle* h, const int32_t* d_draft, int k, int beta, float tau, int32_t* d_accepted,
+                   int32_t* d_bif, void* stream) {
+    if (!h) return SPECDEC_ERR_INVALID_ARG;
+    if (!h->encoded) return fail(h, SPECDEC_ERR_NOT_ENCODED, "verify: no session (call specdec_encode)");
+    if (!d_draft) return fail(h, SPECDEC_ERR_INVALID_ARG, "verify: null drafts");
+    if (k < 1 || k > h->k_cap) return fail(h, SPECDEC_ERR_CAPACITY, "verify: k outside [1, k_max]");
+    if (beta < 1 || !(tau >= 0.f)) return fail(h, SPECDEC_ERR_INVALID_ARG, "verify: beta >= 1 and tau >= 0 required");
+    cudaStream_t st = (cudaStream_t)stream;
+    return DISPATCH(h, verify_impl<bf16>(h, d_draft, k, beta, tau, d_accepted, d_bif, st),
+                    verify_impl<float>(h, d_draft, k, beta, tau, d_accepted, d_bif, st));
+}
+
+int specdec_commit(specdec_handle* h, const int32_t* d_keep, const int32_t* d_next, void* stream) {
+    if (!h) return SPECDEC_ERR_INVALID_ARG;
+    if (!h->encoded) return fail(h, SPECDEC_ERR_NOT_ENCODED, "commit: no session (call specdec_encode)");
+    if (!h->verified) return fail(h, SPECDEC_ERR_INVALID_ARG, "commit: must follow specdec_verify");
+    return commit_impl(h, d_keep, d_next, (cudaStream_t)stream);
+}
+
+int specdec_get_output(specdec_handle* h, int32_t* d_out, int out_stride, int32_t* d_out_len, int32_t* d_finished,
+                       void* stream) {
+    if (!h) return SPECDEC_ERR_INVALID_ARG;
+    if (!h->B) return fail(h, SPECDEC_ERR_NOT_ENCODED, "get_output: no session");
+    if (d_out && out_stride < 1) return fail(h, SPECDEC_ERR_INVALID_ARG, "get_output: out_stride < 1");
+    k_copy_out<<<h->B, 128, 0, (cudaStream_t)stream>>>(h->ses, h->B, d_out, out_stride, d_out_len, d_finished);
+    KCHECK(h);
+    return SPECDEC_OK;
+}
+
+int specdec_generate(specdec_handle* h, const int32_t* d_src, const int32_t* d_src_len, const int32_t* d_max_tgt, int B,
+                     int S_max, int k, int beta, float tau, int32_t* d_out, int out_stride, int32_t* d_out_len,
+                     specdec_stats* h_stats, void* stream) {
+    if (!h) return SPECDEC_ERR_INVALID_ARG;
+    if (!d_src || !d_src_len || !d_out || !d_out_len || B < 1 || S_max < 1 || out_stride < 1)
+        return fail(h, SPECDEC_ERR_INVALID_ARG, "generate: bad argument");
+    if (B > h->B_cap || S_max > h->S_cap) return fail(h, SPECDEC_ERR_CAPACITY, "generate: B or S_max beyond capacity");
+    if (k < 1 || k > h->k_cap) return fail(h, SPECDEC_ERR_CAPACITY, "generate: k outside [1, k_max]");
+    if (beta < 1 || !(tau >= 0.f)) return fail(h, SPECDEC_ERR_INVALID_ARG, "generate: beta >= 1 and tau >= 0 required");
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = DISPATCH(h, generate_impl<bf16>(h, d_src, d_src_len, d_max_tgt, B, S_max, k, beta, tau, d_out, out_stride, d_out_len, h_stats, st),
+                      generate_impl<float>(h, d_src, d_src_len, d_max_tgt, B, S_max, k, beta, tau, d_out, out_stride, d_out_len, h_stats, st));
+    if (h_stats) h_stats->status = rc;
+    return rc;
+}
+
+int specdec_generate_host(specdec_handle* h, const int32_t* h_src, const int32_t* h_src_len, const int32_t* h_max_tgt,
+                          int B, int S_max, int k, int beta, float tau, int32_t* h_out, int out_stride,
+                          int32_t* h_out_len, specdec_stats* h_stats, void* stream) {
+    if (!h) return SPECDEC_ERR_INVALID_ARG;
+    if (!h_src || !h_src_len || !h_out || !h_out_len || B < 1 || S_max < 1 || out_stride < 1)
+        return fail(h, SPECDEC_ERR_INVALID_ARG, "generate_host: bad argument");
+    if (B > h->B_cap || S_max > h->S_cap) return fail(h, SPECDEC_ERR_CAPACITY, "generate_host: B or S_max beyond capacity");
+    cudaStream_t st = (cudaStream_t)stream;
+    int *s_src = h->stage_src, *s_len = h->stage_len, *s_mt = h->stage_mt;
+    CUDA_TRY(h, cudaMemcpyAsync(s_src, h_src, (size_t)B * S_max * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(h, cudaMemcpyAsync(s_len, h_src_len, (size_t)B * 4, cudaMemcpyHostToDevice, st));
+    if (h_max_tgt) CUDA_TRY(h, cudaMemcpyAsync(s_mt, h_max_tgt, (size_t)B * 4, cudaMemcpyHostToDevice, st));
+    if (k < 1 || k > h->k_cap) return fail(h, SPECDEC_ERR_CAPACITY, "generate_host: k outside [1, k_max]");
+    if (beta < 1 || !(tau >= 0.f)) return fail(h, SPECDEC_ERR_INVALID_ARG, "generate_host: beta >= 1 and tau >= 0 required");
+    // the ids and lengths are read straight from the session arrays afterwards
+    const int* mt = h_max_tgt ? s_mt : nullptr;
+    int rc = DISPATCH(h, generate_impl<bf16>(h, s_src, s_len, mt, B, S_max, k, beta, tau, nullptr, 1, nullptr, h_stats, st),
+                      generate_impl<float>(h, s_src, s_len, mt, B, S_max, k, beta, tau, nullptr, 1, nullptr, h_stats, st));
+    if (h_stats) h_stats->status = rc;
+    if (rc != 0) return rc;
+    const int w = std::min(out_stride, h->ses.out_stride);
+    CUDA_TRY(h, cudaMemcpy2DAsync(h_out, (size_t)out_stride * 4, h->ses.out, (size_t)h->ses.out_stride * 4, (size_t)w * 4,
+                                  B, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(h, cudaMemcpyAsync(h_out_len, h->ses.len, (size_t)B * 4, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(h, cudaStreamSynchronize(st));
+    return SPECDEC_OK;
+}
+
+int specdec_accept_scan(const float* d_logits, const int32_t* d_draft, int B, int k, int V, int beta, float tau,
+                        int32_t* d_accepted, int32_t* d_bif, void* stream) {
+    if (!d_logits || !d_draft || !d_accepted || !d_bif || B < 1 || k < 1 || V < 1 || beta < 1 || !(tau >= 0.f))
+        return fail(nullptr, SPECDEC_ERR_INVALID_ARG, "accept_scan: bad argument");
+    k_accept_logits<<<B, 256, 0, (cudaStream_t)stream>>>(d_logits, d_draft, k, V, beta, tau, d_accepted, d_bif);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(nullptr, SPECDEC_ERR_CUDA, std::string("accept_scan: ") + cudaGetErrorString(e));
+    return SPECDEC_OK;
+}
+
+int specdec_debug_logits(specdec_handle* h, int which, float* d_logits, void* stream) {
+    if (!h || !d_logits) return SPECDEC_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    int cnt, rows; const ModelW* m;
+    if (which == 0) { if (!h->verified) return fail(h, SPECDEC_ERR_INVALID_ARG, "debug_logits: no verify pass to replay");
+        cnt = CNT_VERIFY; rows = h->B * (h->last_k + 1); m = &h->ver; }
+    else { if (!h->drafted) return fail(h, SPECDEC_ERR_INVALID_ARG, "debug_logits: no draft pass to replay");
+        cnt = CNT_DRAFT_MASK; rows = h->last_draft_rows_ub; m = &h->dra; }
+    const int d = m->dm.d_model, V = m->dm.vocab;
+    return DISPATCH(h, gemm<bf16>(h, EPI_F32, h->y, d, m->embed, nullptr, V, d, cnt, rows, nullptr, 0, d_logits, st),
+                    gemm<float>(h, EPI_F32, h->y, d, m->embed, nullptr, V, d, cnt, rows, nullptr, 0, d_logits, st));
+}
+
+int specdec_debug_row_stats(specdec_handle* h, float* d_stats, void* stream) {
+    if (!h || !d_stats) return SPECDEC_ERR_INVALID_ARG;
+    if (!h->verified) return fail(h, SPECDEC_ERR_INVALID_ARG, "debug_row_stats: no verify pass");
+    CUDA_TRY(h, cudaMemcpyAsync(d_stats, h->row_stats, (size_t)h->B * (h->last_k + 1) * 6 * 4, cudaMemcpyDeviceToDevice,
+                                (cudaStream_t)stream));
+    return SPECDEC_OK;
+}
+
+}  // extern "C"
