@@ -1,18 +1,387 @@
-// Tensor-core GEMM interface (tcgen05 / TMEM / TMA).  Placeholder until the kernel lands:
-// reports "unavailable" so every contraction runs in the SIMT reference GEMM on the GPU.
+// Tensor-core GEMM for sm_100a:  C[r, n] = sum_k A[r, k] * W[n, k]  (bf16 operands, fp32 accumulate).
+//
+//   * operands are staged by TMA (cp.async.bulk.tensor, 128-byte swizzle) into a ring of shared
+//     memory stages, 64 K-elements (128 B) per row;
+//   * one elected thread issues tcgen05.mma (M = 128 activation rows, N = BN weight rows, K = 16
+//     per instruction) with the accumulator in tensor memory;
+//   * four epilogue warps read the accumulator back with tcgen05.ld (one TMEM lane = one output
+//     row per thread) and apply the fused epilogue: bias / ReLU / residual add / fp32 store / the
+//     per-row vocabulary statistics that replace the logits tensor.
+//
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, warps 2..5 = epilogue.
+// Every mbarrier wait is bounded; on a timeout the CTA flags an error word in global memory,
+// stops waiting everywhere, still releases its tensor memory and returns.
 #pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <map>
 #include <string>
+#include <tuple>
+
 #include "kernels.cuh"
 
 namespace sd {
 
-struct TmaEncoder {
-    bool ready = false;
-    std::string err = "not built";
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// Bounded wait: gives up after ~2e8 clocks, raises the CTA-wide abort flag and the global error word.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err_word,
+                                          int code) {
+    if (*abort_flag) return false;
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > 200000000LL) {
+            *abort_flag = 1;
+            atomicExch(err_word, code);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor: K-major tile, rows of 128 B, 128-byte swizzle, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);        // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                             // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                   // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                             // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                             // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+constexpr int TC_BM = 128, TC_BK = 64, TC_THREADS = 192;
+template <int BN> struct TcCfg {
+    static constexpr int STAGES = BN >= 256 ? 4 : (BN >= 128 ? 6 : 8);
+    static constexpr int STAGE_BYTES = (TC_BM + BN) * TC_BK * 2;
+    static constexpr int SMEM = STAGES * STAGE_BYTES + 1024;
 };
 
-inline bool tc_supported(int, int) { return false; }
-inline int tc_init(TmaEncoder&) { return -1; }
-inline int gemm_tc_launch(TmaEncoder&, int, GemmArgs<bf16>&, int, cudaStream_t, int*) { return -1; }
+template <int EPI, int BN>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, GemmArgs<bf16> g,
+          int* err_word) {
+    using Cfg = TcCfg<BN>;
+    constexpr int STAGES = Cfg::STAGES;
+    const int R = *g.n_rows;
+    const int m0 = blockIdx.y * TC_BM, n0 = blockIdx.x * BN;
+    if (m0 >= R) return;                       // whole CTA leaves before touching barriers or tensor memory
+
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[STAGES], bar_empty[STAGES], bar_acc;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+    const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nkb = g.K / TC_BK;
+
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&bar_full[s]), 1); mbar_init(smem_u32(&bar_empty[s]), 1); }
+        mbar_init(smem_u32(&bar_acc), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), BN < 32 ? 32 : BN);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = tmem_base_s;
+    volatile int* abort_flag = &abort_s;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = kb % STAGES;
+                if (kb >= STAGES) mbar_wait(smem_u32(&bar_empty[s]), ((kb / STAGES) - 1) & 1, abort_flag, err_word, 1);
+                if (*abort_flag) break;
+                const uint32_t a_dst = tiles + s * Cfg::STAGE_BYTES, w_dst = a_dst + TC_BM * TC_BK * 2;
+                const uint32_t bar = smem_u32(&bar_full[s]);
+                mbar_expect_tx(bar, Cfg::STAGE_BYTES);
+                tma_load_2d(a_dst, &tmA, kb * TC_BK, m0, bar);
+                tma_load_2d(w_dst, &tmW, kb * TC_BK, n0, bar);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, BN);
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = kb % STAGES;
+                mbar_wait(smem_u32(&bar_full[s]), (kb / STAGES) & 1, abort_flag, err_word, 2);
+                if (*abort_flag) break;
+                tc_fence_after();
+                const uint32_t a_src = tiles + s * Cfg::STAGE_BYTES, w_src = a_src + TC_BM * TC_BK * 2;
+                const uint64_t ad = umma_desc_k_sw128(a_src), wd = umma_desc_k_sw128(w_src);
+#pragma unroll
+                for (int k4 = 0; k4 < TC_BK / 16; ++k4)      // +32 bytes along K per instruction: 2 address units
+                    umma_bf16(tmem_d, ad + (uint64_t)(k4 * 2), wd + (uint64_t)(k4 * 2), idesc, (kb | k4) ? 1u : 0u);
+                umma_commit(smem_u32(&bar_empty[s]));        // stage reusable once these MMAs have read it
+            }
+            umma_commit(smem_u32(&bar_acc));                 // accumulator complete
+        }
+    } else {
+        const int q = warp & 3;                              // TMEM lane quadrant this warp may read
+        const int r = m0 + q * 32 + lane;
+        const bool live = mbar_wait(smem_u32(&bar_acc), 0, abort_flag, err_word, 3);
+        tc_fence_after();
+        const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16);
+        float v[32];
+        if (EPI == EPI_STATS) {
+            const float ld = (g.ld && r < R) ? g.ld[r] : CUDART_INF_F;
+            const int id = (g.ld_id && r < R) ? g.ld_id[r] : -1;
+            RowPart p; p.mx = -CUDART_INF_F; p.arg = 0x7fffffff; p.sum = 0.f; p.cnt = 0;
+            for (int c = 0; c < BN / 32; ++c) {
+                tmem_ld32(trow + c * 32, v);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const int n = n0 + c * 32 + j;
+                    if (n < g.N) {
+                        const float x = (n == id) ? ld : v[j];   // the draft's column takes the pre-pass value
+                        if (x > p.mx) { p.mx = x; p.arg = n; }
+                        p.cnt += (x > ld) ? 1 : 0;
+                    }
+                }
+            }
+            for (int c = 0; c < BN / 32; ++c) {
+                tmem_ld32(trow + c * 32, v);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const int n = n0 + c * 32 + j;
+                    if (n < g.N) p.sum += expf(((n == id) ? ld : v[j]) - p.mx);
+                }
+            }
+            if (live && r < R) g.part[(size_t)r * g.n_tiles + blockIdx.x] = p;
+        } else {
+            for (int c = 0; c < BN / 32; ++c) {
+                tmem_ld32(trow + c * 32, v);
+                const int nb = n0 + c * 32;
+                if (!live || r >= R) continue;
+                if (g.bias) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] += (nb + j < g.N) ? __ldg(g.bias + nb + j) : 0.f;
+                }
+                const bool full = nb + 32 <= g.N;
+                if (EPI == EPI_STORE || EPI == EPI_RELU) {
+                    bf16* o = g.out + (size_t)r * g.ldo + nb;
+                    if (full && (g.ldo % 8 == 0)) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            __align__(16) bf16 t[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) t[e] = __float2bfloat16_rn(EPI == EPI_RELU ? fmaxf(v[j + e], 0.f) : v[j + e]);
+                            *reinterpret_cast<uint4*>(o + j) = *reinterpret_cast<const uint4*>(t);
+                        }
+                    } else {
+                        for (int j = 0; j < 32; ++j)
+                            if (nb + j < g.N) o[j] = __float2bfloat16_rn(EPI == EPI_RELU ? fmaxf(v[j], 0.f) : v[j]);
+                    }
+                } else {
+                    float* o = g.resid + (size_t)r * g.N + nb;
+                    if (full && (g.N % 4 == 0)) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            float4 t = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                            if (EPI == EPI_RESID) {
+                                const float4 x = *reinterpret_cast<const float4*>(o + j);
+                                t.x += x.x; t.y += x.y; t.z += x.z; t.w += x.w;
+                            }
+                            *reinterpret_cast<float4*>(o + j) = t;
+                        }
+                    } else {
+                        for (int j = 0; j < 32; ++j)
+                            if (nb + j < g.N) o[j] = (EPI == EPI_RESID ? o[j] : 0.f) + v[j];
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_d, BN < 32 ? 32 : BN);
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TmaEncoder {
+    bool ready = false;
+    std::string err = "not initialised";
+    PFN_encodeTiled encode = nullptr;
+    int* err_word = nullptr;            // device word the kernels raise on a wait timeout
+    std::map<std::tuple<const void*, long long, int, int, int>, CUtensorMap> cache;
+
+    // 2-D bf16 tensor [rows, K] with row pitch ld elements; box = 64 x box_rows, 128-byte swizzle.
+    const CUtensorMap* get(const void* base, long long rows, int K, int ld, int box_rows) {
+        auto key = std::make_tuple(base, rows, K, ld, box_rows);
+        auto it = cache.find(key);
+        if (it != cache.end()) return &it->second;
+        CUtensorMap tm;
+        cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+        cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+        cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+        cuuint32_t estr[2] = {1, 1};
+        CUresult rc = encode(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (rc != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)rc); return nullptr; }
+        if (cache.size() > 4096) cache.clear();
+        return &(cache[key] = tm);
+    }
+};
+
+inline bool tc_supported(int N, int K) { return K % TC_BK == 0 && K >= TC_BK && N >= 32; }
+
+template <int EPI, int BN>
+inline cudaError_t tc_set_smem() {
+    return cudaFuncSetAttribute(k_gemm_tc<EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<BN>::SMEM);
+}
+template <int EPI>
+inline cudaError_t tc_set_smem_all() {
+    cudaError_t e = tc_set_smem<EPI, 32>();
+    if (e == cudaSuccess) e = tc_set_smem<EPI, 64>();
+    if (e == cudaSuccess) e = tc_set_smem<EPI, 128>();
+    if (e == cudaSuccess) e = tc_set_smem<EPI, 256>();
+    return e;
+}
+
+inline int tc_init(TmaEncoder& enc, int* err_word) {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+        enc.err = "cannot query the device"; return -1;
+    }
+    if (major != 10) { enc.err = "device is not sm_100"; return -1; }
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess) { enc.err = "cuTensorMapEncodeTiled not found in the driver"; return -1; }
+    enc.encode = (PFN_encodeTiled)fn;
+    cudaError_t e = tc_set_smem_all<EPI_STORE>();
+    if (e == cudaSuccess) e = tc_set_smem_all<EPI_RELU>();
+    if (e == cudaSuccess) e = tc_set_smem_all<EPI_RESID>();
+    if (e == cudaSuccess) e = tc_set_smem_all<EPI_F32>();
+    if (e == cudaSuccess) e = tc_set_smem<EPI_STATS, 128>();
+    if (e != cudaSuccess) { enc.err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return -1; }
+    enc.err_word = err_word;
+    enc.ready = true;
+    enc.err.clear();
+    return 0;
+}
+
+template <int EPI, int BN>
+inline int tc_launch_one(TmaEncoder& enc, GemmArgs<bf16>& g, int rows_ub, cudaStream_t st) {
+    const CUtensorMap* ta = enc.get(g.A, rows_ub, g.K, g.lda, TC_BM);
+    const CUtensorMap* tw = enc.get(g.W, g.N, g.K, g.K, BN);
+    if (!ta || !tw) return -1;
+    dim3 grid((g.N + BN - 1) / BN, (rows_ub + TC_BM - 1) / TC_BM);
+    k_gemm_tc<EPI, BN><<<grid, TC_THREADS, TcCfg<BN>::SMEM, st>>>(*ta, *tw, g, enc.err_word);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { enc.err = std::string("launch: ") + cudaGetErrorString(e); return -1; }
+    return 0;
+}
+
+template <int EPI>
+inline int tc_launch_bn(TmaEncoder& enc, int bn, GemmArgs<bf16>& g, int rows_ub, cudaStream_t st) {
+    switch (bn) {
+        case 256: return tc_launch_one<EPI, 256>(enc, g, rows_ub, st);
+        case 128: return tc_launch_one<EPI, 128>(enc, g, rows_ub, st);
+        case 64: return tc_launch_one<EPI, 64>(enc, g, rows_ub, st);
+        default: return tc_launch_one<EPI, 32>(enc, g, rows_ub, st);
+    }
+}
+
+// Picks the widest N tile that still yields at least one CTA per SM; otherwise the narrowest
+// (most CTAs streaming the weights).
+inline int tc_pick_bn(int N, int rows_ub) {
+    const int m_tiles = (rows_ub + TC_BM - 1) / TC_BM;
+    const int cand[4] = {256, 128, 64, 32};
+    for (int i = 0; i < 4; ++i) {
+        const int bn = cand[i];
+        if (bn > N) continue;
+        if ((long long)((N + bn - 1) / bn) * m_tiles >= 148) return bn;
+    }
+    return 32;
+}
+
+inline int gemm_tc_launch(TmaEncoder& enc, int epi, GemmArgs<bf16>& g, int rows_ub, cudaStream_t st, int* n_tiles_out) {
+    if (!enc.ready) return -1;
+    if (epi == EPI_STATS) {
+        if (g.N < 128) return -2;
+        g.n_tiles = (g.N + 127) / 128;
+        if (n_tiles_out) *n_tiles_out = g.n_tiles;
+        return tc_launch_one<EPI_STATS, 128>(enc, g, rows_ub, st);
+    }
+    const int bn = tc_pick_bn(g.N, rows_ub);
+    switch (epi) {
+        case EPI_STORE: return tc_launch_bn<EPI_STORE>(enc, bn, g, rows_ub, st);
+        case EPI_RELU: return tc_launch_bn<EPI_RELU>(enc, bn, g, rows_ub, st);
+        case EPI_RESID: return tc_launch_bn<EPI_RESID>(enc, bn, g, rows_ub, st);
+        default: return tc_launch_bn<EPI_F32>(enc, bn, g, rows_ub, st);
+    }
+}
 
 }  // namespace sd

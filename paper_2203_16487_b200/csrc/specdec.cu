@@ -280,7 +280,7 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
     g.n_rows = h->ses.counters + cnt; g.out = (T*)out; g.ldo = ldo; g.resid = resid;
     g.part = h->part; g.ld = ldv; g.ld_id = ld_id; g.n_tiles = cdiv(N, 64);
     if constexpr (std::is_same<T, bf16>::value) {
-        if (h->use_tc && sd::tc_supported(N, K)) {
+        if (h->use_tc && sd::tc_supported(N, K) && (epi != EPI_STATS || N >= 128)) {
             int rc = sd::gemm_tc_launch(h->tma, epi, g, rows_ub, st, n_tiles_out);
             if (rc != 0) return fail(h, SPECDEC_ERR_CUDA, "tensor-core GEMM launch failed: " + h->tma.err);
             ++h->launches;
@@ -529,8 +529,11 @@ int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, con
     }
     if (d_out || d_out_len) TRY(specdec_get_output(h, d_out, out_stride, d_out_len, nullptr, st));
     CUDA_TRY(h, cudaMemcpyAsync(h->h_stats, h->ses.stats, 32, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(h, cudaMemcpyAsync(h->h_stats + 4, h->ses.counters + 7, 4, cudaMemcpyDeviceToHost, st));
     mark();
     CUDA_TRY(h, cudaStreamSynchronize(st));
+    if (*(int*)(h->h_stats + 4) != 0)
+        return fail(h, SPECDEC_ERR_TIMEOUT, "a bounded device-side wait gave up (code " + std::to_string(*(int*)(h->h_stats + 4)) + ")");
     if (hs) {
         memset(hs, 0, sizeof(*hs));
         hs->iterations = it;
@@ -615,6 +618,7 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
     }
     h->arena.base = base;
     layout_all(h);
+    cudaMemsetAsync(base, 0, total, st);          // dead rows of every buffer read as zeros, never as NaN patterns
     auto bail = [&](int code, const std::string& msg) { cudaFree(base); delete h; return fail(nullptr, code, msg); };
     Manifest mf;
     for (int i = 0; i < n_weights; ++i)
@@ -663,7 +667,7 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
         }
     }
     if (h->dtype == SPECDEC_DTYPE_BF16) {
-        if (sd::tc_init(h->tma) != 0) h->use_tc = 0;     // reported through specdec_last_error; SIMT GEMM still runs on the GPU
+        if (sd::tc_init(h->tma, h->ses.counters + 7) != 0) h->use_tc = 0;     // reported through specdec_last_error; SIMT GEMM still runs on the GPU
         if (!h->use_tc) h->err = "tensor-core GEMM unavailable: " + h->tma.err;
     } else {
         h->use_tc = 0;

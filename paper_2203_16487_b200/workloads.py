@@ -231,9 +231,10 @@ def config5_prefix_and_rejections(batch: int, j: int, seed: int = 105):
 
 
 def sharp_tiny_models(seed: int = 31):
-    """Tiny models whose embedding table is N(0, 0.2^2): logits are sharp enough that tau binds."""
-    wv = make_weights(TINY_V, seed, False, embed_std=0.2)
-    wd = make_weights(TINY_D, seed + 1, False, embed_std=0.2)
+    """Tiny models whose embedding table is N(0, 0.06^2): top-1 to top-2 logit gaps are about 1,
+    so tau in {0.5, 1, 3} and beta change what is accepted."""
+    wv = make_weights(TINY_V, seed, False, embed_std=0.06)
+    wd = make_weights(TINY_D, seed + 1, False, embed_std=0.06)
     return wv, wd
 
 
