@@ -166,8 +166,20 @@ int specdec_accept_scan(const float* d_logits, const int32_t* d_draft, int B, in
 int specdec_debug_logits(specdec_handle* h, int which, float* d_logits, void* stream);
 int specdec_debug_row_stats(specdec_handle* h, float* d_stats, void* stream);
 
+/* Scripted drafts, a benchmark / test hook with no counterpart in the paper: random-init
+ * models almost never agree, so a workload's acceptance pattern is imposed instead.  After the
+ * drafter pass has run, draft i of a sequence with j committed tokens is replaced by
+ * d_script[b*stride + j + i] wherever that entry is >= 0.  d_script = NULL turns it off. */
+int specdec_set_draft_script(specdec_handle* h, const int32_t* d_script, int B, int stride, void* stream);
+
+/* With option "profile" = 1, every vocabulary-projection launch of draft and verify inside
+ * specdec_generate is bracketed by CUDA events; this returns their summed duration and count
+ * since the option was set. */
+int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches);
+
 /* Options: "gemm" = 0 SIMT reference GEMM, 1 tcgen05 GEMM (bf16 handles; default 1);
- * "graphs" = 0/1 replay draft/verify steps from CUDA graphs inside specdec_generate. */
+ * "graphs" = 0/1 replay draft/verify steps from CUDA graphs inside specdec_generate;
+ * "profile" = 0/1 (see specdec_profile_read). */
 int specdec_set_option(specdec_handle* h, const char* name, int value);
 
 /* Number of kernels the library has launched on this handle since create. */

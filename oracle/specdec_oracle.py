@@ -27,8 +27,9 @@ Pinned (tests/test_oracle_pins.py): greedy equivalence at beta=1, tau=0;
 brute-force log-prob form of Eq. 7-8 on tiny vocabularies; monotonicity in
 beta and tau; block-parallel == sequential rows; cached == from scratch; the
 worked example's iteration structure; the parameter count implied by the
-paper's memory table; a closed-form model with zeroed sublayers; numpy-free
-scalar re-computation of layer norm / attention on tiny shapes.
+paper's memory table; a closed-form model with zeroed sublayers; the whole
+encoder / decoder stack against torch.nn's pre-LN Transformer layers in fp64;
+every weight shown to influence the output.
 Parity unpinned: nothing about translation quality (needs trained weights).
 """
 from __future__ import annotations
@@ -315,10 +316,13 @@ class GenStats:
 def specdec_generate(mv: Model, md: Model, src: Sequence[int], max_tgt: int, k: int,
                      beta: int, tau: float, bos: int, eos: int, mask: int,
                      use_cache: bool = True, draft_fn=None,
-                     keep_trace: bool = False) -> Tuple[List[int], GenStats]:
+                     keep_trace: bool = False, script: Optional[Sequence[int]] = None
+                     ) -> Tuple[List[int], GenStats]:
     """Draft -> verify -> commit until EOS or max_tgt, one sequence.
 
     draft_fn(committed, k) may replace the drafter (scripted drafts in tests).
+    script (benchmark hook, no counterpart in the paper): after the drafter has run,
+    the draft for target index t is replaced by script[t] wherever script[t] >= 0.
     """
     mem_v = encode(mv, src)
     mem_d = encode(md, src) if draft_fn is None else None
@@ -328,6 +332,9 @@ def specdec_generate(mv: Model, md: Model, src: Sequence[int], max_tgt: int, k: 
     done = max_tgt <= 0
     while not done:
         d = draft(md, mem_d, out, k, bos, mask) if draft_fn is None else list(draft_fn(list(out), k))
+        if script is not None:
+            j = len(out)
+            d = [int(script[j + i]) if j + i < len(script) and script[j + i] >= 0 else d[i] for i in range(k)]
         rows = verify_rows(mv, mem_v, out, d, bos, cache)
         a, bif = verify(rows, d, beta, tau)
         n_before = len(out)

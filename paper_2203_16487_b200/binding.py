@@ -23,7 +23,7 @@ EXPORTS = [
     "specdec_create", "specdec_destroy", "specdec_encode", "specdec_draft", "specdec_verify",
     "specdec_commit", "specdec_generate", "specdec_generate_host", "specdec_get_output",
     "specdec_accept_scan", "specdec_debug_logits", "specdec_debug_row_stats", "specdec_set_option",
-    "specdec_launch_count", "specdec_last_error",
+    "specdec_launch_count", "specdec_last_error", "specdec_set_draft_script", "specdec_profile_read",
 ]
 
 
@@ -78,6 +78,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.specdec_debug_logits.argtypes = [vp, i, vp, vp]
     lib.specdec_debug_row_stats.argtypes = [vp, vp, vp]
     lib.specdec_set_option.argtypes = [vp, C.c_char_p, i]
+    lib.specdec_set_draft_script.argtypes = [vp, ip, i, i, vp]
+    lib.specdec_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
     lib.specdec_launch_count.argtypes = [vp]
     lib.specdec_launch_count.restype = C.c_longlong
     lib.specdec_last_error.argtypes = [vp]
@@ -170,6 +172,20 @@ class SpecDec:
 
     def set_option(self, name: str, value: int):
         self._check(self._lib.specdec_set_option(self._h, name.encode(), int(value)))
+
+    def set_draft_script(self, script):
+        """script [B, n] int32 (or None): entries >= 0 replace the drafter's output at that target index."""
+        if script is None:
+            self._check(self._lib.specdec_set_draft_script(self._h, None, 0, 0, _stream()))
+            return
+        t = self._i32(script)
+        self._check(self._lib.specdec_set_draft_script(self._h, _ptr(t), int(t.shape[0]), int(t.shape[1]), _stream()))
+        torch.cuda.current_stream().synchronize()
+
+    def profile_read(self):
+        ms, n = C.c_double(), C.c_longlong()
+        self._check(self._lib.specdec_profile_read(self._h, C.byref(ms), C.byref(n)))
+        return ms.value, n.value
 
     def last_error(self) -> str:
         return self._lib.specdec_last_error(self._h).decode()

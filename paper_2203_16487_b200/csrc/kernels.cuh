@@ -488,6 +488,18 @@ __global__ void k_draft_argmax(const RowPart* __restrict__ part, int n_tiles, co
     if (lane == 0) draft[slot[row]] = arg;
 }
 
+// Scripted drafts (benchmark / test hook): draft i of a sequence with j committed tokens is
+// replaced by script[b, j + i] where that entry is >= 0.  The drafter pass has already run.
+__global__ void k_apply_script(Session s, const int* __restrict__ script, int stride, int B, int k,
+                               int* __restrict__ draft) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= B * k) return;
+    int b = i / k, c = i % k;
+    if (s.finished[b]) return;
+    int p = s.len[b] + c;
+    if (p < stride) { int t = script[(size_t)b * stride + p]; if (t >= 0) draft[i] = t; }
+}
+
 // ------------------------------------------------------------------ commit / rollback (Eq. 3)
 // Appends drafts[0..keep) and the next token, cuts after the first EOS and at max_tgt.
 // Cache rows beyond the new length are simply dead: the next block overwrites them.

@@ -85,6 +85,14 @@ struct specdec_handle {
     std::vector<cudaEvent_t> poll_ev;
     std::vector<cudaEvent_t> time_ev;
     sd::TmaEncoder tma;
+    // scripted drafts (benchmark / test hook) and dominant-kernel timing
+    int* script = nullptr;          // device [B_cap, T_cap + k_cap] or unset
+    bool script_on = false;
+    int profile = 0;
+    std::vector<cudaEvent_t> prof_ev;
+    size_t prof_n = 0;
+    double prof_ms = 0.0;
+    long long prof_launches = 0;
     std::string err;
 };
 
@@ -185,6 +193,7 @@ void layout_all(specdec_handle* h) {
     h->stage_src = (int*)A.take((size_t)h->B_cap * h->S_cap * 4);
     h->stage_len = (int*)A.take((size_t)h->B_cap * 4);
     h->stage_mt = (int*)A.take((size_t)h->B_cap * 4);
+    h->script = (int*)A.take((size_t)h->B_cap * (h->T_cap + h->k_cap) * 4);
     Session& s = h->ses;
     s.len = (int*)A.take((size_t)h->B_cap * 4);
     s.finished = (int*)A.take((size_t)h->B_cap * 4);
@@ -325,6 +334,24 @@ int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* 
 
 #define TRY(expr) do { int rc__ = (expr); if (rc__ != 0) return rc__; } while (0)
 
+// With the "profile" option on, the vocabulary-projection launches are bracketed by event pairs.
+void prof_mark(specdec_handle* h, cudaStream_t st) {
+    if (!h->profile) return;
+    if (h->prof_n >= h->prof_ev.size()) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) return;
+        h->prof_ev.push_back(e);
+    }
+    cudaEventRecord(h->prof_ev[h->prof_n++], st);
+}
+void prof_collect(specdec_handle* h) {
+    for (size_t i = 0; i + 1 < h->prof_n; i += 2) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, h->prof_ev[i], h->prof_ev[i + 1]) == cudaSuccess) { h->prof_ms += t; ++h->prof_launches; }
+    }
+    h->prof_n = 0;
+}
+
 // One pre-LN block on `rows_ub` rows of the residual stream x (encoder: no cross-attention).
 // Self-attention keys come from the block's own QKV rows (contiguous) or, for the verifier,
 // from the paged cache after the block's K/V were scattered into it.
@@ -447,11 +474,17 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
     TRY(block_ffn<T>(h, m, w, h->x2, CNT_DRAFT_MASK, R2, st));
     TRY(ln<T>(h, h->x2, m.dec_lnf_g, m.dec_lnf_b, CNT_DRAFT_MASK, R2, h->y, d, st));
     int n_tiles = 0;
+    prof_mark(h, st);
     TRY(gemm<T>(h, EPI_STATS, h->y, d, m.embed, nullptr, m.dm.vocab, d, CNT_DRAFT_MASK, R2, nullptr, 0, nullptr, st,
                 nullptr, nullptr, &n_tiles));
+    prof_mark(h, st);
     k_draft_argmax<<<cdiv(R2, 4), 128, 0, st>>>(h->part, n_tiles, h->ses.counters + CNT_DRAFT_MASK, h->mrows.slot,
                                                d_draft);
     KCHECK(h);
+    if (h->script_on) {
+        k_apply_script<<<cdiv(B * k, 256), 256, 0, st>>>(h->ses, h->script, h->T_cap + h->k_cap, B, k, d_draft);
+        KCHECK(h);
+    }
     h->drafted = true; h->verified = false;
     h->last_draft_rows_ub = R2;
     return 0;
@@ -479,8 +512,10 @@ int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float ta
                                                  h->ld, h->ld_id);
     KCHECK(h);
     int n_tiles = 0;
+    prof_mark(h, st);
     TRY(gemm<T>(h, EPI_STATS, h->y, d, m.embed, nullptr, m.dm.vocab, d, CNT_VERIFY, M, nullptr, 0, nullptr, st, h->ld,
                 h->ld_id, &n_tiles));
+    prof_mark(h, st);
     k_accept<<<B, 256, (size_t)(k + 1) * sizeof(RowPart), st>>>(h->part, n_tiles, h->ld, h->ld_id, k, beta, tau,
                                                                 h->accepted, h->bif, h->row_stats);
     KCHECK(h);
@@ -532,6 +567,7 @@ int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, con
     CUDA_TRY(h, cudaMemcpyAsync(h->h_stats + 4, h->ses.counters + 7, 4, cudaMemcpyDeviceToHost, st));
     mark();
     CUDA_TRY(h, cudaStreamSynchronize(st));
+    if (h->profile) prof_collect(h);
     if (*(int*)(h->h_stats + 4) != 0)
         return fail(h, SPECDEC_ERR_TIMEOUT, "a bounded device-side wait gave up (code " + std::to_string(*(int*)(h->h_stats + 4)) + ")");
     if (hs) {
@@ -681,6 +717,7 @@ int specdec_destroy(specdec_handle* h) {
     cudaDeviceSynchronize();
     for (auto& e : h->poll_ev) cudaEventDestroy(e);
     for (auto& e : h->time_ev) cudaEventDestroy(e);
+    for (auto& e : h->prof_ev) cudaEventDestroy(e);
     if (h->h_poll) cudaFreeHost(h->h_poll);
     if (h->h_stats) cudaFreeHost(h->h_stats);
     if (h->arena.base) cudaFree(h->arena.base);
@@ -697,6 +734,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         return SPECDEC_OK;
     }
     if (!strcmp(name, "graphs")) { h->use_graphs = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "profile")) { h->profile = value ? 1 : 0; h->prof_n = 0; h->prof_ms = 0.0; h->prof_launches = 0; return SPECDEC_OK; }
     return fail(h, SPECDEC_ERR_INVALID_ARG, std::string("unknown option: ") + name);
 }
 
@@ -791,6 +829,24 @@ int specdec_generate_host(specdec_handle* h, const int32_t* h_src, const int32_t
                                   B, cudaMemcpyDeviceToHost, st));
     CUDA_TRY(h, cudaMemcpyAsync(h_out_len, h->ses.len, (size_t)B * 4, cudaMemcpyDeviceToHost, st));
     CUDA_TRY(h, cudaStreamSynchronize(st));
+    return SPECDEC_OK;
+}
+
+int specdec_set_draft_script(specdec_handle* h, const int32_t* d_script, int B, int stride, void* stream) {
+    if (!h) return SPECDEC_ERR_INVALID_ARG;
+    if (!d_script) { h->script_on = false; return SPECDEC_OK; }
+    if (B < 1 || B > h->B_cap || stride < 1) return fail(h, SPECDEC_ERR_CAPACITY, "set_draft_script: bad B or stride");
+    const int w = std::min(stride, h->T_cap + h->k_cap);
+    CUDA_TRY(h, cudaMemsetAsync(h->script, 0xff, (size_t)h->B_cap * (h->T_cap + h->k_cap) * 4, (cudaStream_t)stream));
+    CUDA_TRY(h, cudaMemcpy2DAsync(h->script, (size_t)(h->T_cap + h->k_cap) * 4, d_script, (size_t)stride * 4, (size_t)w * 4, B,
+                                  cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    h->script_on = true;
+    return SPECDEC_OK;
+}
+
+int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches) {
+    if (!h || !h_ms || !h_launches) return SPECDEC_ERR_INVALID_ARG;
+    *h_ms = h->prof_ms; *h_launches = h->prof_launches;
     return SPECDEC_OK;
 }
 

@@ -1,0 +1,124 @@
+"""Verify-step microbenchmark (Transformer-base verifier decoder, bf16): times specdec_verify alone.
+
+  python -m paper_2203_16487_b200.microbench --batch 1 --k 25 --prefix 64 [--reps 50] [--no-flush] [--draft]
+
+A session is encoded on sources of 64 Zipf ids, a committed prefix of `prefix`
+tokens is built through verify + commit(keep, next), and the verify step is
+then repeated on a fixed draft block (the verifier's own greedy continuation
+with one substitution at a Geometric(mean 6) position).  Each repetition is
+timed with CUDA events on the launching stream; unless --no-flush is given a
+256 MiB buffer is rewritten between repetitions so the weights come from HBM.
+Prints one JSON line with the median time, the algorithmic bytes / flops of the
+step and the achieved fraction of the measured HBM and bf16 peaks.
+--draft times specdec_draft instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+
+import numpy as np
+import torch
+
+from . import binding, workloads as W
+
+
+def algorithmic_work(B: int, k: int, j: int, S: int, dims: W.ModelDims):
+    """Bytes that must move and flops that must run for one verify step."""
+    d, F, V, L = dims.d_model, dims.d_ffn, dims.vocab, dims.dec_layers
+    per_layer = 3 * d * d + 3 * d + d * d + d + d * d + d + d * d + d + 2 * F * d + F + d + 6 * d   # self qkv/o, cross q/o, ffn, 3 LN
+    params = L * per_layer + V * d + 2 * d
+    M = B * (k + 1)
+    kv_read = B * L * (j + S) * 2 * d * 2
+    kv_new = B * L * (k + 1) * 2 * d * 2 * 2
+    bytes_ = params * 2 + kv_read + kv_new + M * d * 2 + B * 8
+    flops = 2.0 * M * (L * (4 * d * d + 2 * d * d + 2 * F * d) + V * d) + 4.0 * B * L * (k + 1) * d * ((j + k + 1) + S)
+    return params, bytes_, flops
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--k", type=int, default=25)
+    ap.add_argument("--prefix", type=int, default=64)
+    ap.add_argument("--src-len", type=int, default=64)
+    ap.add_argument("--reps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--no-flush", action="store_true")
+    ap.add_argument("--draft", action="store_true")
+    ap.add_argument("--gemm", type=int, default=1)
+    args = ap.parse_args()
+    B, k, j, S = args.batch, args.k, args.prefix, args.src_len
+
+    wl = W.config5_microbench(B, S)
+    wv = W.make_weights(wl.verifier, wl.seed_verifier, True)
+    wd = W.make_weights(wl.drafter, wl.seed_drafter, True)
+    sd = binding.SpecDec(wl.verifier, wv, wl.drafter, wd, k_max=max(k, 1), max_batch=B, max_src=S,
+                         max_tgt=j + k + 2, bf16=True)
+    sd.set_option("gemm", args.gemm)
+    src, lens = W.pad_batch(wl.src)
+    sd.encode(src, lens, None)
+    prefix, rej = W.config5_prefix_and_rejections(B, j)
+    prefix = np.stack(prefix) if j > 0 else np.zeros((B, 0), np.int32)
+    # build the committed prefix: verify a block of prefix tokens, keep c of them plus the next one
+    done = 0
+    while done < j:
+        c = min(k, j - done - 1)
+        block = np.zeros((B, k), np.int32)
+        block[:, :c] = prefix[:, done:done + c]
+        sd.verify(block, 1, 0.0)
+        sd.commit(np.full(B, c, np.int32), prefix[:, done + c])
+        done += c + 1
+    out, n, _ = sd.output()
+    assert int(n.min()) == j and int(n.max()) == j
+    # draft block: the verifier's greedy continuation from that prefix, one substitution per sequence
+    drafts = np.zeros((B, k), np.int32)
+    for i in range(k + 1):        # greedy continuation one token at a time through the same entry points
+        acc, bif = sd.verify(drafts, 1, 0.0)
+        a, t = acc.cpu().numpy(), bif.cpu().numpy()
+        if int(a.min()) >= k:
+            break
+        for b in range(B):
+            if a[b] < k:
+                drafts[b, a[b]] = t[b]
+    for b in range(B):
+        if rej[b] <= k:
+            drafts[b, rej[b] - 1] = (drafts[b, rej[b] - 1] + 17) % wl.verifier.vocab
+    d_drafts = torch.from_numpy(drafts).cuda()
+    acc, _ = sd.verify(d_drafts, 3, 1.0)
+    mean_a = float(acc.float().mean())
+
+    flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    times = []
+    for r in range(args.warmup + args.reps):
+        if flush is not None:
+            flush.fill_(r & 0xff)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        if args.draft:
+            sd.draft(k)
+        else:
+            sd.verify(d_drafts, 3, 1.0)
+        e1.record()
+        torch.cuda.synchronize()
+        if r >= args.warmup:
+            times.append(e0.elapsed_time(e1) * 1e3)
+    us = float(np.median(times))
+    params, bytes_, flops = algorithmic_work(B, k, j, S, wl.verifier)
+    peaks = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    hbm, tc, kind = 6650.0, 1590.0, "fallback"
+    if os.path.exists(peaks):
+        p = json.load(open(peaks)); hbm, tc, kind = p["hbm_gbs"], p["bf16_tflops"], "measured"
+    print(json.dumps({
+        "step": "draft" if args.draft else "verify", "batch": B, "k": k, "prefix": j, "src_len": S,
+        "us_median": us, "us_min": float(np.min(times)), "l2_flush": flush is not None, "mean_accepted": mean_a,
+        "algorithmic_MB": bytes_ / 1e6, "algorithmic_GFLOP": flops / 1e9,
+        "hbm_GBs": bytes_ / us / 1e3, "hbm_frac": bytes_ / us / 1e3 / hbm,
+        "tensor_TFLOPs": flops / us / 1e6, "tensor_frac": flops / us / 1e6 / tc, "peaks": kind,
+    }))
+    sd.close()
+
+
+if __name__ == "__main__":
+    main()

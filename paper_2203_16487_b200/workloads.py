@@ -62,10 +62,10 @@ class Workload:
 def round_to_bf16(a: np.ndarray) -> np.ndarray:
     """Round fp32 values to the nearest bf16 (ties to even), returned as fp32."""
     a = np.ascontiguousarray(a, dtype=np.float32)
-    u = a.view(np.uint32).astype(np.uint64)
-    lsb = (u >> 16) & 1
-    u = (u + 0x7FFF + lsb) & 0xFFFF0000
-    return u.astype(np.uint32).view(np.float32).reshape(a.shape)
+    u = a.view(np.uint32)
+    lsb = (u >> np.uint32(16)) & np.uint32(1)
+    u = (u + np.uint32(0x7FFF) + lsb) & np.uint32(0xFFFF0000)      # finite inputs only: no carry out of bit 31
+    return u.view(np.float32).reshape(a.shape)
 
 
 def sinusoid_table(n_pos: int, d: int) -> np.ndarray:
@@ -102,7 +102,7 @@ def make_weights(dims: ModelDims, seed: int, bf16: bool,
     w: Dict[str, np.ndarray] = {}
 
     def mat(name, shape, std=0.02):
-        a = (rng.standard_normal(shape) * std).astype(np.float32)
+        a = rng.standard_normal(shape, dtype=np.float32) * np.float32(std)
         w[name] = round_to_bf16(a) if (bf16 and a.ndim >= 2) else a
 
     def ln(name):
