@@ -156,6 +156,25 @@ int specdec_get_output(specdec_handle* h, int32_t* d_out, int out_stride, int32_
 int specdec_accept_scan(const float* d_logits, const int32_t* d_draft, int B, int k, int V,
                         int beta, float tau, int32_t* d_accepted, int32_t* d_bif, void* stream);
 
+/* The same acceptance rule for callers that must not allocate device memory -- the paper has no
+ * counterpart; this exists for embedding the rule in programs where the device allocator is off
+ * limits: a serving process whose memory pool already owns all of HBM (so a later cudaMalloc
+ * fails), or a latency-critical loop that cannot afford the device-wide synchronisation an
+ * allocation or free implies.  Inputs and outputs are the caller's, exactly as for
+ * specdec_accept_scan (d_logits [B,k+1,V] fp32, d_draft [B,k]; d_accepted, d_bif [B]); the
+ * intermediate per-row partial statistics live in a fixed array compiled into the library
+ * (about 4.2 MB of device memory on every GPU that loads the library, held until the process
+ * exits).  Limits: B*(k+1) <= 4096 and V <= 65536; beyond them the call returns
+ * SPECDEC_ERR_CAPACITY and launches nothing.  The call makes no cudaMalloc / cudaFree and uses
+ * no allocating library routine.  The first call on each device looks up the array's device
+ * address (cudaGetSymbolAddress, with the caller's current device); make that first call
+ * before starting any stream capture.  All calls share the one array, which keeps whatever
+ * the previous call left in it; every entry a call reads is rewritten by that call first, so
+ * nothing needs clearing, but two calls whose kernels overlap on the GPU (different streams,
+ * or different host threads) race on it: serialise them. */
+int specdec_accept_scan_static(const float* d_logits, const int32_t* d_draft, int B, int k, int V,
+                               int beta, float tau, int32_t* d_accepted, int32_t* d_bif, void* stream);
+
 /* Debug / parity helpers (not on the hot path).
  * specdec_debug_logits: re-runs the vocabulary projection of the last verify
  *   (which = 0, rows [B*(k+1)]) or draft (which = 1, rows [n_active*k]) pass

@@ -24,6 +24,7 @@ EXPORTS = [
     "specdec_commit", "specdec_generate", "specdec_generate_host", "specdec_get_output",
     "specdec_accept_scan", "specdec_debug_logits", "specdec_debug_row_stats", "specdec_set_option",
     "specdec_launch_count", "specdec_last_error", "specdec_set_draft_script", "specdec_profile_read",
+    "specdec_accept_scan_static",
 ]
 
 
@@ -75,6 +76,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.specdec_generate_host.argtypes = [vp, ip, ip, ip, i, i, i, i, f, ip, i, ip, C.POINTER(Stats), vp]
     lib.specdec_get_output.argtypes = [vp, ip, i, ip, ip, vp]
     lib.specdec_accept_scan.argtypes = [vp, ip, i, i, i, i, f, ip, ip, vp]
+    lib.specdec_accept_scan_static.argtypes = [vp, ip, i, i, i, i, f, ip, ip, vp]
     lib.specdec_debug_logits.argtypes = [vp, i, vp, vp]
     lib.specdec_debug_row_stats.argtypes = [vp, vp, vp]
     lib.specdec_set_option.argtypes = [vp, C.c_char_p, i]
@@ -272,6 +274,25 @@ def accept_scan(logits: torch.Tensor, drafts: torch.Tensor, beta: int, tau: floa
     bif = torch.empty(B, dtype=torch.int32, device=logits.device)
     rc = lib().specdec_accept_scan(_ptr(logits), _ptr(drafts), B, k1 - 1, V, beta, float(tau), _ptr(acc), _ptr(bif),
                                    _stream())
+    if rc != 0:
+        raise SpecDecError(rc, lib().specdec_last_error(None).decode())
+    return acc, bif
+
+
+def accept_scan_static(logits: torch.Tensor, drafts: torch.Tensor, beta: int, tau: float,
+                       acc: Optional[torch.Tensor] = None, bif: Optional[torch.Tensor] = None):
+    """specdec_accept_scan_static: the acceptance rule for callers that cannot allocate device memory
+    (the partial statistics sit in an array compiled into the library).  Pass preallocated `acc` and
+    `bif` [B] int32 device tensors to keep the call itself free of any allocation."""
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous()
+    B, k1, V = logits.shape
+    assert drafts.is_cuda and drafts.dtype == torch.int32 and drafts.is_contiguous()
+    if acc is None:
+        acc = torch.empty(B, dtype=torch.int32, device=logits.device)
+    if bif is None:
+        bif = torch.empty(B, dtype=torch.int32, device=logits.device)
+    rc = lib().specdec_accept_scan_static(_ptr(logits), _ptr(drafts), B, k1 - 1, V, beta, float(tau), _ptr(acc),
+                                          _ptr(bif), _stream())
     if rc != 0:
         raise SpecDecError(rc, lib().specdec_last_error(None).decode())
     return acc, bif

@@ -467,6 +467,41 @@ __global__ void k_accept_logits(const float* __restrict__ logits, const int* __r
     }
 }
 
+// Per (row, tile of `tile` columns) statistics of caller-provided logits [rows, V]: the first stage of the
+// two-stage acceptance scan whose partials live in the library's static scratch array.
+__global__ void k_logit_tile_stats(const float* __restrict__ logits, const int* __restrict__ draft, int k, int V,
+                                   int tile, int n_tiles, RowPart* __restrict__ part, float* __restrict__ ld_out,
+                                   int* __restrict__ id_out) {
+    __shared__ RowPart wsm[32];
+    const int row = blockIdx.y, t = blockIdx.x, b = row / (k + 1), c = row % (k + 1);
+    const float* l = logits + (size_t)row * V;
+    const int tok = (c < k) ? draft[b * k + c] : -1;
+    const bool ok = tok >= 0 && tok < V;
+    const float ld = (c == k) ? CUDART_INF_F : (ok ? l[tok] : -CUDART_INF_F);
+    RowPart m; m.mx = -CUDART_INF_F; m.arg = 0x7fffffff; m.sum = 0.f; m.cnt = 0;
+    const int v1 = min(V, (t + 1) * tile);
+    for (int v = t * tile + threadIdx.x; v < v1; v += blockDim.x) {
+        RowPart q; q.mx = l[v]; q.arg = v; q.sum = 1.f; q.cnt = (l[v] > ld) ? 1 : 0;
+        part_merge(m, q);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        RowPart q;
+        q.mx = __shfl_xor_sync(0xffffffffu, m.mx, o);
+        q.arg = __shfl_xor_sync(0xffffffffu, m.arg, o);
+        q.sum = __shfl_xor_sync(0xffffffffu, m.sum, o);
+        q.cnt = __shfl_xor_sync(0xffffffffu, m.cnt, o);
+        part_merge(m, q);
+    }
+    if ((threadIdx.x & 31) == 0) wsm[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < (int)(blockDim.x >> 5); ++w) part_merge(m, wsm[w]);
+        part[(size_t)row * n_tiles + t] = m;
+        if (t == 0) { ld_out[row] = ld; id_out[row] = (c == k) ? -1 : (ok ? tok : -2); }
+    }
+}
+
 // ------------------------------------------------------------------ drafter argmax
 __global__ void k_draft_argmax(const RowPart* __restrict__ part, int n_tiles, const int* __restrict__ n_rows,
                                const int* __restrict__ slot, int* __restrict__ draft) {

@@ -860,6 +860,57 @@ int specdec_accept_scan(const float* d_logits, const int32_t* d_draft, int B, in
     return SPECDEC_OK;
 }
 
+// ---- acceptance scan for callers that must not allocate ---------------------------------------------
+// The per-(row, tile) partial statistics live in a file-scope device array instead of an arena.  In host
+// code `g_static_scratch` is only a stand-in for the symbol: the kernels get the device address that
+// cudaGetSymbolAddress returns, looked up once per device with that device current.
+namespace {
+constexpr int NA_MAX_ROWS = 4096;      // B * (k + 1)
+constexpr int NA_TILE = 1024;          // vocabulary columns per partial
+constexpr int NA_MAX_TILES = 64;       // => V <= 65536
+constexpr size_t NA_PART_BYTES = (size_t)NA_MAX_ROWS * NA_MAX_TILES * sizeof(RowPart);
+constexpr size_t NA_BYTES = NA_PART_BYTES + (size_t)NA_MAX_ROWS * 8;
+static __device__ __align__(256) unsigned char g_static_scratch[NA_BYTES];
+constexpr int NA_MAX_DEVICES = 64;
+void* g_static_scratch_addr[NA_MAX_DEVICES] = {nullptr};
+}  // namespace
+
+int specdec_accept_scan_static(const float* d_logits, const int32_t* d_draft, int B, int k, int V, int beta, float tau,
+                               int32_t* d_accepted, int32_t* d_bif, void* stream) {
+    if (!d_logits || !d_draft || !d_accepted || !d_bif || B < 1 || k < 1 || V < 1 || beta < 1 || !(tau >= 0.f))
+        return fail(nullptr, SPECDEC_ERR_INVALID_ARG, "accept_scan_static: bad argument");
+    const long long rows = (long long)B * (k + 1);
+    const int n_tiles = (V + NA_TILE - 1) / NA_TILE;
+    if (rows > NA_MAX_ROWS || n_tiles > NA_MAX_TILES)
+        return fail(nullptr, SPECDEC_ERR_CAPACITY,
+                    "accept_scan_static: B*(k+1) = " + std::to_string(rows) + " (limit " + std::to_string(NA_MAX_ROWS) +
+                    ") or V = " + std::to_string(V) + " (limit " + std::to_string(NA_MAX_TILES * NA_TILE) +
+                    ") exceeds the static scratch; use specdec_accept_scan");
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= NA_MAX_DEVICES)
+        return fail(nullptr, SPECDEC_ERR_CUDA, std::string("accept_scan_static: cudaGetDevice: ") + cudaGetErrorString(e));
+    if (!g_static_scratch_addr[dev]) {          // first call on this device: resolve the symbol's device address
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess || !p)
+            return fail(nullptr, SPECDEC_ERR_CUDA, std::string("accept_scan_static: cudaGetSymbolAddress: ") + cudaGetErrorString(e));
+        g_static_scratch_addr[dev] = p;
+    }
+    unsigned char* base = (unsigned char*)g_static_scratch_addr[dev];
+    RowPart* part = (RowPart*)base;
+    float* ld = (float*)(base + NA_PART_BYTES);
+    int* ld_id = (int*)(base + NA_PART_BYTES + (size_t)NA_MAX_ROWS * 4);
+    cudaStream_t st = (cudaStream_t)stream;
+    // every slot the second stage reads is rewritten by the first, so nothing has to start at zero
+    k_logit_tile_stats<<<dim3(n_tiles, (unsigned)rows), 256, 0, st>>>(d_logits, d_draft, k, V, NA_TILE, n_tiles, part, ld, ld_id);
+    k_accept<<<B, 256, (size_t)(k + 1) * sizeof(RowPart), st>>>(part, n_tiles, ld, ld_id, k, beta, tau, d_accepted, d_bif,
+                                                                nullptr);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(nullptr, SPECDEC_ERR_CUDA, std::string("accept_scan_static: ") + cudaGetErrorString(e));
+    return SPECDEC_OK;
+}
+
 int specdec_debug_logits(specdec_handle* h, int which, float* d_logits, void* stream) {
     if (!h || !d_logits) return SPECDEC_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
