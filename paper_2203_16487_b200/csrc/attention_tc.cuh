@@ -1,0 +1,208 @@
+// Tile attention for bf16 operands and head size 64: one CTA per (32-query tile, head, sequence).
+//
+//   K and V of every visible key are staged once in shared memory (16-byte cp.async, 128-byte rows,
+//   XOR-swizzled chunks), S = Q K^T runs on the tensor cores (mma.sync m16n8k16, fp32 accumulate),
+//   the softmax is single pass with the true row maximum, the un-normalised probabilities are
+//   rounded to bf16 for P V (second tensor-core contraction) and the result is divided by the fp32
+//   sum of the unrounded exponentials -- the same arithmetic as the reference attention kernel.
+//
+// Used for the verifier's causal attention over the paged cache, both cross-attentions, the
+// drafter's bidirectional attention and the encoders.  Work per CTA is 2 * 32 * keys * 64 * 2 flops:
+// far too little to fill a 128-row tcgen05 tile, which is why this contraction uses warp-level MMA.
+#pragma once
+#include "kernels.cuh"
+
+namespace sd {
+
+struct AttnTcArgs {
+    const bf16* q; int q_stride; const int* q_index;     // query row r reads q + (q_index ? q_index[r] : r) * q_stride
+    const bf16* k; const bf16* v; int kv_stride;         // contiguous: key t of sequence b at row kv_off[b] + t
+    const int* kv_off;
+    Paged pg;                                             // paged: row pg.row(b, t)
+    const int* q_off; const int* q_cnt;                   // per sequence: first query row, number of query rows
+    const int* nkeys;                                     // per query row: visible keys (0..nkeys-1)
+    bf16* out; int out_stride;
+    int max_keys;                                         // capacity the shared memory was sized for
+    float scale;
+};
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+// byte offset of 16-byte chunk c (0..7) of row r in a tile of 128-byte rows
+__device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
+
+constexpr int ATT_Q = 32;
+inline size_t attn_tc_smem(int max_keys) {
+    const int nkp = (max_keys + 15) & ~15;
+    return (size_t)ATT_Q * 128 + (size_t)nkp * 256 + (size_t)ATT_Q * (nkp + 4) * 4 + 16;
+}
+
+template <bool PAGED>
+__global__ void __launch_bounds__(128) k_attn_tc(AttnTcArgs a) {
+    extern __shared__ __align__(128) unsigned char sm[];
+    __shared__ int s_nk[ATT_Q];
+    __shared__ float s_sum[ATT_Q];
+    __shared__ int s_nkmax;
+    const int b = blockIdx.z, h = blockIdx.y, qt = blockIdx.x;
+    const int cnt = a.q_cnt[b];
+    if (qt * ATT_Q >= cnt) return;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int r0 = a.q_off[b] + qt * ATT_Q, nq = min(ATT_Q, cnt - qt * ATT_Q);
+
+    if (tid < 32) {
+        int nk = (tid < nq) ? min(a.nkeys[r0 + tid], a.max_keys) : 0;
+        s_nk[tid] = nk;
+        int m = nk;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (tid == 0) s_nkmax = m;
+    }
+    __syncthreads();
+    const int nkmax = s_nkmax;
+    const int nkp = max((nkmax + 15) & ~15, 16);
+    const uint32_t Qs = (uint32_t)__cvta_generic_to_shared(sm), Ks = Qs + ATT_Q * 128, Vs = Ks + nkp * 128;
+    unsigned char* Qp = sm;
+    unsigned char* Kp = sm + ATT_Q * 128;
+    unsigned char* Vp = Kp + nkp * 128;
+    float* Ss = reinterpret_cast<float*>(Vp + nkp * 128);
+    const int sstr = nkp + 4;                    // fp32 row pitch of S
+    const int pstr = nkp + 8;                    // bf16 row pitch of P (lives where K was)
+
+    // ---- stage Q, K, V
+    for (int i = tid; i < ATT_Q * 8; i += 128) {
+        const int r = i >> 3, c = i & 7;
+        if (r < nq) {
+            const size_t qr = a.q_index ? (size_t)a.q_index[r0 + r] : (size_t)(r0 + r);
+            cp_async16(Qs + swz(r, c), a.q + qr * a.q_stride + h * 64 + c * 8);
+        } else {
+            *reinterpret_cast<uint4*>(Qp + swz(r, c)) = make_uint4(0, 0, 0, 0);
+        }
+    }
+    for (int i = tid; i < nkp * 8; i += 128) {
+        const int t = i >> 3, c = i & 7;
+        if (t < nkmax) {
+            const size_t kr = PAGED ? a.pg.row(b, t) : (size_t)(a.kv_off[b] + t);
+            cp_async16(Ks + swz(t, c), a.k + kr * a.kv_stride + h * 64 + c * 8);
+            cp_async16(Vs + swz(t, c), a.v + kr * a.kv_stride + h * 64 + c * 8);
+        } else {
+            *reinterpret_cast<uint4*>(Kp + swz(t, c)) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4*>(Vp + swz(t, c)) = make_uint4(0, 0, 0, 0);
+        }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+
+    const int g = lane >> 2, t4 = lane & 3;
+    // ---- S = scale * Q K^T, masked
+    {
+        uint32_t qf[2][4][4];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                const int r = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = ks * 2 + (lane >> 4);
+                ldsm_x4(Qs + swz(r, c), qf[mt][ks][0], qf[mt][ks][1], qf[mt][ks][2], qf[mt][ks][3]);
+            }
+        for (int nt = warp; nt < nkp / 8; nt += 4) {
+            uint32_t kf[2][4];
+#pragma unroll
+            for (int kk = 0; kk < 2; ++kk) {
+                const int r = nt * 8 + (lane & 7), c = kk * 4 + (lane >> 3);
+                ldsm_x4(Ks + swz(r, c), kf[kk][0], kf[kk][1], kf[kk][2], kf[kk][3]);
+            }
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) {
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) mma_bf16(acc, qf[mt][ks], kf[ks >> 1][(ks & 1) * 2], kf[ks >> 1][(ks & 1) * 2 + 1]);
+                const int ra = mt * 16 + g, rb = ra + 8, col = nt * 8 + t4 * 2;
+                const int na = s_nk[ra], nb = s_nk[rb];
+                Ss[ra * sstr + col] = (col < na) ? acc[0] * a.scale : -CUDART_INF_F;
+                Ss[ra * sstr + col + 1] = (col + 1 < na) ? acc[1] * a.scale : -CUDART_INF_F;
+                Ss[rb * sstr + col] = (col < nb) ? acc[2] * a.scale : -CUDART_INF_F;
+                Ss[rb * sstr + col + 1] = (col + 1 < nb) ? acc[3] * a.scale : -CUDART_INF_F;
+            }
+        }
+    }
+    __syncthreads();
+    // ---- softmax: 4 threads per row; P (bf16, un-normalised) overwrites the K tile
+    {
+        bf16* P = reinterpret_cast<bf16*>(Kp);
+        const int r = tid >> 2, sub = tid & 3;
+        const float* srow = Ss + r * sstr;
+        float m = -CUDART_INF_F;
+        for (int c = sub; c < nkp; c += 4) m = fmaxf(m, srow[c]);
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+        float sum = 0.f;
+        for (int c = sub; c < nkp; c += 4) {
+            const float s = srow[c];
+            const float e = (s == -CUDART_INF_F) ? 0.f : expf(s - m);
+            sum += e;
+            P[r * pstr + c] = __float2bfloat16_rn(e);
+        }
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        if (sub == 0) s_sum[r] = sum;
+    }
+    __syncthreads();
+    // ---- O = P V ; warp w owns head columns 16w .. 16w+15
+    {
+        float acc[2][2][4];
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
+        for (int kt = 0; kt < nkp / 16; ++kt) {
+            uint32_t vf[4];
+            {
+                const int r = kt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = warp * 2 + (lane >> 4);
+                ldsm_x4_t(Vs + swz(r, c), vf[0], vf[1], vf[2], vf[3]);
+            }
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) {
+                uint32_t pf[4];
+                const int r = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = kt * 16 + (lane >> 4) * 8;
+                ldsm_x4(Ks + (uint32_t)(r * pstr + c) * 2, pf[0], pf[1], pf[2], pf[3]);
+                mma_bf16(acc[mt][0], pf, vf[0], vf[1]);
+                mma_bf16(acc[mt][1], pf, vf[2], vf[3]);
+            }
+        }
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int r = mt * 16 + g + half * 8;
+                if (r < nq) {
+                    const float den = s_sum[r];
+                    bf16* o = a.out + (size_t)(r0 + r) * a.out_stride + h * 64 + warp * 16 + t4 * 2;
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt) {
+                        __nv_bfloat162 v2;
+                        v2.x = __float2bfloat16_rn(den > 0.f ? acc[mt][nt][half * 2] / den : 0.f);
+                        v2.y = __float2bfloat16_rn(den > 0.f ? acc[mt][nt][half * 2 + 1] / den : 0.f);
+                        *reinterpret_cast<__nv_bfloat162*>(o + nt * 8) = v2;
+                    }
+                }
+            }
+    }
+}
+
+}  // namespace sd

@@ -57,6 +57,8 @@ struct Rows {
     int* kv_off_cross;  // [B]
     int* src_row;   // mask-only pass: the row of the full pass this row continues
     int* slot;      // mask-only pass: index into the [B,k] draft array
+    int* q_off;     // [B] first row of the sequence in this pass
+    int* q_cnt;     // [B] rows of the sequence in this pass (0: none)
 };
 
 // ------------------------------------------------------------------ row preparation
@@ -65,7 +67,7 @@ __global__ void k_enc_prep(const int* __restrict__ src, const int* __restrict__ 
                            Rows r, int* counters) {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i == 0) counters[CNT_ENC] = B * S_max;
-    if (i < B) { r.kv_off[i] = i * S_max; r.kv_off_cross[i] = i * S_max; }
+    if (i < B) { r.kv_off[i] = i * S_max; r.kv_off_cross[i] = i * S_max; r.q_off[i] = i * S_max; r.q_cnt[i] = src_len[i]; }
     if (i >= B * S_max) return;
     int b = i / S_max, t = i % S_max;
     r.tok[i] = src[i];
@@ -80,7 +82,7 @@ __global__ void k_verify_prep(Session s, const int* __restrict__ draft, int B, i
                               Rows r) {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i == 0) s.counters[CNT_VERIFY] = B * (k + 1);
-    if (i < B) r.kv_off_cross[i] = i * S_max;
+    if (i < B) { r.kv_off_cross[i] = i * S_max; r.q_off[i] = i * (k + 1); r.q_cnt[i] = k + 1; }
     if (i >= B * (k + 1)) return;
     int b = i / (k + 1), c = i % (k + 1);
     int j = s.len[b];
@@ -110,7 +112,9 @@ __global__ void k_draft_prep(Session s, int B, int k, int S_max, int bos, int ma
     __syncthreads();
     for (int b = 0; b < B; ++b) {
         if (threadIdx.x == 0) { all.kv_off[b] = off[b]; all.kv_off_cross[b] = b * S_max;
-                                msk.kv_off[b] = off[b]; msk.kv_off_cross[b] = b * S_max; }
+                                msk.kv_off[b] = off[b]; msk.kv_off_cross[b] = b * S_max;
+                                all.q_off[b] = off[b]; all.q_cnt[b] = off[b + 1] - off[b];
+                                msk.q_off[b] = moff[b]; msk.q_cnt[b] = moff[b + 1] - moff[b]; }
         if (s.finished[b]) continue;
         int j = s.len[b], n = j + 1 + k, sl = s.src_len[b];
         for (int t = threadIdx.x; t < n; t += blockDim.x) {

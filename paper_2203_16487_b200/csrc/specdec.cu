@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "../../include/specdec.h"
+#include "attention_tc.cuh"
 #include "gemm_tc.cuh"
 #include "kernels.cuh"
 
@@ -77,7 +78,8 @@ struct specdec_handle {
     bool encoded = false, verified = false, drafted = false;
     int last_draft_rows_ub = 0;
     // options
-    int use_tc = 1, use_graphs = 0;
+    int use_tc = 1, use_graphs = 0, use_tc_attn = 1;
+    size_t attn_tc_smem_cap = 0;
     long long launches = 0;
     // polling
     int* h_poll = nullptr;          // pinned
@@ -155,7 +157,7 @@ void layout_rows(Arena& A, Rows& r, int n, int B) {
     auto iv = [&](size_t c) { return (int*)A.take(c * 4); };
     r.tok = iv(n); r.pos = iv(n); r.seq = iv(n); r.nk_self = iv(n); r.nk_cross = iv(n);
     r.src_row = iv(n); r.slot = iv(n);
-    r.kv_off = iv(B); r.kv_off_cross = iv(B);
+    r.kv_off = iv(B); r.kv_off_cross = iv(B); r.q_off = iv(B); r.q_cnt = iv(B);
 }
 
 void layout_all(specdec_handle* h) {
@@ -309,16 +311,36 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
     return 0;
 }
 
+// Attention of the pass described by `r`.  bf16 handles with 64-wide heads use the tensor-core tile
+// kernel (one CTA per 32-query tile, head, sequence; q_ub bounds the queries of one sequence);
+// everything else uses the warp-per-(row, head) kernel.
 template <typename T>
 int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* q_index, const void* k, const void* v,
-         int kv_stride, const int* kv_off, const int* seq, const int* nkeys, int cnt, int rows_ub, void* out,
+         int kv_stride, const int* kv_off, const Rows& r, const int* nkeys, int cnt, int rows_ub, int q_ub, void* out,
          int out_stride, int n_heads, int d_head, int max_keys, cudaStream_t st) {
     if (rows_ub <= 0) return 0;
+    if constexpr (std::is_same<T, bf16>::value) {
+        const size_t smem = attn_tc_smem(max_keys);
+        if (h->use_tc_attn && d_head == 64 && smem <= h->attn_tc_smem_cap) {
+            AttnTcArgs a;
+            a.q = (const bf16*)q; a.q_stride = q_stride; a.q_index = q_index;
+            a.k = (const bf16*)k; a.v = (const bf16*)v; a.kv_stride = kv_stride; a.kv_off = kv_off;
+            a.pg.table = h->page_table; a.pg.page_tokens = h->cfg.page_tokens; a.pg.max_pages = h->pages_per_seq;
+            a.q_off = r.q_off; a.q_cnt = r.q_cnt; a.nkeys = nkeys;
+            a.out = (bf16*)out; a.out_stride = out_stride; a.max_keys = max_keys;
+            a.scale = 1.0f / sqrtf((float)d_head);
+            dim3 grid(cdiv(q_ub, ATT_Q), n_heads, h->B);
+            if (paged) k_attn_tc<true><<<grid, 128, smem, st>>>(a);
+            else k_attn_tc<false><<<grid, 128, smem, st>>>(a);
+            KCHECK(h);
+            return 0;
+        }
+    }
     AttnArgs<T> a;
     a.q = (const T*)q; a.q_stride = q_stride; a.q_index = q_index;
     a.k = (const T*)k; a.v = (const T*)v; a.kv_stride = kv_stride; a.kv_off = kv_off;
     a.pg.table = h->page_table; a.pg.page_tokens = h->cfg.page_tokens; a.pg.max_pages = h->pages_per_seq;
-    a.seq = seq; a.nkeys = nkeys; a.n_rows = h->ses.counters + cnt;
+    a.seq = r.seq; a.nkeys = nkeys; a.n_rows = h->ses.counters + cnt;
     a.out = (T*)out; a.out_stride = out_stride;
     a.n_heads = n_heads; a.d_head = d_head; a.max_keys = max_keys;
     a.scale = 1.0f / sqrtf((float)d_head);
@@ -357,7 +379,7 @@ void prof_collect(specdec_handle* h) {
 // from the paged cache after the block's K/V were scattered into it.
 template <typename T>
 int block_self(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, const Rows& r, int cnt, int rows_ub,
-               int layer, bool verify, int max_keys, cudaStream_t st) {
+               int q_ub, int layer, bool verify, int max_keys, cudaStream_t st) {
     const int d = m.dm.d_model, H = m.dm.n_heads, dh = d / H;
     const size_t e = h->esz;
     TRY(ln<T>(h, x, w.ln1_g, w.ln1_b, cnt, rows_ub, h->y, d, st));
@@ -367,11 +389,11 @@ int block_self(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, co
         k_kv_scatter<T><<<rows_ub, 128, 0, st>>>((const T*)h->qkv, r.seq, r.pos, h->ses.counters + cnt, pg,
                                                  (T*)h->kc[layer], (T*)h->vc[layer], d);
         KCHECK(h);
-        TRY(attn<T>(h, true, h->qkv, 3 * d, nullptr, h->kc[layer], h->vc[layer], d, nullptr, r.seq, r.nk_self, cnt,
-                    rows_ub, h->att, d, H, dh, max_keys, st));
+        TRY(attn<T>(h, true, h->qkv, 3 * d, nullptr, h->kc[layer], h->vc[layer], d, nullptr, r, r.nk_self, cnt,
+                    rows_ub, q_ub, h->att, d, H, dh, max_keys, st));
     } else {
         TRY(attn<T>(h, false, h->qkv, 3 * d, nullptr, (char*)h->qkv + (size_t)d * e, (char*)h->qkv + (size_t)2 * d * e,
-                    3 * d, r.kv_off, r.seq, r.nk_self, cnt, rows_ub, h->att, d, H, dh, max_keys, st));
+                    3 * d, r.kv_off, r, r.nk_self, cnt, rows_ub, q_ub, h->att, d, H, dh, max_keys, st));
     }
     TRY(gemm<T>(h, EPI_RESID, h->att, d, w.o_w, w.o_b, d, d, cnt, rows_ub, nullptr, 0, x, st));
     return 0;
@@ -379,13 +401,13 @@ int block_self(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, co
 
 template <typename T>
 int block_cross(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, const Rows& r, int cnt, int rows_ub,
-                int layer, cudaStream_t st) {
+                int q_ub, int layer, cudaStream_t st) {
     const int d = m.dm.d_model, H = m.dm.n_heads, dh = d / H;
     const size_t e = h->esz;
     TRY(ln<T>(h, x, w.lnc_g, w.lnc_b, cnt, rows_ub, h->y, d, st));
     TRY(gemm<T>(h, EPI_STORE, h->y, d, w.cq_w, w.cq_b, d, d, cnt, rows_ub, h->q, d, nullptr, st));
     TRY(attn<T>(h, false, h->q, d, nullptr, m.ckv[layer], (char*)m.ckv[layer] + (size_t)d * e, 2 * d, r.kv_off_cross,
-                r.seq, r.nk_cross, cnt, rows_ub, h->att, d, H, dh, h->S_max, st));
+                r, r.nk_cross, cnt, rows_ub, q_ub, h->att, d, H, dh, h->S_max, st));
     TRY(gemm<T>(h, EPI_RESID, h->att, d, w.co_w, w.co_b, d, d, cnt, rows_ub, nullptr, 0, x, st));
     return 0;
 }
@@ -418,7 +440,7 @@ int encode_model(specdec_handle* h, ModelW& m, const int* d_src, cudaStream_t st
     KCHECK(h);
     TRY(embed<T>(h, m, h->rows, m.pos_enc, CNT_ENC, R, st));
     for (int l = 0; l < m.dm.enc_layers; ++l) {
-        TRY(block_self<T>(h, m, m.enc[l], h->x, h->rows, CNT_ENC, R, l, false, h->S_max, st));
+        TRY(block_self<T>(h, m, m.enc[l], h->x, h->rows, CNT_ENC, R, h->S_max, l, false, h->S_max, st));
         TRY(block_ffn<T>(h, m, m.enc[l], h->x, CNT_ENC, R, st));
     }
     TRY(ln<T>(h, h->x, m.enc_lnf_g, m.enc_lnf_b, CNT_ENC, R, h->mem, d, st));
@@ -456,8 +478,8 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
     KCHECK(h);
     TRY(embed<T>(h, m, h->rows, m.pos_dec, CNT_DRAFT_ALL, R1, st));
     for (int l = 0; l + 1 < L; ++l) {
-        TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_DRAFT_ALL, R1, l, false, max_keys, st));
-        TRY(block_cross<T>(h, m, m.dec[l], h->x, h->rows, CNT_DRAFT_ALL, R1, l, st));
+        TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_DRAFT_ALL, R1, max_keys, l, false, max_keys, st));
+        TRY(block_cross<T>(h, m, m.dec[l], h->x, h->rows, CNT_DRAFT_ALL, R1, max_keys, l, st));
         TRY(block_ffn<T>(h, m, m.dec[l], h->x, CNT_DRAFT_ALL, R1, st));
     }
     // last layer: K/V from every row, queries and everything after them from the k mask rows only
@@ -467,10 +489,10 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
     k_gather_rows<<<R2, 128, 0, st>>>(h->x, h->mrows.src_row, h->ses.counters + CNT_DRAFT_MASK, h->x2, d);
     KCHECK(h);
     TRY(attn<T>(h, false, h->qkv, 3 * d, h->mrows.src_row, (char*)h->qkv + (size_t)d * e,
-                (char*)h->qkv + (size_t)2 * d * e, 3 * d, h->mrows.kv_off, h->mrows.seq, h->mrows.nk_self,
-                CNT_DRAFT_MASK, R2, h->att, d, H, dh, max_keys, st));
+                (char*)h->qkv + (size_t)2 * d * e, 3 * d, h->mrows.kv_off, h->mrows, h->mrows.nk_self,
+                CNT_DRAFT_MASK, R2, k, h->att, d, H, dh, max_keys, st));
     TRY(gemm<T>(h, EPI_RESID, h->att, d, w.o_w, w.o_b, d, d, CNT_DRAFT_MASK, R2, nullptr, 0, h->x2, st));
-    TRY(block_cross<T>(h, m, w, h->x2, h->mrows, CNT_DRAFT_MASK, R2, L - 1, st));
+    TRY(block_cross<T>(h, m, w, h->x2, h->mrows, CNT_DRAFT_MASK, R2, k, L - 1, st));
     TRY(block_ffn<T>(h, m, w, h->x2, CNT_DRAFT_MASK, R2, st));
     TRY(ln<T>(h, h->x2, m.dec_lnf_g, m.dec_lnf_b, CNT_DRAFT_MASK, R2, h->y, d, st));
     int n_tiles = 0;
@@ -503,8 +525,8 @@ int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float ta
     KCHECK(h);
     TRY(embed<T>(h, m, h->rows, m.pos_dec, CNT_VERIFY, M, st));
     for (int l = 0; l < L; ++l) {
-        TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, l, true, max_keys, st));
-        TRY(block_cross<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, l, st));
+        TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, k + 1, l, true, max_keys, st));
+        TRY(block_cross<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, k + 1, l, st));
         TRY(block_ffn<T>(h, m, m.dec[l], h->x, CNT_VERIFY, M, st));
     }
     TRY(ln<T>(h, h->x, m.dec_lnf_g, m.dec_lnf_b, CNT_VERIFY, M, h->y, d, st));
@@ -703,6 +725,13 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
         }
     }
     if (h->dtype == SPECDEC_DTYPE_BF16) {
+        const int max_keys = std::max(h->S_cap, h->T_cap + h->k_cap + 1);
+        h->attn_tc_smem_cap = std::min<size_t>(attn_tc_smem(max_keys), 227 * 1024);
+        if (cudaFuncSetAttribute(k_attn_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess) {
+            cudaGetLastError();
+            h->attn_tc_smem_cap = 48 * 1024;
+        }
         if (sd::tc_init(h->tma, h->ses.counters + 7) != 0) h->use_tc = 0;     // reported through specdec_last_error; SIMT GEMM still runs on the GPU
         if (!h->use_tc) h->err = "tensor-core GEMM unavailable: " + h->tma.err;
     } else {
@@ -733,6 +762,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         h->use_tc = value ? 1 : 0;
         return SPECDEC_OK;
     }
+    if (!strcmp(name, "attn")) { h->use_tc_attn = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "graphs")) { h->use_graphs = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "profile")) { h->profile = value ? 1 : 0; h->prof_n = 0; h->prof_ms = 0.0; h->prof_launches = 0; return SPECDEC_OK; }
     return fail(h, SPECDEC_ERR_INVALID_ARG, std::string("unknown option: ") + name);

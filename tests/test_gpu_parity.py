@@ -227,8 +227,8 @@ MID_V = W.ModelDims(128, 2, 512, 2000, 2, 2, 128)
 MID_D = W.ModelDims(128, 2, 512, 2000, 3, 2, 128)
 
 
-@pytest.mark.parametrize("gemm", [0, 1])
-def test_bf16_mid_lockstep(gemm):
+@pytest.mark.parametrize("gemm,attn", [(0, 0), (1, 0), (0, 1), (1, 1)])
+def test_bf16_mid_lockstep(gemm, attn):
     wv, wd = W.make_weights(MID_V, 21, True), W.make_weights(MID_D, 22, True)
     mv, md = O.model_from(MID_V, wv, mode="bf16"), O.model_from(MID_D, wd, mode="bf16")
     rng = np.random.default_rng(6)
@@ -236,6 +236,7 @@ def test_bf16_mid_lockstep(gemm):
     sd = _handle(MID_V, wv, MID_D, wd, True, k_max=12, max_batch=8, max_src=40, max_tgt=40)
     try:
         sd.set_option("gemm", gemm)
+        sd.set_option("attn", attn)
     except Exception as e:
         pytest.skip(f"tensor-core GEMM not available: {e}")
     rep = lockstep.run(sd, mv, md, srcs, [30, 18, 40, 5, 33], 12, 3, 1.0, margin=1e-3, check_logits_every=2,
