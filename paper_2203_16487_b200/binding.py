@@ -150,6 +150,7 @@ class SpecDec:
         self._h = h
         del keep
         self.B = 0
+        self._bufs = {}
 
     # ------------------------------------------------------------------ helpers
     def _check(self, rc):
@@ -202,16 +203,30 @@ class SpecDec:
         self.B, S = int(src.shape[0]), int(src.shape[1])
         self._check(self._lib.specdec_encode(self._h, _ptr(src), _ptr(src_len), _ptr(mt), self.B, S, _stream()))
 
+    def _buf(self, name, shape):
+        """Persistent device buffers: stable addresses let the library replay its CUDA graphs."""
+        key = (name,) + tuple(shape)
+        if key not in self._bufs:
+            self._bufs[key] = torch.zeros(shape, dtype=torch.int32, device=self.device)
+        return self._bufs[key]
+
     def draft(self, k: int) -> torch.Tensor:
-        out = torch.full((self.B, k), -1, dtype=torch.int32, device=self.device)
+        """Drafts [B,k]; the returned tensor is reused by the next call of the same shape."""
+        out = self._buf("draft", (self.B, k))
+        out.fill_(-1)
         self._check(self._lib.specdec_draft(self._h, k, _ptr(out), _stream()))
         return out
 
     def verify(self, drafts, beta: int, tau: float):
-        drafts = self._i32(drafts)
+        """(accepted [B], bifurcation token [B]); the returned tensors are reused by the next call."""
         k = int(drafts.shape[1])
-        acc = torch.empty(self.B, dtype=torch.int32, device=self.device)
-        bif = torch.empty(self.B, dtype=torch.int32, device=self.device)
+        buf = self._buf("vdraft", (self.B, k))
+        buf.copy_(self._i32(drafts))
+        return self.verify_raw(buf, beta, tau, self._buf("acc", (self.B,)), self._buf("bif", (self.B,)))
+
+    def verify_raw(self, drafts: torch.Tensor, beta: int, tau: float, acc: torch.Tensor, bif: torch.Tensor):
+        """No staging: `drafts` [B,k], `acc`, `bif` [B] are int32 device tensors owned by the caller."""
+        k = int(drafts.shape[1])
         self._check(self._lib.specdec_verify(self._h, _ptr(drafts), k, beta, float(tau), _ptr(acc), _ptr(bif), _stream()))
         return acc, bif
 

@@ -7,6 +7,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <map>
 #include <string>
 #include <type_traits>
 #include <unordered_map>
@@ -78,7 +79,10 @@ struct specdec_handle {
     bool encoded = false, verified = false, drafted = false;
     int last_draft_rows_ub = 0;
     // options
-    int use_tc = 1, use_graphs = 0, use_tc_attn = 1;
+    int use_tc = 1, use_graphs = 1, use_tc_attn = 1;
+    // CUDA graphs of whole draft / verify(+commit) steps, keyed by everything their launches depend on
+    struct GraphEntry { cudaGraphExec_t exec; long long kernels; };
+    std::map<std::vector<long long>, GraphEntry> graphs;
     size_t attn_tc_smem_cap = 0;
     long long launches = 0;
     // polling
@@ -87,6 +91,10 @@ struct specdec_handle {
     std::vector<cudaEvent_t> poll_ev;
     std::vector<cudaEvent_t> time_ev;
     sd::TmaEncoder tma;
+    // work submitted on the legacy default stream (which cannot be captured into a graph) is run on this
+    // stream instead, fenced by events at both ends of the call
+    cudaStream_t own_stream = nullptr;
+    cudaEvent_t fence_in = nullptr, fence_out = nullptr;
     // scripted drafts (benchmark / test hook) and dominant-kernel timing
     int* script = nullptr;          // device [B_cap, T_cap + k_cap] or unset
     bool script_on = false;
@@ -557,6 +565,61 @@ int commit_impl(specdec_handle* h, const int* d_keep, const int* d_next, cudaStr
     return 0;
 }
 
+// Stream a call really runs on: the caller's, or the handle's own when the caller gave a default stream.
+struct StreamScope {
+    specdec_handle* h; cudaStream_t user, st; bool redirected;
+    StreamScope(specdec_handle* h_, void* stream) : h(h_), user((cudaStream_t)stream), st((cudaStream_t)stream), redirected(false) {
+        if ((user == nullptr || user == cudaStreamLegacy || user == cudaStreamPerThread) && h->own_stream) {
+            cudaEventRecord(h->fence_in, user);
+            cudaStreamWaitEvent(h->own_stream, h->fence_in, 0);
+            st = h->own_stream;
+            redirected = true;
+        }
+    }
+    ~StreamScope() {
+        if (redirected) {
+            cudaEventRecord(h->fence_out, st);
+            cudaStreamWaitEvent(user, h->fence_out, 0);
+        }
+    }
+};
+
+void drop_graphs(specdec_handle* h) {
+    for (auto& g : h->graphs) cudaGraphExecDestroy(g.second.exec);
+    h->graphs.clear();
+}
+
+// Runs `body` (a sequence of launches on `st`) through a cached CUDA graph: captured on first use,
+// replayed afterwards.  The key must name everything the launches depend on besides device memory.
+template <typename F>
+int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body) {
+    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->script_on ? 1 : 0);
+    key.push_back(h->B); key.push_back(h->S_max);
+    auto it = h->graphs.find(key);
+    if (it == h->graphs.end()) {
+        const long long before = h->launches;
+        CUDA_TRY(h, cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+        int rc = body();
+        cudaGraph_t g = nullptr;
+        cudaError_t e = cudaStreamEndCapture(st, &g);
+        if (rc != 0) { if (g) cudaGraphDestroy(g); return rc; }
+        if (e != cudaSuccess || !g) return fail(h, SPECDEC_ERR_CUDA, std::string("graph capture: ") + cudaGetErrorString(e));
+        cudaGraphExec_t ex = nullptr;
+        e = cudaGraphInstantiate(&ex, g, 0);
+        cudaGraphDestroy(g);
+        if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("graph instantiate: ") + cudaGetErrorString(e));
+        if (h->graphs.size() > 256) drop_graphs(h);
+        specdec_handle::GraphEntry ge{ex, h->launches - before};
+        h->launches = before;
+        it = h->graphs.emplace(std::move(key), ge).first;
+    }
+    CUDA_TRY(h, cudaGraphLaunch(it->second.exec, st));
+    h->launches += it->second.kernels;
+    return 0;
+}
+
+inline int len_bucket(const specdec_handle* h, int len_ub) { return std::min(h->T_cap, (len_ub + 31) / 32 * 32); }
+
 template <typename T>
 int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, const int* d_max_tgt, int B, int S_max,
                   int k, int beta, float tau, int* d_out, int out_stride, int* d_out_len, specdec_stats* hs,
@@ -570,12 +633,30 @@ int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, con
     const int max_iters = h->T_cap;            // every iteration commits >= 1 token per unfinished sequence
     const int lag = 2, slots = (int)h->poll_ev.size();
     int it = 0;
+    const bool graphs = h->use_graphs && !h->profile;
+    int tau_bits; memcpy(&tau_bits, &tau, 4);
     for (; it < max_iters; ++it) {
-        TRY(draft_impl<T>(h, k, h->g_draft, st));
-        mark();
-        TRY(verify_impl<T>(h, h->g_draft, k, beta, tau, nullptr, nullptr, st));
-        mark();
-        TRY(commit_impl(h, nullptr, nullptr, st));
+        if (graphs) {
+            // the launches depend on the host-side length bound only through its 32-token bucket
+            const int true_ub = h->len_ub, lb = len_bucket(h, true_ub);
+            h->len_ub = lb;
+            TRY(graph_call(h, {1, k, lb}, st, [&]() { return draft_impl<T>(h, k, h->g_draft, st); }));
+            mark();
+            h->len_ub = lb;
+            TRY(graph_call(h, {2, k, lb, beta, tau_bits}, st, [&]() {
+                int rc = verify_impl<T>(h, h->g_draft, k, beta, tau, nullptr, nullptr, st);
+                return rc ? rc : commit_impl(h, nullptr, nullptr, st);
+            }));
+            mark();
+            h->len_ub = std::min(true_ub + k + 1, h->T_cap);
+            h->last_k = k; h->verified = false; h->drafted = false;
+        } else {
+            TRY(draft_impl<T>(h, k, h->g_draft, st));
+            mark();
+            TRY(verify_impl<T>(h, h->g_draft, k, beta, tau, nullptr, nullptr, st));
+            mark();
+            TRY(commit_impl(h, nullptr, nullptr, st));
+        }
         mark();
         CUDA_TRY(h, cudaMemcpyAsync(h->h_poll + (it % slots), h->ses.counters + CNT_ACTIVE, 4, cudaMemcpyDeviceToHost, st));
         CUDA_TRY(h, cudaEventRecord(h->poll_ev[it % slots], st));
@@ -704,6 +785,9 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
     if (ce != cudaSuccess) return bail(SPECDEC_ERR_CUDA, std::string("weight repacking: ") + cudaGetErrorString(ce));
     if (cudaMallocHost((void**)&h->h_poll, 64 * 4) != cudaSuccess || cudaMallocHost((void**)&h->h_stats, 64) != cudaSuccess)
         return bail(SPECDEC_ERR_CUDA, "pinned host allocation failed");
+    cudaStreamCreateWithFlags(&h->own_stream, cudaStreamNonBlocking);
+    cudaEventCreateWithFlags(&h->fence_in, cudaEventDisableTiming);
+    cudaEventCreateWithFlags(&h->fence_out, cudaEventDisableTiming);
     h->poll_ev.resize(8);
     for (auto& e : h->poll_ev) cudaEventCreateWithFlags(&e, cudaEventDisableTiming);
     h->time_ev.resize((size_t)3 * h->T_cap + 8);
@@ -744,6 +828,10 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
 int specdec_destroy(specdec_handle* h) {
     if (!h) return SPECDEC_ERR_INVALID_ARG;
     cudaDeviceSynchronize();
+    drop_graphs(h);
+    if (h->own_stream) cudaStreamDestroy(h->own_stream);
+    if (h->fence_in) cudaEventDestroy(h->fence_in);
+    if (h->fence_out) cudaEventDestroy(h->fence_out);
     for (auto& e : h->poll_ev) cudaEventDestroy(e);
     for (auto& e : h->time_ev) cudaEventDestroy(e);
     for (auto& e : h->prof_ev) cudaEventDestroy(e);
@@ -756,6 +844,7 @@ int specdec_destroy(specdec_handle* h) {
 
 int specdec_set_option(specdec_handle* h, const char* name, int value) {
     if (!h || !name) return SPECDEC_ERR_INVALID_ARG;
+    drop_graphs(h);
     if (!strcmp(name, "gemm")) {
         if (value && (h->dtype != SPECDEC_DTYPE_BF16 || !h->tma.ready))
             return fail(h, SPECDEC_ERR_UNSUPPORTED, "tensor-core GEMM needs a bf16 handle on an sm_100 device");
@@ -775,7 +864,8 @@ int specdec_encode(specdec_handle* h, const int32_t* d_src, const int32_t* d_src
     if (!h) return SPECDEC_ERR_INVALID_ARG;
     if (!d_src || !d_src_len || B < 1 || S_max < 1) return fail(h, SPECDEC_ERR_INVALID_ARG, "encode: bad argument");
     if (B > h->B_cap || S_max > h->S_cap) return fail(h, SPECDEC_ERR_CAPACITY, "encode: B or S_max beyond capacity");
-    cudaStream_t st = (cudaStream_t)stream;
+    StreamScope scope(h, stream);
+    cudaStream_t st = scope.st;
     return DISPATCH(h, encode_impl<bf16>(h, d_src, d_src_len, d_max_tgt, B, S_max, st),
                     encode_impl<float>(h, d_src, d_src_len, d_max_tgt, B, S_max, st));
 }
@@ -785,7 +875,17 @@ int specdec_draft(specdec_handle* h, int k, int32_t* d_draft, void* stream) {
     if (!h->encoded) return fail(h, SPECDEC_ERR_NOT_ENCODED, "draft: no session (call specdec_encode)");
     if (!d_draft) return fail(h, SPECDEC_ERR_INVALID_ARG, "draft: null output");
     if (k < 1 || k > h->k_cap) return fail(h, SPECDEC_ERR_CAPACITY, "draft: k outside [1, k_max]");
-    cudaStream_t st = (cudaStream_t)stream;
+    StreamScope scope(h, stream);
+    cudaStream_t st = scope.st;
+    if (h->use_graphs && !h->profile) {
+        const int true_ub = h->len_ub, lb = len_bucket(h, true_ub);
+        h->len_ub = lb;
+        int rc = graph_call(h, {3, k, lb, (long long)(intptr_t)d_draft}, st, [&]() {
+            return DISPATCH(h, draft_impl<bf16>(h, k, d_draft, st), draft_impl<float>(h, k, d_draft, st)); });
+        h->len_ub = true_ub;
+        h->drafted = true; h->verified = false; h->last_draft_rows_ub = h->B * k;
+        return rc;
+    }
     return DISPATCH(h, draft_impl<bf16>(h, k, d_draft, st), draft_impl<float>(h, k, d_draft, st));
 }
 
@@ -796,7 +896,20 @@ int specdec_verify(specdec_handle* h, const int32_t* d_draft, int k, int beta, f
     if (!d_draft) return fail(h, SPECDEC_ERR_INVALID_ARG, "verify: null drafts");
     if (k < 1 || k > h->k_cap) return fail(h, SPECDEC_ERR_CAPACITY, "verify: k outside [1, k_max]");
     if (beta < 1 || !(tau >= 0.f)) return fail(h, SPECDEC_ERR_INVALID_ARG, "verify: beta >= 1 and tau >= 0 required");
-    cudaStream_t st = (cudaStream_t)stream;
+    StreamScope scope(h, stream);
+    cudaStream_t st = scope.st;
+    if (h->use_graphs && !h->profile) {
+        const int true_ub = h->len_ub, lb = len_bucket(h, true_ub);
+        int tau_bits; memcpy(&tau_bits, &tau, 4);
+        h->len_ub = lb;
+        int rc = graph_call(h, {4, k, lb, beta, tau_bits, (long long)(intptr_t)d_draft, (long long)(intptr_t)d_accepted,
+                                (long long)(intptr_t)d_bif}, st, [&]() {
+            return DISPATCH(h, verify_impl<bf16>(h, d_draft, k, beta, tau, d_accepted, d_bif, st),
+                            verify_impl<float>(h, d_draft, k, beta, tau, d_accepted, d_bif, st)); });
+        h->len_ub = true_ub;
+        h->last_k = k; h->verified = true; h->drafted = false;
+        return rc;
+    }
     return DISPATCH(h, verify_impl<bf16>(h, d_draft, k, beta, tau, d_accepted, d_bif, st),
                     verify_impl<float>(h, d_draft, k, beta, tau, d_accepted, d_bif, st));
 }
@@ -805,7 +918,8 @@ int specdec_commit(specdec_handle* h, const int32_t* d_keep, const int32_t* d_ne
     if (!h) return SPECDEC_ERR_INVALID_ARG;
     if (!h->encoded) return fail(h, SPECDEC_ERR_NOT_ENCODED, "commit: no session (call specdec_encode)");
     if (!h->verified) return fail(h, SPECDEC_ERR_INVALID_ARG, "commit: must follow specdec_verify");
-    return commit_impl(h, d_keep, d_next, (cudaStream_t)stream);
+    StreamScope scope(h, stream);
+    return commit_impl(h, d_keep, d_next, scope.st);
 }
 
 int specdec_get_output(specdec_handle* h, int32_t* d_out, int out_stride, int32_t* d_out_len, int32_t* d_finished,
@@ -813,7 +927,8 @@ int specdec_get_output(specdec_handle* h, int32_t* d_out, int out_stride, int32_
     if (!h) return SPECDEC_ERR_INVALID_ARG;
     if (!h->B) return fail(h, SPECDEC_ERR_NOT_ENCODED, "get_output: no session");
     if (d_out && out_stride < 1) return fail(h, SPECDEC_ERR_INVALID_ARG, "get_output: out_stride < 1");
-    k_copy_out<<<h->B, 128, 0, (cudaStream_t)stream>>>(h->ses, h->B, d_out, out_stride, d_out_len, d_finished);
+    StreamScope scope(h, stream);
+    k_copy_out<<<h->B, 128, 0, scope.st>>>(h->ses, h->B, d_out, out_stride, d_out_len, d_finished);
     KCHECK(h);
     return SPECDEC_OK;
 }
@@ -827,7 +942,8 @@ int specdec_generate(specdec_handle* h, const int32_t* d_src, const int32_t* d_s
     if (B > h->B_cap || S_max > h->S_cap) return fail(h, SPECDEC_ERR_CAPACITY, "generate: B or S_max beyond capacity");
     if (k < 1 || k > h->k_cap) return fail(h, SPECDEC_ERR_CAPACITY, "generate: k outside [1, k_max]");
     if (beta < 1 || !(tau >= 0.f)) return fail(h, SPECDEC_ERR_INVALID_ARG, "generate: beta >= 1 and tau >= 0 required");
-    cudaStream_t st = (cudaStream_t)stream;
+    StreamScope scope(h, stream);
+    cudaStream_t st = scope.st;
     int rc = DISPATCH(h, generate_impl<bf16>(h, d_src, d_src_len, d_max_tgt, B, S_max, k, beta, tau, d_out, out_stride, d_out_len, h_stats, st),
                       generate_impl<float>(h, d_src, d_src_len, d_max_tgt, B, S_max, k, beta, tau, d_out, out_stride, d_out_len, h_stats, st));
     if (h_stats) h_stats->status = rc;
@@ -841,7 +957,8 @@ int specdec_generate_host(specdec_handle* h, const int32_t* h_src, const int32_t
     if (!h_src || !h_src_len || !h_out || !h_out_len || B < 1 || S_max < 1 || out_stride < 1)
         return fail(h, SPECDEC_ERR_INVALID_ARG, "generate_host: bad argument");
     if (B > h->B_cap || S_max > h->S_cap) return fail(h, SPECDEC_ERR_CAPACITY, "generate_host: B or S_max beyond capacity");
-    cudaStream_t st = (cudaStream_t)stream;
+    StreamScope scope(h, stream);
+    cudaStream_t st = scope.st;
     int *s_src = h->stage_src, *s_len = h->stage_len, *s_mt = h->stage_mt;
     CUDA_TRY(h, cudaMemcpyAsync(s_src, h_src, (size_t)B * S_max * 4, cudaMemcpyHostToDevice, st));
     CUDA_TRY(h, cudaMemcpyAsync(s_len, h_src_len, (size_t)B * 4, cudaMemcpyHostToDevice, st));
@@ -866,10 +983,11 @@ int specdec_set_draft_script(specdec_handle* h, const int32_t* d_script, int B, 
     if (!h) return SPECDEC_ERR_INVALID_ARG;
     if (!d_script) { h->script_on = false; return SPECDEC_OK; }
     if (B < 1 || B > h->B_cap || stride < 1) return fail(h, SPECDEC_ERR_CAPACITY, "set_draft_script: bad B or stride");
+    StreamScope scope(h, stream);
     const int w = std::min(stride, h->T_cap + h->k_cap);
-    CUDA_TRY(h, cudaMemsetAsync(h->script, 0xff, (size_t)h->B_cap * (h->T_cap + h->k_cap) * 4, (cudaStream_t)stream));
+    CUDA_TRY(h, cudaMemsetAsync(h->script, 0xff, (size_t)h->B_cap * (h->T_cap + h->k_cap) * 4, scope.st));
     CUDA_TRY(h, cudaMemcpy2DAsync(h->script, (size_t)(h->T_cap + h->k_cap) * 4, d_script, (size_t)stride * 4, (size_t)w * 4, B,
-                                  cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+                                  cudaMemcpyDeviceToDevice, scope.st));
     h->script_on = true;
     return SPECDEC_OK;
 }
@@ -943,7 +1061,8 @@ int specdec_accept_scan_static(const float* d_logits, const int32_t* d_draft, in
 
 int specdec_debug_logits(specdec_handle* h, int which, float* d_logits, void* stream) {
     if (!h || !d_logits) return SPECDEC_ERR_INVALID_ARG;
-    cudaStream_t st = (cudaStream_t)stream;
+    StreamScope scope(h, stream);
+    cudaStream_t st = scope.st;
     int cnt, rows; const ModelW* m;
     if (which == 0) { if (!h->verified) return fail(h, SPECDEC_ERR_INVALID_ARG, "debug_logits: no verify pass to replay");
         cnt = CNT_VERIFY; rows = h->B * (h->last_k + 1); m = &h->ver; }
@@ -957,8 +1076,9 @@ int specdec_debug_logits(specdec_handle* h, int which, float* d_logits, void* st
 int specdec_debug_row_stats(specdec_handle* h, float* d_stats, void* stream) {
     if (!h || !d_stats) return SPECDEC_ERR_INVALID_ARG;
     if (!h->verified) return fail(h, SPECDEC_ERR_INVALID_ARG, "debug_row_stats: no verify pass");
+    StreamScope scope(h, stream);
     CUDA_TRY(h, cudaMemcpyAsync(d_stats, h->row_stats, (size_t)h->B * (h->last_k + 1) * 6 * 4, cudaMemcpyDeviceToDevice,
-                                (cudaStream_t)stream));
+                                scope.st));
     return SPECDEC_OK;
 }
 

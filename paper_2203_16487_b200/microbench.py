@@ -48,6 +48,7 @@ def main():
     ap.add_argument("--no-flush", action="store_true")
     ap.add_argument("--draft", action="store_true")
     ap.add_argument("--gemm", type=int, default=1)
+    ap.add_argument("--graphs", type=int, default=1)
     args = ap.parse_args()
     B, k, j, S = args.batch, args.k, args.prefix, args.src_len
 
@@ -57,6 +58,7 @@ def main():
     sd = binding.SpecDec(wl.verifier, wv, wl.drafter, wd, k_max=max(k, 1), max_batch=B, max_src=S,
                          max_tgt=j + k + 2, bf16=True)
     sd.set_option("gemm", args.gemm)
+    sd.set_option("graphs", args.graphs)
     src, lens = W.pad_batch(wl.src)
     sd.encode(src, lens, None)
     prefix, rej = W.config5_prefix_and_rejections(B, j)
@@ -86,8 +88,10 @@ def main():
         if rej[b] <= k:
             drafts[b, rej[b] - 1] = (drafts[b, rej[b] - 1] + 17) % wl.verifier.vocab
     d_drafts = torch.from_numpy(drafts).cuda()
-    acc, _ = sd.verify(d_drafts, 3, 1.0)
-    mean_a = float(acc.float().mean())
+    acc_t = torch.zeros(B, dtype=torch.int32, device="cuda")
+    bif_t = torch.zeros(B, dtype=torch.int32, device="cuda")
+    sd.verify_raw(d_drafts, 3, 1.0, acc_t, bif_t)
+    mean_a = float(acc_t.float().mean())
 
     flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
     times = []
@@ -99,7 +103,7 @@ def main():
         if args.draft:
             sd.draft(k)
         else:
-            sd.verify(d_drafts, 3, 1.0)
+            sd.verify_raw(d_drafts, 3, 1.0, acc_t, bif_t)
         e1.record()
         torch.cuda.synchronize()
         if r >= args.warmup:

@@ -65,10 +65,11 @@ def test_accept_scan_matches_oracle(V, k, B):
 
 
 # ---------------------------------------------------------------- config 1: tiny fp32
-@pytest.mark.parametrize("beta,tau", [(3, 1.0), (1, 0.0)])
-def test_config1_generate_bit_exact(tiny, beta, tau):
+@pytest.mark.parametrize("beta,tau,graphs", [(3, 1.0, 1), (1, 0.0, 1), (3, 1.0, 0)])
+def test_config1_generate_bit_exact(tiny, beta, tau, graphs):
     wl, wv, wd, mv, md = tiny
     sd = _handle(wl.verifier, wv, wl.drafter, wd, False)
+    sd.set_option("graphs", graphs)
     for s in wl.src:                                         # batch 1, one source at a time
         out, n, st = sd.generate(s[None], [len(s)], [32], wl.k, beta, tau)
         got = out[0, :int(n[0])].cpu().tolist()
