@@ -199,7 +199,8 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
 /* Options: "gemm" = 0 SIMT reference GEMM, 1 tcgen05 GEMM (bf16 handles; default 1);
  * "attn" = 0 warp-per-row reference attention, 1 tensor-core tile attention (bf16, 64-wide heads; default 1);
  * "graphs" = 0/1 replay draft/verify steps from CUDA graphs inside specdec_generate;
- * "profile" = 0/1 (see specdec_profile_read). */
+ * "profile" = 0/1 (see specdec_profile_read); "row_lse" = 0/1 also accumulate the log-sum-exp of
+ * every verifier row (only reported through specdec_debug_row_stats; the rule does not need it). */
 int specdec_set_option(specdec_handle* h, const char* name, int value);
 
 /* Number of kernels the library has launched on this handle since create. */

@@ -8,13 +8,15 @@
 //     row per thread) and apply the fused epilogue: bias / ReLU / residual add / fp32 store / the
 //     per-row vocabulary statistics that replace the logits tensor.
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, warps 2..5 = epilogue.
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, warps 2..9 = epilogue
+// (two warps per TMEM lane quadrant, each taking half of the tile's columns).
 // Every mbarrier wait is bounded; on a timeout the CTA flags an error word in global memory,
 // stops waiting everywhere, still releases its tensor memory and returns.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <map>
 #include <string>
 #include <tuple>
@@ -113,25 +115,53 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-constexpr int TC_BM = 128, TC_BK = 64, TC_THREADS = 192;
+constexpr int TC_BM = 128, TC_BK = 64;
+constexpr int TC_EPI_WARPS = 8;                      // two per TMEM lane quadrant: each takes half the columns
+constexpr int TC_THREADS = (2 + TC_EPI_WARPS) * 32;  // + TMA warp + MMA warp
 template <int BN> struct TcCfg {
     static constexpr int STAGES = BN >= 256 ? 4 : (BN >= 128 ? 6 : 8);
     static constexpr int STAGE_BYTES = (TC_BM + BN) * TC_BK * 2;
     static constexpr int SMEM = STAGES * STAGE_BYTES + 1024;
+    static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;      // two accumulators
 };
 
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// CW consecutive fp32 columns (CW = 16 or 32) of this thread's TMEM lane.
+template <int CW>
+__device__ __forceinline__ void tmem_ld(uint32_t taddr, float* v) {
+    if constexpr (CW == 32) { tmem_ld32(taddr, v); return; }
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Persistent kernel: CTA c works on tiles c, c + gridDim.x, ... (row tile fastest, so CTAs running
+// together share one weight tile).  The TMA ring and the two TMEM accumulators run across tiles, so the
+// epilogue of tile i overlaps the loads and MMAs of tile i + 1.
 template <int EPI, int BN>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, GemmArgs<bf16> g,
           int* err_word) {
     using Cfg = TcCfg<BN>;
     constexpr int STAGES = Cfg::STAGES;
+    constexpr int HALF = BN / 2;                     // columns per epilogue warp
+    constexpr int CW = HALF >= 32 ? 32 : 16;         // columns per TMEM read
     const int R = *g.n_rows;
-    const int m0 = blockIdx.y * TC_BM, n0 = blockIdx.x * BN;
-    if (m0 >= R) return;                       // whole CTA leaves before touching barriers or tensor memory
+    const int m_tiles = (R + TC_BM - 1) / TC_BM, n_tiles = (g.N + BN - 1) / BN;
+    const int total = m_tiles * n_tiles;
+    if ((int)blockIdx.x >= total) return;            // whole CTA leaves before touching barriers or tensor memory
 
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_full[STAGES], bar_empty[STAGES], bar_acc;
+    __shared__ __align__(8) uint64_t bar_full[STAGES], bar_empty[STAGES], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -141,11 +171,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     if (threadIdx.x == 0) {
         abort_s = 0;
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&bar_full[s]), 1); mbar_init(smem_u32(&bar_empty[s]), 1); }
-        mbar_init(smem_u32(&bar_acc), 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bar_acc_full[i]), 1); mbar_init(smem_u32(&bar_acc_empty[i]), TC_EPI_WARPS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), BN < 32 ? 32 : BN);
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), Cfg::TMEM_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -154,113 +184,150 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % STAGES;
-                if (kb >= STAGES) mbar_wait(smem_u32(&bar_empty[s]), ((kb / STAGES) - 1) & 1, abort_flag, err_word, 1);
-                if (*abort_flag) break;
-                const uint32_t a_dst = tiles + s * Cfg::STAGE_BYTES, w_dst = a_dst + TC_BM * TC_BK * 2;
-                const uint32_t bar = smem_u32(&bar_full[s]);
-                mbar_expect_tx(bar, Cfg::STAGE_BYTES);
-                tma_load_2d(a_dst, &tmA, kb * TC_BK, m0, bar);
-                tma_load_2d(w_dst, &tmW, kb * TC_BK, n0, bar);
+            int kbi = 0;                               // k-blocks issued so far, over all tiles
+            for (int t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
+                const int m0 = (t % m_tiles) * TC_BM, n0 = (t / m_tiles) * BN;
+                for (int kb = 0; kb < nkb; ++kb, ++kbi) {
+                    const int s = kbi % STAGES;
+                    if (kbi >= STAGES) mbar_wait(smem_u32(&bar_empty[s]), ((kbi / STAGES) - 1) & 1, abort_flag, err_word, 1);
+                    if (*abort_flag) break;
+                    const uint32_t a_dst = tiles + s * Cfg::STAGE_BYTES, w_dst = a_dst + TC_BM * TC_BK * 2;
+                    const uint32_t bar = smem_u32(&bar_full[s]);
+                    mbar_expect_tx(bar, Cfg::STAGE_BYTES);
+                    tma_load_2d(a_dst, &tmA, kb * TC_BK, m0, bar);
+                    tma_load_2d(w_dst, &tmW, kb * TC_BK, n0, bar);
+                }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, BN);
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % STAGES;
-                mbar_wait(smem_u32(&bar_full[s]), (kb / STAGES) & 1, abort_flag, err_word, 2);
-                if (*abort_flag) break;
+            int kbi = 0, i = 0;
+            for (int t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++i) {
+                const int ab = i & 1;
+                if (i >= 2) mbar_wait(smem_u32(&bar_acc_empty[ab]), ((i >> 1) - 1) & 1, abort_flag, err_word, 4);
                 tc_fence_after();
-                const uint32_t a_src = tiles + s * Cfg::STAGE_BYTES, w_src = a_src + TC_BM * TC_BK * 2;
-                const uint64_t ad = umma_desc_k_sw128(a_src), wd = umma_desc_k_sw128(w_src);
+                const uint32_t acc = tmem_d + ab * BN;
+                for (int kb = 0; kb < nkb; ++kb, ++kbi) {
+                    const int s = kbi % STAGES;
+                    mbar_wait(smem_u32(&bar_full[s]), (kbi / STAGES) & 1, abort_flag, err_word, 2);
+                    if (*abort_flag) break;
+                    tc_fence_after();
+                    const uint32_t a_src = tiles + s * Cfg::STAGE_BYTES, w_src = a_src + TC_BM * TC_BK * 2;
+                    const uint64_t ad = umma_desc_k_sw128(a_src), wd = umma_desc_k_sw128(w_src);
 #pragma unroll
-                for (int k4 = 0; k4 < TC_BK / 16; ++k4)      // +32 bytes along K per instruction: 2 address units
-                    umma_bf16(tmem_d, ad + (uint64_t)(k4 * 2), wd + (uint64_t)(k4 * 2), idesc, (kb | k4) ? 1u : 0u);
-                umma_commit(smem_u32(&bar_empty[s]));        // stage reusable once these MMAs have read it
+                    for (int k4 = 0; k4 < TC_BK / 16; ++k4)      // +32 bytes along K per instruction: 2 address units
+                        umma_bf16(acc, ad + (uint64_t)(k4 * 2), wd + (uint64_t)(k4 * 2), idesc, (kb | k4) ? 1u : 0u);
+                    umma_commit(smem_u32(&bar_empty[s]));        // stage reusable once these MMAs have read it
+                }
+                umma_commit(smem_u32(&bar_acc_full[ab]));        // accumulator of this tile complete
             }
-            umma_commit(smem_u32(&bar_acc));                 // accumulator complete
         }
     } else {
-        const int q = warp & 3;                              // TMEM lane quadrant this warp may read
-        const int r = m0 + q * 32 + lane;
-        const bool live = mbar_wait(smem_u32(&bar_acc), 0, abort_flag, err_word, 3);
-        tc_fence_after();
-        const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16);
-        float v[32];
-        if (EPI == EPI_STATS) {
-            const float ld = (g.ld && r < R) ? g.ld[r] : CUDART_INF_F;
-            const int id = (g.ld_id && r < R) ? g.ld_id[r] : -1;
-            RowPart p; p.mx = -CUDART_INF_F; p.arg = 0x7fffffff; p.sum = 0.f; p.cnt = 0;
-            for (int c = 0; c < BN / 32; ++c) {
-                tmem_ld32(trow + c * 32, v);
+        const int q = warp & 3;                                  // TMEM lane quadrant this warp may read
+        const int half = (warp - 2) >> 2;                        // which half of the tile's columns
+        int i = 0;
+        for (int t = blockIdx.x; t < total; t += gridDim.x, ++i) {
+            const int ab = i & 1;
+            const int m0 = (t % m_tiles) * TC_BM, n_tile = t / m_tiles, n0 = n_tile * BN + half * HALF;
+            const int r = m0 + q * 32 + lane;
+            const bool live = mbar_wait(smem_u32(&bar_acc_full[ab]), (i >> 1) & 1, abort_flag, err_word, 3);
+            tc_fence_after();
+            const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16) + ab * BN + half * HALF;
+            const bool warp_live = live && (m0 + q * 32 < R);    // warp-uniform: any live row in this quadrant
+            float v[CW];
+            if (warp_live && EPI == EPI_STATS) {
+                const float ld = (g.ld && r < R) ? g.ld[r] : CUDART_INF_F;
+                const int id = (g.ld_id && r < R) ? g.ld_id[r] : -1;
+                // four interleaved running statistics shorten the dependent chain; merged in column order
+                float mx[4]; int arg[4]; int cnt = 0;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int n = n0 + c * 32 + j;
-                    if (n < g.N) {
-                        const float x = (n == id) ? ld : v[j];   // the draft's column takes the pre-pass value
-                        if (x > p.mx) { p.mx = x; p.arg = n; }
-                        p.cnt += (x > ld) ? 1 : 0;
+                for (int u = 0; u < 4; ++u) { mx[u] = -CUDART_INF_F; arg[u] = 0x7fffffff; }
+                for (int c = 0; c < HALF / CW; ++c) {
+                    tmem_ld<CW>(trow + c * CW, v);
+#pragma unroll
+                    for (int j = 0; j < CW; ++j) {
+                        const int n = n0 + c * CW + j;
+                        const float x = (n >= g.N) ? -CUDART_INF_F : ((n == id) ? ld : v[j]);   // draft column: pre-pass value
+                        if (x > mx[j & 3]) { mx[j & 3] = x; arg[j & 3] = n; }
+                        cnt += (x > ld) ? 1 : 0;
                     }
                 }
-            }
-            for (int c = 0; c < BN / 32; ++c) {
-                tmem_ld32(trow + c * 32, v);
+                RowPart p; p.mx = mx[0]; p.arg = arg[0]; p.sum = 0.f; p.cnt = cnt;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int n = n0 + c * 32 + j;
-                    if (n < g.N) p.sum += expf(((n == id) ? ld : v[j]) - p.mx);
-                }
-            }
-            if (live && r < R) g.part[(size_t)r * g.n_tiles + blockIdx.x] = p;
-        } else {
-            for (int c = 0; c < BN / 32; ++c) {
-                tmem_ld32(trow + c * 32, v);
-                const int nb = n0 + c * 32;
-                if (!live || r >= R) continue;
-                if (g.bias) {
+                for (int u = 1; u < 4; ++u)
+                    if (mx[u] > p.mx || (mx[u] == p.mx && arg[u] < p.arg)) { p.mx = mx[u]; p.arg = arg[u]; }
+                if (g.want_sum) {
+                    for (int c = 0; c < HALF / CW; ++c) {
+                        tmem_ld<CW>(trow + c * CW, v);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] += (nb + j < g.N) ? __ldg(g.bias + nb + j) : 0.f;
-                }
-                const bool full = nb + 32 <= g.N;
-                if (EPI == EPI_STORE || EPI == EPI_RELU) {
-                    bf16* o = g.out + (size_t)r * g.ldo + nb;
-                    if (full && (g.ldo % 8 == 0)) {
-#pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
-                            __align__(16) bf16 t[8];
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) t[e] = __float2bfloat16_rn(EPI == EPI_RELU ? fmaxf(v[j + e], 0.f) : v[j + e]);
-                            *reinterpret_cast<uint4*>(o + j) = *reinterpret_cast<const uint4*>(t);
+                        for (int j = 0; j < CW; ++j) {
+                            const int n = n0 + c * CW + j;
+                            if (n < g.N) p.sum += expf(((n == id) ? ld : v[j]) - p.mx);
                         }
-                    } else {
-                        for (int j = 0; j < 32; ++j)
-                            if (nb + j < g.N) o[j] = __float2bfloat16_rn(EPI == EPI_RELU ? fmaxf(v[j], 0.f) : v[j]);
                     }
-                } else {
-                    float* o = g.resid + (size_t)r * g.N + nb;
-                    if (full && (g.N % 4 == 0)) {
+                }
+                if (r < R) g.part[(size_t)r * g.n_tiles + n_tile * 2 + half] = p;
+            } else if (warp_live) {
+                for (int c = 0; c < HALF / CW; ++c) {
+                    tmem_ld<CW>(trow + c * CW, v);
+                    const int nb = n0 + c * CW;
+                    if (r >= R) continue;
+                    if (g.bias) {
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            float4 t = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                            if (EPI == EPI_RESID) {
-                                const float4 x = *reinterpret_cast<const float4*>(o + j);
-                                t.x += x.x; t.y += x.y; t.z += x.z; t.w += x.w;
+                        for (int j = 0; j < CW; ++j) v[j] += (nb + j < g.N) ? __ldg(g.bias + nb + j) : 0.f;
+                    }
+                    const bool full = nb + CW <= g.N;
+                    if (EPI == EPI_STORE || EPI == EPI_RELU || EPI == EPI_QKV) {
+                        bf16* o = g.out + (size_t)r * g.ldo + nb;
+                        int ldo_ok = g.ldo % 8 == 0;
+                        if (EPI == EPI_QKV && nb >= g.kv_d) {              // K or V part: straight into the paged cache
+                            const size_t row = g.pg.row(g.seq[r], g.pos[r]);
+                            o = (nb < 2 * g.kv_d ? g.kc + row * g.kv_d + (nb - g.kv_d) : g.vc + row * g.kv_d + (nb - 2 * g.kv_d));
+                            ldo_ok = g.kv_d % 8 == 0;
+                        }
+                        if (full && ldo_ok) {
+#pragma unroll
+                            for (int j = 0; j < CW; j += 8) {
+                                __align__(16) bf16 tb[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) tb[e] = __float2bfloat16_rn(EPI == EPI_RELU ? fmaxf(v[j + e], 0.f) : v[j + e]);
+                                *reinterpret_cast<uint4*>(o + j) = *reinterpret_cast<const uint4*>(tb);
                             }
-                            *reinterpret_cast<float4*>(o + j) = t;
+                        } else {
+                            for (int j = 0; j < CW; ++j)
+                                if (nb + j < g.N) o[j] = __float2bfloat16_rn(EPI == EPI_RELU ? fmaxf(v[j], 0.f) : v[j]);
                         }
                     } else {
-                        for (int j = 0; j < 32; ++j)
-                            if (nb + j < g.N) o[j] = (EPI == EPI_RESID ? o[j] : 0.f) + v[j];
+                        float* o = g.resid + (size_t)r * g.N + nb;
+                        if (full && (g.N % 4 == 0)) {
+                            float4 xin[CW / 4];
+                            if (EPI == EPI_RESID) {
+#pragma unroll
+                                for (int j = 0; j < CW / 4; ++j) xin[j] = *reinterpret_cast<const float4*>(o + j * 4);
+                            }
+#pragma unroll
+                            for (int j = 0; j < CW / 4; ++j) {
+                                float4 tv = make_float4(v[j * 4], v[j * 4 + 1], v[j * 4 + 2], v[j * 4 + 3]);
+                                if (EPI == EPI_RESID) { tv.x += xin[j].x; tv.y += xin[j].y; tv.z += xin[j].z; tv.w += xin[j].w; }
+                                *reinterpret_cast<float4*>(o + j * 4) = tv;
+                            }
+                        } else {
+                            for (int j = 0; j < CW; ++j)
+                                if (nb + j < g.N) o[j] = (EPI == EPI_RESID ? o[j] : 0.f) + v[j];
+                        }
                     }
                 }
             }
+            // this warp is done with the accumulator: hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[ab]));
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem_d, BN < 32 ? 32 : BN);
+    if (warp == 1) tmem_dealloc(tmem_d, Cfg::TMEM_COLS);
 }
 
 // ------------------------------------------------------------------ host side
@@ -273,6 +340,7 @@ struct TmaEncoder {
     std::string err = "not initialised";
     PFN_encodeTiled encode = nullptr;
     int* err_word = nullptr;            // device word the kernels raise on a wait timeout
+    int n_sm = 148;
     std::map<std::tuple<const void*, long long, int, int, int>, CUtensorMap> cache;
 
     // 2-D bf16 tensor [rows, K] with row pitch ld elements; box = 64 x box_rows, 128-byte swizzle.
@@ -315,6 +383,7 @@ inline int tc_init(TmaEncoder& enc, int* err_word) {
         enc.err = "cannot query the device"; return -1;
     }
     if (major != 10) { enc.err = "device is not sm_100"; return -1; }
+    cudaDeviceGetAttribute(&enc.n_sm, cudaDevAttrMultiProcessorCount, dev);
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
@@ -324,6 +393,7 @@ inline int tc_init(TmaEncoder& enc, int* err_word) {
     if (e == cudaSuccess) e = tc_set_smem_all<EPI_RELU>();
     if (e == cudaSuccess) e = tc_set_smem_all<EPI_RESID>();
     if (e == cudaSuccess) e = tc_set_smem_all<EPI_F32>();
+    if (e == cudaSuccess) e = tc_set_smem_all<EPI_QKV>();
     if (e == cudaSuccess) e = tc_set_smem<EPI_STATS, 128>();
     if (e != cudaSuccess) { enc.err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return -1; }
     enc.err_word = err_word;
@@ -337,7 +407,8 @@ inline int tc_launch_one(TmaEncoder& enc, GemmArgs<bf16>& g, int rows_ub, cudaSt
     const CUtensorMap* ta = enc.get(g.A, rows_ub, g.K, g.lda, TC_BM);
     const CUtensorMap* tw = enc.get(g.W, g.N, g.K, g.K, BN);
     if (!ta || !tw) return -1;
-    dim3 grid((g.N + BN - 1) / BN, (rows_ub + TC_BM - 1) / TC_BM);
+    const long long tiles_ub = (long long)((g.N + BN - 1) / BN) * ((rows_ub + TC_BM - 1) / TC_BM);
+    const int grid = (int)std::min<long long>(tiles_ub, enc.n_sm);
     k_gemm_tc<EPI, BN><<<grid, TC_THREADS, TcCfg<BN>::SMEM, st>>>(*ta, *tw, g, enc.err_word);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { enc.err = std::string("launch: ") + cudaGetErrorString(e); return -1; }
@@ -371,7 +442,7 @@ inline int gemm_tc_launch(TmaEncoder& enc, int epi, GemmArgs<bf16>& g, int rows_
     if (!enc.ready) return -1;
     if (epi == EPI_STATS) {
         if (g.N < 128) return -2;
-        g.n_tiles = (g.N + 127) / 128;
+        g.n_tiles = 2 * ((g.N + 127) / 128);          // two column halves per tile
         if (n_tiles_out) *n_tiles_out = g.n_tiles;
         return tc_launch_one<EPI_STATS, 128>(enc, g, rows_ub, st);
     }
@@ -380,6 +451,7 @@ inline int gemm_tc_launch(TmaEncoder& enc, int epi, GemmArgs<bf16>& g, int rows_
         case EPI_STORE: return tc_launch_bn<EPI_STORE>(enc, bn, g, rows_ub, st);
         case EPI_RELU: return tc_launch_bn<EPI_RELU>(enc, bn, g, rows_ub, st);
         case EPI_RESID: return tc_launch_bn<EPI_RESID>(enc, bn, g, rows_ub, st);
+        case EPI_QKV: return tc_launch_bn<EPI_QKV>(enc, bn, g, rows_ub, st);
         default: return tc_launch_bn<EPI_F32>(enc, bn, g, rows_ub, st);
     }
 }

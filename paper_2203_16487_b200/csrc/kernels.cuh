@@ -257,7 +257,7 @@ __global__ void k_attention(AttnArgs<T> a) {
 
 // ------------------------------------------------------------------ GEMM epilogues
 // C[r, n] = sum_k A[r, k] * W[n, k]  (+ bias[n])
-enum { EPI_STORE = 0, EPI_RELU = 1, EPI_RESID = 2, EPI_STATS = 3, EPI_F32 = 4 };
+enum { EPI_STORE = 0, EPI_RELU = 1, EPI_RESID = 2, EPI_STATS = 3, EPI_F32 = 4, EPI_QKV = 5 };
 
 // Partial statistics of one verifier (or drafter) row over one tile of vocabulary columns.
 struct __align__(16) RowPart { float mx; int arg; float sum; int cnt; };
@@ -275,6 +275,10 @@ struct GemmArgs {
     RowPart* part; int n_tiles; // part[r * n_tiles + tile]
     const float* ld;            // [rows] logit of the row's draft from the pre-pass (+inf: none)
     const int* ld_id;           // [rows] the draft's id (-1: none)
+    int want_sum;               // also accumulate sum exp(l - max) (only needed to report log-probabilities)
+    // EPI_QKV: columns [0, kv_d) are stored like EPI_STORE, [kv_d, 2 kv_d) go to the K cache and
+    // [2 kv_d, 3 kv_d) to the V cache at the row's (sequence, position)
+    const int* seq; const int* pos; Paged pg; T* kc; T* vc; int kv_d;
 };
 
 // Merge order of row statistics: larger maximum wins, equal maxima keep the lower id.
@@ -361,10 +365,11 @@ __global__ void __launch_bounds__(256) k_gemm_simt(GemmArgs<T> g) {
                 if (v > p.mx) { p.mx = v; p.arg = n0 + j; }
                 p.cnt += (v > ld) ? 1 : 0;
             }
-            for (int j = 0; j < nn; ++j) {
-                float v = (n0 + j == id) ? ld : Ct[tid][j];
-                p.sum += expf(v - p.mx);
-            }
+            if (g.want_sum)
+                for (int j = 0; j < nn; ++j) {
+                    float v = (n0 + j == id) ? ld : Ct[tid][j];
+                    p.sum += expf(v - p.mx);
+                }
             g.part[(size_t)r * g.n_tiles + blockIdx.x] = p;
         }
     }

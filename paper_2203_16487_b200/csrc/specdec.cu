@@ -79,7 +79,7 @@ struct specdec_handle {
     bool encoded = false, verified = false, drafted = false;
     int last_draft_rows_ub = 0;
     // options
-    int use_tc = 1, use_graphs = 1, use_tc_attn = 1;
+    int use_tc = 1, use_graphs = 1, use_tc_attn = 1, want_lse = 0;
     // CUDA graphs of whole draft / verify(+commit) steps, keyed by everything their launches depend on
     struct GraphEntry { cudaGraphExec_t exec; long long kernels; };
     std::map<std::vector<long long>, GraphEntry> graphs;
@@ -288,16 +288,26 @@ int ln(specdec_handle* h, const float* x, const float* g, const float* b, int cn
     return 0;
 }
 
+// Where the K and V columns of a fused QKV projection go (the verifier's paged cache).
+struct KvDest { const int* seq; const int* pos; void* kc; void* vc; int d; };
+
+template <typename T> bool tc_usable(const specdec_handle* h, int N, int K) {
+    return std::is_same<T, bf16>::value && h->use_tc && sd::tc_supported(N, K);
+}
+
 // out = A W^T (+bias) with one of the epilogues; rows_ub bounds the grid, the live count is on the device.
 template <typename T>
 int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, const float* bias, int N, int K, int cnt,
          int rows_ub, void* out, int ldo, float* resid, cudaStream_t st, const float* ldv = nullptr,
-         const int* ld_id = nullptr, int* n_tiles_out = nullptr) {
+         const int* ld_id = nullptr, int* n_tiles_out = nullptr, const KvDest* kv = nullptr) {
     if (rows_ub <= 0) return 0;
     GemmArgs<T> g;
     g.A = (const T*)A; g.lda = lda; g.W = (const T*)W; g.bias = bias; g.N = N; g.K = K;
     g.n_rows = h->ses.counters + cnt; g.out = (T*)out; g.ldo = ldo; g.resid = resid;
-    g.part = h->part; g.ld = ldv; g.ld_id = ld_id; g.n_tiles = cdiv(N, 64);
+    g.part = h->part; g.ld = ldv; g.ld_id = ld_id; g.n_tiles = cdiv(N, 64); g.want_sum = h->want_lse;
+    g.seq = nullptr; g.pos = nullptr; g.kc = nullptr; g.vc = nullptr; g.kv_d = 0;
+    g.pg.table = h->page_table; g.pg.page_tokens = h->cfg.page_tokens; g.pg.max_pages = h->pages_per_seq;
+    if (kv) { g.seq = kv->seq; g.pos = kv->pos; g.kc = (T*)kv->kc; g.vc = (T*)kv->vc; g.kv_d = kv->d; }
     if constexpr (std::is_same<T, bf16>::value) {
         if (h->use_tc && sd::tc_supported(N, K) && (epi != EPI_STATS || N >= 128)) {
             int rc = sd::gemm_tc_launch(h->tma, epi, g, rows_ub, st, n_tiles_out);
@@ -391,12 +401,21 @@ int block_self(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, co
     const int d = m.dm.d_model, H = m.dm.n_heads, dh = d / H;
     const size_t e = h->esz;
     TRY(ln<T>(h, x, w.ln1_g, w.ln1_b, cnt, rows_ub, h->y, d, st));
-    TRY(gemm<T>(h, EPI_STORE, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, cnt, rows_ub, h->qkv, 3 * d, nullptr, st));
+    if (verify && tc_usable<T>(h, 3 * d, d) && d % 32 == 0) {
+        // K and V columns leave the GEMM epilogue straight into the paged cache
+        KvDest kv{r.seq, r.pos, h->kc[layer], h->vc[layer], d};
+        TRY(gemm<T>(h, EPI_QKV, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, cnt, rows_ub, h->qkv, 3 * d, nullptr, st, nullptr,
+                    nullptr, nullptr, &kv));
+    } else {
+        TRY(gemm<T>(h, EPI_STORE, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, cnt, rows_ub, h->qkv, 3 * d, nullptr, st));
+        if (verify) {
+            Paged pg{h->page_table, h->cfg.page_tokens, h->pages_per_seq};
+            k_kv_scatter<T><<<rows_ub, 128, 0, st>>>((const T*)h->qkv, r.seq, r.pos, h->ses.counters + cnt, pg,
+                                                     (T*)h->kc[layer], (T*)h->vc[layer], d);
+            KCHECK(h);
+        }
+    }
     if (verify) {
-        Paged pg{h->page_table, h->cfg.page_tokens, h->pages_per_seq};
-        k_kv_scatter<T><<<rows_ub, 128, 0, st>>>((const T*)h->qkv, r.seq, r.pos, h->ses.counters + cnt, pg,
-                                                 (T*)h->kc[layer], (T*)h->vc[layer], d);
-        KCHECK(h);
         TRY(attn<T>(h, true, h->qkv, 3 * d, nullptr, h->kc[layer], h->vc[layer], d, nullptr, r, r.nk_self, cnt,
                     rows_ub, q_ub, h->att, d, H, dh, max_keys, st));
     } else {
@@ -593,7 +612,7 @@ void drop_graphs(specdec_handle* h) {
 // replayed afterwards.  The key must name everything the launches depend on besides device memory.
 template <typename F>
 int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body) {
-    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->script_on ? 1 : 0);
+    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->script_on ? 1 : 0);
     key.push_back(h->B); key.push_back(h->S_max);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
@@ -851,6 +870,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         h->use_tc = value ? 1 : 0;
         return SPECDEC_OK;
     }
+    if (!strcmp(name, "row_lse")) { h->want_lse = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "attn")) { h->use_tc_attn = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "graphs")) { h->use_graphs = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "profile")) { h->profile = value ? 1 : 0; h->prof_n = 0; h->prof_ms = 0.0; h->prof_launches = 0; return SPECDEC_OK; }

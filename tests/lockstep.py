@@ -45,6 +45,7 @@ def run(sd, mv: O.Model, md: O.Model, srcs, max_tgt, k, beta, tau, margin: float
         logit_tol: float = 1e-4, draft_fn=None, pad_to: Optional[int] = None) -> Report:
     rep = Report()
     B = len(srcs)
+    sd.set_option("row_lse", 1)
     src, lens = W.pad_batch(srcs, pad_to)
     sd.encode(src, lens, np.asarray(max_tgt, np.int32))
     mem_v = [O.encode(mv, s) for s in srcs]
