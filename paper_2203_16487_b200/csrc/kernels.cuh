@@ -281,6 +281,12 @@ struct GemmArgs {
     const int* seq; const int* pos; Paged pg; T* kc; T* vc; int kv_d;
 };
 
+// Merge of (max, argmax, count) only: used on the hot path, where the sum is not needed.
+__device__ __forceinline__ void part_merge_nosum(RowPart& a, const RowPart& b) {
+    if (b.mx > a.mx || (b.mx == a.mx && b.arg < a.arg)) { a.mx = b.mx; a.arg = b.arg; }
+    a.cnt += b.cnt;
+}
+
 // Merge order of row statistics: larger maximum wins, equal maxima keep the lower id.
 __device__ __forceinline__ void part_merge(RowPart& a, const RowPart& b) {
     float m = fmaxf(a.mx, b.mx);
@@ -399,14 +405,23 @@ __global__ void k_draft_logit(const T* __restrict__ y, const T* __restrict__ E, 
 // finds the first rejected draft.  row_stats (optional) receives 6 floats per row.
 __global__ void k_accept(const RowPart* __restrict__ part, int n_tiles, const float* __restrict__ ld,
                          const int* __restrict__ ld_id, int k, int beta, float tau, int* __restrict__ accepted,
-                         int* __restrict__ bif, float* __restrict__ row_stats) {
+                         int* __restrict__ bif, float* __restrict__ row_stats, int want_sum) {
     extern __shared__ unsigned char sm_acc[];
     RowPart* rs = reinterpret_cast<RowPart*>(sm_acc);       // [k+1]
     const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
     for (int c = warp; c <= k; c += nw) {
         const RowPart* p = part + ((size_t)b * (k + 1) + c) * n_tiles;
         RowPart m; m.mx = -CUDART_INF_F; m.arg = 0x7fffffff; m.sum = 0.f; m.cnt = 0;
-        for (int t = lane; t < n_tiles; t += 32) part_merge(m, p[t]);
+        if (want_sum) {
+            for (int t = lane; t < n_tiles; t += 32) part_merge(m, p[t]);
+        } else {
+            int t = lane;
+            for (; t + 96 < n_tiles; t += 128) {            // four independent loads in flight
+                const RowPart q0 = p[t], q1 = p[t + 32], q2 = p[t + 64], q3 = p[t + 96];
+                part_merge_nosum(m, q0); part_merge_nosum(m, q1); part_merge_nosum(m, q2); part_merge_nosum(m, q3);
+            }
+            for (; t < n_tiles; t += 32) part_merge_nosum(m, p[t]);
+        }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             RowPart q;
@@ -414,7 +429,7 @@ __global__ void k_accept(const RowPart* __restrict__ part, int n_tiles, const fl
             q.arg = __shfl_xor_sync(0xffffffffu, m.arg, o);
             q.sum = __shfl_xor_sync(0xffffffffu, m.sum, o);
             q.cnt = __shfl_xor_sync(0xffffffffu, m.cnt, o);
-            part_merge(m, q);
+            if (want_sum) part_merge(m, q); else part_merge_nosum(m, q);
         }
         if (lane == 0) rs[c] = m;
     }
@@ -433,7 +448,7 @@ __global__ void k_accept(const RowPart* __restrict__ part, int n_tiles, const fl
     if (row_stats)
         for (int c = threadIdx.x; c <= k; c += blockDim.x) {
             float* o = row_stats + ((size_t)b * (k + 1) + c) * 6;
-            o[0] = rs[c].mx; o[1] = (float)rs[c].arg; o[2] = rs[c].mx + logf(rs[c].sum);
+            o[0] = rs[c].mx; o[1] = (float)rs[c].arg; o[2] = want_sum ? rs[c].mx + logf(rs[c].sum) : 0.f;
             o[3] = (float)rs[c].cnt; o[4] = ld[b * (k + 1) + c]; o[5] = (float)ld_id[b * (k + 1) + c];
         }
 }

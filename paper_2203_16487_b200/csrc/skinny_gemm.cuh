@@ -1,0 +1,163 @@
+// Weight-streaming GEMM for a handful of activation rows (M <= 64):  C[r, n] = sum_k A[r, k] W[n, k].
+//
+// At batch 1 a verify block has k+1 = 26 rows, so every layer GEMM is a pass over its weight matrix
+// bounded by HBM, not by math.  This kernel is shaped for that: one CTA per 8 weight rows, so a
+// 512 x 512 projection already spreads over 64 SMs; the eight warps of a CTA split K, each lane
+// streams 16-byte pieces of its weight rows straight from global memory into registers (all loads are
+// issued before anything else happens), the activation rows sit in shared memory, and the products
+// run on warp-level tensor-core MMAs (m16n8k16, fp32 accumulate) with the k index permuted so that a
+// lane's 16 contiguous weight bytes are exactly its B fragments.  The K-split partial sums are added
+// in a fixed order, so results do not depend on timing.
+//
+// Optionally the activation rows are produced in the prologue as LayerNorm(x) (fp32 residual rows in,
+// bf16 operand rows into shared memory), which removes the separate normalisation launch and its
+// round trip through HBM.  Epilogues: bias + store / ReLU / residual add / QKV with K,V scattered into
+// the paged cache.
+#pragma once
+#include "attention_tc.cuh"
+#include "kernels.cuh"
+
+namespace sd {
+
+struct SkinnyArgs {
+    GemmArgs<bf16> g;            // A (bf16 rows) unless ln_x is set; W, bias, N, K, n_rows and the epilogue fields
+    const float* ln_x;           // LayerNorm prologue: fp32 rows [rows, K] ...
+    const float* ln_g; const float* ln_b; float ln_eps;
+    bf16* ln_out;                // ... optionally also written out as bf16 rows [rows, K] (by CTA 0)
+};
+
+constexpr int SK_NB = 8;         // weight rows per CTA
+constexpr int SK_WARPS = 8;
+inline size_t skinny_smem(int MT, int K) { return (size_t)MT * 16 * (K + 8) * 2 + (size_t)SK_WARPS * MT * 16 * SK_NB * 4; }
+
+template <int EPI, int MT, bool LN>
+__global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
+    extern __shared__ __align__(16) unsigned char sk_sm[];
+    const GemmArgs<bf16>& g = a.g;
+    const int K = g.K, N = g.N;
+    const int R = min(*g.n_rows, MT * 16);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t4 = lane & 3;
+    const int n0 = blockIdx.x * SK_NB;
+    const int pitch = K + 8;                                  // bf16 elements per activation row in shared memory
+    bf16* As = reinterpret_cast<bf16*>(sk_sm);
+    float* red = reinterpret_cast<float*>(sk_sm + (size_t)MT * 16 * pitch * 2);
+
+    // K split: warp s takes k in [s * ks, (s + 1) * ks), in super-steps of 32
+    const int nsplit = min(SK_WARPS, K / 32);
+    const int ks = (K / 32 + nsplit - 1) / nsplit * 32;
+    const int k_begin = warp * ks, k_end = min(K, k_begin + ks);
+    constexpr int MAX_SS = 8;                                 // super-steps whose weights are preloaded in registers
+    uint4 wreg[MAX_SS];
+    const bool w_ok = (n0 + gq) < N;
+    const bf16* wrow = g.W + (size_t)(n0 + gq) * K + t4 * 8;
+#pragma unroll
+    for (int ss = 0; ss < MAX_SS; ++ss) {
+        const int k0 = k_begin + ss * 32;
+        wreg[ss] = (w_ok && warp < nsplit && k0 < k_end) ? __ldg(reinterpret_cast<const uint4*>(wrow + k0)) : make_uint4(0, 0, 0, 0);
+    }
+
+    // ---- activation rows into shared memory
+    if (LN) {
+        for (int m = warp; m < MT * 16; m += SK_WARPS) {
+            bf16* dst = As + (size_t)m * pitch;
+            if (m < R) {
+                const float* xr = a.ln_x + (size_t)m * K;
+                float s = 0.f;
+                for (int e = lane * 4; e < K; e += 128) { const float4 v = *reinterpret_cast<const float4*>(xr + e); s += v.x + v.y + v.z + v.w; }
+                const float mu = warp_sum(s) / K;
+                float q = 0.f;
+                for (int e = lane * 4; e < K; e += 128) {
+                    const float4 v = *reinterpret_cast<const float4*>(xr + e);
+                    const float c0 = v.x - mu, c1 = v.y - mu, c2 = v.z - mu, c3 = v.w - mu;
+                    q += c0 * c0 + c1 * c1 + c2 * c2 + c3 * c3;
+                }
+                const float rstd = 1.0f / sqrtf(warp_sum(q) / K + a.ln_eps);
+                for (int e = lane * 4; e < K; e += 128) {
+                    const float4 v = *reinterpret_cast<const float4*>(xr + e);
+                    const float4 gm = *reinterpret_cast<const float4*>(a.ln_g + e), bt = *reinterpret_cast<const float4*>(a.ln_b + e);
+                    __nv_bfloat162 p0, p1;
+                    p0.x = __float2bfloat16_rn((v.x - mu) * rstd * gm.x + bt.x); p0.y = __float2bfloat16_rn((v.y - mu) * rstd * gm.y + bt.y);
+                    p1.x = __float2bfloat16_rn((v.z - mu) * rstd * gm.z + bt.z); p1.y = __float2bfloat16_rn((v.w - mu) * rstd * gm.w + bt.w);
+                    *reinterpret_cast<__nv_bfloat162*>(dst + e) = p0;
+                    *reinterpret_cast<__nv_bfloat162*>(dst + e + 2) = p1;
+                    if (a.ln_out && blockIdx.x == 0) {
+                        *reinterpret_cast<__nv_bfloat162*>(a.ln_out + (size_t)m * K + e) = p0;
+                        *reinterpret_cast<__nv_bfloat162*>(a.ln_out + (size_t)m * K + e + 2) = p1;
+                    }
+                }
+            } else {
+                for (int e = lane * 8; e < K; e += 256) *reinterpret_cast<uint4*>(dst + e) = make_uint4(0, 0, 0, 0);
+            }
+        }
+    } else {
+        const uint32_t as_base = (uint32_t)__cvta_generic_to_shared(As);
+        const int chunks = K / 8;
+        for (int i = tid; i < MT * 16 * chunks; i += SK_WARPS * 32) {
+            const int m = i / chunks, c = i % chunks;
+            if (m < R) cp_async16(as_base + (uint32_t)(m * pitch + c * 8) * 2, g.A + (size_t)m * g.lda + c * 8);
+            else *reinterpret_cast<uint4*>(As + (size_t)m * pitch + c * 8) = make_uint4(0, 0, 0, 0);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();
+
+    // ---- products: per super-step of 32 k, two MMAs per 16-row tile
+    float acc[MT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[mt][e] = 0.f;
+    if (warp < nsplit) {
+        auto step = [&](const uint4& w, int k0) {
+            const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    const uint2 lo = *reinterpret_cast<const uint2*>(As + (size_t)(mt * 16 + gq) * pitch + k0 + t4 * 8 + j * 4);
+                    const uint2 hi = *reinterpret_cast<const uint2*>(As + (size_t)(mt * 16 + gq + 8) * pitch + k0 + t4 * 8 + j * 4);
+                    const uint32_t af[4] = {lo.x, hi.x, lo.y, hi.y};
+                    mma_bf16(acc[mt], af, wv[2 * j], wv[2 * j + 1]);
+                }
+            }
+        };
+#pragma unroll
+        for (int ss = 0; ss < MAX_SS; ++ss) {
+            const int k0 = k_begin + ss * 32;
+            if (k0 < k_end) step(wreg[ss], k0);
+        }
+        for (int k0 = k_begin + MAX_SS * 32; k0 < k_end; k0 += 32) {       // K slices longer than the preloaded part
+            const uint4 w = w_ok ? __ldg(reinterpret_cast<const uint4*>(wrow + k0)) : make_uint4(0, 0, 0, 0);
+            step(w, k0);
+        }
+    }
+    // ---- fixed-order sum over the K split, then the epilogue
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        float* r0 = red + ((size_t)warp * MT * 16 + mt * 16 + gq) * SK_NB + t4 * 2;
+        r0[0] = acc[mt][0]; r0[1] = acc[mt][1];
+        r0[8 * SK_NB] = acc[mt][2]; r0[8 * SK_NB + 1] = acc[mt][3];
+    }
+    __syncthreads();
+    for (int o = tid; o < MT * 16 * SK_NB; o += SK_WARPS * 32) {
+        const int r = o / SK_NB, n = n0 + (o % SK_NB);
+        if (r >= R || n >= N) continue;
+        float v = 0.f;
+        for (int s = 0; s < nsplit; ++s) v += red[(size_t)s * MT * 16 * SK_NB + o];
+        if (g.bias) v += g.bias[n];
+        if (EPI == EPI_STORE) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(v);
+        if (EPI == EPI_RELU) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(fmaxf(v, 0.f));
+        if (EPI == EPI_RESID) g.resid[(size_t)r * N + n] += v;
+        if (EPI == EPI_QKV) {
+            if (n < g.kv_d) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(v);
+            else {
+                const size_t row = g.pg.row(g.seq[r], g.pos[r]);
+                if (n < 2 * g.kv_d) g.kc[row * g.kv_d + (n - g.kv_d)] = __float2bfloat16_rn(v);
+                else g.vc[row * g.kv_d + (n - 2 * g.kv_d)] = __float2bfloat16_rn(v);
+            }
+        }
+    }
+}
+
+}  // namespace sd

@@ -17,6 +17,7 @@
 #include "attention_tc.cuh"
 #include "gemm_tc.cuh"
 #include "kernels.cuh"
+#include "skinny_gemm.cuh"
 
 using namespace sd;
 
@@ -79,7 +80,8 @@ struct specdec_handle {
     bool encoded = false, verified = false, drafted = false;
     int last_draft_rows_ub = 0;
     // options
-    int use_tc = 1, use_graphs = 1, use_tc_attn = 1, want_lse = 0;
+    int use_tc = 1, use_graphs = 1, use_tc_attn = 1, want_lse = 0, use_skinny = 1;
+    size_t skinny_smem_cap = 0;
     // CUDA graphs of whole draft / verify(+commit) steps, keyed by everything their launches depend on
     struct GraphEntry { cudaGraphExec_t exec; long long kernels; };
     std::map<std::vector<long long>, GraphEntry> graphs;
@@ -126,6 +128,8 @@ int fail(specdec_handle* h, int code, const std::string& msg) {
                         " at line " + std::to_string(__LINE__));                            \
         ++h->launches;                                                                      \
     } while (0)
+
+#define TRY(expr) do { int rc__ = (expr); if (rc__ != 0) return rc__; } while (0)
 
 inline int cdiv(int a, int b) { return (a + b - 1) / b; }
 
@@ -295,12 +299,64 @@ template <typename T> bool tc_usable(const specdec_handle* h, int N, int K) {
     return std::is_same<T, bf16>::value && h->use_tc && sd::tc_supported(N, K);
 }
 
+// LayerNorm fused in front of a GEMM: x fp32 rows, gain, bias.
+struct LnSpec { const float* x; const float* g; const float* b; };
+
+// The weight-streaming kernel serves bf16 GEMMs over at most 64 rows (see skinny_gemm.cuh).
+template <typename T>
+bool skinny_ok(const specdec_handle* h, int epi, int rows_ub, int N, int K, bool with_ln) {
+    if (!std::is_same<T, bf16>::value || !h->use_skinny || rows_ub > 64) return false;
+    if (epi != EPI_STORE && epi != EPI_RELU && epi != EPI_RESID && epi != EPI_QKV) return false;
+    if (K % 32 || (with_ln && K % 128)) return false;
+    return skinny_smem(rows_ub <= 32 ? 2 : 4, K) <= h->skinny_smem_cap;
+}
+
+template <int EPI, int MT>
+int skinny_launch_ln(specdec_handle* h, SkinnyArgs& a, cudaStream_t st) {
+    const int grid = cdiv(a.g.N, SK_NB);
+    const size_t smem = skinny_smem(MT, a.g.K);
+    if (a.ln_x) k_skinny<EPI, MT, true><<<grid, SK_WARPS * 32, smem, st>>>(a);
+    else k_skinny<EPI, MT, false><<<grid, SK_WARPS * 32, smem, st>>>(a);
+    KCHECK(h);
+    return 0;
+}
+template <int EPI>
+int skinny_launch_mt(specdec_handle* h, SkinnyArgs& a, int rows_ub, cudaStream_t st) {
+    return rows_ub <= 32 ? skinny_launch_ln<EPI, 2>(h, a, st) : skinny_launch_ln<EPI, 4>(h, a, st);
+}
+int skinny_launch(specdec_handle* h, int epi, SkinnyArgs& a, int rows_ub, cudaStream_t st) {
+    switch (epi) {
+        case EPI_STORE: return skinny_launch_mt<EPI_STORE>(h, a, rows_ub, st);
+        case EPI_RELU: return skinny_launch_mt<EPI_RELU>(h, a, rows_ub, st);
+        case EPI_RESID: return skinny_launch_mt<EPI_RESID>(h, a, rows_ub, st);
+        default: return skinny_launch_mt<EPI_QKV>(h, a, rows_ub, st);
+    }
+}
+template <int EPI, int MT>
+cudaError_t skinny_attr(int bytes) {
+    cudaError_t e = cudaFuncSetAttribute(k_skinny<EPI, MT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_skinny<EPI, MT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    return e;
+}
+template <int EPI>
+cudaError_t skinny_attr_mt(int bytes) {
+    cudaError_t e = skinny_attr<EPI, 2>(bytes);
+    if (e == cudaSuccess) e = skinny_attr<EPI, 4>(bytes);
+    return e;
+}
+
 // out = A W^T (+bias) with one of the epilogues; rows_ub bounds the grid, the live count is on the device.
 template <typename T>
 int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, const float* bias, int N, int K, int cnt,
          int rows_ub, void* out, int ldo, float* resid, cudaStream_t st, const float* ldv = nullptr,
-         const int* ld_id = nullptr, int* n_tiles_out = nullptr, const KvDest* kv = nullptr) {
+         const int* ld_id = nullptr, int* n_tiles_out = nullptr, const KvDest* kv = nullptr,
+         const LnSpec* lnp = nullptr) {
     if (rows_ub <= 0) return 0;
+    const bool skinny = skinny_ok<T>(h, epi, rows_ub, N, K, lnp != nullptr);
+    if (lnp && !skinny) {                       // separate normalisation launch, then a plain GEMM on its output
+        TRY(ln<T>(h, lnp->x, lnp->g, lnp->b, cnt, rows_ub, h->y, K, st));
+        A = h->y; lda = K;
+    }
     GemmArgs<T> g;
     g.A = (const T*)A; g.lda = lda; g.W = (const T*)W; g.bias = bias; g.N = N; g.K = K;
     g.n_rows = h->ses.counters + cnt; g.out = (T*)out; g.ldo = ldo; g.resid = resid;
@@ -308,6 +364,15 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
     g.seq = nullptr; g.pos = nullptr; g.kc = nullptr; g.vc = nullptr; g.kv_d = 0;
     g.pg.table = h->page_table; g.pg.page_tokens = h->cfg.page_tokens; g.pg.max_pages = h->pages_per_seq;
     if (kv) { g.seq = kv->seq; g.pos = kv->pos; g.kc = (T*)kv->kc; g.vc = (T*)kv->vc; g.kv_d = kv->d; }
+    if constexpr (std::is_same<T, bf16>::value) {
+        if (skinny) {
+            SkinnyArgs sa; sa.g = g;
+            sa.ln_x = lnp ? lnp->x : nullptr; sa.ln_g = lnp ? lnp->g : nullptr; sa.ln_b = lnp ? lnp->b : nullptr;
+            sa.ln_eps = 1e-5f; sa.ln_out = nullptr;
+            TRY(skinny_launch(h, epi, sa, rows_ub, st));
+            return 0;
+        }
+    }
     if constexpr (std::is_same<T, bf16>::value) {
         if (h->use_tc && sd::tc_supported(N, K) && (epi != EPI_STATS || N >= 128)) {
             int rc = sd::gemm_tc_launch(h->tma, epi, g, rows_ub, st, n_tiles_out);
@@ -372,7 +437,6 @@ int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* 
     return 0;
 }
 
-#define TRY(expr) do { int rc__ = (expr); if (rc__ != 0) return rc__; } while (0)
 
 // With the "profile" option on, the vocabulary-projection launches are bracketed by event pairs.
 void prof_mark(specdec_handle* h, cudaStream_t st) {
@@ -400,14 +464,15 @@ int block_self(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, co
                int q_ub, int layer, bool verify, int max_keys, cudaStream_t st) {
     const int d = m.dm.d_model, H = m.dm.n_heads, dh = d / H;
     const size_t e = h->esz;
-    TRY(ln<T>(h, x, w.ln1_g, w.ln1_b, cnt, rows_ub, h->y, d, st));
+    const LnSpec l1{x, w.ln1_g, w.ln1_b};
     if (verify && tc_usable<T>(h, 3 * d, d) && d % 32 == 0) {
         // K and V columns leave the GEMM epilogue straight into the paged cache
         KvDest kv{r.seq, r.pos, h->kc[layer], h->vc[layer], d};
         TRY(gemm<T>(h, EPI_QKV, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, cnt, rows_ub, h->qkv, 3 * d, nullptr, st, nullptr,
-                    nullptr, nullptr, &kv));
+                    nullptr, nullptr, &kv, &l1));
     } else {
-        TRY(gemm<T>(h, EPI_STORE, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, cnt, rows_ub, h->qkv, 3 * d, nullptr, st));
+        TRY(gemm<T>(h, EPI_STORE, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, cnt, rows_ub, h->qkv, 3 * d, nullptr, st, nullptr,
+                    nullptr, nullptr, nullptr, &l1));
         if (verify) {
             Paged pg{h->page_table, h->cfg.page_tokens, h->pages_per_seq};
             k_kv_scatter<T><<<rows_ub, 128, 0, st>>>((const T*)h->qkv, r.seq, r.pos, h->ses.counters + cnt, pg,
@@ -431,8 +496,9 @@ int block_cross(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, c
                 int q_ub, int layer, cudaStream_t st) {
     const int d = m.dm.d_model, H = m.dm.n_heads, dh = d / H;
     const size_t e = h->esz;
-    TRY(ln<T>(h, x, w.lnc_g, w.lnc_b, cnt, rows_ub, h->y, d, st));
-    TRY(gemm<T>(h, EPI_STORE, h->y, d, w.cq_w, w.cq_b, d, d, cnt, rows_ub, h->q, d, nullptr, st));
+    const LnSpec lc{x, w.lnc_g, w.lnc_b};
+    TRY(gemm<T>(h, EPI_STORE, h->y, d, w.cq_w, w.cq_b, d, d, cnt, rows_ub, h->q, d, nullptr, st, nullptr, nullptr, nullptr,
+                nullptr, &lc));
     TRY(attn<T>(h, false, h->q, d, nullptr, m.ckv[layer], (char*)m.ckv[layer] + (size_t)d * e, 2 * d, r.kv_off_cross,
                 r, r.nk_cross, cnt, rows_ub, q_ub, h->att, d, H, dh, h->S_max, st));
     TRY(gemm<T>(h, EPI_RESID, h->att, d, w.co_w, w.co_b, d, d, cnt, rows_ub, nullptr, 0, x, st));
@@ -442,8 +508,9 @@ int block_cross(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, c
 template <typename T>
 int block_ffn(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, int cnt, int rows_ub, cudaStream_t st) {
     const int d = m.dm.d_model, f = m.dm.d_ffn;
-    TRY(ln<T>(h, x, w.ln2_g, w.ln2_b, cnt, rows_ub, h->y, d, st));
-    TRY(gemm<T>(h, EPI_RELU, h->y, d, w.w1, w.b1, f, d, cnt, rows_ub, h->hbuf, f, nullptr, st));
+    const LnSpec l2{x, w.ln2_g, w.ln2_b};
+    TRY(gemm<T>(h, EPI_RELU, h->y, d, w.w1, w.b1, f, d, cnt, rows_ub, h->hbuf, f, nullptr, st, nullptr, nullptr, nullptr,
+                nullptr, &l2));
     TRY(gemm<T>(h, EPI_RESID, h->hbuf, f, w.w2, w.b2, d, f, cnt, rows_ub, nullptr, 0, x, st));
     return 0;
 }
@@ -511,8 +578,9 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
     }
     // last layer: K/V from every row, queries and everything after them from the k mask rows only
     const LayerW& w = m.dec[L - 1];
-    TRY(ln<T>(h, h->x, w.ln1_g, w.ln1_b, CNT_DRAFT_ALL, R1, h->y, d, st));
-    TRY(gemm<T>(h, EPI_STORE, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, CNT_DRAFT_ALL, R1, h->qkv, 3 * d, nullptr, st));
+    const LnSpec l1{h->x, w.ln1_g, w.ln1_b};
+    TRY(gemm<T>(h, EPI_STORE, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, CNT_DRAFT_ALL, R1, h->qkv, 3 * d, nullptr, st, nullptr,
+                nullptr, nullptr, nullptr, &l1));
     k_gather_rows<<<R2, 128, 0, st>>>(h->x, h->mrows.src_row, h->ses.counters + CNT_DRAFT_MASK, h->x2, d);
     KCHECK(h);
     TRY(attn<T>(h, false, h->qkv, 3 * d, h->mrows.src_row, (char*)h->qkv + (size_t)d * e,
@@ -565,8 +633,8 @@ int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float ta
     TRY(gemm<T>(h, EPI_STATS, h->y, d, m.embed, nullptr, m.dm.vocab, d, CNT_VERIFY, M, nullptr, 0, nullptr, st, h->ld,
                 h->ld_id, &n_tiles));
     prof_mark(h, st);
-    k_accept<<<B, 256, (size_t)(k + 1) * sizeof(RowPart), st>>>(h->part, n_tiles, h->ld, h->ld_id, k, beta, tau,
-                                                                h->accepted, h->bif, h->row_stats);
+    k_accept<<<B, 1024, (size_t)(k + 1) * sizeof(RowPart), st>>>(h->part, n_tiles, h->ld, h->ld_id, k, beta, tau,
+                                                                 h->accepted, h->bif, h->row_stats, h->want_lse);
     KCHECK(h);
     if (d_accepted) CUDA_TRY(h, cudaMemcpyAsync(d_accepted, h->accepted, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
     if (d_bif) CUDA_TRY(h, cudaMemcpyAsync(d_bif, h->bif, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
@@ -612,7 +680,7 @@ void drop_graphs(specdec_handle* h) {
 // replayed afterwards.  The key must name everything the launches depend on besides device memory.
 template <typename F>
 int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body) {
-    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->script_on ? 1 : 0);
+    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->script_on ? 1 : 0);
     key.push_back(h->B); key.push_back(h->S_max);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
@@ -835,6 +903,17 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
             cudaGetLastError();
             h->attn_tc_smem_cap = 48 * 1024;
         }
+        {
+            const int kmax = std::max(h->d_max, h->f_max);
+            size_t need = std::min<size_t>(skinny_smem(4, kmax), 227 * 1024);
+            if (skinny_smem(2, kmax) > need) need = std::min<size_t>(skinny_smem(2, kmax), 227 * 1024);
+            cudaError_t e = skinny_attr_mt<EPI_STORE>((int)need);
+            if (e == cudaSuccess) e = skinny_attr_mt<EPI_RELU>((int)need);
+            if (e == cudaSuccess) e = skinny_attr_mt<EPI_RESID>((int)need);
+            if (e == cudaSuccess) e = skinny_attr_mt<EPI_QKV>((int)need);
+            if (e != cudaSuccess) { cudaGetLastError(); need = 48 * 1024; }
+            h->skinny_smem_cap = need;
+        }
         if (sd::tc_init(h->tma, h->ses.counters + 7) != 0) h->use_tc = 0;     // reported through specdec_last_error; SIMT GEMM still runs on the GPU
         if (!h->use_tc) h->err = "tensor-core GEMM unavailable: " + h->tma.err;
     } else {
@@ -870,6 +949,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         h->use_tc = value ? 1 : 0;
         return SPECDEC_OK;
     }
+    if (!strcmp(name, "skinny")) { h->use_skinny = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "row_lse")) { h->want_lse = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "attn")) { h->use_tc_attn = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "graphs")) { h->use_graphs = value ? 1 : 0; return SPECDEC_OK; }
@@ -1073,7 +1153,7 @@ int specdec_accept_scan_static(const float* d_logits, const int32_t* d_draft, in
     // every slot the second stage reads is rewritten by the first, so nothing has to start at zero
     k_logit_tile_stats<<<dim3(n_tiles, (unsigned)rows), 256, 0, st>>>(d_logits, d_draft, k, V, NA_TILE, n_tiles, part, ld, ld_id);
     k_accept<<<B, 256, (size_t)(k + 1) * sizeof(RowPart), st>>>(part, n_tiles, ld, ld_id, k, beta, tau, d_accepted, d_bif,
-                                                                nullptr);
+                                                                nullptr, 0);
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(nullptr, SPECDEC_ERR_CUDA, std::string("accept_scan_static: ") + cudaGetErrorString(e));
     return SPECDEC_OK;

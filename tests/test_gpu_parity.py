@@ -249,6 +249,38 @@ def test_bf16_mid_lockstep(gemm, attn):
     sd.close()
 
 
+@pytest.mark.parametrize("nseq,skinny", [(2, 1), (4, 1), (2, 0)])
+def test_bf16_mid_small_batches_weight_streaming_gemm(nseq, skinny):
+    """Passes of at most 64 rows run the weight-streaming GEMM with fused LayerNorm (26 rows: two 16-row
+    tiles; 52 rows: four)."""
+    wv, wd = W.make_weights(MID_V, 21, True), W.make_weights(MID_D, 22, True)
+    mv, md = O.model_from(MID_V, wv, mode="bf16"), O.model_from(MID_D, wd, mode="bf16")
+    rng = np.random.default_rng(8)
+    srcs = [W.zipf_ids(rng, n, 2000) for n in (20, 7, 33, 12)][:nseq]
+    sd = _handle(MID_V, wv, MID_D, wd, True, k_max=12, max_batch=4, max_src=40, max_tgt=24)
+    sd.set_option("skinny", skinny)
+    rep = lockstep.run(sd, mv, md, srcs, [24, 18, 9, 20][:nseq], 12, 3, 1.0, margin=1e-3, check_logits_every=2)
+    print(rep.iterations, rep.draft_near_ties, rep.verify_near_ties, rep.max_logit_err, rep.max_stat_err)
+    assert rep.ok, rep.notes
+    assert rep.max_logit_err < 2e-2 and rep.max_stat_err < 2e-2
+    sd.close()
+
+
+def test_base_shapes_batch1_lockstep():
+    """One config-2 sentence at batch 1 (26-row verify block, K up to 2048 in the weight-streaming GEMM)."""
+    wl = W.config2_translation(1)
+    wv = W.make_weights(wl.verifier, wl.seed_verifier, True)
+    wd = W.make_weights(wl.drafter, wl.seed_drafter, True)
+    mv, md = O.model_from(wl.verifier, wv, mode="bf16"), O.model_from(wl.drafter, wd, mode="bf16")
+    sd = _handle(wl.verifier, wv, wl.drafter, wd, True, k_max=25, max_batch=1, max_src=40, max_tgt=64)
+    rep = lockstep.run(sd, mv, md, wl.src, wl.max_tgt, 25, 3, 1.0, margin=1e-3, check_logits_every=4, max_iters=8)
+    print(rep.iterations, rep.draft_positions, rep.draft_near_ties, rep.verify_rows, rep.verify_near_ties,
+          rep.max_logit_err, rep.max_stat_err, rep.notes[:5])
+    assert rep.ok, rep.notes
+    assert rep.max_logit_err < 2e-2 and rep.max_stat_err < 2e-2
+    sd.close()
+
+
 def test_base_shapes_bf16_lockstep_and_pure_tolerance():
     """Transformer-base shapes (config 2 recipe), a few sentences: lock-step against the oracle with bf16
     operand rounding, and logits against the pure-fp32 oracle within 2e-2 abs / 1e-2 rel."""
