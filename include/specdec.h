@@ -198,6 +198,7 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
 
 /* Options: "gemm" = 0 SIMT reference GEMM, 1 tcgen05 GEMM (bf16 handles; default 1);
  * "skinny" = 0/1 weight-streaming GEMM with fused LayerNorm for passes of at most 64 rows (bf16; default 1);
+ * "pdl" = 0/1 programmatic dependent launch between the kernels of a step (default 1);
  * "attn" = 0 warp-per-row reference attention, 1 tensor-core tile attention (bf16, 64-wide heads; default 1);
  * "graphs" = 0/1 replay draft/verify steps from CUDA graphs inside specdec_generate;
  * "profile" = 0/1 (see specdec_profile_read); "row_lse" = 0/1 also accumulate the log-sum-exp of

@@ -58,6 +58,8 @@ __global__ void __launch_bounds__(128) k_attn_tc(AttnTcArgs a) {
     __shared__ float s_sum[ATT_Q];
     __shared__ int s_nkmax;
     const int b = blockIdx.z, h = blockIdx.y, qt = blockIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();                                   // everything this kernel reads was written by its predecessors
     const int cnt = a.q_cnt[b];
     if (qt * ATT_Q >= cnt) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;

@@ -21,6 +21,13 @@ template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __flo
 // value as the operand type would hold it, back in fp32
 template <typename T> __device__ __forceinline__ float round_as(float v) { return to_f(from_f<T>(v)); }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start
+// while its predecessor is still running.  pdl_wait() blocks until the predecessor grids have completed
+// and their writes are visible; everything a kernel does before it must not depend on them (weights and
+// constants only) and must not write global memory.  Without the attribute both are no-ops.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));

@@ -35,7 +35,6 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
     extern __shared__ __align__(16) unsigned char sk_sm[];
     const GemmArgs<bf16>& g = a.g;
     const int K = g.K, N = g.N;
-    const int R = min(*g.n_rows, MT * 16);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t4 = lane & 3;
     const int n0 = blockIdx.x * SK_NB;
     const int pitch = K + 8;                                  // bf16 elements per activation row in shared memory
@@ -56,33 +55,58 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
         wreg[ss] = (w_ok && warp < nsplit && k0 < k_end) ? __ldg(reinterpret_cast<const uint4*>(wrow + k0)) : make_uint4(0, 0, 0, 0);
     }
 
+    // everything above touched only weights; from here on the predecessor's output is read
+    pdl_launch_dependents();
+    pdl_wait();
+    const int R = min(*g.n_rows, MT * 16);      // the live row count is itself written earlier in the step
     // ---- activation rows into shared memory
     if (LN) {
-        for (int m = warp; m < MT * 16; m += SK_WARPS) {
+        // each warp normalises rows warp, warp + 8, ...; all of its rows are fetched first (one round trip)
+        constexpr int RS = (MT * 16 + SK_WARPS - 1) / SK_WARPS;      // row slots per warp
+        constexpr int CH = 4;                                        // float4 chunks per lane and row: K <= 512
+        float4 xv[RS][CH];
+#pragma unroll
+        for (int s = 0; s < RS; ++s) {
+            const int m = warp + s * SK_WARPS;
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                const int e = lane * 4 + c * 128;
+                xv[s][c] = (m < R && e < K) ? *reinterpret_cast<const float4*>(a.ln_x + (size_t)m * K + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+#pragma unroll
+        for (int s = 0; s < RS; ++s) {
+            const int m = warp + s * SK_WARPS;
+            if (m >= MT * 16) continue;
             bf16* dst = As + (size_t)m * pitch;
             if (m < R) {
-                const float* xr = a.ln_x + (size_t)m * K;
-                float s = 0.f;
-                for (int e = lane * 4; e < K; e += 128) { const float4 v = *reinterpret_cast<const float4*>(xr + e); s += v.x + v.y + v.z + v.w; }
-                const float mu = warp_sum(s) / K;
+                float sum = 0.f;
+#pragma unroll
+                for (int c = 0; c < CH; ++c) sum += xv[s][c].x + xv[s][c].y + xv[s][c].z + xv[s][c].w;   // chunks past K are zero
+                const float mu = warp_sum(sum) / K;
                 float q = 0.f;
-                for (int e = lane * 4; e < K; e += 128) {
-                    const float4 v = *reinterpret_cast<const float4*>(xr + e);
-                    const float c0 = v.x - mu, c1 = v.y - mu, c2 = v.z - mu, c3 = v.w - mu;
-                    q += c0 * c0 + c1 * c1 + c2 * c2 + c3 * c3;
-                }
+#pragma unroll
+                for (int c = 0; c < CH; ++c)
+                    if (lane * 4 + c * 128 < K) {
+                        const float c0 = xv[s][c].x - mu, c1 = xv[s][c].y - mu, c2 = xv[s][c].z - mu, c3 = xv[s][c].w - mu;
+                        q += c0 * c0 + c1 * c1 + c2 * c2 + c3 * c3;
+                    }
                 const float rstd = 1.0f / sqrtf(warp_sum(q) / K + a.ln_eps);
-                for (int e = lane * 4; e < K; e += 128) {
-                    const float4 v = *reinterpret_cast<const float4*>(xr + e);
-                    const float4 gm = *reinterpret_cast<const float4*>(a.ln_g + e), bt = *reinterpret_cast<const float4*>(a.ln_b + e);
-                    __nv_bfloat162 p0, p1;
-                    p0.x = __float2bfloat16_rn((v.x - mu) * rstd * gm.x + bt.x); p0.y = __float2bfloat16_rn((v.y - mu) * rstd * gm.y + bt.y);
-                    p1.x = __float2bfloat16_rn((v.z - mu) * rstd * gm.z + bt.z); p1.y = __float2bfloat16_rn((v.w - mu) * rstd * gm.w + bt.w);
-                    *reinterpret_cast<__nv_bfloat162*>(dst + e) = p0;
-                    *reinterpret_cast<__nv_bfloat162*>(dst + e + 2) = p1;
-                    if (a.ln_out && blockIdx.x == 0) {
-                        *reinterpret_cast<__nv_bfloat162*>(a.ln_out + (size_t)m * K + e) = p0;
-                        *reinterpret_cast<__nv_bfloat162*>(a.ln_out + (size_t)m * K + e + 2) = p1;
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    const int e = lane * 4 + c * 128;
+                    if (e < K) {
+                        const float4 v = xv[s][c];
+                        const float4 gm = *reinterpret_cast<const float4*>(a.ln_g + e), bt = *reinterpret_cast<const float4*>(a.ln_b + e);
+                        __nv_bfloat162 p0, p1;
+                        p0.x = __float2bfloat16_rn((v.x - mu) * rstd * gm.x + bt.x); p0.y = __float2bfloat16_rn((v.y - mu) * rstd * gm.y + bt.y);
+                        p1.x = __float2bfloat16_rn((v.z - mu) * rstd * gm.z + bt.z); p1.y = __float2bfloat16_rn((v.w - mu) * rstd * gm.w + bt.w);
+                        *reinterpret_cast<__nv_bfloat162*>(dst + e) = p0;
+                        *reinterpret_cast<__nv_bfloat162*>(dst + e + 2) = p1;
+                        if (a.ln_out && blockIdx.x == 0) {
+                            *reinterpret_cast<__nv_bfloat162*>(a.ln_out + (size_t)m * K + e) = p0;
+                            *reinterpret_cast<__nv_bfloat162*>(a.ln_out + (size_t)m * K + e + 2) = p1;
+                        }
                     }
                 }
             } else {

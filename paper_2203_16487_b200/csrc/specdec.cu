@@ -80,7 +80,7 @@ struct specdec_handle {
     bool encoded = false, verified = false, drafted = false;
     int last_draft_rows_ub = 0;
     // options
-    int use_tc = 1, use_graphs = 1, use_tc_attn = 1, want_lse = 0, use_skinny = 1;
+    int use_tc = 1, use_graphs = 1, use_tc_attn = 1, want_lse = 0, use_skinny = 1, use_pdl = 1;
     size_t skinny_smem_cap = 0;
     // CUDA graphs of whole draft / verify(+commit) steps, keyed by everything their launches depend on
     struct GraphEntry { cudaGraphExec_t exec; long long kernels; };
@@ -307,16 +307,31 @@ template <typename T>
 bool skinny_ok(const specdec_handle* h, int epi, int rows_ub, int N, int K, bool with_ln) {
     if (!std::is_same<T, bf16>::value || !h->use_skinny || rows_ub > 64) return false;
     if (epi != EPI_STORE && epi != EPI_RELU && epi != EPI_RESID && epi != EPI_QKV) return false;
-    if (K % 32 || (with_ln && K % 128)) return false;
+    if (K % 32 || (with_ln && (K % 128 || K > 512))) return false;
     return skinny_smem(rows_ub <= 32 ? 2 : 4, K) <= h->skinny_smem_cap;
+}
+
+// Launch that lets the kernel start before its predecessor in the stream has finished (the kernel itself
+// calls pdl_wait() before it touches anything the predecessor wrote).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(specdec_handle* h, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                       Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = h->use_pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
 template <int EPI, int MT>
 int skinny_launch_ln(specdec_handle* h, SkinnyArgs& a, cudaStream_t st) {
     const int grid = cdiv(a.g.N, SK_NB);
     const size_t smem = skinny_smem(MT, a.g.K);
-    if (a.ln_x) k_skinny<EPI, MT, true><<<grid, SK_WARPS * 32, smem, st>>>(a);
-    else k_skinny<EPI, MT, false><<<grid, SK_WARPS * 32, smem, st>>>(a);
+    cudaError_t e = a.ln_x ? launch_pdl(h, k_skinny<EPI, MT, true>, dim3(grid), dim3(SK_WARPS * 32), smem, st, a)
+                           : launch_pdl(h, k_skinny<EPI, MT, false>, dim3(grid), dim3(SK_WARPS * 32), smem, st, a);
+    if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("skinny GEMM launch: ") + cudaGetErrorString(e));
     KCHECK(h);
     return 0;
 }
@@ -413,8 +428,9 @@ int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* 
             a.out = (bf16*)out; a.out_stride = out_stride; a.max_keys = max_keys;
             a.scale = 1.0f / sqrtf((float)d_head);
             dim3 grid(cdiv(q_ub, ATT_Q), n_heads, h->B);
-            if (paged) k_attn_tc<true><<<grid, 128, smem, st>>>(a);
-            else k_attn_tc<false><<<grid, 128, smem, st>>>(a);
+            cudaError_t e = paged ? launch_pdl(h, k_attn_tc<true>, grid, dim3(128), smem, st, a)
+                                  : launch_pdl(h, k_attn_tc<false>, grid, dim3(128), smem, st, a);
+            if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(e));
             KCHECK(h);
             return 0;
         }
@@ -680,7 +696,7 @@ void drop_graphs(specdec_handle* h) {
 // replayed afterwards.  The key must name everything the launches depend on besides device memory.
 template <typename F>
 int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body) {
-    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->script_on ? 1 : 0);
+    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->script_on ? 1 : 0);
     key.push_back(h->B); key.push_back(h->S_max);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
@@ -949,6 +965,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         h->use_tc = value ? 1 : 0;
         return SPECDEC_OK;
     }
+    if (!strcmp(name, "pdl")) { h->use_pdl = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "skinny")) { h->use_skinny = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "row_lse")) { h->want_lse = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "attn")) { h->use_tc_attn = value ? 1 : 0; return SPECDEC_OK; }
