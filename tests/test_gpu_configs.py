@@ -1,0 +1,128 @@
+"""GPU parity at the full sizes of the workload recipes (configs 3, 4, 5), on sampled outputs.
+
+The oracle cannot follow 128 sequences for a hundred iterations inside a test, so at full size the
+CUDA path runs the whole batch and a few sampled sequences are compared with the oracle's batch-1
+result; lock-step checks cover every decision on a few sequences.  Tolerances as in
+test_gpu_parity.py (bf16 handles: decisions bit-exact outside 1e-3 margins).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import specdec_oracle as O
+from paper_2203_16487_b200 import workloads as W
+from tests import lockstep
+
+pytestmark = pytest.mark.gpu
+BOS, EOS, MASK = W.BOS_ID, W.EOS_ID, W.MASK_ID
+
+
+@pytest.fixture(scope="module")
+def base():
+    from paper_2203_16487_b200 import binding
+    wv = W.make_weights(W.BASE_V, 1001, True)
+    wd = W.make_weights(W.BASE_D, 1002, True)
+    mv, md = O.model_from(W.BASE_V, wv, mode="bf16"), O.model_from(W.BASE_D, wd, mode="bf16")
+    return binding, wv, wd, mv, md
+
+
+def _prefix_match(a, b):
+    n = 0
+    for x, y in zip(a, b):
+        if x != y:
+            break
+        n += 1
+    return n
+
+
+@pytest.mark.parametrize("batch,beta,tau", [(32, 1, 0.0), (32, 5, 3.0), (128, 3, 1.0)])
+def test_config3_batched_generate_sampled_sequences(base, batch, beta, tau):
+    binding, wv, wd, mv, md = base
+    wl = W.config3_batched(batch, beta, tau)
+    smax, tmax = max(len(s) for s in wl.src), max(wl.max_tgt)
+    sd = binding.SpecDec(W.BASE_V, wv, W.BASE_D, wd, k_max=25, max_batch=batch, max_src=smax, max_tgt=tmax, bf16=True)
+    src, lens = W.pad_batch(wl.src)
+    out, n, st = sd.generate(src, lens, wl.max_tgt, 25, beta, tau)
+    out, n = out.cpu().numpy(), n.cpu().numpy()
+    assert st["emitted"] == int(n.sum()) and (n <= np.array(wl.max_tgt)).all() and (n >= 1).all()
+    assert st["iterations"] <= tmax and st["seq_iterations"] <= st["emitted"]      # >= 1 token per sequence-iteration
+    # sampled sequences against the oracle's batch-1 run (shortest, longest and one in between)
+    order = np.argsort([len(s) for s in wl.src])
+    for b in (int(order[0]), int(order[len(order) // 2]), int(order[-1])):
+        mt = min(wl.max_tgt[b], 24)                     # bounded oracle work; prefixes must agree
+        ref, _ = O.specdec_generate(mv, md, wl.src[b], mt, 25, beta, tau, BOS, EOS, MASK)
+        got = out[b, :n[b]].tolist()[:mt]
+        assert got == ref, (b, _prefix_match(got, ref), got[:8], ref[:8])
+    # batch invariance on the device: the same sequences decoded alone
+    for b in (int(order[1]), int(order[-2])):
+        o1, n1, _ = sd.generate(wl.src[b][None], [len(wl.src[b])], [wl.max_tgt[b]], 25, beta, tau)
+        assert o1[0, :int(n1[0])].cpu().tolist() == out[b, :n[b]].tolist()
+    sd.close()
+
+
+def test_config4_long_sources(base):
+    binding, wv, wd, mv, md = base
+    wl = W.config4_summarization()
+    smax = max(len(s) for s in wl.src)
+    sd = binding.SpecDec(W.BASE_V, wv, W.BASE_D, wd, k_max=25, max_batch=8, max_src=smax, max_tgt=128, bf16=True)
+    # every decision of two long-source sequences for a few iterations (cross-attention over 300-512 keys)
+    rep = lockstep.run(sd, mv, md, wl.src[:2], [128, 128], 25, 3, 1.0, margin=1e-3, check_logits_every=2, max_iters=3)
+    print(rep.iterations, rep.draft_near_ties, rep.verify_near_ties, rep.max_logit_err, rep.max_stat_err, rep.notes[:3])
+    assert rep.ok, rep.notes
+    assert rep.max_logit_err < 2e-2
+    # the whole batch of 8, full length; one sampled sequence against the oracle
+    src, lens = W.pad_batch(wl.src)
+    out, n, st = sd.generate(src, lens, wl.max_tgt, 25, 3, 1.0)
+    assert n.cpu().tolist() == [128] * 8 or st["emitted"] == int(n.sum())
+    ref, _ = O.specdec_generate(mv, md, wl.src[3], 12, 25, 3, 1.0, BOS, EOS, MASK)
+    assert out[3, :12].cpu().tolist() == ref
+    sd.close()
+
+
+@pytest.mark.parametrize("k,prefix", [(5, 64), (50, 64), (25, 256), (10, 0)])
+def test_config5_verify_step_with_scripted_rejections(base, k, prefix):
+    """Drafts = the oracle verifier's greedy continuation with one substitution at position r ~ Geometric(mean 6):
+    the accepted length must be min(r - 1, k) and the bifurcation token the oracle's top-1 there."""
+    binding, wv, wd, mv, md = base
+    B, S = 2, 64
+    wl = W.config5_microbench(B, S)
+    prefixes, rej = W.config5_prefix_and_rejections(B, prefix)
+    sd = binding.SpecDec(W.BASE_V, wv, W.BASE_D, wd, k_max=50, max_batch=B, max_src=S, max_tgt=prefix + 52, bf16=True)
+    src, lens = W.pad_batch(wl.src)
+    sd.encode(src, lens, None)
+    done = 0
+    pre = np.stack(prefixes) if prefix else np.zeros((B, 0), np.int32)
+    kb = 25
+    while done < prefix:                                  # build the prefix through verify + commit(keep, next)
+        c = min(kb, prefix - done - 1)
+        block = np.zeros((B, kb), np.int32); block[:, :c] = pre[:, done:done + c]
+        sd.verify(block, 1, 0.0)
+        sd.commit(np.full(B, c, np.int32), pre[:, done + c])
+        done += c + 1
+    drafts = np.zeros((B, k), np.int32)
+    expect = []
+    for b in range(B):
+        mem = O.encode(mv, wl.src[b])
+        cache = O.new_cache(mv, mem)
+        committed = pre[b].tolist()
+        if committed:
+            O.decoder_rows(mv, [BOS] + committed[:-1], mem, True, cache)
+        g = []
+        for _ in range(k):                                # oracle greedy continuation, one token at a time
+            row = O.decoder_rows(mv, [(committed + g)[-1] if committed + g else BOS], mem, True, cache)[-1]
+            g.append(int(np.argmax(row)))
+        d = list(g)
+        r = int(rej[b])
+        cache.truncate(len(committed))
+        if r <= k:
+            rows = O.verify_rows(mv, mem, committed, g, BOS, cache)
+            cache.truncate(len(committed))
+            d[r - 1] = int(np.argmin(rows[r - 1]))       # the lowest-logit token: rejected under every beta < V
+        drafts[b] = d
+        rows = O.verify_rows(mv, mem, committed, d, BOS, cache)
+        a, t = O.verify(rows, d, 3, 1.0)
+        assert a == min(r - 1, k)
+        expect.append((a, t))
+    acc, bif = sd.verify(drafts, 3, 1.0)
+    assert list(zip(acc.cpu().tolist(), bif.cpu().tolist())) == expect
+    sd.close()
