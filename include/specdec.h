@@ -184,6 +184,9 @@ int specdec_accept_scan_static(const float* d_logits, const int32_t* d_draft, in
  *   the draft's logit (+inf on the bonus row), draft id (-1 on the bonus row). */
 int specdec_debug_logits(specdec_handle* h, int which, float* d_logits, void* stream);
 int specdec_debug_row_stats(specdec_handle* h, float* d_stats, void* stream);
+/* With option "cl_trace" = 1 the cluster decoder kernel records a nanosecond timestamp after each of its
+ * phases (first CTA only); this copies the first n (<= 256) of them to the host.  Synchronises the device. */
+int specdec_debug_cluster_trace(specdec_handle* h, long long* h_out, int n);
 
 /* Scripted drafts, a benchmark / test hook with no counterpart in the paper: random-init
  * models almost never agree, so a workload's acceptance pattern is imposed instead.  After the
@@ -198,6 +201,9 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
 
 /* Options: "gemm" = 0 SIMT reference GEMM, 1 tcgen05 GEMM (bf16 handles; default 1);
  * "skinny" = 0/1 weight-streaming GEMM with fused LayerNorm for passes of at most 64 rows (bf16; default 1);
+ * "cluster" = 0/1 run the verifier's decoder stack as one thread-block-cluster kernel per sequence when the
+ *   batch is at most 8, k + 1 <= 32 and the model has 8 heads of 64 (default 0: measured slower than the
+ *   per-operation kernels, kept for comparison);
  * "pdl" = 0/1 programmatic dependent launch between the kernels of a step (default 1);
  * "attn" = 0 warp-per-row reference attention, 1 tensor-core tile attention (bf16, 64-wide heads; default 1);
  * "graphs" = 0/1 replay draft/verify steps from CUDA graphs inside specdec_generate;

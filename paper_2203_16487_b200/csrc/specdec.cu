@@ -15,6 +15,7 @@
 
 #include "../../include/specdec.h"
 #include "attention_tc.cuh"
+#include "decoder_cluster.cuh"
 #include "gemm_tc.cuh"
 #include "kernels.cuh"
 #include "skinny_gemm.cuh"
@@ -80,7 +81,13 @@ struct specdec_handle {
     bool encoded = false, verified = false, drafted = false;
     int last_draft_rows_ub = 0;
     // options
-    int use_tc = 1, use_graphs = 1, use_tc_attn = 1, want_lse = 0, use_skinny = 1, use_pdl = 1;
+    int use_tc = 1, use_graphs = 1, use_tc_attn = 1, want_lse = 0, use_skinny = 1, use_pdl = 1, use_cluster = 0;
+    // packed weight stream of the cluster decoder kernel (verifier, small batches)
+    unsigned char* cl_stream = nullptr;
+    size_t cl_cta_stride = 0;
+    bool cl_ok = false;
+    long long* cl_trace = nullptr;   // device [256] timestamps of the cluster kernel's phases (option "cl_trace")
+    int want_cl_trace = 0;
     size_t skinny_smem_cap = 0;
     // CUDA graphs of whole draft / verify(+commit) steps, keyed by everything their launches depend on
     struct GraphEntry { cudaGraphExec_t exec; long long kernels; };
@@ -165,6 +172,13 @@ void layout_model(specdec_handle* h, ModelW& m, const specdec_model_dims& dm) {
     for (auto& p : m.ckv) p = A.take((size_t)h->B_cap * h->S_cap * 2 * d * e);
 }
 
+// The cluster decoder kernel needs one CTA per head of 64 columns and operand rows that fit its shared memory.
+bool cl_eligible(const specdec_config& c) {
+    const specdec_model_dims& v = c.verifier;
+    return c.compute_dtype == SPECDEC_DTYPE_BF16 && v.n_heads == CL_C && v.d_model == CL_C * 64 && v.d_model <= 512 &&
+           v.d_ffn % (CL_C * 64) == 0 && v.d_ffn <= 2048 && v.dec_layers <= CL_MAX_LAYERS;
+}
+
 void layout_rows(Arena& A, Rows& r, int n, int B) {
     auto iv = [&](size_t c) { return (int*)A.take(c * 4); };
     r.tok = iv(n); r.pos = iv(n); r.seq = iv(n); r.nk_self = iv(n); r.nk_cross = iv(n);
@@ -208,6 +222,12 @@ void layout_all(specdec_handle* h) {
     h->stage_len = (int*)A.take((size_t)h->B_cap * 4);
     h->stage_mt = (int*)A.take((size_t)h->B_cap * 4);
     h->script = (int*)A.take((size_t)h->B_cap * (h->T_cap + h->k_cap) * 4);
+    if (cl_eligible(h->cfg)) {
+        const specdec_model_dims& v = h->cfg.verifier;
+        h->cl_cta_stride = (size_t)v.dec_layers * cl_stages_per_layer(v.d_model, v.d_ffn) * CL_STAGE;
+        h->cl_stream = (unsigned char*)A.take(h->cl_cta_stride * CL_C);
+        h->cl_trace = (long long*)A.take(256 * 8);
+    }
     Session& s = h->ses;
     s.len = (int*)A.take((size_t)h->B_cap * 4);
     s.finished = (int*)A.take((size_t)h->B_cap * 4);
@@ -635,7 +655,38 @@ int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float ta
     k_verify_prep<<<cdiv(M, 256), 256, 0, st>>>(h->ses, h->v_draft, B, k, h->S_max, h->cfg.bos_id, h->rows);
     KCHECK(h);
     TRY(embed<T>(h, m, h->rows, m.pos_dec, CNT_VERIFY, M, st));
-    for (int l = 0; l < L; ++l) {
+    bool clustered = false;
+    if constexpr (std::is_same<T, bf16>::value) {
+        const int cap = cl_max_keys(m.dm.d_ffn);
+        if (h->cl_ok && h->use_cluster && B <= 8 && k + 1 <= CL_M && max_keys <= cap && h->S_max <= cap) {
+            // the whole decoder stack in one kernel: one cluster of 8 CTAs per sequence
+            ClArgs ca;
+            ca.wstream = h->cl_stream; ca.cta_stride = h->cl_cta_stride; ca.n_layers = L;
+            for (int l = 0; l < L; ++l) {
+                const LayerW& w = m.dec[l];
+                ca.layer[l] = ClLayer{w.ln1_g, w.ln1_b, w.lnc_g, w.lnc_b, w.ln2_g, w.ln2_b, w.qkv_b, w.o_b, w.cq_b, w.co_b, w.b1, w.b2,
+                                      (bf16*)h->kc[l], (bf16*)h->vc[l], (const bf16*)m.ckv[l]};
+            }
+            ca.x = h->x; ca.att = (bf16*)h->att; ca.hbuf = (bf16*)h->hbuf;
+            ca.len = h->ses.len; ca.src_len = h->ses.src_len;
+            ca.pg.table = h->page_table; ca.pg.page_tokens = h->cfg.page_tokens; ca.pg.max_pages = h->pages_per_seq;
+            ca.S_max = h->S_max; ca.k1 = k + 1; ca.d = d; ca.F = m.dm.d_ffn; ca.max_keys = cap; ca.err_word = h->ses.counters + 7;
+            ca.trace = h->want_cl_trace ? h->cl_trace : nullptr;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(B * CL_C); cfg.blockDim = dim3(CL_THREADS); cfg.dynamicSmemBytes = cl_smem_bytes(m.dm.d_ffn); cfg.stream = st;
+            cudaLaunchAttribute attr[2];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = CL_C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[1].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr; cfg.numAttrs = h->use_pdl ? 2 : 1;
+            cudaError_t e = cudaLaunchKernelEx(&cfg, k_decoder_cluster, ca);
+            if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("cluster decoder launch: ") + cudaGetErrorString(e));
+            KCHECK(h);
+            clustered = true;
+        }
+    }
+    for (int l = 0; l < L && !clustered; ++l) {
         TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, k + 1, l, true, max_keys, st));
         TRY(block_cross<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, k + 1, l, st));
         TRY(block_ffn<T>(h, m, m.dec[l], h->x, CNT_VERIFY, M, st));
@@ -696,7 +747,7 @@ void drop_graphs(specdec_handle* h) {
 // replayed afterwards.  The key must name everything the launches depend on besides device memory.
 template <typename F>
 int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body) {
-    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->script_on ? 1 : 0);
+    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
     key.push_back(h->B); key.push_back(h->S_max);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
@@ -930,6 +981,21 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
             if (e != cudaSuccess) { cudaGetLastError(); need = 48 * 1024; }
             h->skinny_smem_cap = need;
         }
+        if (h->cl_stream) {
+            const specdec_model_dims& v = cfg->verifier;
+            const int spl = cl_stages_per_layer(v.d_model, v.d_ffn);
+            for (int l = 0; l < v.dec_layers; ++l) {
+                const LayerW& w = h->ver.dec[l];
+                ClPackSrc ps{(const bf16*)w.qkv_w, (const bf16*)w.o_w, (const bf16*)w.cq_w, (const bf16*)w.co_w, (const bf16*)w.w1, (const bf16*)w.w2};
+                k_cl_pack<<<1024, 256, 0, st>>>(ps, l, v.d_model, v.d_ffn, (uint4*)h->cl_stream, h->cl_cta_stride / 16, spl);
+                ++h->launches;
+            }
+            cudaError_t e = cudaFuncSetAttribute(k_decoder_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cl_smem_bytes(v.d_ffn));
+            if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+            if (e == cudaSuccess) e = cudaGetLastError();
+            h->cl_ok = (e == cudaSuccess);
+            if (!h->cl_ok) cudaGetLastError();
+        }
         if (sd::tc_init(h->tma, h->ses.counters + 7) != 0) h->use_tc = 0;     // reported through specdec_last_error; SIMT GEMM still runs on the GPU
         if (!h->use_tc) h->err = "tensor-core GEMM unavailable: " + h->tma.err;
     } else {
@@ -965,6 +1031,8 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         h->use_tc = value ? 1 : 0;
         return SPECDEC_OK;
     }
+    if (!strcmp(name, "cl_trace")) { h->want_cl_trace = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "pdl")) { h->use_pdl = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "skinny")) { h->use_skinny = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "row_lse")) { h->want_lse = value ? 1 : 0; return SPECDEC_OK; }
@@ -1188,6 +1256,14 @@ int specdec_debug_logits(specdec_handle* h, int which, float* d_logits, void* st
     const int d = m->dm.d_model, V = m->dm.vocab;
     return DISPATCH(h, gemm<bf16>(h, EPI_F32, h->y, d, m->embed, nullptr, V, d, cnt, rows, nullptr, 0, d_logits, st),
                     gemm<float>(h, EPI_F32, h->y, d, m->embed, nullptr, V, d, cnt, rows, nullptr, 0, d_logits, st));
+}
+
+int specdec_debug_cluster_trace(specdec_handle* h, long long* h_out, int n) {
+    if (!h || !h_out || n < 1 || n > 256) return SPECDEC_ERR_INVALID_ARG;
+    if (!h->cl_trace) return fail(h, SPECDEC_ERR_UNSUPPORTED, "cluster decoder kernel not available for this model");
+    CUDA_TRY(h, cudaDeviceSynchronize());
+    CUDA_TRY(h, cudaMemcpy(h_out, h->cl_trace, (size_t)n * 8, cudaMemcpyDeviceToHost));
+    return SPECDEC_OK;
 }
 
 int specdec_debug_row_stats(specdec_handle* h, float* d_stats, void* stream) {

@@ -37,37 +37,17 @@ def algorithmic_work(B: int, k: int, j: int, S: int, dims: W.ModelDims):
     return params, bytes_, flops
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--batch", type=int, default=1)
-    ap.add_argument("--k", type=int, default=25)
-    ap.add_argument("--prefix", type=int, default=64)
-    ap.add_argument("--src-len", type=int, default=64)
-    ap.add_argument("--reps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--no-flush", action="store_true")
-    ap.add_argument("--draft", action="store_true")
-    ap.add_argument("--gemm", type=int, default=1)
-    ap.add_argument("--graphs", type=int, default=1)
-    args = ap.parse_args()
-    B, k, j, S = args.batch, args.k, args.prefix, args.src_len
-
-    wl = W.config5_microbench(B, S)
-    wv = W.make_weights(wl.verifier, wl.seed_verifier, True)
-    wd = W.make_weights(wl.drafter, wl.seed_drafter, True)
-    sd = binding.SpecDec(wl.verifier, wv, wl.drafter, wd, k_max=max(k, 1), max_batch=B, max_src=S,
-                         max_tgt=j + k + 2, bf16=True)
-    sd.set_option("gemm", args.gemm)
-    sd.set_option("graphs", args.graphs)
+def measure(sd, wl, B, k, j, S, reps, warmup, flush, draft=False):
+    """Builds a committed prefix of j tokens, a draft block with scripted rejections, and times the step."""
     src, lens = W.pad_batch(wl.src)
     sd.encode(src, lens, None)
     prefix, rej = W.config5_prefix_and_rejections(B, j)
     prefix = np.stack(prefix) if j > 0 else np.zeros((B, 0), np.int32)
-    # build the committed prefix: verify a block of prefix tokens, keep c of them plus the next one
+    kb = min(k, 25)
     done = 0
-    while done < j:
-        c = min(k, j - done - 1)
-        block = np.zeros((B, k), np.int32)
+    while done < j:            # verify a block of prefix tokens, keep c of them plus the next one
+        c = min(kb, j - done - 1)
+        block = np.zeros((B, kb), np.int32)
         block[:, :c] = prefix[:, done:done + c]
         sd.verify(block, 1, 0.0)
         sd.commit(np.full(B, c, np.int32), prefix[:, done + c])
@@ -76,7 +56,7 @@ def main():
     assert int(n.min()) == j and int(n.max()) == j
     # draft block: the verifier's greedy continuation from that prefix, one substitution per sequence
     drafts = np.zeros((B, k), np.int32)
-    for i in range(k + 1):        # greedy continuation one token at a time through the same entry points
+    for i in range(k + 1):
         acc, bif = sd.verify(drafts, 1, 0.0)
         a, t = acc.cpu().numpy(), bif.cpu().numpy()
         if int(a.min()) >= k:
@@ -92,36 +72,80 @@ def main():
     bif_t = torch.zeros(B, dtype=torch.int32, device="cuda")
     sd.verify_raw(d_drafts, 3, 1.0, acc_t, bif_t)
     mean_a = float(acc_t.float().mean())
-
-    flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
     times = []
-    for r in range(args.warmup + args.reps):
+    for r in range(warmup + reps):
         if flush is not None:
             flush.fill_(r & 0xff)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        if args.draft:
+        if draft:
             sd.draft(k)
         else:
             sd.verify_raw(d_drafts, 3, 1.0, acc_t, bif_t)
         e1.record()
         torch.cuda.synchronize()
-        if r >= args.warmup:
+        if r >= warmup:
             times.append(e0.elapsed_time(e1) * 1e3)
-    us = float(np.median(times))
-    params, bytes_, flops = algorithmic_work(B, k, j, S, wl.verifier)
-    peaks = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
-    hbm, tc, kind = 6650.0, 1590.0, "fallback"
-    if os.path.exists(peaks):
-        p = json.load(open(peaks)); hbm, tc, kind = p["hbm_gbs"], p["bf16_tflops"], "measured"
-    print(json.dumps({
-        "step": "draft" if args.draft else "verify", "batch": B, "k": k, "prefix": j, "src_len": S,
-        "us_median": us, "us_min": float(np.min(times)), "l2_flush": flush is not None, "mean_accepted": mean_a,
-        "algorithmic_MB": bytes_ / 1e6, "algorithmic_GFLOP": flops / 1e9,
-        "hbm_GBs": bytes_ / us / 1e3, "hbm_frac": bytes_ / us / 1e3 / hbm,
-        "tensor_TFLOPs": flops / us / 1e6, "tensor_frac": flops / us / 1e6 / tc, "peaks": kind,
-    }))
-    sd.close()
+    return float(np.median(times)), float(np.min(times)), mean_a
+
+
+def peaks():
+    p = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return d["hbm_gbs"], d["bf16_tflops"], "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--k", type=int, default=25)
+    ap.add_argument("--prefix", type=int, default=64)
+    ap.add_argument("--src-len", type=int, default=64)
+    ap.add_argument("--reps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--no-flush", action="store_true")
+    ap.add_argument("--draft", action="store_true")
+    ap.add_argument("--gemm", type=int, default=1)
+    ap.add_argument("--graphs", type=int, default=1)
+    ap.add_argument("--grid", action="store_true", help="the whole k x prefix x batch grid of the verify microbench")
+    args = ap.parse_args()
+    S = args.src_len
+    hbm, tc, kind = peaks()
+    flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    batches = [1, 8, 64, 128] if args.grid else [args.batch]
+    ks = [5, 10, 25, 50] if args.grid else [args.k]
+    prefixes = [0, 64, 256] if args.grid else [args.prefix]
+    if args.grid:
+        print(f"| B | k | prefix | us/step | MB | GFLOP | HBM GB/s | % of {kind} HBM | TFLOP/s | % of {kind} bf16 | mean accepted |")
+        print("|---|---|---|---|---|---|---|---|---|---|---|")
+    for B in batches:
+        wl = W.config5_microbench(B, S)
+        wv = W.make_weights(wl.verifier, wl.seed_verifier, True)
+        wd = W.make_weights(wl.drafter, wl.seed_drafter, True)
+        sd = binding.SpecDec(wl.verifier, wv, wl.drafter, wd, k_max=max(ks), max_batch=B, max_src=S,
+                             max_tgt=max(prefixes) + max(ks) + 2, bf16=True)
+        del wv, wd
+        sd.set_option("gemm", args.gemm)
+        sd.set_option("graphs", args.graphs)
+        for j in prefixes:
+            for k in ks:
+                us, us_min, mean_a = measure(sd, wl, B, k, j, S, args.reps, args.warmup, flush, args.draft)
+                params, bytes_, flops = algorithmic_work(B, k, j, S, wl.verifier)
+                if args.grid:
+                    print(f"| {B} | {k} | {j} | {us:.1f} | {bytes_ / 1e6:.1f} | {flops / 1e9:.2f} | {bytes_ / us / 1e3:.0f} | "
+                          f"{100 * bytes_ / us / 1e3 / hbm:.1f} | {flops / us / 1e6:.1f} | {100 * flops / us / 1e6 / tc:.1f} | {mean_a:.2f} |",
+                          flush=True)
+                else:
+                    print(json.dumps({
+                        "step": "draft" if args.draft else "verify", "batch": B, "k": k, "prefix": j, "src_len": S,
+                        "us_median": us, "us_min": us_min, "l2_flush": flush is not None, "mean_accepted": mean_a,
+                        "algorithmic_MB": bytes_ / 1e6, "algorithmic_GFLOP": flops / 1e9,
+                        "hbm_GBs": bytes_ / us / 1e3, "hbm_frac": bytes_ / us / 1e3 / hbm,
+                        "tensor_TFLOPs": flops / us / 1e6, "tensor_frac": flops / us / 1e6 / tc, "peaks": kind,
+                    }))
+        sd.close()
 
 
 if __name__ == "__main__":
