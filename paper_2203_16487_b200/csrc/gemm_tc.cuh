@@ -121,7 +121,8 @@ constexpr int TC_THREADS = (2 + TC_EPI_WARPS) * 32;  // + TMA warp + MMA warp
 template <int BN> struct TcCfg {
     static constexpr int STAGES = BN >= 256 ? 4 : (BN >= 128 ? 6 : 8);
     static constexpr int STAGE_BYTES = (TC_BM + BN) * TC_BK * 2;
-    static constexpr int SMEM = STAGES * STAGE_BYTES + 1024;
+    static constexpr int STG_BYTES = TC_EPI_WARPS * 32 * 32 * 4;      // per-warp 32 x 32 fp32 transpose buffers
+    static constexpr int SMEM = STAGES * STAGE_BYTES + STG_BYTES + 1024;
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;      // two accumulators
 };
 
@@ -167,6 +168,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb = g.K / TC_BK;
+    float* stg = reinterpret_cast<float*>(smem_raw + (tiles - smem_u32(smem_raw)) + STAGES * Cfg::STAGE_BYTES) + (warp >= 2 ? warp - 2 : 0) * 1024;
 
     if (threadIdx.x == 0) {
         abort_s = 0;
@@ -236,6 +238,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16) + ab * BN + half * HALF;
             const bool warp_live = live && (m0 + q * 32 < R);    // warp-uniform: any live row in this quadrant
             float v[CW];
+            long long my_cache_row = 0;                          // EPI_QKV: cache row of this lane's output row
+            if (EPI == EPI_QKV && warp_live && r < R) my_cache_row = (long long)g.pg.row(g.seq[r], g.pos[r]);
             if (warp_live && EPI == EPI_STATS) {
                 const float ld = (g.ld && r < R) ? g.ld[r] : CUDART_INF_F;
                 const int id = (g.ld_id && r < R) ? g.ld_id[r] : -1;
@@ -272,50 +276,78 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 for (int c = 0; c < HALF / CW; ++c) {
                     tmem_ld<CW>(trow + c * CW, v);
                     const int nb = n0 + c * CW;
-                    if (r >= R) continue;
                     if (g.bias) {
 #pragma unroll
                         for (int j = 0; j < CW; ++j) v[j] += (nb + j < g.N) ? __ldg(g.bias + nb + j) : 0.f;
                     }
+                    if (EPI == EPI_RELU) {
+#pragma unroll
+                        for (int j = 0; j < CW; ++j) v[j] = fmaxf(v[j], 0.f);
+                    }
                     const bool full = nb + CW <= g.N;
-                    if (EPI == EPI_STORE || EPI == EPI_RELU || EPI == EPI_QKV) {
+                    const bool bf_out = (EPI == EPI_STORE || EPI == EPI_RELU || EPI == EPI_QKV);
+                    if (CW == 32 && full && (bf_out ? (g.ldo % 2 == 0 && (EPI != EPI_QKV || g.kv_d % 32 == 0)) : true)) {
+                        // Transpose through shared memory: a thread owns one output ROW in tensor memory, but global
+                        // memory wants a warp to touch one row at a time.  The 32 x 32 block is written row-wise with
+                        // its 16-byte chunks XOR-swizzled by the row, then read back one row per warp instruction.
+                        float* srow = stg + lane * 32;
+#pragma unroll
+                        for (int j4 = 0; j4 < 8; ++j4)
+                            *reinterpret_cast<float4*>(srow + ((j4 ^ (lane & 7)) << 2)) = make_float4(v[j4 * 4], v[j4 * 4 + 1], v[j4 * 4 + 2], v[j4 * 4 + 3]);
+                        __syncwarp();
+                        const int rbase = m0 + q * 32;
+                        if (!bf_out) {
+                            float* gcol = g.resid + nb + lane;
+#pragma unroll
+                            for (int r8 = 0; r8 < 32; r8 += 8) {
+                                float xin[8];
+                                if (EPI == EPI_RESID) {
+#pragma unroll
+                                    for (int u = 0; u < 8; ++u) xin[u] = (rbase + r8 + u < R) ? gcol[(size_t)(rbase + r8 + u) * g.N] : 0.f;
+                                }
+#pragma unroll
+                                for (int u = 0; u < 8; ++u) {
+                                    const int rr = r8 + u;
+                                    float val = stg[rr * 32 + ((((lane >> 2) ^ (rr & 7))) << 2) + (lane & 3)];
+                                    if (EPI == EPI_RESID) val += xin[u];
+                                    if (rbase + rr < R) gcol[(size_t)(rbase + rr) * g.N] = val;
+                                }
+                            }
+                        } else {
+                            const int hl = lane >> 4, cl = lane & 15;           // half-warp per row, two columns per lane
+#pragma unroll 4
+                            for (int r2 = 0; r2 < 32; r2 += 2) {
+                                const int rr = r2 + hl, gr = rbase + rr;
+                                const long long row_of = (EPI == EPI_QKV) ? __shfl_sync(0xffffffffu, my_cache_row, rr) : 0;
+                                const float2 pv = *reinterpret_cast<const float2*>(stg + rr * 32 + (((cl >> 1) ^ (rr & 7)) << 2) + (cl & 1) * 2);
+                                if (gr < R) {
+                                    bf16* o = g.out + (size_t)gr * g.ldo + nb;
+                                    if (EPI == EPI_QKV && nb >= g.kv_d) {          // K or V part: straight into the paged cache
+                                        const size_t row = (size_t)row_of;
+                                        o = (nb < 2 * g.kv_d ? g.kc + row * g.kv_d + (nb - g.kv_d) : g.vc + row * g.kv_d + (nb - 2 * g.kv_d));
+                                    }
+                                    __nv_bfloat162 b2;
+                                    b2.x = __float2bfloat16_rn(pv.x); b2.y = __float2bfloat16_rn(pv.y);
+                                    *reinterpret_cast<__nv_bfloat162*>(o + cl * 2) = b2;
+                                }
+                            }
+                        }
+                        __syncwarp();
+                        continue;
+                    }
+                    if (r >= R) continue;
+                    if (bf_out) {
                         bf16* o = g.out + (size_t)r * g.ldo + nb;
-                        int ldo_ok = g.ldo % 8 == 0;
-                        if (EPI == EPI_QKV && nb >= g.kv_d) {              // K or V part: straight into the paged cache
+                        if (EPI == EPI_QKV && nb >= g.kv_d) {
                             const size_t row = g.pg.row(g.seq[r], g.pos[r]);
                             o = (nb < 2 * g.kv_d ? g.kc + row * g.kv_d + (nb - g.kv_d) : g.vc + row * g.kv_d + (nb - 2 * g.kv_d));
-                            ldo_ok = g.kv_d % 8 == 0;
                         }
-                        if (full && ldo_ok) {
-#pragma unroll
-                            for (int j = 0; j < CW; j += 8) {
-                                __align__(16) bf16 tb[8];
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) tb[e] = __float2bfloat16_rn(EPI == EPI_RELU ? fmaxf(v[j + e], 0.f) : v[j + e]);
-                                *reinterpret_cast<uint4*>(o + j) = *reinterpret_cast<const uint4*>(tb);
-                            }
-                        } else {
-                            for (int j = 0; j < CW; ++j)
-                                if (nb + j < g.N) o[j] = __float2bfloat16_rn(EPI == EPI_RELU ? fmaxf(v[j], 0.f) : v[j]);
-                        }
+                        for (int j = 0; j < CW; ++j)
+                            if (nb + j < g.N) o[j] = __float2bfloat16_rn(v[j]);
                     } else {
                         float* o = g.resid + (size_t)r * g.N + nb;
-                        if (full && (g.N % 4 == 0)) {
-                            float4 xin[CW / 4];
-                            if (EPI == EPI_RESID) {
-#pragma unroll
-                                for (int j = 0; j < CW / 4; ++j) xin[j] = *reinterpret_cast<const float4*>(o + j * 4);
-                            }
-#pragma unroll
-                            for (int j = 0; j < CW / 4; ++j) {
-                                float4 tv = make_float4(v[j * 4], v[j * 4 + 1], v[j * 4 + 2], v[j * 4 + 3]);
-                                if (EPI == EPI_RESID) { tv.x += xin[j].x; tv.y += xin[j].y; tv.z += xin[j].z; tv.w += xin[j].w; }
-                                *reinterpret_cast<float4*>(o + j * 4) = tv;
-                            }
-                        } else {
-                            for (int j = 0; j < CW; ++j)
-                                if (nb + j < g.N) o[j] = (EPI == EPI_RESID ? o[j] : 0.f) + v[j];
-                        }
+                        for (int j = 0; j < CW; ++j)
+                            if (nb + j < g.N) o[j] = (EPI == EPI_RESID ? o[j] : 0.f) + v[j];
                     }
                 }
             }
@@ -395,6 +427,7 @@ inline int tc_init(TmaEncoder& enc, int* err_word) {
     if (e == cudaSuccess) e = tc_set_smem_all<EPI_F32>();
     if (e == cudaSuccess) e = tc_set_smem_all<EPI_QKV>();
     if (e == cudaSuccess) e = tc_set_smem<EPI_STATS, 128>();
+    if (e == cudaSuccess) e = tc_set_smem<EPI_STATS, 256>();
     if (e != cudaSuccess) { enc.err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return -1; }
     enc.err_word = err_word;
     enc.ready = true;
@@ -425,28 +458,34 @@ inline int tc_launch_bn(TmaEncoder& enc, int bn, GemmArgs<bf16>& g, int rows_ub,
     }
 }
 
-// Picks the widest N tile that still yields at least one CTA per SM; otherwise the narrowest
-// (most CTAs streaming the weights).
-inline int tc_pick_bn(int N, int rows_ub) {
+// Tile width: a CTA ingests (128 + BN) * K * 2 bytes per tile and the SMs are ingest-bound long before
+// they are math-bound, so pick the BN that minimises waves * (128 + BN); ties go to the wider tile.
+inline int tc_pick_bn(int N, int rows_ub, int n_sm) {
     const int m_tiles = (rows_ub + TC_BM - 1) / TC_BM;
     const int cand[4] = {256, 128, 64, 32};
+    int best = 32; long long best_cost = -1;
     for (int i = 0; i < 4; ++i) {
         const int bn = cand[i];
-        if (bn > N) continue;
-        if ((long long)((N + bn - 1) / bn) * m_tiles >= 148) return bn;
+        if (bn > N && bn != 32) continue;
+        if (bn == 32 && m_tiles > 1) continue;                 // the narrow tile only pays for a single row tile
+        const long long tiles = (long long)((N + bn - 1) / bn) * m_tiles;
+        const long long cost = ((tiles + n_sm - 1) / n_sm) * (TC_BM + bn);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
     }
-    return 32;
+    return best;
 }
 
 inline int gemm_tc_launch(TmaEncoder& enc, int epi, GemmArgs<bf16>& g, int rows_ub, cudaStream_t st, int* n_tiles_out) {
     if (!enc.ready) return -1;
     if (epi == EPI_STATS) {
         if (g.N < 128) return -2;
-        g.n_tiles = 2 * ((g.N + 127) / 128);          // two column halves per tile
+        const bool wide = rows_ub > 4 * TC_BM && g.N >= 256;    // many row tiles: wider tiles halve the re-reads of A
+        const int bn = wide ? 256 : 128;
+        g.n_tiles = 2 * ((g.N + bn - 1) / bn);                   // two column halves per tile
         if (n_tiles_out) *n_tiles_out = g.n_tiles;
-        return tc_launch_one<EPI_STATS, 128>(enc, g, rows_ub, st);
+        return wide ? tc_launch_one<EPI_STATS, 256>(enc, g, rows_ub, st) : tc_launch_one<EPI_STATS, 128>(enc, g, rows_ub, st);
     }
-    const int bn = tc_pick_bn(g.N, rows_ub);
+    const int bn = tc_pick_bn(g.N, rows_ub, enc.n_sm);
     switch (epi) {
         case EPI_STORE: return tc_launch_bn<EPI_STORE>(enc, bn, g, rows_ub, st);
         case EPI_RELU: return tc_launch_bn<EPI_RELU>(enc, bn, g, rows_ub, st);

@@ -164,7 +164,8 @@ __global__ void k_gather_rows(const float* __restrict__ x, const int* __restrict
     for (int e = threadIdx.x; e < d; e += blockDim.x) out[(size_t)row * d + e] = s[e];
 }
 
-// One warp per row; biased variance, eps inside the square root.
+// One warp per row; biased variance, eps inside the square root.  Rows of up to 512 elements
+// (a multiple of 128) are held in registers, so the row is read from memory once.
 template <typename T>
 __global__ void k_layernorm(const float* __restrict__ x, const float* __restrict__ g, const float* __restrict__ b,
                             const int* __restrict__ n_rows, T* __restrict__ y, int d, float eps) {
@@ -172,6 +173,39 @@ __global__ void k_layernorm(const float* __restrict__ x, const float* __restrict
     int lane = threadIdx.x & 31;
     if (row >= *n_rows) return;
     const float* xr = x + (size_t)row * d;
+    if (d % 128 == 0 && d <= 512) {
+        float4 v[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int e = lane * 4 + c * 128;
+            v[c] = e < d ? *reinterpret_cast<const float4*>(xr + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float s = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) s += v[c].x + v[c].y + v[c].z + v[c].w;
+        const float mu = warp_sum(s) / d;
+        float q = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            if (lane * 4 + c * 128 < d) {
+                const float c0 = v[c].x - mu, c1 = v[c].y - mu, c2 = v[c].z - mu, c3 = v[c].w - mu;
+                q += c0 * c0 + c1 * c1 + c2 * c2 + c3 * c3;
+            }
+        const float rstd = 1.0f / sqrtf(warp_sum(q) / d + eps);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int e = lane * 4 + c * 128;
+            if (e < d) {
+                const float4 gm = *reinterpret_cast<const float4*>(g + e), bt = *reinterpret_cast<const float4*>(b + e);
+                T* o = y + (size_t)row * d + e;
+                o[0] = from_f<T>((v[c].x - mu) * rstd * gm.x + bt.x);
+                o[1] = from_f<T>((v[c].y - mu) * rstd * gm.y + bt.y);
+                o[2] = from_f<T>((v[c].z - mu) * rstd * gm.z + bt.z);
+                o[3] = from_f<T>((v[c].w - mu) * rstd * gm.w + bt.w);
+            }
+        }
+        return;
+    }
     float s = 0.f;
     for (int e = lane; e < d; e += 32) s += xr[e];
     float mu = warp_sum(s) / d;

@@ -307,7 +307,7 @@ template <typename T>
 int ln(specdec_handle* h, const float* x, const float* g, const float* b, int cnt, int rows_ub, void* y, int d,
        cudaStream_t st) {
     if (rows_ub <= 0) return 0;
-    k_layernorm<T><<<cdiv(rows_ub, 4), 128, 0, st>>>(x, g, b, h->ses.counters + cnt, (T*)y, d, 1e-5f);
+    k_layernorm<T><<<cdiv(rows_ub, 8), 256, 0, st>>>(x, g, b, h->ses.counters + cnt, (T*)y, d, 1e-5f);
     KCHECK(h);
     return 0;
 }
