@@ -298,7 +298,10 @@ def run_ours(args):
     roof = ({"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak}
             if bound_hbm else
             {"bound": "tensor", "achieved": tf, "peak": tc_peak, "unit": "TFLOP/s", "frac": tf / tc_peak})
-    roof.update({"traffic": None, "kernel": "k_gemm_tc<EPI_STATS,128> (vocabulary projection + row statistics)",
+    # DRAM bytes of one launch from the ncu capture summarised in profiles/vocab_stats_kernel_b1_ncu.md
+    # (dram__bytes_read.sum + dram__bytes_write.sum at 26 rows); none was taken at other row counts
+    traffic = 33613824 if B == 1 else None
+    roof.update({"traffic": traffic, "kernel": "k_gemm_tc<EPI_STATS> (vocabulary projection + row statistics, verify step)",
                  "peak_kind": f"of {peak_kind}", "launches_timed": int(vocab_n), "us_per_launch": per_launch_ms * 1e3,
                  "algorithmic_bytes_per_launch": alg_bytes})
 

@@ -194,9 +194,9 @@ int specdec_debug_cluster_trace(specdec_handle* h, long long* h_out, int n);
  * d_script[b*stride + j + i] wherever that entry is >= 0.  d_script = NULL turns it off. */
 int specdec_set_draft_script(specdec_handle* h, const int32_t* d_script, int B, int stride, void* stream);
 
-/* With option "profile" = 1, every vocabulary-projection launch of draft and verify inside
- * specdec_generate is bracketed by CUDA events; this returns their summed duration and count
- * since the option was set. */
+/* With option "profile" = 1, every vocabulary-projection launch of the verify step (B*(k+1) rows)
+ * inside specdec_generate is bracketed by CUDA events; this returns their summed duration and
+ * count since the option was set. */
 int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches);
 
 /* Options: "gemm" = 0 SIMT reference GEMM, 1 tcgen05 GEMM (bf16 handles; default 1);

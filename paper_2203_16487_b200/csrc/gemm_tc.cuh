@@ -115,6 +115,9 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+__device__ __forceinline__ void tc_stamp(long long* trace, int slot) {
+    if (trace && blockIdx.x == 0) { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); trace[slot] = t; }
+}
 constexpr int TC_BM = 128, TC_BK = 64;
 constexpr int TC_EPI_WARPS = 8;                      // two per TMEM lane quadrant: each takes half the columns
 constexpr int TC_THREADS = (2 + TC_EPI_WARPS) * 32;  // + TMA warp + MMA warp
@@ -155,6 +158,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     using Cfg = TcCfg<BN>;
     constexpr int STAGES = Cfg::STAGES;
     constexpr int HALF = BN / 2;                     // columns per epilogue warp
+    if (threadIdx.x == 0) tc_stamp(g.trace, 0);
     constexpr int CW = HALF >= 32 ? 32 : 16;         // columns per TMEM read
     const int R = *g.n_rows;
     const int m_tiles = (R + TC_BM - 1) / TC_BM, n_tiles = (g.N + BN - 1) / BN;
@@ -183,6 +187,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     tc_fence_after();
     const uint32_t tmem_d = tmem_base_s;
     volatile int* abort_flag = &abort_s;
+    if (threadIdx.x == 0) tc_stamp(g.trace, 1);
 
     if (warp == 0) {
         if (lane == 0) {
@@ -198,8 +203,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     mbar_expect_tx(bar, Cfg::STAGE_BYTES);
                     tma_load_2d(a_dst, &tmA, kb * TC_BK, m0, bar);
                     tma_load_2d(w_dst, &tmW, kb * TC_BK, n0, bar);
+                    if (kbi == 0) tc_stamp(g.trace, 2);
                 }
             }
+            tc_stamp(g.trace, 3);
         }
     } else if (warp == 1) {
         if (lane == 0) {
@@ -214,6 +221,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     const int s = kbi % STAGES;
                     mbar_wait(smem_u32(&bar_full[s]), (kbi / STAGES) & 1, abort_flag, err_word, 2);
                     if (*abort_flag) break;
+                    if (kbi == 0) tc_stamp(g.trace, 4);
                     tc_fence_after();
                     const uint32_t a_src = tiles + s * Cfg::STAGE_BYTES, w_src = a_src + TC_BM * TC_BK * 2;
                     const uint64_t ad = umma_desc_k_sw128(a_src), wd = umma_desc_k_sw128(w_src);
@@ -223,6 +231,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     umma_commit(smem_u32(&bar_empty[s]));        // stage reusable once these MMAs have read it
                 }
                 umma_commit(smem_u32(&bar_acc_full[ab]));        // accumulator of this tile complete
+                tc_stamp(g.trace, 5 + (i > 0));
             }
         }
     } else {
@@ -234,6 +243,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             const int m0 = (t % m_tiles) * TC_BM, n_tile = t / m_tiles, n0 = n_tile * BN + half * HALF;
             const int r = m0 + q * 32 + lane;
             const bool live = mbar_wait(smem_u32(&bar_acc_full[ab]), (i >> 1) & 1, abort_flag, err_word, 3);
+            if (threadIdx.x == 64) tc_stamp(g.trace, 7 + 2 * (i > 0));
             tc_fence_after();
             const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16) + ab * BN + half * HALF;
             const bool warp_live = live && (m0 + q * 32 < R);    // warp-uniform: any live row in this quadrant
@@ -355,11 +365,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[ab]));
+            if (threadIdx.x == 64) tc_stamp(g.trace, 8 + 2 * (i > 0));
         }
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_d, Cfg::TMEM_COLS);
+    if (threadIdx.x == 0) tc_stamp(g.trace, 11);
 }
 
 // ------------------------------------------------------------------ host side

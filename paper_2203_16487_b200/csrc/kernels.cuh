@@ -320,6 +320,7 @@ struct GemmArgs {
     // EPI_QKV: columns [0, kv_d) are stored like EPI_STORE, [kv_d, 2 kv_d) go to the K cache and
     // [2 kv_d, 3 kv_d) to the V cache at the row's (sequence, position)
     const int* seq; const int* pos; Paged pg; T* kc; T* vc; int kv_d;
+    long long* trace;           // optional: CTA 0 records %globaltimer at a few points (debugging aid)
 };
 
 // Merge of (max, argmax, count) only: used on the hot path, where the sum is not needed.

@@ -398,6 +398,7 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
     g.part = h->part; g.ld = ldv; g.ld_id = ld_id; g.n_tiles = cdiv(N, 64); g.want_sum = h->want_lse;
     g.seq = nullptr; g.pos = nullptr; g.kc = nullptr; g.vc = nullptr; g.kv_d = 0;
     g.pg.table = h->page_table; g.pg.page_tokens = h->cfg.page_tokens; g.pg.max_pages = h->pages_per_seq;
+    g.trace = (h->want_cl_trace && epi == EPI_STATS && h->cl_trace) ? h->cl_trace + 200 : nullptr;
     if (kv) { g.seq = kv->seq; g.pos = kv->pos; g.kc = (T*)kv->kc; g.vc = (T*)kv->vc; g.kv_d = kv->d; }
     if constexpr (std::is_same<T, bf16>::value) {
         if (skinny) {
@@ -627,10 +628,8 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
     TRY(block_ffn<T>(h, m, w, h->x2, CNT_DRAFT_MASK, R2, st));
     TRY(ln<T>(h, h->x2, m.dec_lnf_g, m.dec_lnf_b, CNT_DRAFT_MASK, R2, h->y, d, st));
     int n_tiles = 0;
-    prof_mark(h, st);
     TRY(gemm<T>(h, EPI_STATS, h->y, d, m.embed, nullptr, m.dm.vocab, d, CNT_DRAFT_MASK, R2, nullptr, 0, nullptr, st,
                 nullptr, nullptr, &n_tiles));
-    prof_mark(h, st);
     k_draft_argmax<<<cdiv(R2, 4), 128, 0, st>>>(h->part, n_tiles, h->ses.counters + CNT_DRAFT_MASK, h->mrows.slot,
                                                d_draft);
     KCHECK(h);
@@ -772,6 +771,22 @@ int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F
     return 0;
 }
 
+// encode through a CUDA graph: the inputs are first copied into the handle's own staging buffers so that the
+// captured launches never depend on the caller's pointers
+template <typename T>
+int encode_staged(specdec_handle* h, const int* d_src, const int* d_src_len, const int* d_max_tgt, int B, int S_max,
+                  cudaStream_t st) {
+    if (!h->use_graphs || h->profile) return encode_impl<T>(h, d_src, d_src_len, d_max_tgt, B, S_max, st);
+    if (d_src != h->stage_src) CUDA_TRY(h, cudaMemcpyAsync(h->stage_src, d_src, (size_t)B * S_max * 4, cudaMemcpyDeviceToDevice, st));
+    if (d_src_len != h->stage_len) CUDA_TRY(h, cudaMemcpyAsync(h->stage_len, d_src_len, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
+    if (d_max_tgt && d_max_tgt != h->stage_mt) CUDA_TRY(h, cudaMemcpyAsync(h->stage_mt, d_max_tgt, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
+    h->B = B; h->S_max = S_max;
+    TRY(graph_call(h, {5, d_max_tgt ? 1 : 0}, st, [&]() {
+        return encode_impl<T>(h, h->stage_src, h->stage_len, d_max_tgt ? h->stage_mt : nullptr, B, S_max, st); }));
+    h->len_ub = 0; h->encoded = true; h->verified = false; h->drafted = false;
+    return 0;
+}
+
 inline int len_bucket(const specdec_handle* h, int len_ub) { return std::min(h->T_cap, (len_ub + 31) / 32 * 32); }
 
 template <typename T>
@@ -782,7 +797,7 @@ int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, con
     size_t ev = 0;
     auto mark = [&]() { if (timed && ev < h->time_ev.size()) cudaEventRecord(h->time_ev[ev++], st); };
     mark();
-    TRY(encode_impl<T>(h, d_src, d_src_len, d_max_tgt, B, S_max, st));
+    TRY(encode_staged<T>(h, d_src, d_src_len, d_max_tgt, B, S_max, st));
     mark();
     const int max_iters = h->T_cap;            // every iteration commits >= 1 token per unfinished sequence
     const int lag = 2, slots = (int)h->poll_ev.size();
@@ -1051,8 +1066,8 @@ int specdec_encode(specdec_handle* h, const int32_t* d_src, const int32_t* d_src
     if (B > h->B_cap || S_max > h->S_cap) return fail(h, SPECDEC_ERR_CAPACITY, "encode: B or S_max beyond capacity");
     StreamScope scope(h, stream);
     cudaStream_t st = scope.st;
-    return DISPATCH(h, encode_impl<bf16>(h, d_src, d_src_len, d_max_tgt, B, S_max, st),
-                    encode_impl<float>(h, d_src, d_src_len, d_max_tgt, B, S_max, st));
+    return DISPATCH(h, encode_staged<bf16>(h, d_src, d_src_len, d_max_tgt, B, S_max, st),
+                    encode_staged<float>(h, d_src, d_src_len, d_max_tgt, B, S_max, st));
 }
 
 int specdec_draft(specdec_handle* h, int k, int32_t* d_draft, void* stream) {
