@@ -120,7 +120,7 @@ int specdec_draft(specdec_handle* h, int k, int32_t* d_draft, void* stream);
  * its score <= tau (Eq. 8).  d_accepted [B] receives the accepted length in
  * [0,k]; d_bif [B] the verifier's top-1 token on the row after the accepted
  * prefix (the replacement at the bifurcation, or the bonus token when a = k).
- * Does not commit.  beta >= 1, tau >= 0, 1 <= k <= k_max. */
+ * Does not commit.  beta >= 1, tau >= 0, 0 <= k <= k_max (k = 0: one row, the next greedy token). */
 int specdec_verify(specdec_handle* h, const int32_t* d_draft, int k, int beta, float tau,
                    int32_t* d_accepted, int32_t* d_bif, void* stream);
 
@@ -133,7 +133,9 @@ int specdec_commit(specdec_handle* h, const int32_t* d_keep, const int32_t* d_ne
 
 /* encode + (draft -> verify -> commit) until every sequence is finished.
  * d_out [B,out_stride] int32 receives the generated ids (without BOS),
- * d_out_len [B] their count.  h_stats may be NULL.  Synchronises `stream`. */
+ * d_out_len [B] their count.  h_stats may be NULL.  Synchronises `stream`.
+ * k = 0 is plain greedy autoregressive decoding with the verifier alone (no drafter pass, one-row
+ * verify blocks): the baseline SpecDec is compared with. */
 int specdec_generate(specdec_handle* h, const int32_t* d_src, const int32_t* d_src_len,
                      const int32_t* d_max_tgt, int B, int S_max, int k, int beta, float tau,
                      int32_t* d_out, int out_stride, int32_t* d_out_len,

@@ -385,6 +385,7 @@ struct TmaEncoder {
     PFN_encodeTiled encode = nullptr;
     int* err_word = nullptr;            // device word the kernels raise on a wait timeout
     int n_sm = 148;
+    int force_bn = 0;                   // experiments: 0 = choose, else 32 / 64 / 128 / 256
     std::map<std::tuple<const void*, long long, int, int, int>, CUtensorMap> cache;
 
     // 2-D bf16 tensor [rows, K] with row pitch ld elements; box = 64 x box_rows, 128-byte swizzle.
@@ -471,7 +472,8 @@ inline int tc_launch_bn(TmaEncoder& enc, int bn, GemmArgs<bf16>& g, int rows_ub,
 }
 
 // Tile width: a CTA ingests (128 + BN) * K * 2 bytes per tile and the SMs are ingest-bound long before
-// they are math-bound, so pick the BN that minimises waves * (128 + BN); ties go to the wider tile.
+// they are math-bound, so pick the BN that minimises waves * (128 + BN); ties go to the narrower tile
+// (more tiles per CTA, so more of the epilogue overlaps the next tile's loads).
 inline int tc_pick_bn(int N, int rows_ub, int n_sm) {
     const int m_tiles = (rows_ub + TC_BM - 1) / TC_BM;
     const int cand[4] = {256, 128, 64, 32};
@@ -482,7 +484,7 @@ inline int tc_pick_bn(int N, int rows_ub, int n_sm) {
         if (bn == 32 && m_tiles > 1) continue;                 // the narrow tile only pays for a single row tile
         const long long tiles = (long long)((N + bn - 1) / bn) * m_tiles;
         const long long cost = ((tiles + n_sm - 1) / n_sm) * (TC_BM + bn);
-        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
+        if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best = bn; }
     }
     return best;
 }
@@ -497,7 +499,7 @@ inline int gemm_tc_launch(TmaEncoder& enc, int epi, GemmArgs<bf16>& g, int rows_
         if (n_tiles_out) *n_tiles_out = g.n_tiles;
         return wide ? tc_launch_one<EPI_STATS, 256>(enc, g, rows_ub, st) : tc_launch_one<EPI_STATS, 128>(enc, g, rows_ub, st);
     }
-    const int bn = tc_pick_bn(g.N, rows_ub, enc.n_sm);
+    const int bn = (enc.force_bn && enc.force_bn <= g.N) ? enc.force_bn : tc_pick_bn(g.N, rows_ub, enc.n_sm);
     switch (epi) {
         case EPI_STORE: return tc_launch_bn<EPI_STORE>(enc, bn, g, rows_ub, st);
         case EPI_RELU: return tc_launch_bn<EPI_RELU>(enc, bn, g, rows_ub, st);

@@ -310,6 +310,7 @@ struct GemmArgs {
     const float* bias;          // [N] or null
     int N, K;
     const int* n_rows;          // device row count
+    int rows_static;            // >= 0: the row count is known on the host (saves a dependent load); else read n_rows
     T* out; int ldo;            // EPI_STORE / EPI_RELU
     float* resid;               // EPI_RESID: resid[r, n] += value ; EPI_F32: resid[r, n] = value (ld = N)
     // EPI_STATS

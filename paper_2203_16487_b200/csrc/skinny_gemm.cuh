@@ -24,7 +24,12 @@ struct SkinnyArgs {
     const float* ln_x;           // LayerNorm prologue: fp32 rows [rows, K] ...
     const float* ln_g; const float* ln_b; float ln_eps;
     bf16* ln_out;                // ... optionally also written out as bf16 rows [rows, K] (by CTA 0)
+    long long* trace;            // optional: CTA 0 records %globaltimer at a few points (debugging aid)
 };
+
+__device__ __forceinline__ void sk_stamp(long long* trace, int slot) {
+    if (trace && blockIdx.x == 0 && threadIdx.x == 0) { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); trace[slot] = t; }
+}
 
 constexpr int SK_NB = 8;         // weight rows per CTA
 constexpr int SK_WARPS = 8;
@@ -36,6 +41,7 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
     const GemmArgs<bf16>& g = a.g;
     const int K = g.K, N = g.N;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t4 = lane & 3;
+    sk_stamp(a.trace, 0);
     const int n0 = blockIdx.x * SK_NB;
     const int pitch = K + 8;                                  // bf16 elements per activation row in shared memory
     bf16* As = reinterpret_cast<bf16*>(sk_sm);
@@ -55,10 +61,23 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
         wreg[ss] = (w_ok && warp < nsplit && k0 < k_end) ? __ldg(reinterpret_cast<const uint4*>(wrow + k0)) : make_uint4(0, 0, 0, 0);
     }
 
+    // bias and LayerNorm parameters are weights too: fetch them before waiting for the predecessor
+    const float bias_v = (g.bias && n0 + (tid & 7) < N) ? __ldg(g.bias + n0 + (tid & 7)) : 0.f;
+    float4 lgam[4], lbet[4];
+    if (LN) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int e = lane * 4 + c * 128;
+            lgam[c] = e < K ? __ldg(reinterpret_cast<const float4*>(a.ln_g + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            lbet[c] = e < K ? __ldg(reinterpret_cast<const float4*>(a.ln_b + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
     // everything above touched only weights; from here on the predecessor's output is read
+    sk_stamp(a.trace, 1);
     pdl_launch_dependents();
     pdl_wait();
-    const int R = min(*g.n_rows, MT * 16);      // the live row count is itself written earlier in the step
+    sk_stamp(a.trace, 2);
+    const int R = min(g.rows_static >= 0 ? g.rows_static : *g.n_rows, MT * 16);   // a device-side count is itself written earlier in the step
     // ---- activation rows into shared memory
     if (LN) {
         // each warp normalises rows warp, warp + 8, ...; all of its rows are fetched first (one round trip)
@@ -97,7 +116,7 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
                     const int e = lane * 4 + c * 128;
                     if (e < K) {
                         const float4 v = xv[s][c];
-                        const float4 gm = *reinterpret_cast<const float4*>(a.ln_g + e), bt = *reinterpret_cast<const float4*>(a.ln_b + e);
+                        const float4 gm = lgam[c], bt = lbet[c];
                         __nv_bfloat162 p0, p1;
                         p0.x = __float2bfloat16_rn((v.x - mu) * rstd * gm.x + bt.x); p0.y = __float2bfloat16_rn((v.y - mu) * rstd * gm.y + bt.y);
                         p1.x = __float2bfloat16_rn((v.z - mu) * rstd * gm.z + bt.z); p1.y = __float2bfloat16_rn((v.w - mu) * rstd * gm.w + bt.w);
@@ -125,6 +144,7 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
         asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
     __syncthreads();
+    sk_stamp(a.trace, 3);
 
     // ---- products: per super-step of 32 k, two MMAs per 16-row tile
     float acc[MT][4];
@@ -146,16 +166,25 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
                 }
             }
         };
+        // chunks of MAX_SS super-steps: the next chunk's weights are in flight while this one is multiplied
+        for (int cb = k_begin; cb < k_end; cb += MAX_SS * 32) {
+            uint4 wnext[MAX_SS];
+            const int nb = cb + MAX_SS * 32;
 #pragma unroll
-        for (int ss = 0; ss < MAX_SS; ++ss) {
-            const int k0 = k_begin + ss * 32;
-            if (k0 < k_end) step(wreg[ss], k0);
-        }
-        for (int k0 = k_begin + MAX_SS * 32; k0 < k_end; k0 += 32) {       // K slices longer than the preloaded part
-            const uint4 w = w_ok ? __ldg(reinterpret_cast<const uint4*>(wrow + k0)) : make_uint4(0, 0, 0, 0);
-            step(w, k0);
+            for (int ss = 0; ss < MAX_SS; ++ss) {
+                const int k0 = nb + ss * 32;
+                wnext[ss] = (w_ok && k0 < k_end) ? __ldg(reinterpret_cast<const uint4*>(wrow + k0)) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int ss = 0; ss < MAX_SS; ++ss) {
+                const int k0 = cb + ss * 32;
+                if (k0 < k_end) step(wreg[ss], k0);
+            }
+#pragma unroll
+            for (int ss = 0; ss < MAX_SS; ++ss) wreg[ss] = wnext[ss];
         }
     }
+    sk_stamp(a.trace, 4);
     // ---- fixed-order sum over the K split, then the epilogue
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
@@ -169,7 +198,7 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
         if (r >= R || n >= N) continue;
         float v = 0.f;
         for (int s = 0; s < nsplit; ++s) v += red[(size_t)s * MT * 16 * SK_NB + o];
-        if (g.bias) v += g.bias[n];
+        v += bias_v;
         if (EPI == EPI_STORE) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(v);
         if (EPI == EPI_RELU) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(fmaxf(v, 0.f));
         if (EPI == EPI_RESID) g.resid[(size_t)r * N + n] += v;
@@ -182,6 +211,7 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
             }
         }
     }
+    sk_stamp(a.trace, 5);
 }
 
 }  // namespace sd

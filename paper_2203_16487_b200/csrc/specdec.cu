@@ -394,7 +394,7 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
     }
     GemmArgs<T> g;
     g.A = (const T*)A; g.lda = lda; g.W = (const T*)W; g.bias = bias; g.N = N; g.K = K;
-    g.n_rows = h->ses.counters + cnt; g.out = (T*)out; g.ldo = ldo; g.resid = resid;
+    g.n_rows = h->ses.counters + cnt; g.rows_static = (cnt == CNT_VERIFY || cnt == CNT_ENC) ? rows_ub : -1; g.out = (T*)out; g.ldo = ldo; g.resid = resid;
     g.part = h->part; g.ld = ldv; g.ld_id = ld_id; g.n_tiles = cdiv(N, 64); g.want_sum = h->want_lse;
     g.seq = nullptr; g.pos = nullptr; g.kc = nullptr; g.vc = nullptr; g.kv_d = 0;
     g.pg.table = h->page_table; g.pg.page_tokens = h->cfg.page_tokens; g.pg.max_pages = h->pages_per_seq;
@@ -405,6 +405,7 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
             SkinnyArgs sa; sa.g = g;
             sa.ln_x = lnp ? lnp->x : nullptr; sa.ln_g = lnp ? lnp->g : nullptr; sa.ln_b = lnp ? lnp->b : nullptr;
             sa.ln_eps = 1e-5f; sa.ln_out = nullptr;
+            sa.trace = (h->want_cl_trace && h->cl_trace) ? h->cl_trace + 216 + 6 * (epi == EPI_RELU ? 0 : epi == EPI_RESID ? 1 : epi == EPI_QKV ? 2 : 3) : nullptr;
             TRY(skinny_launch(h, epi, sa, rows_ub, st));
             return 0;
         }
@@ -649,7 +650,7 @@ int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float ta
     ModelW& m = h->ver;
     const int B = h->B, d = m.dm.d_model, L = m.dm.dec_layers, M = B * (k + 1);
     const int max_keys = std::min(h->len_ub, h->T_cap) + k + 1;
-    if (d_draft != h->v_draft)
+    if (d_draft != h->v_draft && k > 0)
         CUDA_TRY(h, cudaMemcpyAsync(h->v_draft, d_draft, (size_t)B * k * 4, cudaMemcpyDeviceToDevice, st));
     k_verify_prep<<<cdiv(M, 256), 256, 0, st>>>(h->ses, h->v_draft, B, k, h->S_max, h->cfg.bos_id, h->rows);
     KCHECK(h);
@@ -809,7 +810,7 @@ int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, con
             // the launches depend on the host-side length bound only through its 32-token bucket
             const int true_ub = h->len_ub, lb = len_bucket(h, true_ub);
             h->len_ub = lb;
-            TRY(graph_call(h, {1, k, lb}, st, [&]() { return draft_impl<T>(h, k, h->g_draft, st); }));
+            if (k > 0) TRY(graph_call(h, {1, k, lb}, st, [&]() { return draft_impl<T>(h, k, h->g_draft, st); }));
             mark();
             h->len_ub = lb;
             TRY(graph_call(h, {2, k, lb, beta, tau_bits}, st, [&]() {
@@ -820,7 +821,7 @@ int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, con
             h->len_ub = std::min(true_ub + k + 1, h->T_cap);
             h->last_k = k; h->verified = false; h->drafted = false;
         } else {
-            TRY(draft_impl<T>(h, k, h->g_draft, st));
+            if (k > 0) TRY(draft_impl<T>(h, k, h->g_draft, st));
             mark();
             TRY(verify_impl<T>(h, h->g_draft, k, beta, tau, nullptr, nullptr, st));
             mark();
@@ -1047,6 +1048,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         return SPECDEC_OK;
     }
     if (!strcmp(name, "cl_trace")) { h->want_cl_trace = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "pdl")) { h->use_pdl = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "skinny")) { h->use_skinny = value ? 1 : 0; return SPECDEC_OK; }
@@ -1093,8 +1095,8 @@ int specdec_verify(specdec_handle* h, const int32_t* d_draft, int k, int beta, f
                    int32_t* d_bif, void* stream) {
     if (!h) return SPECDEC_ERR_INVALID_ARG;
     if (!h->encoded) return fail(h, SPECDEC_ERR_NOT_ENCODED, "verify: no session (call specdec_encode)");
-    if (!d_draft) return fail(h, SPECDEC_ERR_INVALID_ARG, "verify: null drafts");
-    if (k < 1 || k > h->k_cap) return fail(h, SPECDEC_ERR_CAPACITY, "verify: k outside [1, k_max]");
+    if (!d_draft && k > 0) return fail(h, SPECDEC_ERR_INVALID_ARG, "verify: null drafts");
+    if (k < 0 || k > h->k_cap) return fail(h, SPECDEC_ERR_CAPACITY, "verify: k outside [0, k_max]");
     if (beta < 1 || !(tau >= 0.f)) return fail(h, SPECDEC_ERR_INVALID_ARG, "verify: beta >= 1 and tau >= 0 required");
     StreamScope scope(h, stream);
     cudaStream_t st = scope.st;
@@ -1140,7 +1142,7 @@ int specdec_generate(specdec_handle* h, const int32_t* d_src, const int32_t* d_s
     if (!d_src || !d_src_len || !d_out || !d_out_len || B < 1 || S_max < 1 || out_stride < 1)
         return fail(h, SPECDEC_ERR_INVALID_ARG, "generate: bad argument");
     if (B > h->B_cap || S_max > h->S_cap) return fail(h, SPECDEC_ERR_CAPACITY, "generate: B or S_max beyond capacity");
-    if (k < 1 || k > h->k_cap) return fail(h, SPECDEC_ERR_CAPACITY, "generate: k outside [1, k_max]");
+    if (k < 0 || k > h->k_cap) return fail(h, SPECDEC_ERR_CAPACITY, "generate: k outside [0, k_max]");
     if (beta < 1 || !(tau >= 0.f)) return fail(h, SPECDEC_ERR_INVALID_ARG, "generate: beta >= 1 and tau >= 0 required");
     StreamScope scope(h, stream);
     cudaStream_t st = scope.st;
@@ -1163,7 +1165,7 @@ int specdec_generate_host(specdec_handle* h, const int32_t* h_src, const int32_t
     CUDA_TRY(h, cudaMemcpyAsync(s_src, h_src, (size_t)B * S_max * 4, cudaMemcpyHostToDevice, st));
     CUDA_TRY(h, cudaMemcpyAsync(s_len, h_src_len, (size_t)B * 4, cudaMemcpyHostToDevice, st));
     if (h_max_tgt) CUDA_TRY(h, cudaMemcpyAsync(s_mt, h_max_tgt, (size_t)B * 4, cudaMemcpyHostToDevice, st));
-    if (k < 1 || k > h->k_cap) return fail(h, SPECDEC_ERR_CAPACITY, "generate_host: k outside [1, k_max]");
+    if (k < 0 || k > h->k_cap) return fail(h, SPECDEC_ERR_CAPACITY, "generate_host: k outside [0, k_max]");
     if (beta < 1 || !(tau >= 0.f)) return fail(h, SPECDEC_ERR_INVALID_ARG, "generate_host: beta >= 1 and tau >= 0 required");
     // the ids and lengths are read straight from the session arrays afterwards
     const int* mt = h_max_tgt ? s_mt : nullptr;

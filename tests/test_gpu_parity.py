@@ -88,6 +88,18 @@ def test_config1_generate_bit_exact(tiny, beta, tau, graphs):
     sd.close()
 
 
+def test_k0_is_greedy_autoregressive_decoding(tiny):
+    """k = 0 runs the verifier alone, one row per step: the greedy baseline of the paper's comparisons."""
+    wl, wv, wd, mv, md = tiny
+    sd = _handle(wl.verifier, wv, wl.drafter, wd, False)
+    src, lens = W.pad_batch(wl.src)
+    out, n, st = sd.generate(src, lens, wl.max_tgt, 0, 1, 0.0)
+    for b, s in enumerate(wl.src):
+        assert out[b, :int(n[b])].cpu().tolist() == O.greedy_decode(mv, s, 32, BOS, EOS)
+    assert st["drafted"] == 0 and st["accepted"] == 0 and st["emitted"] == int(n.sum()) == st["seq_iterations"]
+    sd.close()
+
+
 def test_tiny_lockstep_logits_and_stats(tiny):
     wl, wv, wd, mv, md = tiny
     sd = _handle(wl.verifier, wv, wl.drafter, wd, False)
