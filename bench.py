@@ -56,6 +56,13 @@ def workload(batch: int):
     return wl, name
 
 
+def config_of(name: str, batch: int, world: int) -> dict:
+    return {"workload": name, "batch": batch, "k": K_BLOCK, "beta": BETA, "tau": TAU,
+            "acceptance": f"scripted: greedy continuation, rejection every Geometric(mean {GEO_MEAN:g}) positions",
+            "l2": "each step streams 248 MB of bf16 weights (both models) > 126 MB L2; no explicit flush",
+            "parallelism": f"replicas x{world}"}
+
+
 def make_script(greedy: np.ndarray, n: int, rng: np.random.Generator, vocab: int, width: int) -> np.ndarray:
     """Greedy continuation with a token the verifier rejects every Geometric(mean 6) positions."""
     s = np.full(width, -1, np.int32)
@@ -163,7 +170,7 @@ def run_reference(args):
         "impl": "reference", "metric": "generated tokens/s", "value": v, "unit": "tokens/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / max(args.steps, 1),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": name, "k": K_BLOCK, "beta": BETA, "tau": TAU, "batch": 1},
+        "config": config_of(name, 1, 1),
         "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": cores_used(), "kind": "oracle", "sample": sample},
         "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -311,10 +318,7 @@ def run_ours(args):
         "metric": "generated tokens/s", "value": toks_all / (ms_max * 1e-3), "unit": "tokens/s",
         "n_gpus": world, "steps": K_, "warmup": W_, "ms_per_step": ms_max / max(K_, 1),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": name, "batch": B, "k": K_BLOCK, "beta": BETA, "tau": TAU,
-                   "acceptance": f"scripted: greedy continuation, rejection every Geometric(mean {GEO_MEAN:g}) positions",
-                   "l2": "each step streams 248 MB of bf16 weights (both models) > 126 MB L2; no explicit flush",
-                   "parallelism": f"replicas x{world}"},
+        "config": config_of(name, B, world),
         "e2e": {"value": e_toks_all / (e_ms_max * 1e-3), "unit": "tokens/s",
                 "h2d_bytes_per_step": int(B * max_src * 4 + B * 8), "d2h_bytes_per_step": int(B * max_tgt * 4 + B * 4)},
         "gpu_launches": int(launches),

@@ -31,38 +31,41 @@ __device__ __forceinline__ void sk_stamp(long long* trace, int slot) {
     if (trace && blockIdx.x == 0 && threadIdx.x == 0) { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); trace[slot] = t; }
 }
 
-constexpr int SK_NB = 8;         // weight rows per CTA
+constexpr int SK_NB = 8;         // weight rows per 8-row group
 constexpr int SK_WARPS = 8;
+// G groups of 8 weight rows per CTA; the 8 warps are G groups x (8 / G) K-splits
 inline size_t skinny_smem(int MT, int K) { return (size_t)MT * 16 * (K + 8) * 2 + (size_t)SK_WARPS * MT * 16 * SK_NB * 4; }
 
-template <int EPI, int MT, bool LN>
+template <int EPI, int MT, bool LN, int G>
 __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
     extern __shared__ __align__(16) unsigned char sk_sm[];
     const GemmArgs<bf16>& g = a.g;
     const int K = g.K, N = g.N;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t4 = lane & 3;
     sk_stamp(a.trace, 0);
-    const int n0 = blockIdx.x * SK_NB;
+    constexpr int SPL = SK_WARPS / G;                          // K-splits per group
+    const int grp = warp % G, spl = warp / G;
+    const int n0 = blockIdx.x * (SK_NB * G);                  // first weight row of this CTA
     const int pitch = K + 8;                                  // bf16 elements per activation row in shared memory
     bf16* As = reinterpret_cast<bf16*>(sk_sm);
     float* red = reinterpret_cast<float*>(sk_sm + (size_t)MT * 16 * pitch * 2);
 
     // K split: warp s takes k in [s * ks, (s + 1) * ks), in super-steps of 32
-    const int nsplit = min(SK_WARPS, K / 32);
+    const int nsplit = min(SPL, K / 32);
     const int ks = (K / 32 + nsplit - 1) / nsplit * 32;
-    const int k_begin = warp * ks, k_end = min(K, k_begin + ks);
+    const int k_begin = spl * ks, k_end = min(K, k_begin + ks);
     constexpr int MAX_SS = 8;                                 // super-steps whose weights are preloaded in registers
     uint4 wreg[MAX_SS];
-    const bool w_ok = (n0 + gq) < N;
-    const bf16* wrow = g.W + (size_t)(n0 + gq) * K + t4 * 8;
+    const bool w_ok = (n0 + grp * SK_NB + gq) < N;
+    const bf16* wrow = g.W + (size_t)(n0 + grp * SK_NB + gq) * K + t4 * 8;
 #pragma unroll
     for (int ss = 0; ss < MAX_SS; ++ss) {
         const int k0 = k_begin + ss * 32;
-        wreg[ss] = (w_ok && warp < nsplit && k0 < k_end) ? __ldg(reinterpret_cast<const uint4*>(wrow + k0)) : make_uint4(0, 0, 0, 0);
+        wreg[ss] = (w_ok && spl < nsplit && k0 < k_end) ? __ldg(reinterpret_cast<const uint4*>(wrow + k0)) : make_uint4(0, 0, 0, 0);
     }
 
     // bias and LayerNorm parameters are weights too: fetch them before waiting for the predecessor
-    const float bias_v = (g.bias && n0 + (tid & 7) < N) ? __ldg(g.bias + n0 + (tid & 7)) : 0.f;
+    const float bias_v = (g.bias && n0 + (tid % (SK_NB * G)) < N) ? __ldg(g.bias + n0 + (tid % (SK_NB * G))) : 0.f;
     float4 lgam[4], lbet[4];
     if (LN) {
 #pragma unroll
@@ -152,7 +155,7 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[mt][e] = 0.f;
-    if (warp < nsplit) {
+    if (spl < nsplit) {
         auto step = [&](const uint4& w, int k0) {
             const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
@@ -188,16 +191,16 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
     // ---- fixed-order sum over the K split, then the epilogue
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
-        float* r0 = red + ((size_t)warp * MT * 16 + mt * 16 + gq) * SK_NB + t4 * 2;
+        float* r0 = red + ((size_t)spl * MT * 16 + mt * 16 + gq) * (SK_NB * G) + grp * SK_NB + t4 * 2;
         r0[0] = acc[mt][0]; r0[1] = acc[mt][1];
-        r0[8 * SK_NB] = acc[mt][2]; r0[8 * SK_NB + 1] = acc[mt][3];
+        r0[8 * SK_NB * G] = acc[mt][2]; r0[8 * SK_NB * G + 1] = acc[mt][3];
     }
     __syncthreads();
-    for (int o = tid; o < MT * 16 * SK_NB; o += SK_WARPS * 32) {
-        const int r = o / SK_NB, n = n0 + (o % SK_NB);
+    for (int o = tid; o < MT * 16 * SK_NB * G; o += SK_WARPS * 32) {
+        const int r = o / (SK_NB * G), n = n0 + (o % (SK_NB * G));
         if (r >= R || n >= N) continue;
         float v = 0.f;
-        for (int s = 0; s < nsplit; ++s) v += red[(size_t)s * MT * 16 * SK_NB + o];
+        for (int s = 0; s < nsplit; ++s) v += red[(size_t)s * MT * 16 * SK_NB * G + o];
         v += bias_v;
         if (EPI == EPI_STORE) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(v);
         if (EPI == EPI_RELU) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(fmaxf(v, 0.f));

@@ -89,6 +89,7 @@ struct specdec_handle {
     long long* cl_trace = nullptr;   // device [256] timestamps of the cluster kernel's phases (option "cl_trace")
     int want_cl_trace = 0;
     size_t skinny_smem_cap = 0;
+    int skinny_groups = 1;          // 8-row weight groups per CTA of the weight-streaming GEMM (1, 2 or 4)
     // CUDA graphs of whole draft / verify(+commit) steps, keyed by everything their launches depend on
     struct GraphEntry { cudaGraphExec_t exec; long long kernels; };
     std::map<std::vector<long long>, GraphEntry> graphs;
@@ -345,15 +346,23 @@ cudaError_t launch_pdl(specdec_handle* h, void (*kernel)(KArgs...), dim3 grid, d
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
-template <int EPI, int MT>
-int skinny_launch_ln(specdec_handle* h, SkinnyArgs& a, cudaStream_t st) {
-    const int grid = cdiv(a.g.N, SK_NB);
+template <int EPI, int MT, int G>
+int skinny_launch_g(specdec_handle* h, SkinnyArgs& a, cudaStream_t st) {
+    const int grid = cdiv(a.g.N, SK_NB * G);
     const size_t smem = skinny_smem(MT, a.g.K);
-    cudaError_t e = a.ln_x ? launch_pdl(h, k_skinny<EPI, MT, true>, dim3(grid), dim3(SK_WARPS * 32), smem, st, a)
-                           : launch_pdl(h, k_skinny<EPI, MT, false>, dim3(grid), dim3(SK_WARPS * 32), smem, st, a);
+    cudaError_t e = a.ln_x ? launch_pdl(h, k_skinny<EPI, MT, true, G>, dim3(grid), dim3(SK_WARPS * 32), smem, st, a)
+                           : launch_pdl(h, k_skinny<EPI, MT, false, G>, dim3(grid), dim3(SK_WARPS * 32), smem, st, a);
     if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("skinny GEMM launch: ") + cudaGetErrorString(e));
     KCHECK(h);
     return 0;
+}
+template <int EPI, int MT>
+int skinny_launch_ln(specdec_handle* h, SkinnyArgs& a, cudaStream_t st) {
+    switch (h->skinny_groups) {
+        case 4: return skinny_launch_g<EPI, MT, 4>(h, a, st);
+        case 2: return skinny_launch_g<EPI, MT, 2>(h, a, st);
+        default: return skinny_launch_g<EPI, MT, 1>(h, a, st);
+    }
 }
 template <int EPI>
 int skinny_launch_mt(specdec_handle* h, SkinnyArgs& a, int rows_ub, cudaStream_t st) {
@@ -369,8 +378,11 @@ int skinny_launch(specdec_handle* h, int epi, SkinnyArgs& a, int rows_ub, cudaSt
 }
 template <int EPI, int MT>
 cudaError_t skinny_attr(int bytes) {
-    cudaError_t e = cudaFuncSetAttribute(k_skinny<EPI, MT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_skinny<EPI, MT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaError_t e = cudaSuccess;
+    auto set = [&](auto* f) { if (e == cudaSuccess) e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes); };
+    set(k_skinny<EPI, MT, true, 1>); set(k_skinny<EPI, MT, false, 1>);
+    set(k_skinny<EPI, MT, true, 2>); set(k_skinny<EPI, MT, false, 2>);
+    set(k_skinny<EPI, MT, true, 4>); set(k_skinny<EPI, MT, false, 4>);
     return e;
 }
 template <int EPI>
@@ -747,7 +759,7 @@ void drop_graphs(specdec_handle* h) {
 // replayed afterwards.  The key must name everything the launches depend on besides device memory.
 template <typename F>
 int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body) {
-    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
+    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
     key.push_back(h->B); key.push_back(h->S_max);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
@@ -1048,6 +1060,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         return SPECDEC_OK;
     }
     if (!strcmp(name, "cl_trace")) { h->want_cl_trace = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "skinny_groups")) { h->skinny_groups = (value == 2 || value == 4) ? value : 1; return SPECDEC_OK; }
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "pdl")) { h->use_pdl = value ? 1 : 0; return SPECDEC_OK; }
