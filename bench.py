@@ -202,6 +202,8 @@ def run_ours(args):
     sd = binding.SpecDec(wl.verifier, wv, wl.drafter, wd, k_max=K_BLOCK, max_batch=B, max_src=max_src,
                          max_tgt=max_tgt, bf16=True, device=f"cuda:{local}")
     del wv, wd
+    if args.poll_lag is not None:
+        sd.set_option("poll_lag", args.poll_lag)
 
     # the step stream: rank r takes batches r, r + world, ... (replicas; no data-path collective)
     n_total = args.warmup + args.steps
@@ -361,6 +363,7 @@ def main():
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--poll-lag", type=int, default=None, help="experiments: iterations the host runs ahead of the finish counter")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

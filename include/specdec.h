@@ -206,6 +206,8 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
  * "cluster" = 0/1 run the verifier's decoder stack as one thread-block-cluster kernel per sequence when the
  *   batch is at most 8, k + 1 <= 32 and the model has 8 heads of 64 (default 0: measured slower than the
  *   per-operation kernels, kept for comparison);
+ * "poll_lag" = n: specdec_generate reads the unfinished-sequences counter n iterations late (0: waits for it
+ *   after every iteration; default 0 up to batch 4, else 2);
  * "pdl" = 0/1 programmatic dependent launch between the kernels of a step (default 1);
  * "attn" = 0 warp-per-row reference attention, 1 tensor-core tile attention (bf16, 64-wide heads; default 1);
  * "graphs" = 0/1 replay draft/verify steps from CUDA graphs inside specdec_generate;

@@ -89,6 +89,7 @@ struct specdec_handle {
     long long* cl_trace = nullptr;   // device [256] timestamps of the cluster kernel's phases (option "cl_trace")
     int want_cl_trace = 0;
     size_t skinny_smem_cap = 0;
+    int poll_lag = -1;              // -1: chosen by batch size
     int skinny_groups = 1;          // 8-row weight groups per CTA of the weight-streaming GEMM (1, 2 or 4)
     // CUDA graphs of whole draft / verify(+commit) steps, keyed by everything their launches depend on
     struct GraphEntry { cudaGraphExec_t exec; long long kernels; };
@@ -329,7 +330,7 @@ bool skinny_ok(const specdec_handle* h, int epi, int rows_ub, int N, int K, bool
     if (!std::is_same<T, bf16>::value || !h->use_skinny || rows_ub > 64) return false;
     if (epi != EPI_STORE && epi != EPI_RELU && epi != EPI_RESID && epi != EPI_QKV) return false;
     if (K % 32 || (with_ln && (K % 128 || K > 512))) return false;
-    return skinny_smem(rows_ub <= 32 ? 2 : 4, K) <= h->skinny_smem_cap;
+    return skinny_smem(rows_ub <= 32 ? 2 : (rows_ub <= 48 ? 3 : 4), K) <= h->skinny_smem_cap;
 }
 
 // Launch that lets the kernel start before its predecessor in the stream has finished (the kernel itself
@@ -358,15 +359,12 @@ int skinny_launch_g(specdec_handle* h, SkinnyArgs& a, cudaStream_t st) {
 }
 template <int EPI, int MT>
 int skinny_launch_ln(specdec_handle* h, SkinnyArgs& a, cudaStream_t st) {
-    switch (h->skinny_groups) {
-        case 4: return skinny_launch_g<EPI, MT, 4>(h, a, st);
-        case 2: return skinny_launch_g<EPI, MT, 2>(h, a, st);
-        default: return skinny_launch_g<EPI, MT, 1>(h, a, st);
-    }
+    return skinny_launch_g<EPI, MT, 1>(h, a, st);
 }
 template <int EPI>
 int skinny_launch_mt(specdec_handle* h, SkinnyArgs& a, int rows_ub, cudaStream_t st) {
-    return rows_ub <= 32 ? skinny_launch_ln<EPI, 2>(h, a, st) : skinny_launch_ln<EPI, 4>(h, a, st);
+    return rows_ub <= 32 ? skinny_launch_ln<EPI, 2>(h, a, st)
+         : rows_ub <= 48 ? skinny_launch_ln<EPI, 3>(h, a, st) : skinny_launch_ln<EPI, 4>(h, a, st);
 }
 int skinny_launch(specdec_handle* h, int epi, SkinnyArgs& a, int rows_ub, cudaStream_t st) {
     switch (epi) {
@@ -381,13 +379,12 @@ cudaError_t skinny_attr(int bytes) {
     cudaError_t e = cudaSuccess;
     auto set = [&](auto* f) { if (e == cudaSuccess) e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes); };
     set(k_skinny<EPI, MT, true, 1>); set(k_skinny<EPI, MT, false, 1>);
-    set(k_skinny<EPI, MT, true, 2>); set(k_skinny<EPI, MT, false, 2>);
-    set(k_skinny<EPI, MT, true, 4>); set(k_skinny<EPI, MT, false, 4>);
     return e;
 }
 template <int EPI>
 cudaError_t skinny_attr_mt(int bytes) {
     cudaError_t e = skinny_attr<EPI, 2>(bytes);
+    if (e == cudaSuccess) e = skinny_attr<EPI, 3>(bytes);
     if (e == cudaSuccess) e = skinny_attr<EPI, 4>(bytes);
     return e;
 }
@@ -813,7 +810,9 @@ int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, con
     TRY(encode_staged<T>(h, d_src, d_src_len, d_max_tgt, B, S_max, st));
     mark();
     const int max_iters = h->T_cap;            // every iteration commits >= 1 token per unfinished sequence
-    const int lag = 2, slots = (int)h->poll_ev.size();
+    // how many iterations the host runs ahead of the "unfinished sequences" counter it reads back: every iteration
+    // launched after the last sequence finished is wasted work, every wait for the counter is a bubble
+    const int lag = h->poll_lag >= 0 ? h->poll_lag : (B <= 4 ? 0 : 2), slots = (int)h->poll_ev.size();
     int it = 0;
     const bool graphs = h->use_graphs && !h->profile;
     int tau_bits; memcpy(&tau_bits, &tau, 4);
@@ -1060,7 +1059,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         return SPECDEC_OK;
     }
     if (!strcmp(name, "cl_trace")) { h->want_cl_trace = value ? 1 : 0; return SPECDEC_OK; }
-    if (!strcmp(name, "skinny_groups")) { h->skinny_groups = (value == 2 || value == 4) ? value : 1; return SPECDEC_OK; }
+    if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "pdl")) { h->use_pdl = value ? 1 : 0; return SPECDEC_OK; }
