@@ -62,8 +62,11 @@ struct specdec_handle {
     // capacities
     int B_cap, S_cap, T_cap, k_cap, R_cap, R2_cap, M_cap, d_max, f_max, v_max, pages_per_seq, n_tiles_cap;
     // activations
-    float *x, *x2;
+    float *x, *x2;                          // the workspace in use (one of ws[0], ws[1])
     void *y, *qkv, *att, *q, *hbuf, *mem;
+    struct WorkSet { float* x; void *y, *qkv, *att, *q, *hbuf, *mem; } ws[2];   // ws[1]: second encoder, own stream
+    cudaStream_t enc_stream = nullptr;
+    cudaEvent_t enc_fork = nullptr, enc_join = nullptr;
     // verifier KV cache
     std::vector<void*> kc, vc;
     int* page_table;
@@ -203,6 +206,13 @@ void layout_all(specdec_handle* h) {
     h->q = A.take(R * d * e);
     h->hbuf = A.take(R * f * e);
     h->mem = A.take((size_t)h->B_cap * h->S_cap * d * e);
+    h->ws[0] = {h->x, h->y, h->qkv, h->att, h->q, h->hbuf, h->mem};
+    {   // a second, encoder-sized workspace so the two encoders can run side by side
+        const size_t Re = (size_t)h->B_cap * h->S_cap;
+        specdec_handle::WorkSet& w = h->ws[1];
+        w.x = (float*)A.take(Re * d * 4); w.y = A.take(Re * d * e); w.qkv = A.take(Re * 3 * d * e); w.att = A.take(Re * d * e);
+        w.q = A.take(Re * d * e); w.hbuf = A.take(Re * f * e); w.mem = A.take(Re * d * e);
+    }
     const size_t cache_rows = (size_t)h->B_cap * h->pages_per_seq * h->cfg.page_tokens;
     h->kc.resize(h->cfg.verifier.dec_layers);
     h->vc.resize(h->cfg.verifier.dec_layers);
@@ -574,11 +584,14 @@ int embed(specdec_handle* h, const ModelW& m, const Rows& r, const float* pos_ta
 }
 
 // ---------------------------------------------------------------- encode
+void use_workset(specdec_handle* h, int i) {
+    const specdec_handle::WorkSet& w = h->ws[i];
+    h->x = w.x; h->y = w.y; h->qkv = w.qkv; h->att = w.att; h->q = w.q; h->hbuf = w.hbuf; h->mem = w.mem;
+}
+
 template <typename T>
-int encode_model(specdec_handle* h, ModelW& m, const int* d_src, cudaStream_t st) {
+int encode_model(specdec_handle* h, ModelW& m, cudaStream_t st) {
     const int R = h->B * h->S_max, d = m.dm.d_model;
-    k_enc_prep<<<cdiv(R, 256), 256, 0, st>>>(d_src, h->ses.src_len, h->B, h->S_max, h->rows, h->ses.counters);
-    KCHECK(h);
     TRY(embed<T>(h, m, h->rows, m.pos_enc, CNT_ENC, R, st));
     for (int l = 0; l < m.dm.enc_layers; ++l) {
         TRY(block_self<T>(h, m, m.enc[l], h->x, h->rows, CNT_ENC, R, h->S_max, l, false, h->S_max, st));
@@ -600,8 +613,29 @@ int encode_impl(specdec_handle* h, const int* d_src, const int* d_src_len, const
     KCHECK(h);
     k_count_active<<<1, 32, 0, st>>>(h->ses, B);
     KCHECK(h);
-    TRY(encode_model<T>(h, h->ver, d_src, st));
-    TRY(encode_model<T>(h, h->dra, d_src, st));
+    {
+        const int R = B * S_max;
+        k_enc_prep<<<cdiv(R, 256), 256, 0, st>>>(d_src, h->ses.src_len, B, S_max, h->rows, h->ses.counters);
+        KCHECK(h);
+    }
+    // the two encoders are independent: the drafter's runs on a second stream in its own workspace
+    const bool side = h->enc_stream != nullptr;
+    cudaStream_t st2 = side ? h->enc_stream : st;
+    if (side) {
+        CUDA_TRY(h, cudaEventRecord(h->enc_fork, st));
+        CUDA_TRY(h, cudaStreamWaitEvent(st2, h->enc_fork, 0));
+    }
+    int rc = encode_model<T>(h, h->ver, st);
+    if (rc == 0) {
+        if (side) use_workset(h, 1);
+        rc = encode_model<T>(h, h->dra, st2);
+        use_workset(h, 0);
+    }
+    if (side) {
+        cudaEventRecord(h->enc_join, st2);
+        cudaStreamWaitEvent(st, h->enc_join, 0);
+    }
+    if (rc != 0) return rc;
     h->encoded = true;
     return 0;
 }
@@ -967,6 +1001,9 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
     if (cudaMallocHost((void**)&h->h_poll, 64 * 4) != cudaSuccess || cudaMallocHost((void**)&h->h_stats, 64) != cudaSuccess)
         return bail(SPECDEC_ERR_CUDA, "pinned host allocation failed");
     cudaStreamCreateWithFlags(&h->own_stream, cudaStreamNonBlocking);
+    cudaStreamCreateWithFlags(&h->enc_stream, cudaStreamNonBlocking);
+    cudaEventCreateWithFlags(&h->enc_fork, cudaEventDisableTiming);
+    cudaEventCreateWithFlags(&h->enc_join, cudaEventDisableTiming);
     cudaEventCreateWithFlags(&h->fence_in, cudaEventDisableTiming);
     cudaEventCreateWithFlags(&h->fence_out, cudaEventDisableTiming);
     h->poll_ev.resize(8);
@@ -1037,6 +1074,9 @@ int specdec_destroy(specdec_handle* h) {
     cudaDeviceSynchronize();
     drop_graphs(h);
     if (h->own_stream) cudaStreamDestroy(h->own_stream);
+    if (h->enc_stream) cudaStreamDestroy(h->enc_stream);
+    if (h->enc_fork) cudaEventDestroy(h->enc_fork);
+    if (h->enc_join) cudaEventDestroy(h->enc_join);
     if (h->fence_in) cudaEventDestroy(h->fence_in);
     if (h->fence_out) cudaEventDestroy(h->fence_out);
     for (auto& e : h->poll_ev) cudaEventDestroy(e);
