@@ -208,6 +208,9 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
  *   per-operation kernels, kept for comparison);
  * "poll_lag" = n: specdec_generate reads the unfinished-sequences counter n iterations late (0: waits for it
  *   after every iteration; default 0 up to batch 4, else 2);
+ * "fused_attn" = 0/1 attention + output projection + residual as one 8-CTA-cluster kernel per sequence for
+ *   blocks of at most 32 query rows and models with 8 heads of 64 (default 0: measured slower than the two
+ *   separate kernels at batch 1 and at batch 128, kept for comparison);
  * "pdl" = 0/1 programmatic dependent launch between the kernels of a step (default 1);
  * "attn" = 0 warp-per-row reference attention, 1 tensor-core tile attention (bf16, 64-wide heads; default 1);
  * "graphs" = 0/1 replay draft/verify steps from CUDA graphs inside specdec_generate;

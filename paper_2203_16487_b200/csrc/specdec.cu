@@ -14,6 +14,7 @@
 #include <vector>
 
 #include "../../include/specdec.h"
+#include "attention_oproj.cuh"
 #include "attention_tc.cuh"
 #include "decoder_cluster.cuh"
 #include "gemm_tc.cuh"
@@ -93,6 +94,8 @@ struct specdec_handle {
     int want_cl_trace = 0;
     size_t skinny_smem_cap = 0;
     int poll_lag = -1;              // -1: chosen by batch size
+    int use_fused_attn = 0;         // attention + output projection as one cluster kernel (measured slower: off)
+    size_t attn_proj_smem_cap = 0;
     int skinny_groups = 1;          // 8-row weight groups per CTA of the weight-streaming GEMM (1, 2 or 4)
     // CUDA graphs of whole draft / verify(+commit) steps, keyed by everything their launches depend on
     struct GraphEntry { cudaGraphExec_t exec; long long kernels; };
@@ -513,6 +516,40 @@ void prof_collect(specdec_handle* h) {
     h->prof_n = 0;
 }
 
+// Attention + output projection + residual as one 8-CTA-cluster kernel per sequence (see attention_oproj.cuh).
+// Returns 1 if it was launched, 0 if the shapes do not qualify, < 0 on error.
+template <typename T>
+int fused_attn_proj(specdec_handle* h, bool paged, const void* q, int q_stride, const int* q_index, const void* k,
+                    const void* v, int kv_stride, const int* kv_off, const Rows& r, const int* nkeys, int q_ub,
+                    int n_heads, int d_head, int max_keys, const void* wo, const float* bo, float* x, int d, cudaStream_t st) {
+    if constexpr (!std::is_same<T, bf16>::value) return 0;
+    else {
+        if (!h->use_fused_attn || !h->use_tc_attn || n_heads != AP_HEADS || d_head != 64 || d != AP_HEADS * 64 || q_ub > ATT_Q) return 0;
+        const size_t smem = attn_proj_smem(max_keys, d);
+        if (smem > h->attn_proj_smem_cap) return 0;
+        AttnProjArgs p;
+        AttnTcArgs& a = p.at;
+        a.q = (const bf16*)q; a.q_stride = q_stride; a.q_index = q_index;
+        a.k = (const bf16*)k; a.v = (const bf16*)v; a.kv_stride = kv_stride; a.kv_off = kv_off;
+        a.pg.table = h->page_table; a.pg.page_tokens = h->cfg.page_tokens; a.pg.max_pages = h->pages_per_seq;
+        a.q_off = r.q_off; a.q_cnt = r.q_cnt; a.nkeys = nkeys; a.out = nullptr; a.out_stride = 0; a.max_keys = max_keys;
+        a.scale = 1.0f / sqrtf((float)d_head);
+        p.wo = (const bf16*)wo; p.bo = bo; p.x = x; p.d = d;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(AP_HEADS, h->B); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = AP_HEADS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = h->use_pdl ? 2 : 1;
+        cudaError_t e = paged ? cudaLaunchKernelEx(&cfg, k_attn_proj<true>, p) : cudaLaunchKernelEx(&cfg, k_attn_proj<false>, p);
+        if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("attention+projection launch: ") + cudaGetErrorString(e));
+        KCHECK(h);
+        return 1;
+    }
+}
+
 // One pre-LN block on `rows_ub` rows of the residual stream x (encoder: no cross-attention).
 // Self-attention keys come from the block's own QKV rows (contiguous) or, for the verifier,
 // from the paged cache after the block's K/V were scattered into it.
@@ -538,6 +575,10 @@ int block_self(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, co
         }
     }
     if (verify) {
+        const int f = fused_attn_proj<T>(h, true, h->qkv, 3 * d, nullptr, h->kc[layer], h->vc[layer], d, nullptr, r, r.nk_self,
+                                         q_ub, H, dh, max_keys, w.o_w, w.o_b, x, d, st);
+        if (f < 0) return f;
+        if (f == 1) return 0;
         TRY(attn<T>(h, true, h->qkv, 3 * d, nullptr, h->kc[layer], h->vc[layer], d, nullptr, r, r.nk_self, cnt,
                     rows_ub, q_ub, h->att, d, H, dh, max_keys, st));
     } else {
@@ -556,6 +597,12 @@ int block_cross(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, c
     const LnSpec lc{x, w.lnc_g, w.lnc_b};
     TRY(gemm<T>(h, EPI_STORE, h->y, d, w.cq_w, w.cq_b, d, d, cnt, rows_ub, h->q, d, nullptr, st, nullptr, nullptr, nullptr,
                 nullptr, &lc));
+    {
+        const int f = fused_attn_proj<T>(h, false, h->q, d, nullptr, m.ckv[layer], (char*)m.ckv[layer] + (size_t)d * e, 2 * d,
+                                         r.kv_off_cross, r, r.nk_cross, q_ub, H, dh, h->S_max, w.co_w, w.co_b, x, d, st);
+        if (f < 0) return f;
+        if (f == 1) return 0;
+    }
     TRY(attn<T>(h, false, h->q, d, nullptr, m.ckv[layer], (char*)m.ckv[layer] + (size_t)d * e, 2 * d, r.kv_off_cross,
                 r, r.nk_cross, cnt, rows_ub, q_ub, h->att, d, H, dh, h->S_max, st));
     TRY(gemm<T>(h, EPI_RESID, h->att, d, w.co_w, w.co_b, d, d, cnt, rows_ub, nullptr, 0, x, st));
@@ -664,10 +711,18 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
                 nullptr, nullptr, nullptr, &l1));
     k_gather_rows<<<R2, 128, 0, st>>>(h->x, h->mrows.src_row, h->ses.counters + CNT_DRAFT_MASK, h->x2, d);
     KCHECK(h);
-    TRY(attn<T>(h, false, h->qkv, 3 * d, h->mrows.src_row, (char*)h->qkv + (size_t)d * e,
-                (char*)h->qkv + (size_t)2 * d * e, 3 * d, h->mrows.kv_off, h->mrows, h->mrows.nk_self,
-                CNT_DRAFT_MASK, R2, k, h->att, d, H, dh, max_keys, st));
-    TRY(gemm<T>(h, EPI_RESID, h->att, d, w.o_w, w.o_b, d, d, CNT_DRAFT_MASK, R2, nullptr, 0, h->x2, st));
+    {
+        const int f = fused_attn_proj<T>(h, false, h->qkv, 3 * d, h->mrows.src_row, (char*)h->qkv + (size_t)d * e,
+                                         (char*)h->qkv + (size_t)2 * d * e, 3 * d, h->mrows.kv_off, h->mrows, h->mrows.nk_self, k,
+                                         H, dh, max_keys, w.o_w, w.o_b, h->x2, d, st);
+        if (f < 0) return f;
+        if (f == 0) {
+            TRY(attn<T>(h, false, h->qkv, 3 * d, h->mrows.src_row, (char*)h->qkv + (size_t)d * e,
+                        (char*)h->qkv + (size_t)2 * d * e, 3 * d, h->mrows.kv_off, h->mrows, h->mrows.nk_self,
+                        CNT_DRAFT_MASK, R2, k, h->att, d, H, dh, max_keys, st));
+            TRY(gemm<T>(h, EPI_RESID, h->att, d, w.o_w, w.o_b, d, d, CNT_DRAFT_MASK, R2, nullptr, 0, h->x2, st));
+        }
+    }
     TRY(block_cross<T>(h, m, w, h->x2, h->mrows, CNT_DRAFT_MASK, R2, k, L - 1, st));
     TRY(block_ffn<T>(h, m, w, h->x2, CNT_DRAFT_MASK, R2, st));
     TRY(ln<T>(h, h->x2, m.dec_lnf_g, m.dec_lnf_b, CNT_DRAFT_MASK, R2, h->y, d, st));
@@ -790,7 +845,7 @@ void drop_graphs(specdec_handle* h) {
 // replayed afterwards.  The key must name everything the launches depend on besides device memory.
 template <typename F>
 int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body) {
-    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
+    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->use_fused_attn); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
     key.push_back(h->B); key.push_back(h->S_max);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
@@ -1060,6 +1115,16 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
             h->cl_ok = (e == cudaSuccess);
             if (!h->cl_ok) cudaGetLastError();
         }
+        {
+            const int max_keys = std::max(h->S_cap, h->T_cap + h->k_cap + 1);
+            size_t cap = std::min<size_t>(attn_proj_smem(max_keys, cfg->verifier.d_model), 227 * 1024);
+            if (cudaFuncSetAttribute(k_attn_proj<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cap) != cudaSuccess ||
+                cudaFuncSetAttribute(k_attn_proj<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cap) != cudaSuccess) {
+                cudaGetLastError();
+                cap = 0;
+            }
+            h->attn_proj_smem_cap = cap;
+        }
         if (sd::tc_init(h->tma, h->ses.counters + 7) != 0) h->use_tc = 0;     // reported through specdec_last_error; SIMT GEMM still runs on the GPU
         if (!h->use_tc) h->err = "tensor-core GEMM unavailable: " + h->tma.err;
     } else {
@@ -1099,6 +1164,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         return SPECDEC_OK;
     }
     if (!strcmp(name, "cl_trace")) { h->want_cl_trace = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "fused_attn")) { h->use_fused_attn = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }

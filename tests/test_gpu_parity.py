@@ -278,16 +278,18 @@ def test_bf16_mid_small_batches_weight_streaming_gemm(nseq, skinny):
     sd.close()
 
 
-@pytest.mark.parametrize("cluster", [1, 0])
-def test_base_shapes_batch1_lockstep(cluster):
+@pytest.mark.parametrize("cluster,fused", [(1, 0), (0, 0), (0, 1)])
+def test_base_shapes_batch1_lockstep(cluster, fused):
     """One config-2 sentence at batch 1 (26-row verify block): the decoder stack as one cluster kernel
-    (cluster = 1) or as per-operation kernels with the weight-streaming GEMM (cluster = 0)."""
+    (cluster = 1) or as per-operation kernels with the weight-streaming GEMM (cluster = 0), optionally with
+    attention and its output projection fused into one cluster kernel (fused = 1)."""
     wl = W.config2_translation(1)
     wv = W.make_weights(wl.verifier, wl.seed_verifier, True)
     wd = W.make_weights(wl.drafter, wl.seed_drafter, True)
     mv, md = O.model_from(wl.verifier, wv, mode="bf16"), O.model_from(wl.drafter, wd, mode="bf16")
     sd = _handle(wl.verifier, wv, wl.drafter, wd, True, k_max=25, max_batch=1, max_src=40, max_tgt=64)
     sd.set_option("cluster", cluster)
+    sd.set_option("fused_attn", fused)
     rep = lockstep.run(sd, mv, md, wl.src, wl.max_tgt, 25, 3, 1.0, margin=1e-3, check_logits_every=4, max_iters=8)
     print(rep.iterations, rep.draft_positions, rep.draft_near_ties, rep.verify_rows, rep.verify_near_ties,
           rep.max_logit_err, rep.max_stat_err, rep.notes[:5])
