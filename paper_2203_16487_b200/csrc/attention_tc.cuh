@@ -21,6 +21,8 @@ struct AttnTcArgs {
     Paged pg;                                             // paged: row pg.row(b, t)
     const int* q_off; const int* q_cnt;                   // per sequence: first query row, number of query rows
     const int* nkeys;                                     // per query row: visible keys (0..nkeys-1)
+    const int* pre_keys;                                  // per sequence (or null): keys 0..pre-1 were written before this
+                                                          // step began, so they may be fetched before the dependency wait
     bf16* out; int out_stride;
     int max_keys;                                         // capacity the shared memory was sized for
     float scale;
@@ -58,8 +60,8 @@ __global__ void __launch_bounds__(128) k_attn_tc(AttnTcArgs a) {
     __shared__ float s_sum[ATT_Q];
     __shared__ int s_nkmax;
     const int b = blockIdx.z, h = blockIdx.y, qt = blockIdx.x;
-    pdl_launch_dependents();
-    pdl_wait();                                   // everything this kernel reads was written by its predecessors
+    // Row metadata, page table and sequence lengths are written at the start of the step, before the first
+    // kernel of the programmatic-launch chain can begin, so they may be read before the dependency wait.
     const int cnt = a.q_cnt[b];
     if (qt * ATT_Q >= cnt) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -84,7 +86,17 @@ __global__ void __launch_bounds__(128) k_attn_tc(AttnTcArgs a) {
     const int sstr = nkp + 4;                    // fp32 row pitch of S
     const int pstr = nkp + 8;                    // bf16 row pitch of P (lives where K was)
 
-    // ---- stage Q, K, V
+    // ---- stage K, V of the keys that predate this step (cached prefix, encoder memory) before the wait ...
+    const int npre = a.pre_keys ? min(a.pre_keys[b], nkmax) : 0;
+    for (int i = tid; i < npre * 8; i += 128) {
+        const int t = i >> 3, c = i & 7;
+        const size_t kr = PAGED ? a.pg.row(b, t) : (size_t)(a.kv_off[b] + t);
+        cp_async16(Ks + swz(t, c), a.k + kr * a.kv_stride + h * 64 + c * 8);
+        cp_async16(Vs + swz(t, c), a.v + kr * a.kv_stride + h * 64 + c * 8);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    pdl_launch_dependents();
+    pdl_wait();                                   // ... and everything the predecessor kernels wrote after it
     for (int i = tid; i < ATT_Q * 8; i += 128) {
         const int r = i >> 3, c = i & 7;
         if (r < nq) {
@@ -94,7 +106,7 @@ __global__ void __launch_bounds__(128) k_attn_tc(AttnTcArgs a) {
             *reinterpret_cast<uint4*>(Qp + swz(r, c)) = make_uint4(0, 0, 0, 0);
         }
     }
-    for (int i = tid; i < nkp * 8; i += 128) {
+    for (int i = tid + npre * 8; i < nkp * 8; i += 128) {
         const int t = i >> 3, c = i & 7;
         if (t < nkmax) {
             const size_t kr = PAGED ? a.pg.row(b, t) : (size_t)(a.kv_off[b] + t);

@@ -459,7 +459,7 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
 template <typename T>
 int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* q_index, const void* k, const void* v,
          int kv_stride, const int* kv_off, const Rows& r, const int* nkeys, int cnt, int rows_ub, int q_ub, void* out,
-         int out_stride, int n_heads, int d_head, int max_keys, cudaStream_t st) {
+         int out_stride, int n_heads, int d_head, int max_keys, cudaStream_t st, const int* pre_keys = nullptr) {
     if (rows_ub <= 0) return 0;
     if constexpr (std::is_same<T, bf16>::value) {
         const size_t smem = attn_tc_smem(max_keys);
@@ -468,7 +468,7 @@ int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* 
             a.q = (const bf16*)q; a.q_stride = q_stride; a.q_index = q_index;
             a.k = (const bf16*)k; a.v = (const bf16*)v; a.kv_stride = kv_stride; a.kv_off = kv_off;
             a.pg.table = h->page_table; a.pg.page_tokens = h->cfg.page_tokens; a.pg.max_pages = h->pages_per_seq;
-            a.q_off = r.q_off; a.q_cnt = r.q_cnt; a.nkeys = nkeys;
+            a.q_off = r.q_off; a.q_cnt = r.q_cnt; a.nkeys = nkeys; a.pre_keys = h->use_pdl ? pre_keys : nullptr;
             a.out = (bf16*)out; a.out_stride = out_stride; a.max_keys = max_keys;
             a.scale = 1.0f / sqrtf((float)d_head);
             dim3 grid(cdiv(q_ub, ATT_Q), n_heads, h->B);
@@ -532,7 +532,7 @@ int fused_attn_proj(specdec_handle* h, bool paged, const void* q, int q_stride, 
         a.q = (const bf16*)q; a.q_stride = q_stride; a.q_index = q_index;
         a.k = (const bf16*)k; a.v = (const bf16*)v; a.kv_stride = kv_stride; a.kv_off = kv_off;
         a.pg.table = h->page_table; a.pg.page_tokens = h->cfg.page_tokens; a.pg.max_pages = h->pages_per_seq;
-        a.q_off = r.q_off; a.q_cnt = r.q_cnt; a.nkeys = nkeys; a.out = nullptr; a.out_stride = 0; a.max_keys = max_keys;
+        a.q_off = r.q_off; a.q_cnt = r.q_cnt; a.nkeys = nkeys; a.pre_keys = nullptr; a.out = nullptr; a.out_stride = 0; a.max_keys = max_keys;
         a.scale = 1.0f / sqrtf((float)d_head);
         p.wo = (const bf16*)wo; p.bo = bo; p.x = x; p.d = d;
         cudaLaunchConfig_t cfg = {};
@@ -580,7 +580,7 @@ int block_self(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, co
         if (f < 0) return f;
         if (f == 1) return 0;
         TRY(attn<T>(h, true, h->qkv, 3 * d, nullptr, h->kc[layer], h->vc[layer], d, nullptr, r, r.nk_self, cnt,
-                    rows_ub, q_ub, h->att, d, H, dh, max_keys, st));
+                    rows_ub, q_ub, h->att, d, H, dh, max_keys, st, h->ses.len));      // cached prefix: positions < len
     } else {
         TRY(attn<T>(h, false, h->qkv, 3 * d, nullptr, (char*)h->qkv + (size_t)d * e, (char*)h->qkv + (size_t)2 * d * e,
                     3 * d, r.kv_off, r, r.nk_self, cnt, rows_ub, q_ub, h->att, d, H, dh, max_keys, st));
@@ -604,7 +604,7 @@ int block_cross(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, c
         if (f == 1) return 0;
     }
     TRY(attn<T>(h, false, h->q, d, nullptr, m.ckv[layer], (char*)m.ckv[layer] + (size_t)d * e, 2 * d, r.kv_off_cross,
-                r, r.nk_cross, cnt, rows_ub, q_ub, h->att, d, H, dh, h->S_max, st));
+                r, r.nk_cross, cnt, rows_ub, q_ub, h->att, d, H, dh, h->S_max, st, h->ses.src_len));   // encoder K/V: all of it
     TRY(gemm<T>(h, EPI_RESID, h->att, d, w.co_w, w.co_b, d, d, cnt, rows_ub, nullptr, 0, x, st));
     return 0;
 }
