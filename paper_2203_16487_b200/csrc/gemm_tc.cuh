@@ -160,7 +160,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     constexpr int HALF = BN / 2;                     // columns per epilogue warp
     if (threadIdx.x == 0) tc_stamp(g.trace, 0);
     constexpr int CW = HALF >= 32 ? 32 : 16;         // columns per TMEM read
-    const int R = *g.n_rows;
+    // With a row count known on the host the kernel can set itself up and start streaming weight tiles before
+    // its predecessor has finished (programmatic dependent launch); a device-side count must be waited for.
+    const bool early = g.rows_static >= 0;
+    if (!early) pdl_wait();
+    const int R = early ? g.rows_static : *g.n_rows;
     const int m_tiles = (R + TC_BM - 1) / TC_BM, n_tiles = (g.N + BN - 1) / BN;
     const int total = m_tiles * n_tiles;
     if ((int)blockIdx.x >= total) return;            // whole CTA leaves before touching barriers or tensor memory
@@ -188,6 +192,19 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     const uint32_t tmem_d = tmem_base_s;
     volatile int* abort_flag = &abort_s;
     if (threadIdx.x == 0) tc_stamp(g.trace, 1);
+    int pre = 0;                                       // stages whose weight half was requested before the wait
+    if (early) {
+        if (threadIdx.x == 0) {
+            const int n0 = ((int)blockIdx.x / m_tiles) * BN;
+            for (; pre < STAGES && pre < nkb; ++pre) {
+                const uint32_t bar = smem_u32(&bar_full[pre]);
+                mbar_expect_tx(bar, Cfg::STAGE_BYTES);
+                tma_load_2d(tiles + pre * Cfg::STAGE_BYTES + TC_BM * TC_BK * 2, &tmW, pre * TC_BK, n0, bar);
+            }
+        }
+        pdl_launch_dependents();
+        pdl_wait();                                    // activations, residual and outputs belong to the predecessors until here
+    }
 
     if (warp == 0) {
         if (lane == 0) {
@@ -200,9 +217,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     if (*abort_flag) break;
                     const uint32_t a_dst = tiles + s * Cfg::STAGE_BYTES, w_dst = a_dst + TC_BM * TC_BK * 2;
                     const uint32_t bar = smem_u32(&bar_full[s]);
-                    mbar_expect_tx(bar, Cfg::STAGE_BYTES);
+                    if (kbi >= pre) {
+                        mbar_expect_tx(bar, Cfg::STAGE_BYTES);
+                        tma_load_2d(w_dst, &tmW, kb * TC_BK, n0, bar);
+                    }
                     tma_load_2d(a_dst, &tmA, kb * TC_BK, m0, bar);
-                    tma_load_2d(w_dst, &tmW, kb * TC_BK, n0, bar);
                     if (kbi == 0) tc_stamp(g.trace, 2);
                 }
             }
@@ -386,6 +405,7 @@ struct TmaEncoder {
     int* err_word = nullptr;            // device word the kernels raise on a wait timeout
     int n_sm = 148;
     int force_bn = 0;                   // experiments: 0 = choose, else 32 / 64 / 128 / 256
+    bool pdl = true;                    // launch with programmatic stream serialization
     std::map<std::tuple<const void*, long long, int, int, int>, CUtensorMap> cache;
 
     // 2-D bf16 tensor [rows, K] with row pitch ld elements; box = 64 x box_rows, 128-byte swizzle.
@@ -455,8 +475,14 @@ inline int tc_launch_one(TmaEncoder& enc, GemmArgs<bf16>& g, int rows_ub, cudaSt
     if (!ta || !tw) return -1;
     const long long tiles_ub = (long long)((g.N + BN - 1) / BN) * ((rows_ub + TC_BM - 1) / TC_BM);
     const int grid = (int)std::min<long long>(tiles_ub, enc.n_sm);
-    k_gemm_tc<EPI, BN><<<grid, TC_THREADS, TcCfg<BN>::SMEM, st>>>(*ta, *tw, g, enc.err_word);
-    cudaError_t e = cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = TcCfg<BN>::SMEM; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = enc.pdl ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_gemm_tc<EPI, BN>, *ta, *tw, g, enc.err_word);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { enc.err = std::string("launch: ") + cudaGetErrorString(e); return -1; }
     return 0;
 }

@@ -171,6 +171,8 @@ __global__ void k_layernorm(const float* __restrict__ x, const float* __restrict
                             const int* __restrict__ n_rows, T* __restrict__ y, int d, float eps) {
     int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     int lane = threadIdx.x & 31;
+    pdl_launch_dependents();
+    pdl_wait();
     if (row >= *n_rows) return;
     const float* xr = x + (size_t)row * d;
     if (d % 128 == 0 && d <= 512) {

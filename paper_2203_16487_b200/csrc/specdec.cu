@@ -318,11 +318,29 @@ void load_model(specdec_handle* h, ModelW& m, const std::string& pre, Manifest& 
 }
 
 // ---------------------------------------------------------------- launch helpers
+// Launch that lets the kernel start before its predecessor in the stream has finished (the kernel itself
+// calls pdl_wait() before it touches anything the predecessor wrote).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(specdec_handle* h, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                       Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = h->use_pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 template <typename T>
 int ln(specdec_handle* h, const float* x, const float* g, const float* b, int cnt, int rows_ub, void* y, int d,
        cudaStream_t st) {
     if (rows_ub <= 0) return 0;
-    k_layernorm<T><<<cdiv(rows_ub, 8), 256, 0, st>>>(x, g, b, h->ses.counters + cnt, (T*)y, d, 1e-5f);
+    {
+        cudaError_t e = launch_pdl(h, k_layernorm<T>, dim3(cdiv(rows_ub, 8)), dim3(256), 0, st, x, g, b,
+                                   (const int*)(h->ses.counters + cnt), (T*)y, d, 1e-5f);
+        if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("layer norm launch: ") + cudaGetErrorString(e));
+    }
     KCHECK(h);
     return 0;
 }
@@ -344,20 +362,6 @@ bool skinny_ok(const specdec_handle* h, int epi, int rows_ub, int N, int K, bool
     if (epi != EPI_STORE && epi != EPI_RELU && epi != EPI_RESID && epi != EPI_QKV) return false;
     if (K % 32 || (with_ln && (K % 128 || K > 512))) return false;
     return skinny_smem(rows_ub <= 32 ? 2 : (rows_ub <= 48 ? 3 : 4), K) <= h->skinny_smem_cap;
-}
-
-// Launch that lets the kernel start before its predecessor in the stream has finished (the kernel itself
-// calls pdl_wait() before it touches anything the predecessor wrote).
-template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(specdec_handle* h, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
-                       Args... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = h->use_pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
 template <int EPI, int MT, int G>
@@ -1168,7 +1172,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
     if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }
-    if (!strcmp(name, "pdl")) { h->use_pdl = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "pdl")) { h->use_pdl = value ? 1 : 0; h->tma.pdl = value != 0; return SPECDEC_OK; }
     if (!strcmp(name, "skinny")) { h->use_skinny = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "row_lse")) { h->want_lse = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "attn")) { h->use_tc_attn = value ? 1 : 0; return SPECDEC_OK; }
