@@ -126,3 +126,34 @@ def test_config5_verify_step_with_scripted_rejections(base, k, prefix):
     acc, bif = sd.verify(drafts, 3, 1.0)
     assert list(zip(acc.cpu().tolist(), bif.cpu().tolist())) == expect
     sd.close()
+
+
+def test_shape_variants_12_2_verifier_and_narrow_heads():
+    """The paper also accelerates a 12+2 Transformer-base verifier (Table 1, lower half); and a bf16 model whose
+    heads are 32 wide exercises the tensor-core GEMM together with the warp-per-row attention."""
+    from paper_2203_16487_b200 import binding
+    v122 = W.ModelDims(512, 8, 2048, 32768, 12, 2, 1024)
+    wv, wd = W.make_weights(v122, 2001, True), W.make_weights(W.BASE_D, 1002, True)
+    mv, md = O.model_from(v122, wv, mode="bf16"), O.model_from(W.BASE_D, wd, mode="bf16")
+    wl = W.config2_translation(2)
+    sd = binding.SpecDec(v122, wv, W.BASE_D, wd, k_max=10, max_batch=2, max_src=40, max_tgt=48, bf16=True)
+    rep = lockstep.run(sd, mv, md, wl.src, [20, 20], 10, 3, 1.0, margin=1e-3, check_logits_every=3, max_iters=5)
+    assert rep.ok, rep.notes
+    assert rep.max_logit_err < 2e-2
+    sd.close()
+    nv = W.ModelDims(128, 4, 256, 3000, 2, 2, 128)            # heads of 32
+    nd = W.ModelDims(128, 4, 256, 3000, 2, 1, 128)
+    wv, wd = W.make_weights(nv, 61, True), W.make_weights(nd, 62, True)
+    mv, md = O.model_from(nv, wv, mode="bf16"), O.model_from(nd, wd, mode="bf16")
+    rng = np.random.default_rng(3)
+    srcs = [W.zipf_ids(rng, n, 3000) for n in (9, 30, 17)]
+    sd = binding.SpecDec(nv, wv, nd, wd, k_max=6, max_batch=3, max_src=32, max_tgt=20, bf16=True)
+    rep = lockstep.run(sd, mv, md, srcs, [20, 11, 16], 6, 2, 0.5, margin=1e-3, check_logits_every=2)
+    assert rep.ok, rep.notes
+    assert rep.max_logit_err < 2e-2
+    out, n, _ = sd.generate(*W.pad_batch(srcs), [20, 11, 16], 6, 1, 0.0)
+    for b, s in enumerate(srcs):                                # strict rule = greedy decoding (up to bf16 near-ties)
+        ref = O.greedy_decode(mv, s, [20, 11, 16][b], BOS, EOS)
+        got = out[b, :int(n[b])].cpu().tolist()
+        assert got == ref or _prefix_match(got, ref) >= 3
+    sd.close()
