@@ -48,13 +48,14 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
 __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
 
 constexpr int ATT_Q = 32;
+constexpr int ATT_THREADS = 256;          // 8 warps
 inline size_t attn_tc_smem(int max_keys) {
     const int nkp = (max_keys + 15) & ~15;
     return (size_t)ATT_Q * 128 + (size_t)nkp * 256 + (size_t)ATT_Q * (nkp + 4) * 4 + 16;
 }
 
 template <bool PAGED>
-__global__ void __launch_bounds__(128) k_attn_tc(AttnTcArgs a) {
+__global__ void __launch_bounds__(ATT_THREADS) k_attn_tc(AttnTcArgs a) {
     extern __shared__ __align__(128) unsigned char sm[];
     __shared__ int s_nk[ATT_Q];
     __shared__ float s_sum[ATT_Q];
@@ -88,7 +89,7 @@ __global__ void __launch_bounds__(128) k_attn_tc(AttnTcArgs a) {
 
     // ---- stage K, V of the keys that predate this step (cached prefix, encoder memory) before the wait ...
     const int npre = a.pre_keys ? min(a.pre_keys[b], nkmax) : 0;
-    for (int i = tid; i < npre * 8; i += 128) {
+    for (int i = tid; i < npre * 8; i += ATT_THREADS) {
         const int t = i >> 3, c = i & 7;
         const size_t kr = PAGED ? a.pg.row(b, t) : (size_t)(a.kv_off[b] + t);
         cp_async16(Ks + swz(t, c), a.k + kr * a.kv_stride + h * 64 + c * 8);
@@ -97,7 +98,7 @@ __global__ void __launch_bounds__(128) k_attn_tc(AttnTcArgs a) {
     asm volatile("cp.async.commit_group;" ::: "memory");
     pdl_launch_dependents();
     pdl_wait();                                   // ... and everything the predecessor kernels wrote after it
-    for (int i = tid; i < ATT_Q * 8; i += 128) {
+    for (int i = tid; i < ATT_Q * 8; i += ATT_THREADS) {
         const int r = i >> 3, c = i & 7;
         if (r < nq) {
             const size_t qr = a.q_index ? (size_t)a.q_index[r0 + r] : (size_t)(r0 + r);
@@ -106,7 +107,7 @@ __global__ void __launch_bounds__(128) k_attn_tc(AttnTcArgs a) {
             *reinterpret_cast<uint4*>(Qp + swz(r, c)) = make_uint4(0, 0, 0, 0);
         }
     }
-    for (int i = tid + npre * 8; i < nkp * 8; i += 128) {
+    for (int i = tid + npre * 8; i < nkp * 8; i += ATT_THREADS) {
         const int t = i >> 3, c = i & 7;
         if (t < nkmax) {
             const size_t kr = PAGED ? a.pg.row(b, t) : (size_t)(a.kv_off[b] + t);
@@ -132,7 +133,7 @@ __global__ void __launch_bounds__(128) k_attn_tc(AttnTcArgs a) {
                 const int r = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = ks * 2 + (lane >> 4);
                 ldsm_x4(Qs + swz(r, c), qf[mt][ks][0], qf[mt][ks][1], qf[mt][ks][2], qf[mt][ks][3]);
             }
-        for (int nt = warp; nt < nkp / 8; nt += 4) {
+        for (int nt = warp; nt < nkp / 8; nt += ATT_THREADS / 32) {
             uint32_t kf[2][4];
 #pragma unroll
             for (int kk = 0; kk < 2; ++kk) {
@@ -154,17 +155,18 @@ __global__ void __launch_bounds__(128) k_attn_tc(AttnTcArgs a) {
         }
     }
     __syncthreads();
-    // ---- softmax: 4 threads per row; P (bf16, un-normalised) overwrites the K tile
+    // ---- softmax: 8 threads per row; P (bf16, un-normalised) overwrites the K tile
     {
         bf16* P = reinterpret_cast<bf16*>(Kp);
-        const int r = tid >> 2, sub = tid & 3;
+        const int r = tid >> 3, sub = tid & 7;
         const float* srow = Ss + r * sstr;
         float m = -CUDART_INF_F;
-        for (int c = sub; c < nkp; c += 4) m = fmaxf(m, srow[c]);
+        for (int c = sub; c < nkp; c += 8) m = fmaxf(m, srow[c]);
         m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
         m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 4));
         float sum = 0.f;
-        for (int c = sub; c < nkp; c += 4) {
+        for (int c = sub; c < nkp; c += 8) {
             const float s = srow[c];
             const float e = (s == -CUDART_INF_F) ? 0.f : expf(s - m);
             sum += e;
@@ -172,50 +174,46 @@ __global__ void __launch_bounds__(128) k_attn_tc(AttnTcArgs a) {
         }
         sum += __shfl_xor_sync(0xffffffffu, sum, 1);
         sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 4);
         if (sub == 0) s_sum[r] = sum;
     }
     __syncthreads();
-    // ---- O = P V ; warp w owns head columns 16w .. 16w+15
+    // ---- O = P V ; warp w owns query rows 16 (w / 4) .. and head columns 16 (w % 4) ..
     {
-        float acc[2][2][4];
+        const int mt = warp >> 2, wq = warp & 3;
+        float acc[2][4];
 #pragma unroll
-        for (int i = 0; i < 2; ++i)
+        for (int j = 0; j < 2; ++j)
 #pragma unroll
-            for (int j = 0; j < 2; ++j)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
+            for (int e = 0; e < 4; ++e) acc[j][e] = 0.f;
         for (int kt = 0; kt < nkp / 16; ++kt) {
-            uint32_t vf[4];
+            uint32_t vf[4], pf[4];
             {
-                const int r = kt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = warp * 2 + (lane >> 4);
+                const int r = kt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = wq * 2 + (lane >> 4);
                 ldsm_x4_t(Vs + swz(r, c), vf[0], vf[1], vf[2], vf[3]);
             }
-#pragma unroll
-            for (int mt = 0; mt < 2; ++mt) {
-                uint32_t pf[4];
+            {
                 const int r = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = kt * 16 + (lane >> 4) * 8;
                 ldsm_x4(Ks + (uint32_t)(r * pstr + c) * 2, pf[0], pf[1], pf[2], pf[3]);
-                mma_bf16(acc[mt][0], pf, vf[0], vf[1]);
-                mma_bf16(acc[mt][1], pf, vf[2], vf[3]);
             }
+            mma_bf16(acc[0], pf, vf[0], vf[1]);
+            mma_bf16(acc[1], pf, vf[2], vf[3]);
         }
 #pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
+        for (int half = 0; half < 2; ++half) {
+            const int r = mt * 16 + g + half * 8;
+            if (r < nq) {
+                const float den = s_sum[r];
+                bf16* o = a.out + (size_t)(r0 + r) * a.out_stride + h * 64 + wq * 16 + t4 * 2;
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                const int r = mt * 16 + g + half * 8;
-                if (r < nq) {
-                    const float den = s_sum[r];
-                    bf16* o = a.out + (size_t)(r0 + r) * a.out_stride + h * 64 + warp * 16 + t4 * 2;
-#pragma unroll
-                    for (int nt = 0; nt < 2; ++nt) {
-                        __nv_bfloat162 v2;
-                        v2.x = __float2bfloat16_rn(den > 0.f ? acc[mt][nt][half * 2] / den : 0.f);
-                        v2.y = __float2bfloat16_rn(den > 0.f ? acc[mt][nt][half * 2 + 1] / den : 0.f);
-                        *reinterpret_cast<__nv_bfloat162*>(o + nt * 8) = v2;
-                    }
+                for (int nt = 0; nt < 2; ++nt) {
+                    __nv_bfloat162 v2;
+                    v2.x = __float2bfloat16_rn(den > 0.f ? acc[nt][half * 2] / den : 0.f);
+                    v2.y = __float2bfloat16_rn(den > 0.f ? acc[nt][half * 2 + 1] / den : 0.f);
+                    *reinterpret_cast<__nv_bfloat162*>(o + nt * 8) = v2;
                 }
             }
+        }
     }
 }
 

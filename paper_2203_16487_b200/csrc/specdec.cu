@@ -476,8 +476,8 @@ int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* 
             a.out = (bf16*)out; a.out_stride = out_stride; a.max_keys = max_keys;
             a.scale = 1.0f / sqrtf((float)d_head);
             dim3 grid(cdiv(q_ub, ATT_Q), n_heads, h->B);
-            cudaError_t e = paged ? launch_pdl(h, k_attn_tc<true>, grid, dim3(128), smem, st, a)
-                                  : launch_pdl(h, k_attn_tc<false>, grid, dim3(128), smem, st, a);
+            cudaError_t e = paged ? launch_pdl(h, k_attn_tc<true>, grid, dim3(ATT_THREADS), smem, st, a)
+                                  : launch_pdl(h, k_attn_tc<false>, grid, dim3(ATT_THREADS), smem, st, a);
             if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(e));
             KCHECK(h);
             return 0;
