@@ -59,6 +59,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
 }
+constexpr int TC_BM = 128, TC_BK = 64;
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -118,15 +119,19 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
 __device__ __forceinline__ void tc_stamp(long long* trace, int slot) {
     if (trace && blockIdx.x == 0) { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); trace[slot] = t; }
 }
-constexpr int TC_BM = 128, TC_BK = 64;
 constexpr int TC_EPI_WARPS = 8;                      // two per TMEM lane quadrant: each takes half the columns
 constexpr int TC_THREADS = (2 + TC_EPI_WARPS) * 32;  // + TMA warp + MMA warp
-template <int BN> struct TcCfg {
-    static constexpr int STAGES = BN >= 256 ? 4 : (BN >= 128 ? 6 : 8);
-    static constexpr int STAGE_BYTES = (TC_BM + BN) * TC_BK * 2;
-    static constexpr int STG_BYTES = TC_EPI_WARPS * 32 * 32 * 4;      // per-warp 32 x 32 fp32 transpose buffers
+// AR = rows of the activation box a stage holds (the MMA always spans 128 rows; with AR < 128 the rows beyond
+// the box are whatever shared memory holds and only feed accumulator lanes that nobody reads).  STG = the
+// epilogue needs its transpose buffers.
+template <int BN, int AR = 128, bool STG = true> struct TcCfg {
+    static constexpr int STAGE_BYTES = (AR + BN) * TC_BK * 2;
+    static constexpr int STG_BYTES = STG ? TC_EPI_WARPS * 32 * 32 * 4 : 0;   // per-warp 32 x 32 fp32 transpose buffers
+    static_assert(BN >= 128 - AR, "the 128-row MMA read of a short activation box must stay inside its stage");
+    static constexpr int FIT = (232448 - 1024 - STG_BYTES) / STAGE_BYTES;
+    static constexpr int STAGES = AR < 128 || !STG ? (FIT > 8 ? 8 : FIT) : (BN > 128 ? 4 : (BN >= 128 ? 6 : 8));
     static constexpr int SMEM = STAGES * STAGE_BYTES + STG_BYTES + 1024;
-    static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;      // two accumulators
+    static constexpr int TMEM_COLS = 2 * BN <= 32 ? 32 : (2 * BN <= 64 ? 64 : (2 * BN <= 128 ? 128 : (2 * BN <= 256 ? 256 : 512)));  // two accumulators, power of two
 };
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
@@ -151,21 +156,23 @@ __device__ __forceinline__ void tmem_ld(uint32_t taddr, float* v) {
 // Persistent kernel: CTA c works on tiles c, c + gridDim.x, ... (row tile fastest, so CTAs running
 // together share one weight tile).  The TMA ring and the two TMEM accumulators run across tiles, so the
 // epilogue of tile i overlaps the loads and MMAs of tile i + 1.
-template <int EPI, int BN>
+template <int EPI, int BN, int AR = 128>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, GemmArgs<bf16> g,
           int* err_word) {
-    using Cfg = TcCfg<BN>;
+    using Cfg = TcCfg<BN, AR, EPI != EPI_STATS>;
     constexpr int STAGES = Cfg::STAGES;
+    constexpr int A_BYTES = AR * TC_BK * 2;          // activation part of a stage
     constexpr int HALF = BN / 2;                     // columns per epilogue warp
     if (threadIdx.x == 0) tc_stamp(g.trace, 0);
-    constexpr int CW = HALF >= 32 ? 32 : 16;         // columns per TMEM read
+    constexpr int CW = HALF % 32 == 0 ? 32 : 16;     // columns per TMEM read
     // With a row count known on the host the kernel can set itself up and start streaming weight tiles before
     // its predecessor has finished (programmatic dependent launch); a device-side count must be waited for.
-    const bool early = g.rows_static >= 0;
+    // So can a launch whose rows fit one row tile whatever their count (one_m_tile): the count is read later.
+    const bool early = g.rows_static >= 0 || g.one_m_tile;
     if (!early) pdl_wait();
-    const int R = early ? g.rows_static : *g.n_rows;
-    const int m_tiles = (R + TC_BM - 1) / TC_BM, n_tiles = (g.N + BN - 1) / BN;
+    int R = g.rows_static >= 0 ? g.rows_static : (early ? 0 : *g.n_rows);
+    const int m_tiles = g.one_m_tile ? 1 : (R + TC_BM - 1) / TC_BM, n_tiles = (g.N + BN - 1) / BN;
     const int total = m_tiles * n_tiles;
     if ((int)blockIdx.x >= total) return;            // whole CTA leaves before touching barriers or tensor memory
 
@@ -184,14 +191,15 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bar_acc_full[i]), 1); mbar_init(smem_u32(&bar_acc_empty[i]), TC_EPI_WARPS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        tc_stamp(g.trace, 12);
     }
-    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), Cfg::TMEM_COLS);
+    if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_s), Cfg::TMEM_COLS); if (lane == 0) tc_stamp(g.trace, 13); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_d = tmem_base_s;
     volatile int* abort_flag = &abort_s;
-    if (threadIdx.x == 0) tc_stamp(g.trace, 1);
+    if (threadIdx.x == 0 && tmem_d != 0xffffffffu) tc_stamp(g.trace, 1);   // (the test pins the stamp behind the read)
     int pre = 0;                                       // stages whose weight half was requested before the wait
     if (early) {
         if (threadIdx.x == 0) {
@@ -199,11 +207,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             for (; pre < STAGES && pre < nkb; ++pre) {
                 const uint32_t bar = smem_u32(&bar_full[pre]);
                 mbar_expect_tx(bar, Cfg::STAGE_BYTES);
-                tma_load_2d(tiles + pre * Cfg::STAGE_BYTES + TC_BM * TC_BK * 2, &tmW, pre * TC_BK, n0, bar);
+                tma_load_2d(tiles + pre * Cfg::STAGE_BYTES + A_BYTES, &tmW, pre * TC_BK, n0, bar);
             }
         }
         pdl_launch_dependents();
         pdl_wait();                                    // activations, residual and outputs belong to the predecessors until here
+        if (g.rows_static < 0) R = *g.n_rows;
     }
 
     if (warp == 0) {
@@ -215,7 +224,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     const int s = kbi % STAGES;
                     if (kbi >= STAGES) mbar_wait(smem_u32(&bar_empty[s]), ((kbi / STAGES) - 1) & 1, abort_flag, err_word, 1);
                     if (*abort_flag) break;
-                    const uint32_t a_dst = tiles + s * Cfg::STAGE_BYTES, w_dst = a_dst + TC_BM * TC_BK * 2;
+                    const uint32_t a_dst = tiles + s * Cfg::STAGE_BYTES, w_dst = a_dst + A_BYTES;
                     const uint32_t bar = smem_u32(&bar_full[s]);
                     if (kbi >= pre) {
                         mbar_expect_tx(bar, Cfg::STAGE_BYTES);
@@ -242,7 +251,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     if (*abort_flag) break;
                     if (kbi == 0) tc_stamp(g.trace, 4);
                     tc_fence_after();
-                    const uint32_t a_src = tiles + s * Cfg::STAGE_BYTES, w_src = a_src + TC_BM * TC_BK * 2;
+                    const uint32_t a_src = tiles + s * Cfg::STAGE_BYTES, w_src = a_src + A_BYTES;
                     const uint64_t ad = umma_desc_k_sw128(a_src), wd = umma_desc_k_sw128(w_src);
 #pragma unroll
                     for (int k4 = 0; k4 < TC_BK / 16; ++k4)      // +32 bytes along K per instruction: 2 address units
@@ -256,11 +265,32 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     } else {
         const int q = warp & 3;                                  // TMEM lane quadrant this warp may read
         const int half = (warp - 2) >> 2;                        // which half of the tile's columns
+        constexpr bool bf_out = (EPI == EPI_STORE || EPI == EPI_RELU || EPI == EPI_QKV);
+        constexpr int NCH = HALF / CW;                           // column chunks per warp and tile
+        // 16-byte accesses after the transpose need aligned rows
+        const bool vec_ok = CW == 32 && (bf_out ? (g.ldo % 8 == 0 && (EPI != EPI_QKV || g.kv_d % 32 == 0)) : (g.N % 4 == 0));
         int i = 0;
         for (int t = blockIdx.x; t < total; t += gridDim.x, ++i) {
             const int ab = i & 1;
             const int m0 = (t % m_tiles) * TC_BM, n_tile = t / m_tiles, n0 = n_tile * BN + half * HALF;
             const int r = m0 + q * 32 + lane;
+            const int rbase = m0 + q * 32;
+            // EPI_RESID: the residual values of the first two column chunks are requested before the accumulator
+            // is awaited, so their latency hides behind the MMAs
+            float4 xin[2][8];
+            if (EPI == EPI_RESID && vec_ok && rbase < R) {
+#pragma unroll
+                for (int c = 0; c < (NCH < 2 ? NCH : 2); ++c) {
+                    const int nb = n0 + c * CW;
+                    if (nb + CW <= g.N) {
+#pragma unroll
+                        for (int ps = 0; ps < 8; ++ps) {
+                            const int gr = rbase + ps * 4 + (lane >> 3);
+                            xin[c][ps] = gr < R ? *reinterpret_cast<const float4*>(g.resid + (size_t)gr * g.N + nb + (lane & 7) * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+                    }
+                }
+            }
             const bool live = mbar_wait(smem_u32(&bar_acc_full[ab]), (i >> 1) & 1, abort_flag, err_word, 3);
             if (threadIdx.x == 64) tc_stamp(g.trace, 7 + 2 * (i > 0));
             tc_fence_after();
@@ -302,9 +332,74 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 }
                 if (r < R) g.part[(size_t)r * g.n_tiles + n_tile * 2 + half] = p;
             } else if (warp_live) {
-                for (int c = 0; c < HALF / CW; ++c) {
-                    tmem_ld<CW>(trow + c * CW, v);
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
                     const int nb = n0 + c * CW;
+                    if (EPI == EPI_RESID && c >= 2 && vec_ok && nb + CW <= g.N) {      // chunks 0 and 1 were requested before the wait
+#pragma unroll
+                        for (int ps = 0; ps < 8; ++ps) {
+                            const int gr = rbase + ps * 4 + (lane >> 3);
+                            xin[c & 1][ps] = gr < R ? *reinterpret_cast<const float4*>(g.resid + (size_t)gr * g.N + nb + (lane & 7) * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+                    }
+                    tmem_ld<CW>(trow + c * CW, v);
+                    if (CW == 32 && vec_ok && nb + CW <= g.N) {
+                        // Transpose through shared memory: a thread owns one output ROW in tensor memory, but global
+                        // memory wants neighbouring lanes on neighbouring addresses.  The 32 x 32 block is written row-wise
+                        // with its 16-byte chunks XOR-swizzled by the row, then read back 16 bytes of output per lane.
+                        float* srow = stg + lane * 32;
+#pragma unroll
+                        for (int j4 = 0; j4 < 8; ++j4)
+                            *reinterpret_cast<float4*>(srow + ((j4 ^ (lane & 7)) << 2)) = make_float4(v[j4 * 4], v[j4 * 4 + 1], v[j4 * 4 + 2], v[j4 * 4 + 3]);
+                        __syncwarp();
+                        if (!bf_out) {
+                            // fp32 rows: 8 lanes per row (4 columns each), 4 rows per pass
+                            const int l8 = lane & 7, rsub = lane >> 3;
+                            const float4 bz = g.bias ? __ldg(reinterpret_cast<const float4*>(g.bias + nb) + l8) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                            for (int ps = 0; ps < 8; ++ps) {
+                                const int rr = ps * 4 + rsub, gr = rbase + rr;
+                                float4 a = *reinterpret_cast<const float4*>(stg + rr * 32 + ((l8 ^ (rr & 7)) << 2));
+                                a.x += bz.x; a.y += bz.y; a.z += bz.z; a.w += bz.w;
+                                if (EPI == EPI_RESID) { const float4 x = xin[c & 1][ps]; a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w; }
+                                if (gr < R) *reinterpret_cast<float4*>(g.resid + (size_t)gr * g.N + nb + l8 * 4) = a;
+                            }
+                        } else {
+                            // bf16 rows: 4 lanes per row (8 columns = 16 bytes each), 8 rows per pass
+                            const int c4 = lane & 3, rsub = lane >> 2;
+                            float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
+                            if (g.bias) { b0 = __ldg(reinterpret_cast<const float4*>(g.bias + nb) + 2 * c4); b1 = __ldg(reinterpret_cast<const float4*>(g.bias + nb) + 2 * c4 + 1); }
+#pragma unroll
+                            for (int ps = 0; ps < 4; ++ps) {
+                                const int rr = ps * 8 + rsub, gr = rbase + rr;
+                                const long long row_of = (EPI == EPI_QKV) ? __shfl_sync(0xffffffffu, my_cache_row, rr) : 0;
+                                float4 a0 = *reinterpret_cast<const float4*>(stg + rr * 32 + (((2 * c4) ^ (rr & 7)) << 2));
+                                float4 a1 = *reinterpret_cast<const float4*>(stg + rr * 32 + (((2 * c4 + 1) ^ (rr & 7)) << 2));
+                                a0.x += b0.x; a0.y += b0.y; a0.z += b0.z; a0.w += b0.w;
+                                a1.x += b1.x; a1.y += b1.y; a1.z += b1.z; a1.w += b1.w;
+                                if (EPI == EPI_RELU) {
+                                    a0.x = fmaxf(a0.x, 0.f); a0.y = fmaxf(a0.y, 0.f); a0.z = fmaxf(a0.z, 0.f); a0.w = fmaxf(a0.w, 0.f);
+                                    a1.x = fmaxf(a1.x, 0.f); a1.y = fmaxf(a1.y, 0.f); a1.z = fmaxf(a1.z, 0.f); a1.w = fmaxf(a1.w, 0.f);
+                                }
+                                if (gr < R) {
+                                    bf16* o = g.out + (size_t)gr * g.ldo + nb;
+                                    if (EPI == EPI_QKV && nb >= g.kv_d) {          // K or V part: straight into the paged cache
+                                        const size_t row = (size_t)row_of;
+                                        o = (nb < 2 * g.kv_d ? g.kc + row * g.kv_d + (nb - g.kv_d) : g.vc + row * g.kv_d + (nb - 2 * g.kv_d));
+                                    }
+                                    __nv_bfloat162 p0 = __floats2bfloat162_rn(a0.x, a0.y), p1 = __floats2bfloat162_rn(a0.z, a0.w);
+                                    __nv_bfloat162 p2 = __floats2bfloat162_rn(a1.x, a1.y), p3 = __floats2bfloat162_rn(a1.z, a1.w);
+                                    uint4 pk;
+                                    pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+                                    pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+                                    *reinterpret_cast<uint4*>(o + c4 * 8) = pk;
+                                }
+                            }
+                        }
+                        __syncwarp();
+                        continue;
+                    }
+                    // ragged or unaligned chunk: one row per thread, element by element
                     if (g.bias) {
 #pragma unroll
                         for (int j = 0; j < CW; ++j) v[j] += (nb + j < g.N) ? __ldg(g.bias + nb + j) : 0.f;
@@ -312,57 +407,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     if (EPI == EPI_RELU) {
 #pragma unroll
                         for (int j = 0; j < CW; ++j) v[j] = fmaxf(v[j], 0.f);
-                    }
-                    const bool full = nb + CW <= g.N;
-                    const bool bf_out = (EPI == EPI_STORE || EPI == EPI_RELU || EPI == EPI_QKV);
-                    if (CW == 32 && full && (bf_out ? (g.ldo % 2 == 0 && (EPI != EPI_QKV || g.kv_d % 32 == 0)) : true)) {
-                        // Transpose through shared memory: a thread owns one output ROW in tensor memory, but global
-                        // memory wants a warp to touch one row at a time.  The 32 x 32 block is written row-wise with
-                        // its 16-byte chunks XOR-swizzled by the row, then read back one row per warp instruction.
-                        float* srow = stg + lane * 32;
-#pragma unroll
-                        for (int j4 = 0; j4 < 8; ++j4)
-                            *reinterpret_cast<float4*>(srow + ((j4 ^ (lane & 7)) << 2)) = make_float4(v[j4 * 4], v[j4 * 4 + 1], v[j4 * 4 + 2], v[j4 * 4 + 3]);
-                        __syncwarp();
-                        const int rbase = m0 + q * 32;
-                        if (!bf_out) {
-                            float* gcol = g.resid + nb + lane;
-#pragma unroll
-                            for (int r8 = 0; r8 < 32; r8 += 8) {
-                                float xin[8];
-                                if (EPI == EPI_RESID) {
-#pragma unroll
-                                    for (int u = 0; u < 8; ++u) xin[u] = (rbase + r8 + u < R) ? gcol[(size_t)(rbase + r8 + u) * g.N] : 0.f;
-                                }
-#pragma unroll
-                                for (int u = 0; u < 8; ++u) {
-                                    const int rr = r8 + u;
-                                    float val = stg[rr * 32 + ((((lane >> 2) ^ (rr & 7))) << 2) + (lane & 3)];
-                                    if (EPI == EPI_RESID) val += xin[u];
-                                    if (rbase + rr < R) gcol[(size_t)(rbase + rr) * g.N] = val;
-                                }
-                            }
-                        } else {
-                            const int hl = lane >> 4, cl = lane & 15;           // half-warp per row, two columns per lane
-#pragma unroll 4
-                            for (int r2 = 0; r2 < 32; r2 += 2) {
-                                const int rr = r2 + hl, gr = rbase + rr;
-                                const long long row_of = (EPI == EPI_QKV) ? __shfl_sync(0xffffffffu, my_cache_row, rr) : 0;
-                                const float2 pv = *reinterpret_cast<const float2*>(stg + rr * 32 + (((cl >> 1) ^ (rr & 7)) << 2) + (cl & 1) * 2);
-                                if (gr < R) {
-                                    bf16* o = g.out + (size_t)gr * g.ldo + nb;
-                                    if (EPI == EPI_QKV && nb >= g.kv_d) {          // K or V part: straight into the paged cache
-                                        const size_t row = (size_t)row_of;
-                                        o = (nb < 2 * g.kv_d ? g.kc + row * g.kv_d + (nb - g.kv_d) : g.vc + row * g.kv_d + (nb - 2 * g.kv_d));
-                                    }
-                                    __nv_bfloat162 b2;
-                                    b2.x = __float2bfloat16_rn(pv.x); b2.y = __float2bfloat16_rn(pv.y);
-                                    *reinterpret_cast<__nv_bfloat162*>(o + cl * 2) = b2;
-                                }
-                            }
-                        }
-                        __syncwarp();
-                        continue;
                     }
                     if (r >= R) continue;
                     if (bf_out) {
@@ -429,9 +473,10 @@ struct TmaEncoder {
 
 inline bool tc_supported(int N, int K) { return K % TC_BK == 0 && K >= TC_BK && N >= 32; }
 
-template <int EPI, int BN>
+template <int EPI, int BN, int AR = 128>
 inline cudaError_t tc_set_smem() {
-    return cudaFuncSetAttribute(k_gemm_tc<EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<BN>::SMEM);
+    return cudaFuncSetAttribute(k_gemm_tc<EPI, BN, AR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                TcCfg<BN, AR, EPI != EPI_STATS>::SMEM);
 }
 template <int EPI>
 inline cudaError_t tc_set_smem_all() {
@@ -460,6 +505,9 @@ inline int tc_init(TmaEncoder& enc, int* err_word) {
     if (e == cudaSuccess) e = tc_set_smem_all<EPI_F32>();
     if (e == cudaSuccess) e = tc_set_smem_all<EPI_QKV>();
     if (e == cudaSuccess) e = tc_set_smem<EPI_STATS, 128>();
+    if (e == cudaSuccess) e = tc_set_smem<EPI_STATS, 224, 32>();
+    if (e == cudaSuccess) e = tc_set_smem<EPI_STATS, 224, 64>();
+    if (e == cudaSuccess) e = tc_set_smem<EPI_STATS, 224, 128>();
     if (e == cudaSuccess) e = tc_set_smem<EPI_STATS, 256>();
     if (e != cudaSuccess) { enc.err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e); return -1; }
     enc.err_word = err_word;
@@ -468,20 +516,20 @@ inline int tc_init(TmaEncoder& enc, int* err_word) {
     return 0;
 }
 
-template <int EPI, int BN>
+template <int EPI, int BN, int AR = 128>
 inline int tc_launch_one(TmaEncoder& enc, GemmArgs<bf16>& g, int rows_ub, cudaStream_t st) {
-    const CUtensorMap* ta = enc.get(g.A, rows_ub, g.K, g.lda, TC_BM);
+    const CUtensorMap* ta = enc.get(g.A, rows_ub, g.K, g.lda, AR);
     const CUtensorMap* tw = enc.get(g.W, g.N, g.K, g.K, BN);
     if (!ta || !tw) return -1;
     const long long tiles_ub = (long long)((g.N + BN - 1) / BN) * ((rows_ub + TC_BM - 1) / TC_BM);
     const int grid = (int)std::min<long long>(tiles_ub, enc.n_sm);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = TcCfg<BN>::SMEM; cfg.stream = st;
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = TcCfg<BN, AR, EPI != EPI_STATS>::SMEM; cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = enc.pdl ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, k_gemm_tc<EPI, BN>, *ta, *tw, g, enc.err_word);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_gemm_tc<EPI, BN, AR>, *ta, *tw, g, enc.err_word);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { enc.err = std::string("launch: ") + cudaGetErrorString(e); return -1; }
     return 0;
@@ -520,12 +568,23 @@ inline int gemm_tc_launch(TmaEncoder& enc, int epi, GemmArgs<bf16>& g, int rows_
     if (epi == EPI_STATS) {
         if (g.N < 128) return -2;
         const bool wide = rows_ub > 4 * TC_BM && g.N >= 256;    // many row tiles: wider tiles halve the re-reads of A
-        const int bn = wide ? 256 : 128;
+        int bn = wide ? 256 : 128;
+        // One row tile is pure weight streaming: when 128-wide tiles need a second, part-empty wave but 224-wide
+        // ones fit in one, every SM streams one equal slice of the matrix (32768 columns = 147 tiles of 224).
+        if (rows_ub <= TC_BM && (g.N + 127) / 128 > enc.n_sm && (g.N + 223) / 224 <= enc.n_sm) bn = 224;
+        if (enc.force_bn == 128 || enc.force_bn == 256 || (enc.force_bn == 224 && rows_ub <= TC_BM)) bn = enc.force_bn;
         g.n_tiles = 2 * ((g.N + bn - 1) / bn);                   // two column halves per tile
         if (n_tiles_out) *n_tiles_out = g.n_tiles;
-        return wide ? tc_launch_one<EPI_STATS, 256>(enc, g, rows_ub, st) : tc_launch_one<EPI_STATS, 128>(enc, g, rows_ub, st);
+        g.one_m_tile = (bn == 224);
+        if (bn == 224)      // one tile per CTA: the ring is as deep as shared memory allows, most of it requested up front
+            return rows_ub <= 32 ? tc_launch_one<EPI_STATS, 224, 32>(enc, g, rows_ub, st)
+                 : rows_ub <= 64 ? tc_launch_one<EPI_STATS, 224, 64>(enc, g, rows_ub, st)
+                                 : tc_launch_one<EPI_STATS, 224, 128>(enc, g, rows_ub, st);
+        return bn == 256 ? tc_launch_one<EPI_STATS, 256>(enc, g, rows_ub, st) : tc_launch_one<EPI_STATS, 128>(enc, g, rows_ub, st);
     }
-    const int bn = (enc.force_bn && enc.force_bn <= g.N) ? enc.force_bn : tc_pick_bn(g.N, rows_ub, enc.n_sm);
+    const int fb = enc.force_bn;
+    const bool forced = (fb == 32 || fb == 64 || fb == 128 || fb == 256) && fb <= g.N;
+    const int bn = forced ? fb : tc_pick_bn(g.N, rows_ub, enc.n_sm);
     switch (epi) {
         case EPI_STORE: return tc_launch_bn<EPI_STORE>(enc, bn, g, rows_ub, st);
         case EPI_RELU: return tc_launch_bn<EPI_RELU>(enc, bn, g, rows_ub, st);

@@ -55,9 +55,26 @@ int main(int argc,char**argv){
     printf("bulk SB=%d NS=%d ctas=%d: %.1f GB/s per CTA, %.1f GB/s total (%s)\n",SB,NS,c,per/ms/1e6,per*c/ms/1e6,cudaGetErrorString(cudaGetLastError()));
   }
   for(int c: ctas) for(int th: {256,1024}){
-    size_t per=(size_t)8<<20; float ms;
+    size_t per=(size_t)8<<20; if (per*c>total) per=total/c/4096*4096; float ms;   // stay inside the buffer
     k_ldg<<<c,th>>>((const uint4*)buf,per/16,sink); cudaDeviceSynchronize(); cudaEventRecord(e0); k_ldg<<<c,th>>>((const uint4*)buf,per/16,sink); cudaEventRecord(e1); cudaEventSynchronize(e1); cudaEventElapsedTime(&ms,e0,e1);
     printf("ldg threads=%d ctas=%d: %.1f GB/s per CTA, %.1f GB/s total\n",th,c,per/ms/1e6,per*c/ms/1e6);
+  }
+  // One-shot short stream: every SM pulls 224 KB once (33 MB in all, the size of the vocabulary matrix), after the
+  // L2 was filled with (a) clean lines by a read sweep, (b) dirty lines by a write sweep.  "empty" is the
+  // event-to-event time of a kernel that does nothing.
+  {
+    unsigned char* big; cudaMalloc(&big,(size_t)512<<20); cudaMemset(big,2,(size_t)512<<20);
+    const int SB=32768; const size_t per=(size_t)7*SB; size_t smem=(size_t)7*SB; float ms;
+    cudaFuncSetAttribute(k_bulk<7>,cudaFuncAttributeMaxDynamicSharedMemorySize,(int)smem);
+    for(int mode=0; mode<3; mode++) for(int rep=0; rep<3; rep++){
+      if(mode==0) k_ldg<<<592,1024>>>((const uint4*)big,((size_t)512<<20)/16/592,sink);
+      if(mode==1) cudaMemsetAsync(big,rep,(size_t)512<<20);
+      cudaDeviceSynchronize();
+      cudaEventRecord(e0);
+      if(mode==2) k_bulk<7><<<148,32,smem>>>(buf,0,SB,sink); else k_bulk<7><<<148,32,smem>>>(buf,per,SB,sink);
+      cudaEventRecord(e1); cudaEventSynchronize(e1); cudaEventElapsedTime(&ms,e0,e1);
+      printf("one-shot 148 x 224 KB after %s: %.2f us  (%.0f GB/s incl. launch)  (%s)\n", mode==0?"clean read sweep":mode==1?"dirty write sweep":"nothing (empty kernel)", ms*1e3, mode==2?0.0:per*148/ms/1e6, cudaGetErrorString(cudaGetLastError()));
+    }
   }
   return 0;
 }

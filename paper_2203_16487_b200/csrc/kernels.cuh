@@ -313,6 +313,7 @@ struct GemmArgs {
     int N, K;
     const int* n_rows;          // device row count
     int rows_static;            // >= 0: the row count is known on the host (saves a dependent load); else read n_rows
+    int one_m_tile;             // tensor-core path: the rows fit one 128-row tile whatever n_rows says
     T* out; int ldo;            // EPI_STORE / EPI_RELU
     float* resid;               // EPI_RESID: resid[r, n] += value ; EPI_F32: resid[r, n] = value (ld = N)
     // EPI_STATS

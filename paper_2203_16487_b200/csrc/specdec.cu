@@ -421,10 +421,11 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
     GemmArgs<T> g;
     g.A = (const T*)A; g.lda = lda; g.W = (const T*)W; g.bias = bias; g.N = N; g.K = K;
     g.n_rows = h->ses.counters + cnt; g.rows_static = (cnt == CNT_VERIFY || cnt == CNT_ENC) ? rows_ub : -1; g.out = (T*)out; g.ldo = ldo; g.resid = resid;
+    g.one_m_tile = 0;
     g.part = h->part; g.ld = ldv; g.ld_id = ld_id; g.n_tiles = cdiv(N, 64); g.want_sum = h->want_lse;
     g.seq = nullptr; g.pos = nullptr; g.kc = nullptr; g.vc = nullptr; g.kv_d = 0;
     g.pg.table = h->page_table; g.pg.page_tokens = h->cfg.page_tokens; g.pg.max_pages = h->pages_per_seq;
-    g.trace = (h->want_cl_trace && epi == EPI_STATS && h->cl_trace) ? h->cl_trace + 200 : nullptr;
+    g.trace = (h->want_cl_trace && h->cl_trace && epi == (h->want_cl_trace >= 10 ? h->want_cl_trace - 10 : EPI_STATS)) ? h->cl_trace + 200 : nullptr;
     if (kv) { g.seq = kv->seq; g.pos = kv->pos; g.kc = (T*)kv->kc; g.vc = (T*)kv->vc; g.kv_d = kv->d; }
     if constexpr (std::is_same<T, bf16>::value) {
         if (skinny) {
@@ -1167,7 +1168,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         h->use_tc = value ? 1 : 0;
         return SPECDEC_OK;
     }
-    if (!strcmp(name, "cl_trace")) { h->want_cl_trace = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "cl_trace")) { h->want_cl_trace = value; return SPECDEC_OK; }   // 10 + e: time the tensor-core GEMM with epilogue e instead of the vocabulary one
     if (!strcmp(name, "fused_attn")) { h->use_fused_attn = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }

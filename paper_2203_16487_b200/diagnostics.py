@@ -19,11 +19,11 @@ import torch
 from . import binding, workloads as W
 
 
-def _handle(k=25):
-    wl = W.config5_microbench(1, 64)
+def _handle(k=25, batch=1):
+    wl = W.config5_microbench(batch, 64)
     wv = W.make_weights(wl.verifier, wl.seed_verifier, True)
     wd = W.make_weights(wl.drafter, wl.seed_drafter, True)
-    sd = binding.SpecDec(wl.verifier, wv, wl.drafter, wd, k_max=k, max_batch=1, max_src=64, max_tgt=100, bf16=True)
+    sd = binding.SpecDec(wl.verifier, wv, wl.drafter, wd, k_max=k, max_batch=batch, max_src=64, max_tgt=100, bf16=True)
     src, lens = W.pad_batch(wl.src)
     return sd, src, lens
 
@@ -48,18 +48,21 @@ def cluster_trace(reps=20):
     sd.close()
 
 
-def vocab_trace(reps=20):
-    sd, src, lens = _handle()
+def vocab_trace(reps=20, opts=(), batch=1):
+    sd, src, lens = _handle(batch=batch)
     sd.set_option("cl_trace", 1); sd.set_option("graphs", 0)
+    for name, value in opts:
+        sd.set_option(name, value)
     sd.encode(src, lens, None)
-    drafts = np.arange(100, 125, dtype=np.int32)[None]
+    drafts = np.tile(np.arange(100, 125, dtype=np.int32)[None], (batch, 1))
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     for it in range(reps):
         flush.fill_(it & 0xff)
         sd.verify(drafts, 3, 1.0)
     torch.cuda.synchronize()
-    t = np.array(sd.cluster_trace(256), dtype=np.int64)[200:212]
-    names = ["kernel entry", "barriers + TMEM ready", "first TMA issued", "all TMA issued", "first stage landed",
+    t = np.array(sd.cluster_trace(256), dtype=np.int64)[200:214]
+    t = np.concatenate([t[:1], t[12:14], t[1:12]])
+    names = ["kernel entry", "mbarriers initialised", "TMEM allocated", "barriers + TMEM ready", "first TMA issued", "all TMA issued", "first stage landed",
              "tile 0 MMAs committed", "last tile MMAs committed", "epilogue tile 0 start", "epilogue tile 0 end",
              "epilogue tile 1 start", "epilogue tile 1 end", "exit"]
     for n, x in zip(names, t):
@@ -80,10 +83,12 @@ if __name__ == "__main__":
     ap.add_argument("--cluster-trace", action="store_true")
     ap.add_argument("--vocab-trace", action="store_true")
     ap.add_argument("--ingest-probe", action="store_true")
+    ap.add_argument("--batch", type=int, default=1, help="vocab trace: sequences in the verify step")
+    ap.add_argument("--opt", action="append", default=[], help="library option name=value (repeatable), vocab trace only")
     a = ap.parse_args()
     if a.cluster_trace:
         cluster_trace()
     if a.vocab_trace:
-        vocab_trace()
+        vocab_trace(batch=a.batch, opts=[(o.split("=")[0], int(o.split("=")[1])) for o in a.opt])
     if a.ingest_probe:
         ingest_probe()

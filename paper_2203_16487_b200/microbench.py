@@ -110,6 +110,7 @@ def main():
     ap.add_argument("--gemm", type=int, default=1)
     ap.add_argument("--graphs", type=int, default=1)
     ap.add_argument("--tc-bn", type=int, default=0, help="force the N tile of the tensor-core GEMM (experiments)")
+    ap.add_argument("--opt", action="append", default=[], help="library option name=value (repeatable; experiments)")
     ap.add_argument("--grid", action="store_true", help="the whole k x prefix x batch grid of the verify microbench")
     args = ap.parse_args()
     S = args.src_len
@@ -131,6 +132,8 @@ def main():
         sd.set_option("gemm", args.gemm)
         sd.set_option("graphs", args.graphs)
         sd.set_option("tc_bn", args.tc_bn)
+        for o in args.opt:
+            sd.set_option(o.split("=")[0], int(o.split("=")[1]))
         for j in prefixes:
             for k in ks:
                 us, us_min, mean_a = measure(sd, wl, B, k, j, S, args.reps, args.warmup, flush, args.draft)
