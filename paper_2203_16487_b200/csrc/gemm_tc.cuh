@@ -291,17 +291,30 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     }
                 }
             }
+            // ... and so are this lane's bias columns, its cache row and its draft logit
+            float4 bzv[NCH][2];
+            if (EPI != EPI_STATS && vec_ok && g.bias) {
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    const int nb = n0 + c * CW;
+                    if (nb + CW <= g.N) {
+                        const float4* bp = reinterpret_cast<const float4*>(g.bias + nb);
+                        if (bf_out) { bzv[c][0] = __ldg(bp + 2 * (lane & 3)); bzv[c][1] = __ldg(bp + 2 * (lane & 3) + 1); }
+                        else bzv[c][0] = __ldg(bp + (lane & 7));
+                    }
+                }
+            }
+            long long my_cache_row = 0;                          // EPI_QKV: cache row of this lane's output row
+            if (EPI == EPI_QKV && r < R) my_cache_row = (long long)g.pg.row(g.seq[r], g.pos[r]);
+            float ld = CUDART_INF_F; int id = -1;                // EPI_STATS: pre-pass logit and id of the row's draft
+            if (EPI == EPI_STATS && r < R) { if (g.ld) ld = g.ld[r]; if (g.ld_id) id = g.ld_id[r]; }
             const bool live = mbar_wait(smem_u32(&bar_acc_full[ab]), (i >> 1) & 1, abort_flag, err_word, 3);
             if (threadIdx.x == 64) tc_stamp(g.trace, 7 + 2 * (i > 0));
             tc_fence_after();
             const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16) + ab * BN + half * HALF;
             const bool warp_live = live && (m0 + q * 32 < R);    // warp-uniform: any live row in this quadrant
             float v[CW];
-            long long my_cache_row = 0;                          // EPI_QKV: cache row of this lane's output row
-            if (EPI == EPI_QKV && warp_live && r < R) my_cache_row = (long long)g.pg.row(g.seq[r], g.pos[r]);
             if (warp_live && EPI == EPI_STATS) {
-                const float ld = (g.ld && r < R) ? g.ld[r] : CUDART_INF_F;
-                const int id = (g.ld_id && r < R) ? g.ld_id[r] : -1;
                 // four interleaved running statistics shorten the dependent chain; merged in column order
                 float mx[4]; int arg[4]; int cnt = 0;
 #pragma unroll
@@ -355,7 +368,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                         if (!bf_out) {
                             // fp32 rows: 8 lanes per row (4 columns each), 4 rows per pass
                             const int l8 = lane & 7, rsub = lane >> 3;
-                            const float4 bz = g.bias ? __ldg(reinterpret_cast<const float4*>(g.bias + nb) + l8) : make_float4(0.f, 0.f, 0.f, 0.f);
+                            const float4 bz = g.bias ? bzv[c][0] : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                             for (int ps = 0; ps < 8; ++ps) {
                                 const int rr = ps * 4 + rsub, gr = rbase + rr;
@@ -368,7 +381,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                             // bf16 rows: 4 lanes per row (8 columns = 16 bytes each), 8 rows per pass
                             const int c4 = lane & 3, rsub = lane >> 2;
                             float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
-                            if (g.bias) { b0 = __ldg(reinterpret_cast<const float4*>(g.bias + nb) + 2 * c4); b1 = __ldg(reinterpret_cast<const float4*>(g.bias + nb) + 2 * c4 + 1); }
+                            if (g.bias) { b0 = bzv[c][0]; b1 = bzv[c][1]; }
 #pragma unroll
                             for (int ps = 0; ps < 4; ++ps) {
                                 const int rr = ps * 8 + rsub, gr = rbase + rr;
