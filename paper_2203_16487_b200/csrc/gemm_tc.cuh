@@ -560,15 +560,17 @@ inline int tc_launch_bn(TmaEncoder& enc, int bn, GemmArgs<bf16>& g, int rows_ub,
 
 // Tile width: a CTA ingests (128 + BN) * K * 2 bytes per tile and the SMs are ingest-bound long before
 // they are math-bound, so pick the BN that minimises waves * (128 + BN); ties go to the narrower tile
-// (more tiles per CTA, so more of the epilogue overlaps the next tile's loads).
+// (more tiles per CTA, so more of the epilogue overlaps the next tile's loads).  32-wide tiles are for
+// matrices narrower than 64 only: their 16-column epilogue halves cannot use the 16-byte store path, and a
+// verify step over 78 rows measured 649 us with them against 399 us with 64-wide tiles.
 inline int tc_pick_bn(int N, int rows_ub, int n_sm) {
     const int m_tiles = (rows_ub + TC_BM - 1) / TC_BM;
-    const int cand[4] = {256, 128, 64, 32};
-    int best = 32; long long best_cost = -1;
-    for (int i = 0; i < 4; ++i) {
+    if (N < 64) return 32;
+    const int cand[3] = {256, 128, 64};
+    int best = 64; long long best_cost = -1;
+    for (int i = 0; i < 3; ++i) {
         const int bn = cand[i];
-        if (bn > N && bn != 32) continue;
-        if (bn == 32 && m_tiles > 1) continue;                 // the narrow tile only pays for a single row tile
+        if (bn > N && bn != 64) continue;
         const long long tiles = (long long)((N + bn - 1) / bn) * m_tiles;
         const long long cost = ((tiles + n_sm - 1) / n_sm) * (TC_BM + bn);
         if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best = bn; }

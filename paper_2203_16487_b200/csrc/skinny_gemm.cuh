@@ -1,4 +1,4 @@
-// Weight-streaming GEMM for a handful of activation rows (M <= 64):  C[r, n] = sum_k A[r, k] W[n, k].
+// Weight-streaming GEMM for a handful of activation rows (the library uses it for M <= 32):  C[r, n] = sum_k A[r, k] W[n, k].
 //
 // At batch 1 a verify block has k+1 = 26 rows, so every layer GEMM is a pass over its weight matrix
 // bounded by HBM, not by math.  This kernel is shaped for that: one CTA per 8 weight rows, so a

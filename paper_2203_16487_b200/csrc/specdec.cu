@@ -355,13 +355,16 @@ template <typename T> bool tc_usable(const specdec_handle* h, int N, int K) {
 // LayerNorm fused in front of a GEMM: x fp32 rows, gain, bias.
 struct LnSpec { const float* x; const float* g; const float* b; };
 
-// The weight-streaming kernel serves bf16 GEMMs over at most 64 rows (see skinny_gemm.cuh).
+// The weight-streaming kernel serves bf16 GEMMs over at most 32 rows (see skinny_gemm.cuh): measured on a
+// verify step, 26 rows take 362 us with it against 391 us with 64-wide tensor-core tiles, but 52 rows take
+// 500 us against 391 us, so anything beyond two 16-row tiles goes to the tile GEMM.
+constexpr int SK_ROWS_MAX = 32;
 template <typename T>
 bool skinny_ok(const specdec_handle* h, int epi, int rows_ub, int N, int K, bool with_ln) {
-    if (!std::is_same<T, bf16>::value || !h->use_skinny || rows_ub > 64) return false;
+    if (!std::is_same<T, bf16>::value || !h->use_skinny || rows_ub > SK_ROWS_MAX) return false;
     if (epi != EPI_STORE && epi != EPI_RELU && epi != EPI_RESID && epi != EPI_QKV) return false;
     if (K % 32 || (with_ln && (K % 128 || K > 512))) return false;
-    return skinny_smem(rows_ub <= 32 ? 2 : (rows_ub <= 48 ? 3 : 4), K) <= h->skinny_smem_cap;
+    return skinny_smem(2, K) <= h->skinny_smem_cap;
 }
 
 template <int EPI, int MT, int G>
@@ -380,8 +383,8 @@ int skinny_launch_ln(specdec_handle* h, SkinnyArgs& a, cudaStream_t st) {
 }
 template <int EPI>
 int skinny_launch_mt(specdec_handle* h, SkinnyArgs& a, int rows_ub, cudaStream_t st) {
-    return rows_ub <= 32 ? skinny_launch_ln<EPI, 2>(h, a, st)
-         : rows_ub <= 48 ? skinny_launch_ln<EPI, 3>(h, a, st) : skinny_launch_ln<EPI, 4>(h, a, st);
+    (void)rows_ub;
+    return skinny_launch_ln<EPI, 2>(h, a, st);
 }
 int skinny_launch(specdec_handle* h, int epi, SkinnyArgs& a, int rows_ub, cudaStream_t st) {
     switch (epi) {
@@ -399,12 +402,7 @@ cudaError_t skinny_attr(int bytes) {
     return e;
 }
 template <int EPI>
-cudaError_t skinny_attr_mt(int bytes) {
-    cudaError_t e = skinny_attr<EPI, 2>(bytes);
-    if (e == cudaSuccess) e = skinny_attr<EPI, 3>(bytes);
-    if (e == cudaSuccess) e = skinny_attr<EPI, 4>(bytes);
-    return e;
-}
+cudaError_t skinny_attr_mt(int bytes) { return skinny_attr<EPI, 2>(bytes); }
 
 // out = A W^T (+bias) with one of the epilogues; rows_ub bounds the grid, the live count is on the device.
 template <typename T>
@@ -1096,8 +1094,7 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
         }
         {
             const int kmax = std::max(h->d_max, h->f_max);
-            size_t need = std::min<size_t>(skinny_smem(4, kmax), 227 * 1024);
-            if (skinny_smem(2, kmax) > need) need = std::min<size_t>(skinny_smem(2, kmax), 227 * 1024);
+            size_t need = std::min<size_t>(skinny_smem(2, kmax), 227 * 1024);
             cudaError_t e = skinny_attr_mt<EPI_STORE>((int)need);
             if (e == cudaSuccess) e = skinny_attr_mt<EPI_RELU>((int)need);
             if (e == cudaSuccess) e = skinny_attr_mt<EPI_RESID>((int)need);

@@ -263,8 +263,8 @@ def test_bf16_mid_lockstep(gemm, attn):
 
 @pytest.mark.parametrize("nseq,skinny", [(2, 1), (4, 1), (2, 0)])
 def test_bf16_mid_small_batches_weight_streaming_gemm(nseq, skinny):
-    """Passes of at most 64 rows run the weight-streaming GEMM with fused LayerNorm (26 rows: two 16-row
-    tiles; 52 rows: four)."""
+    """Passes of at most 32 rows run the weight-streaming GEMM with fused LayerNorm (26 rows: two 16-row
+    tiles); 52 rows run one 128-row tile of the tensor-core GEMM with 64-wide column tiles."""
     wv, wd = W.make_weights(MID_V, 21, True), W.make_weights(MID_D, 22, True)
     mv, md = O.model_from(MID_V, wv, mode="bf16"), O.model_from(MID_D, wd, mode="bf16")
     rng = np.random.default_rng(8)
