@@ -48,14 +48,17 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
 __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
 
 constexpr int ATT_Q = 32;
-constexpr int ATT_THREADS = 256;          // 8 warps
+// NW warps per CTA: 8 when few CTAs are in flight (each CTA is one latency chain: more warps shorten it) or
+// when shared memory leaves room for one or two CTAs per SM; 4 when the SMs are saturated with CTAs anyway
+// (fewer duplicated fragment loads per CTA).
 inline size_t attn_tc_smem(int max_keys) {
     const int nkp = (max_keys + 15) & ~15;
     return (size_t)ATT_Q * 128 + (size_t)nkp * 256 + (size_t)ATT_Q * (nkp + 4) * 4 + 16;
 }
 
-template <bool PAGED>
-__global__ void __launch_bounds__(ATT_THREADS) k_attn_tc(AttnTcArgs a) {
+template <bool PAGED, int NW>
+__global__ void __launch_bounds__(NW * 32) k_attn_tc(AttnTcArgs a) {
+    constexpr int ATT_THREADS = NW * 32;
     extern __shared__ __align__(128) unsigned char sm[];
     __shared__ int s_nk[ATT_Q];
     __shared__ float s_sum[ATT_Q];
@@ -155,58 +158,60 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_tc(AttnTcArgs a) {
         }
     }
     __syncthreads();
-    // ---- softmax: 8 threads per row; P (bf16, un-normalised) overwrites the K tile
+    // ---- softmax: NW threads per row; P (bf16, un-normalised) overwrites the K tile
     {
         bf16* P = reinterpret_cast<bf16*>(Kp);
-        const int r = tid >> 3, sub = tid & 7;
+        const int r = tid / NW, sub = tid % NW;
         const float* srow = Ss + r * sstr;
         float m = -CUDART_INF_F;
-        for (int c = sub; c < nkp; c += 8) m = fmaxf(m, srow[c]);
-        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 4));
+        for (int c = sub; c < nkp; c += NW) m = fmaxf(m, srow[c]);
+#pragma unroll
+        for (int o = 1; o < NW; o <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
         float sum = 0.f;
-        for (int c = sub; c < nkp; c += 8) {
+        for (int c = sub; c < nkp; c += NW) {
             const float s = srow[c];
             const float e = (s == -CUDART_INF_F) ? 0.f : expf(s - m);
             sum += e;
             P[r * pstr + c] = __float2bfloat16_rn(e);
         }
-        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-        sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+#pragma unroll
+        for (int o = 1; o < NW; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
         if (sub == 0) s_sum[r] = sum;
     }
     __syncthreads();
-    // ---- O = P V ; warp w owns query rows 16 (w / 4) .. and head columns 16 (w % 4) ..
+    // ---- O = P V ; warp w owns query rows 16 (w / (NW / 2)) .. and 128 / NW head columns
     {
-        const int mt = warp >> 2, wq = warp & 3;
-        float acc[2][4];
+        constexpr int WPM = NW / 2;                  // warps per 16-row query tile
+        constexpr int NV = 64 / WPM / 16;            // 16-column groups per warp
+        const int mt = warp / WPM, wq = warp % WPM;
+        float acc[2 * NV][4];
 #pragma unroll
-        for (int j = 0; j < 2; ++j)
+        for (int j = 0; j < 2 * NV; ++j)
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[j][e] = 0.f;
         for (int kt = 0; kt < nkp / 16; ++kt) {
-            uint32_t vf[4], pf[4];
-            {
-                const int r = kt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = wq * 2 + (lane >> 4);
-                ldsm_x4_t(Vs + swz(r, c), vf[0], vf[1], vf[2], vf[3]);
-            }
+            uint32_t pf[4];
             {
                 const int r = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = kt * 16 + (lane >> 4) * 8;
                 ldsm_x4(Ks + (uint32_t)(r * pstr + c) * 2, pf[0], pf[1], pf[2], pf[3]);
             }
-            mma_bf16(acc[0], pf, vf[0], vf[1]);
-            mma_bf16(acc[1], pf, vf[2], vf[3]);
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                uint32_t vf[4];
+                const int r = kt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = (wq * NV + v) * 2 + (lane >> 4);
+                ldsm_x4_t(Vs + swz(r, c), vf[0], vf[1], vf[2], vf[3]);
+                mma_bf16(acc[2 * v], pf, vf[0], vf[1]);
+                mma_bf16(acc[2 * v + 1], pf, vf[2], vf[3]);
+            }
         }
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
             const int r = mt * 16 + g + half * 8;
             if (r < nq) {
                 const float den = s_sum[r];
-                bf16* o = a.out + (size_t)(r0 + r) * a.out_stride + h * 64 + wq * 16 + t4 * 2;
+                bf16* o = a.out + (size_t)(r0 + r) * a.out_stride + h * 64 + wq * (NV * 16) + t4 * 2;
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt) {
+                for (int nt = 0; nt < 2 * NV; ++nt) {
                     __nv_bfloat162 v2;
                     v2.x = __float2bfloat16_rn(den > 0.f ? acc[nt][half * 2] / den : 0.f);
                     v2.y = __float2bfloat16_rn(den > 0.f ? acc[nt][half * 2 + 1] / den : 0.f);

@@ -96,6 +96,7 @@ struct specdec_handle {
     int poll_lag = -1;              // -1: chosen by batch size
     int use_fused_attn = 0;         // attention + output projection as one cluster kernel (measured slower: off)
     size_t attn_proj_smem_cap = 0;
+    int attn_warps = 0;             // 0 = choose per launch, else 4 or 8 warps per tile-attention CTA (option "attn_warps")
     int skinny_groups = 1;          // 8-row weight groups per CTA of the weight-streaming GEMM (1, 2 or 4)
     // CUDA graphs of whole draft / verify(+commit) steps, keyed by everything their launches depend on
     struct GraphEntry { cudaGraphExec_t exec; long long kernels; };
@@ -475,8 +476,13 @@ int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* 
             a.out = (bf16*)out; a.out_stride = out_stride; a.max_keys = max_keys;
             a.scale = 1.0f / sqrtf((float)d_head);
             dim3 grid(cdiv(q_ub, ATT_Q), n_heads, h->B);
-            cudaError_t e = paged ? launch_pdl(h, k_attn_tc<true>, grid, dim3(ATT_THREADS), smem, st, a)
-                                  : launch_pdl(h, k_attn_tc<false>, grid, dim3(ATT_THREADS), smem, st, a);
+            // 4 warps when the SMs are saturated with CTAs anyway, 8 when a CTA's own latency chain is what counts
+            const long long ctas = (long long)grid.x * grid.y * grid.z, per_sm = (long long)(227 * 1024) / (long long)(smem + 1024);
+            const bool wide = h->attn_warps ? h->attn_warps == 8 : (per_sm <= 2 || ctas < 4LL * h->tma.n_sm);
+            cudaError_t e = wide ? (paged ? launch_pdl(h, k_attn_tc<true, 8>, grid, dim3(256), smem, st, a)
+                                          : launch_pdl(h, k_attn_tc<false, 8>, grid, dim3(256), smem, st, a))
+                                 : (paged ? launch_pdl(h, k_attn_tc<true, 4>, grid, dim3(128), smem, st, a)
+                                          : launch_pdl(h, k_attn_tc<false, 4>, grid, dim3(128), smem, st, a));
             if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(e));
             KCHECK(h);
             return 0;
@@ -848,7 +854,7 @@ void drop_graphs(specdec_handle* h) {
 // replayed afterwards.  The key must name everything the launches depend on besides device memory.
 template <typename F>
 int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body) {
-    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->use_fused_attn); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
+    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->attn_warps); key.push_back(h->use_fused_attn); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
     key.push_back(h->B); key.push_back(h->S_max);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
@@ -1087,8 +1093,10 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
     if (h->dtype == SPECDEC_DTYPE_BF16) {
         const int max_keys = std::max(h->S_cap, h->T_cap + h->k_cap + 1);
         h->attn_tc_smem_cap = std::min<size_t>(attn_tc_smem(max_keys), 227 * 1024);
-        if (cudaFuncSetAttribute(k_attn_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
-            cudaFuncSetAttribute(k_attn_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess) {
+        if (cudaFuncSetAttribute(k_attn_tc<true, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_tc<false, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_tc<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_tc<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess) {
             cudaGetLastError();
             h->attn_tc_smem_cap = 48 * 1024;
         }
@@ -1170,6 +1178,10 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
     if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "attn_warps")) {
+        if (value != 0 && value != 4 && value != 8) return fail(h, SPECDEC_ERR_INVALID_ARG, "attn_warps must be 0, 4 or 8");
+        h->attn_warps = value; return SPECDEC_OK;
+    }
     if (!strcmp(name, "pdl")) { h->use_pdl = value ? 1 : 0; h->tma.pdl = value != 0; return SPECDEC_OK; }
     if (!strcmp(name, "skinny")) { h->use_skinny = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "row_lse")) { h->want_lse = value ? 1 : 0; return SPECDEC_OK; }
