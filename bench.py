@@ -300,7 +300,11 @@ def run_ours(args):
     acc = sum(s["accepted"] for s in stats)
     d, V = wl.verifier.d_model, wl.verifier.vocab
     rows = B * (K_BLOCK + 1)
-    alg_bytes = V * d * 2 + rows * d * 2 + rows * (V // 128) * 16 + rows * 8
+    # column halves per row that the kernel writes 16-byte partial statistics for: one 224-wide tile per SM up to
+    # 128 rows, 128-wide tiles up to 512 rows, 256-wide above (the library's tile rule for this kernel)
+    tile = 224 if rows <= 128 else (128 if rows <= 512 else 256)
+    n_part = 2 * ((V + tile - 1) // tile)
+    alg_bytes = V * d * 2 + rows * d * 2 + rows * n_part * 16 + rows * 8
     per_launch_ms = vocab_ms / max(vocab_n, 1)
     achieved = alg_bytes / (per_launch_ms * 1e-3) / 1e9 if per_launch_ms > 0 else 0.0
     flops = 2.0 * rows * d * V
@@ -311,7 +315,7 @@ def run_ours(args):
             {"bound": "tensor", "achieved": tf, "peak": tc_peak, "unit": "TFLOP/s", "frac": tf / tc_peak})
     # DRAM bytes of one launch from the ncu capture summarised in profiles/vocab_stats_kernel_b1_ncu.md
     # (dram__bytes_read.sum + dram__bytes_write.sum at 26 rows); none was taken at other row counts
-    traffic = 33613824 if B == 1 else None
+    traffic = 33608960 if B == 1 else None
     roof.update({"traffic": traffic, "kernel": "k_gemm_tc<EPI_STATS> (vocabulary projection + row statistics, verify step)",
                  "peak_kind": f"of {peak_kind}", "launches_timed": int(vocab_n), "us_per_launch": per_launch_ms * 1e3,
                  "algorithmic_bytes_per_launch": alg_bytes})
