@@ -153,6 +153,189 @@ __device__ __forceinline__ void tmem_ld(uint32_t taddr, float* v) {
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// One tile of the epilogue, for one of the eight epilogue warps: q = the TMEM lane quadrant the warp may read,
+// half = which half of the tile's BN columns it takes; tmem_acc = the tile's accumulator.  Requests what it can
+// before waiting for the accumulator (residual tile, bias, cache rows, draft logits), then reads tensor memory
+// chunk by chunk.  The caller hands the accumulator back afterwards.
+template <int EPI, int BN>
+__device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R, int m0, int n_tile, int q, int half, int lane,
+                                                 uint32_t tmem_acc, float* stg, uint32_t bar_acc_full_addr, uint32_t parity,
+                                                 volatile int* abort_flag, int* err_word, bool later_tile) {
+    constexpr int HALF = BN / 2;                     // columns per epilogue warp
+    constexpr int CW = HALF % 32 == 0 ? 32 : 16;     // columns per TMEM read
+    constexpr bool bf_out = (EPI == EPI_STORE || EPI == EPI_RELU || EPI == EPI_QKV);
+    constexpr int NCH = HALF / CW;                   // column chunks per warp and tile
+    // 16-byte accesses after the transpose need aligned rows
+    const bool vec_ok = CW == 32 && (bf_out ? (g.ldo % 8 == 0 && (EPI != EPI_QKV || g.kv_d % 32 == 0)) : (g.N % 4 == 0));
+    const int n0 = n_tile * BN + half * HALF;
+    const int r = m0 + q * 32 + lane;
+    const int rbase = m0 + q * 32;
+    // EPI_RESID: the residual values of the first two column chunks are requested before the accumulator
+    // is awaited, so their latency hides behind the MMAs
+    float4 xin[2][8];
+    if (EPI == EPI_RESID && vec_ok && rbase < R) {
+#pragma unroll
+        for (int c = 0; c < (NCH < 2 ? NCH : 2); ++c) {
+            const int nb = n0 + c * CW;
+            if (nb + CW <= g.N) {
+#pragma unroll
+                for (int ps = 0; ps < 8; ++ps) {
+                    const int gr = rbase + ps * 4 + (lane >> 3);
+                    xin[c][ps] = gr < R ? *reinterpret_cast<const float4*>(g.resid + (size_t)gr * g.N + nb + (lane & 7) * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+        }
+    }
+    // ... and so are this lane's bias columns, its cache row and its draft logit
+    float4 bzv[NCH][2];
+    if (EPI != EPI_STATS && vec_ok && g.bias) {
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+            const int nb = n0 + c * CW;
+            if (nb + CW <= g.N) {
+                const float4* bp = reinterpret_cast<const float4*>(g.bias + nb);
+                if (bf_out) { bzv[c][0] = __ldg(bp + 2 * (lane & 3)); bzv[c][1] = __ldg(bp + 2 * (lane & 3) + 1); }
+                else bzv[c][0] = __ldg(bp + (lane & 7));
+            }
+        }
+    }
+    long long my_cache_row = 0;                          // EPI_QKV: cache row of this lane's output row
+    if (EPI == EPI_QKV && r < R) my_cache_row = (long long)g.pg.row(g.seq[r], g.pos[r]);
+    float ld = CUDART_INF_F; int id = -1;                // EPI_STATS: pre-pass logit and id of the row's draft
+    if (EPI == EPI_STATS && r < R) { if (g.ld) ld = g.ld[r]; if (g.ld_id) id = g.ld_id[r]; }
+    const bool live = mbar_wait(bar_acc_full_addr, parity, abort_flag, err_word, 3);
+    if (threadIdx.x == 64) tc_stamp(g.trace, 7 + 2 * (later_tile ? 1 : 0));
+    tc_fence_after();
+    const uint32_t trow = tmem_acc + ((uint32_t)(q * 32) << 16) + half * HALF;
+    const bool warp_live = live && (m0 + q * 32 < R);    // warp-uniform: any live row in this quadrant
+    float v[CW];
+    if (warp_live && EPI == EPI_STATS) {
+        // four interleaved running statistics shorten the dependent chain; merged in column order
+        float mx[4]; int arg[4]; int cnt = 0;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { mx[u] = -CUDART_INF_F; arg[u] = 0x7fffffff; }
+        for (int c = 0; c < HALF / CW; ++c) {
+            tmem_ld<CW>(trow + c * CW, v);
+#pragma unroll
+            for (int j = 0; j < CW; ++j) {
+                const int n = n0 + c * CW + j;
+                const float x = (n >= g.N) ? -CUDART_INF_F : ((n == id) ? ld : v[j]);   // draft column: pre-pass value
+                if (x > mx[j & 3]) { mx[j & 3] = x; arg[j & 3] = n; }
+                cnt += (x > ld) ? 1 : 0;
+            }
+        }
+        RowPart p; p.mx = mx[0]; p.arg = arg[0]; p.sum = 0.f; p.cnt = cnt;
+#pragma unroll
+        for (int u = 1; u < 4; ++u)
+            if (mx[u] > p.mx || (mx[u] == p.mx && arg[u] < p.arg)) { p.mx = mx[u]; p.arg = arg[u]; }
+        if (g.want_sum) {
+            for (int c = 0; c < HALF / CW; ++c) {
+                tmem_ld<CW>(trow + c * CW, v);
+#pragma unroll
+                for (int j = 0; j < CW; ++j) {
+                    const int n = n0 + c * CW + j;
+                    if (n < g.N) p.sum += expf(((n == id) ? ld : v[j]) - p.mx);
+                }
+            }
+        }
+        if (r < R) g.part[(size_t)r * g.n_tiles + n_tile * 2 + half] = p;
+    } else if (warp_live) {
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+            const int nb = n0 + c * CW;
+            if (EPI == EPI_RESID && c >= 2 && vec_ok && nb + CW <= g.N) {      // chunks 0 and 1 were requested before the wait
+#pragma unroll
+                for (int ps = 0; ps < 8; ++ps) {
+                    const int gr = rbase + ps * 4 + (lane >> 3);
+                    xin[c & 1][ps] = gr < R ? *reinterpret_cast<const float4*>(g.resid + (size_t)gr * g.N + nb + (lane & 7) * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+            tmem_ld<CW>(trow + c * CW, v);
+            if (CW == 32 && vec_ok && nb + CW <= g.N) {
+                // Transpose through shared memory: a thread owns one output ROW in tensor memory, but global
+                // memory wants neighbouring lanes on neighbouring addresses.  The 32 x 32 block is written row-wise
+                // with its 16-byte chunks XOR-swizzled by the row, then read back 16 bytes of output per lane.
+                float* srow = stg + lane * 32;
+#pragma unroll
+                for (int j4 = 0; j4 < 8; ++j4)
+                    *reinterpret_cast<float4*>(srow + ((j4 ^ (lane & 7)) << 2)) = make_float4(v[j4 * 4], v[j4 * 4 + 1], v[j4 * 4 + 2], v[j4 * 4 + 3]);
+                __syncwarp();
+                if (!bf_out) {
+                    // fp32 rows: 8 lanes per row (4 columns each), 4 rows per pass
+                    const int l8 = lane & 7, rsub = lane >> 3;
+                    const float4 bz = g.bias ? bzv[c][0] : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int ps = 0; ps < 8; ++ps) {
+                        const int rr = ps * 4 + rsub, gr = rbase + rr;
+                        float4 a = *reinterpret_cast<const float4*>(stg + rr * 32 + ((l8 ^ (rr & 7)) << 2));
+                        a.x += bz.x; a.y += bz.y; a.z += bz.z; a.w += bz.w;
+                        if (EPI == EPI_RESID) { const float4 x = xin[c & 1][ps]; a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w; }
+                        if (gr < R) *reinterpret_cast<float4*>(g.resid + (size_t)gr * g.N + nb + l8 * 4) = a;
+                    }
+                } else {
+                    // bf16 rows: 4 lanes per row (8 columns = 16 bytes each), 8 rows per pass
+                    const int c4 = lane & 3, rsub = lane >> 2;
+                    float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
+                    if (g.bias) { b0 = bzv[c][0]; b1 = bzv[c][1]; }
+#pragma unroll
+                    for (int ps = 0; ps < 4; ++ps) {
+                        const int rr = ps * 8 + rsub, gr = rbase + rr;
+                        const long long row_of = (EPI == EPI_QKV) ? __shfl_sync(0xffffffffu, my_cache_row, rr) : 0;
+                        float4 a0 = *reinterpret_cast<const float4*>(stg + rr * 32 + (((2 * c4) ^ (rr & 7)) << 2));
+                        float4 a1 = *reinterpret_cast<const float4*>(stg + rr * 32 + (((2 * c4 + 1) ^ (rr & 7)) << 2));
+                        a0.x += b0.x; a0.y += b0.y; a0.z += b0.z; a0.w += b0.w;
+                        a1.x += b1.x; a1.y += b1.y; a1.z += b1.z; a1.w += b1.w;
+                        if (EPI == EPI_RELU) {
+                            a0.x = fmaxf(a0.x, 0.f); a0.y = fmaxf(a0.y, 0.f); a0.z = fmaxf(a0.z, 0.f); a0.w = fmaxf(a0.w, 0.f);
+                            a1.x = fmaxf(a1.x, 0.f); a1.y = fmaxf(a1.y, 0.f); a1.z = fmaxf(a1.z, 0.f); a1.w = fmaxf(a1.w, 0.f);
+                        }
+                        if (gr < R) {
+                            bf16* o = g.out + (size_t)gr * g.ldo + nb;
+                            if (EPI == EPI_QKV && nb >= g.kv_d) {          // K or V part: straight into the paged cache
+                                const size_t row = (size_t)row_of;
+                                o = (nb < 2 * g.kv_d ? g.kc + row * g.kv_d + (nb - g.kv_d) : g.vc + row * g.kv_d + (nb - 2 * g.kv_d));
+                            }
+                            __nv_bfloat162 p0 = __floats2bfloat162_rn(a0.x, a0.y), p1 = __floats2bfloat162_rn(a0.z, a0.w);
+                            __nv_bfloat162 p2 = __floats2bfloat162_rn(a1.x, a1.y), p3 = __floats2bfloat162_rn(a1.z, a1.w);
+                            uint4 pk;
+                            pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+                            pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+                            *reinterpret_cast<uint4*>(o + c4 * 8) = pk;
+                        }
+                    }
+                }
+                __syncwarp();
+                continue;
+            }
+            // ragged or unaligned chunk: one row per thread, element by element
+            if (g.bias) {
+#pragma unroll
+                for (int j = 0; j < CW; ++j) v[j] += (nb + j < g.N) ? __ldg(g.bias + nb + j) : 0.f;
+            }
+            if (EPI == EPI_RELU) {
+#pragma unroll
+                for (int j = 0; j < CW; ++j) v[j] = fmaxf(v[j], 0.f);
+            }
+            if (r >= R) continue;
+            if (bf_out) {
+                bf16* o = g.out + (size_t)r * g.ldo + nb;
+                if (EPI == EPI_QKV && nb >= g.kv_d) {
+                    const size_t row = g.pg.row(g.seq[r], g.pos[r]);
+                    o = (nb < 2 * g.kv_d ? g.kc + row * g.kv_d + (nb - g.kv_d) : g.vc + row * g.kv_d + (nb - 2 * g.kv_d));
+                }
+                for (int j = 0; j < CW; ++j)
+                    if (nb + j < g.N) o[j] = __float2bfloat16_rn(v[j]);
+            } else {
+                float* o = g.resid + (size_t)r * g.N + nb;
+                for (int j = 0; j < CW; ++j)
+                    if (nb + j < g.N) o[j] = (EPI == EPI_RESID ? o[j] : 0.f) + v[j];
+            }
+        }
+    }
+    tc_fence_before();
+    __syncwarp();
+}
+
 // Persistent kernel: CTA c works on tiles c, c + gridDim.x, ... (row tile fastest, so CTAs running
 // together share one weight tile).  The TMA ring and the two TMEM accumulators run across tiles, so the
 // epilogue of tile i overlaps the loads and MMAs of tile i + 1.
@@ -163,9 +346,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     using Cfg = TcCfg<BN, AR, EPI != EPI_STATS>;
     constexpr int STAGES = Cfg::STAGES;
     constexpr int A_BYTES = AR * TC_BK * 2;          // activation part of a stage
-    constexpr int HALF = BN / 2;                     // columns per epilogue warp
     if (threadIdx.x == 0) tc_stamp(g.trace, 0);
-    constexpr int CW = HALF % 32 == 0 ? 32 : 16;     // columns per TMEM read
     // With a row count known on the host the kernel can set itself up and start streaming weight tiles before
     // its predecessor has finished (programmatic dependent launch); a device-side count must be waited for.
     // So can a launch whose rows fit one row tile whatever their count (one_m_tile): the count is read later.
@@ -265,181 +446,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     } else {
         const int q = warp & 3;                                  // TMEM lane quadrant this warp may read
         const int half = (warp - 2) >> 2;                        // which half of the tile's columns
-        constexpr bool bf_out = (EPI == EPI_STORE || EPI == EPI_RELU || EPI == EPI_QKV);
-        constexpr int NCH = HALF / CW;                           // column chunks per warp and tile
-        // 16-byte accesses after the transpose need aligned rows
-        const bool vec_ok = CW == 32 && (bf_out ? (g.ldo % 8 == 0 && (EPI != EPI_QKV || g.kv_d % 32 == 0)) : (g.N % 4 == 0));
         int i = 0;
         for (int t = blockIdx.x; t < total; t += gridDim.x, ++i) {
             const int ab = i & 1;
-            const int m0 = (t % m_tiles) * TC_BM, n_tile = t / m_tiles, n0 = n_tile * BN + half * HALF;
-            const int r = m0 + q * 32 + lane;
-            const int rbase = m0 + q * 32;
-            // EPI_RESID: the residual values of the first two column chunks are requested before the accumulator
-            // is awaited, so their latency hides behind the MMAs
-            float4 xin[2][8];
-            if (EPI == EPI_RESID && vec_ok && rbase < R) {
-#pragma unroll
-                for (int c = 0; c < (NCH < 2 ? NCH : 2); ++c) {
-                    const int nb = n0 + c * CW;
-                    if (nb + CW <= g.N) {
-#pragma unroll
-                        for (int ps = 0; ps < 8; ++ps) {
-                            const int gr = rbase + ps * 4 + (lane >> 3);
-                            xin[c][ps] = gr < R ? *reinterpret_cast<const float4*>(g.resid + (size_t)gr * g.N + nb + (lane & 7) * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
-                    }
-                }
-            }
-            // ... and so are this lane's bias columns, its cache row and its draft logit
-            float4 bzv[NCH][2];
-            if (EPI != EPI_STATS && vec_ok && g.bias) {
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    const int nb = n0 + c * CW;
-                    if (nb + CW <= g.N) {
-                        const float4* bp = reinterpret_cast<const float4*>(g.bias + nb);
-                        if (bf_out) { bzv[c][0] = __ldg(bp + 2 * (lane & 3)); bzv[c][1] = __ldg(bp + 2 * (lane & 3) + 1); }
-                        else bzv[c][0] = __ldg(bp + (lane & 7));
-                    }
-                }
-            }
-            long long my_cache_row = 0;                          // EPI_QKV: cache row of this lane's output row
-            if (EPI == EPI_QKV && r < R) my_cache_row = (long long)g.pg.row(g.seq[r], g.pos[r]);
-            float ld = CUDART_INF_F; int id = -1;                // EPI_STATS: pre-pass logit and id of the row's draft
-            if (EPI == EPI_STATS && r < R) { if (g.ld) ld = g.ld[r]; if (g.ld_id) id = g.ld_id[r]; }
-            const bool live = mbar_wait(smem_u32(&bar_acc_full[ab]), (i >> 1) & 1, abort_flag, err_word, 3);
-            if (threadIdx.x == 64) tc_stamp(g.trace, 7 + 2 * (i > 0));
-            tc_fence_after();
-            const uint32_t trow = tmem_d + ((uint32_t)(q * 32) << 16) + ab * BN + half * HALF;
-            const bool warp_live = live && (m0 + q * 32 < R);    // warp-uniform: any live row in this quadrant
-            float v[CW];
-            if (warp_live && EPI == EPI_STATS) {
-                // four interleaved running statistics shorten the dependent chain; merged in column order
-                float mx[4]; int arg[4]; int cnt = 0;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) { mx[u] = -CUDART_INF_F; arg[u] = 0x7fffffff; }
-                for (int c = 0; c < HALF / CW; ++c) {
-                    tmem_ld<CW>(trow + c * CW, v);
-#pragma unroll
-                    for (int j = 0; j < CW; ++j) {
-                        const int n = n0 + c * CW + j;
-                        const float x = (n >= g.N) ? -CUDART_INF_F : ((n == id) ? ld : v[j]);   // draft column: pre-pass value
-                        if (x > mx[j & 3]) { mx[j & 3] = x; arg[j & 3] = n; }
-                        cnt += (x > ld) ? 1 : 0;
-                    }
-                }
-                RowPart p; p.mx = mx[0]; p.arg = arg[0]; p.sum = 0.f; p.cnt = cnt;
-#pragma unroll
-                for (int u = 1; u < 4; ++u)
-                    if (mx[u] > p.mx || (mx[u] == p.mx && arg[u] < p.arg)) { p.mx = mx[u]; p.arg = arg[u]; }
-                if (g.want_sum) {
-                    for (int c = 0; c < HALF / CW; ++c) {
-                        tmem_ld<CW>(trow + c * CW, v);
-#pragma unroll
-                        for (int j = 0; j < CW; ++j) {
-                            const int n = n0 + c * CW + j;
-                            if (n < g.N) p.sum += expf(((n == id) ? ld : v[j]) - p.mx);
-                        }
-                    }
-                }
-                if (r < R) g.part[(size_t)r * g.n_tiles + n_tile * 2 + half] = p;
-            } else if (warp_live) {
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    const int nb = n0 + c * CW;
-                    if (EPI == EPI_RESID && c >= 2 && vec_ok && nb + CW <= g.N) {      // chunks 0 and 1 were requested before the wait
-#pragma unroll
-                        for (int ps = 0; ps < 8; ++ps) {
-                            const int gr = rbase + ps * 4 + (lane >> 3);
-                            xin[c & 1][ps] = gr < R ? *reinterpret_cast<const float4*>(g.resid + (size_t)gr * g.N + nb + (lane & 7) * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
-                    }
-                    tmem_ld<CW>(trow + c * CW, v);
-                    if (CW == 32 && vec_ok && nb + CW <= g.N) {
-                        // Transpose through shared memory: a thread owns one output ROW in tensor memory, but global
-                        // memory wants neighbouring lanes on neighbouring addresses.  The 32 x 32 block is written row-wise
-                        // with its 16-byte chunks XOR-swizzled by the row, then read back 16 bytes of output per lane.
-                        float* srow = stg + lane * 32;
-#pragma unroll
-                        for (int j4 = 0; j4 < 8; ++j4)
-                            *reinterpret_cast<float4*>(srow + ((j4 ^ (lane & 7)) << 2)) = make_float4(v[j4 * 4], v[j4 * 4 + 1], v[j4 * 4 + 2], v[j4 * 4 + 3]);
-                        __syncwarp();
-                        if (!bf_out) {
-                            // fp32 rows: 8 lanes per row (4 columns each), 4 rows per pass
-                            const int l8 = lane & 7, rsub = lane >> 3;
-                            const float4 bz = g.bias ? bzv[c][0] : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                            for (int ps = 0; ps < 8; ++ps) {
-                                const int rr = ps * 4 + rsub, gr = rbase + rr;
-                                float4 a = *reinterpret_cast<const float4*>(stg + rr * 32 + ((l8 ^ (rr & 7)) << 2));
-                                a.x += bz.x; a.y += bz.y; a.z += bz.z; a.w += bz.w;
-                                if (EPI == EPI_RESID) { const float4 x = xin[c & 1][ps]; a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w; }
-                                if (gr < R) *reinterpret_cast<float4*>(g.resid + (size_t)gr * g.N + nb + l8 * 4) = a;
-                            }
-                        } else {
-                            // bf16 rows: 4 lanes per row (8 columns = 16 bytes each), 8 rows per pass
-                            const int c4 = lane & 3, rsub = lane >> 2;
-                            float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
-                            if (g.bias) { b0 = bzv[c][0]; b1 = bzv[c][1]; }
-#pragma unroll
-                            for (int ps = 0; ps < 4; ++ps) {
-                                const int rr = ps * 8 + rsub, gr = rbase + rr;
-                                const long long row_of = (EPI == EPI_QKV) ? __shfl_sync(0xffffffffu, my_cache_row, rr) : 0;
-                                float4 a0 = *reinterpret_cast<const float4*>(stg + rr * 32 + (((2 * c4) ^ (rr & 7)) << 2));
-                                float4 a1 = *reinterpret_cast<const float4*>(stg + rr * 32 + (((2 * c4 + 1) ^ (rr & 7)) << 2));
-                                a0.x += b0.x; a0.y += b0.y; a0.z += b0.z; a0.w += b0.w;
-                                a1.x += b1.x; a1.y += b1.y; a1.z += b1.z; a1.w += b1.w;
-                                if (EPI == EPI_RELU) {
-                                    a0.x = fmaxf(a0.x, 0.f); a0.y = fmaxf(a0.y, 0.f); a0.z = fmaxf(a0.z, 0.f); a0.w = fmaxf(a0.w, 0.f);
-                                    a1.x = fmaxf(a1.x, 0.f); a1.y = fmaxf(a1.y, 0.f); a1.z = fmaxf(a1.z, 0.f); a1.w = fmaxf(a1.w, 0.f);
-                                }
-                                if (gr < R) {
-                                    bf16* o = g.out + (size_t)gr * g.ldo + nb;
-                                    if (EPI == EPI_QKV && nb >= g.kv_d) {          // K or V part: straight into the paged cache
-                                        const size_t row = (size_t)row_of;
-                                        o = (nb < 2 * g.kv_d ? g.kc + row * g.kv_d + (nb - g.kv_d) : g.vc + row * g.kv_d + (nb - 2 * g.kv_d));
-                                    }
-                                    __nv_bfloat162 p0 = __floats2bfloat162_rn(a0.x, a0.y), p1 = __floats2bfloat162_rn(a0.z, a0.w);
-                                    __nv_bfloat162 p2 = __floats2bfloat162_rn(a1.x, a1.y), p3 = __floats2bfloat162_rn(a1.z, a1.w);
-                                    uint4 pk;
-                                    pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
-                                    pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
-                                    *reinterpret_cast<uint4*>(o + c4 * 8) = pk;
-                                }
-                            }
-                        }
-                        __syncwarp();
-                        continue;
-                    }
-                    // ragged or unaligned chunk: one row per thread, element by element
-                    if (g.bias) {
-#pragma unroll
-                        for (int j = 0; j < CW; ++j) v[j] += (nb + j < g.N) ? __ldg(g.bias + nb + j) : 0.f;
-                    }
-                    if (EPI == EPI_RELU) {
-#pragma unroll
-                        for (int j = 0; j < CW; ++j) v[j] = fmaxf(v[j], 0.f);
-                    }
-                    if (r >= R) continue;
-                    if (bf_out) {
-                        bf16* o = g.out + (size_t)r * g.ldo + nb;
-                        if (EPI == EPI_QKV && nb >= g.kv_d) {
-                            const size_t row = g.pg.row(g.seq[r], g.pos[r]);
-                            o = (nb < 2 * g.kv_d ? g.kc + row * g.kv_d + (nb - g.kv_d) : g.vc + row * g.kv_d + (nb - 2 * g.kv_d));
-                        }
-                        for (int j = 0; j < CW; ++j)
-                            if (nb + j < g.N) o[j] = __float2bfloat16_rn(v[j]);
-                    } else {
-                        float* o = g.resid + (size_t)r * g.N + nb;
-                        for (int j = 0; j < CW; ++j)
-                            if (nb + j < g.N) o[j] = (EPI == EPI_RESID ? o[j] : 0.f) + v[j];
-                    }
-                }
-            }
+            const int m0 = (t % m_tiles) * TC_BM, n_tile = t / m_tiles;
+            tc_epilogue_tile<EPI, BN>(g, R, m0, n_tile, q, half, lane, tmem_d + ab * BN, stg, smem_u32(&bar_acc_full[ab]),
+                                      (i >> 1) & 1, abort_flag, err_word, i > 0);
             // this warp is done with the accumulator: hand it back to the MMA warp
-            tc_fence_before();
-            __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[ab]));
             if (threadIdx.x == 64) tc_stamp(g.trace, 8 + 2 * (i > 0));
         }

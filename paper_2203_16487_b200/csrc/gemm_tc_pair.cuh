@@ -1,0 +1,246 @@
+// Two-SM variant of the tensor-core GEMM (tcgen05 cta_group::2) for the wide GEMMs over many rows.
+//
+// A cluster of two CTAs works on one 256-row x BN-column tile.  Each CTA stages its own 128 activation
+// rows and HALF of the weight tile (BN / 2 weight rows); one thread of the leader CTA (cluster rank 0)
+// issues tcgen05.mma.cta_group::2 with M = 256, which reads both CTAs' shared memory and leaves rows
+// 0..127 of the result in the leader's tensor memory and rows 128..255 in the peer's.  A CTA therefore
+// ingests (128 + BN / 2) * K * 2 bytes per 128 x BN outputs instead of (128 + BN) * K * 2: the single-SM
+// kernel is bound by exactly that ingest, not by the MMAs.
+//
+// Synchronisation (every wait is bounded, as in the single-SM kernel):
+//   full[s]      in the leader: its producer expects the bytes of BOTH CTAs' loads; both CTAs' TMA loads
+//                (cta_group::2 form, no multicast) complete their bytes on it;
+//   empty[s]     in each CTA, acc_full[i] in each CTA: signalled by the leader's MMA thread with one
+//                multicast tcgen05.commit (same barrier offset in both CTAs);
+//   acc_empty[i] in the leader: the eight epilogue warps of both CTAs arrive on it (the peer's remotely).
+// Cluster barriers bracket the kernel so that no CTA touches the other's barriers before they exist or
+// leaves while the other may still read its shared memory.
+#pragma once
+#include "gemm_tc.cuh"
+
+namespace sd {
+
+__device__ __forceinline__ uint32_t pair_cta_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t pair_map(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void pair_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA tile load into this CTA's shared memory whose bytes are counted on a barrier given by its cluster address
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar_cluster) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar_cluster), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+// arrives, once the MMAs issued so far have completed, on the barrier at this offset in both CTAs of the pair
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+
+template <int BN, bool STG = true> struct TcPairCfg {
+    static constexpr int BNH = BN / 2;                                    // weight rows a CTA stages per tile
+    static constexpr int STAGE_BYTES = (TC_BM + BNH) * TC_BK * 2;
+    static constexpr int STG_BYTES = STG ? TC_EPI_WARPS * 32 * 32 * 4 : 0;
+    static constexpr int FIT = (232448 - 1024 - STG_BYTES) / STAGE_BYTES;
+    static constexpr int STAGES = FIT > 8 ? 8 : FIT;
+    static constexpr int SMEM = STAGES * STAGE_BYTES + STG_BYTES + 1024;
+    static constexpr int TMEM_COLS = 2 * BN <= 128 ? 128 : (2 * BN <= 256 ? 256 : 512);   // two accumulators
+    static_assert(BN % 32 == 0 && BN >= 64 && BN <= 256, "pair tile width");
+};
+
+// Persistent over pair tiles: pair p works on tiles p, p + pairs, ... (row pair fastest, so pairs running
+// together share one weight tile).  Ring and accumulators run across tiles as in the single-SM kernel.
+template <int EPI, int BN>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
+k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, GemmArgs<bf16> g,
+               int* err_word) {
+    using Cfg = TcPairCfg<BN, EPI != EPI_STATS>;
+    constexpr int STAGES = Cfg::STAGES, BNH = Cfg::BNH;
+    constexpr int A_BYTES = TC_BM * TC_BK * 2;
+    const bool early = g.rows_static >= 0;
+    if (!early) pdl_wait();
+    const int R = early ? g.rows_static : *g.n_rows;
+    const int m_pairs = (R + 2 * TC_BM - 1) / (2 * TC_BM), n_tiles = (g.N + BN - 1) / BN;
+    const int total = m_pairs * n_tiles;
+    const int pair = (int)blockIdx.x >> 1, pairs = (int)gridDim.x >> 1;
+    if (pair >= total) return;                       // both CTAs of the pair leave together, before any cluster barrier
+
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[STAGES], bar_empty[STAGES], bar_acc_full[2], bar_acc_empty[2];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+    const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = pair_cta_rank();
+    const bool leader = rank == 0;
+    const int nkb = g.K / TC_BK;
+    float* stg = reinterpret_cast<float*>(smem_raw + (tiles - smem_u32(smem_raw)) + STAGES * Cfg::STAGE_BYTES) + (warp >= 2 ? warp - 2 : 0) * 1024;
+
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&bar_full[s]), 1); mbar_init(smem_u32(&bar_empty[s]), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bar_acc_full[i]), 1); mbar_init(smem_u32(&bar_acc_empty[i]), 2 * TC_EPI_WARPS); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc_pair(smem_u32(&tmem_base_s), Cfg::TMEM_COLS);
+    tc_fence_before();
+    pair_sync();                                     // both CTAs' barriers and tensor memory exist from here on
+    tc_fence_after();
+    const uint32_t tmem_d = tmem_base_s;
+    volatile int* abort_flag = &abort_s;
+    int pre = 0;                                     // stages whose weight halves were requested before the wait
+    if (early) {
+        if (threadIdx.x == 0) {
+            const int n0 = (pair / m_pairs) * BN + (int)rank * BNH;
+            for (; pre < STAGES && pre < nkb; ++pre) {
+                if (leader) mbar_expect_tx(smem_u32(&bar_full[pre]), 2 * Cfg::STAGE_BYTES);
+                tma_load_2d_pair(tiles + pre * Cfg::STAGE_BYTES + A_BYTES, &tmW, pre * TC_BK, n0, pair_map(smem_u32(&bar_full[pre]), 0));
+            }
+        }
+        pdl_launch_dependents();
+        pdl_wait();                                  // activations, residual and outputs belong to the predecessors until here
+    }
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int kbi = 0;
+            for (int t = pair; t < total && !*abort_flag; t += pairs) {
+                const int m0 = (t % m_pairs) * 2 * TC_BM + (int)rank * TC_BM, n0 = (t / m_pairs) * BN + (int)rank * BNH;
+                for (int kb = 0; kb < nkb; ++kb, ++kbi) {
+                    const int s = kbi % STAGES;
+                    if (kbi >= STAGES) mbar_wait(smem_u32(&bar_empty[s]), ((kbi / STAGES) - 1) & 1, abort_flag, err_word, 1);
+                    if (*abort_flag) break;
+                    const uint32_t a_dst = tiles + s * Cfg::STAGE_BYTES, w_dst = a_dst + A_BYTES;
+                    const uint32_t bar = pair_map(smem_u32(&bar_full[s]), 0);
+                    if (kbi >= pre) {
+                        if (leader) mbar_expect_tx(smem_u32(&bar_full[s]), 2 * Cfg::STAGE_BYTES);
+                        tma_load_2d_pair(w_dst, &tmW, kb * TC_BK, n0, bar);
+                    }
+                    tma_load_2d_pair(a_dst, &tmA, kb * TC_BK, m0, bar);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && leader) {
+            constexpr uint32_t idesc = umma_idesc_bf16(2 * TC_BM, BN);
+            int kbi = 0, i = 0;
+            for (int t = pair; t < total && !*abort_flag; t += pairs, ++i) {
+                const int ab = i & 1;
+                if (i >= 2) mbar_wait(smem_u32(&bar_acc_empty[ab]), ((i >> 1) - 1) & 1, abort_flag, err_word, 4);
+                tc_fence_after();
+                const uint32_t acc = tmem_d + ab * BN;
+                for (int kb = 0; kb < nkb; ++kb, ++kbi) {
+                    const int s = kbi % STAGES;
+                    mbar_wait(smem_u32(&bar_full[s]), (kbi / STAGES) & 1, abort_flag, err_word, 2);
+                    if (*abort_flag) break;
+                    tc_fence_after();
+                    const uint32_t a_src = tiles + s * Cfg::STAGE_BYTES, w_src = a_src + A_BYTES;
+                    const uint64_t ad = umma_desc_k_sw128(a_src), wd = umma_desc_k_sw128(w_src);
+#pragma unroll
+                    for (int k4 = 0; k4 < TC_BK / 16; ++k4)
+                        umma_bf16_pair(acc, ad + (uint64_t)(k4 * 2), wd + (uint64_t)(k4 * 2), idesc, (kb | k4) ? 1u : 0u);
+                    umma_commit_pair(smem_u32(&bar_empty[s]));       // both CTAs may refill the stage
+                }
+                umma_commit_pair(smem_u32(&bar_acc_full[ab]));       // both CTAs' halves of the accumulator are complete
+            }
+        }
+    } else {
+        const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
+        int i = 0;
+        for (int t = pair; t < total; t += pairs, ++i) {
+            const int ab = i & 1;
+            const int m0 = (t % m_pairs) * 2 * TC_BM + (int)rank * TC_BM, n_tile = t / m_pairs;
+            tc_epilogue_tile<EPI, BN>(g, R, m0, n_tile, q, half, lane, tmem_d + ab * BN, stg, smem_u32(&bar_acc_full[ab]),
+                                      (i >> 1) & 1, abort_flag, err_word, i > 0);
+            if (lane == 0) mbar_arrive_cluster(pair_map(smem_u32(&bar_acc_empty[ab]), 0));
+        }
+    }
+    tc_fence_before();
+    pair_sync();                                     // nobody reads the other's memory or barriers past this point
+    if (warp == 1) tmem_dealloc_pair(tmem_d, Cfg::TMEM_COLS);
+}
+
+// ------------------------------------------------------------------ host side
+template <int EPI, int BN>
+inline cudaError_t tc_pair_set_smem() {
+    return cudaFuncSetAttribute(k_gemm_tc_pair<EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                TcPairCfg<BN, EPI != EPI_STATS>::SMEM);
+}
+inline cudaError_t tc_pair_init() {
+    cudaError_t e = tc_pair_set_smem<EPI_QKV, 256>();
+    if (e == cudaSuccess) e = tc_pair_set_smem<EPI_RELU, 256>();
+    if (e == cudaSuccess) e = tc_pair_set_smem<EPI_STORE, 256>();
+    if (e == cudaSuccess) e = tc_pair_set_smem<EPI_STATS, 256>();
+    return e;
+}
+
+// Worth it for wide weight matrices over many rows: the weight half of the ingest is what the pair saves.
+inline bool tc_pair_wanted(int epi, int N, int K, int rows_ub) {
+    if (epi != EPI_QKV && epi != EPI_RELU && epi != EPI_STORE && epi != EPI_STATS) return false;
+    return rows_ub >= 4 * 2 * TC_BM && N >= 1024 && N % 128 == 0 && K % TC_BK == 0;
+}
+
+template <int EPI, int BN>
+inline int tc_pair_launch_one(TmaEncoder& enc, GemmArgs<bf16>& g, int rows_ub, cudaStream_t st) {
+    const CUtensorMap* ta = enc.get(g.A, rows_ub, g.K, g.lda, TC_BM);
+    const CUtensorMap* tw = enc.get(g.W, g.N, g.K, g.K, BN / 2);
+    if (!ta || !tw) return -1;
+    const long long tiles_ub = (long long)((g.N + BN - 1) / BN) * ((rows_ub + 2 * TC_BM - 1) / (2 * TC_BM));
+    const int grid = 2 * (int)std::min<long long>(tiles_ub, enc.n_sm / 2);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(TC_THREADS);
+    cfg.dynamicSmemBytes = TcPairCfg<BN, EPI != EPI_STATS>::SMEM; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = enc.pdl ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_gemm_tc_pair<EPI, BN>, *ta, *tw, g, enc.err_word);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) { enc.err = std::string("pair launch: ") + cudaGetErrorString(e); return -1; }
+    return 0;
+}
+
+inline int gemm_tc_pair_launch(TmaEncoder& enc, int epi, GemmArgs<bf16>& g, int rows_ub, cudaStream_t st, int* n_tiles_out) {
+    if (!enc.ready) return -1;
+    g.one_m_tile = 0;
+    switch (epi) {
+        case EPI_QKV: return tc_pair_launch_one<EPI_QKV, 256>(enc, g, rows_ub, st);
+        case EPI_RELU: return tc_pair_launch_one<EPI_RELU, 256>(enc, g, rows_ub, st);
+        case EPI_STORE: return tc_pair_launch_one<EPI_STORE, 256>(enc, g, rows_ub, st);
+        case EPI_STATS:
+            g.n_tiles = 2 * ((g.N + 255) / 256);
+            if (n_tiles_out) *n_tiles_out = g.n_tiles;
+            return tc_pair_launch_one<EPI_STATS, 256>(enc, g, rows_ub, st);
+        default: return -2;
+    }
+}
+
+}  // namespace sd

@@ -18,6 +18,7 @@
 #include "attention_tc.cuh"
 #include "decoder_cluster.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_tc_pair.cuh"
 #include "kernels.cuh"
 #include "skinny_gemm.cuh"
 
@@ -96,6 +97,8 @@ struct specdec_handle {
     int poll_lag = -1;              // -1: chosen by batch size
     int use_fused_attn = 0;         // attention + output projection as one cluster kernel (measured slower: off)
     size_t attn_proj_smem_cap = 0;
+    bool pair_ready = false;
+    int use_pair = 0;               // two-SM tiles (cta_group::2) for wide GEMMs over many rows (option "pair")
     int attn_warps = 0;             // 0 = choose per launch, else 4 or 8 warps per tile-attention CTA (option "attn_warps")
     int skinny_groups = 1;          // 8-row weight groups per CTA of the weight-streaming GEMM (1, 2 or 4)
     // CUDA graphs of whole draft / verify(+commit) steps, keyed by everything their launches depend on
@@ -438,7 +441,9 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
     }
     if constexpr (std::is_same<T, bf16>::value) {
         if (h->use_tc && sd::tc_supported(N, K) && (epi != EPI_STATS || N >= 128)) {
-            int rc = sd::gemm_tc_launch(h->tma, epi, g, rows_ub, st, n_tiles_out);
+            int rc = (h->use_pair && sd::tc_pair_wanted(epi, N, K, rows_ub))
+                         ? sd::gemm_tc_pair_launch(h->tma, epi, g, rows_ub, st, n_tiles_out)
+                         : sd::gemm_tc_launch(h->tma, epi, g, rows_ub, st, n_tiles_out);
             if (rc != 0) return fail(h, SPECDEC_ERR_CUDA, "tensor-core GEMM launch failed: " + h->tma.err);
             ++h->launches;
             return 0;
@@ -854,7 +859,7 @@ void drop_graphs(specdec_handle* h) {
 // replayed afterwards.  The key must name everything the launches depend on besides device memory.
 template <typename F>
 int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body) {
-    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->attn_warps); key.push_back(h->use_fused_attn); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
+    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->use_pair); key.push_back(h->attn_warps); key.push_back(h->use_fused_attn); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
     key.push_back(h->B); key.push_back(h->S_max);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
@@ -1136,6 +1141,8 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
             h->attn_proj_smem_cap = cap;
         }
         if (sd::tc_init(h->tma, h->ses.counters + 7) != 0) h->use_tc = 0;     // reported through specdec_last_error; SIMT GEMM still runs on the GPU
+        h->pair_ready = h->use_tc && sd::tc_pair_init() == cudaSuccess;
+        if (!h->pair_ready) cudaGetLastError();
         if (!h->use_tc) h->err = "tensor-core GEMM unavailable: " + h->tma.err;
     } else {
         h->use_tc = 0;
@@ -1178,6 +1185,10 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
     if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "pair")) {
+        if (value && !h->pair_ready) return fail(h, SPECDEC_ERR_UNSUPPORTED, "two-SM GEMM tiles are not available on this handle");
+        h->use_pair = value ? 1 : 0; return SPECDEC_OK;
+    }
     if (!strcmp(name, "attn_warps")) {
         if (value != 0 && value != 4 && value != 8) return fail(h, SPECDEC_ERR_INVALID_ARG, "attn_warps must be 0, 4 or 8");
         h->attn_warps = value; return SPECDEC_OK;
