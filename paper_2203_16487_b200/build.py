@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 SRC = os.path.join(HERE, "csrc", "specdec.cu")
 LIB = os.path.join(HERE, "libspecdec_b200.so")
-DEPS = [SRC] + [os.path.join(HERE, "csrc", f) for f in ("kernels.cuh", "gemm_tc.cuh", "attention_tc.cuh", "skinny_gemm.cuh", "decoder_cluster.cuh", "attention_oproj.cuh")] + \
+DEPS = [SRC] + sorted(os.path.join(HERE, "csrc", f) for f in os.listdir(os.path.join(HERE, "csrc")) if f.endswith(".cuh")) + \
        [os.path.join(os.path.dirname(HERE), "include", "specdec.h")]
 
 

@@ -431,6 +431,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     mbar_wait(smem_u32(&bar_full[s]), (kbi / STAGES) & 1, abort_flag, err_word, 2);
                     if (*abort_flag) break;
                     if (kbi == 0) tc_stamp(g.trace, 4);
+                    if (kbi < 16) tc_stamp(g.trace, 40 + kbi);          // landing cadence of the first k-blocks
                     tc_fence_after();
                     const uint32_t a_src = tiles + s * Cfg::STAGE_BYTES, w_src = a_src + A_BYTES;
                     const uint64_t ad = umma_desc_k_sw128(a_src), wd = umma_desc_k_sw128(w_src);

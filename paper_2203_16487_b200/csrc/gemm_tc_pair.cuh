@@ -83,6 +83,7 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     using Cfg = TcPairCfg<BN, EPI != EPI_STATS>;
     constexpr int STAGES = Cfg::STAGES, BNH = Cfg::BNH;
     constexpr int A_BYTES = TC_BM * TC_BK * 2;
+    if (threadIdx.x == 0) tc_stamp(g.trace, 0);
     const bool early = g.rows_static >= 0;
     if (!early) pdl_wait();
     const int R = early ? g.rows_static : *g.n_rows;
@@ -115,6 +116,7 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem_d = tmem_base_s;
     volatile int* abort_flag = &abort_s;
+    if (threadIdx.x == 0 && tmem_d != 0xffffffffu) tc_stamp(g.trace, 1);
     int pre = 0;                                     // stages whose weight halves were requested before the wait
     if (early) {
         if (threadIdx.x == 0) {
@@ -144,8 +146,10 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         tma_load_2d_pair(w_dst, &tmW, kb * TC_BK, n0, bar);
                     }
                     tma_load_2d_pair(a_dst, &tmA, kb * TC_BK, m0, bar);
+                    if (kbi == 0) tc_stamp(g.trace, 2);
                 }
             }
+            tc_stamp(g.trace, 3);
         }
     } else if (warp == 1) {
         if (lane == 0 && leader) {
@@ -160,6 +164,7 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const int s = kbi % STAGES;
                     mbar_wait(smem_u32(&bar_full[s]), (kbi / STAGES) & 1, abort_flag, err_word, 2);
                     if (*abort_flag) break;
+                    if (kbi == 0) tc_stamp(g.trace, 4);
                     tc_fence_after();
                     const uint32_t a_src = tiles + s * Cfg::STAGE_BYTES, w_src = a_src + A_BYTES;
                     const uint64_t ad = umma_desc_k_sw128(a_src), wd = umma_desc_k_sw128(w_src);
@@ -169,6 +174,7 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     umma_commit_pair(smem_u32(&bar_empty[s]));       // both CTAs may refill the stage
                 }
                 umma_commit_pair(smem_u32(&bar_acc_full[ab]));       // both CTAs' halves of the accumulator are complete
+                tc_stamp(g.trace, 5 + (i > 0));
             }
         }
     } else {
@@ -181,11 +187,13 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             tc_epilogue_tile<EPI, BN>(g, R, m0, n_tile, q, half, lane, tmem_d + ab * BN, stg, smem_u32(&bar_acc_full[ab]),
                                       (i >> 1) & 1, abort_flag, err_word, i > 0);
             if (lane == 0) mbar_arrive_cluster(pair_map(smem_u32(&bar_acc_empty[ab]), 0));
+            if (threadIdx.x == 64) tc_stamp(g.trace, 8 + 2 * (i > 0));
         }
     }
     tc_fence_before();
     pair_sync();                                     // nobody reads the other's memory or barriers past this point
     if (warp == 1) tmem_dealloc_pair(tmem_d, Cfg::TMEM_COLS);
+    if (threadIdx.x == 0) tc_stamp(g.trace, 11);
 }
 
 // ------------------------------------------------------------------ host side

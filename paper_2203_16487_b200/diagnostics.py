@@ -61,6 +61,8 @@ def vocab_trace(reps=20, opts=(), batch=1):
         sd.verify(drafts, 3, 1.0)
     torch.cuda.synchronize()
     t = np.array(sd.cluster_trace(256), dtype=np.int64)[200:214]
+    tt = np.array(sd.cluster_trace(256), dtype=np.int64)
+    print("k-block landings (us since entry):", [round((x - t[0]) / 1e3, 2) for x in tt[240:256]])
     t = np.concatenate([t[:1], t[12:14], t[1:12]])
     names = ["kernel entry", "mbarriers initialised", "TMEM allocated", "barriers + TMEM ready", "first TMA issued", "all TMA issued", "first stage landed",
              "tile 0 MMAs committed", "last tile MMAs committed", "epilogue tile 0 start", "epilogue tile 0 end",
