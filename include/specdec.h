@@ -202,7 +202,12 @@ int specdec_set_draft_script(specdec_handle* h, const int32_t* d_script, int B, 
 int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches);
 
 /* Options: "gemm" = 0 SIMT reference GEMM, 1 tcgen05 GEMM (bf16 handles; default 1);
- * "skinny" = 0/1 weight-streaming GEMM with fused LayerNorm for passes of at most 64 rows (bf16; default 1);
+ * "skinny" = 0/1 weight-streaming GEMM with fused LayerNorm for passes of at most 32 rows (bf16; default 1);
+ * "pair" = 0/1 two-SM tensor-core tiles (256 rows x 256 columns per CTA pair) for GEMMs with at least 1024 rows
+ *   and 1024 columns (default 0: same results bit for bit, measured no faster than single-SM tiles at these
+ *   sizes, kept for comparison);
+ * "attn_warps" = 0 choose per launch, 4 or 8 warps per CTA of the tile attention (default 0);
+ * "tc_bn" = 0 choose, else force the column width of the tensor-core GEMM tiles (64 / 128 / 256; experiments);
  * "cluster" = 0/1 run the verifier's decoder stack as one thread-block-cluster kernel per sequence when the
  *   batch is at most 8, k + 1 <= 32 and the model has 8 heads of 64 (default 0: measured slower than the
  *   per-operation kernels, kept for comparison);
