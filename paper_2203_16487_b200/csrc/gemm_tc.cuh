@@ -46,8 +46,8 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait: gives up after ~2e8 clocks, raises the CTA-wide abort flag and the global error word.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err_word,
                                           int code) {
+    if (mbar_try_wait(bar, parity)) return true;      // fast path: no other shared-memory access
     if (*abort_flag) return false;
-    if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -426,20 +426,27 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 if (i >= 2) mbar_wait(smem_u32(&bar_acc_empty[ab]), ((i >> 1) - 1) & 1, abort_flag, err_word, 4);
                 tc_fence_after();
                 const uint32_t acc = tmem_d + ab * BN;
-                for (int kb = 0; kb < nkb; ++kb, ++kbi) {
+                // The tensor pipe accepts one MMA at a time from this thread, so whatever the thread does between
+                // two k-blocks is time the pipe idles: the barrier of the NEXT stage is tested before the MMAs of
+                // this one are issued (its latency hides behind them), and the loop carries nothing else.
+                bool ok = mbar_wait(smem_u32(&bar_full[kbi % STAGES]), (kbi / STAGES) & 1, abort_flag, err_word, 2);
+                if (kbi == 0) tc_stamp(g.trace, 4);
+                for (int kb = 0; kb < nkb && ok; ++kb, ++kbi) {
                     const int s = kbi % STAGES;
-                    mbar_wait(smem_u32(&bar_full[s]), (kbi / STAGES) & 1, abort_flag, err_word, 2);
-                    if (*abort_flag) break;
-                    if (kbi == 0) tc_stamp(g.trace, 4);
+                    const int sn = (kbi + 1) % STAGES;
+                    const uint32_t next_bar = smem_u32(&bar_full[sn]), next_par = ((kbi + 1) / STAGES) & 1;
+                    const bool more = kb + 1 < nkb;
+                    const uint32_t early_ok = more ? mbar_try_wait(next_bar, next_par) : 1u;
                     if (kbi < 16) tc_stamp(g.trace, 40 + kbi);          // landing cadence of the first k-blocks
-                    tc_fence_after();
                     const uint32_t a_src = tiles + s * Cfg::STAGE_BYTES, w_src = a_src + A_BYTES;
                     const uint64_t ad = umma_desc_k_sw128(a_src), wd = umma_desc_k_sw128(w_src);
 #pragma unroll
                     for (int k4 = 0; k4 < TC_BK / 16; ++k4)      // +32 bytes along K per instruction: 2 address units
                         umma_bf16(acc, ad + (uint64_t)(k4 * 2), wd + (uint64_t)(k4 * 2), idesc, (kb | k4) ? 1u : 0u);
                     umma_commit(smem_u32(&bar_empty[s]));        // stage reusable once these MMAs have read it
+                    if (!early_ok) ok = mbar_wait(next_bar, next_par, abort_flag, err_word, 2);
                 }
+                if (!ok) break;
                 umma_commit(smem_u32(&bar_acc_full[ab]));        // accumulator of this tile complete
                 tc_stamp(g.trace, 5 + (i > 0));
             }

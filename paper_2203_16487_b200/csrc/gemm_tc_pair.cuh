@@ -196,6 +196,150 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (threadIdx.x == 0) tc_stamp(g.trace, 11);
 }
 
+// Vocabulary projection + row statistics on two-SM tiles with the activation rows RESIDENT in shared memory:
+// a pair of CTAs takes a contiguous run of (row pair, column tile) tiles, column tile fastest, so its 2 x 128
+// activation rows (K <= 512: at most 128 KB per CTA) are loaded once per row pair and only the weight halves
+// (128 rows x 64 per k-block and CTA) stream through the ring.  Per k-block a CTA then ingests 16 KB instead of
+// 32 KB (two-SM tile with streamed activations) or 48 KB (single-SM 128 x 256 tile).
+constexpr int VP_BN = 256, VP_BNH = 128, VP_MAX_STAGES = 8;
+constexpr int VP_KB_BYTES = TC_BM * TC_BK * 2;                    // 16 KB: one k-block of 128 rows, activations or weights
+inline int vp_stages(int K) {
+    const int fit = (232448 - 1024 - (K / TC_BK) * VP_KB_BYTES) / VP_KB_BYTES;
+    return fit > VP_MAX_STAGES ? VP_MAX_STAGES : fit;
+}
+inline size_t vp_smem(int K) { return (size_t)(K / TC_BK + vp_stages(K)) * VP_KB_BYTES + 1024; }
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
+k_vocab_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, GemmArgs<bf16> g,
+             int* err_word, int stages) {
+    if (threadIdx.x == 0) tc_stamp(g.trace, 0);
+    const bool early = g.rows_static >= 0;
+    if (!early) pdl_wait();
+    const int R = early ? g.rows_static : *g.n_rows;
+    const int m_pairs = (R + 2 * TC_BM - 1) / (2 * TC_BM), n_tiles = (g.N + VP_BN - 1) / VP_BN;
+    const int total = m_pairs * n_tiles;
+    const int pair = (int)blockIdx.x >> 1, pairs = (int)gridDim.x >> 1;
+    const int per = (total + pairs - 1) / pairs;     // contiguous run of tiles per pair, column tile fastest
+    const int t_begin = pair * per, t_end = min(total, t_begin + per);
+    if (t_begin >= t_end) return;                    // both CTAs of the pair leave together, before any cluster barrier
+
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_w_full[VP_MAX_STAGES], bar_w_empty[VP_MAX_STAGES], bar_a_full, bar_a_empty,
+        bar_acc_full[2], bar_acc_empty[2];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = pair_cta_rank();
+    const bool leader = rank == 0;
+    const int nkb = g.K / TC_BK;
+    const uint32_t a_base = (smem_u32(smem_raw) + 1023u) & ~1023u, w_base = a_base + nkb * VP_KB_BYTES;
+
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        for (int s = 0; s < VP_MAX_STAGES; ++s) { mbar_init(smem_u32(&bar_w_full[s]), 1); mbar_init(smem_u32(&bar_w_empty[s]), 1); }
+        mbar_init(smem_u32(&bar_a_full), 1); mbar_init(smem_u32(&bar_a_empty), 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bar_acc_full[i]), 1); mbar_init(smem_u32(&bar_acc_empty[i]), 2 * TC_EPI_WARPS); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc_pair(smem_u32(&tmem_base_s), 512);
+    tc_fence_before();
+    pair_sync();
+    tc_fence_after();
+    const uint32_t tmem_d = tmem_base_s;
+    volatile int* abort_flag = &abort_s;
+    if (threadIdx.x == 0 && tmem_d != 0xffffffffu) tc_stamp(g.trace, 1);
+    int pre = 0;                                     // ring stages requested before the wait (weights only)
+    if (early) {
+        if (threadIdx.x == 0) {
+            const int n0 = (t_begin % n_tiles) * VP_BN + (int)rank * VP_BNH;
+            for (; pre < stages && pre < nkb; ++pre) {
+                if (leader) mbar_expect_tx(smem_u32(&bar_w_full[pre]), 2 * VP_KB_BYTES);
+                tma_load_2d_pair(w_base + pre * VP_KB_BYTES, &tmW, pre * TC_BK, n0, pair_map(smem_u32(&bar_w_full[pre]), 0));
+            }
+        }
+        pdl_launch_dependents();
+        pdl_wait();
+    }
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int kbi = 0, a_loads = 0, cur_m = -1;
+            for (int t = t_begin; t < t_end && !*abort_flag; ++t) {
+                const int m_pair = t / n_tiles, n0 = (t % n_tiles) * VP_BN + (int)rank * VP_BNH;
+                if (m_pair != cur_m) {               // new row pair: replace the resident activation rows
+                    if (a_loads > 0) mbar_wait(smem_u32(&bar_a_empty), (a_loads - 1) & 1, abort_flag, err_word, 5);
+                    if (*abort_flag) break;
+                    if (leader) mbar_expect_tx(smem_u32(&bar_a_full), 2 * nkb * VP_KB_BYTES);
+                    const uint32_t abar = pair_map(smem_u32(&bar_a_full), 0);
+                    for (int kb = 0; kb < nkb; ++kb)
+                        tma_load_2d_pair(a_base + kb * VP_KB_BYTES, &tmA, kb * TC_BK, m_pair * 2 * TC_BM + (int)rank * TC_BM, abar);
+                    cur_m = m_pair; ++a_loads;
+                    if (a_loads == 1) tc_stamp(g.trace, 2);
+                }
+                for (int kb = 0; kb < nkb; ++kb, ++kbi) {
+                    const int s = kbi % stages;
+                    if (kbi >= stages) mbar_wait(smem_u32(&bar_w_empty[s]), ((kbi / stages) - 1) & 1, abort_flag, err_word, 1);
+                    if (*abort_flag) break;
+                    if (kbi >= pre) {
+                        if (leader) mbar_expect_tx(smem_u32(&bar_w_full[s]), 2 * VP_KB_BYTES);
+                        tma_load_2d_pair(w_base + s * VP_KB_BYTES, &tmW, kb * TC_BK, n0, pair_map(smem_u32(&bar_w_full[s]), 0));
+                    }
+                }
+            }
+            tc_stamp(g.trace, 3);
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && leader) {
+            constexpr uint32_t idesc = umma_idesc_bf16(2 * TC_BM, VP_BN);
+            int kbi = 0, i = 0, a_uses = 0, cur_m = -1;
+            for (int t = t_begin; t < t_end && !*abort_flag; ++t, ++i) {
+                const int ab = i & 1, m_pair = t / n_tiles;
+                if (i >= 2) mbar_wait(smem_u32(&bar_acc_empty[ab]), ((i >> 1) - 1) & 1, abort_flag, err_word, 4);
+                if (m_pair != cur_m) {
+                    mbar_wait(smem_u32(&bar_a_full), a_uses & 1, abort_flag, err_word, 6);
+                    cur_m = m_pair; ++a_uses;
+                }
+                if (*abort_flag) break;
+                tc_fence_after();
+                const uint32_t acc = tmem_d + ab * VP_BN;
+                for (int kb = 0; kb < nkb; ++kb, ++kbi) {
+                    const int s = kbi % stages;
+                    mbar_wait(smem_u32(&bar_w_full[s]), (kbi / stages) & 1, abort_flag, err_word, 2);
+                    if (*abort_flag) break;
+                    if (kbi == 0) tc_stamp(g.trace, 4);
+                    if (kbi < 16) tc_stamp(g.trace, 40 + kbi);
+                    tc_fence_after();
+                    const uint64_t ad = umma_desc_k_sw128(a_base + kb * VP_KB_BYTES), wd = umma_desc_k_sw128(w_base + s * VP_KB_BYTES);
+#pragma unroll
+                    for (int k4 = 0; k4 < TC_BK / 16; ++k4)
+                        umma_bf16_pair(acc, ad + (uint64_t)(k4 * 2), wd + (uint64_t)(k4 * 2), idesc, (kb | k4) ? 1u : 0u);
+                    umma_commit_pair(smem_u32(&bar_w_empty[s]));
+                }
+                if (t + 1 == t_end || (t + 1) / n_tiles != m_pair) umma_commit_pair(smem_u32(&bar_a_empty));   // rows may be replaced
+                umma_commit_pair(smem_u32(&bar_acc_full[ab]));
+                tc_stamp(g.trace, 5 + (i > 0));
+            }
+        }
+    } else {
+        const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
+        int i = 0;
+        for (int t = t_begin; t < t_end; ++t, ++i) {
+            const int ab = i & 1;
+            const int m0 = (t / n_tiles) * 2 * TC_BM + (int)rank * TC_BM, n_tile = t % n_tiles;
+            tc_epilogue_tile<EPI_STATS, VP_BN>(g, R, m0, n_tile, q, half, lane, tmem_d + ab * VP_BN, nullptr,
+                                               smem_u32(&bar_acc_full[ab]), (i >> 1) & 1, abort_flag, err_word, i > 0);
+            if (lane == 0) mbar_arrive_cluster(pair_map(smem_u32(&bar_acc_empty[ab]), 0));
+            if (threadIdx.x == 64) tc_stamp(g.trace, 8 + 2 * (i > 0));
+        }
+    }
+    tc_fence_before();
+    pair_sync();
+    if (warp == 1) tmem_dealloc_pair(tmem_d, 512);
+    if (threadIdx.x == 0) tc_stamp(g.trace, 11);
+}
+
 // ------------------------------------------------------------------ host side
 template <int EPI, int BN>
 inline cudaError_t tc_pair_set_smem() {
@@ -207,6 +351,7 @@ inline cudaError_t tc_pair_init() {
     if (e == cudaSuccess) e = tc_pair_set_smem<EPI_RELU, 256>();
     if (e == cudaSuccess) e = tc_pair_set_smem<EPI_STORE, 256>();
     if (e == cudaSuccess) e = tc_pair_set_smem<EPI_STATS, 256>();
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_vocab_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);
     return e;
 }
 
@@ -236,6 +381,24 @@ inline int tc_pair_launch_one(TmaEncoder& enc, GemmArgs<bf16>& g, int rows_ub, c
     return 0;
 }
 
+inline int vocab_pair_launch(TmaEncoder& enc, GemmArgs<bf16>& g, int rows_ub, cudaStream_t st) {
+    const CUtensorMap* ta = enc.get(g.A, rows_ub, g.K, g.lda, TC_BM);
+    const CUtensorMap* tw = enc.get(g.W, g.N, g.K, g.K, VP_BNH);
+    if (!ta || !tw) return -1;
+    const long long tiles_ub = (long long)((g.N + VP_BN - 1) / VP_BN) * ((rows_ub + 2 * TC_BM - 1) / (2 * TC_BM));
+    const int grid = 2 * (int)std::min<long long>(tiles_ub, enc.n_sm / 2);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = vp_smem(g.K); cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = enc.pdl ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_vocab_pair, *ta, *tw, g, enc.err_word, vp_stages(g.K));
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) { enc.err = std::string("vocabulary pair launch: ") + cudaGetErrorString(e); return -1; }
+    return 0;
+}
+
 inline int gemm_tc_pair_launch(TmaEncoder& enc, int epi, GemmArgs<bf16>& g, int rows_ub, cudaStream_t st, int* n_tiles_out) {
     if (!enc.ready) return -1;
     g.one_m_tile = 0;
@@ -246,6 +409,7 @@ inline int gemm_tc_pair_launch(TmaEncoder& enc, int epi, GemmArgs<bf16>& g, int 
         case EPI_STATS:
             g.n_tiles = 2 * ((g.N + 255) / 256);
             if (n_tiles_out) *n_tiles_out = g.n_tiles;
+            if (g.K <= 512 && vp_stages(g.K) >= 4) return vocab_pair_launch(enc, g, rows_ub, st);
             return tc_pair_launch_one<EPI_STATS, 256>(enc, g, rows_ub, st);
         default: return -2;
     }
