@@ -160,19 +160,21 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (i >= 2) mbar_wait(smem_u32(&bar_acc_empty[ab]), ((i >> 1) - 1) & 1, abort_flag, err_word, 4);
                 tc_fence_after();
                 const uint32_t acc = tmem_d + ab * BN;
-                for (int kb = 0; kb < nkb; ++kb, ++kbi) {
-                    const int s = kbi % STAGES;
-                    mbar_wait(smem_u32(&bar_full[s]), (kbi / STAGES) & 1, abort_flag, err_word, 2);
-                    if (*abort_flag) break;
-                    if (kbi == 0) tc_stamp(g.trace, 4);
-                    tc_fence_after();
+                bool ok = mbar_wait(smem_u32(&bar_full[kbi % STAGES]), (kbi / STAGES) & 1, abort_flag, err_word, 2);
+                if (kbi == 0) tc_stamp(g.trace, 4);
+                for (int kb = 0; kb < nkb && ok; ++kb, ++kbi) {   // next stage's barrier is tested before this stage's MMAs
+                    const int s = kbi % STAGES, sn = (kbi + 1) % STAGES;
+                    const uint32_t next_bar = smem_u32(&bar_full[sn]), next_par = ((kbi + 1) / STAGES) & 1;
+                    const uint32_t early_ok = (kb + 1 < nkb) ? mbar_try_wait(next_bar, next_par) : 1u;
                     const uint32_t a_src = tiles + s * Cfg::STAGE_BYTES, w_src = a_src + A_BYTES;
                     const uint64_t ad = umma_desc_k_sw128(a_src), wd = umma_desc_k_sw128(w_src);
 #pragma unroll
                     for (int k4 = 0; k4 < TC_BK / 16; ++k4)
                         umma_bf16_pair(acc, ad + (uint64_t)(k4 * 2), wd + (uint64_t)(k4 * 2), idesc, (kb | k4) ? 1u : 0u);
                     umma_commit_pair(smem_u32(&bar_empty[s]));       // both CTAs may refill the stage
+                    if (!early_ok) ok = mbar_wait(next_bar, next_par, abort_flag, err_word, 2);
                 }
+                if (!ok) break;
                 umma_commit_pair(smem_u32(&bar_acc_full[ab]));       // both CTAs' halves of the accumulator are complete
                 tc_stamp(g.trace, 5 + (i > 0));
             }
@@ -303,19 +305,21 @@ k_vocab_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 if (*abort_flag) break;
                 tc_fence_after();
                 const uint32_t acc = tmem_d + ab * VP_BN;
-                for (int kb = 0; kb < nkb; ++kb, ++kbi) {
-                    const int s = kbi % stages;
-                    mbar_wait(smem_u32(&bar_w_full[s]), (kbi / stages) & 1, abort_flag, err_word, 2);
-                    if (*abort_flag) break;
-                    if (kbi == 0) tc_stamp(g.trace, 4);
+                bool ok = mbar_wait(smem_u32(&bar_w_full[kbi % stages]), (kbi / stages) & 1, abort_flag, err_word, 2);
+                if (kbi == 0) tc_stamp(g.trace, 4);
+                for (int kb = 0; kb < nkb && ok; ++kb, ++kbi) {   // next stage's barrier is tested before this stage's MMAs
+                    const int s = kbi % stages, sn = (kbi + 1) % stages;
+                    const uint32_t next_bar = smem_u32(&bar_w_full[sn]), next_par = ((kbi + 1) / stages) & 1;
+                    const uint32_t early_ok = (kb + 1 < nkb) ? mbar_try_wait(next_bar, next_par) : 1u;
                     if (kbi < 16) tc_stamp(g.trace, 40 + kbi);
-                    tc_fence_after();
                     const uint64_t ad = umma_desc_k_sw128(a_base + kb * VP_KB_BYTES), wd = umma_desc_k_sw128(w_base + s * VP_KB_BYTES);
 #pragma unroll
                     for (int k4 = 0; k4 < TC_BK / 16; ++k4)
                         umma_bf16_pair(acc, ad + (uint64_t)(k4 * 2), wd + (uint64_t)(k4 * 2), idesc, (kb | k4) ? 1u : 0u);
                     umma_commit_pair(smem_u32(&bar_w_empty[s]));
+                    if (!early_ok) ok = mbar_wait(next_bar, next_par, abort_flag, err_word, 2);
                 }
+                if (!ok) break;
                 if (t + 1 == t_end || (t + 1) / n_tiles != m_pair) umma_commit_pair(smem_u32(&bar_a_empty));   // rows may be replaced
                 umma_commit_pair(smem_u32(&bar_acc_full[ab]));
                 tc_stamp(g.trace, 5 + (i > 0));
