@@ -517,6 +517,7 @@ inline cudaError_t tc_set_smem_all() {
     cudaError_t e = tc_set_smem<EPI, 32>();
     if (e == cudaSuccess) e = tc_set_smem<EPI, 64>();
     if (e == cudaSuccess) e = tc_set_smem<EPI, 128>();
+    if (e == cudaSuccess) e = tc_set_smem<EPI, 192>();
     if (e == cudaSuccess) e = tc_set_smem<EPI, 256>();
     return e;
 }
@@ -573,6 +574,7 @@ template <int EPI>
 inline int tc_launch_bn(TmaEncoder& enc, int bn, GemmArgs<bf16>& g, int rows_ub, cudaStream_t st) {
     switch (bn) {
         case 256: return tc_launch_one<EPI, 256>(enc, g, rows_ub, st);
+        case 192: return tc_launch_one<EPI, 192>(enc, g, rows_ub, st);
         case 128: return tc_launch_one<EPI, 128>(enc, g, rows_ub, st);
         case 64: return tc_launch_one<EPI, 64>(enc, g, rows_ub, st);
         default: return tc_launch_one<EPI, 32>(enc, g, rows_ub, st);
@@ -587,9 +589,9 @@ inline int tc_launch_bn(TmaEncoder& enc, int bn, GemmArgs<bf16>& g, int rows_ub,
 inline int tc_pick_bn(int N, int rows_ub, int n_sm) {
     const int m_tiles = (rows_ub + TC_BM - 1) / TC_BM;
     if (N < 64) return 32;
-    const int cand[3] = {256, 128, 64};
+    const int cand[4] = {256, 192, 128, 64};
     int best = 64; long long best_cost = -1;
-    for (int i = 0; i < 3; ++i) {
+    for (int i = 0; i < 4; ++i) {
         const int bn = cand[i];
         if (bn > N && bn != 64) continue;
         const long long tiles = (long long)((N + bn - 1) / bn) * m_tiles;
@@ -619,7 +621,7 @@ inline int gemm_tc_launch(TmaEncoder& enc, int epi, GemmArgs<bf16>& g, int rows_
         return bn == 256 ? tc_launch_one<EPI_STATS, 256>(enc, g, rows_ub, st) : tc_launch_one<EPI_STATS, 128>(enc, g, rows_ub, st);
     }
     const int fb = enc.force_bn;
-    const bool forced = (fb == 32 || fb == 64 || fb == 128 || fb == 256) && fb <= g.N;
+    const bool forced = (fb == 32 || fb == 64 || fb == 128 || fb == 192 || fb == 256) && fb <= g.N;
     const int bn = forced ? fb : tc_pick_bn(g.N, rows_ub, enc.n_sm);
     switch (epi) {
         case EPI_STORE: return tc_launch_bn<EPI_STORE>(enc, bn, g, rows_ub, st);
