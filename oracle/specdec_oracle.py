@@ -16,20 +16,25 @@ computes in np.float32 by default; pass dtype=np.float64 to measure its own
 rounding noise.  `mode="bf16"` additionally rounds values to bf16 at the points
 where the CUDA path feeds bf16 operands to its tensor-core contractions
 (normalised activations, Q/K/V, un-normalised attention probabilities,
-attention output, ReLU output, encoder memory); accumulation stays in `dtype`.
+attention output, feed-forward activation output, encoder memory); accumulation
+stays in `dtype`.
 
 The paper gives only layer counts and 512/2048 widths (Section 4.1).  The rest
 of the architecture is a stated reading: pre-LN blocks, ReLU, eps 1e-5,
 sqrt(d)-scaled shared embeddings plus a position table, biases everywhere, tied
-output projection without bias, argmax ties to the lowest id.
+output projection without bias, argmax ties to the lowest id.  `act="gelu"`
+switches the feed-forward activation to the exact (erf) GELU for the BART-base
+shaped pair of the summarisation experiment (Section 5.2; BART's dimensions are
+public knowledge, not the paper's: 768 wide, 12 heads, 3072 inner, 50265 ids,
+learned position tables, which here are simply the pos_enc / pos_dec weights).
 
 Pinned (tests/test_oracle_pins.py): greedy equivalence at beta=1, tau=0;
 brute-force log-prob form of Eq. 7-8 on tiny vocabularies; monotonicity in
 beta and tau; block-parallel == sequential rows; cached == from scratch; the
 worked example's iteration structure; the parameter count implied by the
 paper's memory table; a closed-form model with zeroed sublayers; the whole
-encoder / decoder stack against torch.nn's pre-LN Transformer layers in fp64;
-every weight shown to influence the output.
+encoder / decoder stack against torch.nn's pre-LN Transformer layers in fp64
+(ReLU and GELU); every weight shown to influence the output.
 Parity unpinned: nothing about translation quality (needs trained weights).
 """
 from __future__ import annotations
@@ -38,6 +43,7 @@ from dataclasses import dataclass, field
 from typing import Dict, List, Optional, Sequence, Tuple
 
 import numpy as np
+from scipy.special import erf as _erf      # library routine: the error function of the exact GELU
 
 LN_EPS = 1e-5
 
@@ -71,6 +77,7 @@ class Model:
     w: Dict[str, np.ndarray]
     dtype: type = np.float32
     mode: str = "pure"            # "pure" | "bf16"
+    act: str = "relu"             # feed-forward activation: "relu" (Transformer-base, Section 4.1) | "gelu" (BART-base, Section 5.2)
 
     def __post_init__(self):
         self.w = {k: np.asarray(v, dtype=self.dtype) for k, v in self.w.items()}
@@ -79,9 +86,9 @@ class Model:
         return bf16_round(a) if self.mode == "bf16" else a
 
 
-def model_from(dims, weights, dtype=np.float32, mode="pure") -> Model:
+def model_from(dims, weights, dtype=np.float32, mode="pure", act="relu") -> Model:
     return Model(dims.d_model, dims.n_heads, dims.d_ffn, dims.vocab,
-                 dims.enc_layers, dims.dec_layers, weights, dtype, mode)
+                 dims.enc_layers, dims.dec_layers, weights, dtype, mode, act)
 
 
 # ----------------------------------------------------------------------------
@@ -124,8 +131,14 @@ def embed(m: Model, tokens: Sequence[int], positions: Sequence[int], table: str)
     return m.w["embed"][tok] * m.dtype(np.sqrt(m.d_model)) + m.w[table][pos]
 
 
+def gelu(x: np.ndarray) -> np.ndarray:
+    """x * Phi(x) with the exact normal CDF (the erf form), in the dtype of x."""
+    return (x * (x.dtype.type(0.5) * (x.dtype.type(1) + _erf(x * x.dtype.type(1.0 / np.sqrt(2.0)))))).astype(x.dtype)
+
+
 def ffn(m: Model, y: np.ndarray, p: str) -> np.ndarray:
-    hdn = np.maximum(y @ m.w[p + ".w1"].T + m.w[p + ".b1"], 0)
+    pre = y @ m.w[p + ".w1"].T + m.w[p + ".b1"]
+    hdn = gelu(pre) if m.act == "gelu" else np.maximum(pre, 0)
     return m.r(hdn) @ m.w[p + ".w2"].T + m.w[p + ".b2"]
 
 

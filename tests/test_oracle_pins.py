@@ -42,7 +42,7 @@ def test_parameter_count_matches_memory_table():
     assert W.count_params(wd) == 63_015_936
 
 
-def _torch_stack(m: O.Model):
+def _torch_stack(m: O.Model, act="relu"):
     """The same weights loaded into torch.nn pre-LN Transformer layers (fp64)."""
     d, H, F = m.d_model, m.n_heads, m.d_ffn
     t = lambda a: torch.tensor(np.asarray(a, dtype=np.float64))
@@ -61,11 +61,11 @@ def _torch_stack(m: O.Model):
 
     enc, dec = [], []
     for l in range(m.enc_layers):
-        L = torch.nn.TransformerEncoderLayer(d, H, F, 0.0, norm_first=True, batch_first=True).double()
+        L = torch.nn.TransformerEncoderLayer(d, H, F, 0.0, activation=act, norm_first=True, batch_first=True).double()
         load_attn(L.self_attn, f"enc.{l}.self"); load_common(L, f"enc.{l}", L.norm2)
         enc.append(L.eval())
     for l in range(m.dec_layers):
-        L = torch.nn.TransformerDecoderLayer(d, H, F, 0.0, norm_first=True, batch_first=True).double()
+        L = torch.nn.TransformerDecoderLayer(d, H, F, 0.0, activation=act, norm_first=True, batch_first=True).double()
         load_attn(L.self_attn, f"dec.{l}.self"); load_attn(L.multihead_attn, f"dec.{l}.cross")
         load_common(L, f"dec.{l}", L.norm3)
         L.norm2.weight.data = t(m.w[f"dec.{l}.ln_cross.g"]); L.norm2.bias.data = t(m.w[f"dec.{l}.ln_cross.b"])
@@ -73,13 +73,14 @@ def _torch_stack(m: O.Model):
     return enc, dec
 
 
-@pytest.mark.parametrize("causal", [True, False])
-def test_stack_equals_torch_library_layers(tiny, causal):
+@pytest.mark.parametrize("causal,act", [(True, "relu"), (False, "relu"), (True, "gelu"), (False, "gelu")])
+def test_stack_equals_torch_library_layers(tiny, causal, act):
     """Encoder memory and decoder logits equal torch.nn's pre-LN Transformer layers
-    fed the same weights (library routine as the independent definition)."""
+    fed the same weights (library routine as the independent definition), for both
+    feed-forward activations (torch's "gelu" is the exact erf form)."""
     wl, mv, _ = tiny
-    m = O.model_from(wl.verifier, mv.w, dtype=np.float64)
-    enc, dec = _torch_stack(m)
+    m = O.model_from(wl.verifier, mv.w, dtype=np.float64, act=act)
+    enc, dec = _torch_stack(m, act)
     t = lambda a: torch.tensor(np.asarray(a, dtype=np.float64))
     src = wl.src[0]
     tokens = [BOS, 17, 230, 5, 999, MASK, MASK]
@@ -102,7 +103,8 @@ def test_stack_equals_torch_library_layers(tiny, causal):
     logits = O.decoder_rows(m, tokens, mem_o, causal)
     np.testing.assert_allclose(logits, logits_ref, rtol=0, atol=1e-10)
     # and the fp32 oracle agrees with its fp64 self to rounding noise
-    l32 = O.decoder_rows(mv, tokens, O.encode(mv, src), causal)
+    m32 = O.model_from(wl.verifier, mv.w, act=act)
+    l32 = O.decoder_rows(m32, tokens, O.encode(m32, src), causal)
     assert np.abs(l32 - logits_ref).max() < 2e-5
 
 
