@@ -44,9 +44,13 @@ extern "C" {
 #define SPECDEC_DTYPE_F32   0
 #define SPECDEC_DTYPE_BF16  1
 
+#define SPECDEC_ACT_RELU    0
+#define SPECDEC_ACT_GELU    1
+
 typedef struct specdec_handle specdec_handle;
 
-/* One encoder-decoder Transformer (pre-LN, ReLU, shared embedding table). */
+/* One encoder-decoder Transformer (pre-LN, shared embedding table; position tables are weights, so
+ * sinusoidal and learned positions are both just data). */
 typedef struct {
     int d_model, n_heads, d_ffn, vocab;
     int enc_layers, dec_layers;
@@ -62,6 +66,9 @@ typedef struct {
     int compute_dtype;                 /* SPECDEC_DTYPE_F32: fp32 operands (SIMT kernels);
                                           SPECDEC_DTYPE_BF16: bf16 operands, fp32 accumulation
                                           (tcgen05 tensor-core GEMMs)                          */
+    int ffn_activation;                /* SPECDEC_ACT_RELU (Transformer-base, Section 4.1) or SPECDEC_ACT_GELU:
+                                          the exact GELU x * Phi(x), for the BART-base-shaped pair of the
+                                          summarisation experiment (Section 5.2); both models use it    */
 } specdec_config;
 
 /* One named weight.  `d_ptr` is a DEVICE pointer to fp32 data, row-major.

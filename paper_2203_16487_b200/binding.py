@@ -36,7 +36,7 @@ class ModelDims(C.Structure):
 class Config(C.Structure):
     _fields_ = [("verifier", ModelDims), ("drafter", ModelDims)] + [(n, C.c_int) for n in (
         "k_max", "max_batch", "max_src", "max_tgt", "page_tokens",
-        "pad_id", "bos_id", "eos_id", "mask_id", "compute_dtype")]
+        "pad_id", "bos_id", "eos_id", "mask_id", "compute_dtype", "ffn_activation")]
 
 
 class Tensor(C.Structure):
@@ -126,7 +126,8 @@ class SpecDec:
 
     def __init__(self, verifier_dims, verifier_w: Dict[str, np.ndarray], drafter_dims,
                  drafter_w: Dict[str, np.ndarray], *, k_max: int, max_batch: int, max_src: int, max_tgt: int,
-                 bf16: bool, page_tokens: int = 16, pad_id=0, bos_id=1, eos_id=2, mask_id=3, device="cuda:0"):
+                 bf16: bool, page_tokens: int = 16, pad_id=0, bos_id=1, eos_id=2, mask_id=3, device="cuda:0",
+                 activation: str = "relu"):
         if not torch.cuda.is_available():
             raise RuntimeError("SpecDec needs a CUDA device: the library has no CPU path")
         self._lib = lib()
@@ -134,7 +135,7 @@ class SpecDec:
         self.k_max, self.max_batch, self.max_src, self.max_tgt = k_max, max_batch, max_src, max_tgt
         self.vocab = verifier_dims.vocab
         cfg = Config(_dims(verifier_dims), _dims(drafter_dims), k_max, max_batch, max_src, max_tgt, page_tokens,
-                     pad_id, bos_id, eos_id, mask_id, 1 if bf16 else 0)
+                     pad_id, bos_id, eos_id, mask_id, 1 if bf16 else 0, {"relu": 0, "gelu": 1}[activation])
         keep, tensors = [], []
         for prefix, w in (("verifier.", verifier_w), ("drafter.", drafter_w)):
             for name, a in w.items():

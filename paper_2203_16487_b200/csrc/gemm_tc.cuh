@@ -286,8 +286,8 @@ __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R,
                         a0.x += b0.x; a0.y += b0.y; a0.z += b0.z; a0.w += b0.w;
                         a1.x += b1.x; a1.y += b1.y; a1.z += b1.z; a1.w += b1.w;
                         if (EPI == EPI_RELU) {
-                            a0.x = fmaxf(a0.x, 0.f); a0.y = fmaxf(a0.y, 0.f); a0.z = fmaxf(a0.z, 0.f); a0.w = fmaxf(a0.w, 0.f);
-                            a1.x = fmaxf(a1.x, 0.f); a1.y = fmaxf(a1.y, 0.f); a1.z = fmaxf(a1.z, 0.f); a1.w = fmaxf(a1.w, 0.f);
+                            a0.x = ffn_act(a0.x, g.act); a0.y = ffn_act(a0.y, g.act); a0.z = ffn_act(a0.z, g.act); a0.w = ffn_act(a0.w, g.act);
+                            a1.x = ffn_act(a1.x, g.act); a1.y = ffn_act(a1.y, g.act); a1.z = ffn_act(a1.z, g.act); a1.w = ffn_act(a1.w, g.act);
                         }
                         if (gr < R) {
                             bf16* o = g.out + (size_t)gr * g.ldo + nb;
@@ -314,7 +314,7 @@ __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R,
             }
             if (EPI == EPI_RELU) {
 #pragma unroll
-                for (int j = 0; j < CW; ++j) v[j] = fmaxf(v[j], 0.f);
+                for (int j = 0; j < CW; ++j) v[j] = ffn_act(v[j], g.act);
             }
             if (r >= R) continue;
             if (bf_out) {

@@ -175,27 +175,27 @@ __global__ void k_layernorm(const float* __restrict__ x, const float* __restrict
     pdl_wait();
     if (row >= *n_rows) return;
     const float* xr = x + (size_t)row * d;
-    if (d % 128 == 0 && d <= 512) {
-        float4 v[4];
+    if (d % 128 == 0 && d <= 1024) {
+        float4 v[8];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 8; ++c) {
             const int e = lane * 4 + c * 128;
             v[c] = e < d ? *reinterpret_cast<const float4*>(xr + e) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         float s = 0.f;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) s += v[c].x + v[c].y + v[c].z + v[c].w;
+        for (int c = 0; c < 8; ++c) s += v[c].x + v[c].y + v[c].z + v[c].w;
         const float mu = warp_sum(s) / d;
         float q = 0.f;
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+        for (int c = 0; c < 8; ++c)
             if (lane * 4 + c * 128 < d) {
                 const float c0 = v[c].x - mu, c1 = v[c].y - mu, c2 = v[c].z - mu, c3 = v[c].w - mu;
                 q += c0 * c0 + c1 * c1 + c2 * c2 + c3 * c3;
             }
         const float rstd = 1.0f / sqrtf(warp_sum(q) / d + eps);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 8; ++c) {
             const int e = lane * 4 + c * 128;
             if (e < d) {
                 const float4 gm = *reinterpret_cast<const float4*>(g + e), bt = *reinterpret_cast<const float4*>(b + e);
@@ -300,7 +300,12 @@ __global__ void k_attention(AttnArgs<T> a) {
 
 // ------------------------------------------------------------------ GEMM epilogues
 // C[r, n] = sum_k A[r, k] * W[n, k]  (+ bias[n])
-enum { EPI_STORE = 0, EPI_RELU = 1, EPI_RESID = 2, EPI_STATS = 3, EPI_F32 = 4, EPI_QKV = 5 };
+enum { EPI_STORE = 0, EPI_RELU = 1, EPI_RESID = 2, EPI_STATS = 3, EPI_F32 = 4, EPI_QKV = 5 };   // EPI_RELU = the feed-forward activation
+
+// Feed-forward activation of EPI_RELU: ReLU (act = 0) or the exact GELU x * Phi(x) (act = 1).
+__device__ __forceinline__ float ffn_act(float x, int act) {
+    return act ? 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)) : fmaxf(x, 0.f);
+}
 
 // Partial statistics of one verifier (or drafter) row over one tile of vocabulary columns.
 struct __align__(16) RowPart { float mx; int arg; float sum; int cnt; };
@@ -315,6 +320,7 @@ struct GemmArgs {
     int rows_static;            // >= 0: the row count is known on the host (saves a dependent load); else read n_rows
     int one_m_tile;             // tensor-core path: the rows fit one 128-row tile whatever n_rows says
     T* out; int ldo;            // EPI_STORE / EPI_RELU
+    int act;                    // EPI_RELU: 0 ReLU, 1 exact GELU
     float* resid;               // EPI_RESID: resid[r, n] += value ; EPI_F32: resid[r, n] = value (ld = N)
     // EPI_STATS
     RowPart* part; int n_tiles; // part[r * n_tiles + tile]
@@ -397,7 +403,7 @@ __global__ void __launch_bounds__(256) k_gemm_simt(GemmArgs<T> g) {
                 Ct[ty * 4 + i][tx * 4 + j] = v;
             } else if (r < R && n < g.N) {
                 if (EPI == EPI_STORE) g.out[(size_t)r * g.ldo + n] = from_f<T>(v);
-                if (EPI == EPI_RELU) g.out[(size_t)r * g.ldo + n] = from_f<T>(fmaxf(v, 0.f));
+                if (EPI == EPI_RELU) g.out[(size_t)r * g.ldo + n] = from_f<T>(ffn_act(v, g.act));
                 if (EPI == EPI_RESID) g.resid[(size_t)r * g.N + n] += v;
                 if (EPI == EPI_F32) g.resid[(size_t)r * g.N + n] = v;
             }

@@ -187,7 +187,7 @@ void layout_model(specdec_handle* h, ModelW& m, const specdec_model_dims& dm) {
 // The cluster decoder kernel needs one CTA per head of 64 columns and operand rows that fit its shared memory.
 bool cl_eligible(const specdec_config& c) {
     const specdec_model_dims& v = c.verifier;
-    return c.compute_dtype == SPECDEC_DTYPE_BF16 && v.n_heads == CL_C && v.d_model == CL_C * 64 && v.d_model <= 512 &&
+    return c.compute_dtype == SPECDEC_DTYPE_BF16 && c.ffn_activation == SPECDEC_ACT_RELU && v.n_heads == CL_C && v.d_model == CL_C * 64 && v.d_model <= 512 &&
            v.d_ffn % (CL_C * 64) == 0 && v.d_ffn <= 2048 && v.dec_layers <= CL_MAX_LAYERS;
 }
 
@@ -423,7 +423,7 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
     GemmArgs<T> g;
     g.A = (const T*)A; g.lda = lda; g.W = (const T*)W; g.bias = bias; g.N = N; g.K = K;
     g.n_rows = h->ses.counters + cnt; g.rows_static = (cnt == CNT_VERIFY || cnt == CNT_ENC) ? rows_ub : -1; g.out = (T*)out; g.ldo = ldo; g.resid = resid;
-    g.one_m_tile = 0;
+    g.one_m_tile = 0; g.act = h->cfg.ffn_activation;
     g.part = h->part; g.ld = ldv; g.ld_id = ld_id; g.n_tiles = cdiv(N, 64); g.want_sum = h->want_lse;
     g.seq = nullptr; g.pos = nullptr; g.kc = nullptr; g.vc = nullptr; g.kv_d = 0;
     g.pg.table = h->page_table; g.pg.page_tokens = h->cfg.page_tokens; g.pg.max_pages = h->pages_per_seq;
@@ -1007,6 +1007,8 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
         return fail(nullptr, SPECDEC_ERR_INVALID_ARG, "page_tokens must be a power of two");
     if (cfg->compute_dtype != SPECDEC_DTYPE_F32 && cfg->compute_dtype != SPECDEC_DTYPE_BF16)
         return fail(nullptr, SPECDEC_ERR_INVALID_ARG, "compute_dtype must be 0 (fp32) or 1 (bf16)");
+    if (cfg->ffn_activation != SPECDEC_ACT_RELU && cfg->ffn_activation != SPECDEC_ACT_GELU)
+        return fail(nullptr, SPECDEC_ERR_INVALID_ARG, "ffn_activation must be 0 (ReLU) or 1 (GELU)");
     if (cfg->verifier.vocab != cfg->drafter.vocab)
         return fail(nullptr, SPECDEC_ERR_INVALID_ARG, "verifier and drafter must share the vocabulary");
     const int need_pos = cfg->max_tgt + cfg->k_max + 1;

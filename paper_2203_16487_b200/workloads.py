@@ -85,7 +85,7 @@ def sinusoid_table(n_pos: int, d: int) -> np.ndarray:
 
 
 def make_weights(dims: ModelDims, seed: int, bf16: bool,
-                 embed_std: float = 0.02) -> Dict[str, np.ndarray]:
+                 embed_std: float = 0.02, learned_pos: bool = False) -> Dict[str, np.ndarray]:
     """Random-init weights N(0, 0.02^2); LN gain 1 + N(0, 0.02^2).
 
     Names (row-major [out, in], y = x W^T + b):
@@ -95,7 +95,8 @@ def make_weights(dims: ModelDims, seed: int, bf16: bool,
       enc.{l}.ffn.{w1,b1,w2,b2}  enc.ln_f.{g,b}
       dec.{l}. ... same plus  ln_cross.{g,b}  cross.{q,k,v,o}.{w,b} ;  dec.ln_f.{g,b}
     With bf16=True every matrix (ndim >= 2, position tables excepted) is rounded
-    once to bf16-representable values.
+    once to bf16-representable values.  learned_pos=True draws the position tables
+    N(0, 0.02^2) instead of evaluating sinusoids (BART-style learned positions).
     """
     rng = np.random.default_rng(seed)
     d, f, v = dims.d_model, dims.d_ffn, dims.vocab
@@ -119,8 +120,12 @@ def make_weights(dims: ModelDims, seed: int, bf16: bool,
         mat(prefix + ".w2", (d, f)); mat(prefix + ".b2", (d,))
 
     mat("embed", (v, d), embed_std)
-    w["pos_enc"] = sinusoid_table(dims.max_pos, d)
-    w["pos_dec"] = sinusoid_table(dims.max_pos, d)
+    if learned_pos:
+        w["pos_enc"] = rng.standard_normal((dims.max_pos, d), dtype=np.float32) * np.float32(0.02)
+        w["pos_dec"] = rng.standard_normal((dims.max_pos, d), dtype=np.float32) * np.float32(0.02)
+    else:
+        w["pos_enc"] = sinusoid_table(dims.max_pos, d)
+        w["pos_dec"] = sinusoid_table(dims.max_pos, d)
     for l in range(dims.enc_layers):
         ln(f"enc.{l}.ln1"); attn(f"enc.{l}.self"); ln(f"enc.{l}.ln2"); ffn(f"enc.{l}.ffn")
     ln("enc.ln_f")
@@ -170,6 +175,10 @@ TINY_V = ModelDims(64, 4, 256, 1000, 2, 2, 64)
 TINY_D = ModelDims(64, 4, 256, 1000, 2, 1, 64)
 BASE_V = ModelDims(512, 8, 2048, 32768, 6, 6, 1024)
 BASE_D = ModelDims(512, 8, 2048, 32768, 12, 2, 1024)
+# BART-base shapes (public model card, not the paper): 768 wide, 12 heads, 3072 inner, 50265 ids, GELU, learned
+# positions; the drafter starts from the BART-base encoder (Section 5.2), so 6 encoder layers + 2 decoder layers.
+BART_V = ModelDims(768, 12, 3072, 50265, 6, 6, 1026)
+BART_D = ModelDims(768, 12, 3072, 50265, 6, 2, 1026)
 
 
 def config1_tiny(beta: int = 3, tau: float = 1.0) -> Workload:
@@ -206,6 +215,15 @@ def config4_summarization(batch: int = 8) -> Workload:
     wl.src = make_sources(rng, 8, 300, 512, BASE_V.vocab)[:batch]
     wl.max_tgt = [128] * len(wl.src)
     return wl
+
+
+def config_bart_summarization(batch: int = 4, lo: int = 300, hi: int = 512) -> Workload:
+    """BART-base-shaped pair on paragraph-length sources (the summarisation setting of Section 5.2); weights via
+    make_weights(..., learned_pos=True), handle / oracle with the GELU activation."""
+    rng = np.random.default_rng(106)
+    src = make_sources(rng, batch, lo, hi, BART_V.vocab)
+    return Workload("config_bart_summarization", BART_V, BART_D, 25, 3, 1.0, True, 3001, 3002, 106, src,
+                    [128] * batch)
 
 
 def config5_microbench(batch: int, src_len: int = 64) -> Workload:

@@ -45,5 +45,8 @@ def test_no_device_means_error_not_fallback():
     # argument validation happens before any device work
     cfg.page_tokens = 12
     assert lib.specdec_create(C.byref(cfg), t, 1, None, C.byref(h)) == -1
+    cfg.page_tokens, cfg.ffn_activation = 16, 7
+    assert lib.specdec_create(C.byref(cfg), t, 1, None, C.byref(h)) == -1
+    assert b"ffn_activation" in lib.specdec_last_error(None)
     with pytest.raises(RuntimeError):
         binding.SpecDec(None, {}, None, {}, k_max=1, max_batch=1, max_src=1, max_tgt=1, bf16=False)

@@ -159,3 +159,28 @@ def test_shape_variants_12_2_verifier_and_narrow_heads():
         got = out[b, :int(n[b])].cpu().tolist()
         assert got == ref or _prefix_match(got, ref) >= 3
     sd.close()
+
+
+def test_bart_base_shaped_pair_gelu_learned_positions():
+    """The summarisation experiment's model family (Section 5.2): BART-base shapes (768 wide, 12 heads, 3072 inner,
+    50265 ids: an odd vocabulary with a ragged last column tile), exact GELU, learned position tables, a drafter
+    with the 6-layer encoder.  Lock-step against the oracle, then a batched generate with one sampled sequence."""
+    from paper_2203_16487_b200 import binding
+    wl = W.config_bart_summarization(3, 40, 150)
+    wv = W.make_weights(wl.verifier, wl.seed_verifier, True, learned_pos=True)
+    wd = W.make_weights(wl.drafter, wl.seed_drafter, True, learned_pos=True)
+    mv = O.model_from(wl.verifier, wv, mode="bf16", act="gelu")
+    md = O.model_from(wl.drafter, wd, mode="bf16", act="gelu")
+    smax = max(len(s) for s in wl.src)
+    sd = binding.SpecDec(wl.verifier, wv, wl.drafter, wd, k_max=25, max_batch=3, max_src=smax, max_tgt=40, bf16=True,
+                         activation="gelu")
+    rep = lockstep.run(sd, mv, md, wl.src[:2], [40, 40], 25, 3, 1.0, margin=1e-3, check_logits_every=2, max_iters=3)
+    print(rep.iterations, rep.draft_near_ties, rep.verify_near_ties, rep.max_logit_err, rep.max_stat_err, rep.notes[:3])
+    assert rep.ok, rep.notes
+    assert rep.max_logit_err < 2e-2
+    src, lens = W.pad_batch(wl.src)
+    out, n, st = sd.generate(src, lens, [40, 30, 20], 25, 3, 1.0)
+    assert st["emitted"] == int(n.sum()) and n.cpu().tolist() == [40, 30, 20]
+    ref, _ = O.specdec_generate(mv, md, wl.src[2], 10, 25, 3, 1.0, BOS, EOS, MASK)
+    assert out[2, :10].cpu().tolist() == ref
+    sd.close()
