@@ -110,6 +110,8 @@ def main():
     ap.add_argument("--gemm", type=int, default=1)
     ap.add_argument("--graphs", type=int, default=1)
     ap.add_argument("--tc-bn", type=int, default=0, help="force the N tile of the tensor-core GEMM (experiments)")
+    ap.add_argument("--model", choices=["base", "bart"], default="base",
+                    help="Transformer-base pair (default) or the BART-base-shaped pair (GELU, learned positions)")
     ap.add_argument("--opt", action="append", default=[], help="library option name=value (repeatable; experiments)")
     ap.add_argument("--grid", action="store_true", help="the whole k x prefix x batch grid of the verify microbench")
     args = ap.parse_args()
@@ -124,10 +126,14 @@ def main():
         print("|---|---|---|---|---|---|---|---|---|---|---|")
     for B in batches:
         wl = W.config5_microbench(B, S)
-        wv = W.make_weights(wl.verifier, wl.seed_verifier, True)
-        wd = W.make_weights(wl.drafter, wl.seed_drafter, True)
+        bart = args.model == "bart"
+        if bart:
+            wl.verifier, wl.drafter = W.BART_V, W.BART_D
+            wl.src = [W.zipf_ids(np.random.default_rng(105 + b), S, W.BART_V.vocab) for b in range(B)]
+        wv = W.make_weights(wl.verifier, wl.seed_verifier, True, learned_pos=bart)
+        wd = W.make_weights(wl.drafter, wl.seed_drafter, True, learned_pos=bart)
         sd = binding.SpecDec(wl.verifier, wv, wl.drafter, wd, k_max=max(ks), max_batch=B, max_src=S,
-                             max_tgt=max(prefixes) + max(ks) + 2, bf16=True)
+                             max_tgt=max(prefixes) + max(ks) + 2, bf16=True, activation="gelu" if bart else "relu")
         del wv, wd
         sd.set_option("gemm", args.gemm)
         sd.set_option("graphs", args.graphs)
