@@ -213,6 +213,10 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
  * "pair" = 0/1 two-SM tensor-core tiles (256 rows x 256 columns per CTA pair) for GEMMs with at least 1024 rows
  *   and 1024 columns (default 0: same results bit for bit, measured no faster than single-SM tiles at these
  *   sizes, kept for comparison);
+ * "ln_fuse" = 0/1 apply the LayerNorm that reads the residual stream next inside the residual GEMM that
+ *   writes it (tensor-core path: the CTAs of a row tile form a cluster and exchange per-row sums through
+ *   distributed shared memory; default 0: correct, but its longer single-tile tail costs more than the
+ *   separate LayerNorm launch it removes: 743 vs 688 us per 128-sequence verify step);
  * "attn_warps" = 0 choose per launch, 4 or 8 warps per CTA of the tile attention (default 0);
  * "tc_bn" = 0 choose, else force the column width of the tensor-core GEMM tiles (64 / 128 / 256; experiments);
  * "cluster" = 0/1 run the verifier's decoder stack as one thread-block-cluster kernel per sequence when the

@@ -124,12 +124,12 @@ constexpr int TC_THREADS = (2 + TC_EPI_WARPS) * 32;  // + TMA warp + MMA warp
 // AR = rows of the activation box a stage holds (the MMA always spans 128 rows; with AR < 128 the rows beyond
 // the box are whatever shared memory holds and only feed accumulator lanes that nobody reads).  STG = the
 // epilogue needs its transpose buffers.
-template <int BN, int AR = 128, bool STG = true> struct TcCfg {
+template <int BN, int AR = 128, bool STG = true, bool LNF = false> struct TcCfg {   // LNF: room for the row statistics
     static constexpr int STAGE_BYTES = (AR + BN) * TC_BK * 2;
     static constexpr int STG_BYTES = STG ? TC_EPI_WARPS * 32 * 32 * 4 : 0;   // per-warp 32 x 32 fp32 transpose buffers
     static_assert(BN >= 128 - AR, "the 128-row MMA read of a short activation box must stay inside its stage");
     static constexpr int FIT = (232448 - 1024 - STG_BYTES) / STAGE_BYTES;
-    static constexpr int STAGES = AR < 128 || !STG ? (FIT > 8 ? 8 : FIT) : (BN > 128 ? 4 : (BN >= 128 ? 6 : 8));
+    static constexpr int STAGES = (AR < 128 || !STG ? (FIT > 8 ? 8 : FIT) : (BN > 128 ? 4 : (BN >= 128 ? 6 : 8))) - (LNF ? 1 : 0);
     static constexpr int SMEM = STAGES * STAGE_BYTES + STG_BYTES + 1024;
     static constexpr int TMEM_COLS = 2 * BN <= 32 ? 32 : (2 * BN <= 64 ? 64 : (2 * BN <= 128 ? 128 : (2 * BN <= 256 ? 256 : 512)));  // two accumulators, power of two
 };
@@ -153,17 +153,41 @@ __device__ __forceinline__ void tmem_ld(uint32_t taddr, float* v) {
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+__device__ __forceinline__ void tc_cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t tc_cluster_nctas() {
+    uint32_t n;
+    asm volatile("mov.u32 %0, %%cluster_nctaid.x;" : "=r"(n));
+    return n;
+}
+// Two floats to shared-memory address `local_addr` of CTA `rank` of this cluster, counted (8 bytes) on the mbarrier at
+// `local_bar` of that same CTA: the receiver learns of the data through its own barrier, no cluster-wide fence needed.
+__device__ __forceinline__ void tc_st_peer2(uint32_t local_addr, uint32_t local_bar, uint32_t rank, float a, float b) {
+    uint32_t ra, rb;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rb) : "r"(local_bar), "r"(rank));
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
+                 ::"r"(ra), "f"(a), "f"(b), "r"(rb) : "memory");
+}
+
 // One tile of the epilogue, for one of the eight epilogue warps: q = the TMEM lane quadrant the warp may read,
 // half = which half of the tile's BN columns it takes; tmem_acc = the tile's accumulator.  Requests what it can
 // before waiting for the accumulator (residual tile, bias, cache rows, draft logits), then reads tensor memory
 // chunk by chunk.  The caller hands the accumulator back afterwards.
-template <int EPI, int BN>
+// LNF (residual epilogue only): bias and residual are added while a thread still owns a whole row (so its sum and sum
+// of squares over the warp's columns need no shuffles), the pair is written into EVERY cluster peer's
+// ln_part[row][2 * rank + half], and the new residual values stay in `keep` for the fused LayerNorm that follows.
+template <int EPI, int BN, bool LNF = false>
 __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R, int m0, int n_tile, int q, int half, int lane,
                                                  uint32_t tmem_acc, float* stg, uint32_t bar_acc_full_addr, uint32_t parity,
-                                                 volatile int* abort_flag, int* err_word, bool later_tile) {
+                                                 volatile int* abort_flag, int* err_word, bool later_tile,
+                                                 float* ln_part = nullptr, float4 (*keep)[8] = nullptr,
+                                                 const float* bias_s = nullptr, uint32_t ln_bar = 0) {
+    static_assert(!LNF || (EPI == EPI_RESID && BN <= 128 && BN % 64 == 0), "fused LayerNorm: residual epilogue, 64 or 128 columns");
     constexpr int HALF = BN / 2;                     // columns per epilogue warp
     constexpr int CW = HALF % 32 == 0 ? 32 : 16;     // columns per TMEM read
-    constexpr bool bf_out = (EPI == EPI_STORE || EPI == EPI_RELU || EPI == EPI_QKV);
+    constexpr bool bf_out = (EPI == EPI_STORE || EPI == EPI_RELU || EPI == EPI_GELU || EPI == EPI_QKV);
     constexpr int NCH = HALF / CW;                   // column chunks per warp and tile
     // 16-byte accesses after the transpose need aligned rows
     const bool vec_ok = CW == 32 && (bf_out ? (g.ldo % 8 == 0 && (EPI != EPI_QKV || g.kv_d % 32 == 0)) : (g.N % 4 == 0));
@@ -180,12 +204,17 @@ __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R,
             if (nb + CW <= g.N) {
 #pragma unroll
                 for (int ps = 0; ps < 8; ++ps) {
-                    const int gr = rbase + ps * 4 + (lane >> 3);
-                    xin[c][ps] = gr < R ? *reinterpret_cast<const float4*>(g.resid + (size_t)gr * g.N + nb + (lane & 7) * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    if constexpr (LNF) {             // row layout: this thread's own row, columns 4 ps .. 4 ps + 3 of the chunk
+                        xin[c][ps] = r < R ? *reinterpret_cast<const float4*>(g.resid + (size_t)r * g.N + nb + ps * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    } else {
+                        const int gr = rbase + ps * 4 + (lane >> 3);
+                        xin[c][ps] = gr < R ? *reinterpret_cast<const float4*>(g.resid + (size_t)gr * g.N + nb + (lane & 7) * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
                 }
             }
         }
     }
+    float ln_s1 = 0.f, ln_s2 = 0.f;                  // LNF: sum and sum of squares of this thread's row over the warp's columns
     // ... and so are this lane's bias columns, its cache row and its draft logit
     float4 bzv[NCH][2];
     if (EPI != EPI_STATS && vec_ok && g.bias) {
@@ -251,6 +280,16 @@ __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R,
                 }
             }
             tmem_ld<CW>(trow + c * CW, v);
+            if constexpr (LNF) {
+#pragma unroll
+                for (int j4 = 0; j4 < 8; ++j4) {
+                    const float4 bz = *reinterpret_cast<const float4*>(bias_s + half * HALF + c * CW + j4 * 4);   // staged at set-up
+                    const float4 x = xin[c & 1][j4];
+                    v[j4 * 4] += bz.x + x.x; v[j4 * 4 + 1] += bz.y + x.y; v[j4 * 4 + 2] += bz.z + x.z; v[j4 * 4 + 3] += bz.w + x.w;
+                    ln_s1 += (v[j4 * 4] + v[j4 * 4 + 1]) + (v[j4 * 4 + 2] + v[j4 * 4 + 3]);
+                    ln_s2 += (v[j4 * 4] * v[j4 * 4] + v[j4 * 4 + 1] * v[j4 * 4 + 1]) + (v[j4 * 4 + 2] * v[j4 * 4 + 2] + v[j4 * 4 + 3] * v[j4 * 4 + 3]);
+                }
+            }
             if (CW == 32 && vec_ok && nb + CW <= g.N) {
                 // Transpose through shared memory: a thread owns one output ROW in tensor memory, but global
                 // memory wants neighbouring lanes on neighbouring addresses.  The 32 x 32 block is written row-wise
@@ -268,9 +307,12 @@ __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R,
                     for (int ps = 0; ps < 8; ++ps) {
                         const int rr = ps * 4 + rsub, gr = rbase + rr;
                         float4 a = *reinterpret_cast<const float4*>(stg + rr * 32 + ((l8 ^ (rr & 7)) << 2));
-                        a.x += bz.x; a.y += bz.y; a.z += bz.z; a.w += bz.w;
-                        if (EPI == EPI_RESID) { const float4 x = xin[c & 1][ps]; a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w; }
+                        if constexpr (!LNF) {
+                            a.x += bz.x; a.y += bz.y; a.z += bz.z; a.w += bz.w;
+                            if (EPI == EPI_RESID) { const float4 x = xin[c & 1][ps]; a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w; }
+                        }
                         if (gr < R) *reinterpret_cast<float4*>(g.resid + (size_t)gr * g.N + nb + l8 * 4) = a;
+                        if constexpr (LNF) keep[c][ps] = a;
                     }
                 } else {
                     // bf16 rows: 4 lanes per row (8 columns = 16 bytes each), 8 rows per pass
@@ -286,8 +328,12 @@ __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R,
                         a0.x += b0.x; a0.y += b0.y; a0.z += b0.z; a0.w += b0.w;
                         a1.x += b1.x; a1.y += b1.y; a1.z += b1.z; a1.w += b1.w;
                         if (EPI == EPI_RELU) {
-                            a0.x = ffn_act(a0.x, g.act); a0.y = ffn_act(a0.y, g.act); a0.z = ffn_act(a0.z, g.act); a0.w = ffn_act(a0.w, g.act);
-                            a1.x = ffn_act(a1.x, g.act); a1.y = ffn_act(a1.y, g.act); a1.z = ffn_act(a1.z, g.act); a1.w = ffn_act(a1.w, g.act);
+                            a0.x = fmaxf(a0.x, 0.f); a0.y = fmaxf(a0.y, 0.f); a0.z = fmaxf(a0.z, 0.f); a0.w = fmaxf(a0.w, 0.f);
+                            a1.x = fmaxf(a1.x, 0.f); a1.y = fmaxf(a1.y, 0.f); a1.z = fmaxf(a1.z, 0.f); a1.w = fmaxf(a1.w, 0.f);
+                        }
+                        if (EPI == EPI_GELU) {
+                            a0.x = ffn_act(a0.x, 1); a0.y = ffn_act(a0.y, 1); a0.z = ffn_act(a0.z, 1); a0.w = ffn_act(a0.w, 1);
+                            a1.x = ffn_act(a1.x, 1); a1.y = ffn_act(a1.y, 1); a1.z = ffn_act(a1.z, 1); a1.w = ffn_act(a1.w, 1);
                         }
                         if (gr < R) {
                             bf16* o = g.out + (size_t)gr * g.ldo + nb;
@@ -312,9 +358,9 @@ __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R,
 #pragma unroll
                 for (int j = 0; j < CW; ++j) v[j] += (nb + j < g.N) ? __ldg(g.bias + nb + j) : 0.f;
             }
-            if (EPI == EPI_RELU) {
+            if (EPI == EPI_RELU || EPI == EPI_GELU) {
 #pragma unroll
-                for (int j = 0; j < CW; ++j) v[j] = ffn_act(v[j], g.act);
+                for (int j = 0; j < CW; ++j) v[j] = ffn_act(v[j], EPI == EPI_GELU ? 1 : 0);
             }
             if (r >= R) continue;
             if (bf_out) {
@@ -332,6 +378,11 @@ __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R,
             }
         }
     }
+    if constexpr (LNF) {                             // this row's partial statistics into every peer's table; every warp
+        const uint32_t nct = tc_cluster_nctas();     // sends (rows past the end send what they have) so the byte count is fixed
+        const uint32_t slot = smem_u32(ln_part + ((q * 32 + lane) * 16 + n_tile * 2 + half) * 2);
+        for (uint32_t rk = 0; rk < nct; ++rk) tc_st_peer2(slot, ln_bar, rk, ln_s1, ln_s2);
+    }
     tc_fence_before();
     __syncwarp();
 }
@@ -339,11 +390,17 @@ __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R,
 // Persistent kernel: CTA c works on tiles c, c + gridDim.x, ... (row tile fastest, so CTAs running
 // together share one weight tile).  The TMA ring and the two TMEM accumulators run across tiles, so the
 // epilogue of tile i overlaps the loads and MMAs of tile i + 1.
-template <int EPI, int BN, int AR = 128>
+//
+// LNF (residual epilogue, N = the model width): the LayerNorm that consumes the new residual stream is applied in the
+// same kernel.  The CTAs of one row tile form a cluster (N / BN of them, one tile each, column tile = cluster rank);
+// each writes per-row sums and sums of squares of its columns into every peer's shared memory (distributed shared
+// memory stores), and after one cluster barrier every CTA has the whole row's statistics locally and normalises the values it still holds in registers into
+// g.ln_out (bf16).  Sums are added in a fixed order; the variance is E[x^2] - mean^2 in fp32.
+template <int EPI, int BN, int AR = 128, bool LNF = false>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, GemmArgs<bf16> g,
           int* err_word) {
-    using Cfg = TcCfg<BN, AR, EPI != EPI_STATS>;
+    using Cfg = TcCfg<BN, AR, EPI != EPI_STATS, LNF>;
     constexpr int STAGES = Cfg::STAGES;
     constexpr int A_BYTES = AR * TC_BK * 2;          // activation part of a stage
     if (threadIdx.x == 0) tc_stamp(g.trace, 0);
@@ -361,6 +418,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     __shared__ __align__(8) uint64_t bar_full[STAGES], bar_empty[STAGES], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
+    __shared__ __align__(16) float ln_part_s[LNF ? TC_BM * 32 : 1];  // [row][2 * cluster rank + column half][sum, sum of squares]
+    __shared__ float ln_mr_s[LNF ? TC_BM * 2 : 1];                   // [row][mean, 1 / std]
+    __shared__ __align__(16) float bias_s[LNF ? BN : 1];             // LNF: this tile's bias columns
+    __shared__ __align__(8) uint64_t bar_ln;                         // LNF: counts the peers' statistics as they arrive
+    float4 keep[2][8];                                               // LNF: this thread's new residual values
     const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb = g.K / TC_BK;
@@ -375,8 +437,20 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         tc_stamp(g.trace, 12);
     }
     if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_s), Cfg::TMEM_COLS); if (lane == 0) tc_stamp(g.trace, 13); }
-    tc_fence_before();
-    __syncthreads();
+    if constexpr (LNF) {
+        const int nt0 = ((int)blockIdx.x % n_tiles) * BN;
+        for (int i = threadIdx.x; i < BN; i += TC_THREADS) bias_s[i] = g.bias ? __ldg(g.bias + nt0 + i) : 0.f;   // a weight: before the wait
+        if (threadIdx.x == 0) {
+            mbar_init(smem_u32(&bar_ln), 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            mbar_expect_tx(smem_u32(&bar_ln), tc_cluster_nctas() * TC_EPI_WARPS * 32 * 8);   // 8 bytes from every epilogue thread of every peer
+        }
+        tc_fence_before();
+        tc_cluster_sync();                           // peers' barriers exist before anybody sends (all of this precedes the dependency wait)
+    } else {
+        tc_fence_before();
+        __syncthreads();
+    }
     tc_fence_after();
     const uint32_t tmem_d = tmem_base_s;
     volatile int* abort_flag = &abort_s;
@@ -384,7 +458,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     int pre = 0;                                       // stages whose weight half was requested before the wait
     if (early) {
         if (threadIdx.x == 0) {
-            const int n0 = ((int)blockIdx.x / m_tiles) * BN;
+            const int n0 = (LNF ? (int)blockIdx.x % n_tiles : (int)blockIdx.x / m_tiles) * BN;
             for (; pre < STAGES && pre < nkb; ++pre) {
                 const uint32_t bar = smem_u32(&bar_full[pre]);
                 mbar_expect_tx(bar, Cfg::STAGE_BYTES);
@@ -400,7 +474,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         if (lane == 0) {
             int kbi = 0;                               // k-blocks issued so far, over all tiles
             for (int t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
-                const int m0 = (t % m_tiles) * TC_BM, n0 = (t / m_tiles) * BN;
+                const int m0 = (LNF ? t / n_tiles : t % m_tiles) * TC_BM, n0 = (LNF ? t % n_tiles : t / m_tiles) * BN;
                 for (int kb = 0; kb < nkb; ++kb, ++kbi) {
                     const int s = kbi % STAGES;
                     if (kbi >= STAGES) mbar_wait(smem_u32(&bar_empty[s]), ((kbi / STAGES) - 1) & 1, abort_flag, err_word, 1);
@@ -457,16 +531,59 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         int i = 0;
         for (int t = blockIdx.x; t < total; t += gridDim.x, ++i) {
             const int ab = i & 1;
-            const int m0 = (t % m_tiles) * TC_BM, n_tile = t / m_tiles;
-            tc_epilogue_tile<EPI, BN>(g, R, m0, n_tile, q, half, lane, tmem_d + ab * BN, stg, smem_u32(&bar_acc_full[ab]),
-                                      (i >> 1) & 1, abort_flag, err_word, i > 0);
+            const int m0 = (LNF ? t / n_tiles : t % m_tiles) * TC_BM, n_tile = LNF ? t % n_tiles : t / m_tiles;
+            tc_epilogue_tile<EPI, BN, LNF>(g, R, m0, n_tile, q, half, lane, tmem_d + ab * BN, stg, smem_u32(&bar_acc_full[ab]),
+                                           (i >> 1) & 1, abort_flag, err_word, i > 0, ln_part_s, keep, bias_s, smem_u32(&bar_ln));
             // this warp is done with the accumulator: hand it back to the MMA warp
             if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[ab]));
             if (threadIdx.x == 64) tc_stamp(g.trace, 8 + 2 * (i > 0));
         }
     }
-    tc_fence_before();
-    __syncthreads();
+    if constexpr (LNF) {
+        if (warp >= 2) {
+            const int q = warp & 3, half = (warp - 2) >> 2;
+            const int m0 = ((int)blockIdx.x / n_tiles) * TC_BM, n_tile = (int)blockIdx.x % n_tiles;
+            if (half == 0) {                         // one thread per row: the whole row's statistics, slots in a fixed order
+                mbar_wait(smem_u32(&bar_ln), 0, abort_flag, err_word, 7);   // every peer's partial sums have landed here
+                const int row = q * 32 + lane;
+                const float* pr = ln_part_s + row * 32;
+                float s1 = 0.f, s2 = 0.f;
+                for (int sl = 0; sl < 2 * n_tiles; ++sl) { s1 += pr[sl * 2]; s2 += pr[sl * 2 + 1]; }
+                const float mu = s1 / g.N;
+                const float var = fmaxf(s2 / g.N - mu * mu, 0.f);
+                ln_mr_s[row * 2] = mu;
+                ln_mr_s[row * 2 + 1] = 1.0f / sqrtf(var + g.ln_eps);
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(TC_EPI_WARPS * 32) : "memory");     // the eight epilogue warps only
+            constexpr int HALF = BN / 2, NCH = HALF / 32;
+            const int l8 = lane & 7, rsub = lane >> 3, rbase = m0 + q * 32;
+            if (rbase < R) {
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    const int nb = n_tile * BN + half * HALF + c * 32;
+                    const float4 gm = __ldg(reinterpret_cast<const float4*>(g.ln_g + nb) + l8);
+                    const float4 bt = __ldg(reinterpret_cast<const float4*>(g.ln_b + nb) + l8);
+#pragma unroll
+                    for (int ps = 0; ps < 8; ++ps) {
+                        const int rr = ps * 4 + rsub, gr = rbase + rr;
+                        const float mu = ln_mr_s[(q * 32 + rr) * 2], rstd = ln_mr_s[(q * 32 + rr) * 2 + 1];
+                        const float4 a = keep[c][ps];
+                        if (gr < R) {
+                            __nv_bfloat162 p0 = __floats2bfloat162_rn((a.x - mu) * rstd * gm.x + bt.x, (a.y - mu) * rstd * gm.y + bt.y);
+                            __nv_bfloat162 p1 = __floats2bfloat162_rn((a.z - mu) * rstd * gm.z + bt.z, (a.w - mu) * rstd * gm.w + bt.w);
+                            uint2 pk; pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+                            *reinterpret_cast<uint2*>(g.ln_out + (size_t)gr * g.N + nb + l8 * 4) = pk;
+                        }
+                    }
+                }
+            }
+        }
+        tc_fence_before();
+        __syncthreads();                             // (peers only ever WROTE into this CTA, before the cluster barrier)
+    } else {
+        tc_fence_before();
+        __syncthreads();
+    }
     if (warp == 1) tmem_dealloc(tmem_d, Cfg::TMEM_COLS);
     if (threadIdx.x == 0) tc_stamp(g.trace, 11);
 }
@@ -536,9 +653,12 @@ inline int tc_init(TmaEncoder& enc, int* err_word) {
     enc.encode = (PFN_encodeTiled)fn;
     cudaError_t e = tc_set_smem_all<EPI_STORE>();
     if (e == cudaSuccess) e = tc_set_smem_all<EPI_RELU>();
+    if (e == cudaSuccess) e = tc_set_smem_all<EPI_GELU>();
     if (e == cudaSuccess) e = tc_set_smem_all<EPI_RESID>();
     if (e == cudaSuccess) e = tc_set_smem_all<EPI_F32>();
     if (e == cudaSuccess) e = tc_set_smem_all<EPI_QKV>();
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_tc<EPI_RESID, 64, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<64, 128, true, true>::SMEM);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_tc<EPI_RESID, 128, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<128, 128, true, true>::SMEM);
     if (e == cudaSuccess) e = tc_set_smem<EPI_STATS, 128>();
     if (e == cudaSuccess) e = tc_set_smem<EPI_STATS, 224, 32>();
     if (e == cudaSuccess) e = tc_set_smem<EPI_STATS, 224, 64>();
@@ -568,6 +688,35 @@ inline int tc_launch_one(TmaEncoder& enc, GemmArgs<bf16>& g, int rows_ub, cudaSt
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { enc.err = std::string("launch: ") + cudaGetErrorString(e); return -1; }
     return 0;
+}
+
+// Residual GEMM with the following LayerNorm fused (see k_gemm_tc, LNF): one cluster of N / BN CTAs per row tile.
+inline bool tc_ln_fusable(int N, int K) { return N % 128 == 0 && N <= 1024 && K % TC_BK == 0 && K >= TC_BK; }
+template <int BN>
+inline int tc_launch_ln_one(TmaEncoder& enc, GemmArgs<bf16>& g, int rows_ub, cudaStream_t st) {
+    const CUtensorMap* ta = enc.get(g.A, rows_ub, g.K, g.lda, TC_BM);
+    const CUtensorMap* tw = enc.get(g.W, g.N, g.K, g.K, BN);
+    if (!ta || !tw) return -1;
+    const int n_tiles = g.N / BN, m_tiles = (rows_ub + TC_BM - 1) / TC_BM;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_tiles * m_tiles); cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = TcCfg<BN, 128, true, true>::SMEM; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = n_tiles; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = enc.pdl ? 2 : 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_gemm_tc<EPI_RESID, BN, 128, true>, *ta, *tw, g, enc.err_word);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) { enc.err = std::string("launch (fused LayerNorm): ") + cudaGetErrorString(e); return -1; }
+    return 0;
+}
+inline int gemm_tc_launch_ln(TmaEncoder& enc, GemmArgs<bf16>& g, int rows_ub, cudaStream_t st) {
+    if (!enc.ready) return -1;
+    g.one_m_tile = 0;
+    // 64-wide tiles (clusters of up to 8) while there are few row tiles, 128-wide otherwise and for wide models
+    const bool narrow = rows_ub <= 2 * TC_BM && g.N <= 512;
+    return narrow ? tc_launch_ln_one<64>(enc, g, rows_ub, st) : tc_launch_ln_one<128>(enc, g, rows_ub, st);
 }
 
 template <int EPI>
@@ -626,6 +775,7 @@ inline int gemm_tc_launch(TmaEncoder& enc, int epi, GemmArgs<bf16>& g, int rows_
     switch (epi) {
         case EPI_STORE: return tc_launch_bn<EPI_STORE>(enc, bn, g, rows_ub, st);
         case EPI_RELU: return tc_launch_bn<EPI_RELU>(enc, bn, g, rows_ub, st);
+        case EPI_GELU: return tc_launch_bn<EPI_GELU>(enc, bn, g, rows_ub, st);
         case EPI_RESID: return tc_launch_bn<EPI_RESID>(enc, bn, g, rows_ub, st);
         case EPI_QKV: return tc_launch_bn<EPI_QKV>(enc, bn, g, rows_ub, st);
         default: return tc_launch_bn<EPI_F32>(enc, bn, g, rows_ub, st);

@@ -361,7 +361,7 @@ inline cudaError_t tc_pair_init() {
 
 // Worth it for wide weight matrices over many rows: the weight half of the ingest is what the pair saves.
 inline bool tc_pair_wanted(int epi, int N, int K, int rows_ub) {
-    if (epi != EPI_QKV && epi != EPI_RELU && epi != EPI_STORE && epi != EPI_STATS) return false;
+    if (epi != EPI_QKV && epi != EPI_RELU && epi != EPI_STORE && epi != EPI_STATS) return false;   // (the GELU variant stays on single-SM tiles)
     return rows_ub >= 4 * 2 * TC_BM && N >= 1024 && N % 128 == 0 && K % TC_BK == 0;
 }
 

@@ -164,7 +164,43 @@ __global__ void k_gather_rows(const float* __restrict__ x, const int* __restrict
     for (int e = threadIdx.x; e < d; e += blockDim.x) out[(size_t)row * d + e] = s[e];
 }
 
-// One warp per row; biased variance, eps inside the square root.  Rows of up to 512 elements
+// Register-resident row of up to NC * 128 elements (one warp per row).
+template <typename T, int NC>
+__device__ __forceinline__ void ln_row_regs(const float* __restrict__ xr, const float* __restrict__ g, const float* __restrict__ b,
+                                            T* __restrict__ y, int row, int d, float eps, int lane) {
+    float4 v[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const int e = lane * 4 + c * 128;
+        v[c] = e < d ? *reinterpret_cast<const float4*>(xr + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) s += v[c].x + v[c].y + v[c].z + v[c].w;
+    const float mu = warp_sum(s) / d;
+    float q = 0.f;
+#pragma unroll
+    for (int c = 0; c < NC; ++c)
+        if (lane * 4 + c * 128 < d) {
+            const float c0 = v[c].x - mu, c1 = v[c].y - mu, c2 = v[c].z - mu, c3 = v[c].w - mu;
+            q += c0 * c0 + c1 * c1 + c2 * c2 + c3 * c3;
+        }
+    const float rstd = 1.0f / sqrtf(warp_sum(q) / d + eps);
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const int e = lane * 4 + c * 128;
+        if (e < d) {
+            const float4 gm = *reinterpret_cast<const float4*>(g + e), bt = *reinterpret_cast<const float4*>(b + e);
+            T* o = y + (size_t)row * d + e;
+            o[0] = from_f<T>((v[c].x - mu) * rstd * gm.x + bt.x);
+            o[1] = from_f<T>((v[c].y - mu) * rstd * gm.y + bt.y);
+            o[2] = from_f<T>((v[c].z - mu) * rstd * gm.z + bt.z);
+            o[3] = from_f<T>((v[c].w - mu) * rstd * gm.w + bt.w);
+        }
+    }
+}
+
+// One warp per row; biased variance, eps inside the square root.  Rows of up to 1024 elements
 // (a multiple of 128) are held in registers, so the row is read from memory once.
 template <typename T>
 __global__ void k_layernorm(const float* __restrict__ x, const float* __restrict__ g, const float* __restrict__ b,
@@ -175,39 +211,8 @@ __global__ void k_layernorm(const float* __restrict__ x, const float* __restrict
     pdl_wait();
     if (row >= *n_rows) return;
     const float* xr = x + (size_t)row * d;
-    if (d % 128 == 0 && d <= 1024) {
-        float4 v[8];
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            const int e = lane * 4 + c * 128;
-            v[c] = e < d ? *reinterpret_cast<const float4*>(xr + e) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        float s = 0.f;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) s += v[c].x + v[c].y + v[c].z + v[c].w;
-        const float mu = warp_sum(s) / d;
-        float q = 0.f;
-#pragma unroll
-        for (int c = 0; c < 8; ++c)
-            if (lane * 4 + c * 128 < d) {
-                const float c0 = v[c].x - mu, c1 = v[c].y - mu, c2 = v[c].z - mu, c3 = v[c].w - mu;
-                q += c0 * c0 + c1 * c1 + c2 * c2 + c3 * c3;
-            }
-        const float rstd = 1.0f / sqrtf(warp_sum(q) / d + eps);
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            const int e = lane * 4 + c * 128;
-            if (e < d) {
-                const float4 gm = *reinterpret_cast<const float4*>(g + e), bt = *reinterpret_cast<const float4*>(b + e);
-                T* o = y + (size_t)row * d + e;
-                o[0] = from_f<T>((v[c].x - mu) * rstd * gm.x + bt.x);
-                o[1] = from_f<T>((v[c].y - mu) * rstd * gm.y + bt.y);
-                o[2] = from_f<T>((v[c].z - mu) * rstd * gm.z + bt.z);
-                o[3] = from_f<T>((v[c].w - mu) * rstd * gm.w + bt.w);
-            }
-        }
-        return;
-    }
+    if (d % 128 == 0 && d <= 512) { ln_row_regs<T, 4>(xr, g, b, y, row, d, eps, lane); return; }
+    if (d % 128 == 0 && d <= 1024) { ln_row_regs<T, 8>(xr, g, b, y, row, d, eps, lane); return; }
     float s = 0.f;
     for (int e = lane; e < d; e += 32) s += xr[e];
     float mu = warp_sum(s) / d;
@@ -300,7 +305,7 @@ __global__ void k_attention(AttnArgs<T> a) {
 
 // ------------------------------------------------------------------ GEMM epilogues
 // C[r, n] = sum_k A[r, k] * W[n, k]  (+ bias[n])
-enum { EPI_STORE = 0, EPI_RELU = 1, EPI_RESID = 2, EPI_STATS = 3, EPI_F32 = 4, EPI_QKV = 5 };   // EPI_RELU = the feed-forward activation
+enum { EPI_STORE = 0, EPI_RELU = 1, EPI_RESID = 2, EPI_STATS = 3, EPI_F32 = 4, EPI_QKV = 5, EPI_GELU = 6 };   // EPI_RELU / EPI_GELU = the feed-forward activation (separate kernels: erff costs registers)
 
 // Feed-forward activation of EPI_RELU: ReLU (act = 0) or the exact GELU x * Phi(x) (act = 1).
 __device__ __forceinline__ float ffn_act(float x, int act) {
@@ -321,6 +326,8 @@ struct GemmArgs {
     int one_m_tile;             // tensor-core path: the rows fit one 128-row tile whatever n_rows says
     T* out; int ldo;            // EPI_STORE / EPI_RELU
     int act;                    // EPI_RELU: 0 ReLU, 1 exact GELU
+    // EPI_RESID on the tensor-core path, optional: also write LayerNorm(new residual rows) as bf16 [rows, N]
+    const float* ln_g; const float* ln_b; float ln_eps; T* ln_out;
     float* resid;               // EPI_RESID: resid[r, n] += value ; EPI_F32: resid[r, n] = value (ld = N)
     // EPI_STATS
     RowPart* part; int n_tiles; // part[r * n_tiles + tile]

@@ -203,7 +203,8 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
         for (int s = 0; s < nsplit; ++s) v += red[(size_t)s * MT * 16 * SK_NB * G + o];
         v += bias_v;
         if (EPI == EPI_STORE) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(v);
-        if (EPI == EPI_RELU) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(ffn_act(v, g.act));
+        if (EPI == EPI_RELU) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(fmaxf(v, 0.f));
+        if (EPI == EPI_GELU) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(ffn_act(v, 1));
         if (EPI == EPI_RESID) g.resid[(size_t)r * N + n] += v;
         if (EPI == EPI_QKV) {
             if (n < g.kv_d) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(v);

@@ -97,6 +97,12 @@ struct specdec_handle {
     int poll_lag = -1;              // -1: chosen by batch size
     int use_fused_attn = 0;         // attention + output projection as one cluster kernel (measured slower: off)
     size_t attn_proj_smem_cap = 0;
+    // LayerNorm fused into the residual GEMM that feeds it (tensor-core path): what the next residual GEMM should
+    // also produce, and what the last one did produce
+    struct NextLn { const float* g; const float* b; void* out; };
+    NextLn next_ln = {nullptr, nullptr, nullptr};
+    const float* fused_x = nullptr; const float* fused_g = nullptr; const void* fused_out = nullptr;
+    int use_ln_fuse = 0;            // option "ln_fuse": measured slower than the separate LayerNorm launch, kept for comparison
     bool pair_ready = false;
     int use_pair = 0;               // two-SM tiles (cta_group::2) for wide GEMMs over many rows (option "pair")
     int attn_warps = 0;             // 0 = choose per launch, else 4 or 8 warps per tile-attention CTA (option "attn_warps")
@@ -349,6 +355,14 @@ int ln(specdec_handle* h, const float* x, const float* g, const float* b, int cn
     return 0;
 }
 
+// LayerNorm of rows x into y, unless the residual GEMM that produced x already wrote exactly that.
+template <typename T>
+int ln_or_fused(specdec_handle* h, const float* x, const float* g, const float* b, int cnt, int rows_ub, void* y, int d,
+                cudaStream_t st) {
+    if (x == h->fused_x && g == h->fused_g && y == h->fused_out) return 0;
+    return ln<T>(h, x, g, b, cnt, rows_ub, y, d, st);
+}
+
 // Where the K and V columns of a fused QKV projection go (the verifier's paged cache).
 struct KvDest { const int* seq; const int* pos; void* kc; void* vc; int d; };
 
@@ -366,7 +380,7 @@ constexpr int SK_ROWS_MAX = 32;
 template <typename T>
 bool skinny_ok(const specdec_handle* h, int epi, int rows_ub, int N, int K, bool with_ln) {
     if (!std::is_same<T, bf16>::value || !h->use_skinny || rows_ub > SK_ROWS_MAX) return false;
-    if (epi != EPI_STORE && epi != EPI_RELU && epi != EPI_RESID && epi != EPI_QKV) return false;
+    if (epi != EPI_STORE && epi != EPI_RELU && epi != EPI_GELU && epi != EPI_RESID && epi != EPI_QKV) return false;
     if (K % 32 || (with_ln && (K % 128 || K > 512))) return false;
     return skinny_smem(2, K) <= h->skinny_smem_cap;
 }
@@ -394,6 +408,7 @@ int skinny_launch(specdec_handle* h, int epi, SkinnyArgs& a, int rows_ub, cudaSt
     switch (epi) {
         case EPI_STORE: return skinny_launch_mt<EPI_STORE>(h, a, rows_ub, st);
         case EPI_RELU: return skinny_launch_mt<EPI_RELU>(h, a, rows_ub, st);
+        case EPI_GELU: return skinny_launch_mt<EPI_GELU>(h, a, rows_ub, st);
         case EPI_RESID: return skinny_launch_mt<EPI_RESID>(h, a, rows_ub, st);
         default: return skinny_launch_mt<EPI_QKV>(h, a, rows_ub, st);
     }
@@ -417,13 +432,16 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
     if (rows_ub <= 0) return 0;
     const bool skinny = skinny_ok<T>(h, epi, rows_ub, N, K, lnp != nullptr);
     if (lnp && !skinny) {                       // separate normalisation launch, then a plain GEMM on its output
-        TRY(ln<T>(h, lnp->x, lnp->g, lnp->b, cnt, rows_ub, h->y, K, st));
+        TRY(ln_or_fused<T>(h, lnp->x, lnp->g, lnp->b, cnt, rows_ub, h->y, K, st));
         A = h->y; lda = K;
     }
+    const specdec_handle::NextLn want_ln = h->next_ln;
+    if (epi == EPI_RESID) { h->fused_x = nullptr; h->next_ln = {nullptr, nullptr, nullptr}; }   // the residual rows change
     GemmArgs<T> g;
     g.A = (const T*)A; g.lda = lda; g.W = (const T*)W; g.bias = bias; g.N = N; g.K = K;
     g.n_rows = h->ses.counters + cnt; g.rows_static = (cnt == CNT_VERIFY || cnt == CNT_ENC) ? rows_ub : -1; g.out = (T*)out; g.ldo = ldo; g.resid = resid;
     g.one_m_tile = 0; g.act = h->cfg.ffn_activation;
+    g.ln_g = nullptr; g.ln_b = nullptr; g.ln_eps = 1e-5f; g.ln_out = nullptr;
     g.part = h->part; g.ld = ldv; g.ld_id = ld_id; g.n_tiles = cdiv(N, 64); g.want_sum = h->want_lse;
     g.seq = nullptr; g.pos = nullptr; g.kc = nullptr; g.vc = nullptr; g.kv_d = 0;
     g.pg.table = h->page_table; g.pg.page_tokens = h->cfg.page_tokens; g.pg.max_pages = h->pages_per_seq;
@@ -434,13 +452,21 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
             SkinnyArgs sa; sa.g = g;
             sa.ln_x = lnp ? lnp->x : nullptr; sa.ln_g = lnp ? lnp->g : nullptr; sa.ln_b = lnp ? lnp->b : nullptr;
             sa.ln_eps = 1e-5f; sa.ln_out = nullptr;
-            sa.trace = (h->want_cl_trace && h->cl_trace) ? h->cl_trace + 216 + 6 * (epi == EPI_RELU ? 0 : epi == EPI_RESID ? 1 : epi == EPI_QKV ? 2 : 3) : nullptr;
+            sa.trace = (h->want_cl_trace && h->cl_trace) ? h->cl_trace + 216 + 6 * ((epi == EPI_RELU || epi == EPI_GELU) ? 0 : epi == EPI_RESID ? 1 : epi == EPI_QKV ? 2 : 3) : nullptr;
             TRY(skinny_launch(h, epi, sa, rows_ub, st));
             return 0;
         }
     }
     if constexpr (std::is_same<T, bf16>::value) {
         if (h->use_tc && sd::tc_supported(N, K) && (epi != EPI_STATS || N >= 128)) {
+            if (epi == EPI_RESID && h->use_ln_fuse && want_ln.g && want_ln.out && sd::tc_ln_fusable(N, K)) {
+                g.ln_g = want_ln.g; g.ln_b = want_ln.b; g.ln_out = (T*)want_ln.out;
+                if (sd::gemm_tc_launch_ln(h->tma, g, rows_ub, st) != 0)
+                    return fail(h, SPECDEC_ERR_CUDA, "tensor-core GEMM launch failed: " + h->tma.err);
+                h->fused_x = resid; h->fused_g = want_ln.g; h->fused_out = want_ln.out;
+                ++h->launches;
+                return 0;
+            }
             int rc = (h->use_pair && sd::tc_pair_wanted(epi, N, K, rows_ub))
                          ? sd::gemm_tc_pair_launch(h->tma, epi, g, rows_ub, st, n_tiles_out)
                          : sd::gemm_tc_launch(h->tma, epi, g, rows_ub, st, n_tiles_out);
@@ -453,7 +479,7 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
     dim3 grid(cdiv(N, 64), cdiv(rows_ub, 64));
     switch (epi) {
         case EPI_STORE: k_gemm_simt<T, EPI_STORE><<<grid, 256, 0, st>>>(g); break;
-        case EPI_RELU: k_gemm_simt<T, EPI_RELU><<<grid, 256, 0, st>>>(g); break;
+        case EPI_RELU: case EPI_GELU: k_gemm_simt<T, EPI_RELU><<<grid, 256, 0, st>>>(g); break;   // activation chosen by g.act
         case EPI_RESID: k_gemm_simt<T, EPI_RESID><<<grid, 256, 0, st>>>(g); break;
         case EPI_STATS: k_gemm_simt<T, EPI_STATS><<<grid, 256, 0, st>>>(g); break;
         default: k_gemm_simt<T, EPI_F32><<<grid, 256, 0, st>>>(g); break;
@@ -560,6 +586,7 @@ int fused_attn_proj(specdec_handle* h, bool paged, const void* q, int q_stride, 
         cudaError_t e = paged ? cudaLaunchKernelEx(&cfg, k_attn_proj<true>, p) : cudaLaunchKernelEx(&cfg, k_attn_proj<false>, p);
         if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("attention+projection launch: ") + cudaGetErrorString(e));
         KCHECK(h);
+        h->fused_x = nullptr; h->next_ln = {nullptr, nullptr, nullptr};    // this kernel rewrote the residual rows
         return 1;
     }
 }
@@ -569,7 +596,8 @@ int fused_attn_proj(specdec_handle* h, bool paged, const void* q, int q_stride, 
 // from the paged cache after the block's K/V were scattered into it.
 template <typename T>
 int block_self(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, const Rows& r, int cnt, int rows_ub,
-               int q_ub, int layer, bool verify, int max_keys, cudaStream_t st) {
+               int q_ub, int layer, bool verify, int max_keys, cudaStream_t st, const float* next_g = nullptr,
+               const float* next_b = nullptr) {
     const int d = m.dm.d_model, H = m.dm.n_heads, dh = d / H;
     const size_t e = h->esz;
     const LnSpec l1{x, w.ln1_g, w.ln1_b};
@@ -599,6 +627,7 @@ int block_self(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, co
         TRY(attn<T>(h, false, h->qkv, 3 * d, nullptr, (char*)h->qkv + (size_t)d * e, (char*)h->qkv + (size_t)2 * d * e,
                     3 * d, r.kv_off, r, r.nk_self, cnt, rows_ub, q_ub, h->att, d, H, dh, max_keys, st));
     }
+    h->next_ln = {next_g, next_b, h->y};             // the LayerNorm that reads the residual stream next
     TRY(gemm<T>(h, EPI_RESID, h->att, d, w.o_w, w.o_b, d, d, cnt, rows_ub, nullptr, 0, x, st));
     return 0;
 }
@@ -619,16 +648,19 @@ int block_cross(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, c
     }
     TRY(attn<T>(h, false, h->q, d, nullptr, m.ckv[layer], (char*)m.ckv[layer] + (size_t)d * e, 2 * d, r.kv_off_cross,
                 r, r.nk_cross, cnt, rows_ub, q_ub, h->att, d, H, dh, h->S_max, st, h->ses.src_len));   // encoder K/V: all of it
+    h->next_ln = {w.ln2_g, w.ln2_b, h->y};           // the feed-forward sublayer's LayerNorm comes next
     TRY(gemm<T>(h, EPI_RESID, h->att, d, w.co_w, w.co_b, d, d, cnt, rows_ub, nullptr, 0, x, st));
     return 0;
 }
 
 template <typename T>
-int block_ffn(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, int cnt, int rows_ub, cudaStream_t st) {
+int block_ffn(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, int cnt, int rows_ub, cudaStream_t st,
+              const float* next_g = nullptr, const float* next_b = nullptr, void* next_out = nullptr) {
     const int d = m.dm.d_model, f = m.dm.d_ffn;
     const LnSpec l2{x, w.ln2_g, w.ln2_b};
-    TRY(gemm<T>(h, EPI_RELU, h->y, d, w.w1, w.b1, f, d, cnt, rows_ub, h->hbuf, f, nullptr, st, nullptr, nullptr, nullptr,
+    TRY(gemm<T>(h, h->cfg.ffn_activation == SPECDEC_ACT_GELU ? EPI_GELU : EPI_RELU, h->y, d, w.w1, w.b1, f, d, cnt, rows_ub, h->hbuf, f, nullptr, st, nullptr, nullptr, nullptr,
                 nullptr, &l2));
+    h->next_ln = {next_g, next_b, next_out ? next_out : h->y};
     TRY(gemm<T>(h, EPI_RESID, h->hbuf, f, w.w2, w.b2, d, f, cnt, rows_ub, nullptr, 0, x, st));
     return 0;
 }
@@ -638,6 +670,7 @@ int embed(specdec_handle* h, const ModelW& m, const Rows& r, const float* pos_ta
           cudaStream_t st) {
     if (rows_ub <= 0) return 0;
     const int d = m.dm.d_model;
+    h->fused_x = nullptr;                            // new residual rows: nothing normalised is pending
     k_embed<T><<<rows_ub, 128, 0, st>>>(r.tok, r.pos, h->ses.counters + cnt, (const T*)m.embed, pos_table, h->x, d,
                                         sqrtf((float)d), m.dm.vocab, m.dm.max_pos);
     KCHECK(h);
@@ -655,10 +688,12 @@ int encode_model(specdec_handle* h, ModelW& m, cudaStream_t st) {
     const int R = h->B * h->S_max, d = m.dm.d_model;
     TRY(embed<T>(h, m, h->rows, m.pos_enc, CNT_ENC, R, st));
     for (int l = 0; l < m.dm.enc_layers; ++l) {
-        TRY(block_self<T>(h, m, m.enc[l], h->x, h->rows, CNT_ENC, R, h->S_max, l, false, h->S_max, st));
-        TRY(block_ffn<T>(h, m, m.enc[l], h->x, CNT_ENC, R, st));
+        const bool last = l + 1 == m.dm.enc_layers;
+        TRY(block_self<T>(h, m, m.enc[l], h->x, h->rows, CNT_ENC, R, h->S_max, l, false, h->S_max, st, m.enc[l].ln2_g, m.enc[l].ln2_b));
+        TRY(block_ffn<T>(h, m, m.enc[l], h->x, CNT_ENC, R, st, last ? m.enc_lnf_g : m.enc[l + 1].ln1_g,
+                         last ? m.enc_lnf_b : m.enc[l + 1].ln1_b, last ? h->mem : nullptr));
     }
-    TRY(ln<T>(h, h->x, m.enc_lnf_g, m.enc_lnf_b, CNT_ENC, R, h->mem, d, st));
+    TRY(ln_or_fused<T>(h, h->x, m.enc_lnf_g, m.enc_lnf_b, CNT_ENC, R, h->mem, d, st));
     for (int l = 0; l < m.dm.dec_layers; ++l)
         TRY(gemm<T>(h, EPI_STORE, h->mem, d, m.dec[l].ckv_w, m.dec[l].ckv_b, 2 * d, d, CNT_ENC, R, m.ckv[l], 2 * d,
                     nullptr, st));
@@ -714,9 +749,9 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
     KCHECK(h);
     TRY(embed<T>(h, m, h->rows, m.pos_dec, CNT_DRAFT_ALL, R1, st));
     for (int l = 0; l + 1 < L; ++l) {
-        TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_DRAFT_ALL, R1, max_keys, l, false, max_keys, st));
+        TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_DRAFT_ALL, R1, max_keys, l, false, max_keys, st, m.dec[l].lnc_g, m.dec[l].lnc_b));
         TRY(block_cross<T>(h, m, m.dec[l], h->x, h->rows, CNT_DRAFT_ALL, R1, max_keys, l, st));
-        TRY(block_ffn<T>(h, m, m.dec[l], h->x, CNT_DRAFT_ALL, R1, st));
+        TRY(block_ffn<T>(h, m, m.dec[l], h->x, CNT_DRAFT_ALL, R1, st, m.dec[l + 1].ln1_g, m.dec[l + 1].ln1_b));
     }
     // last layer: K/V from every row, queries and everything after them from the k mask rows only
     const LayerW& w = m.dec[L - 1];
@@ -738,8 +773,8 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
         }
     }
     TRY(block_cross<T>(h, m, w, h->x2, h->mrows, CNT_DRAFT_MASK, R2, k, L - 1, st));
-    TRY(block_ffn<T>(h, m, w, h->x2, CNT_DRAFT_MASK, R2, st));
-    TRY(ln<T>(h, h->x2, m.dec_lnf_g, m.dec_lnf_b, CNT_DRAFT_MASK, R2, h->y, d, st));
+    TRY(block_ffn<T>(h, m, w, h->x2, CNT_DRAFT_MASK, R2, st, m.dec_lnf_g, m.dec_lnf_b));
+    TRY(ln_or_fused<T>(h, h->x2, m.dec_lnf_g, m.dec_lnf_b, CNT_DRAFT_MASK, R2, h->y, d, st));
     int n_tiles = 0;
     TRY(gemm<T>(h, EPI_STATS, h->y, d, m.embed, nullptr, m.dm.vocab, d, CNT_DRAFT_MASK, R2, nullptr, 0, nullptr, st,
                 nullptr, nullptr, &n_tiles));
@@ -799,11 +834,13 @@ int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float ta
         }
     }
     for (int l = 0; l < L && !clustered; ++l) {
-        TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, k + 1, l, true, max_keys, st));
+        const bool last = l + 1 == L;
+        TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, k + 1, l, true, max_keys, st, m.dec[l].lnc_g, m.dec[l].lnc_b));
         TRY(block_cross<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, k + 1, l, st));
-        TRY(block_ffn<T>(h, m, m.dec[l], h->x, CNT_VERIFY, M, st));
+        TRY(block_ffn<T>(h, m, m.dec[l], h->x, CNT_VERIFY, M, st, last ? m.dec_lnf_g : m.dec[l + 1].ln1_g,
+                         last ? m.dec_lnf_b : m.dec[l + 1].ln1_b));
     }
-    TRY(ln<T>(h, h->x, m.dec_lnf_g, m.dec_lnf_b, CNT_VERIFY, M, h->y, d, st));
+    TRY(ln_or_fused<T>(h, h->x, m.dec_lnf_g, m.dec_lnf_b, CNT_VERIFY, M, h->y, d, st));
     k_draft_logit<T><<<cdiv(M, 4), 128, 0, st>>>((const T*)h->y, (const T*)m.embed, h->v_draft, B, k, d, m.dm.vocab,
                                                  h->ld, h->ld_id);
     KCHECK(h);
@@ -859,7 +896,7 @@ void drop_graphs(specdec_handle* h) {
 // replayed afterwards.  The key must name everything the launches depend on besides device memory.
 template <typename F>
 int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body) {
-    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->use_pair); key.push_back(h->attn_warps); key.push_back(h->use_fused_attn); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
+    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->use_ln_fuse); key.push_back(h->use_pair); key.push_back(h->attn_warps); key.push_back(h->use_fused_attn); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
     key.push_back(h->B); key.push_back(h->S_max);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
@@ -1111,6 +1148,7 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
             const int kmax = std::max(h->d_max, h->f_max);
             size_t need = std::min<size_t>(skinny_smem(2, kmax), 227 * 1024);
             cudaError_t e = skinny_attr_mt<EPI_STORE>((int)need);
+            if (e == cudaSuccess) e = skinny_attr_mt<EPI_GELU>((int)need);
             if (e == cudaSuccess) e = skinny_attr_mt<EPI_RELU>((int)need);
             if (e == cudaSuccess) e = skinny_attr_mt<EPI_RESID>((int)need);
             if (e == cudaSuccess) e = skinny_attr_mt<EPI_QKV>((int)need);
@@ -1187,6 +1225,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
     if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "ln_fuse")) { h->use_ln_fuse = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "pair")) {
         if (value && !h->pair_ready) return fail(h, SPECDEC_ERR_UNSUPPORTED, "two-SM GEMM tiles are not available on this handle");
         h->use_pair = value ? 1 : 0; return SPECDEC_OK;

@@ -37,12 +37,14 @@ def _prefix_match(a, b):
 
 @pytest.mark.parametrize("batch,beta,tau,pair", [(32, 1, 0.0, 0), (32, 5, 3.0, 0), (128, 3, 1.0, 0), (128, 3, 1.0, 1)])
 def test_config3_batched_generate_sampled_sequences(base, batch, beta, tau, pair):
-    """pair = 1: the wide GEMMs over many rows (QKV, FFN1, vocabulary, encoder K/V) run as two-SM tiles."""
+    """pair = 1: the wide GEMMs over many rows (QKV, FFN1, vocabulary, encoder K/V) run as two-SM tiles, and every
+    LayerNorm is applied inside the residual GEMM before it (clusters of four CTAs per row tile)."""
     binding, wv, wd, mv, md = base
     wl = W.config3_batched(batch, beta, tau)
     smax, tmax = max(len(s) for s in wl.src), max(wl.max_tgt)
     sd = binding.SpecDec(W.BASE_V, wv, W.BASE_D, wd, k_max=25, max_batch=batch, max_src=smax, max_tgt=tmax, bf16=True)
     sd.set_option("pair", pair)
+    sd.set_option("ln_fuse", pair)
     src, lens = W.pad_batch(wl.src)
     out, n, st = sd.generate(src, lens, wl.max_tgt, 25, beta, tau)
     out, n = out.cpu().numpy(), n.cpu().numpy()

@@ -261,7 +261,7 @@ def test_bf16_mid_lockstep(gemm, attn):
     sd.close()
 
 
-@pytest.mark.parametrize("nseq,skinny", [(2, 1), (4, 1), (2, 0)])
+@pytest.mark.parametrize("nseq,skinny", [(2, 1), (4, 1), (2, 0), (4, 2)])
 def test_bf16_mid_small_batches_weight_streaming_gemm(nseq, skinny):
     """Passes of at most 32 rows run the weight-streaming GEMM with fused LayerNorm (26 rows: two 16-row
     tiles); 52 rows run one 128-row tile of the tensor-core GEMM with 64-wide column tiles."""
@@ -270,7 +270,8 @@ def test_bf16_mid_small_batches_weight_streaming_gemm(nseq, skinny):
     rng = np.random.default_rng(8)
     srcs = [W.zipf_ids(rng, n, 2000) for n in (20, 7, 33, 12)][:nseq]
     sd = _handle(MID_V, wv, MID_D, wd, True, k_max=12, max_batch=4, max_src=40, max_tgt=24)
-    sd.set_option("skinny", skinny)
+    sd.set_option("skinny", min(skinny, 1))
+    sd.set_option("ln_fuse", 1 if skinny == 2 else 0)      # 2: also fuse each LayerNorm into the residual GEMM before it
     rep = lockstep.run(sd, mv, md, srcs, [24, 18, 9, 20][:nseq], 12, 3, 1.0, margin=1e-3, check_logits_every=2)
     print(rep.iterations, rep.draft_near_ties, rep.verify_near_ties, rep.max_logit_err, rep.max_stat_err)
     assert rep.ok, rep.notes
