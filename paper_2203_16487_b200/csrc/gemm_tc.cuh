@@ -117,7 +117,9 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
 }
 
 __device__ __forceinline__ void tc_stamp(long long* trace, int slot) {
-    if (trace && blockIdx.x == 0) { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); trace[slot] = t; }
+    if (trace && blockIdx.x == 0 && (unsigned)slot < 56u) {          // the trace window holds 56 slots
+        long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); trace[slot] = t;
+    }
 }
 constexpr int TC_EPI_WARPS = 8;                      // two per TMEM lane quadrant: each takes half the columns
 constexpr int TC_THREADS = (2 + TC_EPI_WARPS) * 32;  // + TMA warp + MMA warp
