@@ -217,6 +217,8 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
  *   writes it (tensor-core path: the CTAs of a row tile form a cluster and exchange per-row sums through
  *   distributed shared memory; default 0: correct, but its longer single-tile tail costs more than the
  *   separate LayerNorm launch it removes: 743 vs 688 us per 128-sequence verify step);
+ * "attn_rs" = 0 never / 1 choose (default) / 2 whenever the keys allow: tile attention keeps the scores in the MMA
+ *   accumulators through the softmax instead of a shared-memory tile (smaller footprint, more CTAs per SM);
  * "attn_warps" = 0 choose per launch, 4 or 8 warps per CTA of the tile attention (default 0);
  * "tc_bn" = 0 choose, else force the column width of the tensor-core GEMM tiles (64 / 128 / 256; experiments);
  * "cluster" = 0/1 run the verifier's decoder stack as one thread-block-cluster kernel per sequence when the

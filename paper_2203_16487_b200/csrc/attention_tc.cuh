@@ -55,10 +55,19 @@ inline size_t attn_tc_smem(int max_keys) {
     const int nkp = (max_keys + 15) & ~15;
     return (size_t)ATT_Q * 128 + (size_t)nkp * 256 + (size_t)ATT_Q * (nkp + 4) * 4 + 16;
 }
+// RS ("register scores"): with at most ATT_RS_TILES 8-key tiles per warp the scores stay in the MMA accumulators
+// through the softmax, so shared memory holds Q, K and V only (a third less at 96 keys: more CTAs per SM).
+constexpr int ATT_RS_TILES = 6;
+inline int attn_tc_rs_max_keys(int warps) { return warps * ATT_RS_TILES * 8; }
+inline size_t attn_tc_smem_rs(int max_keys) {
+    const int nkp = (max_keys + 15) & ~15;
+    return (size_t)ATT_Q * 128 + (size_t)nkp * 256 + 16;
+}
 
-template <bool PAGED, int NW>
+template <bool PAGED, int NW, bool RS = false>
 __global__ void __launch_bounds__(NW * 32) k_attn_tc(AttnTcArgs a) {
     constexpr int ATT_THREADS = NW * 32;
+    __shared__ float s_wmax[RS ? NW * ATT_Q : 1], s_wsum[RS ? NW * ATT_Q : 1];   // RS: per-warp row maxima and sums
     extern __shared__ __align__(128) unsigned char sm[];
     __shared__ int s_nk[ATT_Q];
     __shared__ float s_sum[ATT_Q];
@@ -126,6 +135,95 @@ __global__ void __launch_bounds__(NW * 32) k_attn_tc(AttnTcArgs a) {
     __syncthreads();
 
     const int g = lane >> 2, t4 = lane & 3;
+    if constexpr (RS) {
+        // ---- S = scale * Q K^T in registers: warp w takes key tiles w, w + NW, ...
+        uint32_t qf[2][4][4];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                const int r = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = ks * 2 + (lane >> 4);
+                ldsm_x4(Qs + swz(r, c), qf[mt][ks][0], qf[mt][ks][1], qf[mt][ks][2], qf[mt][ks][3]);
+            }
+        float sc[2][ATT_RS_TILES][4];
+        float rmax[2][2] = {{-CUDART_INF_F, -CUDART_INF_F}, {-CUDART_INF_F, -CUDART_INF_F}};   // [mt][row g / row g + 8]
+        int nkr[2][2];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) { nkr[mt][0] = s_nk[mt * 16 + g]; nkr[mt][1] = s_nk[mt * 16 + g + 8]; }
+#pragma unroll
+        for (int j = 0; j < ATT_RS_TILES; ++j) {
+            const int nt = warp + j * NW;
+            if (nt < nkp / 8) {
+                uint32_t kf[2][4];
+#pragma unroll
+                for (int kk = 0; kk < 2; ++kk) {
+                    const int r = nt * 8 + (lane & 7), c = kk * 4 + (lane >> 3);
+                    ldsm_x4(Ks + swz(r, c), kf[kk][0], kf[kk][1], kf[kk][2], kf[kk][3]);
+                }
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) mma_bf16(acc, qf[mt][ks], kf[ks >> 1][(ks & 1) * 2], kf[ks >> 1][(ks & 1) * 2 + 1]);
+                    const int col = nt * 8 + t4 * 2;
+                    sc[mt][j][0] = (col < nkr[mt][0]) ? acc[0] * a.scale : -CUDART_INF_F;
+                    sc[mt][j][1] = (col + 1 < nkr[mt][0]) ? acc[1] * a.scale : -CUDART_INF_F;
+                    sc[mt][j][2] = (col < nkr[mt][1]) ? acc[2] * a.scale : -CUDART_INF_F;
+                    sc[mt][j][3] = (col + 1 < nkr[mt][1]) ? acc[3] * a.scale : -CUDART_INF_F;
+                    rmax[mt][0] = fmaxf(rmax[mt][0], fmaxf(sc[mt][j][0], sc[mt][j][1]));
+                    rmax[mt][1] = fmaxf(rmax[mt][1], fmaxf(sc[mt][j][2], sc[mt][j][3]));
+                }
+            } else {
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) sc[mt][j][e] = -CUDART_INF_F;
+            }
+        }
+        // row maximum: across the four lanes that share a row, then across warps through shared memory
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int hb = 0; hb < 2; ++hb) {
+                float m = rmax[mt][hb];
+                m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+                m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+                if (t4 == 0) s_wmax[warp * ATT_Q + mt * 16 + hb * 8 + g] = m;
+            }
+        __syncthreads();                              // every warp is also done reading K: P may overwrite it
+        bf16* P = reinterpret_cast<bf16*>(Kp);
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int hb = 0; hb < 2; ++hb) {
+                const int row = mt * 16 + hb * 8 + g;
+                float m = -CUDART_INF_F;
+#pragma unroll
+                for (int w = 0; w < NW; ++w) m = fmaxf(m, s_wmax[w * ATT_Q + row]);
+                float sum = 0.f;
+#pragma unroll
+                for (int j = 0; j < ATT_RS_TILES; ++j) {
+                    const int nt = warp + j * NW;
+                    if (nt < nkp / 8) {
+                        const float s0 = sc[mt][j][hb * 2], s1 = sc[mt][j][hb * 2 + 1];
+                        const float e0 = (s0 == -CUDART_INF_F) ? 0.f : expf(s0 - m), e1 = (s1 == -CUDART_INF_F) ? 0.f : expf(s1 - m);
+                        sum += e0 + e1;
+                        *reinterpret_cast<__nv_bfloat162*>(P + row * pstr + nt * 8 + t4 * 2) = __floats2bfloat162_rn(e0, e1);
+                    }
+                }
+                sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+                sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                if (t4 == 0) s_wsum[warp * ATT_Q + row] = sum;
+            }
+        __syncthreads();
+        if (tid < ATT_Q) {                            // normaliser of a row: the warps' sums in a fixed order
+            float t = 0.f;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) t += s_wsum[w * ATT_Q + tid];
+            s_sum[tid] = t;
+        }
+        __syncthreads();
+    } else {
     // ---- S = scale * Q K^T, masked
     {
         uint32_t qf[2][4][4];
@@ -179,6 +277,7 @@ __global__ void __launch_bounds__(NW * 32) k_attn_tc(AttnTcArgs a) {
         if (sub == 0) s_sum[r] = sum;
     }
     __syncthreads();
+    }
     // ---- O = P V ; warp w owns query rows 16 (w / (NW / 2)) .. and 128 / NW head columns
     {
         constexpr int WPM = NW / 2;                  // warps per 16-row query tile

@@ -105,6 +105,7 @@ struct specdec_handle {
     int use_ln_fuse = 0;            // option "ln_fuse": measured slower than the separate LayerNorm launch, kept for comparison
     bool pair_ready = false;
     int use_pair = 0;               // two-SM tiles (cta_group::2) for wide GEMMs over many rows (option "pair")
+    int attn_rs = 1;                // tile attention keeps the scores in registers when the keys allow (option "attn_rs")
     int attn_warps = 0;             // 0 = choose per launch, else 4 or 8 warps per tile-attention CTA (option "attn_warps")
     int skinny_groups = 1;          // 8-row weight groups per CTA of the weight-streaming GEMM (1, 2 or 4)
     // CUDA graphs of whole draft / verify(+commit) steps, keyed by everything their launches depend on
@@ -507,13 +508,29 @@ int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* 
             a.out = (bf16*)out; a.out_stride = out_stride; a.max_keys = max_keys;
             a.scale = 1.0f / sqrtf((float)d_head);
             dim3 grid(cdiv(q_ub, ATT_Q), n_heads, h->B);
-            // 4 warps when the SMs are saturated with CTAs anyway, 8 when a CTA's own latency chain is what counts
-            const long long ctas = (long long)grid.x * grid.y * grid.z, per_sm = (long long)(227 * 1024) / (long long)(smem + 1024);
-            const bool wide = h->attn_warps ? h->attn_warps == 8 : (per_sm <= 2 || ctas < 4LL * h->tma.n_sm);
-            cudaError_t e = wide ? (paged ? launch_pdl(h, k_attn_tc<true, 8>, grid, dim3(256), smem, st, a)
-                                          : launch_pdl(h, k_attn_tc<false, 8>, grid, dim3(256), smem, st, a))
-                                 : (paged ? launch_pdl(h, k_attn_tc<true, 4>, grid, dim3(128), smem, st, a)
-                                          : launch_pdl(h, k_attn_tc<false, 4>, grid, dim3(128), smem, st, a));
+            // 4 warps when the SMs are saturated with CTAs anyway, 8 when a CTA's own latency chain is what counts;
+            // scores stay in registers (smaller shared memory: more CTAs per SM) when the keys fit 6 tiles per warp
+            const long long ctas = (long long)grid.x * grid.y * grid.z;
+            const int nkp = (max_keys + 15) & ~15;
+            auto per_sm_of = [](size_t sm) { return (long long)(227 * 1024) / (long long)(sm + 1024); };
+            // (measured: the register variant is slower per CTA, 357 -> 387 us per batch-1 step, and pays off only where
+            // shared memory held the occupancy down: 1018 -> 873 us per step at batch 128 over a 256-token prefix)
+            bool rs = nkp <= attn_tc_rs_max_keys(8) &&
+                      (h->attn_rs == 2 || (h->attn_rs == 1 && per_sm_of(smem) <= 2 && ctas > 2LL * h->tma.n_sm));
+            size_t smem_l = rs ? attn_tc_smem_rs(max_keys) : smem;
+            bool wide = h->attn_warps ? h->attn_warps == 8 : (per_sm_of(smem_l) <= 2 || ctas < 4LL * h->tma.n_sm);
+            if (rs && !wide && nkp > attn_tc_rs_max_keys(4)) {       // too many keys for four warps' registers
+                if (h->attn_warps == 4) { rs = false; smem_l = smem; } else wide = true;
+            }
+            cudaError_t e;
+            if (rs) e = wide ? (paged ? launch_pdl(h, k_attn_tc<true, 8, true>, grid, dim3(256), smem_l, st, a)
+                                      : launch_pdl(h, k_attn_tc<false, 8, true>, grid, dim3(256), smem_l, st, a))
+                             : (paged ? launch_pdl(h, k_attn_tc<true, 4, true>, grid, dim3(128), smem_l, st, a)
+                                      : launch_pdl(h, k_attn_tc<false, 4, true>, grid, dim3(128), smem_l, st, a));
+            else e = wide ? (paged ? launch_pdl(h, k_attn_tc<true, 8>, grid, dim3(256), smem, st, a)
+                                   : launch_pdl(h, k_attn_tc<false, 8>, grid, dim3(256), smem, st, a))
+                          : (paged ? launch_pdl(h, k_attn_tc<true, 4>, grid, dim3(128), smem, st, a)
+                                   : launch_pdl(h, k_attn_tc<false, 4>, grid, dim3(128), smem, st, a));
             if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(e));
             KCHECK(h);
             return 0;
@@ -896,7 +913,7 @@ void drop_graphs(specdec_handle* h) {
 // replayed afterwards.  The key must name everything the launches depend on besides device memory.
 template <typename F>
 int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body) {
-    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->use_ln_fuse); key.push_back(h->use_pair); key.push_back(h->attn_warps); key.push_back(h->use_fused_attn); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
+    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->use_ln_fuse); key.push_back(h->use_pair); key.push_back(h->attn_warps); key.push_back(h->attn_rs); key.push_back(h->use_fused_attn); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
     key.push_back(h->B); key.push_back(h->S_max);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
@@ -1140,7 +1157,11 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
         if (cudaFuncSetAttribute(k_attn_tc<true, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
             cudaFuncSetAttribute(k_attn_tc<false, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
             cudaFuncSetAttribute(k_attn_tc<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
-            cudaFuncSetAttribute(k_attn_tc<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess) {
+            cudaFuncSetAttribute(k_attn_tc<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_tc<true, 8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_tc<false, 8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_tc<true, 4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
+            cudaFuncSetAttribute(k_attn_tc<false, 4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess) {
             cudaGetLastError();
             h->attn_tc_smem_cap = 48 * 1024;
         }
@@ -1230,6 +1251,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         if (value && !h->pair_ready) return fail(h, SPECDEC_ERR_UNSUPPORTED, "two-SM GEMM tiles are not available on this handle");
         h->use_pair = value ? 1 : 0; return SPECDEC_OK;
     }
+    if (!strcmp(name, "attn_rs")) { h->attn_rs = value < 0 ? 0 : (value > 2 ? 2 : value); return SPECDEC_OK; }   // 0 never, 1 choose, 2 whenever possible
     if (!strcmp(name, "attn_warps")) {
         if (value != 0 && value != 4 && value != 8) return fail(h, SPECDEC_ERR_INVALID_ARG, "attn_warps must be 0, 4 or 8");
         h->attn_warps = value; return SPECDEC_OK;

@@ -45,6 +45,7 @@ def test_config3_batched_generate_sampled_sequences(base, batch, beta, tau, pair
     sd = binding.SpecDec(W.BASE_V, wv, W.BASE_D, wd, k_max=25, max_batch=batch, max_src=smax, max_tgt=tmax, bf16=True)
     sd.set_option("pair", pair)
     sd.set_option("ln_fuse", pair)
+    sd.set_option("attn_rs", 2 if pair else 1)             # 2: attention scores stay in registers wherever the keys allow
     src, lens = W.pad_batch(wl.src)
     out, n, st = sd.generate(src, lens, wl.max_tgt, 25, beta, tau)
     out, n = out.cpu().numpy(), n.cpu().numpy()
