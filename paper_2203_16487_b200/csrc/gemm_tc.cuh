@@ -177,15 +177,13 @@ __device__ __forceinline__ void tc_st_peer2(uint32_t local_addr, uint32_t local_
 // half = which half of the tile's BN columns it takes; tmem_acc = the tile's accumulator.  Requests what it can
 // before waiting for the accumulator (residual tile, bias, cache rows, draft logits), then reads tensor memory
 // chunk by chunk.  The caller hands the accumulator back afterwards.
-// LNF (residual epilogue only): bias and residual are added while a thread still owns a whole row (so its sum and sum
-// of squares over the warp's columns need no shuffles), the pair is written into EVERY cluster peer's
-// ln_part[row][2 * rank + half], and the new residual values stay in `keep` for the fused LayerNorm that follows.
+// LNF (residual epilogue only): per row, the sum and sum of squares of the new residual values over the warp's columns
+// are written into EVERY cluster peer's ln_part[row][2 * rank + half] for the fused LayerNorm that follows.
 template <int EPI, int BN, bool LNF = false>
 __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R, int m0, int n_tile, int q, int half, int lane,
                                                  uint32_t tmem_acc, float* stg, uint32_t bar_acc_full_addr, uint32_t parity,
                                                  volatile int* abort_flag, int* err_word, bool later_tile,
-                                                 float* ln_part = nullptr, float4 (*keep)[8] = nullptr,
-                                                 const float* bias_s = nullptr, uint32_t ln_bar = 0) {
+                                                 float* ln_part = nullptr, uint32_t ln_bar = 0) {
     static_assert(!LNF || (EPI == EPI_RESID && BN <= 128 && BN % 64 == 0), "fused LayerNorm: residual epilogue, 64 or 128 columns");
     constexpr int HALF = BN / 2;                     // columns per epilogue warp
     constexpr int CW = HALF % 32 == 0 ? 32 : 16;     // columns per TMEM read
@@ -206,17 +204,15 @@ __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R,
             if (nb + CW <= g.N) {
 #pragma unroll
                 for (int ps = 0; ps < 8; ++ps) {
-                    if constexpr (LNF) {             // row layout: this thread's own row, columns 4 ps .. 4 ps + 3 of the chunk
-                        xin[c][ps] = r < R ? *reinterpret_cast<const float4*>(g.resid + (size_t)r * g.N + nb + ps * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-                    } else {
-                        const int gr = rbase + ps * 4 + (lane >> 3);
-                        xin[c][ps] = gr < R ? *reinterpret_cast<const float4*>(g.resid + (size_t)gr * g.N + nb + (lane & 7) * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
+                    const int gr = rbase + ps * 4 + (lane >> 3);
+                    xin[c][ps] = gr < R ? *reinterpret_cast<const float4*>(g.resid + (size_t)gr * g.N + nb + (lane & 7) * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
         }
     }
-    float ln_s1 = 0.f, ln_s2 = 0.f;                  // LNF: sum and sum of squares of this thread's row over the warp's columns
+    float ln_s1[8], ln_s2[8];                        // LNF: per pass, sum and sum of squares of row 4 ps + lane / 8 over this lane's columns
+#pragma unroll
+    for (int ps = 0; ps < 8; ++ps) { ln_s1[ps] = 0.f; ln_s2[ps] = 0.f; }
     // ... and so are this lane's bias columns, its cache row and its draft logit
     float4 bzv[NCH][2];
     if (EPI != EPI_STATS && vec_ok && g.bias) {
@@ -282,16 +278,6 @@ __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R,
                 }
             }
             tmem_ld<CW>(trow + c * CW, v);
-            if constexpr (LNF) {
-#pragma unroll
-                for (int j4 = 0; j4 < 8; ++j4) {
-                    const float4 bz = *reinterpret_cast<const float4*>(bias_s + half * HALF + c * CW + j4 * 4);   // staged at set-up
-                    const float4 x = xin[c & 1][j4];
-                    v[j4 * 4] += bz.x + x.x; v[j4 * 4 + 1] += bz.y + x.y; v[j4 * 4 + 2] += bz.z + x.z; v[j4 * 4 + 3] += bz.w + x.w;
-                    ln_s1 += (v[j4 * 4] + v[j4 * 4 + 1]) + (v[j4 * 4 + 2] + v[j4 * 4 + 3]);
-                    ln_s2 += (v[j4 * 4] * v[j4 * 4] + v[j4 * 4 + 1] * v[j4 * 4 + 1]) + (v[j4 * 4 + 2] * v[j4 * 4 + 2] + v[j4 * 4 + 3] * v[j4 * 4 + 3]);
-                }
-            }
             if (CW == 32 && vec_ok && nb + CW <= g.N) {
                 // Transpose through shared memory: a thread owns one output ROW in tensor memory, but global
                 // memory wants neighbouring lanes on neighbouring addresses.  The 32 x 32 block is written row-wise
@@ -309,12 +295,13 @@ __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R,
                     for (int ps = 0; ps < 8; ++ps) {
                         const int rr = ps * 4 + rsub, gr = rbase + rr;
                         float4 a = *reinterpret_cast<const float4*>(stg + rr * 32 + ((l8 ^ (rr & 7)) << 2));
-                        if constexpr (!LNF) {
-                            a.x += bz.x; a.y += bz.y; a.z += bz.z; a.w += bz.w;
-                            if (EPI == EPI_RESID) { const float4 x = xin[c & 1][ps]; a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w; }
-                        }
+                        a.x += bz.x; a.y += bz.y; a.z += bz.z; a.w += bz.w;
+                        if (EPI == EPI_RESID) { const float4 x = xin[c & 1][ps]; a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w; }
                         if (gr < R) *reinterpret_cast<float4*>(g.resid + (size_t)gr * g.N + nb + l8 * 4) = a;
-                        if constexpr (LNF) keep[c][ps] = a;
+                        if constexpr (LNF) {
+                            ln_s1[ps] += (a.x + a.y) + (a.z + a.w);
+                            ln_s2[ps] += (a.x * a.x + a.y * a.y) + (a.z * a.z + a.w * a.w);
+                        }
                     }
                 } else {
                     // bf16 rows: 4 lanes per row (8 columns = 16 bytes each), 8 rows per pass
@@ -380,10 +367,19 @@ __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R,
             }
         }
     }
-    if constexpr (LNF) {                             // this row's partial statistics into every peer's table; every warp
+    if constexpr (LNF) {                             // each row's partial statistics into every peer's table; every warp
         const uint32_t nct = tc_cluster_nctas();     // sends (rows past the end send what they have) so the byte count is fixed
-        const uint32_t slot = smem_u32(ln_part + ((q * 32 + lane) * 16 + n_tile * 2 + half) * 2);
-        for (uint32_t rk = 0; rk < nct; ++rk) tc_st_peer2(slot, ln_bar, rk, ln_s1, ln_s2);
+#pragma unroll
+        for (int ps = 0; ps < 8; ++ps) {
+            float s1 = ln_s1[ps], s2 = ln_s2[ps];
+#pragma unroll
+            for (int o = 1; o < 8; o <<= 1) { s1 += __shfl_xor_sync(0xffffffffu, s1, o); s2 += __shfl_xor_sync(0xffffffffu, s2, o); }
+            if ((lane & 7) == 0) {
+                const int rr = ps * 4 + (lane >> 3);
+                const uint32_t slot = smem_u32(ln_part + ((q * 32 + rr) * 16 + n_tile * 2 + half) * 2);
+                for (uint32_t rk = 0; rk < nct; ++rk) tc_st_peer2(slot, ln_bar, rk, s1, s2);
+            }
+        }
     }
     tc_fence_before();
     __syncwarp();
@@ -422,9 +418,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     __shared__ int abort_s;
     __shared__ __align__(16) float ln_part_s[LNF ? TC_BM * 32 : 1];  // [row][2 * cluster rank + column half][sum, sum of squares]
     __shared__ float ln_mr_s[LNF ? TC_BM * 2 : 1];                   // [row][mean, 1 / std]
-    __shared__ __align__(16) float bias_s[LNF ? BN : 1];             // LNF: this tile's bias columns
     __shared__ __align__(8) uint64_t bar_ln;                         // LNF: counts the peers' statistics as they arrive
-    float4 keep[2][8];                                               // LNF: this thread's new residual values
     const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb = g.K / TC_BK;
@@ -440,12 +434,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     }
     if (warp == 1) { tmem_alloc(smem_u32(&tmem_base_s), Cfg::TMEM_COLS); if (lane == 0) tc_stamp(g.trace, 13); }
     if constexpr (LNF) {
-        const int nt0 = ((int)blockIdx.x % n_tiles) * BN;
-        for (int i = threadIdx.x; i < BN; i += TC_THREADS) bias_s[i] = g.bias ? __ldg(g.bias + nt0 + i) : 0.f;   // a weight: before the wait
         if (threadIdx.x == 0) {
             mbar_init(smem_u32(&bar_ln), 1);
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-            mbar_expect_tx(smem_u32(&bar_ln), tc_cluster_nctas() * TC_EPI_WARPS * 32 * 8);   // 8 bytes from every epilogue thread of every peer
+            mbar_expect_tx(smem_u32(&bar_ln), tc_cluster_nctas() * TC_BM * 2 * 8);   // 8 bytes per row and column half from every peer
         }
         tc_fence_before();
         tc_cluster_sync();                           // peers' barriers exist before anybody sends (all of this precedes the dependency wait)
@@ -535,7 +527,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             const int ab = i & 1;
             const int m0 = (LNF ? t / n_tiles : t % m_tiles) * TC_BM, n_tile = LNF ? t % n_tiles : t / m_tiles;
             tc_epilogue_tile<EPI, BN, LNF>(g, R, m0, n_tile, q, half, lane, tmem_d + ab * BN, stg, smem_u32(&bar_acc_full[ab]),
-                                           (i >> 1) & 1, abort_flag, err_word, i > 0, ln_part_s, keep, bias_s, smem_u32(&bar_ln));
+                                           (i >> 1) & 1, abort_flag, err_word, i > 0, ln_part_s, smem_u32(&bar_ln));
             // this warp is done with the accumulator: hand it back to the MMA warp
             if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[ab]));
             if (threadIdx.x == 64) tc_stamp(g.trace, 8 + 2 * (i > 0));
@@ -569,8 +561,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     for (int ps = 0; ps < 8; ++ps) {
                         const int rr = ps * 4 + rsub, gr = rbase + rr;
                         const float mu = ln_mr_s[(q * 32 + rr) * 2], rstd = ln_mr_s[(q * 32 + rr) * 2 + 1];
-                        const float4 a = keep[c][ps];
                         if (gr < R) {
+                            const float4 a = *reinterpret_cast<const float4*>(g.resid + (size_t)gr * g.N + nb + l8 * 4);   // written by this thread above
                             __nv_bfloat162 p0 = __floats2bfloat162_rn((a.x - mu) * rstd * gm.x + bt.x, (a.y - mu) * rstd * gm.y + bt.y);
                             __nv_bfloat162 p1 = __floats2bfloat162_rn((a.z - mu) * rstd * gm.z + bt.z, (a.w - mu) * rstd * gm.w + bt.w);
                             uint2 pk; pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
