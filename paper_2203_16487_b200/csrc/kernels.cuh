@@ -164,9 +164,10 @@ __global__ void k_gather_rows(const float* __restrict__ x, const int* __restrict
     for (int e = threadIdx.x; e < d; e += blockDim.x) out[(size_t)row * d + e] = s[e];
 }
 
-// Register-resident row of up to NC * 128 elements (one warp per row).
+// Register-resident row of up to NC * 128 elements (one warp per row).  gm / bt = this lane's gain and bias columns,
+// fetched by the caller before the dependency wait (they are weights).
 template <typename T, int NC>
-__device__ __forceinline__ void ln_row_regs(const float* __restrict__ xr, const float* __restrict__ g, const float* __restrict__ b,
+__device__ __forceinline__ void ln_row_regs(const float* __restrict__ xr, const float4* gm, const float4* bt,
                                             T* __restrict__ y, int row, int d, float eps, int lane) {
     float4 v[NC];
 #pragma unroll
@@ -190,12 +191,11 @@ __device__ __forceinline__ void ln_row_regs(const float* __restrict__ xr, const 
     for (int c = 0; c < NC; ++c) {
         const int e = lane * 4 + c * 128;
         if (e < d) {
-            const float4 gm = *reinterpret_cast<const float4*>(g + e), bt = *reinterpret_cast<const float4*>(b + e);
             T* o = y + (size_t)row * d + e;
-            o[0] = from_f<T>((v[c].x - mu) * rstd * gm.x + bt.x);
-            o[1] = from_f<T>((v[c].y - mu) * rstd * gm.y + bt.y);
-            o[2] = from_f<T>((v[c].z - mu) * rstd * gm.z + bt.z);
-            o[3] = from_f<T>((v[c].w - mu) * rstd * gm.w + bt.w);
+            o[0] = from_f<T>((v[c].x - mu) * rstd * gm[c].x + bt[c].x);
+            o[1] = from_f<T>((v[c].y - mu) * rstd * gm[c].y + bt[c].y);
+            o[2] = from_f<T>((v[c].z - mu) * rstd * gm[c].z + bt[c].z);
+            o[3] = from_f<T>((v[c].w - mu) * rstd * gm[c].w + bt[c].w);
         }
     }
 }
@@ -207,12 +207,24 @@ __global__ void k_layernorm(const float* __restrict__ x, const float* __restrict
                             const int* __restrict__ n_rows, T* __restrict__ y, int d, float eps) {
     int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     int lane = threadIdx.x & 31;
+    const bool regs4 = d % 128 == 0 && d <= 512, regs8 = d % 128 == 0 && d <= 1024;
+    float4 gm[8], bt[8];                             // gain and bias are weights: fetched before the dependency wait
+    if (regs8) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const int e = lane * 4 + c * 128;
+            if (c < 4 || !regs4) {
+                gm[c] = e < d ? __ldg(reinterpret_cast<const float4*>(g + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                bt[c] = e < d ? __ldg(reinterpret_cast<const float4*>(b + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+    }
     pdl_launch_dependents();
     pdl_wait();
     if (row >= *n_rows) return;
     const float* xr = x + (size_t)row * d;
-    if (d % 128 == 0 && d <= 512) { ln_row_regs<T, 4>(xr, g, b, y, row, d, eps, lane); return; }
-    if (d % 128 == 0 && d <= 1024) { ln_row_regs<T, 8>(xr, g, b, y, row, d, eps, lane); return; }
+    if (regs4) { ln_row_regs<T, 4>(xr, gm, bt, y, row, d, eps, lane); return; }
+    if (regs8) { ln_row_regs<T, 8>(xr, gm, bt, y, row, d, eps, lane); return; }
     float s = 0.f;
     for (int e = lane; e < d; e += 32) s += xr[e];
     float mu = warp_sum(s) / d;
