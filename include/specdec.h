@@ -217,6 +217,10 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
  *   writes it (tensor-core path: the CTAs of a row tile form a cluster and exchange per-row sums through
  *   distributed shared memory; default 0: correct, but its longer single-tile tail costs more than the
  *   separate LayerNorm launch it removes: 743 vs 688 us per 128-sequence verify step);
+ * "ln_rows" = 0/1 tensor-core GEMMs over at most 128 rows normalise their input rows themselves (eight warps write
+ *   the bf16 operand tile in the tensor core's swizzled layout) instead of reading the output of a LayerNorm launch
+ *   (default 0: correct, but every CTA repeating the normalisation costs more than the launch: 407 vs 358 us per
+ *   2-sequence verify step, 491 vs 377 us at 4 sequences);
  * "attn_rs" = 0 never / 1 choose (default) / 2 whenever the keys allow: tile attention keeps the scores in the MMA
  *   accumulators through the softmax instead of a shared-memory tile (smaller footprint, more CTAs per SM);
  * "attn_warps" = 0 choose per launch, 4 or 8 warps per CTA of the tile attention (default 0);

@@ -18,6 +18,7 @@
 #include "attention_tc.cuh"
 #include "decoder_cluster.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_tc_lnrows.cuh"
 #include "gemm_tc_pair.cuh"
 #include "kernels.cuh"
 #include "skinny_gemm.cuh"
@@ -103,6 +104,8 @@ struct specdec_handle {
     NextLn next_ln = {nullptr, nullptr, nullptr};
     const float* fused_x = nullptr; const float* fused_g = nullptr; const void* fused_out = nullptr;
     int use_ln_fuse = 0;            // option "ln_fuse": measured slower than the separate LayerNorm launch, kept for comparison
+    bool lnrows_ready = false;
+    int use_ln_rows = 0;            // option "ln_rows": GEMMs over at most 128 rows normalise their input rows themselves (measured slower: off)
     bool pair_ready = false;
     int use_pair = 0;               // two-SM tiles (cta_group::2) for wide GEMMs over many rows (option "pair")
     int attn_rs = 1;                // tile attention keeps the scores in registers when the keys allow (option "attn_rs")
@@ -432,7 +435,12 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
          const LnSpec* lnp = nullptr) {
     if (rows_ub <= 0) return 0;
     const bool skinny = skinny_ok<T>(h, epi, rows_ub, N, K, lnp != nullptr);
-    if (lnp && !skinny) {                       // separate normalisation launch, then a plain GEMM on its output
+    // At most 128 rows on the tensor-core path: the GEMM normalises its input rows itself (gemm_tc_lnrows.cuh)
+    bool ln_rows = false;
+    if constexpr (std::is_same<T, bf16>::value)
+        ln_rows = lnp && !skinny && h->use_tc && h->lnrows_ready && h->use_ln_rows && sd::lr_supported(epi, N, K, rows_ub) &&
+                  !(lnp->x == h->fused_x && lnp->g == h->fused_g && h->y == h->fused_out);
+    if (lnp && !skinny && !ln_rows) {           // separate normalisation launch, then a plain GEMM on its output
         TRY(ln_or_fused<T>(h, lnp->x, lnp->g, lnp->b, cnt, rows_ub, h->y, K, st));
         A = h->y; lda = K;
     }
@@ -459,6 +467,13 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
         }
     }
     if constexpr (std::is_same<T, bf16>::value) {
+        if (ln_rows) {
+            sd::LnRowsArgs la{lnp->x, lnp->g, lnp->b, 1e-5f};
+            if (sd::lr_launch(h->tma, epi, g, la, st) != 0)
+                return fail(h, SPECDEC_ERR_CUDA, "tensor-core GEMM launch failed: " + h->tma.err);
+            ++h->launches;
+            return 0;
+        }
         if (h->use_tc && sd::tc_supported(N, K) && (epi != EPI_STATS || N >= 128)) {
             if (epi == EPI_RESID && h->use_ln_fuse && want_ln.g && want_ln.out && sd::tc_ln_fusable(N, K)) {
                 g.ln_g = want_ln.g; g.ln_b = want_ln.b; g.ln_out = (T*)want_ln.out;
@@ -913,7 +928,7 @@ void drop_graphs(specdec_handle* h) {
 // replayed afterwards.  The key must name everything the launches depend on besides device memory.
 template <typename F>
 int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body) {
-    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->use_ln_fuse); key.push_back(h->use_pair); key.push_back(h->attn_warps); key.push_back(h->attn_rs); key.push_back(h->use_fused_attn); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
+    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->use_ln_fuse); key.push_back(h->use_ln_rows); key.push_back(h->use_pair); key.push_back(h->attn_warps); key.push_back(h->attn_rs); key.push_back(h->use_fused_attn); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
     key.push_back(h->B); key.push_back(h->S_max);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
@@ -1202,6 +1217,8 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
             h->attn_proj_smem_cap = cap;
         }
         if (sd::tc_init(h->tma, h->ses.counters + 7) != 0) h->use_tc = 0;     // reported through specdec_last_error; SIMT GEMM still runs on the GPU
+        h->lnrows_ready = h->use_tc && sd::lr_init() == cudaSuccess;
+        if (!h->lnrows_ready) cudaGetLastError();
         h->pair_ready = h->use_tc && sd::tc_pair_init() == cudaSuccess;
         if (!h->pair_ready) cudaGetLastError();
         if (!h->use_tc) h->err = "tensor-core GEMM unavailable: " + h->tma.err;
@@ -1246,6 +1263,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
     if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "ln_rows")) { h->use_ln_rows = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "ln_fuse")) { h->use_ln_fuse = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "pair")) {
         if (value && !h->pair_ready) return fail(h, SPECDEC_ERR_UNSUPPORTED, "two-SM GEMM tiles are not available on this handle");

@@ -273,6 +273,7 @@ def test_bf16_mid_small_batches_weight_streaming_gemm(nseq, skinny):
     sd.set_option("skinny", min(skinny, 1))
     sd.set_option("ln_fuse", 1 if skinny == 2 else 0)      # 2: also fuse each LayerNorm into the residual GEMM before it
     sd.set_option("attn_rs", 2 if skinny == 2 else 1)      # ... and keep attention scores in registers wherever possible
+    sd.set_option("ln_rows", 1 if skinny in (0, 2) else 0) # 0 / 2: GEMMs over at most 128 rows normalise their own input rows
     rep = lockstep.run(sd, mv, md, srcs, [24, 18, 9, 20][:nseq], 12, 3, 1.0, margin=1e-3, check_logits_every=2)
     print(rep.iterations, rep.draft_near_ties, rep.verify_near_ties, rep.max_logit_err, rep.max_stat_err)
     assert rep.ok, rep.notes
