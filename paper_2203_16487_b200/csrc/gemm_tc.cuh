@@ -766,6 +766,7 @@ inline int gemm_tc_launch(TmaEncoder& enc, int epi, GemmArgs<bf16>& g, int rows_
     const int fb = enc.force_bn;
     const bool forced = (fb == 32 || fb == 64 || fb == 128 || fb == 192 || fb == 256) && fb <= g.N;
     const int bn = forced ? fb : tc_pick_bn(g.N, rows_ub, enc.n_sm);
+    g.one_m_tile = rows_ub <= TC_BM;        // one row tile whatever the device-side count says: set up and prefetch before the wait
     switch (epi) {
         case EPI_STORE: return tc_launch_bn<EPI_STORE>(enc, bn, g, rows_ub, st);
         case EPI_RELU: return tc_launch_bn<EPI_RELU>(enc, bn, g, rows_ub, st);
