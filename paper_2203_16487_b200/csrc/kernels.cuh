@@ -150,6 +150,8 @@ __global__ void k_embed(const int* __restrict__ tok, const int* __restrict__ pos
                         const T* __restrict__ E, const float* __restrict__ P, float* __restrict__ x, int d,
                         float scale, int vocab, int max_pos) {
     int row = blockIdx.x;
+    pdl_launch_dependents();                       // writes x only, which every successor reads after its own wait
+    pdl_wait();
     if (row >= *n_rows) return;
     int t = min(max(tok[row], 0), vocab - 1), p = min(max(pos[row], 0), max_pos - 1);
     for (int e = threadIdx.x; e < d; e += blockDim.x)
@@ -159,6 +161,8 @@ __global__ void k_embed(const int* __restrict__ tok, const int* __restrict__ pos
 __global__ void k_gather_rows(const float* __restrict__ x, const int* __restrict__ src_row,
                               const int* __restrict__ n_rows, float* __restrict__ out, int d) {
     int row = blockIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
     if (row >= *n_rows) return;
     const float* s = x + (size_t)src_row[row] * d;
     for (int e = threadIdx.x; e < d; e += blockDim.x) out[(size_t)row * d + e] = s[e];
@@ -460,6 +464,8 @@ __global__ void k_draft_logit(const T* __restrict__ y, const T* __restrict__ E, 
                               int B, int k, int d, int vocab, float* __restrict__ ld, int* __restrict__ ld_id) {
     int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     int lane = threadIdx.x & 31;
+    pdl_launch_dependents();
+    pdl_wait();
     if (row >= B * (k + 1)) return;
     int b = row / (k + 1), c = row % (k + 1);
     if (c == k) { if (lane == 0) { ld[row] = CUDART_INF_F; ld_id[row] = -1; } return; }
@@ -480,6 +486,8 @@ __global__ void k_accept(const RowPart* __restrict__ part, int n_tiles, const fl
     extern __shared__ unsigned char sm_acc[];
     RowPart* rs = reinterpret_cast<RowPart*>(sm_acc);       // [k+1]
     const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    pdl_launch_dependents();
+    pdl_wait();
     for (int c = warp; c <= k; c += nw) {
         const RowPart* p = part + ((size_t)b * (k + 1) + c) * n_tiles;
         RowPart m; m.mx = -CUDART_INF_F; m.arg = 0x7fffffff; m.sum = 0.f; m.cnt = 0;
@@ -602,6 +610,8 @@ __global__ void k_draft_argmax(const RowPart* __restrict__ part, int n_tiles, co
                                const int* __restrict__ slot, int* __restrict__ draft) {
     int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     int lane = threadIdx.x & 31;
+    pdl_launch_dependents();
+    pdl_wait();
     if (row >= *n_rows) return;
     const RowPart* p = part + (size_t)row * n_tiles;
     float mx = -CUDART_INF_F; int arg = 0x7fffffff;
@@ -623,6 +633,7 @@ __global__ void k_draft_argmax(const RowPart* __restrict__ part, int n_tiles, co
 __global__ void k_apply_script(Session s, const int* __restrict__ script, int stride, int B, int k,
                                int* __restrict__ draft) {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_wait();
     if (i >= B * k) return;
     int b = i / k, c = i % k;
     if (s.finished[b]) return;
@@ -636,6 +647,7 @@ __global__ void k_apply_script(Session s, const int* __restrict__ script, int st
 __global__ void k_commit(Session s, const int* __restrict__ draft, const int* __restrict__ keep,
                          const int* __restrict__ next, int B, int k, int eos) {
     int b = blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_wait();                                    // no early trigger: the lengths written here are read by later kernels BEFORE their waits
     if (b >= B || s.finished[b]) return;
     int j = s.len[b];
     const int mt = s.max_tgt[b];

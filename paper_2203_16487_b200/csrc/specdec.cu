@@ -703,8 +703,8 @@ int embed(specdec_handle* h, const ModelW& m, const Rows& r, const float* pos_ta
     if (rows_ub <= 0) return 0;
     const int d = m.dm.d_model;
     h->fused_x = nullptr;                            // new residual rows: nothing normalised is pending
-    k_embed<T><<<rows_ub, 128, 0, st>>>(r.tok, r.pos, h->ses.counters + cnt, (const T*)m.embed, pos_table, h->x, d,
-                                        sqrtf((float)d), m.dm.vocab, m.dm.max_pos);
+    CUDA_TRY(h, launch_pdl(h, k_embed<T>, dim3(rows_ub), dim3(128), 0, st, (const int*)r.tok, (const int*)r.pos, (const int*)(h->ses.counters + cnt), (const T*)m.embed, (const float*)pos_table, h->x, d,
+                                        sqrtf((float)d), m.dm.vocab, m.dm.max_pos));
     KCHECK(h);
     return 0;
 }
@@ -790,7 +790,7 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
     const LnSpec l1{h->x, w.ln1_g, w.ln1_b};
     TRY(gemm<T>(h, EPI_STORE, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, CNT_DRAFT_ALL, R1, h->qkv, 3 * d, nullptr, st, nullptr,
                 nullptr, nullptr, nullptr, &l1));
-    k_gather_rows<<<R2, 128, 0, st>>>(h->x, h->mrows.src_row, h->ses.counters + CNT_DRAFT_MASK, h->x2, d);
+    CUDA_TRY(h, launch_pdl(h, k_gather_rows, dim3(R2), dim3(128), 0, st, (const float*)h->x, (const int*)h->mrows.src_row, (const int*)(h->ses.counters + CNT_DRAFT_MASK), h->x2, d));
     KCHECK(h);
     {
         const int f = fused_attn_proj<T>(h, false, h->qkv, 3 * d, h->mrows.src_row, (char*)h->qkv + (size_t)d * e,
@@ -810,11 +810,11 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
     int n_tiles = 0;
     TRY(gemm<T>(h, EPI_STATS, h->y, d, m.embed, nullptr, m.dm.vocab, d, CNT_DRAFT_MASK, R2, nullptr, 0, nullptr, st,
                 nullptr, nullptr, &n_tiles));
-    k_draft_argmax<<<cdiv(R2, 4), 128, 0, st>>>(h->part, n_tiles, h->ses.counters + CNT_DRAFT_MASK, h->mrows.slot,
-                                               d_draft);
+    CUDA_TRY(h, launch_pdl(h, k_draft_argmax, dim3(cdiv(R2, 4)), dim3(128), 0, st, (const RowPart*)h->part, n_tiles,
+                           (const int*)(h->ses.counters + CNT_DRAFT_MASK), (const int*)h->mrows.slot, d_draft));
     KCHECK(h);
     if (h->script_on) {
-        k_apply_script<<<cdiv(B * k, 256), 256, 0, st>>>(h->ses, h->script, h->T_cap + h->k_cap, B, k, d_draft);
+        CUDA_TRY(h, launch_pdl(h, k_apply_script, dim3(cdiv(B * k, 256)), dim3(256), 0, st, h->ses, (const int*)h->script, h->T_cap + h->k_cap, B, k, d_draft));
         KCHECK(h);
     }
     h->drafted = true; h->verified = false;
@@ -873,16 +873,16 @@ int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float ta
                          last ? m.dec_lnf_b : m.dec[l + 1].ln1_b));
     }
     TRY(ln_or_fused<T>(h, h->x, m.dec_lnf_g, m.dec_lnf_b, CNT_VERIFY, M, h->y, d, st));
-    k_draft_logit<T><<<cdiv(M, 4), 128, 0, st>>>((const T*)h->y, (const T*)m.embed, h->v_draft, B, k, d, m.dm.vocab,
-                                                 h->ld, h->ld_id);
+    CUDA_TRY(h, launch_pdl(h, k_draft_logit<T>, dim3(cdiv(M, 4)), dim3(128), 0, st, (const T*)h->y, (const T*)m.embed,
+                           (const int*)h->v_draft, B, k, d, m.dm.vocab, h->ld, h->ld_id));
     KCHECK(h);
     int n_tiles = 0;
     prof_mark(h, st);
     TRY(gemm<T>(h, EPI_STATS, h->y, d, m.embed, nullptr, m.dm.vocab, d, CNT_VERIFY, M, nullptr, 0, nullptr, st, h->ld,
                 h->ld_id, &n_tiles));
     prof_mark(h, st);
-    k_accept<<<B, 1024, (size_t)(k + 1) * sizeof(RowPart), st>>>(h->part, n_tiles, h->ld, h->ld_id, k, beta, tau,
-                                                                 h->accepted, h->bif, h->row_stats, h->want_lse);
+    CUDA_TRY(h, launch_pdl(h, k_accept, dim3(B), dim3(1024), (size_t)(k + 1) * sizeof(RowPart), st, (const RowPart*)h->part, n_tiles,
+                           (const float*)h->ld, (const int*)h->ld_id, k, beta, tau, h->accepted, h->bif, h->row_stats, h->want_lse));
     KCHECK(h);
     if (d_accepted) CUDA_TRY(h, cudaMemcpyAsync(d_accepted, h->accepted, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
     if (d_bif) CUDA_TRY(h, cudaMemcpyAsync(d_bif, h->bif, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
@@ -892,8 +892,8 @@ int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float ta
 
 int commit_impl(specdec_handle* h, const int* d_keep, const int* d_next, cudaStream_t st) {
     const int k = h->last_k;
-    k_commit<<<cdiv(h->B, 128), 128, 0, st>>>(h->ses, h->v_draft, d_keep ? d_keep : h->accepted,
-                                             d_next ? d_next : h->bif, h->B, k, h->cfg.eos_id);
+    CUDA_TRY(h, launch_pdl(h, k_commit, dim3(cdiv(h->B, 128)), dim3(128), 0, st, h->ses, (const int*)h->v_draft,
+                           (const int*)(d_keep ? d_keep : h->accepted), (const int*)(d_next ? d_next : h->bif), h->B, k, h->cfg.eos_id));
     KCHECK(h);
     h->len_ub = std::min(h->len_ub + k + 1, h->T_cap);
     h->verified = false;
