@@ -988,25 +988,26 @@ int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, con
     int it = 0;
     const bool graphs = h->use_graphs && !h->profile;
     int tau_bits; memcpy(&tau_bits, &tau, 4);
+    // the drafter writes its block straight into the verifier's draft buffer: no copy between the two steps
     for (; it < max_iters; ++it) {
         if (graphs) {
             // the launches depend on the host-side length bound only through its 32-token bucket
             const int true_ub = h->len_ub, lb = len_bucket(h, true_ub);
             h->len_ub = lb;
-            if (k > 0) TRY(graph_call(h, {1, k, lb}, st, [&]() { return draft_impl<T>(h, k, h->g_draft, st); }));
+            if (k > 0) TRY(graph_call(h, {1, k, lb}, st, [&]() { return draft_impl<T>(h, k, h->v_draft, st); }));
             mark();
             h->len_ub = lb;
             TRY(graph_call(h, {2, k, lb, beta, tau_bits}, st, [&]() {
-                int rc = verify_impl<T>(h, h->g_draft, k, beta, tau, nullptr, nullptr, st);
+                int rc = verify_impl<T>(h, h->v_draft, k, beta, tau, nullptr, nullptr, st);
                 return rc ? rc : commit_impl(h, nullptr, nullptr, st);
             }));
             mark();
             h->len_ub = std::min(true_ub + k + 1, h->T_cap);
             h->last_k = k; h->verified = false; h->drafted = false;
         } else {
-            if (k > 0) TRY(draft_impl<T>(h, k, h->g_draft, st));
+            if (k > 0) TRY(draft_impl<T>(h, k, h->v_draft, st));
             mark();
-            TRY(verify_impl<T>(h, h->g_draft, k, beta, tau, nullptr, nullptr, st));
+            TRY(verify_impl<T>(h, h->v_draft, k, beta, tau, nullptr, nullptr, st));
             mark();
             TRY(commit_impl(h, nullptr, nullptr, st));
         }
