@@ -8,6 +8,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <math_constants.h>
+#include <type_traits>
 
 namespace sd {
 
@@ -464,15 +465,38 @@ __global__ void k_draft_logit(const T* __restrict__ y, const T* __restrict__ E, 
                               int B, int k, int d, int vocab, float* __restrict__ ld, int* __restrict__ ld_id) {
     int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     int lane = threadIdx.x & 31;
+    // The draft ids were written before this step's kernel chain began and the embedding table is a weight: with bf16
+    // rows of at most 512 columns a lane fetches its 16 columns of the draft's embedding row before the dependency wait.
+    const bool vec = std::is_same<T, bf16>::value && d % 16 == 0 && d <= 512;
+    const bool in_range = row < B * (k + 1);
+    const int b = in_range ? row / (k + 1) : 0, c = in_range ? row % (k + 1) : k;
+    const int tok = (in_range && c < k) ? draft[b * k + c] : -1;
+    const bool ok = tok >= 0 && tok < vocab;
+    uint4 ev[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+    if (vec && ok && lane * 16 < d) {
+        const uint4* ep = reinterpret_cast<const uint4*>(E + (size_t)tok * d + lane * 16);
+        ev[0] = __ldg(ep); ev[1] = __ldg(ep + 1);
+    }
     pdl_launch_dependents();
     pdl_wait();
-    if (row >= B * (k + 1)) return;
-    int b = row / (k + 1), c = row % (k + 1);
+    if (!in_range) return;
     if (c == k) { if (lane == 0) { ld[row] = CUDART_INF_F; ld_id[row] = -1; } return; }
-    int tok = draft[b * k + c];
-    bool ok = tok >= 0 && tok < vocab;
     float s = 0.f;
-    if (ok) for (int e = lane; e < d; e += 32) s = fmaf(to_f(y[(size_t)row * d + e]), to_f(E[(size_t)tok * d + e]), s);
+    if (vec) {
+        if (ok && lane * 16 < d) {
+            const uint4* yp = reinterpret_cast<const uint4*>(y + (size_t)row * d + lane * 16);
+            const uint4 yv[2] = {yp[0], yp[1]};
+            const __nv_bfloat162* e2 = reinterpret_cast<const __nv_bfloat162*>(ev);
+            const __nv_bfloat162* y2 = reinterpret_cast<const __nv_bfloat162*>(yv);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float2 a = __bfloat1622float2(y2[i]), w = __bfloat1622float2(e2[i]);
+                s = fmaf(a.x, w.x, s); s = fmaf(a.y, w.y, s);
+            }
+        }
+    } else if (ok) {
+        for (int e = lane; e < d; e += 32) s = fmaf(to_f(y[(size_t)row * d + e]), to_f(E[(size_t)tok * d + e]), s);
+    }
     s = warp_sum(s);
     if (lane == 0) { ld[row] = ok ? s : -CUDART_INF_F; ld_id[row] = ok ? tok : -2; }
 }
