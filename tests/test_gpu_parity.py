@@ -88,6 +88,26 @@ def test_config1_generate_bit_exact(tiny, beta, tau, graphs):
     sd.close()
 
 
+def test_degenerate_shapes_bit_exact(tiny):
+    """One-token sources, k = 1 and k = k_max, target budgets of 0, 1 and 2 tokens in one batch, a rule that accepts
+    everything (beta = V, huge tau) and the strict one: each sequence must equal the oracle's batch-1 run."""
+    wl, wv, wd, mv, md = tiny
+    V = wl.verifier.vocab
+    srcs = [np.array([7], np.int32), np.array([901], np.int32), wl.src[0][:2], wl.src[1]]
+    budgets = [0, 1, 2, 5]
+    sd = _handle(wl.verifier, wv, wl.drafter, wd, False)
+    src, lens = W.pad_batch(srcs)
+    for k in (1, 8):
+        for beta, tau in ((V, 1e30), (1, 0.0), (2, 0.25)):
+            out, n, st = sd.generate(src, lens, budgets, k, beta, tau)
+            assert n.cpu().tolist()[0] == 0
+            for b, s in enumerate(srcs):
+                ref, _ = O.specdec_generate(mv, md, s, budgets[b], k, beta, tau, BOS, EOS, MASK)
+                assert out[b, :int(n[b])].cpu().tolist() == ref, (k, beta, tau, b)
+            assert st["emitted"] == int(n.sum())
+    sd.close()
+
+
 def test_k0_is_greedy_autoregressive_decoding(tiny):
     """k = 0 runs the verifier alone, one row per step: the greedy baseline of the paper's comparisons."""
     wl, wv, wd, mv, md = tiny

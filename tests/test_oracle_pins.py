@@ -108,6 +108,18 @@ def test_stack_equals_torch_library_layers(tiny, causal, act):
     assert np.abs(l32 - logits_ref).max() < 2e-5
 
 
+def test_gelu_closed_form_values():
+    """x * Phi(x): Phi(1) = 0.841344746068543 (standard normal table), odd part x / 2, limits 0 and x."""
+    x = np.array([0.0, 1.0, -1.0, 2.0, 30.0, -30.0], dtype=np.float64)
+    g = O.gelu(x)
+    assert g[0] == 0.0
+    assert abs(g[1] - 0.841344746068543) < 1e-15 and abs(g[2] + (1.0 - 0.841344746068543)) < 1e-15
+    assert abs(g[3] - 2.0 * 0.977249868051821) < 1e-14
+    assert g[4] == 30.0 and g[5] == 0.0
+    np.testing.assert_allclose(O.gelu(x) - O.gelu(-x), x, rtol=0, atol=1e-14)       # gelu(x) - gelu(-x) = x
+    assert O.gelu(x.astype(np.float32)).dtype == np.float32
+
+
 def test_every_weight_is_used(tiny):
     """Perturbing any single weight tensor changes the verifier logits (no dropped term)."""
     wl, mv, _ = tiny
