@@ -348,7 +348,7 @@ def run_ours(args):
         O, mv, md = oracle_models(wl1)
         rng = np.random.default_rng(7)
         n_s, ctoks, csecs = 0, 0, 0.0
-        while n_s < 64 and csecs < 12.0:
+        while n_s < 128 and csecs < 15.0:              # a bounded sample: 10-20 s of CPU work
             n, t, _ = oracle_step(O, mv, md, wl1, n_s, rng)
             ctoks += n; csecs += t; n_s += 1
         line["cpu_baseline"] = {"value": ctoks / csecs, "unit": "tokens/s", "cores": cores_used(), "kind": "oracle",
