@@ -15,6 +15,7 @@
 // the paged cache.
 #pragma once
 #include "attention_tc.cuh"
+#include "gemm_tc.cuh"
 #include "kernels.cuh"
 
 namespace sd {
@@ -25,6 +26,7 @@ struct SkinnyArgs {
     const float* ln_g; const float* ln_b; float ln_eps;
     bf16* ln_out;                // ... optionally also written out as bf16 rows [rows, K] (by CTA 0)
     long long* trace;            // optional: CTA 0 records %globaltimer at a few points (debugging aid)
+    int* err_word;               // raised when a bounded wait gives up
 };
 
 __device__ __forceinline__ void sk_stamp(long long* trace, int slot) {
@@ -36,7 +38,20 @@ constexpr int SK_WARPS = 8;
 // G groups of 8 weight rows per CTA; the 8 warps are G groups x (8 / G) K-splits
 inline size_t skinny_smem(int MT, int K) { return (size_t)MT * 16 * (K + 8) * 2 + (size_t)SK_WARPS * MT * 16 * SK_NB * 4; }
 
-template <int EPI, int MT, bool LN, int G>
+// CL (with LN, clusters of 8 CTAs along the weight rows): every CTA of the grid needs the same normalised rows, and
+// 200 CTAs each reading the same 26 x 2 KB at the same moment queue up on the same L2 lines.  With CL each CTA of a
+// cluster normalises only the rows r, r + 8, ... (r = its cluster rank) and sends them to its seven peers'
+// shared memory (st.async, counted on the receiver's mbarrier): one eighth of the L2 requests, and no CTA
+// repeats another's arithmetic.
+__device__ __forceinline__ void sk_st_peer(uint32_t local_addr, uint32_t local_bar, uint32_t rank, uint32_t lo, uint32_t hi) {
+    uint32_t ra, rb;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rb) : "r"(local_bar), "r"(rank));
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.b32 [%0], {%1, %2}, [%3];"
+                 ::"r"(ra), "r"(lo), "r"(hi), "r"(rb) : "memory");
+}
+
+template <int EPI, int MT, bool LN, int G, bool CL = false>
 __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
     extern __shared__ __align__(16) unsigned char sk_sm[];
     const GemmArgs<bf16>& g = a.g;
@@ -75,6 +90,16 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
             lbet[c] = e < K ? __ldg(reinterpret_cast<const float4*>(a.ln_b + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
     }
+    __shared__ __align__(8) uint64_t row_bar;                 // CL: counts the peers' rows as they arrive
+    __shared__ int row_abort;
+    if constexpr (CL) {
+        if (tid == 0) {
+            row_abort = 0;
+            mbar_init(smem_u32(&row_bar), 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        tc_cluster_sync();                                    // every peer's barrier exists before anybody sends
+    }
     // everything above touched only weights; from here on the predecessor's output is read
     sk_stamp(a.trace, 1);
     pdl_launch_dependents();
@@ -82,7 +107,57 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
     sk_stamp(a.trace, 2);
     const int R = min(g.rows_static >= 0 ? g.rows_static : *g.n_rows, MT * 16);   // a device-side count is itself written earlier in the step
     // ---- activation rows into shared memory
-    if (LN) {
+    if (LN && CL) {
+        uint32_t rank;
+        asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+        const int own = (R > (int)rank) ? (R - 1 - (int)rank) / 8 + 1 : 0;      // rows rank, rank + 8, ... below R
+        if (tid == 0) mbar_expect_tx(smem_u32(&row_bar), (uint32_t)(R - own) * K * 2);
+        const int m = (int)rank + 8 * warp;                   // warps 0..3: one row each (MT * 16 = 32 rows at most)
+        if (warp < MT * 2 && m < R) {
+            float4 xv[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int e = lane * 4 + c * 128;
+                xv[c] = e < K ? *reinterpret_cast<const float4*>(a.ln_x + (size_t)m * K + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) sum += xv[c].x + xv[c].y + xv[c].z + xv[c].w;
+            const float mu = warp_sum(sum) / K;
+            float q = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (lane * 4 + c * 128 < K) {
+                    const float c0 = xv[c].x - mu, c1 = xv[c].y - mu, c2 = xv[c].z - mu, c3 = xv[c].w - mu;
+                    q += c0 * c0 + c1 * c1 + c2 * c2 + c3 * c3;
+                }
+            const float rstd = 1.0f / sqrtf(warp_sum(q) / K + a.ln_eps);
+            bf16* dst = As + (size_t)m * pitch;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int e = lane * 4 + c * 128;
+                if (e < K) {
+                    const float4 v = xv[c];
+                    const float4 gm = lgam[c], bt = lbet[c];
+                    __nv_bfloat162 p0, p1;
+                    p0.x = __float2bfloat16_rn((v.x - mu) * rstd * gm.x + bt.x); p0.y = __float2bfloat16_rn((v.y - mu) * rstd * gm.y + bt.y);
+                    p1.x = __float2bfloat16_rn((v.z - mu) * rstd * gm.z + bt.z); p1.y = __float2bfloat16_rn((v.w - mu) * rstd * gm.w + bt.w);
+                    const uint32_t lo = *reinterpret_cast<uint32_t*>(&p0), hi = *reinterpret_cast<uint32_t*>(&p1);
+                    *reinterpret_cast<uint2*>(dst + e) = make_uint2(lo, hi);
+                    const uint32_t la = smem_u32(dst + e);
+#pragma unroll
+                    for (uint32_t rk = 0; rk < 8; ++rk)
+                        if (rk != rank) sk_st_peer(la, smem_u32(&row_bar), rk, lo, hi);
+                }
+            }
+        }
+        // rows past the end are zeroed locally by the idle warps
+        for (int i = tid; i < (MT * 16 - R) * (K / 8); i += SK_WARPS * 32) {
+            const int mm = R + i / (K / 8), c = i % (K / 8);
+            *reinterpret_cast<uint4*>(As + (size_t)mm * pitch + c * 8) = make_uint4(0, 0, 0, 0);
+        }
+        mbar_wait(smem_u32(&row_bar), 0, &row_abort, a.err_word, 8);             // the peers' rows have landed
+    } else if (LN) {
         // each warp normalises rows warp, warp + 8, ...; all of its rows are fetched first (one round trip)
         constexpr int RS = (MT * 16 + SK_WARPS - 1) / SK_WARPS;      // row slots per warp
         constexpr int CH = 4;                                        // float4 chunks per lane and row: K <= 512

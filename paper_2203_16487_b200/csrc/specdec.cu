@@ -104,6 +104,7 @@ struct specdec_handle {
     NextLn next_ln = {nullptr, nullptr, nullptr};
     const float* fused_x = nullptr; const float* fused_g = nullptr; const void* fused_out = nullptr;
     int use_ln_fuse = 0;            // option "ln_fuse": measured slower than the separate LayerNorm launch, kept for comparison
+    int use_sk_cluster = 1;         // option "sk_cluster": LayerNorm-fused weight-streaming GEMMs share the normalised rows in clusters of 8
     bool lnrows_ready = false;
     int use_ln_rows = 0;            // option "ln_rows": GEMMs over at most 128 rows normalise their input rows themselves (measured slower: off)
     bool pair_ready = false;
@@ -393,8 +394,22 @@ template <int EPI, int MT, int G>
 int skinny_launch_g(specdec_handle* h, SkinnyArgs& a, cudaStream_t st) {
     const int grid = cdiv(a.g.N, SK_NB * G);
     const size_t smem = skinny_smem(MT, a.g.K);
-    cudaError_t e = a.ln_x ? launch_pdl(h, k_skinny<EPI, MT, true, G>, dim3(grid), dim3(SK_WARPS * 32), smem, st, a)
-                           : launch_pdl(h, k_skinny<EPI, MT, false, G>, dim3(grid), dim3(SK_WARPS * 32), smem, st, a);
+    cudaError_t e;
+    if (a.ln_x && G == 1 && h->use_sk_cluster && grid % 8 == 0 && a.g.K % 128 == 0) {
+        // clusters of 8 CTAs share the LayerNorm of the input rows (see skinny_gemm.cuh)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(SK_WARPS * 32); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 8; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = h->use_pdl ? 2 : 1;
+        e = cudaLaunchKernelEx(&cfg, k_skinny<EPI, MT, true, 1, true>, a);
+    } else {
+        e = a.ln_x ? launch_pdl(h, k_skinny<EPI, MT, true, G>, dim3(grid), dim3(SK_WARPS * 32), smem, st, a)
+                   : launch_pdl(h, k_skinny<EPI, MT, false, G>, dim3(grid), dim3(SK_WARPS * 32), smem, st, a);
+    }
     if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("skinny GEMM launch: ") + cudaGetErrorString(e));
     KCHECK(h);
     return 0;
@@ -421,7 +436,7 @@ template <int EPI, int MT>
 cudaError_t skinny_attr(int bytes) {
     cudaError_t e = cudaSuccess;
     auto set = [&](auto* f) { if (e == cudaSuccess) e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes); };
-    set(k_skinny<EPI, MT, true, 1>); set(k_skinny<EPI, MT, false, 1>);
+    set(k_skinny<EPI, MT, true, 1>); set(k_skinny<EPI, MT, false, 1>); set(k_skinny<EPI, MT, true, 1, true>);
     return e;
 }
 template <int EPI>
@@ -460,7 +475,7 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
         if (skinny) {
             SkinnyArgs sa; sa.g = g;
             sa.ln_x = lnp ? lnp->x : nullptr; sa.ln_g = lnp ? lnp->g : nullptr; sa.ln_b = lnp ? lnp->b : nullptr;
-            sa.ln_eps = 1e-5f; sa.ln_out = nullptr;
+            sa.ln_eps = 1e-5f; sa.ln_out = nullptr; sa.err_word = h->ses.counters + 7;
             sa.trace = (h->want_cl_trace && h->cl_trace) ? h->cl_trace + 216 + 6 * ((epi == EPI_RELU || epi == EPI_GELU) ? 0 : epi == EPI_RESID ? 1 : epi == EPI_QKV ? 2 : 3) : nullptr;
             TRY(skinny_launch(h, epi, sa, rows_ub, st));
             return 0;
@@ -928,7 +943,7 @@ void drop_graphs(specdec_handle* h) {
 // replayed afterwards.  The key must name everything the launches depend on besides device memory.
 template <typename F>
 int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body) {
-    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->use_ln_fuse); key.push_back(h->use_ln_rows); key.push_back(h->use_pair); key.push_back(h->attn_warps); key.push_back(h->attn_rs); key.push_back(h->use_fused_attn); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
+    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->use_ln_fuse); key.push_back(h->use_ln_rows); key.push_back(h->use_sk_cluster); key.push_back(h->use_pair); key.push_back(h->attn_warps); key.push_back(h->attn_rs); key.push_back(h->use_fused_attn); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
     key.push_back(h->B); key.push_back(h->S_max);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
@@ -1264,6 +1279,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
     if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "sk_cluster")) { h->use_sk_cluster = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "ln_rows")) { h->use_ln_rows = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "ln_fuse")) { h->use_ln_fuse = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "pair")) {
