@@ -51,6 +51,14 @@ __device__ __forceinline__ void sk_st_peer(uint32_t local_addr, uint32_t local_b
                  ::"r"(ra), "r"(lo), "r"(hi), "r"(rb) : "memory");
 }
 
+__device__ __forceinline__ void sk_st_peer16(uint32_t local_addr, uint32_t local_bar, uint32_t rank, uint4 v) {
+    uint32_t ra, rb;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rb) : "r"(local_bar), "r"(rank));
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+                 ::"r"(ra), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(rb) : "memory");
+}
+
 template <int EPI, int MT, bool LN, int G, bool CL = false>
 __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
     extern __shared__ __align__(16) unsigned char sk_sm[];
@@ -210,6 +218,30 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
                 for (int e = lane * 8; e < K; e += 256) *reinterpret_cast<uint4*>(dst + e) = make_uint4(0, 0, 0, 0);
             }
         }
+    } else if (CL) {
+        // plain rows, shared the same way: this CTA fetches rows rank, rank + 8, ... and sends them to its peers
+        uint32_t rank;
+        asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+        const int own = (R > (int)rank) ? (R - 1 - (int)rank) / 8 + 1 : 0;
+        if (tid == 0) mbar_expect_tx(smem_u32(&row_bar), (uint32_t)(R - own) * K * 2);
+        const int m = (int)rank + 8 * (warp >> 1), hf = warp & 1;     // two warps per row: halves of its 16-byte pieces
+        if ((warp >> 1) < MT * 2 && m < R) {
+            const int pieces = K / 8;                                 // 16-byte pieces per row
+            for (int p0 = hf * 32 + lane; p0 < pieces; p0 += 64) {
+                const uint4 v = *reinterpret_cast<const uint4*>(g.A + (size_t)m * g.lda + p0 * 8);
+                bf16* dst = As + (size_t)m * pitch + p0 * 8;
+                *reinterpret_cast<uint4*>(dst) = v;
+                const uint32_t la = smem_u32(dst);
+#pragma unroll
+                for (uint32_t rk = 0; rk < 8; ++rk)
+                    if (rk != rank) sk_st_peer16(la, smem_u32(&row_bar), rk, v);
+            }
+        }
+        for (int i = tid; i < (MT * 16 - R) * (K / 8); i += SK_WARPS * 32) {
+            const int mm = R + i / (K / 8), c = i % (K / 8);
+            *reinterpret_cast<uint4*>(As + (size_t)mm * pitch + c * 8) = make_uint4(0, 0, 0, 0);
+        }
+        mbar_wait(smem_u32(&row_bar), 0, &row_abort, a.err_word, 8);
     } else {
         const uint32_t as_base = (uint32_t)__cvta_generic_to_shared(As);
         const int chunks = K / 8;

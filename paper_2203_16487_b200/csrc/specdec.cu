@@ -104,7 +104,7 @@ struct specdec_handle {
     NextLn next_ln = {nullptr, nullptr, nullptr};
     const float* fused_x = nullptr; const float* fused_g = nullptr; const void* fused_out = nullptr;
     int use_ln_fuse = 0;            // option "ln_fuse": measured slower than the separate LayerNorm launch, kept for comparison
-    int use_sk_cluster = 1;         // option "sk_cluster": LayerNorm-fused weight-streaming GEMMs share the normalised rows in clusters of 8
+    int use_sk_cluster = 1;         // option "sk_cluster": 1 = LayerNorm-fused weight-streaming GEMMs share the normalised rows in clusters of 8; 2 = the plain ones too (measured slower)
     bool lnrows_ready = false;
     int use_ln_rows = 0;            // option "ln_rows": GEMMs over at most 128 rows normalise their input rows themselves (measured slower: off)
     bool pair_ready = false;
@@ -395,8 +395,8 @@ int skinny_launch_g(specdec_handle* h, SkinnyArgs& a, cudaStream_t st) {
     const int grid = cdiv(a.g.N, SK_NB * G);
     const size_t smem = skinny_smem(MT, a.g.K);
     cudaError_t e;
-    if (a.ln_x && G == 1 && h->use_sk_cluster && grid % 8 == 0 && a.g.K % 128 == 0) {
-        // clusters of 8 CTAs share the LayerNorm of the input rows (see skinny_gemm.cuh)
+    if (G == 1 && h->use_sk_cluster && grid % 8 == 0 && (a.ln_x ? a.g.K % 128 == 0 : (a.g.K % 8 == 0 && a.g.lda % 8 == 0 && h->use_sk_cluster >= 2))) {
+        // clusters of 8 CTAs share the (normalised) input rows (see skinny_gemm.cuh)
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(grid); cfg.blockDim = dim3(SK_WARPS * 32); cfg.dynamicSmemBytes = smem; cfg.stream = st;
         cudaLaunchAttribute attr[2];
@@ -405,7 +405,8 @@ int skinny_launch_g(specdec_handle* h, SkinnyArgs& a, cudaStream_t st) {
         attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr; cfg.numAttrs = h->use_pdl ? 2 : 1;
-        e = cudaLaunchKernelEx(&cfg, k_skinny<EPI, MT, true, 1, true>, a);
+        e = a.ln_x ? cudaLaunchKernelEx(&cfg, k_skinny<EPI, MT, true, 1, true>, a)
+                   : cudaLaunchKernelEx(&cfg, k_skinny<EPI, MT, false, 1, true>, a);
     } else {
         e = a.ln_x ? launch_pdl(h, k_skinny<EPI, MT, true, G>, dim3(grid), dim3(SK_WARPS * 32), smem, st, a)
                    : launch_pdl(h, k_skinny<EPI, MT, false, G>, dim3(grid), dim3(SK_WARPS * 32), smem, st, a);
@@ -436,7 +437,7 @@ template <int EPI, int MT>
 cudaError_t skinny_attr(int bytes) {
     cudaError_t e = cudaSuccess;
     auto set = [&](auto* f) { if (e == cudaSuccess) e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes); };
-    set(k_skinny<EPI, MT, true, 1>); set(k_skinny<EPI, MT, false, 1>); set(k_skinny<EPI, MT, true, 1, true>);
+    set(k_skinny<EPI, MT, true, 1>); set(k_skinny<EPI, MT, false, 1>); set(k_skinny<EPI, MT, true, 1, true>); set(k_skinny<EPI, MT, false, 1, true>);
     return e;
 }
 template <int EPI>
@@ -1279,7 +1280,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
     if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }
-    if (!strcmp(name, "sk_cluster")) { h->use_sk_cluster = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "sk_cluster")) { h->use_sk_cluster = value < 0 ? 0 : value; return SPECDEC_OK; }   // 0 off, 1 LayerNorm-fused kernels, 2 all
     if (!strcmp(name, "ln_rows")) { h->use_ln_rows = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "ln_fuse")) { h->use_ln_fuse = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "pair")) {
