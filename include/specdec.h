@@ -219,8 +219,8 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
  *   separate LayerNorm launch it removes: 743 vs 688 us per 128-sequence verify step);
  * "sk_cluster" = 0 off / 1 (default) / 2: the weight-streaming GEMMs with fused LayerNorm run in clusters of 8 CTAs
  *   that each normalise an eighth of the input rows and send them to their peers' shared memory (instead of every
- *   CTA of the grid reading and normalising all rows: 348 -> 272 us per batch-1 verify step); 2 shares the rows
- *   of the plain weight-streaming GEMMs the same way (measured slower: 287 us);
+ *   CTA of the grid reading and normalising all rows: 348 -> 272 us per batch-1 verify step); 2 / 3 also share the rows
+ *   of the plain weight-streaming GEMMs (2: those with K <= 512, no gain; 3: all, slower: 287 us);
  * "ln_rows" = 0/1 tensor-core GEMMs over at most 128 rows normalise their input rows themselves (eight warps write
  *   the bf16 operand tile in the tensor core's swizzled layout) instead of reading the output of a LayerNorm launch
  *   (default 0: correct, but every CTA repeating the normalisation costs more than the launch: 407 vs 358 us per

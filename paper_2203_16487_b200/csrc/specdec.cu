@@ -378,7 +378,8 @@ template <typename T> bool tc_usable(const specdec_handle* h, int N, int K) {
 // LayerNorm fused in front of a GEMM: x fp32 rows, gain, bias.
 struct LnSpec { const float* x; const float* g; const float* b; };
 
-// The weight-streaming kernel serves bf16 GEMMs over at most 32 rows (see skinny_gemm.cuh): measured on a
+// The weight-streaming kernel serves bf16 GEMMs over at most 32 rows (see skinny_gemm.cuh; 64-row variants of its
+// row-sharing LayerNorm kernels were tried too: 422 vs 356 us per 2-sequence verify step): measured on a
 // verify step, 26 rows take 362 us with it against 391 us with 64-wide tensor-core tiles, but 52 rows take
 // 500 us against 391 us, so anything beyond two 16-row tiles goes to the tile GEMM.
 constexpr int SK_ROWS_MAX = 32;
@@ -395,7 +396,7 @@ int skinny_launch_g(specdec_handle* h, SkinnyArgs& a, cudaStream_t st) {
     const int grid = cdiv(a.g.N, SK_NB * G);
     const size_t smem = skinny_smem(MT, a.g.K);
     cudaError_t e;
-    if (G == 1 && h->use_sk_cluster && grid % 8 == 0 && (a.ln_x ? a.g.K % 128 == 0 : (a.g.K % 8 == 0 && a.g.lda % 8 == 0 && h->use_sk_cluster >= 2))) {
+    if (G == 1 && h->use_sk_cluster && grid % 8 == 0 && (a.ln_x ? a.g.K % 128 == 0 : (a.g.K % 8 == 0 && a.g.lda % 8 == 0 && (h->use_sk_cluster >= 3 || (h->use_sk_cluster == 2 && a.g.K <= 512))))) {
         // clusters of 8 CTAs share the (normalised) input rows (see skinny_gemm.cuh)
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(grid); cfg.blockDim = dim3(SK_WARPS * 32); cfg.dynamicSmemBytes = smem; cfg.stream = st;
@@ -1280,7 +1281,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
     if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }
-    if (!strcmp(name, "sk_cluster")) { h->use_sk_cluster = value < 0 ? 0 : value; return SPECDEC_OK; }   // 0 off, 1 LayerNorm-fused kernels, 2 all
+    if (!strcmp(name, "sk_cluster")) { h->use_sk_cluster = value < 0 ? 0 : value; return SPECDEC_OK; }   // 0 off, 1 LayerNorm-fused kernels, 2 + plain ones with K <= 512, 3 all
     if (!strcmp(name, "ln_rows")) { h->use_ln_rows = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "ln_fuse")) { h->use_ln_fuse = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "pair")) {
