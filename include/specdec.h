@@ -222,9 +222,10 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
  *   CTA of the grid reading and normalising all rows: 348 -> 272 us per batch-1 verify step); 2 / 3 also share the rows
  *   of the plain weight-streaming GEMMs (2: those with K <= 512, no gain; 3: all, slower: 287 us);
  * "ln_rows" = 0/1 tensor-core GEMMs over at most 128 rows normalise their input rows themselves (eight warps write
- *   the bf16 operand tile in the tensor core's swizzled layout) instead of reading the output of a LayerNorm launch
- *   (default 0: correct, but every CTA repeating the normalisation costs more than the launch: 407 vs 358 us per
- *   2-sequence verify step, 491 vs 377 us at 4 sequences);
+ *   the bf16 operand tile in the tensor core's swizzled layout) instead of reading the output of a LayerNorm launch;
+ *   the CTAs form clusters of up to 8 that each normalise a share of the rows and send them to their peers' shared
+ *   memory (default 0: correct, but the 16-byte remote stores of 50-100 KB per CTA cost more than the launch they
+ *   replace: 365 vs 356 us per 2-sequence verify step, 426 vs 375 us at 4 sequences);
  * "attn_rs" = 0 never / 1 choose (default) / 2 whenever the keys allow: tile attention keeps the scores in the MMA
  *   accumulators through the softmax instead of a shared-memory tile (smaller footprint, more CTAs per SM);
  * "attn_warps" = 0 choose per launch, 4 or 8 warps per CTA of the tile attention (default 0);

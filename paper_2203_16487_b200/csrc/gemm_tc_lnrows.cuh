@@ -3,10 +3,13 @@
 //
 // Passes of a few dozen rows (a batch-1..4 verify block, the drafter's first layer, short encoder inputs) are
 // chains of small kernels, and a separate LayerNorm launch costs about as much as the GEMM it feeds.  Here one
-// CTA per 64 weight rows normalises ALL activation rows itself: its eight epilogue warps read the fp32 rows,
-// compute the statistics (two passes over registers, as the stand-alone kernel does) and write the bf16 operand
-// straight into shared memory in the layout the tensor core reads (128-byte rows, 16-byte chunks XOR-swizzled by
-// the row within 8-row groups: what a 128B-swizzled TMA load would have produced).  The whole weight tile
+// CTA per 64 weight rows; the CTAs form clusters of up to 8, and each CTA normalises only the rows rank, rank + C, ...
+// of its cluster: its eight epilogue warps read those fp32 rows, compute the statistics (two passes over registers,
+// as the stand-alone kernel does) and write the bf16 operand into shared memory in the layout the tensor core reads
+// (128-byte rows, 16-byte chunks XOR-swizzled by the row within 8-row groups: what a 128B-swizzled TMA load would
+// have produced) -- their own and, with st.async counted on the receiver's mbarrier, every peer's.  (Every CTA of
+// the grid normalising all rows itself was tried first and lost to the separate LayerNorm launch: all CTAs queue up
+// on the same L2 lines.)  The whole weight tile
 // (64 x K) fits the ring and is requested before the programmatic-launch dependency wait, so after the wait the
 // kernel is: read rows, normalise, K / 16 MMAs, epilogue.  Rows past the count are left as they are in shared
 // memory: they only feed accumulator lanes nobody reads.
@@ -24,6 +27,14 @@ inline size_t lr_smem(int K) { return (size_t)(K / TC_BK) * (LR_A_KB_BYTES + LR_
 inline bool lr_supported(int epi, int N, int K, int rows_ub) {
     return rows_ub <= TC_BM && K % TC_BK == 0 && K >= TC_BK && K <= LR_MAX_KB * TC_BK && N % LR_BN == 0 &&
            (epi == EPI_STORE || epi == EPI_RELU || epi == EPI_GELU || epi == EPI_QKV);
+}
+
+__device__ __forceinline__ void lr_st_peer16(uint32_t local_addr, uint32_t local_bar, uint32_t rank, uint4 v) {
+    uint32_t ra, rb;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rb) : "r"(local_bar), "r"(rank));
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+                 ::"r"(ra), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(rb) : "memory");
 }
 
 struct LnRowsArgs { const float* x; const float* gam; const float* bet; float eps; };
@@ -45,15 +56,18 @@ k_gemm_tc_lnrows(const __grid_constant__ CUtensorMap tmW, GemmArgs<bf16> g, LnRo
     if (threadIdx.x == 0) {
         abort_s = 0;
         for (int s = 0; s < LR_MAX_KB; ++s) mbar_init(smem_u32(&bar_w[s]), 1);
-        mbar_init(smem_u32(&bar_a), TC_EPI_WARPS);
+        mbar_init(smem_u32(&bar_a), TC_EPI_WARPS + 1);      // eight local warps + the thread that announces the peers' bytes
         mbar_init(smem_u32(&bar_acc), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), 64);
     tc_fence_before();
-    __syncthreads();
+    tc_cluster_sync();                               // peers' barriers exist before anybody sends (still before the dependency wait)
     tc_fence_after();
+    uint32_t rank;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    const uint32_t csize = tc_cluster_nctas();
     const uint32_t tmem_d = tmem_base_s;
     volatile int* abort_flag = &abort_s;
     // weights and LayerNorm parameters before the dependency wait
@@ -76,11 +90,14 @@ k_gemm_tc_lnrows(const __grid_constant__ CUtensorMap tmW, GemmArgs<bf16> g, LnRo
     pdl_launch_dependents();
     pdl_wait();
     const int R = min(g.rows_static >= 0 ? g.rows_static : *g.n_rows, TC_BM);
+    const int own = (R > (int)rank) ? (R - 1 - (int)rank) / (int)csize + 1 : 0;       // rows rank, rank + csize, ... below R
+    if (threadIdx.x == 0) mbar_expect_tx(smem_u32(&bar_a), (uint32_t)(R - own) * K * 2);
 
     if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, LR_BN);
             bool ok = mbar_wait(smem_u32(&bar_a), 0, abort_flag, err_word, 9);      // the normalised rows are in place
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             tc_fence_after();
             for (int kb = 0; kb < nkb && ok; ++kb) {
                 ok = mbar_wait(smem_u32(&bar_w[kb]), 0, abort_flag, err_word, 2);
@@ -95,11 +112,12 @@ k_gemm_tc_lnrows(const __grid_constant__ CUtensorMap tmW, GemmArgs<bf16> g, LnRo
     } else if (warp >= 2) {
         // ---- LayerNorm of rows (warp - 2), (warp - 2) + 8, ... into the operand tile
         const int w8 = warp - 2;
-        for (int r0 = w8; r0 < R; r0 += 4 * TC_EPI_WARPS) {        // four rows in flight per warp: one round trip
+        const int rstep = TC_EPI_WARPS * (int)csize;                // this CTA's rows: rank + csize * (w8 + 8 i)
+        for (int r0 = (int)rank + (int)csize * w8; r0 < R; r0 += 4 * rstep) {   // four rows in flight per warp: one round trip
             float4 v[4][4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const int r = r0 + i * TC_EPI_WARPS;
+                const int r = r0 + i * rstep;
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
                     v[i][c] = (r < R && col_ok) ? *(reinterpret_cast<const float4*>(ln.x + (size_t)r * K + lane * 16) + c)
@@ -107,7 +125,7 @@ k_gemm_tc_lnrows(const __grid_constant__ CUtensorMap tmW, GemmArgs<bf16> g, LnRo
             }
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const int r = r0 + i * TC_EPI_WARPS;
+                const int r = r0 + i * rstep;
                 if (r >= R) break;                                 // warp-uniform
                 float s = 0.f;
 #pragma unroll
@@ -133,8 +151,16 @@ k_gemm_tc_lnrows(const __grid_constant__ CUtensorMap tmW, GemmArgs<bf16> g, LnRo
                     // columns 16 lane .. : k-block lane / 4, 16-byte chunks 2 (lane % 4) and 2 (lane % 4) + 1 of the 128-byte row
                     uint8_t* rowp = a_ptr + (lane >> 2) * LR_A_KB_BYTES + r * 128;
                     const int c0 = (lane & 3) * 2;
-                    *reinterpret_cast<uint4*>(rowp + ((c0 ^ (r & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                    *reinterpret_cast<uint4*>(rowp + (((c0 + 1) ^ (r & 7)) << 4)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                    uint8_t* q0 = rowp + ((c0 ^ (r & 7)) << 4);
+                    uint8_t* q1 = rowp + (((c0 + 1) ^ (r & 7)) << 4);
+                    const uint4 v0 = make_uint4(pk[0], pk[1], pk[2], pk[3]), v1 = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                    *reinterpret_cast<uint4*>(q0) = v0;
+                    *reinterpret_cast<uint4*>(q1) = v1;
+                    for (uint32_t rk = 0; rk < csize; ++rk)
+                        if (rk != rank) {
+                            lr_st_peer16(smem_u32(q0), smem_u32(&bar_a), rk, v0);
+                            lr_st_peer16(smem_u32(q1), smem_u32(&bar_a), rk, v1);
+                        }
                 }
             }
         }
@@ -156,10 +182,14 @@ inline int lr_launch_one(TmaEncoder& enc, GemmArgs<bf16>& g, const LnRowsArgs& l
     if (!tw) return -1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(g.N / LR_BN); cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = lr_smem(g.K); cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = enc.pdl ? 1 : 0;
+    const int ctas = g.N / LR_BN;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = ctas % 8 == 0 ? 8 : (ctas % 4 == 0 ? 4 : (ctas % 2 == 0 ? 2 : 1));
+    attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = enc.pdl ? 2 : 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, k_gemm_tc_lnrows<EPI>, *tw, g, ln, enc.err_word);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { enc.err = std::string("launch (LayerNorm rows): ") + cudaGetErrorString(e); return -1; }
