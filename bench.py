@@ -204,6 +204,9 @@ def run_ours(args):
     del wv, wd
     if args.poll_lag is not None:
         sd.set_option("poll_lag", args.poll_lag)
+    for kv in args.opt:
+        name, _, val = kv.partition("=")
+        sd.set_option(name, int(val))
 
     # the step stream: rank r takes batches r, r + world, ... (replicas; no data-path collective)
     n_total = args.warmup + args.steps
@@ -290,6 +293,11 @@ def run_ours(args):
     timed_pass(W_, K_, host=False)
     vocab_ms, vocab_n = sd.profile_read()
     sd.set_option("profile", 0)
+    # per-phase times: a pass of its own, because an event after every phase keeps the host from queueing whole
+    # iterations ahead (the timed pass above records none)
+    sd.set_option("stats_timing", 1)
+    _, _, ph_stats = timed_pass(W_, K_, host=False)
+    sd.set_option("stats_timing", 0)
 
     toks_all, ms_max = replicas.reduce_job(toks, ms, dev)
     e_toks_all, e_ms_max = replicas.reduce_job(e_toks, e_ms, dev)
@@ -334,7 +342,9 @@ def run_ours(args):
         "tok_per_iteration": {"accepted": acc / max(seq_it, 1), "emitted": toks / max(seq_it, 1)},
         "iterations": it,
         "scripted_runs_differing_from_greedy": diverged[0],
-        "ms_breakdown": {k: sum(s[k] for s in stats) / max(K_, 1) for k in ("ms_encode", "ms_draft", "ms_verify", "ms_commit")},
+        "ms_breakdown": dict({k: sum(s[k] for s in ph_stats) / max(K_, 1) for k in ("ms_encode", "ms_draft", "ms_verify", "ms_commit", "ms_total")},
+                             note="separate untimed pass with an event after every phase (option stats_timing): each iteration "
+                                  "then waits for the host, so ms_total here exceeds ms_per_step"),
         "unscripted": {"value": n_toks_all / (n_ms_max * 1e-3), "unit": "tokens/s",
                        "tok_per_iteration": sum(s["emitted"] for s in n_stats) / max(sum(s["seq_iterations"] for s in n_stats), 1)},
     }
@@ -368,6 +378,7 @@ def main():
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--opt", action="append", default=[], help="experiments: name=value passed to specdec_set_option")
     ap.add_argument("--poll-lag", type=int, default=None, help="experiments: iterations the host runs ahead of the finish counter")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

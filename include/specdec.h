@@ -90,10 +90,10 @@ typedef struct {
  * accepted / seq_iterations (or emitted / seq_iterations counting the
  * bifurcation token); t_d, t_v are ms_draft, ms_verify per iteration. */
 typedef struct {
-    long long iterations;              /* draft->verify->commit rounds launched               */
+    long long iterations;              /* draft->verify->commit rounds that ran               */
     long long seq_iterations;          /* sum over rounds of sequences still decoding         */
     long long drafted, accepted, emitted;
-    double    ms_encode, ms_draft, ms_verify, ms_commit, ms_total;
+    double    ms_encode, ms_draft, ms_verify, ms_commit, ms_total;   /* draft / verify / commit: option "stats_timing" only */
     int       status;
 } specdec_stats;
 
@@ -234,7 +234,16 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
  *   batch is at most 8, k + 1 <= 32 and the model has 8 heads of 64 (default 0: measured slower than the
  *   per-operation kernels, kept for comparison);
  * "poll_lag" = n: specdec_generate reads the unfinished-sequences counter n iterations late (0: waits for it
- *   after every iteration; default 0 up to batch 4, else 2);
+ *   after every iteration; default 2 with gated iteration graphs, else 0 up to batch 4 and 2 above);
+ * "poll_flag" = 0/1 specdec_generate learns of each commit from a word the commit kernel writes into pinned host
+ *   memory, on which the host spins (default 1), instead of a 4-byte copy and an event per iteration;
+ * "gate" = 0 never / 1 above batch 4 (default) / 2 always: specdec_generate launches each draft -> verify -> commit iteration as ONE CUDA graph whose kernels
+ *   sit in the body of a conditional IF node behind a one-thread kernel that tests the unfinished-sequences
+ *   counter: the host queues iterations ahead of the counter it reads back, and an iteration queued after the
+ *   last sequence finished costs that one kernel (needs "graphs" = 1 and "stats_timing" = 0; at batch 1 the
+ *   conditional node costs more per iteration, about 15 us, than the wait it removes);
+ * "stats_timing" = 0/1 specdec_generate records an event after every draft, verify and commit phase and fills
+ *   ms_draft / ms_verify / ms_commit (default 0: only ms_encode and ms_total; 1 turns the gated graphs off);
  * "fused_attn" = 0/1 attention + output projection + residual as one 8-CTA-cluster kernel per sequence for
  *   blocks of at most 32 query rows and models with 8 heads of 64 (default 0: measured slower than the two
  *   separate kernels at batch 1 and at batch 128, kept for comparison);

@@ -52,7 +52,7 @@ struct Session {
                        //      2 verify rows, 3 encoder rows, 4 unfinished sequences
     unsigned long long* stats;  // [4]: seq_iterations, drafted, accepted, emitted
 };
-enum { CNT_DRAFT_ALL = 0, CNT_DRAFT_MASK = 1, CNT_VERIFY = 2, CNT_ENC = 3, CNT_ACTIVE = 4 };
+enum { CNT_DRAFT_ALL = 0, CNT_DRAFT_MASK = 1, CNT_VERIFY = 2, CNT_ENC = 3, CNT_ACTIVE = 4, CNT_TICKET = 5, CNT_SEQ = 6 };
 
 // Per-row metadata of the pass being run.
 struct Rows {
@@ -669,29 +669,43 @@ __global__ void k_apply_script(Session s, const int* __restrict__ script, int st
 // Appends drafts[0..keep) and the next token, cuts after the first EOS and at max_tgt.
 // Cache rows beyond the new length are simply dead: the next block overwrites them.
 __global__ void k_commit(Session s, const int* __restrict__ draft, const int* __restrict__ keep,
-                         const int* __restrict__ next, int B, int k, int eos) {
+                         const int* __restrict__ next, int B, int k, int eos, unsigned long long* post) {
     int b = blockIdx.x * blockDim.x + threadIdx.x;
     pdl_wait();                                    // no early trigger: the lengths written here are read by later kernels BEFORE their waits
-    if (b >= B || s.finished[b]) return;
-    int j = s.len[b];
-    const int mt = s.max_tgt[b];
-    const int a = min(max(keep[b], 0), k);
-    bool fin = false;
-    int n0 = j;
-    for (int c = 0; c <= a && !fin; ++c) {
-        if (j >= mt) { fin = true; break; }
-        int tok = (c < a) ? draft[b * k + c] : next[b];
-        s.out[(size_t)b * s.out_stride + j] = tok;
-        ++j;
-        if (tok == eos) fin = true;
+    if (b < B && !s.finished[b]) {
+        int j = s.len[b];
+        const int mt = s.max_tgt[b];
+        const int a = min(max(keep[b], 0), k);
+        bool fin = false;
+        int n0 = j;
+        for (int c = 0; c <= a && !fin; ++c) {
+            if (j >= mt) { fin = true; break; }
+            int tok = (c < a) ? draft[b * k + c] : next[b];
+            s.out[(size_t)b * s.out_stride + j] = tok;
+            ++j;
+            if (tok == eos) fin = true;
+        }
+        if (j >= mt) fin = true;
+        s.len[b] = j;
+        atomicAdd(&s.stats[0], 1ull);
+        atomicAdd(&s.stats[1], (unsigned long long)k);
+        atomicAdd(&s.stats[2], (unsigned long long)a);
+        atomicAdd(&s.stats[3], (unsigned long long)(j - n0));
+        if (fin) { s.finished[b] = 1; atomicSub(&s.counters[CNT_ACTIVE], 1); }
     }
-    if (j >= mt) fin = true;
-    s.len[b] = j;
-    atomicAdd(&s.stats[0], 1ull);
-    atomicAdd(&s.stats[1], (unsigned long long)k);
-    atomicAdd(&s.stats[2], (unsigned long long)a);
-    atomicAdd(&s.stats[3], (unsigned long long)(j - n0));
-    if (fin) { s.finished[b] = 1; atomicSub(&s.counters[CNT_ACTIVE], 1); }
+    // the last block to get here posts (commits of this handle so far) << 32 | (sequences still decoding) to the
+    // host-mapped word the generation loop polls: no copy, no event between the iterations
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(&s.counters[CNT_TICKET], 1) == (int)gridDim.x - 1) {
+            s.counters[CNT_TICKET] = 0;
+            const int seq = ++s.counters[CNT_SEQ];
+            const int active = atomicAdd(&s.counters[CNT_ACTIVE], 0);
+            *reinterpret_cast<volatile unsigned long long*>(post) = ((unsigned long long)(unsigned)seq << 32) | (unsigned)active;
+            __threadfence_system();
+        }
+    }
 }
 
 __global__ void k_session_init(Session s, const int* __restrict__ src_len, const int* __restrict__ max_tgt, int B,
@@ -713,6 +727,7 @@ __global__ void k_count_active(Session s, int B) {
         int n = 0;
         for (int b = 0; b < B; ++b) n += s.finished[b] ? 0 : 1;
         s.counters[CNT_ACTIVE] = n;
+        s.counters[CNT_TICKET] = 0;
     }
 }
 

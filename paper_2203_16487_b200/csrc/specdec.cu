@@ -7,6 +7,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <chrono>
 #include <map>
 #include <string>
 #include <type_traits>
@@ -96,6 +97,9 @@ struct specdec_handle {
     int want_cl_trace = 0;
     size_t skinny_smem_cap = 0;
     int poll_lag = -1;              // -1: chosen by batch size
+    int stats_timing = 0;           // 1: specdec_generate records an event after every phase (option "stats_timing")
+    int use_gate = 1;               // whole iterations as one graph behind a device-side IF node (option "gate")
+    bool gate_ok = true;            // false once building such a graph failed: the plain graphs are used from then on
     int use_fused_attn = 0;         // attention + output projection as one cluster kernel (measured slower: off)
     size_t attn_proj_smem_cap = 0;
     // LayerNorm fused into the residual GEMM that feeds it (tensor-core path): what the next residual GEMM should
@@ -119,6 +123,9 @@ struct specdec_handle {
     long long launches = 0;
     // polling
     int* h_poll = nullptr;          // pinned
+    unsigned long long* h_post = nullptr;   // pinned, written by k_commit: (commits of this handle so far) << 32 | unfinished sequences
+    unsigned commits_issued = 0;    // commit kernels launched so far: what the posted count reaches once the stream drains
+    int poll_flag = 1;              // the generation loop polls h_post instead of copying the counter back (option "poll_flag")
     unsigned long long* h_stats = nullptr;  // pinned [4]
     std::vector<cudaEvent_t> poll_ev;
     std::vector<cudaEvent_t> time_ev;
@@ -910,7 +917,7 @@ int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float ta
 int commit_impl(specdec_handle* h, const int* d_keep, const int* d_next, cudaStream_t st) {
     const int k = h->last_k;
     CUDA_TRY(h, launch_pdl(h, k_commit, dim3(cdiv(h->B, 128)), dim3(128), 0, st, h->ses, (const int*)h->v_draft,
-                           (const int*)(d_keep ? d_keep : h->accepted), (const int*)(d_next ? d_next : h->bif), h->B, k, h->cfg.eos_id));
+                           (const int*)(d_keep ? d_keep : h->accepted), (const int*)(d_next ? d_next : h->bif), h->B, k, h->cfg.eos_id, h->h_post));
     KCHECK(h);
     h->len_ub = std::min(h->len_ub + k + 1, h->T_cap);
     h->verified = false;
@@ -943,10 +950,18 @@ void drop_graphs(specdec_handle* h) {
 
 // Runs `body` (a sequence of launches on `st`) through a cached CUDA graph: captured on first use,
 // replayed afterwards.  The key must name everything the launches depend on besides device memory.
+inline void graph_key_tail(const specdec_handle* h, std::vector<long long>& key) {
+    for (long long v : {(long long)h->use_tc, (long long)h->use_tc_attn, (long long)h->want_lse, (long long)h->use_skinny,
+                        (long long)h->use_pdl, (long long)h->use_ln_fuse, (long long)h->use_ln_rows, (long long)h->use_sk_cluster,
+                        (long long)h->use_pair, (long long)h->attn_warps, (long long)h->attn_rs, (long long)h->use_fused_attn,
+                        (long long)h->skinny_groups, (long long)h->use_cluster, (long long)h->want_cl_trace,
+                        (long long)(h->script_on ? 1 : 0), (long long)h->B, (long long)h->S_max})
+        key.push_back(v);
+}
+
 template <typename F>
 int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body) {
-    key.push_back(h->use_tc); key.push_back(h->use_tc_attn); key.push_back(h->want_lse); key.push_back(h->use_skinny); key.push_back(h->use_pdl); key.push_back(h->use_ln_fuse); key.push_back(h->use_ln_rows); key.push_back(h->use_sk_cluster); key.push_back(h->use_pair); key.push_back(h->attn_warps); key.push_back(h->attn_rs); key.push_back(h->use_fused_attn); key.push_back(h->skinny_groups); key.push_back(h->use_cluster); key.push_back(h->want_cl_trace); key.push_back(h->script_on ? 1 : 0);
-    key.push_back(h->B); key.push_back(h->S_max);
+    graph_key_tail(h, key);
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
         const long long before = h->launches;
@@ -967,6 +982,57 @@ int graph_call(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F
     }
     CUDA_TRY(h, cudaGraphLaunch(it->second.exec, st));
     h->launches += it->second.kernels;
+    return 0;
+}
+
+// One kernel in front of an IF node: the body runs only while a sequence is still decoding.
+__global__ void k_gate(const int* __restrict__ counters, cudaGraphConditionalHandle cond) {
+    if (threadIdx.x == 0) cudaGraphSetConditional(cond, counters[CNT_ACTIVE] > 0 ? 1u : 0u);
+}
+
+// A whole draft -> verify -> commit iteration as ONE graph whose launches sit in the body of a conditional node:
+// the host can queue iterations ahead of the "unfinished sequences" counter it reads back (no bubble between
+// iterations), and an iteration queued after the last sequence finished costs one tiny kernel instead of a full pass.
+// Returns 1 (nothing launched) when such a graph cannot be built here; the caller then uses the plain graphs.
+template <typename F>
+int graph_call_gated(specdec_handle* h, std::vector<long long> key, cudaStream_t st, F body, long long* kernels_out) {
+    graph_key_tail(h, key);
+    auto it = h->graphs.find(key);
+    if (it == h->graphs.end()) {
+        const long long before = h->launches;
+        cudaGraph_t g = nullptr, bg = nullptr;
+        cudaGraphConditionalHandle cond;
+        cudaGraphNode_t gate_node, if_node;
+        auto give_up = [&](const char*) { if (g) cudaGraphDestroy(g); cudaGetLastError(); h->gate_ok = false; h->launches = before; return 1; };
+        if (cudaGraphCreate(&g, 0) != cudaSuccess) return give_up("create");
+        if (cudaGraphConditionalHandleCreate(&cond, g, 0, cudaGraphCondAssignDefault) != cudaSuccess) return give_up("handle");
+        const int* counters = h->ses.counters;
+        void* gate_args[] = {(void*)&counters, (void*)&cond};
+        cudaKernelNodeParams kp{};
+        kp.func = (void*)k_gate; kp.gridDim = dim3(1); kp.blockDim = dim3(32); kp.sharedMemBytes = 0; kp.kernelParams = gate_args;
+        if (cudaGraphAddKernelNode(&gate_node, g, nullptr, 0, &kp) != cudaSuccess) return give_up("gate");
+        cudaGraphNodeParams cp{};
+        cp.type = cudaGraphNodeTypeConditional;
+        cp.conditional.handle = cond; cp.conditional.type = cudaGraphCondTypeIf; cp.conditional.size = 1;
+        if (cudaGraphAddNode(&if_node, g, &gate_node, 1, &cp) != cudaSuccess) return give_up("if node");
+        bg = cp.conditional.phGraph_out[0];
+        if (cudaStreamBeginCaptureToGraph(st, bg, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return give_up("capture");
+        int rc = body();
+        cudaGraph_t got = nullptr;
+        cudaError_t e = cudaStreamEndCapture(st, &got);
+        if (rc != 0) { cudaGraphDestroy(g); h->launches = before; return rc; }
+        if (e != cudaSuccess) return give_up("end capture");
+        cudaGraphExec_t ex = nullptr;
+        if (cudaGraphInstantiate(&ex, g, 0) != cudaSuccess) return give_up("instantiate");
+        cudaGraphDestroy(g);
+        if (h->graphs.size() > 256) drop_graphs(h);
+        specdec_handle::GraphEntry ge{ex, h->launches - before + 1};
+        h->launches = before;
+        it = h->graphs.emplace(std::move(key), ge).first;
+    }
+    CUDA_TRY(h, cudaGraphLaunch(it->second.exec, st));
+    h->launches += it->second.kernels;
+    *kernels_out = it->second.kernels;
     return 0;
 }
 
@@ -992,33 +1058,73 @@ template <typename T>
 int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, const int* d_max_tgt, int B, int S_max,
                   int k, int beta, float tau, int* d_out, int out_stride, int* d_out_len, specdec_stats* hs,
                   cudaStream_t st) {
-    const bool timed = hs != nullptr;
+    const bool timed = hs != nullptr, phases = timed && h->stats_timing;
     size_t ev = 0;
-    auto mark = [&]() { if (timed && ev < h->time_ev.size()) cudaEventRecord(h->time_ev[ev++], st); };
-    mark();
+    auto mark_always = [&]() { if (timed && ev < h->time_ev.size()) cudaEventRecord(h->time_ev[ev++], st); };
+    auto mark = [&]() { if (phases) mark_always(); };
+    mark_always();
     TRY(encode_staged<T>(h, d_src, d_src_len, d_max_tgt, B, S_max, st));
-    mark();
+    mark_always();
     const int max_iters = h->T_cap;            // every iteration commits >= 1 token per unfinished sequence
-    // how many iterations the host runs ahead of the "unfinished sequences" counter it reads back: every iteration
-    // launched after the last sequence finished is wasted work, every wait for the counter is a bubble
-    const int lag = h->poll_lag >= 0 ? h->poll_lag : (B <= 4 ? 0 : 2), slots = (int)h->poll_ev.size();
-    int it = 0;
     const bool graphs = h->use_graphs && !h->profile;
+    // the conditional node costs more per iteration than the bubble it removes: worth it only where the host ran
+    // ahead anyway (larger batches), to make the iterations queued after the last sequence finished free
+    bool gated = graphs && h->gate_ok && !phases && (h->use_gate == 1 ? B > 4 : h->use_gate == 2);
+    // how many iterations the host runs ahead of the "unfinished sequences" counter it reads back.  Plain graphs:
+    // every iteration launched after the last sequence finished is wasted work, every wait for the counter is a
+    // bubble.  Gated graphs: an iteration too many costs one small kernel, so the host always runs ahead.
+    const int slots = (int)h->poll_ev.size();
+    int lag = h->poll_lag >= 0 ? std::min(h->poll_lag, slots - 1) : (gated ? 2 : (B <= 4 ? 0 : 2));
+    int it = 0, skipped = 0;
+    long long skipped_kernels = 0;
+    const bool flag = h->poll_flag != 0;
+    if (flag && cudaStreamQuery(st) == cudaSuccess) h->commits_issued = (unsigned)(*(volatile unsigned long long*)h->h_post >> 32);
+    const unsigned commits_base = h->commits_issued;
+    std::vector<long long> it_kernels;
     int tau_bits; memcpy(&tau_bits, &tau, 4);
     // the drafter writes its block straight into the verifier's draft buffer: no copy between the two steps
     for (; it < max_iters; ++it) {
         if (graphs) {
             // the launches depend on the host-side length bound only through its 32-token bucket
             const int true_ub = h->len_ub, lb = len_bucket(h, true_ub);
-            h->len_ub = lb;
-            if (k > 0) TRY(graph_call(h, {1, k, lb}, st, [&]() { return draft_impl<T>(h, k, h->v_draft, st); }));
-            mark();
-            h->len_ub = lb;
-            TRY(graph_call(h, {2, k, lb, beta, tau_bits}, st, [&]() {
-                int rc = verify_impl<T>(h, h->v_draft, k, beta, tau, nullptr, nullptr, st);
-                return rc ? rc : commit_impl(h, nullptr, nullptr, st);
-            }));
-            mark();
+            bool done = false;
+            if (gated) {
+                h->len_ub = lb;
+                long long nk = 0;
+                int rc = graph_call_gated(h, {3, k, lb, beta, tau_bits}, st, [&]() {
+                    int r = k > 0 ? draft_impl<T>(h, k, h->v_draft, st) : 0;
+                    h->len_ub = lb;
+                    if (!r) r = verify_impl<T>(h, h->v_draft, k, beta, tau, nullptr, nullptr, st);
+                    return r ? r : commit_impl(h, nullptr, nullptr, st);
+                }, &nk);
+                if (rc == 1) { gated = false; if (h->poll_lag < 0) lag = std::min(lag, B <= 4 ? 0 : 2); }
+                else if (rc != 0) return rc;
+                else { done = true; it_kernels.push_back(nk); }
+            }
+            if (!done && !phases) {
+                // one graph per iteration: no graph-to-graph gap between the drafter and the verifier
+                h->len_ub = lb;
+                TRY(graph_call(h, {4, k, lb, beta, tau_bits}, st, [&]() {
+                    int r = k > 0 ? draft_impl<T>(h, k, h->v_draft, st) : 0;
+                    h->len_ub = lb;
+                    if (!r) r = verify_impl<T>(h, h->v_draft, k, beta, tau, nullptr, nullptr, st);
+                    return r ? r : commit_impl(h, nullptr, nullptr, st);
+                }));
+                it_kernels.push_back(0);
+                done = true;
+            }
+            if (!done) {
+                h->len_ub = lb;
+                if (k > 0) TRY(graph_call(h, {1, k, lb}, st, [&]() { return draft_impl<T>(h, k, h->v_draft, st); }));
+                mark();
+                h->len_ub = lb;
+                TRY(graph_call(h, {2, k, lb, beta, tau_bits}, st, [&]() {
+                    int rc = verify_impl<T>(h, h->v_draft, k, beta, tau, nullptr, nullptr, st);
+                    return rc ? rc : commit_impl(h, nullptr, nullptr, st);
+                }));
+                mark();
+                it_kernels.push_back(0);
+            }
             h->len_ub = std::min(true_ub + k + 1, h->T_cap);
             h->last_k = k; h->verified = false; h->drafted = false;
         } else {
@@ -1027,33 +1133,69 @@ int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, con
             TRY(verify_impl<T>(h, h->v_draft, k, beta, tau, nullptr, nullptr, st));
             mark();
             TRY(commit_impl(h, nullptr, nullptr, st));
+            it_kernels.push_back(0);
         }
         mark();
-        CUDA_TRY(h, cudaMemcpyAsync(h->h_poll + (it % slots), h->ses.counters + CNT_ACTIVE, 4, cudaMemcpyDeviceToHost, st));
-        CUDA_TRY(h, cudaEventRecord(h->poll_ev[it % slots], st));
+        int active_seen = 1;
+        if (flag) {
+            // spin on the word k_commit posts; a look at the stream now and then surfaces a failed launch
+            if (it >= lag) {
+                const unsigned want = commits_base + (unsigned)(it - lag + 1);
+                const auto t0 = std::chrono::steady_clock::now();
+                for (unsigned spins = 1;; ++spins) {
+                    const unsigned long long v = *(volatile unsigned long long*)h->h_post;
+                    if ((int)((unsigned)(v >> 32) - want) >= 0) { active_seen = (int)(unsigned)v; break; }
+                    if ((spins & 0xfffu) == 0) {
+                        cudaError_t q = cudaStreamQuery(st);
+                        if (q != cudaSuccess && q != cudaErrorNotReady) return fail(h, SPECDEC_ERR_CUDA, std::string("generate: ") + cudaGetErrorString(q));
+                        if (q == cudaSuccess) {       // the stream drained: the word must be there now
+                            const unsigned long long v2 = *(volatile unsigned long long*)h->h_post;
+                            if ((int)((unsigned)(v2 >> 32) - want) >= 0) { active_seen = (int)(unsigned)v2; break; }
+                            return fail(h, SPECDEC_ERR_CUDA, "generate: the commit kernel did not post its counter");
+                        }
+                        if (std::chrono::steady_clock::now() - t0 > std::chrono::seconds(60))
+                            return fail(h, SPECDEC_ERR_TIMEOUT, "generate: no commit within 60 s");
+                    }
+                }
+            }
+        } else {
+            CUDA_TRY(h, cudaMemcpyAsync(h->h_poll + (it % slots), h->ses.counters + CNT_ACTIVE, 4, cudaMemcpyDeviceToHost, st));
+            CUDA_TRY(h, cudaEventRecord(h->poll_ev[it % slots], st));
+            if (it >= lag) {
+                CUDA_TRY(h, cudaEventSynchronize(h->poll_ev[(it - lag) % slots]));
+                active_seen = h->h_poll[(it - lag) % slots];
+            }
+        }
         if (it >= lag) {
-            CUDA_TRY(h, cudaEventSynchronize(h->poll_ev[(it - lag) % slots]));
-            if (h->h_poll[(it - lag) % slots] == 0) { ++it; break; }
+            if (active_seen == 0) {
+                // iterations it - lag + 1 .. it found nothing to do: behind a gate only the gate kernel ran
+                for (int j = it - lag + 1; j <= it; ++j)
+                    if (it_kernels[j] > 0) { ++skipped; skipped_kernels += it_kernels[j] - 1; }
+                ++it;
+                break;
+            }
         }
     }
+    h->launches -= skipped_kernels;
     if (d_out || d_out_len) TRY(specdec_get_output(h, d_out, out_stride, d_out_len, nullptr, st));
     CUDA_TRY(h, cudaMemcpyAsync(h->h_stats, h->ses.stats, 32, cudaMemcpyDeviceToHost, st));
     CUDA_TRY(h, cudaMemcpyAsync(h->h_stats + 4, h->ses.counters + 7, 4, cudaMemcpyDeviceToHost, st));
-    mark();
+    mark_always();
     CUDA_TRY(h, cudaStreamSynchronize(st));
+    h->commits_issued = (unsigned)(*(volatile unsigned long long*)h->h_post >> 32);    // gated iterations that found nothing to do posted nothing
     if (h->profile) prof_collect(h);
     if (*(int*)(h->h_stats + 4) != 0)
         return fail(h, SPECDEC_ERR_TIMEOUT, "a bounded device-side wait gave up (code " + std::to_string(*(int*)(h->h_stats + 4)) + ")");
     if (hs) {
         memset(hs, 0, sizeof(*hs));
-        hs->iterations = it;
+        hs->iterations = it - skipped;
         hs->seq_iterations = (long long)h->h_stats[0];
         hs->drafted = (long long)h->h_stats[1];
         hs->accepted = (long long)h->h_stats[2];
         hs->emitted = (long long)h->h_stats[3];
         auto ms = [&](size_t a, size_t b) { float t = 0.f; if (b < ev) cudaEventElapsedTime(&t, h->time_ev[a], h->time_ev[b]); return (double)t; };
         hs->ms_encode = ms(0, 1);
-        for (int i = 0; i < it; ++i) {
+        for (int i = 0; i < it && phases; ++i) {
             size_t b0 = 1 + (size_t)i * 3;
             hs->ms_draft += ms(b0, b0 + 1);
             hs->ms_verify += ms(b0 + 1, b0 + 2);
@@ -1156,6 +1298,8 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
     ce = cudaStreamSynchronize(st);
     if (ce == cudaSuccess) ce = cudaGetLastError();
     if (ce != cudaSuccess) return bail(SPECDEC_ERR_CUDA, std::string("weight repacking: ") + cudaGetErrorString(ce));
+    if (cudaMallocHost((void**)&h->h_post, 64) != cudaSuccess) return bail(SPECDEC_ERR_CUDA, "pinned host allocation failed");
+    *h->h_post = 0ull;
     if (cudaMallocHost((void**)&h->h_poll, 64 * 4) != cudaSuccess || cudaMallocHost((void**)&h->h_stats, 64) != cudaSuccess)
         return bail(SPECDEC_ERR_CUDA, "pinned host allocation failed");
     cudaStreamCreateWithFlags(&h->own_stream, cudaStreamNonBlocking);
@@ -1261,6 +1405,7 @@ int specdec_destroy(specdec_handle* h) {
     for (auto& e : h->time_ev) cudaEventDestroy(e);
     for (auto& e : h->prof_ev) cudaEventDestroy(e);
     if (h->h_poll) cudaFreeHost(h->h_poll);
+    if (h->h_post) cudaFreeHost(h->h_post);
     if (h->h_stats) cudaFreeHost(h->h_stats);
     if (h->arena.base) cudaFree(h->arena.base);
     delete h;
@@ -1279,6 +1424,9 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
     if (!strcmp(name, "cl_trace")) { h->want_cl_trace = value; return SPECDEC_OK; }   // 10 + e: time the tensor-core GEMM with epilogue e instead of the vocabulary one
     if (!strcmp(name, "fused_attn")) { h->use_fused_attn = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
+    if (!strcmp(name, "stats_timing")) { h->stats_timing = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "poll_flag")) { h->poll_flag = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "gate")) { h->use_gate = value; return SPECDEC_OK; }
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "sk_cluster")) { h->use_sk_cluster = value < 0 ? 0 : value; return SPECDEC_OK; }   // 0 off, 1 LayerNorm-fused kernels, 2 + plain ones with K <= 512, 3 all
@@ -1364,7 +1512,9 @@ int specdec_commit(specdec_handle* h, const int32_t* d_keep, const int32_t* d_ne
     if (!h->encoded) return fail(h, SPECDEC_ERR_NOT_ENCODED, "commit: no session (call specdec_encode)");
     if (!h->verified) return fail(h, SPECDEC_ERR_INVALID_ARG, "commit: must follow specdec_verify");
     StreamScope scope(h, stream);
-    return commit_impl(h, d_keep, d_next, scope.st);
+    int rc = commit_impl(h, d_keep, d_next, scope.st);
+    if (rc == 0) ++h->commits_issued;
+    return rc;
 }
 
 int specdec_get_output(specdec_handle* h, int32_t* d_out, int out_stride, int32_t* d_out_len, int32_t* d_finished,
