@@ -228,6 +228,11 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
  *   replace: 365 vs 356 us per 2-sequence verify step, 426 vs 375 us at 4 sequences);
  * "attn_rs" = 0 never / 1 choose (default) / 2 whenever the keys allow: tile attention keeps the scores in the MMA
  *   accumulators through the softmax instead of a shared-memory tile (smaller footprint, more CTAs per SM);
+ * "attn_stream" = 0 never / 1 by rule (default) / 2 always / 3 always with the two-stage ring: tile attention that
+ *   walks the keys in blocks of 64 with a running maximum (shared memory independent of the key count) instead of
+ *   staging every key at once.  Rule: where the one-shot kernel cannot hold the keys (about 590), and beyond
+ *   "attn_stream_keys" keys (default 320) when the launch has at least 4 CTAs per SM (1180 -> 942 us per
+ *   128-sequence verify step over 512-token sources; with few CTAs the block-by-block walk is the slower one);
  * "attn_warps" = 0 choose per launch, 4 or 8 warps per CTA of the tile attention (default 0);
  * "tc_bn" = 0 choose, else force the column width of the tensor-core GEMM tiles (64 / 128 / 256; experiments);
  * "cluster" = 0/1 run the verifier's decoder stack as one thread-block-cluster kernel per sequence when the

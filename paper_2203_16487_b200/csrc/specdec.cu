@@ -16,6 +16,7 @@
 
 #include "../../include/specdec.h"
 #include "attention_oproj.cuh"
+#include "attention_stream.cuh"
 #include "attention_tc.cuh"
 #include "decoder_cluster.cuh"
 #include "gemm_tc.cuh"
@@ -114,6 +115,8 @@ struct specdec_handle {
     bool pair_ready = false;
     int use_pair = 0;               // two-SM tiles (cta_group::2) for wide GEMMs over many rows (option "pair")
     int attn_rs = 1;                // tile attention keeps the scores in registers when the keys allow (option "attn_rs")
+    int attn_stream = 1;            // streaming tile attention: 0 never, 1 by rule, 2 always, 3 always with the 2-stage ring (option "attn_stream")
+    int attn_stream_keys = 320;     // option "attn_stream_keys"
     int attn_warps = 0;             // 0 = choose per launch, else 4 or 8 warps per tile-attention CTA (option "attn_warps")
     int skinny_groups = 1;          // 8-row weight groups per CTA of the weight-streaming GEMM (1, 2 or 4)
     // CUDA graphs of whole draft / verify(+commit) steps, keyed by everything their launches depend on
@@ -538,7 +541,15 @@ int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* 
     if (rows_ub <= 0) return 0;
     if constexpr (std::is_same<T, bf16>::value) {
         const size_t smem = attn_tc_smem(max_keys);
-        if (h->use_tc_attn && d_head == 64 && smem <= h->attn_tc_smem_cap) {
+        // the streaming kernel where the one-shot kernel cannot hold the keys, and where the SMs are full of CTAs
+        // and the keys are many (its small footprint keeps the occupancy up; with few CTAs its block-by-block walk
+        // is slower than one big request)
+        const long long attn_ctas = (long long)cdiv(q_ub, ATT_Q) * n_heads * h->B;
+        const bool stream = h->use_tc_attn && d_head == 64 &&
+                            (h->attn_stream >= 2 ||
+                             (h->attn_stream == 1 && (smem > h->attn_tc_smem_cap ||
+                                                      (max_keys > h->attn_stream_keys && attn_ctas >= 4LL * h->tma.n_sm))));
+        if (stream || (h->use_tc_attn && d_head == 64 && smem <= h->attn_tc_smem_cap)) {
             AttnTcArgs a;
             a.q = (const bf16*)q; a.q_stride = q_stride; a.q_index = q_index;
             a.k = (const bf16*)k; a.v = (const bf16*)v; a.kv_stride = kv_stride; a.kv_off = kv_off;
@@ -547,6 +558,16 @@ int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* 
             a.out = (bf16*)out; a.out_stride = out_stride; a.max_keys = max_keys;
             a.scale = 1.0f / sqrtf((float)d_head);
             dim3 grid(cdiv(q_ub, ATT_Q), n_heads, h->B);
+            if (stream) {          // key blocks through a ring of stages: shared memory independent of the key count
+                const bool deep = h->attn_stream != 3 && (long long)grid.x * grid.y * grid.z < 4LL * h->tma.n_sm;    // few CTAs: more bytes in flight per CTA
+                cudaError_t e = deep ? (paged ? launch_pdl(h, k_attn_stream<true, 4>, grid, dim3(128), (size_t)ats_smem(4), st, a)
+                                              : launch_pdl(h, k_attn_stream<false, 4>, grid, dim3(128), (size_t)ats_smem(4), st, a))
+                                     : (paged ? launch_pdl(h, k_attn_stream<true, 2>, grid, dim3(128), (size_t)ats_smem(2), st, a)
+                                              : launch_pdl(h, k_attn_stream<false, 2>, grid, dim3(128), (size_t)ats_smem(2), st, a));
+                if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(e));
+                KCHECK(h);
+                return 0;
+            }
             // 4 warps when the SMs are saturated with CTAs anyway, 8 when a CTA's own latency chain is what counts;
             // scores stay in registers (smaller shared memory: more CTAs per SM) when the keys fit 6 tiles per warp
             const long long ctas = (long long)grid.x * grid.y * grid.z;
@@ -953,7 +974,7 @@ void drop_graphs(specdec_handle* h) {
 inline void graph_key_tail(const specdec_handle* h, std::vector<long long>& key) {
     for (long long v : {(long long)h->use_tc, (long long)h->use_tc_attn, (long long)h->want_lse, (long long)h->use_skinny,
                         (long long)h->use_pdl, (long long)h->use_ln_fuse, (long long)h->use_ln_rows, (long long)h->use_sk_cluster,
-                        (long long)h->use_pair, (long long)h->attn_warps, (long long)h->attn_rs, (long long)h->use_fused_attn,
+                        (long long)h->use_pair, (long long)h->attn_stream, (long long)h->attn_stream_keys, (long long)h->attn_warps, (long long)h->attn_rs, (long long)h->use_fused_attn,
                         (long long)h->skinny_groups, (long long)h->use_cluster, (long long)h->want_cl_trace,
                         (long long)(h->script_on ? 1 : 0), (long long)h->B, (long long)h->S_max})
         key.push_back(v);
@@ -1331,6 +1352,8 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
     if (h->dtype == SPECDEC_DTYPE_BF16) {
         const int max_keys = std::max(h->S_cap, h->T_cap + h->k_cap + 1);
         h->attn_tc_smem_cap = std::min<size_t>(attn_tc_smem(max_keys), 227 * 1024);
+        cudaFuncSetAttribute(k_attn_stream<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, ats_smem(4));
+        cudaFuncSetAttribute(k_attn_stream<false, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, ats_smem(4));
         if (cudaFuncSetAttribute(k_attn_tc<true, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
             cudaFuncSetAttribute(k_attn_tc<false, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
             cudaFuncSetAttribute(k_attn_tc<true, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->attn_tc_smem_cap) != cudaSuccess ||
@@ -1436,6 +1459,8 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         if (value && !h->pair_ready) return fail(h, SPECDEC_ERR_UNSUPPORTED, "two-SM GEMM tiles are not available on this handle");
         h->use_pair = value ? 1 : 0; return SPECDEC_OK;
     }
+    if (!strcmp(name, "attn_stream")) { h->attn_stream = value < 0 ? 0 : (value > 3 ? 3 : value); return SPECDEC_OK; }
+    if (!strcmp(name, "attn_stream_keys")) { h->attn_stream_keys = value; return SPECDEC_OK; }
     if (!strcmp(name, "attn_rs")) { h->attn_rs = value < 0 ? 0 : (value > 2 ? 2 : value); return SPECDEC_OK; }   // 0 never, 1 choose, 2 whenever possible
     if (!strcmp(name, "attn_warps")) {
         if (value != 0 && value != 4 && value != 8) return fail(h, SPECDEC_ERR_INVALID_ARG, "attn_warps must be 0, 4 or 8");

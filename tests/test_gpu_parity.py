@@ -301,6 +301,30 @@ def test_bf16_mid_small_batches_weight_streaming_gemm(nseq, skinny):
     sd.close()
 
 
+@pytest.mark.parametrize("long_keys,mode", [(False, 2), (True, 2), (True, 3)])
+def test_bf16_streaming_attention(long_keys, mode):
+    """The streaming tile attention (key blocks of 64 through a two-stage ring, running maximum) against the
+    oracle's one-pass softmax: forced on for the short case (a single, partly filled block), and over sources of
+    up to 200 tokens and targets past 64 (several blocks, ragged last block, causal mask crossing a block edge)."""
+    dv = W.ModelDims(128, 2, 512, 2000, 2, 2, 256)
+    dd = W.ModelDims(128, 2, 512, 2000, 3, 2, 256)
+    wv, wd = W.make_weights(dv, 31, True), W.make_weights(dd, 32, True)
+    mv, md = O.model_from(dv, wv, mode="bf16"), O.model_from(dd, wd, mode="bf16")
+    rng = np.random.default_rng(9)
+    if long_keys:
+        lens, tgts, max_src, max_tgt = (150, 97, 200, 64), [90, 70, 40, 80], 200, 96
+    else:
+        lens, tgts, max_src, max_tgt = (20, 7, 33, 12), [24, 18, 9, 20], 40, 24
+    srcs = [W.zipf_ids(rng, n, 2000) for n in lens]
+    sd = _handle(dv, wv, dd, wd, True, k_max=12, max_batch=4, max_src=max_src, max_tgt=max_tgt)
+    sd.set_option("attn_stream", mode)                       # 2: four-stage ring here (few CTAs), 3: the two-stage ring
+    rep = lockstep.run(sd, mv, md, srcs, tgts, 12, 3, 1.0, margin=1e-3, check_logits_every=2)
+    print(rep.iterations, rep.draft_near_ties, rep.verify_near_ties, rep.max_logit_err, rep.max_stat_err)
+    assert rep.ok, rep.notes
+    assert rep.max_logit_err < 2e-2 and rep.max_stat_err < 2e-2
+    sd.close()
+
+
 @pytest.mark.parametrize("cluster,fused", [(1, 0), (0, 0), (0, 1)])
 def test_base_shapes_batch1_lockstep(cluster, fused):
     """One config-2 sentence at batch 1 (26-row verify block): the decoder stack as one cluster kernel
