@@ -22,6 +22,7 @@
 #include "gemm_tc.cuh"
 #include "gemm_tc_lnrows.cuh"
 #include "gemm_tc_pair.cuh"
+#include "gemm_tc_splitk.cuh"
 #include "kernels.cuh"
 #include "skinny_gemm.cuh"
 
@@ -111,6 +112,8 @@ struct specdec_handle {
     int use_ln_fuse = 0;            // option "ln_fuse": measured slower than the separate LayerNorm launch, kept for comparison
     int use_sk_cluster = 1;         // option "sk_cluster": 1 = LayerNorm-fused weight-streaming GEMMs share the normalised rows in clusters of 8; 2 = the plain ones too (measured slower)
     bool lnrows_ready = false;
+    bool splitk_ready = false;
+    int use_splitk = 1;             // residual GEMMs over <= 128 rows with K >= 1024 split K across a cluster of 4 (option "splitk")
     int use_ln_rows = 0;            // option "ln_rows": GEMMs over at most 128 rows normalise their input rows themselves (measured slower: off)
     bool pair_ready = false;
     int use_pair = 0;               // two-SM tiles (cta_group::2) for wide GEMMs over many rows (option "pair")
@@ -507,6 +510,12 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
                 if (sd::gemm_tc_launch_ln(h->tma, g, rows_ub, st) != 0)
                     return fail(h, SPECDEC_ERR_CUDA, "tensor-core GEMM launch failed: " + h->tma.err);
                 h->fused_x = resid; h->fused_g = want_ln.g; h->fused_out = want_ln.out;
+                ++h->launches;
+                return 0;
+            }
+            if (epi == EPI_RESID && h->use_splitk && h->splitk_ready && sd::spk_supported(N, K, rows_ub)) {
+                if (sd::spk_launch(h->tma, g, rows_ub, st) != 0)
+                    return fail(h, SPECDEC_ERR_CUDA, "tensor-core GEMM launch failed: " + h->tma.err);
                 ++h->launches;
                 return 0;
             }
@@ -974,7 +983,7 @@ void drop_graphs(specdec_handle* h) {
 inline void graph_key_tail(const specdec_handle* h, std::vector<long long>& key) {
     for (long long v : {(long long)h->use_tc, (long long)h->use_tc_attn, (long long)h->want_lse, (long long)h->use_skinny,
                         (long long)h->use_pdl, (long long)h->use_ln_fuse, (long long)h->use_ln_rows, (long long)h->use_sk_cluster,
-                        (long long)h->use_pair, (long long)h->attn_stream, (long long)h->attn_stream_keys, (long long)h->attn_warps, (long long)h->attn_rs, (long long)h->use_fused_attn,
+                        (long long)h->use_pair, (long long)h->use_splitk, (long long)h->attn_stream, (long long)h->attn_stream_keys, (long long)h->attn_warps, (long long)h->attn_rs, (long long)h->use_fused_attn,
                         (long long)h->skinny_groups, (long long)h->use_cluster, (long long)h->want_cl_trace,
                         (long long)(h->script_on ? 1 : 0), (long long)h->B, (long long)h->S_max})
         key.push_back(v);
@@ -1404,6 +1413,8 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
         if (sd::tc_init(h->tma, h->ses.counters + 7) != 0) h->use_tc = 0;     // reported through specdec_last_error; SIMT GEMM still runs on the GPU
         h->lnrows_ready = h->use_tc && sd::lr_init() == cudaSuccess;
         if (!h->lnrows_ready) cudaGetLastError();
+        h->splitk_ready = h->use_tc && sd::spk_init() == cudaSuccess;
+        if (!h->splitk_ready) cudaGetLastError();
         h->pair_ready = h->use_tc && sd::tc_pair_init() == cudaSuccess;
         if (!h->pair_ready) cudaGetLastError();
         if (!h->use_tc) h->err = "tensor-core GEMM unavailable: " + h->tma.err;
@@ -1459,6 +1470,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         if (value && !h->pair_ready) return fail(h, SPECDEC_ERR_UNSUPPORTED, "two-SM GEMM tiles are not available on this handle");
         h->use_pair = value ? 1 : 0; return SPECDEC_OK;
     }
+    if (!strcmp(name, "splitk")) { h->use_splitk = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "attn_stream")) { h->attn_stream = value < 0 ? 0 : (value > 3 ? 3 : value); return SPECDEC_OK; }
     if (!strcmp(name, "attn_stream_keys")) { h->attn_stream_keys = value; return SPECDEC_OK; }
     if (!strcmp(name, "attn_rs")) { h->attn_rs = value < 0 ? 0 : (value > 2 ? 2 : value); return SPECDEC_OK; }   // 0 never, 1 choose, 2 whenever possible
