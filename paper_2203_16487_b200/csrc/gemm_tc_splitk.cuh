@@ -1,5 +1,6 @@
-// Residual GEMM over at most 128 rows with a long reduction (FFN2: K = 4 d), split along K inside a cluster:
-//     resid[r, n] += x[r, :] . W[n, :] + bias[n],   x bf16 [R <= 128, K], W bf16 [N, K], resid fp32 [R, N].
+// Residual GEMM over a few 128-row tiles with a long reduction (FFN2: K = 4 d), split along K inside a cluster:
+//     resid[r, n] += x[r, :] . W[n, :] + bias[n],   x bf16 [R, K], W bf16 [N, K], resid fp32 [R, N],
+// for row counts whose tiles x N / 64 x SPLIT CTAs still fit one wave.
 //
 // With 64-wide column tiles such a GEMM has N / 64 CTAs (8 for d = 512), each walking the whole K: 32 k-blocks at
 // the tensor core's 0.35 us per block is what the kernel costs.  Here SPLIT CTAs of a cluster share one column
@@ -30,8 +31,10 @@ inline int spk_split(int K) {
         if (K % (s * TC_BK) == 0 && K / (s * TC_BK) <= SPK_MAX_KB) return s;
     return 0;
 }
-inline bool spk_supported(int N, int K, int rows_ub) {
-    return rows_ub <= TC_BM && N % SPK_BN == 0 && K >= 1024 && spk_split(K) != 0;
+inline bool spk_supported(int N, int K, int rows_ub, int n_sm) {
+    const int split = spk_split(K);
+    return split != 0 && N % SPK_BN == 0 && K >= 1024 &&
+           (long long)((rows_ub + TC_BM - 1) / TC_BM) * (N / SPK_BN) * split <= n_sm;
 }
 
 template <int SPLIT>
@@ -48,7 +51,7 @@ k_gemm_tc_splitk(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint32_t rank;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
-    const int n_tile = blockIdx.x / SPLIT, kb0 = (int)rank * nkb;
+    const int n_tile = blockIdx.x / SPLIT, kb0 = (int)rank * nkb, m0 = blockIdx.y * TC_BM;
 
     if (threadIdx.x == 0) {
         abort_s = 0;
@@ -72,10 +75,11 @@ k_gemm_tc_splitk(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
     pdl_launch_dependents();
     pdl_wait();
-    const int R = min(g.rows_static >= 0 ? g.rows_static : *g.n_rows, TC_BM);
+    // rows of this CTA's 128-row tile (none: the tile still runs, on zero-filled rows, and stores nothing)
+    const int R = min(max((g.rows_static >= 0 ? g.rows_static : *g.n_rows) - m0, 0), TC_BM);
     if (threadIdx.x == 0) {
         for (int kb = 0; kb < nkb; ++kb)
-            tma_load_2d(a_base + kb * SPK_A_KB, &tmA, (kb0 + kb) * TC_BK, 0, smem_u32(&bar_full[kb]));
+            tma_load_2d(a_base + kb * SPK_A_KB, &tmA, (kb0 + kb) * TC_BK, m0, smem_u32(&bar_full[kb]));
         if (rank == 0) mbar_expect_tx(smem_u32(&bar_part), (uint32_t)(SPLIT - 1) * R * SPK_BN * 4);
     }
     const int q = warp & 3, half = (warp - 2) >> 2, row = q * 32 + lane;
@@ -86,7 +90,7 @@ k_gemm_tc_splitk(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             bz[j] = g.bias ? __ldg(reinterpret_cast<const float4*>(g.bias + n0) + j) : make_float4(0.f, 0.f, 0.f, 0.f);
-            xin[j] = row < R ? *(reinterpret_cast<const float4*>(g.resid + (size_t)row * g.N + n0) + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+            xin[j] = row < R ? *(reinterpret_cast<const float4*>(g.resid + (size_t)(m0 + row) * g.N + n0) + j) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
     }
     bool ok = true;
@@ -142,7 +146,7 @@ k_gemm_tc_splitk(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     }
                     a.x += bz[j].x; a.y += bz[j].y; a.z += bz[j].z; a.w += bz[j].w;
                     a.x += xin[j].x; a.y += xin[j].y; a.z += xin[j].z; a.w += xin[j].w;
-                    *(reinterpret_cast<float4*>(g.resid + (size_t)row * g.N + n0) + j) = a;
+                    *(reinterpret_cast<float4*>(g.resid + (size_t)(m0 + row) * g.N + n0) + j) = a;
                 }
             }
         }
@@ -165,7 +169,7 @@ inline int spk_launch(TmaEncoder& enc, GemmArgs<bf16>& g, int rows_ub, cudaStrea
     const CUtensorMap* tw = enc.get(g.W, g.N, g.K, g.K, SPK_BN);
     if (!ta || !tw || split == 0) return -1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(g.N / SPK_BN * split); cfg.blockDim = dim3(TC_THREADS);
+    cfg.gridDim = dim3(g.N / SPK_BN * split, (rows_ub + TC_BM - 1) / TC_BM); cfg.blockDim = dim3(TC_THREADS);
     cfg.dynamicSmemBytes = spk_smem(g.K / TC_BK / split, split); cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;

@@ -113,7 +113,7 @@ struct specdec_handle {
     int use_sk_cluster = 1;         // option "sk_cluster": 1 = LayerNorm-fused weight-streaming GEMMs share the normalised rows in clusters of 8; 2 = the plain ones too (measured slower)
     bool lnrows_ready = false;
     bool splitk_ready = false;
-    int use_splitk = 1;             // residual GEMMs over <= 128 rows with K >= 1024 split K across a cluster of 4 (option "splitk")
+    int use_splitk = 1;             // residual GEMMs with K >= 1024 over few row tiles split K across a cluster of 4 / 6 CTAs (option "splitk")
     int use_ln_rows = 0;            // option "ln_rows": GEMMs over at most 128 rows normalise their input rows themselves (measured slower: off)
     bool pair_ready = false;
     int use_pair = 0;               // two-SM tiles (cta_group::2) for wide GEMMs over many rows (option "pair")
@@ -513,7 +513,7 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
                 ++h->launches;
                 return 0;
             }
-            if (epi == EPI_RESID && h->use_splitk && h->splitk_ready && sd::spk_supported(N, K, rows_ub)) {
+            if (epi == EPI_RESID && h->use_splitk && h->splitk_ready && sd::spk_supported(N, K, rows_ub, h->tma.n_sm)) {
                 if (sd::spk_launch(h->tma, g, rows_ub, st) != 0)
                     return fail(h, SPECDEC_ERR_CUDA, "tensor-core GEMM launch failed: " + h->tma.err);
                 ++h->launches;
