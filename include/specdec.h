@@ -228,6 +228,10 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
  *   replace: 365 vs 356 us per 2-sequence verify step, 426 vs 375 us at 4 sequences);
  * "attn_rs" = 0 never / 1 choose (default) / 2 whenever the keys allow: tile attention keeps the scores in the MMA
  *   accumulators through the softmax instead of a shared-memory tile (smaller footprint, more CTAs per SM);
+ * "splitk" = 0/1 residual GEMMs with K >= 1024 (FFN2) whose row tiles x N / 64 column tiles x 4 (K <= 2048) or 6
+ *   (K = 3072) CTAs fit one wave run split along K: the CTAs of a cluster share a column tile and rank 0 adds their
+ *   fp32 partials in rank order (default 1: 356 -> 324 us per 2-sequence verify step, 479 -> 416 us with 768-wide
+ *   models; encoders and the drafter's first layer gain the same way);
  * "attn_stream" = 0 never / 1 by rule (default) / 2 always / 3 always with the two-stage ring: tile attention that
  *   walks the keys in blocks of 64 with a running maximum (shared memory independent of the key count) instead of
  *   staging every key at once.  Rule: where the one-shot kernel cannot hold the keys (about 590), and beyond

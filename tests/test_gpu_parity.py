@@ -88,6 +88,43 @@ def test_config1_generate_bit_exact(tiny, beta, tau, graphs):
     sd.close()
 
 
+@pytest.mark.parametrize("opts", [
+    {"gate": 0, "poll_flag": 0},                    # plain graphs, the counter copied back after every iteration
+    {"gate": 0, "poll_flag": 0, "poll_lag": 2},     # ... read two iterations late: two wasted iterations at the end
+    {"gate": 0, "poll_flag": 1, "poll_lag": 1},     # the commit kernel's posted word, one iteration late
+    {"gate": 2, "poll_flag": 1},                    # every iteration behind a device-side IF node, host two ahead
+    {"gate": 2, "poll_flag": 0, "poll_lag": 3},
+    {"stats_timing": 1},                            # an event after every phase: separate draft / verify graphs
+    {"graphs": 0},
+])
+def test_generate_loop_variants_bit_exact(tiny, opts):
+    """Every way the host can drive the draft -> verify -> commit loop gives the oracle's sequences and counters
+    (Algorithm 1 is the same; only who waits for whom changes)."""
+    wl, wv, wd, mv, md = tiny
+    sd = _handle(wl.verifier, wv, wl.drafter, wd, False)
+    for name, val in opts.items():
+        sd.set_option(name, val)
+    src, lens = W.pad_batch(wl.src)
+    refs = [O.specdec_generate(mv, md, s, 32, wl.k, 3, 1.0, BOS, EOS, MASK) for s in wl.src]
+    for rep in range(2):                                     # the second call replays the graphs the first one built
+        out, n, st = sd.generate(src, lens, wl.max_tgt, wl.k, 3, 1.0)
+        for b, (ref, _) in enumerate(refs):
+            assert out[b, :int(n[b])].cpu().tolist() == ref
+        assert st["emitted"] == sum(len(r) for r, _ in refs)
+        assert st["accepted"] == sum(o.accepted for _, o in refs)
+        assert st["seq_iterations"] == sum(o.iterations for _, o in refs)
+        longest = max(o.iterations for _, o in refs)
+        wasted = opts.get("poll_lag", 0) if opts.get("gate", 1) == 0 else 0      # behind the gate they do not run
+        assert st["iterations"] == min(longest + wasted, 32)            # the loop never runs past max_tgt iterations
+        assert st["ms_total"] > 0 and st["ms_encode"] > 0
+        assert (st["ms_verify"] > 0) == bool(opts.get("stats_timing", 0))
+    # one sentence at a time after the batch: the posted commit count carries over between calls
+    for s, (ref, _) in zip(wl.src, refs):
+        out, n, _ = sd.generate(s[None], [len(s)], [32], wl.k, 3, 1.0)
+        assert out[0, :int(n[0])].cpu().tolist() == ref
+    sd.close()
+
+
 def test_degenerate_shapes_bit_exact(tiny):
     """One-token sources, k = 1 and k = k_max, target budgets of 0, 1 and 2 tokens in one batch, a rule that accepts
     everything (beta = V, huge tau) and the strict one: each sequence must equal the oracle's batch-1 run."""
