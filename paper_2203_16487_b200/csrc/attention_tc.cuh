@@ -101,33 +101,36 @@ __global__ void __launch_bounds__(NW * 32) k_attn_tc(AttnTcArgs a) {
 
     // ---- stage K, V of the keys that predate this step (cached prefix, encoder memory) before the wait ...
     const int npre = a.pre_keys ? min(a.pre_keys[b], nkmax) : 0;
-    for (int i = tid; i < npre * 8; i += ATT_THREADS) {
-        const int t = i >> 3, c = i & 7;
-        const size_t kr = PAGED ? a.pg.row(b, t) : (size_t)(a.kv_off[b] + t);
-        cp_async16(Ks + swz(t, c), a.k + kr * a.kv_stride + h * 64 + c * 8);
-        cp_async16(Vs + swz(t, c), a.v + kr * a.kv_stride + h * 64 + c * 8);
+    // a thread keeps its 16-byte chunk of the 128-byte head slice and walks the keys: one row lookup per request pair
+    const int c8 = tid & 7, t0 = tid >> 3;
+    constexpr int TSTEP = ATT_THREADS / 8;
+    const bf16* kcol = a.k + h * 64 + c8 * 8;
+    const bf16* vcol = a.v + h * 64 + c8 * 8;
+    for (int t = t0; t < npre; t += TSTEP) {
+        const size_t off = (PAGED ? a.pg.row(b, t) : (size_t)(a.kv_off[b] + t)) * a.kv_stride;
+        cp_async16(Ks + swz(t, c8), kcol + off);
+        cp_async16(Vs + swz(t, c8), vcol + off);
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
     pdl_launch_dependents();
     pdl_wait();                                   // ... and everything the predecessor kernels wrote after it
-    for (int i = tid; i < ATT_Q * 8; i += ATT_THREADS) {
-        const int r = i >> 3, c = i & 7;
+    for (int r = t0; r < ATT_Q; r += TSTEP) {
         if (r < nq) {
             const size_t qr = a.q_index ? (size_t)a.q_index[r0 + r] : (size_t)(r0 + r);
-            cp_async16(Qs + swz(r, c), a.q + qr * a.q_stride + h * 64 + c * 8);
+            cp_async16(Qs + swz(r, c8), a.q + qr * a.q_stride + h * 64 + c8 * 8);
         } else {
-            *reinterpret_cast<uint4*>(Qp + swz(r, c)) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4*>(Qp + swz(r, c8)) = make_uint4(0, 0, 0, 0);
         }
     }
-    for (int i = tid + npre * 8; i < nkp * 8; i += ATT_THREADS) {
-        const int t = i >> 3, c = i & 7;
+    for (int t = t0; t < nkp; t += TSTEP) {
+        if (t < npre) continue;
         if (t < nkmax) {
-            const size_t kr = PAGED ? a.pg.row(b, t) : (size_t)(a.kv_off[b] + t);
-            cp_async16(Ks + swz(t, c), a.k + kr * a.kv_stride + h * 64 + c * 8);
-            cp_async16(Vs + swz(t, c), a.v + kr * a.kv_stride + h * 64 + c * 8);
+            const size_t off = (PAGED ? a.pg.row(b, t) : (size_t)(a.kv_off[b] + t)) * a.kv_stride;
+            cp_async16(Ks + swz(t, c8), kcol + off);
+            cp_async16(Vs + swz(t, c8), vcol + off);
         } else {
-            *reinterpret_cast<uint4*>(Kp + swz(t, c)) = make_uint4(0, 0, 0, 0);
-            *reinterpret_cast<uint4*>(Vp + swz(t, c)) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4*>(Kp + swz(t, c8)) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4*>(Vp + swz(t, c8)) = make_uint4(0, 0, 0, 0);
         }
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
@@ -256,21 +259,28 @@ __global__ void __launch_bounds__(NW * 32) k_attn_tc(AttnTcArgs a) {
         }
     }
     __syncthreads();
-    // ---- softmax: NW threads per row; P (bf16, un-normalised) overwrites the K tile
+    // ---- softmax: NW threads per row, four scores at a time; P (bf16, un-normalised) overwrites the K tile
     {
         bf16* P = reinterpret_cast<bf16*>(Kp);
         const int r = tid / NW, sub = tid % NW;
-        const float* srow = Ss + r * sstr;
+        const float4* srow = reinterpret_cast<const float4*>(Ss + r * sstr);
         float m = -CUDART_INF_F;
-        for (int c = sub; c < nkp; c += NW) m = fmaxf(m, srow[c]);
+        for (int c = sub; c < nkp / 4; c += NW) {
+            const float4 s4 = srow[c];
+            m = fmaxf(m, fmaxf(fmaxf(s4.x, s4.y), fmaxf(s4.z, s4.w)));
+        }
 #pragma unroll
         for (int o = 1; o < NW; o <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        // exp(s - m) as 2^((s - m) log2 e); a masked score is -inf and gives 0, a row without keys keeps sum 0
+        const float mb = (m == -CUDART_INF_F) ? 0.f : m * 1.4426950408889634f;
         float sum = 0.f;
-        for (int c = sub; c < nkp; c += NW) {
-            const float s = srow[c];
-            const float e = (s == -CUDART_INF_F) ? 0.f : expf(s - m);
-            sum += e;
-            P[r * pstr + c] = __float2bfloat16_rn(e);
+        for (int c = sub; c < nkp / 4; c += NW) {
+            const float4 s4 = srow[c];
+            const float e0 = exp2f(fmaf(s4.x, 1.4426950408889634f, -mb)), e1 = exp2f(fmaf(s4.y, 1.4426950408889634f, -mb));
+            const float e2 = exp2f(fmaf(s4.z, 1.4426950408889634f, -mb)), e3 = exp2f(fmaf(s4.w, 1.4426950408889634f, -mb));
+            sum += (e0 + e1) + (e2 + e3);
+            __nv_bfloat162 p01 = __floats2bfloat162_rn(e0, e1), p23 = __floats2bfloat162_rn(e2, e3);
+            *reinterpret_cast<uint2*>(P + r * pstr + c * 4) = make_uint2(*reinterpret_cast<uint32_t*>(&p01), *reinterpret_cast<uint32_t*>(&p23));
         }
 #pragma unroll
         for (int o = 1; o < NW; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
@@ -307,15 +317,11 @@ __global__ void __launch_bounds__(NW * 32) k_attn_tc(AttnTcArgs a) {
         for (int half = 0; half < 2; ++half) {
             const int r = mt * 16 + g + half * 8;
             if (r < nq) {
-                const float den = s_sum[r];
+                const float den = s_sum[r], inv = den > 0.f ? 1.0f / den : 0.f;
                 bf16* o = a.out + (size_t)(r0 + r) * a.out_stride + h * 64 + wq * (NV * 16) + t4 * 2;
 #pragma unroll
-                for (int nt = 0; nt < 2 * NV; ++nt) {
-                    __nv_bfloat162 v2;
-                    v2.x = __float2bfloat16_rn(den > 0.f ? acc[nt][half * 2] / den : 0.f);
-                    v2.y = __float2bfloat16_rn(den > 0.f ? acc[nt][half * 2 + 1] / den : 0.f);
-                    *reinterpret_cast<__nv_bfloat162*>(o + nt * 8) = v2;
-                }
+                for (int nt = 0; nt < 2 * NV; ++nt)
+                    *reinterpret_cast<__nv_bfloat162*>(o + nt * 8) = __floats2bfloat162_rn(acc[nt][half * 2] * inv, acc[nt][half * 2 + 1] * inv);
             }
         }
     }

@@ -243,8 +243,10 @@ __global__ void k_layernorm(const float* __restrict__ x, const float* __restrict
 struct Paged {
     const int* table;   // [B, max_pages] page ids
     int page_tokens, max_pages;
+    // page_tokens is a power of two (checked when the handle is created): shift and mask, no integer division
     __device__ __forceinline__ size_t row(int b, int t) const {
-        return (size_t)table[b * max_pages + t / page_tokens] * page_tokens + (t % page_tokens);
+        const int sh = 31 - __clz(page_tokens);
+        return ((size_t)table[b * max_pages + (t >> sh)] << sh) + (size_t)(t & (page_tokens - 1));
     }
 };
 

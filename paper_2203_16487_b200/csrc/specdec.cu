@@ -113,6 +113,8 @@ struct specdec_handle {
     int use_sk_cluster = 1;         // option "sk_cluster": 1 = LayerNorm-fused weight-streaming GEMMs share the normalised rows in clusters of 8; 2 = the plain ones too (measured slower)
     bool lnrows_ready = false;
     bool splitk_ready = false;
+    int diag_repeat = 0;            // diagnostics: launch every attention (1) / LayerNorm (2) kernel twice (same result) to
+                                    // read its cost inside the pipeline off the step time (option "diag_repeat")
     int use_splitk = 1;             // residual GEMMs with K >= 1024 over few row tiles split K across a cluster of 4 / 6 CTAs (option "splitk")
     int use_ln_rows = 0;            // option "ln_rows": GEMMs over at most 128 rows normalise their input rows themselves (measured slower: off)
     bool pair_ready = false;
@@ -378,7 +380,9 @@ template <typename T>
 int ln_or_fused(specdec_handle* h, const float* x, const float* g, const float* b, int cnt, int rows_ub, void* y, int d,
                 cudaStream_t st) {
     if (x == h->fused_x && g == h->fused_g && y == h->fused_out) return 0;
-    return ln<T>(h, x, g, b, cnt, rows_ub, y, d, st);
+    TRY(ln<T>(h, x, g, b, cnt, rows_ub, y, d, st));
+    if (h->diag_repeat & 2) TRY(ln<T>(h, x, g, b, cnt, rows_ub, y, d, st));
+    return 0;
 }
 
 // Where the K and V columns of a fused QKV projection go (the verifier's paged cache).
@@ -544,7 +548,7 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
 // kernel (one CTA per 32-query tile, head, sequence; q_ub bounds the queries of one sequence);
 // everything else uses the warp-per-(row, head) kernel.
 template <typename T>
-int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* q_index, const void* k, const void* v,
+int attn_once(specdec_handle* h, bool paged, const void* q, int q_stride, const int* q_index, const void* k, const void* v,
          int kv_stride, const int* kv_off, const Rows& r, const int* nkeys, int cnt, int rows_ub, int q_ub, void* out,
          int out_stride, int n_heads, int d_head, int max_keys, cudaStream_t st, const int* pre_keys = nullptr) {
     if (rows_ub <= 0) return 0;
@@ -584,8 +588,11 @@ int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* 
             auto per_sm_of = [](size_t sm) { return (long long)(227 * 1024) / (long long)(sm + 1024); };
             // (measured: the register variant is slower per CTA, 357 -> 387 us per batch-1 step, and pays off only where
             // shared memory held the occupancy down: 1018 -> 873 us per step at batch 128 over a 256-token prefix)
+            // ... or where it saves a whole wave of CTAs (batch 128 over 90 keys: 5 CTAs per SM hold 740 of the 1024)
+            auto waves_of = [&](size_t sm) { const long long slots = std::max(1LL, per_sm_of(sm)) * h->tma.n_sm; return (ctas + slots - 1) / slots; };
             bool rs = nkp <= attn_tc_rs_max_keys(8) &&
-                      (h->attn_rs == 2 || (h->attn_rs == 1 && per_sm_of(smem) <= 2 && ctas > 2LL * h->tma.n_sm));
+                      (h->attn_rs == 2 || (h->attn_rs == 1 && ((per_sm_of(smem) <= 2 && ctas > 2LL * h->tma.n_sm) ||
+                                                               waves_of(attn_tc_smem_rs(max_keys)) < waves_of(smem))));
             size_t smem_l = rs ? attn_tc_smem_rs(max_keys) : smem;
             bool wide = h->attn_warps ? h->attn_warps == 8 : (per_sm_of(smem_l) <= 2 || ctas < 4LL * h->tma.n_sm);
             if (rs && !wide && nkp > attn_tc_rs_max_keys(4)) {       // too many keys for four warps' registers
@@ -623,6 +630,18 @@ int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* 
     return 0;
 }
 
+
+template <typename T>
+int attn(specdec_handle* h, bool paged, const void* q, int q_stride, const int* q_index, const void* k, const void* v,
+         int kv_stride, const int* kv_off, const Rows& r, const int* nkeys, int cnt, int rows_ub, int q_ub, void* out,
+         int out_stride, int n_heads, int d_head, int max_keys, cudaStream_t st, const int* pre_keys = nullptr) {
+    TRY(attn_once<T>(h, paged, q, q_stride, q_index, k, v, kv_stride, kv_off, r, nkeys, cnt, rows_ub, q_ub, out, out_stride,
+                     n_heads, d_head, max_keys, st, pre_keys));
+    if (h->diag_repeat & 1)
+        TRY(attn_once<T>(h, paged, q, q_stride, q_index, k, v, kv_stride, kv_off, r, nkeys, cnt, rows_ub, q_ub, out, out_stride,
+                         n_heads, d_head, max_keys, st, pre_keys));
+    return 0;
+}
 
 // With the "profile" option on, the vocabulary-projection launches are bracketed by event pairs.
 void prof_mark(specdec_handle* h, cudaStream_t st) {
@@ -983,7 +1002,7 @@ void drop_graphs(specdec_handle* h) {
 inline void graph_key_tail(const specdec_handle* h, std::vector<long long>& key) {
     for (long long v : {(long long)h->use_tc, (long long)h->use_tc_attn, (long long)h->want_lse, (long long)h->use_skinny,
                         (long long)h->use_pdl, (long long)h->use_ln_fuse, (long long)h->use_ln_rows, (long long)h->use_sk_cluster,
-                        (long long)h->use_pair, (long long)h->use_splitk, (long long)h->attn_stream, (long long)h->attn_stream_keys, (long long)h->attn_warps, (long long)h->attn_rs, (long long)h->use_fused_attn,
+                        (long long)h->use_pair, (long long)h->diag_repeat, (long long)h->use_splitk, (long long)h->attn_stream, (long long)h->attn_stream_keys, (long long)h->attn_warps, (long long)h->attn_rs, (long long)h->use_fused_attn,
                         (long long)h->skinny_groups, (long long)h->use_cluster, (long long)h->want_cl_trace,
                         (long long)(h->script_on ? 1 : 0), (long long)h->B, (long long)h->S_max})
         key.push_back(v);
@@ -1470,6 +1489,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         if (value && !h->pair_ready) return fail(h, SPECDEC_ERR_UNSUPPORTED, "two-SM GEMM tiles are not available on this handle");
         h->use_pair = value ? 1 : 0; return SPECDEC_OK;
     }
+    if (!strcmp(name, "diag_repeat")) { h->diag_repeat = value; return SPECDEC_OK; }
     if (!strcmp(name, "splitk")) { h->use_splitk = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "attn_stream")) { h->attn_stream = value < 0 ? 0 : (value > 3 ? 3 : value); return SPECDEC_OK; }
     if (!strcmp(name, "attn_stream_keys")) { h->attn_stream_keys = value; return SPECDEC_OK; }
