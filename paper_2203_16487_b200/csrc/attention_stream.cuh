@@ -150,13 +150,13 @@ __global__ void __launch_bounds__(128) k_attn_stream(AttnTcArgs a) {
             l_run[0] *= al0; l_run[1] *= al1;
 #pragma unroll
             for (int j = 0; j < 8; ++j) { acc[j][0] *= al0; acc[j][1] *= al0; acc[j][2] *= al1; acc[j][3] *= al1; }
+            constexpr float L2E = 1.4426950408889634f;
+            const float mb0 = (mn0 == -CUDART_INF_F) ? 0.f : mn0 * L2E, mb1 = (mn1 == -CUDART_INF_F) ? 0.f : mn1 * L2E;
             uint32_t pf[2][4];
 #pragma unroll
             for (int nt = 0; nt < 4; ++nt) {
-                const float e0 = (sc[nt][0] == -CUDART_INF_F) ? 0.f : expf(sc[nt][0] - mn0);
-                const float e1 = (sc[nt][1] == -CUDART_INF_F) ? 0.f : expf(sc[nt][1] - mn0);
-                const float e2 = (sc[nt][2] == -CUDART_INF_F) ? 0.f : expf(sc[nt][2] - mn1);
-                const float e3 = (sc[nt][3] == -CUDART_INF_F) ? 0.f : expf(sc[nt][3] - mn1);
+                const float e0 = exp2f(fmaf(sc[nt][0], L2E, -mb0)), e1 = exp2f(fmaf(sc[nt][1], L2E, -mb0));   // -inf scores give 0
+                const float e2 = exp2f(fmaf(sc[nt][2], L2E, -mb1)), e3 = exp2f(fmaf(sc[nt][3], L2E, -mb1));
                 l_run[0] += e0 + e1; l_run[1] += e2 + e3;
                 __nv_bfloat162 p01 = __floats2bfloat162_rn(e0, e1), p23 = __floats2bfloat162_rn(e2, e3);
                 // accumulator layout of an 8-key tile = half of the A fragment of a 16-key step
@@ -201,17 +201,14 @@ __global__ void __launch_bounds__(128) k_attn_stream(AttnTcArgs a) {
             const float m1 = mML[rr * 2], l1 = mML[rr * 2 + 1], m0 = m_run[half], l0 = l_run[half];
             const float m = fmaxf(m0, m1);
             const float f0 = (m0 == -CUDART_INF_F) ? 0.f : expf(m0 - m), f1 = (m1 == -CUDART_INF_F) ? 0.f : expf(m1 - m);
-            const float den = l0 * f0 + l1 * f1;
+            const float den = l0 * f0 + l1 * f1, inv = den > 0.f ? 1.0f / den : 0.f;
             if (r < nq) {
                 bf16* o = a.out + (size_t)(r0 + r) * a.out_stride + h * 64 + t4 * 2;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const float2 o1 = *reinterpret_cast<const float2*>(mO + rr * 64 + j * 8 + t4 * 2);
                     const float x = acc[j][half * 2] * f0 + o1.x * f1, y = acc[j][half * 2 + 1] * f0 + o1.y * f1;
-                    __nv_bfloat162 v2;
-                    v2.x = __float2bfloat16_rn(den > 0.f ? x / den : 0.f);
-                    v2.y = __float2bfloat16_rn(den > 0.f ? y / den : 0.f);
-                    *reinterpret_cast<__nv_bfloat162*>(o + j * 8) = v2;
+                    *reinterpret_cast<__nv_bfloat162*>(o + j * 8) = __floats2bfloat162_rn(x * inv, y * inv);
                 }
             }
         }

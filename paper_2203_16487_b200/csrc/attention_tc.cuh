@@ -203,13 +203,14 @@ __global__ void __launch_bounds__(NW * 32) k_attn_tc(AttnTcArgs a) {
                 float m = -CUDART_INF_F;
 #pragma unroll
                 for (int w = 0; w < NW; ++w) m = fmaxf(m, s_wmax[w * ATT_Q + row]);
+                const float mb = (m == -CUDART_INF_F) ? 0.f : m * 1.4426950408889634f;     // masked scores (-inf) give 0
                 float sum = 0.f;
 #pragma unroll
                 for (int j = 0; j < ATT_RS_TILES; ++j) {
                     const int nt = warp + j * NW;
                     if (nt < nkp / 8) {
                         const float s0 = sc[mt][j][hb * 2], s1 = sc[mt][j][hb * 2 + 1];
-                        const float e0 = (s0 == -CUDART_INF_F) ? 0.f : expf(s0 - m), e1 = (s1 == -CUDART_INF_F) ? 0.f : expf(s1 - m);
+                        const float e0 = exp2f(fmaf(s0, 1.4426950408889634f, -mb)), e1 = exp2f(fmaf(s1, 1.4426950408889634f, -mb));
                         sum += e0 + e1;
                         *reinterpret_cast<__nv_bfloat162*>(P + row * pstr + nt * 8 + t4 * 2) = __floats2bfloat162_rn(e0, e1);
                     }
@@ -237,6 +238,9 @@ __global__ void __launch_bounds__(NW * 32) k_attn_tc(AttnTcArgs a) {
                 const int r = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = ks * 2 + (lane >> 4);
                 ldsm_x4(Qs + swz(r, c), qf[mt][ks][0], qf[mt][ks][1], qf[mt][ks][2], qf[mt][ks][3]);
             }
+        int nkr[2][2];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) { nkr[mt][0] = s_nk[mt * 16 + g]; nkr[mt][1] = s_nk[mt * 16 + g + 8]; }
         for (int nt = warp; nt < nkp / 8; nt += ATT_THREADS / 32) {
             uint32_t kf[2][4];
 #pragma unroll
@@ -250,11 +254,11 @@ __global__ void __launch_bounds__(NW * 32) k_attn_tc(AttnTcArgs a) {
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) mma_bf16(acc, qf[mt][ks], kf[ks >> 1][(ks & 1) * 2], kf[ks >> 1][(ks & 1) * 2 + 1]);
                 const int ra = mt * 16 + g, rb = ra + 8, col = nt * 8 + t4 * 2;
-                const int na = s_nk[ra], nb = s_nk[rb];
-                Ss[ra * sstr + col] = (col < na) ? acc[0] * a.scale : -CUDART_INF_F;
-                Ss[ra * sstr + col + 1] = (col + 1 < na) ? acc[1] * a.scale : -CUDART_INF_F;
-                Ss[rb * sstr + col] = (col < nb) ? acc[2] * a.scale : -CUDART_INF_F;
-                Ss[rb * sstr + col + 1] = (col + 1 < nb) ? acc[3] * a.scale : -CUDART_INF_F;
+                const int na = nkr[mt][0], nb = nkr[mt][1];
+                *reinterpret_cast<float2*>(Ss + ra * sstr + col) =
+                    make_float2((col < na) ? acc[0] * a.scale : -CUDART_INF_F, (col + 1 < na) ? acc[1] * a.scale : -CUDART_INF_F);
+                *reinterpret_cast<float2*>(Ss + rb * sstr + col) =
+                    make_float2((col < nb) ? acc[2] * a.scale : -CUDART_INF_F, (col + 1 < nb) ? acc[3] * a.scale : -CUDART_INF_F);
             }
         }
     }
