@@ -468,7 +468,9 @@ int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, cons
          const int* ld_id = nullptr, int* n_tiles_out = nullptr, const KvDest* kv = nullptr,
          const LnSpec* lnp = nullptr) {
     if (rows_ub <= 0) return 0;
-    const bool skinny = skinny_ok<T>(h, epi, rows_ub, N, K, lnp != nullptr);
+    // (not in the encoders: the two encoders run side by side on two streams, and the weight-streaming kernels' 64-256
+    // CTAs per launch get in each other's way there -- 440 us against 386 us with 8-32-CTA tile GEMMs for a 32-token source)
+    const bool skinny = cnt != CNT_ENC && skinny_ok<T>(h, epi, rows_ub, N, K, lnp != nullptr);
     // At most 128 rows on the tensor-core path: the GEMM normalises its input rows itself (gemm_tc_lnrows.cuh)
     bool ln_rows = false;
     if constexpr (std::is_same<T, bf16>::value)
