@@ -113,7 +113,7 @@ struct specdec_handle {
     int use_sk_cluster = 1;         // option "sk_cluster": 1 = LayerNorm-fused weight-streaming GEMMs share the normalised rows in clusters of 8; 2 = the plain ones too (measured slower)
     bool lnrows_ready = false;
     bool splitk_ready = false;
-    int diag_repeat = 0;            // diagnostics: launch every attention (1) / LayerNorm (2) kernel twice (same result) to
+    int diag_repeat = 0;            // diagnostics: launch every attention (1) / LayerNorm (2) / non-residual GEMM (4) / vocabulary (8) kernel twice (same result) to
                                     // read its cost inside the pipeline off the step time (option "diag_repeat")
     int use_splitk = 1;             // residual GEMMs with K >= 1024 over few row tiles split K across a cluster of 4 / 6 CTAs (option "splitk")
     int use_ln_rows = 0;            // option "ln_rows": GEMMs over at most 128 rows normalise their input rows themselves (measured slower: off)
@@ -463,10 +463,28 @@ cudaError_t skinny_attr_mt(int bytes) { return skinny_attr<EPI, 2>(bytes); }
 
 // out = A W^T (+bias) with one of the epilogues; rows_ub bounds the grid, the live count is on the device.
 template <typename T>
+int gemm_once(specdec_handle* h, int epi, const void* A, int lda, const void* W, const float* bias, int N, int K, int cnt,
+              int rows_ub, void* out, int ldo, float* resid, cudaStream_t st, const float* ldv, const int* ld_id,
+              int* n_tiles_out, const KvDest* kv, const LnSpec* lnp);
+
+template <typename T>
 int gemm(specdec_handle* h, int epi, const void* A, int lda, const void* W, const float* bias, int N, int K, int cnt,
          int rows_ub, void* out, int ldo, float* resid, cudaStream_t st, const float* ldv = nullptr,
          const int* ld_id = nullptr, int* n_tiles_out = nullptr, const KvDest* kv = nullptr,
          const LnSpec* lnp = nullptr) {
+    TRY(gemm_once<T>(h, epi, A, lda, W, bias, N, K, cnt, rows_ub, out, ldo, resid, st, ldv, ld_id, n_tiles_out, kv, lnp));
+    // diagnostics: GEMMs that only write outputs (no residual accumulation) can run twice with the same result
+    if ((h->diag_repeat & 4) && epi != EPI_RESID && epi != EPI_STATS)
+        TRY(gemm_once<T>(h, epi, A, lda, W, bias, N, K, cnt, rows_ub, out, ldo, resid, st, ldv, ld_id, n_tiles_out, kv, lnp));
+    if ((h->diag_repeat & 8) && epi == EPI_STATS)
+        TRY(gemm_once<T>(h, epi, A, lda, W, bias, N, K, cnt, rows_ub, out, ldo, resid, st, ldv, ld_id, n_tiles_out, kv, lnp));
+    return 0;
+}
+
+template <typename T>
+int gemm_once(specdec_handle* h, int epi, const void* A, int lda, const void* W, const float* bias, int N, int K, int cnt,
+              int rows_ub, void* out, int ldo, float* resid, cudaStream_t st, const float* ldv, const int* ld_id,
+              int* n_tiles_out, const KvDest* kv, const LnSpec* lnp) {
     if (rows_ub <= 0) return 0;
     // (not in the encoders: the two encoders run side by side on two streams, and the weight-streaming kernels' 64-256
     // CTAs per launch get in each other's way there -- 440 us against 386 us with 8-32-CTA tile GEMMs for a 32-token source)

@@ -2,6 +2,7 @@
 
   python -m paper_2203_16487_b200.diagnostics --cluster-trace   # per-phase time inside the cluster decoder kernel
   python -m paper_2203_16487_b200.diagnostics --vocab-trace     # time line of one CTA of the vocabulary GEMM
+  python -m paper_2203_16487_b200.diagnostics --boundary-probe  # cost of a dependency between two small kernels, two ways to wait
   python -m paper_2203_16487_b200.diagnostics --ingest-probe    # bytes per second one / eight / all SMs can pull from HBM
 
 The traces use the library's "cl_trace" option: the kernels record the global nanosecond timer at a few
@@ -80,11 +81,20 @@ def ingest_probe():
     subprocess.check_call([exe])
 
 
+def boundary_probe():
+    here = os.path.dirname(os.path.abspath(__file__))
+    exe = "/tmp/specdec_boundary_probe"
+    subprocess.check_call(["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-o", exe,
+                           os.path.join(here, "csrc", "boundary_probe.cu")])
+    subprocess.check_call([exe])
+
+
 if __name__ == "__main__":
     ap = argparse.ArgumentParser()
     ap.add_argument("--cluster-trace", action="store_true")
     ap.add_argument("--vocab-trace", action="store_true")
     ap.add_argument("--ingest-probe", action="store_true")
+    ap.add_argument("--boundary-probe", action="store_true")
     ap.add_argument("--batch", type=int, default=1, help="vocab trace: sequences in the verify step")
     ap.add_argument("--opt", action="append", default=[], help="library option name=value (repeatable), vocab trace only")
     a = ap.parse_args()
@@ -94,3 +104,5 @@ if __name__ == "__main__":
         vocab_trace(batch=a.batch, opts=[(o.split("=")[0], int(o.split("=")[1])) for o in a.opt])
     if a.ingest_probe:
         ingest_probe()
+    if a.boundary_probe:
+        boundary_probe()
