@@ -160,10 +160,8 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
             }
         }
         // rows past the end are zeroed locally by the idle warps
-        for (int i = tid; i < (MT * 16 - R) * (K / 8); i += SK_WARPS * 32) {
-            const int mm = R + i / (K / 8), c = i % (K / 8);
-            *reinterpret_cast<uint4*>(As + (size_t)mm * pitch + c * 8) = make_uint4(0, 0, 0, 0);
-        }
+        for (int mm = R + warp; mm < MT * 16; mm += SK_WARPS)
+            for (int c = lane; c < K / 8; c += 32) *reinterpret_cast<uint4*>(As + (size_t)mm * pitch + c * 8) = make_uint4(0, 0, 0, 0);
         mbar_wait(smem_u32(&row_bar), 0, &row_abort, a.err_word, 8);             // the peers' rows have landed
     } else if (LN) {
         // each warp normalises rows warp, warp + 8, ...; all of its rows are fetched first (one round trip)
@@ -237,16 +235,18 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
                     if (rk != rank) sk_st_peer16(la, smem_u32(&row_bar), rk, v);
             }
         }
-        for (int i = tid; i < (MT * 16 - R) * (K / 8); i += SK_WARPS * 32) {
-            const int mm = R + i / (K / 8), c = i % (K / 8);
-            *reinterpret_cast<uint4*>(As + (size_t)mm * pitch + c * 8) = make_uint4(0, 0, 0, 0);
-        }
+        for (int mm = R + warp; mm < MT * 16; mm += SK_WARPS)
+            for (int c = lane; c < K / 8; c += 32) *reinterpret_cast<uint4*>(As + (size_t)mm * pitch + c * 8) = make_uint4(0, 0, 0, 0);
         mbar_wait(smem_u32(&row_bar), 0, &row_abort, a.err_word, 8);
     } else {
         const uint32_t as_base = (uint32_t)__cvta_generic_to_shared(As);
         const int chunks = K / 8;
+        // (row, 16-byte piece) of request i without an integer division where K / 8 is a power of two (it is for the
+        // usual widths; up to 32 requests per thread when K = 2048)
+        const bool p2 = (chunks & (chunks - 1)) == 0;
+        const int sh = 31 - __clz(chunks);
         for (int i = tid; i < MT * 16 * chunks; i += SK_WARPS * 32) {
-            const int m = i / chunks, c = i % chunks;
+            const int m = p2 ? (i >> sh) : i / chunks, c = p2 ? (i & (chunks - 1)) : i % chunks;
             if (m < R) cp_async16(as_base + (uint32_t)(m * pitch + c * 8) * 2, g.A + (size_t)m * g.lda + c * 8);
             else *reinterpret_cast<uint4*>(As + (size_t)m * pitch + c * 8) = make_uint4(0, 0, 0, 0);
         }
