@@ -36,7 +36,11 @@ __device__ __forceinline__ void sk_stamp(long long* trace, int slot) {
 constexpr int SK_NB = 8;         // weight rows per 8-row group
 constexpr int SK_WARPS = 8;
 // G groups of 8 weight rows per CTA; the 8 warps are G groups x (8 / G) K-splits
-inline size_t skinny_smem(int MT, int K) { return (size_t)MT * 16 * (K + 8) * 2 + (size_t)SK_WARPS * MT * 16 * SK_NB * 4; }
+// Row pitch of the activation tile in shared memory: K + 32 bf16, i.e. 16 words past a multiple of 32.  A quarter warp
+// (rows g, g + 1 x the four 16-byte pieces of a super-step) then reads all 32 banks once per 16-byte load; with the
+// earlier K + 8 and 8-byte loads every load was a 4-way bank conflict (the MMA phase of FFN2 took 2.6 us).
+constexpr int SK_PAD = 32;
+inline size_t skinny_smem(int MT, int K) { return (size_t)MT * 16 * (K + SK_PAD) * 2 + (size_t)SK_WARPS * MT * 16 * SK_NB * 4; }
 
 // CL (with LN, clusters of 8 CTAs along the weight rows): every CTA of the grid needs the same normalised rows, and
 // 200 CTAs each reading the same 26 x 2 KB at the same moment queue up on the same L2 lines.  With CL each CTA of a
@@ -69,7 +73,7 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
     constexpr int SPL = SK_WARPS / G;                          // K-splits per group
     const int grp = warp % G, spl = warp / G;
     const int n0 = blockIdx.x * (SK_NB * G);                  // first weight row of this CTA
-    const int pitch = K + 8;                                  // bf16 elements per activation row in shared memory
+    const int pitch = K + SK_PAD;                             // bf16 elements per activation row in shared memory
     bf16* As = reinterpret_cast<bf16*>(sk_sm);
     float* red = reinterpret_cast<float*>(sk_sm + (size_t)MT * 16 * pitch * 2);
 
@@ -266,14 +270,13 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
         auto step = [&](const uint4& w, int k0) {
             const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-            for (int j = 0; j < 2; ++j) {
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    const uint2 lo = *reinterpret_cast<const uint2*>(As + (size_t)(mt * 16 + gq) * pitch + k0 + t4 * 8 + j * 4);
-                    const uint2 hi = *reinterpret_cast<const uint2*>(As + (size_t)(mt * 16 + gq + 8) * pitch + k0 + t4 * 8 + j * 4);
-                    const uint32_t af[4] = {lo.x, hi.x, lo.y, hi.y};
-                    mma_bf16(acc[mt], af, wv[2 * j], wv[2 * j + 1]);
-                }
+            for (int mt = 0; mt < MT; ++mt) {
+                // the lane's 8 consecutive k of rows g and g + 8: both MMAs of the super-step from one 16-byte load each
+                const uint4 lo = *reinterpret_cast<const uint4*>(As + (size_t)(mt * 16 + gq) * pitch + k0 + t4 * 8);
+                const uint4 hi = *reinterpret_cast<const uint4*>(As + (size_t)(mt * 16 + gq + 8) * pitch + k0 + t4 * 8);
+                const uint32_t a0[4] = {lo.x, hi.x, lo.y, hi.y}, a1[4] = {lo.z, hi.z, lo.w, hi.w};
+                mma_bf16(acc[mt], a0, wv[0], wv[1]);
+                mma_bf16(acc[mt], a1, wv[2], wv[3]);
             }
         };
         // chunks of MAX_SS super-steps: the next chunk's weights are in flight while this one is multiplied
