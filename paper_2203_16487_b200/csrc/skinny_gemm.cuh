@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
 #pragma unroll
     for (int ss = 0; ss < MAX_SS; ++ss) {
         const int k0 = k_begin + ss * 32;
-        wreg[ss] = (w_ok && spl < nsplit && k0 < k_end) ? __ldg(reinterpret_cast<const uint4*>(wrow + k0)) : make_uint4(0, 0, 0, 0);
+        wreg[ss] = (w_ok && spl < nsplit && k0 < k_end) ? ldg_pinned(reinterpret_cast<const uint4*>(wrow + k0)) : make_uint4(0, 0, 0, 0);
     }
 
     // bias and LayerNorm parameters are weights too: fetch them before waiting for the predecessor
@@ -118,6 +118,13 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
     pdl_wait();
     sk_stamp(a.trace, 2);
     const int R = min(g.rows_static >= 0 ? g.rows_static : *g.n_rows, MT * 16);   // a device-side count is itself written earlier in the step
+    // residual epilogue with one output per thread: its old value is requested now, not after the products
+    constexpr bool ONE_OUT = (MT * 16 * SK_NB * G == SK_WARPS * 32);
+    float x_old = 0.f;
+    if (EPI == EPI_RESID && ONE_OUT) {
+        const int r = tid / (SK_NB * G), n = n0 + (tid % (SK_NB * G));
+        if (r < R && n < N) x_old = g.resid[(size_t)r * N + n];
+    }
     // ---- activation rows into shared memory
     if (LN && CL) {
         uint32_t rank;
@@ -261,13 +268,17 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
     sk_stamp(a.trace, 3);
 
     // ---- products: per super-step of 32 k, two MMAs per 16-row tile
-    float acc[MT][4];
+    // four accumulator chains per 16-row tile (the two MMAs of a super-step x even / odd super-steps): an mma.sync takes
+    // on the order of 100 clocks to return here, and one chain of 2 K / 32 / 8 dependent MMAs was most of this phase
+    float acc4[MT][4][4];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) acc[mt][e] = 0.f;
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc4[mt][c][e] = 0.f;
     if (spl < nsplit) {
-        auto step = [&](const uint4& w, int k0) {
+        auto step = [&](const uint4& w, int k0, int par) {
             const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
@@ -275,8 +286,8 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
                 const uint4 lo = *reinterpret_cast<const uint4*>(As + (size_t)(mt * 16 + gq) * pitch + k0 + t4 * 8);
                 const uint4 hi = *reinterpret_cast<const uint4*>(As + (size_t)(mt * 16 + gq + 8) * pitch + k0 + t4 * 8);
                 const uint32_t a0[4] = {lo.x, hi.x, lo.y, hi.y}, a1[4] = {lo.z, hi.z, lo.w, hi.w};
-                mma_bf16(acc[mt], a0, wv[0], wv[1]);
-                mma_bf16(acc[mt], a1, wv[2], wv[3]);
+                mma_bf16(acc4[mt][par * 2], a0, wv[0], wv[1]);
+                mma_bf16(acc4[mt][par * 2 + 1], a1, wv[2], wv[3]);
             }
         };
         // chunks of MAX_SS super-steps: the next chunk's weights are in flight while this one is multiplied
@@ -291,12 +302,17 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
 #pragma unroll
             for (int ss = 0; ss < MAX_SS; ++ss) {
                 const int k0 = cb + ss * 32;
-                if (k0 < k_end) step(wreg[ss], k0);
+                if (k0 < k_end) step(wreg[ss], k0, ss & 1);
             }
 #pragma unroll
             for (int ss = 0; ss < MAX_SS; ++ss) wreg[ss] = wnext[ss];
         }
     }
+    float acc[MT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[mt][e] = (acc4[mt][0][e] + acc4[mt][1][e]) + (acc4[mt][2][e] + acc4[mt][3][e]);
     sk_stamp(a.trace, 4);
     // ---- fixed-order sum over the K split, then the epilogue
 #pragma unroll
@@ -315,7 +331,7 @@ __global__ void __launch_bounds__(SK_WARPS * 32) k_skinny(SkinnyArgs a) {
         if (EPI == EPI_STORE) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(v);
         if (EPI == EPI_RELU) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(fmaxf(v, 0.f));
         if (EPI == EPI_GELU) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(ffn_act(v, 1));
-        if (EPI == EPI_RESID) g.resid[(size_t)r * N + n] += v;
+        if (EPI == EPI_RESID) { if (ONE_OUT) g.resid[(size_t)r * N + n] = x_old + v; else g.resid[(size_t)r * N + n] += v; }
         if (EPI == EPI_QKV) {
             if (n < g.kv_d) g.out[(size_t)r * g.ldo + n] = __float2bfloat16_rn(v);
             else {
