@@ -396,7 +396,8 @@ template <typename T> bool tc_usable(const specdec_handle* h, int N, int K) {
 struct LnSpec { const float* x; const float* g; const float* b; };
 
 // The weight-streaming kernel serves bf16 GEMMs over at most 32 rows (see skinny_gemm.cuh; 64-row variants of its
-// row-sharing LayerNorm kernels were tried too: 422 vs 356 us per 2-sequence verify step): measured on a
+// row-sharing LayerNorm kernels were tried too: 422 vs 356 us per 2-sequence verify step, and 360 vs 315 us after the
+// kernel's bank conflicts were gone): measured on a
 // verify step, 26 rows take 362 us with it against 391 us with 64-wide tensor-core tiles, but 52 rows take
 // 500 us against 391 us, so anything beyond two 16-row tiles goes to the tile GEMM.
 constexpr int SK_ROWS_MAX = 32;
