@@ -870,8 +870,7 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
     const size_t e = h->esz;
     const int len_ub = std::min(h->len_ub, h->T_cap);
     const int R1 = B * (len_ub + 1 + k), R2 = B * k, max_keys = len_ub + 1 + k;
-    k_draft_prep<<<1, 256, (2 * B + 2) * sizeof(int), st>>>(h->ses, B, k, h->S_max, h->cfg.bos_id, h->cfg.mask_id,
-                                                          h->rows, h->mrows);
+    k_draft_prep<<<B, 128, 0, st>>>(h->ses, B, k, h->S_max, h->cfg.bos_id, h->cfg.mask_id, h->rows, h->mrows);
     KCHECK(h);
     TRY(embed<T>(h, m, h->rows, m.pos_dec, CNT_DRAFT_ALL, R1, st));
     for (int l = 0; l + 1 < L; ++l) {
