@@ -228,6 +228,9 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
  *   replace: 365 vs 356 us per 2-sequence verify step, 426 vs 375 us at 4 sequences);
  * "attn_rs" = 0 never / 1 choose (default) / 2 whenever the keys allow: tile attention keeps the scores in the MMA
  *   accumulators through the softmax instead of a shared-memory tile (smaller footprint, more CTAs per SM);
+ * "diag_repeat" = bit mask, diagnostics: launch every attention (1), LayerNorm (2), GEMM without residual
+ *   accumulation (4) or vocabulary kernel (8) twice in a row -- same result -- so that the step time rises by that
+ *   class's cost inside the pipeline (default 0);
  * "splitk" = 0/1 residual GEMMs with K >= 1024 (FFN2) whose row tiles x N / 64 column tiles x 4 (K <= 2048) or 6
  *   (K = 3072) CTAs fit one wave run split along K: the CTAs of a cluster share a column tile and rank 0 adds their
  *   fp32 partials in rank order (default 1: 356 -> 324 us per 2-sequence verify step, 479 -> 416 us with 768-wide
