@@ -609,11 +609,9 @@ int attn_once(specdec_handle* h, bool paged, const void* q, int q_stride, const 
             auto per_sm_of = [](size_t sm) { return (long long)(227 * 1024) / (long long)(sm + 1024); };
             // (measured: the register variant is slower per CTA, 357 -> 387 us per batch-1 step, and pays off only where
             // shared memory held the occupancy down: 1018 -> 873 us per step at batch 128 over a 256-token prefix)
-            // ... or where it saves a whole wave of CTAs (batch 128 over 90 keys: 5 CTAs per SM hold 740 of the 1024)
-            auto waves_of = [&](size_t sm) { const long long slots = std::max(1LL, per_sm_of(sm)) * h->tma.n_sm; return (ctas + slots - 1) / slots; };
+            // (choosing it wherever it saves a wave of CTAs was tried too: 479 vs 469 us per 128-sequence draft step)
             bool rs = nkp <= attn_tc_rs_max_keys(8) &&
-                      (h->attn_rs == 2 || (h->attn_rs == 1 && ((per_sm_of(smem) <= 2 && ctas > 2LL * h->tma.n_sm) ||
-                                                               waves_of(attn_tc_smem_rs(max_keys)) < waves_of(smem))));
+                      (h->attn_rs == 2 || (h->attn_rs == 1 && per_sm_of(smem) <= 2 && ctas > 2LL * h->tma.n_sm));
             size_t smem_l = rs ? attn_tc_smem_rs(max_keys) : smem;
             bool wide = h->attn_warps ? h->attn_warps == 8 : (per_sm_of(smem_l) <= 2 || ctas < 4LL * h->tma.n_sm);
             if (rs && !wide && nkp > attn_tc_rs_max_keys(4)) {       // too many keys for four warps' registers
