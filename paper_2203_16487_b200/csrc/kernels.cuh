@@ -684,7 +684,17 @@ __global__ void k_draft_argmax(const RowPart* __restrict__ part, int n_tiles, co
     if (row >= *n_rows) return;
     const RowPart* p = part + (size_t)row * n_tiles;
     float mx = -CUDART_INF_F; int arg = 0x7fffffff;
-    for (int t = lane; t < n_tiles; t += 32) {
+    const int slot_of_row = slot[row];              // written before the step's kernel chain; requested with the partials
+    int t = lane;
+    for (; t + 224 < n_tiles; t += 256) {           // eight independent loads in flight (merge order unchanged)
+        RowPart q[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) q[i] = p[t + 32 * i];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (q[i].mx > mx || (q[i].mx == mx && q[i].arg < arg)) { mx = q[i].mx; arg = q[i].arg; }
+    }
+    for (; t < n_tiles; t += 32) {
         RowPart q = p[t];
         if (q.mx > mx || (q.mx == mx && q.arg < arg)) { mx = q.mx; arg = q.arg; }
     }
@@ -694,7 +704,7 @@ __global__ void k_draft_argmax(const RowPart* __restrict__ part, int n_tiles, co
         int oa = __shfl_xor_sync(0xffffffffu, arg, o);
         if (om > mx || (om == mx && oa < arg)) { mx = om; arg = oa; }
     }
-    if (lane == 0) draft[slot[row]] = arg;
+    if (lane == 0) draft[slot_of_row] = arg;
 }
 
 // Scripted drafts (benchmark / test hook): draft i of a sequence with j committed tokens is
