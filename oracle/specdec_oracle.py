@@ -34,7 +34,9 @@ beta and tau; block-parallel == sequential rows; cached == from scratch; the
 worked example's iteration structure; the parameter count implied by the
 paper's memory table; a closed-form model with zeroed sublayers; the whole
 encoder / decoder stack against torch.nn's pre-LN Transformer layers in fp64
-(ReLU and GELU); every weight shown to influence the output.
+(ReLU and GELU); every weight shown to influence the output; the points at
+which mode="bf16" rounds (a recorder in place of bf16_round); decision_margins
+on hand-worked rows.
 Parity unpinned: nothing about translation quality (needs trained weights).
 """
 from __future__ import annotations

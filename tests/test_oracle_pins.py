@@ -369,3 +369,133 @@ def test_batch_of_independent_sequences_and_modes(tiny):
     lp = O.decoder_rows(mp, [BOS, 4, 5, 6], O.encode(mp, src), True)
     lb = O.decoder_rows(mb, [BOS, 4, 5, 6], O.encode(mb, src), True)
     assert 0 < np.abs(lp - lb).max() < 2e-2
+
+
+# ---------------------------------------------------------------- near-tie classification helper
+def test_decision_margins_hand_cases():
+    """decision_margins on rows written by hand; every expected triple below was worked out on paper.
+
+    Row values (index = token id):  [5.0, 4.0, 3.0, 2.0, 1.0, 0.0]
+    """
+    row = np.array([5.0, 4.0, 3.0, 2.0, 1.0, 0.0], np.float32)
+    inf = float("inf")
+    # beta = 2: the draft must have fewer than 2 entries above it.
+    # draft = token 1 (4.0): one entry above -> accepted by rank; it flips when it drops to the best outsider, 3.0:
+    # rank margin 1.0.  tau = 1.25: (5 - 4) - 1.25 = -0.25 -> tau margin 0.25.  top-1 minus top-2 = 1.0.
+    assert O.decision_margins(row, 1, 2, 1.25) == pytest.approx((1.0, 0.25, 1.0))
+    # draft = token 2 (3.0): two entries above -> rejected by rank; it flips when it reaches the 2nd value, 4.0:
+    # rank margin 1.0.  tau = 1.75: (5 - 3) - 1.75 = +0.25 -> 0.25.
+    assert O.decision_margins(row, 2, 2, 1.75) == pytest.approx((1.0, 0.25, 1.0))
+    # a draft 0.25 above the (beta+1)-th value: beta = 3, values [5, 4, 3.25(draft), 3, ...]
+    r2 = np.array([5.0, 4.0, 3.0, 3.25, 1.0], np.float32)
+    assert O.decision_margins(r2, 3, 3, 10.0) == pytest.approx((0.25, 10.0 - 1.75, 1.0))
+    # a draft 0.25 below the beta-th value: beta = 2, values [5, 4, 3.75(draft)]
+    r3 = np.array([5.0, 3.75, 4.0], np.float32)
+    assert O.decision_margins(r3, 1, 2, 0.0) == pytest.approx((0.25, 1.25, 1.0))
+    # the draft is the top-1 itself with beta = 1: it flips when it falls to the runner-up
+    assert O.decision_margins(row, 0, 1, 0.0) == pytest.approx((1.0, 0.0, 1.0))
+    # two-way tie at the top: the argmax gap is 0; a tied draft is accepted under beta = 1 (no entry strictly above)
+    # and sits exactly on the outsider's value (margin 0)
+    r4 = np.array([2.0, 7.0, 7.0, 1.0], np.float32)
+    assert O.decision_margins(r4, 2, 1, 0.0) == pytest.approx((0.0, 0.0, 0.0))
+    # beta as large as the vocabulary: nothing can push the draft out by rank
+    assert O.decision_margins(row, 5, 6, 2.0)[0] == inf
+    # the bonus row has no draft: only the argmax gap applies
+    assert O.decision_margins(row, None, 3, 1.0) == (inf, inf, 1.0)
+    # consistency with the rule itself: moving the draft's logit across the rank margin flips accept_length
+    for tok, beta in [(1, 2), (2, 2), (3, 3), (4, 1)]:
+        m_rank, _, _ = O.decision_margins(row, tok, beta, 1e9)
+        before = O.accept_length(row[None], [tok], beta, 1e9)
+        for sign in (+1, -1):
+            moved = row.copy(); moved[tok] += sign * (m_rank + 0.01)
+            after = O.accept_length(moved[None], [tok], beta, 1e9)
+            if (sign > 0) == (before == 0):        # towards the threshold: must flip
+                assert after != before, (tok, beta, sign)
+        short = row.copy(); short[tok] += (0.5 * m_rank if before == 0 else -0.5 * m_rank)
+        assert O.accept_length(short[None], [tok], beta, 1e9) == before
+
+
+# ---------------------------------------------------------------- where mode="bf16" rounds
+def test_bf16_mode_rounds_exactly_the_contraction_operands(monkeypatch):
+    """The bf16 mode may round only values that the CUDA path feeds to a tensor-core contraction as a bf16 operand:
+    normalised activations, Q / K / V (cached and new), the un-normalised probabilities exp(s - max), the attention
+    output, the feed-forward activation output, the encoder memory and the cross-attention K / V.  Logits and the
+    residual stream are never rounded (Section 3.2: the rule is evaluated on the verifier's scores as computed).
+
+    The rounding routine is replaced by a recorder; what it is handed is recognised by shape and by properties that
+    follow from the definition of each quantity (unit LayerNorm gains: zero mean, unit variance rows; probabilities:
+    row maximum exactly 1, all in (0, 1]; ReLU output: non-negative with zeros)."""
+    import inspect
+    d, H, F, V, L = 32, 2, 96, 50, 2
+    dims = W.ModelDims(d, H, F, V, 1, L, 32)
+    w = W.make_weights(dims, 5, False)
+    for n in w:
+        if ".ln" in n or "ln_f" in n:
+            w[n] = np.ones_like(w[n]) if n.endswith(".g") else np.zeros_like(w[n])
+    calls = []
+    real = O.bf16_round
+
+    def recorder(a):
+        fn = next(f.function for f in inspect.stack()[2:] if f.function != "<genexpr>")     # the oracle function that rounds
+        calls.append((fn, np.array(a, copy=True)))
+        return real(a)
+
+    monkeypatch.setattr(O, "bf16_round", recorder)
+    m = O.model_from(dims, w, mode="bf16")
+    S, j, T = 7, 3, 5
+    src = list(range(4, 4 + S))
+
+    def is_ln(a):
+        return a.shape[-1] == d and np.allclose(a.mean(-1), 0, atol=1e-5) and np.allclose(a.var(-1), 1, atol=1e-3)
+
+    def is_prob(a, keys):
+        return a.shape[-1] == keys and np.all(a.max(-1) == 1.0) and np.all(a >= 0) and np.all(a <= 1)
+
+    # ---- encoder: per layer LN, q, k, v, H probability tiles, attention output, LN, activation; then the memory
+    mem = O.encode(m, src)
+    kinds = [(f, a.shape) for f, a in calls]
+    per_enc = [("encode", (S, d))] * 4 + [("attention", (S, S))] * H + [("encode", (S, d))] * 2 + [("ffn", (S, F))]
+    assert kinds == per_enc * dims.enc_layers + [("encode", (S, d))]
+    assert is_ln(calls[0][1]) and is_ln(calls[4 + H + 1][1]) and is_ln(calls[-1][1])
+    assert all(is_prob(a, S) for f, a in calls if f == "attention")
+    act = [a for f, a in calls if f == "ffn"][0]
+    assert act.min() == 0.0 and (act == 0).mean() > 0.2
+    assert np.array_equal(mem, real(calls[-1][1]))                       # the memory is the rounded final LayerNorm
+    # ---- cross K / V once per decoder layer
+    calls.clear()
+    cache = O.new_cache(m, mem)
+    assert [(f, a.shape) for f, a in calls] == [("new_cache", (S, d))] * (2 * L)
+    # ---- a cached causal block of T rows after j cached positions
+    O.decoder_rows(m, [1] + list(range(4, 4 + j - 1)), mem, True, cache)
+    calls.clear()
+    logits = O.decoder_rows(m, list(range(9, 9 + T)), mem, True, cache)
+    kinds = [(f, a.shape) for f, a in calls]
+    per_dec = ([("decoder_rows", (T, d))] * 4 + [("attention", (T, j + T))] * H + [("decoder_rows", (T, d))] * 3
+               + [("attention", (T, S))] * H + [("decoder_rows", (T, d))] * 2 + [("ffn", (T, F))])
+    assert kinds == per_dec * L + [("decoder_rows", (T, d))]
+    n_per = len(per_dec)
+    for l in range(L):
+        blk = calls[l * n_per:(l + 1) * n_per]
+        assert is_ln(blk[0][1]) and is_ln(blk[4 + H + 1][1]) and is_ln(blk[4 + H + 3 + H + 1][1])
+        assert all(is_prob(a, j + T) for f, a in blk[4:4 + H])
+        # causal: row i sees j + i + 1 keys, the rest carry probability exactly 0
+        assert all(np.count_nonzero(a[i]) == j + i + 1 for f, a in blk[4:4 + H] for i in range(T))
+        assert all(is_prob(a, S) for f, a in blk[4 + H + 3:4 + H + 3 + H])
+        assert blk[-1][1].min() == 0.0
+        # q, k, v handed over are linear images of the rounded LayerNorm output
+        y = real(blk[0][1])
+        for idx, nm in zip((1, 2, 3), "qkv"):
+            assert np.allclose(blk[idx][1], y @ m.w[f"dec.{l}.self.{nm}.w"].T + m.w[f"dec.{l}.self.{nm}.b"], atol=1e-5)
+        # the cache holds the rounded K / V of the block
+        assert np.array_equal(cache.k[l][j:], real(blk[2][1])) and np.array_equal(cache.v[l][j:], real(blk[3][1]))
+    assert is_ln(calls[-1][1])
+    # logits never pass through the rounding: nothing V wide was recorded, and the result is the exact product
+    assert all(a.shape[-1] != V for f, a in calls)
+    assert np.array_equal(logits, real(calls[-1][1]) @ m.w["embed"].T)
+    assert not np.array_equal(logits, real(logits))
+    # with rounding switched off the same code path is the pure model: all rounding goes through this one routine
+    monkeypatch.setattr(O, "bf16_round", lambda a: a)
+    mp = O.model_from(dims, w, mode="pure")
+    memp = O.encode(mp, src)
+    assert np.array_equal(O.encode(m, src), memp)
+    assert np.array_equal(O.decoder_rows(m, [1, 4, 5], memp, True), O.decoder_rows(mp, [1, 4, 5], memp, True))
