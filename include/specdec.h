@@ -38,7 +38,11 @@ extern "C" {
 #define SPECDEC_ERR_CAPACITY      -3   /* B / S / k / max_tgt beyond create-time limits  */
 #define SPECDEC_ERR_NOT_ENCODED   -4
 #define SPECDEC_ERR_CUDA          -5
-#define SPECDEC_ERR_TIMEOUT       -6   /* a bounded device-side wait gave up             */
+#define SPECDEC_ERR_TIMEOUT       -6   /* a bounded device-side wait gave up.  specdec_generate reports it itself;
+                                          the asynchronous step calls report it one call late: specdec_commit and
+                                          specdec_get_output fetch the device's error word, and the next call on the
+                                          handle that finds it set returns this code and clears it.  The handle stays
+                                          usable: start over with specdec_encode                                      */
 #define SPECDEC_ERR_UNSUPPORTED   -7
 
 #define SPECDEC_DTYPE_F32   0
@@ -173,7 +177,7 @@ int specdec_accept_scan(const float* d_logits, const int32_t* d_draft, int B, in
  * specdec_accept_scan (d_logits [B,k+1,V] fp32, d_draft [B,k]; d_accepted, d_bif [B]); the
  * intermediate per-row partial statistics live in a fixed array compiled into the library
  * (about 4.2 MB of device memory on every GPU that loads the library, held until the process
- * exits).  Limits: B*(k+1) <= 4096 and V <= 65536; beyond them the call returns
+ * exits).  Limits: B*(k+1) <= 4096, V <= 65536 and k+1 <= 2048; beyond them the call returns
  * SPECDEC_ERR_CAPACITY and launches nothing.  The call makes no cudaMalloc / cudaFree and uses
  * no allocating library routine.  The first call on each device looks up the array's device
  * address (cudaGetSymbolAddress, with the caller's current device); make that first call
@@ -193,9 +197,9 @@ int specdec_accept_scan_static(const float* d_logits, const int32_t* d_draft, in
  *   the draft's logit (+inf on the bonus row), draft id (-1 on the bonus row). */
 int specdec_debug_logits(specdec_handle* h, int which, float* d_logits, void* stream);
 int specdec_debug_row_stats(specdec_handle* h, float* d_stats, void* stream);
-/* With option "cl_trace" = 1 the cluster decoder kernel records a nanosecond timestamp after each of its
- * phases (first CTA only); this copies the first n (<= 256) of them to the host.  Synchronises the device. */
-int specdec_debug_cluster_trace(specdec_handle* h, long long* h_out, int n);
+/* With option "trace" != 0 the first CTA of some kernels records nanosecond time stamps of its phases into a
+ * 256-entry device array; this copies the first n (<= 256) entries to the host.  Synchronises the device. */
+int specdec_debug_trace(specdec_handle* h, long long* h_out, int n);
 
 /* Scripted drafts, a benchmark / test hook with no counterpart in the paper: random-init
  * models almost never agree, so a workload's acceptance pattern is imposed instead.  After the
@@ -208,62 +212,36 @@ int specdec_set_draft_script(specdec_handle* h, const int32_t* d_script, int B, 
  * count since the option was set. */
 int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches);
 
-/* Options: "gemm" = 0 SIMT reference GEMM, 1 tcgen05 GEMM (bf16 handles; default 1);
- * "skinny" = 0/1 weight-streaming GEMM with fused LayerNorm for passes of at most 32 rows (bf16; default 1);
- * "pair" = 0/1 two-SM tensor-core tiles (256 rows x 256 columns per CTA pair) for GEMMs with at least 1024 rows
- *   and 1024 columns (default 0: same results bit for bit, measured no faster than single-SM tiles at these
- *   sizes, kept for comparison);
- * "ln_fuse" = 0/1 apply the LayerNorm that reads the residual stream next inside the residual GEMM that
- *   writes it (tensor-core path: the CTAs of a row tile form a cluster and exchange per-row sums through
- *   distributed shared memory; default 0: correct, but its longer single-tile tail costs more than the
- *   separate LayerNorm launch it removes: 743 vs 688 us per 128-sequence verify step);
- * "sk_cluster" = 0 off / 1 (default) / 2: the weight-streaming GEMMs with fused LayerNorm run in clusters of 8 CTAs
- *   that each normalise an eighth of the input rows and send them to their peers' shared memory (instead of every
- *   CTA of the grid reading and normalising all rows: 348 -> 272 us per batch-1 verify step); 2 / 3 also share the rows
- *   of the plain weight-streaming GEMMs (2: those with K <= 512, no gain; 3: all, slower: 287 us);
- * "ln_rows" = 0/1 tensor-core GEMMs over at most 128 rows normalise their input rows themselves (eight warps write
- *   the bf16 operand tile in the tensor core's swizzled layout) instead of reading the output of a LayerNorm launch;
- *   the CTAs form clusters of up to 8 that each normalise a share of the rows and send them to their peers' shared
- *   memory (default 0: correct, but the 16-byte remote stores of 50-100 KB per CTA cost more than the launch they
- *   replace: 365 vs 356 us per 2-sequence verify step, 426 vs 375 us at 4 sequences);
- * "attn_rs" = 0 never / 1 choose (default) / 2 whenever the keys allow: tile attention keeps the scores in the MMA
- *   accumulators through the softmax instead of a shared-memory tile (smaller footprint, more CTAs per SM);
- * "diag_repeat" = bit mask, diagnostics: launch every attention (1), LayerNorm (2), GEMM without residual
- *   accumulation (4) or vocabulary kernel (8) twice in a row -- same result -- so that the step time rises by that
- *   class's cost inside the pipeline (default 0);
- * "splitk" = 0/1 residual GEMMs with K >= 1024 (FFN2) whose row tiles x N / 64 column tiles x 4 (K <= 2048) or 6
- *   (K = 3072) CTAs fit one wave run split along K: the CTAs of a cluster share a column tile and rank 0 adds their
- *   fp32 partials in rank order (default 1: 356 -> 324 us per 2-sequence verify step, 479 -> 416 us with 768-wide
- *   models; encoders and the drafter's first layer gain the same way);
- * "attn_stream" = 0 never / 1 by rule (default) / 2 always / 3 always with the two-stage ring: tile attention that
- *   walks the keys in blocks of 64 with a running maximum (shared memory independent of the key count) instead of
- *   staging every key at once.  Rule: where the one-shot kernel cannot hold the keys (about 590), and beyond
- *   "attn_stream_keys" keys (default 320) when the launch has at least 4 CTAs per SM (1180 -> 942 us per
- *   128-sequence verify step over 512-token sources; with few CTAs the block-by-block walk is the slower one);
- * "attn_warps" = 0 choose per launch, 4 or 8 warps per CTA of the tile attention (default 0);
- * "tc_bn" = 0 choose, else force the column width of the tensor-core GEMM tiles (64 / 128 / 256; experiments);
- * "cluster" = 0/1 run the verifier's decoder stack as one thread-block-cluster kernel per sequence when the
- *   batch is at most 8, k + 1 <= 32 and the model has 8 heads of 64 (default 0: measured slower than the
- *   per-operation kernels, kept for comparison);
- * "poll_lag" = n: specdec_generate reads the unfinished-sequences counter n iterations late (0: waits for it
- *   after every iteration; default 2 with gated iteration graphs, else 0 up to batch 4 and 2 above);
- * "poll_flag" = 0/1 specdec_generate learns of each commit from a word the commit kernel writes into pinned host
- *   memory, on which the host spins (default 1), instead of a 4-byte copy and an event per iteration;
- * "gate" = 0 never / 1 above batch 4 (default) / 2 always: specdec_generate launches each draft -> verify -> commit iteration as ONE CUDA graph whose kernels
- *   sit in the body of a conditional IF node behind a one-thread kernel that tests the unfinished-sequences
- *   counter: the host queues iterations ahead of the counter it reads back, and an iteration queued after the
- *   last sequence finished costs that one kernel (needs "graphs" = 1 and "stats_timing" = 0; at batch 1 the
- *   conditional node costs more per iteration, about 15 us, than the wait it removes);
- * "stats_timing" = 0/1 specdec_generate records an event after every draft, verify and commit phase and fills
- *   ms_draft / ms_verify / ms_commit (default 0: only ms_encode and ms_total; 1 turns the gated graphs off);
- * "fused_attn" = 0/1 attention + output projection + residual as one 8-CTA-cluster kernel per sequence for
- *   blocks of at most 32 query rows and models with 8 heads of 64 (default 0: measured slower than the two
- *   separate kernels at batch 1 and at batch 128, kept for comparison);
- * "pdl" = 0/1 programmatic dependent launch between the kernels of a step (default 1);
- * "attn" = 0 warp-per-row reference attention, 1 tensor-core tile attention (bf16, 64-wide heads; default 1);
- * "graphs" = 0/1 replay draft/verify steps from CUDA graphs inside specdec_generate;
- * "profile" = 0/1 (see specdec_profile_read); "row_lse" = 0/1 also accumulate the log-sum-exp of
- * every verifier row (only reported through specdec_debug_row_stats; the rule does not need it). */
+/* Options (experiments and on-device cross-checks; every combination computes the same result):
+ * "gemm"         0 SIMT reference GEMM / 1 tcgen05 tensor-core GEMM (bf16 handles; default 1)
+ * "attn"         0 warp-per-row reference attention / 1 tensor-core tile attention (bf16, 64-wide heads; default 1)
+ * "skinny"       0/1 weight-streaming GEMM with fused LayerNorm for passes of at most 32 rows (default 1)
+ * "sk_cluster"   0 off / 1 (default): those GEMMs run in clusters of 8 CTAs that share the normalised input rows
+ *                through distributed shared memory; 2 / 3 also the GEMMs without a LayerNorm (K <= 512 / all)
+ * "fused_step"   0 never / 1 (default) where it applies: the verifier's decoder stack of a step as ONE kernel, one
+ *                16-CTA cluster per sequence (verify blocks of at most 32 rows, 8 heads of 64, at most 8 sequences)
+ * "pair"         0/1 two-SM tensor-core tiles (cta_group::2) for GEMMs with >= 1024 rows and columns (default 0)
+ * "ln_fuse"      0/1 the LayerNorm that reads the residual stream next runs inside the residual GEMM (default 0)
+ * "splitk"       0/1 residual GEMMs with K >= 1024 over few row tiles split K across a cluster (default 1)
+ * "attn_rs"      0 never / 1 by rule (default) / 2 whenever the keys allow: scores stay in the MMA accumulators
+ * "attn_stream"  0 never / 1 by rule (default) / 2 always / 3 always, two-stage ring: attention walks the keys in
+ *                blocks of 64 with a running maximum; "attn_stream_keys" (default 320) is the rule's threshold
+ * "attn_warps"   0 choose per launch (default), 4 or 8 warps per tile-attention CTA
+ * "tc_bn"        0 choose (default), else the column width of the tensor-core tiles (64 / 128 / 256)
+ * "pdl"          0/1 programmatic dependent launch between the kernels of a step (default 1)
+ * "graphs"       0/1 replay steps from CUDA graphs (default 1)
+ * "gate"         0 never / 1 above batch 4 (default) / 2 always: each iteration of specdec_generate is one graph
+ *                behind a device-side IF node, so the host can queue iterations ahead of the counter it reads
+ * "poll_flag"    0/1 specdec_generate learns of each commit from a word in pinned host memory (default 1)
+ * "poll_lag"     n: specdec_generate reads the unfinished-sequences counter n iterations late (default: by batch)
+ * "stats_timing" 0/1 fill ms_draft / ms_verify / ms_commit of specdec_stats (default 0; turns the gate off)
+ * "profile"      0/1 see specdec_profile_read
+ * "row_lse"      0/1 also accumulate the log-sum-exp of every verifier row (reported by specdec_debug_row_stats)
+ * "diag_repeat"  bit mask: launch every attention (1), LayerNorm (2), non-residual GEMM (4), vocabulary kernel (8)
+ *                twice in a row (same result), so the step time rises by that class's cost inside the pipeline
+ * "trace"        see specdec_debug_trace
+ * "inject_error" code: test hook -- the next specdec_verify / specdec_generate finds this code in the device error
+ *                word, as if a bounded device-side wait had given up (no kernel waits, nothing faults) */
 int specdec_set_option(specdec_handle* h, const char* name, int value);
 
 /* Number of kernels the library has launched on this handle since create. */

@@ -24,7 +24,7 @@ EXPORTS = [
     "specdec_commit", "specdec_generate", "specdec_generate_host", "specdec_get_output",
     "specdec_accept_scan", "specdec_debug_logits", "specdec_debug_row_stats", "specdec_set_option",
     "specdec_launch_count", "specdec_last_error", "specdec_set_draft_script", "specdec_profile_read",
-    "specdec_accept_scan_static", "specdec_debug_cluster_trace",
+    "specdec_accept_scan_static", "specdec_debug_trace",
 ]
 
 
@@ -58,9 +58,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     if path == LIB_PATH and _build.needs_build():
         try:
             _build.build()              # compile step (nvcc, sm_100a); not a fallback
-        except Exception as e:          # keep a usable older build only if one exists
-            if not os.path.exists(path):
-                raise RuntimeError(f"cannot build {path}: {e}") from e
+        except Exception as e:          # a stale library must never pass for the current source
+            raise RuntimeError(f"cannot build {path}: {e}") from e
     if not os.path.exists(path):
         raise RuntimeError(f"{path} is missing: build it with `python -m paper_2203_16487_b200.build` "
                            "(there is no fallback path)")
@@ -79,7 +78,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.specdec_accept_scan_static.argtypes = [vp, ip, i, i, i, i, f, ip, ip, vp]
     lib.specdec_debug_logits.argtypes = [vp, i, vp, vp]
     lib.specdec_debug_row_stats.argtypes = [vp, vp, vp]
-    lib.specdec_debug_cluster_trace.argtypes = [vp, C.POINTER(C.c_longlong), i]
+    lib.specdec_debug_trace.argtypes = [vp, C.POINTER(C.c_longlong), i]
     lib.specdec_set_option.argtypes = [vp, C.c_char_p, i]
     lib.specdec_set_draft_script.argtypes = [vp, ip, i, i, vp]
     lib.specdec_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
@@ -192,9 +191,9 @@ class SpecDec:
         self._check(self._lib.specdec_profile_read(self._h, C.byref(ms), C.byref(n)))
         return ms.value, n.value
 
-    def cluster_trace(self, n: int):
+    def trace(self, n: int):
         buf = (C.c_longlong * n)()
-        self._check(self._lib.specdec_debug_cluster_trace(self._h, buf, n))
+        self._check(self._lib.specdec_debug_trace(self._h, buf, n))
         return list(buf)
 
     def last_error(self) -> str:

@@ -24,7 +24,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "--use_fast_math" if False else "-DSPECDEC_PRECISE_MATH", "-shared", "-Xcompiler", "-fPIC",
+           "-DSPECDEC_PRECISE_MATH", "-shared", "-Xcompiler", "-fPIC",
            "-cudart", "static", "-o", LIB, SRC]
     if verbose:
         cmd.insert(1, "-Xptxas"); cmd.insert(2, "-v")

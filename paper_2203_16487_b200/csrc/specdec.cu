@@ -15,12 +15,9 @@
 #include <vector>
 
 #include "../../include/specdec.h"
-#include "attention_oproj.cuh"
 #include "attention_stream.cuh"
 #include "attention_tc.cuh"
-#include "decoder_cluster.cuh"
 #include "gemm_tc.cuh"
-#include "gemm_tc_lnrows.cuh"
 #include "gemm_tc_pair.cuh"
 #include "gemm_tc_splitk.cuh"
 #include "kernels.cuh"
@@ -90,20 +87,15 @@ struct specdec_handle {
     bool encoded = false, verified = false, drafted = false;
     int last_draft_rows_ub = 0;
     // options
-    int use_tc = 1, use_graphs = 1, use_tc_attn = 1, want_lse = 0, use_skinny = 1, use_pdl = 1, use_cluster = 0;
-    // packed weight stream of the cluster decoder kernel (verifier, small batches)
-    unsigned char* cl_stream = nullptr;
-    size_t cl_cta_stride = 0;
-    bool cl_ok = false;
-    long long* cl_trace = nullptr;   // device [256] timestamps of the cluster kernel's phases (option "cl_trace")
-    int want_cl_trace = 0;
+    int use_tc = 1, use_graphs = 1, use_tc_attn = 1, want_lse = 0, use_skinny = 1, use_pdl = 1;
+    int use_fused_step = 1;         // the verifier's decoder stack of a step as one cluster kernel per sequence (option "fused_step")
+    long long* trace_buf = nullptr; // device [256] in-kernel time stamps (option "trace")
+    int want_trace = 0;
     size_t skinny_smem_cap = 0;
     int poll_lag = -1;              // -1: chosen by batch size
     int stats_timing = 0;           // 1: specdec_generate records an event after every phase (option "stats_timing")
     int use_gate = 1;               // whole iterations as one graph behind a device-side IF node (option "gate")
     bool gate_ok = true;            // false once building such a graph failed: the plain graphs are used from then on
-    int use_fused_attn = 0;         // attention + output projection as one cluster kernel (measured slower: off)
-    size_t attn_proj_smem_cap = 0;
     // LayerNorm fused into the residual GEMM that feeds it (tensor-core path): what the next residual GEMM should
     // also produce, and what the last one did produce
     struct NextLn { const float* g; const float* b; void* out; };
@@ -111,12 +103,10 @@ struct specdec_handle {
     const float* fused_x = nullptr; const float* fused_g = nullptr; const void* fused_out = nullptr;
     int use_ln_fuse = 0;            // option "ln_fuse": measured slower than the separate LayerNorm launch, kept for comparison
     int use_sk_cluster = 1;         // option "sk_cluster": 1 = LayerNorm-fused weight-streaming GEMMs share the normalised rows in clusters of 8; 2 = the plain ones too (measured slower)
-    bool lnrows_ready = false;
     bool splitk_ready = false;
     int diag_repeat = 0;            // diagnostics: launch every attention (1) / LayerNorm (2) / non-residual GEMM (4) / vocabulary (8) kernel twice (same result) to
                                     // read its cost inside the pipeline off the step time (option "diag_repeat")
     int use_splitk = 1;             // residual GEMMs with K >= 1024 over few row tiles split K across a cluster of 4 / 6 CTAs (option "splitk")
-    int use_ln_rows = 0;            // option "ln_rows": GEMMs over at most 128 rows normalise their input rows themselves (measured slower: off)
     bool pair_ready = false;
     int use_pair = 0;               // two-SM tiles (cta_group::2) for wide GEMMs over many rows (option "pair")
     int attn_rs = 1;                // tile attention keeps the scores in registers when the keys allow (option "attn_rs")
@@ -136,6 +126,9 @@ struct specdec_handle {
     int poll_flag = 1;              // the generation loop polls h_post instead of copying the counter back (option "poll_flag")
     unsigned long long* h_stats = nullptr;  // pinned [4]
     std::vector<cudaEvent_t> poll_ev;
+    // device error word (counters[7], raised by bounded device-side waits) mirrored into pinned memory: h_poll[ERRW_SLOT]
+    cudaEvent_t errw_ev = nullptr;
+    bool errw_pending = false;      // a copy of the word is in flight
     std::vector<cudaEvent_t> time_ev;
     sd::TmaEncoder tma;
     // work submitted on the legacy default stream (which cannot be captured into a graph) is run on this
@@ -154,6 +147,8 @@ struct specdec_handle {
 };
 
 namespace {
+
+constexpr int ERRW_SLOT = 32;       // index into h_poll of the error word's host mirror
 
 int fail(specdec_handle* h, int code, const std::string& msg) {
     if (h) h->err = msg; else g_create_error = msg;
@@ -177,6 +172,26 @@ int fail(specdec_handle* h, int code, const std::string& msg) {
 #define TRY(expr) do { int rc__ = (expr); if (rc__ != 0) return rc__; } while (0)
 
 inline int cdiv(int a, int b) { return (a + b - 1) / b; }
+
+// Bounded device-side waits raise a code in counters[7].  The step calls (draft / verify / commit / get_output) are
+// asynchronous, so they report it one call late: commit and get_output queue a 4-byte copy of the word into pinned
+// memory, and every step call first looks at the last copy that has landed.  Reporting clears the word.
+int errw_check(specdec_handle* h, cudaStream_t st, const char* who) {
+    if (h->errw_pending) {
+        if (cudaEventQuery(h->errw_ev) != cudaSuccess) { cudaGetLastError(); return 0; }
+        h->errw_pending = false;
+    }
+    const int code = ((volatile int*)h->h_poll)[ERRW_SLOT];
+    if (code == 0) return 0;
+    h->h_poll[ERRW_SLOT] = 0;
+    cudaMemsetAsync(h->ses.counters + 7, 0, 4, st);
+    return fail(h, SPECDEC_ERR_TIMEOUT, std::string(who) + ": a bounded device-side wait gave up (code " + std::to_string(code) + ")");
+}
+void errw_fetch(specdec_handle* h, cudaStream_t st) {
+    if (h->errw_pending) return;
+    if (cudaMemcpyAsync(h->h_poll + ERRW_SLOT, h->ses.counters + 7, 4, cudaMemcpyDeviceToHost, st) == cudaSuccess &&
+        cudaEventRecord(h->errw_ev, st) == cudaSuccess) h->errw_pending = true;
+}
 
 // ---------------------------------------------------------------- layout of the arena
 void layout_model(specdec_handle* h, ModelW& m, const specdec_model_dims& dm) {
@@ -208,13 +223,6 @@ void layout_model(specdec_handle* h, ModelW& m, const specdec_model_dims& dm) {
     m.enc_lnf_g = vec(d); m.enc_lnf_b = vec(d); m.dec_lnf_g = vec(d); m.dec_lnf_b = vec(d);
     m.ckv.resize(dm.dec_layers);
     for (auto& p : m.ckv) p = A.take((size_t)h->B_cap * h->S_cap * 2 * d * e);
-}
-
-// The cluster decoder kernel needs one CTA per head of 64 columns and operand rows that fit its shared memory.
-bool cl_eligible(const specdec_config& c) {
-    const specdec_model_dims& v = c.verifier;
-    return c.compute_dtype == SPECDEC_DTYPE_BF16 && c.ffn_activation == SPECDEC_ACT_RELU && v.n_heads == CL_C && v.d_model == CL_C * 64 && v.d_model <= 512 &&
-           v.d_ffn % (CL_C * 64) == 0 && v.d_ffn <= 2048 && v.dec_layers <= CL_MAX_LAYERS;
 }
 
 void layout_rows(Arena& A, Rows& r, int n, int B) {
@@ -267,12 +275,7 @@ void layout_all(specdec_handle* h) {
     h->stage_len = (int*)A.take((size_t)h->B_cap * 4);
     h->stage_mt = (int*)A.take((size_t)h->B_cap * 4);
     h->script = (int*)A.take((size_t)h->B_cap * (h->T_cap + h->k_cap) * 4);
-    if (cl_eligible(h->cfg)) {
-        const specdec_model_dims& v = h->cfg.verifier;
-        h->cl_cta_stride = (size_t)v.dec_layers * cl_stages_per_layer(v.d_model, v.d_ffn) * CL_STAGE;
-        h->cl_stream = (unsigned char*)A.take(h->cl_cta_stride * CL_C);
-        h->cl_trace = (long long*)A.take(256 * 8);
-    }
+    h->trace_buf = (long long*)A.take(256 * 8);
     Session& s = h->ses;
     s.len = (int*)A.take((size_t)h->B_cap * 4);
     s.finished = (int*)A.take((size_t)h->B_cap * 4);
@@ -490,12 +493,7 @@ int gemm_once(specdec_handle* h, int epi, const void* A, int lda, const void* W,
     // (not in the encoders: the two encoders run side by side on two streams, and the weight-streaming kernels' 64-256
     // CTAs per launch get in each other's way there -- 440 us against 386 us with 8-32-CTA tile GEMMs for a 32-token source)
     const bool skinny = cnt != CNT_ENC && skinny_ok<T>(h, epi, rows_ub, N, K, lnp != nullptr);
-    // At most 128 rows on the tensor-core path: the GEMM normalises its input rows itself (gemm_tc_lnrows.cuh)
-    bool ln_rows = false;
-    if constexpr (std::is_same<T, bf16>::value)
-        ln_rows = lnp && !skinny && h->use_tc && h->lnrows_ready && h->use_ln_rows && sd::lr_supported(epi, N, K, rows_ub) &&
-                  !(lnp->x == h->fused_x && lnp->g == h->fused_g && h->y == h->fused_out);
-    if (lnp && !skinny && !ln_rows) {           // separate normalisation launch, then a plain GEMM on its output
+    if (lnp && !skinny) {           // separate normalisation launch, then a plain GEMM on its output
         TRY(ln_or_fused<T>(h, lnp->x, lnp->g, lnp->b, cnt, rows_ub, h->y, K, st));
         A = h->y; lda = K;
     }
@@ -509,26 +507,19 @@ int gemm_once(specdec_handle* h, int epi, const void* A, int lda, const void* W,
     g.part = h->part; g.ld = ldv; g.ld_id = ld_id; g.n_tiles = cdiv(N, 64); g.want_sum = h->want_lse;
     g.seq = nullptr; g.pos = nullptr; g.kc = nullptr; g.vc = nullptr; g.kv_d = 0;
     g.pg.table = h->page_table; g.pg.page_tokens = h->cfg.page_tokens; g.pg.max_pages = h->pages_per_seq;
-    g.trace = (h->want_cl_trace && h->cl_trace && epi == (h->want_cl_trace >= 10 ? h->want_cl_trace - 10 : EPI_STATS)) ? h->cl_trace + 200 : nullptr;
+    g.trace = (h->want_trace && epi == (h->want_trace >= 10 ? h->want_trace - 10 : EPI_STATS)) ? h->trace_buf + 200 : nullptr;
     if (kv) { g.seq = kv->seq; g.pos = kv->pos; g.kc = (T*)kv->kc; g.vc = (T*)kv->vc; g.kv_d = kv->d; }
     if constexpr (std::is_same<T, bf16>::value) {
         if (skinny) {
             SkinnyArgs sa; sa.g = g;
             sa.ln_x = lnp ? lnp->x : nullptr; sa.ln_g = lnp ? lnp->g : nullptr; sa.ln_b = lnp ? lnp->b : nullptr;
             sa.ln_eps = 1e-5f; sa.ln_out = nullptr; sa.err_word = h->ses.counters + 7;
-            sa.trace = (h->want_cl_trace && h->cl_trace) ? h->cl_trace + 216 + 6 * ((epi == EPI_RELU || epi == EPI_GELU) ? 0 : epi == EPI_RESID ? 1 : epi == EPI_QKV ? 2 : 3) : nullptr;
+            sa.trace = h->want_trace ? h->trace_buf + 216 + 6 * ((epi == EPI_RELU || epi == EPI_GELU) ? 0 : epi == EPI_RESID ? 1 : epi == EPI_QKV ? 2 : 3) : nullptr;
             TRY(skinny_launch(h, epi, sa, rows_ub, st));
             return 0;
         }
     }
     if constexpr (std::is_same<T, bf16>::value) {
-        if (ln_rows) {
-            sd::LnRowsArgs la{lnp->x, lnp->g, lnp->b, 1e-5f};
-            if (sd::lr_launch(h->tma, epi, g, la, st) != 0)
-                return fail(h, SPECDEC_ERR_CUDA, "tensor-core GEMM launch failed: " + h->tma.err);
-            ++h->launches;
-            return 0;
-        }
         if (h->use_tc && sd::tc_supported(N, K) && (epi != EPI_STATS || N >= 128)) {
             if (epi == EPI_RESID && h->use_ln_fuse && want_ln.g && want_ln.out && sd::tc_ln_fusable(N, K)) {
                 g.ln_g = want_ln.g; g.ln_b = want_ln.b; g.ln_out = (T*)want_ln.out;
@@ -680,41 +671,6 @@ void prof_collect(specdec_handle* h) {
     h->prof_n = 0;
 }
 
-// Attention + output projection + residual as one 8-CTA-cluster kernel per sequence (see attention_oproj.cuh).
-// Returns 1 if it was launched, 0 if the shapes do not qualify, < 0 on error.
-template <typename T>
-int fused_attn_proj(specdec_handle* h, bool paged, const void* q, int q_stride, const int* q_index, const void* k,
-                    const void* v, int kv_stride, const int* kv_off, const Rows& r, const int* nkeys, int q_ub,
-                    int n_heads, int d_head, int max_keys, const void* wo, const float* bo, float* x, int d, cudaStream_t st) {
-    if constexpr (!std::is_same<T, bf16>::value) return 0;
-    else {
-        if (!h->use_fused_attn || !h->use_tc_attn || n_heads != AP_HEADS || d_head != 64 || d != AP_HEADS * 64 || q_ub > ATT_Q) return 0;
-        const size_t smem = attn_proj_smem(max_keys, d);
-        if (smem > h->attn_proj_smem_cap) return 0;
-        AttnProjArgs p;
-        AttnTcArgs& a = p.at;
-        a.q = (const bf16*)q; a.q_stride = q_stride; a.q_index = q_index;
-        a.k = (const bf16*)k; a.v = (const bf16*)v; a.kv_stride = kv_stride; a.kv_off = kv_off;
-        a.pg.table = h->page_table; a.pg.page_tokens = h->cfg.page_tokens; a.pg.max_pages = h->pages_per_seq;
-        a.q_off = r.q_off; a.q_cnt = r.q_cnt; a.nkeys = nkeys; a.pre_keys = nullptr; a.out = nullptr; a.out_stride = 0; a.max_keys = max_keys;
-        a.scale = 1.0f / sqrtf((float)d_head);
-        p.wo = (const bf16*)wo; p.bo = bo; p.x = x; p.d = d;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(AP_HEADS, h->B); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = smem; cfg.stream = st;
-        cudaLaunchAttribute attr[2];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = AP_HEADS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[1].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr; cfg.numAttrs = h->use_pdl ? 2 : 1;
-        cudaError_t e = paged ? cudaLaunchKernelEx(&cfg, k_attn_proj<true>, p) : cudaLaunchKernelEx(&cfg, k_attn_proj<false>, p);
-        if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("attention+projection launch: ") + cudaGetErrorString(e));
-        KCHECK(h);
-        h->fused_x = nullptr; h->next_ln = {nullptr, nullptr, nullptr};    // this kernel rewrote the residual rows
-        return 1;
-    }
-}
-
 // One pre-LN block on `rows_ub` rows of the residual stream x (encoder: no cross-attention).
 // Self-attention keys come from the block's own QKV rows (contiguous) or, for the verifier,
 // from the paged cache after the block's K/V were scattered into it.
@@ -741,10 +697,6 @@ int block_self(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, co
         }
     }
     if (verify) {
-        const int f = fused_attn_proj<T>(h, true, h->qkv, 3 * d, nullptr, h->kc[layer], h->vc[layer], d, nullptr, r, r.nk_self,
-                                         q_ub, H, dh, max_keys, w.o_w, w.o_b, x, d, st);
-        if (f < 0) return f;
-        if (f == 1) return 0;
         TRY(attn<T>(h, true, h->qkv, 3 * d, nullptr, h->kc[layer], h->vc[layer], d, nullptr, r, r.nk_self, cnt,
                     rows_ub, q_ub, h->att, d, H, dh, max_keys, st, h->ses.len));      // cached prefix: positions < len
     } else {
@@ -764,12 +716,6 @@ int block_cross(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, c
     const LnSpec lc{x, w.lnc_g, w.lnc_b};
     TRY(gemm<T>(h, EPI_STORE, h->y, d, w.cq_w, w.cq_b, d, d, cnt, rows_ub, h->q, d, nullptr, st, nullptr, nullptr, nullptr,
                 nullptr, &lc));
-    {
-        const int f = fused_attn_proj<T>(h, false, h->q, d, nullptr, m.ckv[layer], (char*)m.ckv[layer] + (size_t)d * e, 2 * d,
-                                         r.kv_off_cross, r, r.nk_cross, q_ub, H, dh, h->S_max, w.co_w, w.co_b, x, d, st);
-        if (f < 0) return f;
-        if (f == 1) return 0;
-    }
     TRY(attn<T>(h, false, h->q, d, nullptr, m.ckv[layer], (char*)m.ckv[layer] + (size_t)d * e, 2 * d, r.kv_off_cross,
                 r, r.nk_cross, cnt, rows_ub, q_ub, h->att, d, H, dh, h->S_max, st, h->ses.src_len));   // encoder K/V: all of it
     h->next_ln = {w.ln2_g, w.ln2_b, h->y};           // the feed-forward sublayer's LayerNorm comes next
@@ -883,18 +829,10 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
                 nullptr, nullptr, nullptr, &l1));
     CUDA_TRY(h, launch_pdl(h, k_gather_rows, dim3(R2), dim3(128), 0, st, (const float*)h->x, (const int*)h->mrows.src_row, (const int*)(h->ses.counters + CNT_DRAFT_MASK), h->x2, d));
     KCHECK(h);
-    {
-        const int f = fused_attn_proj<T>(h, false, h->qkv, 3 * d, h->mrows.src_row, (char*)h->qkv + (size_t)d * e,
-                                         (char*)h->qkv + (size_t)2 * d * e, 3 * d, h->mrows.kv_off, h->mrows, h->mrows.nk_self, k,
-                                         H, dh, max_keys, w.o_w, w.o_b, h->x2, d, st);
-        if (f < 0) return f;
-        if (f == 0) {
-            TRY(attn<T>(h, false, h->qkv, 3 * d, h->mrows.src_row, (char*)h->qkv + (size_t)d * e,
-                        (char*)h->qkv + (size_t)2 * d * e, 3 * d, h->mrows.kv_off, h->mrows, h->mrows.nk_self,
-                        CNT_DRAFT_MASK, R2, k, h->att, d, H, dh, max_keys, st));
-            TRY(gemm<T>(h, EPI_RESID, h->att, d, w.o_w, w.o_b, d, d, CNT_DRAFT_MASK, R2, nullptr, 0, h->x2, st));
-        }
-    }
+    TRY(attn<T>(h, false, h->qkv, 3 * d, h->mrows.src_row, (char*)h->qkv + (size_t)d * e,
+                (char*)h->qkv + (size_t)2 * d * e, 3 * d, h->mrows.kv_off, h->mrows, h->mrows.nk_self,
+                CNT_DRAFT_MASK, R2, k, h->att, d, H, dh, max_keys, st));
+    TRY(gemm<T>(h, EPI_RESID, h->att, d, w.o_w, w.o_b, d, d, CNT_DRAFT_MASK, R2, nullptr, 0, h->x2, st));
     TRY(block_cross<T>(h, m, w, h->x2, h->mrows, CNT_DRAFT_MASK, R2, k, L - 1, st));
     TRY(block_ffn<T>(h, m, w, h->x2, CNT_DRAFT_MASK, R2, st, m.dec_lnf_g, m.dec_lnf_b));
     TRY(ln_or_fused<T>(h, h->x2, m.dec_lnf_g, m.dec_lnf_b, CNT_DRAFT_MASK, R2, h->y, d, st));
@@ -925,38 +863,7 @@ int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float ta
     k_verify_prep<<<cdiv(M, 256), 256, 0, st>>>(h->ses, h->v_draft, B, k, h->S_max, h->cfg.bos_id, h->rows);
     KCHECK(h);
     TRY(embed<T>(h, m, h->rows, m.pos_dec, CNT_VERIFY, M, st));
-    bool clustered = false;
-    if constexpr (std::is_same<T, bf16>::value) {
-        const int cap = cl_max_keys(m.dm.d_ffn);
-        if (h->cl_ok && h->use_cluster && B <= 8 && k + 1 <= CL_M && max_keys <= cap && h->S_max <= cap) {
-            // the whole decoder stack in one kernel: one cluster of 8 CTAs per sequence
-            ClArgs ca;
-            ca.wstream = h->cl_stream; ca.cta_stride = h->cl_cta_stride; ca.n_layers = L;
-            for (int l = 0; l < L; ++l) {
-                const LayerW& w = m.dec[l];
-                ca.layer[l] = ClLayer{w.ln1_g, w.ln1_b, w.lnc_g, w.lnc_b, w.ln2_g, w.ln2_b, w.qkv_b, w.o_b, w.cq_b, w.co_b, w.b1, w.b2,
-                                      (bf16*)h->kc[l], (bf16*)h->vc[l], (const bf16*)m.ckv[l]};
-            }
-            ca.x = h->x; ca.att = (bf16*)h->att; ca.hbuf = (bf16*)h->hbuf;
-            ca.len = h->ses.len; ca.src_len = h->ses.src_len;
-            ca.pg.table = h->page_table; ca.pg.page_tokens = h->cfg.page_tokens; ca.pg.max_pages = h->pages_per_seq;
-            ca.S_max = h->S_max; ca.k1 = k + 1; ca.d = d; ca.F = m.dm.d_ffn; ca.max_keys = cap; ca.err_word = h->ses.counters + 7;
-            ca.trace = h->want_cl_trace ? h->cl_trace : nullptr;
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(B * CL_C); cfg.blockDim = dim3(CL_THREADS); cfg.dynamicSmemBytes = cl_smem_bytes(m.dm.d_ffn); cfg.stream = st;
-            cudaLaunchAttribute attr[2];
-            attr[0].id = cudaLaunchAttributeClusterDimension;
-            attr[0].val.clusterDim.x = CL_C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-            attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-            attr[1].val.programmaticStreamSerializationAllowed = 1;
-            cfg.attrs = attr; cfg.numAttrs = h->use_pdl ? 2 : 1;
-            cudaError_t e = cudaLaunchKernelEx(&cfg, k_decoder_cluster, ca);
-            if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("cluster decoder launch: ") + cudaGetErrorString(e));
-            KCHECK(h);
-            clustered = true;
-        }
-    }
-    for (int l = 0; l < L && !clustered; ++l) {
+    for (int l = 0; l < L; ++l) {
         const bool last = l + 1 == L;
         TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, k + 1, l, true, max_keys, st, m.dec[l].lnc_g, m.dec[l].lnc_b));
         TRY(block_cross<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, k + 1, l, st));
@@ -1019,9 +926,9 @@ void drop_graphs(specdec_handle* h) {
 // replayed afterwards.  The key must name everything the launches depend on besides device memory.
 inline void graph_key_tail(const specdec_handle* h, std::vector<long long>& key) {
     for (long long v : {(long long)h->use_tc, (long long)h->use_tc_attn, (long long)h->want_lse, (long long)h->use_skinny,
-                        (long long)h->use_pdl, (long long)h->use_ln_fuse, (long long)h->use_ln_rows, (long long)h->use_sk_cluster,
-                        (long long)h->use_pair, (long long)h->diag_repeat, (long long)h->use_splitk, (long long)h->attn_stream, (long long)h->attn_stream_keys, (long long)h->attn_warps, (long long)h->attn_rs, (long long)h->use_fused_attn,
-                        (long long)h->skinny_groups, (long long)h->use_cluster, (long long)h->want_cl_trace,
+                        (long long)h->use_pdl, (long long)h->use_ln_fuse, (long long)h->use_sk_cluster,
+                        (long long)h->use_pair, (long long)h->diag_repeat, (long long)h->use_splitk, (long long)h->attn_stream, (long long)h->attn_stream_keys, (long long)h->attn_warps, (long long)h->attn_rs,
+                        (long long)h->skinny_groups, (long long)h->want_trace, (long long)h->use_fused_step,
                         (long long)(h->script_on ? 1 : 0), (long long)h->B, (long long)h->S_max})
         key.push_back(v);
 }
@@ -1122,7 +1029,7 @@ int encode_staged(specdec_handle* h, const int* d_src, const int* d_src_len, con
 inline int len_bucket(const specdec_handle* h, int len_ub) { return std::min(h->T_cap, (len_ub + 31) / 32 * 32); }
 
 template <typename T>
-int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, const int* d_max_tgt, int B, int S_max,
+int generate_loop(specdec_handle* h, const int* d_src, const int* d_src_len, const int* d_max_tgt, int B, int S_max,
                   int k, int beta, float tau, int* d_out, int out_stride, int* d_out_len, specdec_stats* hs,
                   cudaStream_t st) {
     const bool timed = hs != nullptr, phases = timed && h->stats_timing;
@@ -1218,6 +1125,12 @@ int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, con
                         if (q == cudaSuccess) {       // the stream drained: the word must be there now
                             const unsigned long long v2 = *(volatile unsigned long long*)h->h_post;
                             if ((int)((unsigned)(v2 >> 32) - want) >= 0) { active_seen = (int)(unsigned)v2; break; }
+                            // behind a gate no commit kernel runs once nothing is left to decode (for instance when
+                            // every budget was zero from the start): ask the device
+                            int active_now = -1;
+                            CUDA_TRY(h, cudaMemcpyAsync(&active_now, h->ses.counters + CNT_ACTIVE, 4, cudaMemcpyDeviceToHost, st));
+                            CUDA_TRY(h, cudaStreamSynchronize(st));
+                            if (active_now == 0) { active_seen = 0; break; }
                             return fail(h, SPECDEC_ERR_CUDA, "generate: the commit kernel did not post its counter");
                         }
                         if (std::chrono::steady_clock::now() - t0 > std::chrono::seconds(60))
@@ -1252,7 +1165,7 @@ int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, con
     h->commits_issued = (unsigned)(*(volatile unsigned long long*)h->h_post >> 32);    // gated iterations that found nothing to do posted nothing
     if (h->profile) prof_collect(h);
     if (*(int*)(h->h_stats + 4) != 0)
-        return fail(h, SPECDEC_ERR_TIMEOUT, "a bounded device-side wait gave up (code " + std::to_string(*(int*)(h->h_stats + 4)) + ")");
+        return fail(h, SPECDEC_ERR_TIMEOUT, "generate: a bounded device-side wait gave up (code " + std::to_string(*(int*)(h->h_stats + 4)) + ")");
     if (hs) {
         memset(hs, 0, sizeof(*hs));
         hs->iterations = it - skipped;
@@ -1271,6 +1184,27 @@ int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, con
         hs->ms_total = ms(0, ev - 1);
     }
     return 0;
+}
+
+template <typename T>
+int generate_impl(specdec_handle* h, const int* d_src, const int* d_src_len, const int* d_max_tgt, int B, int S_max,
+                  int k, int beta, float tau, int* d_out, int out_stride, int* d_out_len, specdec_stats* hs,
+                  cudaStream_t st) {
+    TRY(errw_check(h, st, "generate"));
+    const int rc = generate_loop<T>(h, d_src, d_src_len, d_max_tgt, B, S_max, k, beta, tau, d_out, out_stride, d_out_len, hs, st);
+    if (rc != 0) {
+        // leave the handle usable: drain the stream, take the commit count from what was really posted, and clear the
+        // error word now that it has been reported
+        const std::string msg = h->err;
+        cudaStreamSynchronize(st);
+        cudaGetLastError();
+        h->commits_issued = (unsigned)(*(volatile unsigned long long*)h->h_post >> 32);
+        cudaMemsetAsync(h->ses.counters + 7, 0, 4, st);
+        h->h_poll[ERRW_SLOT] = 0; h->errw_pending = false;
+        h->encoded = false; h->verified = false; h->drafted = false;
+        h->err = msg;
+    }
+    return rc;
 }
 
 int check_model(const specdec_model_dims& m, const char* who, std::string& why) {
@@ -1375,6 +1309,8 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
     cudaEventCreateWithFlags(&h->enc_join, cudaEventDisableTiming);
     cudaEventCreateWithFlags(&h->fence_in, cudaEventDisableTiming);
     cudaEventCreateWithFlags(&h->fence_out, cudaEventDisableTiming);
+    cudaEventCreateWithFlags(&h->errw_ev, cudaEventDisableTiming);
+    memset(h->h_poll, 0, 64 * 4);
     h->poll_ev.resize(8);
     for (auto& e : h->poll_ev) cudaEventCreateWithFlags(&e, cudaEventDisableTiming);
     h->time_ev.resize((size_t)3 * h->T_cap + 8);
@@ -1422,34 +1358,7 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
             if (e != cudaSuccess) { cudaGetLastError(); need = 48 * 1024; }
             h->skinny_smem_cap = need;
         }
-        if (h->cl_stream) {
-            const specdec_model_dims& v = cfg->verifier;
-            const int spl = cl_stages_per_layer(v.d_model, v.d_ffn);
-            for (int l = 0; l < v.dec_layers; ++l) {
-                const LayerW& w = h->ver.dec[l];
-                ClPackSrc ps{(const bf16*)w.qkv_w, (const bf16*)w.o_w, (const bf16*)w.cq_w, (const bf16*)w.co_w, (const bf16*)w.w1, (const bf16*)w.w2};
-                k_cl_pack<<<1024, 256, 0, st>>>(ps, l, v.d_model, v.d_ffn, (uint4*)h->cl_stream, h->cl_cta_stride / 16, spl);
-                ++h->launches;
-            }
-            cudaError_t e = cudaFuncSetAttribute(k_decoder_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cl_smem_bytes(v.d_ffn));
-            if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-            if (e == cudaSuccess) e = cudaGetLastError();
-            h->cl_ok = (e == cudaSuccess);
-            if (!h->cl_ok) cudaGetLastError();
-        }
-        {
-            const int max_keys = std::max(h->S_cap, h->T_cap + h->k_cap + 1);
-            size_t cap = std::min<size_t>(attn_proj_smem(max_keys, cfg->verifier.d_model), 227 * 1024);
-            if (cudaFuncSetAttribute(k_attn_proj<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cap) != cudaSuccess ||
-                cudaFuncSetAttribute(k_attn_proj<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cap) != cudaSuccess) {
-                cudaGetLastError();
-                cap = 0;
-            }
-            h->attn_proj_smem_cap = cap;
-        }
         if (sd::tc_init(h->tma, h->ses.counters + 7) != 0) h->use_tc = 0;     // reported through specdec_last_error; SIMT GEMM still runs on the GPU
-        h->lnrows_ready = h->use_tc && sd::lr_init() == cudaSuccess;
-        if (!h->lnrows_ready) cudaGetLastError();
         h->splitk_ready = h->use_tc && sd::spk_init() == cudaSuccess;
         if (!h->splitk_ready) cudaGetLastError();
         h->pair_ready = h->use_tc && sd::tc_pair_init() == cudaSuccess;
@@ -1472,6 +1381,7 @@ int specdec_destroy(specdec_handle* h) {
     if (h->enc_join) cudaEventDestroy(h->enc_join);
     if (h->fence_in) cudaEventDestroy(h->fence_in);
     if (h->fence_out) cudaEventDestroy(h->fence_out);
+    if (h->errw_ev) cudaEventDestroy(h->errw_ev);
     for (auto& e : h->poll_ev) cudaEventDestroy(e);
     for (auto& e : h->time_ev) cudaEventDestroy(e);
     for (auto& e : h->prof_ev) cudaEventDestroy(e);
@@ -1492,16 +1402,21 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         h->use_tc = value ? 1 : 0;
         return SPECDEC_OK;
     }
-    if (!strcmp(name, "cl_trace")) { h->want_cl_trace = value; return SPECDEC_OK; }   // 10 + e: time the tensor-core GEMM with epilogue e instead of the vocabulary one
-    if (!strcmp(name, "fused_attn")) { h->use_fused_attn = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "trace")) { h->want_trace = value; return SPECDEC_OK; }   // 10 + e: stamp the tensor-core GEMM with epilogue e instead of the vocabulary one
+    if (!strcmp(name, "inject_error")) {
+        // test hook: the error word reads as if a bounded device-side wait had given up; nothing waits, nothing faults
+        CUDA_TRY(h, cudaDeviceSynchronize());
+        CUDA_TRY(h, cudaMemcpy(h->ses.counters + 7, &value, 4, cudaMemcpyHostToDevice));
+        h->h_poll[ERRW_SLOT] = value; h->errw_pending = false;
+        return SPECDEC_OK;
+    }
+    if (!strcmp(name, "fused_step")) { h->use_fused_step = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
     if (!strcmp(name, "stats_timing")) { h->stats_timing = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "poll_flag")) { h->poll_flag = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "gate")) { h->use_gate = value; return SPECDEC_OK; }
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
-    if (!strcmp(name, "cluster")) { h->use_cluster = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "sk_cluster")) { h->use_sk_cluster = value < 0 ? 0 : value; return SPECDEC_OK; }   // 0 off, 1 LayerNorm-fused kernels, 2 + plain ones with K <= 512, 3 all
-    if (!strcmp(name, "ln_rows")) { h->use_ln_rows = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "ln_fuse")) { h->use_ln_fuse = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "pair")) {
         if (value && !h->pair_ready) return fail(h, SPECDEC_ERR_UNSUPPORTED, "two-SM GEMM tiles are not available on this handle");
@@ -1534,6 +1449,7 @@ int specdec_encode(specdec_handle* h, const int32_t* d_src, const int32_t* d_src
     if (B > h->B_cap || S_max > h->S_cap) return fail(h, SPECDEC_ERR_CAPACITY, "encode: B or S_max beyond capacity");
     StreamScope scope(h, stream);
     cudaStream_t st = scope.st;
+    TRY(errw_check(h, st, "encode"));
     return DISPATCH(h, encode_staged<bf16>(h, d_src, d_src_len, d_max_tgt, B, S_max, st),
                     encode_staged<float>(h, d_src, d_src_len, d_max_tgt, B, S_max, st));
 }
@@ -1545,6 +1461,7 @@ int specdec_draft(specdec_handle* h, int k, int32_t* d_draft, void* stream) {
     if (k < 1 || k > h->k_cap) return fail(h, SPECDEC_ERR_CAPACITY, "draft: k outside [1, k_max]");
     StreamScope scope(h, stream);
     cudaStream_t st = scope.st;
+    TRY(errw_check(h, st, "draft"));
     if (h->use_graphs && !h->profile) {
         const int true_ub = h->len_ub, lb = len_bucket(h, true_ub);
         h->len_ub = lb;
@@ -1566,6 +1483,7 @@ int specdec_verify(specdec_handle* h, const int32_t* d_draft, int k, int beta, f
     if (beta < 1 || !(tau >= 0.f)) return fail(h, SPECDEC_ERR_INVALID_ARG, "verify: beta >= 1 and tau >= 0 required");
     StreamScope scope(h, stream);
     cudaStream_t st = scope.st;
+    TRY(errw_check(h, st, "verify"));
     if (h->use_graphs && !h->profile) {
         const int true_ub = h->len_ub, lb = len_bucket(h, true_ub);
         int tau_bits; memcpy(&tau_bits, &tau, 4);
@@ -1587,8 +1505,9 @@ int specdec_commit(specdec_handle* h, const int32_t* d_keep, const int32_t* d_ne
     if (!h->encoded) return fail(h, SPECDEC_ERR_NOT_ENCODED, "commit: no session (call specdec_encode)");
     if (!h->verified) return fail(h, SPECDEC_ERR_INVALID_ARG, "commit: must follow specdec_verify");
     StreamScope scope(h, stream);
+    TRY(errw_check(h, scope.st, "commit"));
     int rc = commit_impl(h, d_keep, d_next, scope.st);
-    if (rc == 0) ++h->commits_issued;
+    if (rc == 0) { ++h->commits_issued; errw_fetch(h, scope.st); }
     return rc;
 }
 
@@ -1600,6 +1519,8 @@ int specdec_get_output(specdec_handle* h, int32_t* d_out, int out_stride, int32_
     StreamScope scope(h, stream);
     k_copy_out<<<h->B, 128, 0, scope.st>>>(h->ses, h->B, d_out, out_stride, d_out_len, d_finished);
     KCHECK(h);
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(scope.st, &cs) == cudaSuccess && cs == cudaStreamCaptureStatusNone) errw_fetch(h, scope.st);
     return SPECDEC_OK;
 }
 
@@ -1686,6 +1607,7 @@ namespace {
 constexpr int NA_MAX_ROWS = 4096;      // B * (k + 1)
 constexpr int NA_TILE = 1024;          // vocabulary columns per partial
 constexpr int NA_MAX_TILES = 64;       // => V <= 65536
+constexpr int NA_MAX_BLOCK = 2048;     // k + 1: 2048 records of 16 bytes + the kernel's static 256 bytes stay below the 48 KB default
 constexpr size_t NA_PART_BYTES = (size_t)NA_MAX_ROWS * NA_MAX_TILES * sizeof(RowPart);
 constexpr size_t NA_BYTES = NA_PART_BYTES + (size_t)NA_MAX_ROWS * 8;
 static __device__ __align__(256) unsigned char g_static_scratch[NA_BYTES];
@@ -1699,10 +1621,12 @@ int specdec_accept_scan_static(const float* d_logits, const int32_t* d_draft, in
         return fail(nullptr, SPECDEC_ERR_INVALID_ARG, "accept_scan_static: bad argument");
     const long long rows = (long long)B * (k + 1);
     const int n_tiles = (V + NA_TILE - 1) / NA_TILE;
-    if (rows > NA_MAX_ROWS || n_tiles > NA_MAX_TILES)
+    // the second stage keeps one merged record per row of a sequence in (default-sized) dynamic shared memory
+    if (rows > NA_MAX_ROWS || n_tiles > NA_MAX_TILES || k + 1 > NA_MAX_BLOCK)
         return fail(nullptr, SPECDEC_ERR_CAPACITY,
                     "accept_scan_static: B*(k+1) = " + std::to_string(rows) + " (limit " + std::to_string(NA_MAX_ROWS) +
-                    ") or V = " + std::to_string(V) + " (limit " + std::to_string(NA_MAX_TILES * NA_TILE) +
+                    "), V = " + std::to_string(V) + " (limit " + std::to_string(NA_MAX_TILES * NA_TILE) +
+                    ") or k+1 = " + std::to_string(k + 1) + " (limit " + std::to_string(NA_MAX_BLOCK) +
                     ") exceeds the static scratch; use specdec_accept_scan");
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
@@ -1743,11 +1667,10 @@ int specdec_debug_logits(specdec_handle* h, int which, float* d_logits, void* st
                     gemm<float>(h, EPI_F32, h->y, d, m->embed, nullptr, V, d, cnt, rows, nullptr, 0, d_logits, st));
 }
 
-int specdec_debug_cluster_trace(specdec_handle* h, long long* h_out, int n) {
+int specdec_debug_trace(specdec_handle* h, long long* h_out, int n) {
     if (!h || !h_out || n < 1 || n > 256) return SPECDEC_ERR_INVALID_ARG;
-    if (!h->cl_trace) return fail(h, SPECDEC_ERR_UNSUPPORTED, "cluster decoder kernel not available for this model");
     CUDA_TRY(h, cudaDeviceSynchronize());
-    CUDA_TRY(h, cudaMemcpy(h_out, h->cl_trace, (size_t)n * 8, cudaMemcpyDeviceToHost));
+    CUDA_TRY(h, cudaMemcpy(h_out, h->trace_buf, (size_t)n * 8, cudaMemcpyDeviceToHost));
     return SPECDEC_OK;
 }
 
