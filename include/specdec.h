@@ -218,8 +218,6 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
  * "skinny"       0/1 weight-streaming GEMM with fused LayerNorm for passes of at most 32 rows (default 1)
  * "sk_cluster"   0 off / 1 (default): those GEMMs run in clusters of 8 CTAs that share the normalised input rows
  *                through distributed shared memory; 2 / 3 also the GEMMs without a LayerNorm (K <= 512 / all)
- * "fused_step"   0 never / 1 (default) where it applies: the verifier's decoder stack of a step as ONE kernel, one
- *                16-CTA cluster per sequence (verify blocks of at most 32 rows, 8 heads of 64, at most 8 sequences)
  * "pair"         0/1 two-SM tensor-core tiles (cta_group::2) for GEMMs with >= 1024 rows and columns (default 0)
  * "ln_fuse"      0/1 the LayerNorm that reads the residual stream next runs inside the residual GEMM (default 0)
  * "splitk"       0/1 residual GEMMs with K >= 1024 over few row tiles split K across a cluster (default 1)

@@ -88,7 +88,6 @@ struct specdec_handle {
     int last_draft_rows_ub = 0;
     // options
     int use_tc = 1, use_graphs = 1, use_tc_attn = 1, want_lse = 0, use_skinny = 1, use_pdl = 1;
-    int use_fused_step = 1;         // the verifier's decoder stack of a step as one cluster kernel per sequence (option "fused_step")
     long long* trace_buf = nullptr; // device [256] in-kernel time stamps (option "trace")
     int want_trace = 0;
     size_t skinny_smem_cap = 0;
@@ -928,7 +927,7 @@ inline void graph_key_tail(const specdec_handle* h, std::vector<long long>& key)
     for (long long v : {(long long)h->use_tc, (long long)h->use_tc_attn, (long long)h->want_lse, (long long)h->use_skinny,
                         (long long)h->use_pdl, (long long)h->use_ln_fuse, (long long)h->use_sk_cluster,
                         (long long)h->use_pair, (long long)h->diag_repeat, (long long)h->use_splitk, (long long)h->attn_stream, (long long)h->attn_stream_keys, (long long)h->attn_warps, (long long)h->attn_rs,
-                        (long long)h->skinny_groups, (long long)h->want_trace, (long long)h->use_fused_step,
+                        (long long)h->skinny_groups, (long long)h->want_trace,
                         (long long)(h->script_on ? 1 : 0), (long long)h->B, (long long)h->S_max})
         key.push_back(v);
 }
@@ -1410,7 +1409,6 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         h->h_poll[ERRW_SLOT] = value; h->errw_pending = false;
         return SPECDEC_OK;
     }
-    if (!strcmp(name, "fused_step")) { h->use_fused_step = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
     if (!strcmp(name, "stats_timing")) { h->stats_timing = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "poll_flag")) { h->poll_flag = value ? 1 : 0; return SPECDEC_OK; }

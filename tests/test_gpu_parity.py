@@ -361,16 +361,16 @@ def test_bf16_streaming_attention(long_keys, mode):
     sd.close()
 
 
-@pytest.mark.parametrize("fused_step", [1, 0])
-def test_base_shapes_batch1_lockstep(fused_step):
-    """One config-2 sentence at batch 1 (26-row verify block): the verifier's decoder stack as one cluster kernel
-    per sequence (fused_step = 1, the default) or as per-operation kernels with the weight-streaming GEMM."""
+@pytest.mark.parametrize("sk_cluster", [1, 0])
+def test_base_shapes_batch1_lockstep(sk_cluster):
+    """One config-2 sentence at batch 1 (26-row verify block): per-operation kernels with the weight-streaming GEMM,
+    its LayerNorm prologue shared across clusters of 8 CTAs (the default) or computed by every CTA."""
     wl = W.config2_translation(1)
     wv = W.make_weights(wl.verifier, wl.seed_verifier, True)
     wd = W.make_weights(wl.drafter, wl.seed_drafter, True)
     mv, md = O.model_from(wl.verifier, wv, mode="bf16"), O.model_from(wl.drafter, wd, mode="bf16")
     sd = _handle(wl.verifier, wv, wl.drafter, wd, True, k_max=25, max_batch=1, max_src=40, max_tgt=64)
-    sd.set_option("fused_step", fused_step)
+    sd.set_option("sk_cluster", sk_cluster)
     rep = lockstep.run(sd, mv, md, wl.src, wl.max_tgt, 25, 3, 1.0, margin=1e-3, check_logits_every=4, max_iters=8)
     print(rep.iterations, rep.draft_positions, rep.draft_near_ties, rep.verify_rows, rep.verify_near_ties,
           rep.max_logit_err, rep.max_stat_err, rep.notes[:5])
