@@ -4,8 +4,12 @@
 One step = one call of specdec_generate (encode + every draft/verify/commit round
 until the sequences finish) on one batch of the translation-shaped workload
 (Transformer-base verifier 6+6, drafter 12+2, d=512, vocab 32768, k=25, beta=3,
-tau=1.0; sources of 20..40 Zipf ids; batch 1 by default, --batch 128 for the
-padded-batch shape with sources of 10..80 ids).  Random-init models almost never
+tau=1.0; sources of 20..40 Zipf ids at batch 1).  The default run also carries the
+metric's second half in the same line: `roofline` = one verify step at (batch 1,
+k = 25, 64 committed tokens) against the HBM roofline, and `batch128` = tokens/s
+on the padded batch of 128 (sources of 10..80 ids) with its verify step against
+the bf16 tensor roofline.  The timed region repeats the K-step stream until it is
+at least two seconds long.  Random-init models almost never
 agree, so the acceptance pattern of the paper's regime is imposed through the
 library's scripted-draft hook: the drafter runs in full, then its output is
 replaced by the verifier's own greedy continuation with a rejected token every
@@ -177,23 +181,13 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------ CUDA arm
-def run_ours(args):
-    import torch
-    import torch.distributed as dist
-    from paper_2203_16487_b200 import binding
+MIN_TIMED_MS = 2000.0          # the timed region repeats the K-step stream until it is at least this long
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+def tokens_leg(torch, binding, B: int, K_: int, W_: int, rank: int, world: int, local: int, opts, poll_lag, want_breakdown: bool):
+    """Generated tokens/s of specdec_generate on the batch-B workload: device-resident inputs, host buffers (e2e),
+    the unscripted drafter, greedy autoregressive decoding (k = 0) and the per-phase split."""
     dev = torch.device("cuda", local)
-    hbm_peak, tc_peak, peak_kind = load_peaks()
-
-    B = args.batch
     wl, name = workload(B)
     wv = W.make_weights(wl.verifier, wl.seed_verifier, True)
     wd = W.make_weights(wl.drafter, wl.seed_drafter, True)
@@ -202,14 +196,14 @@ def run_ours(args):
     sd = binding.SpecDec(wl.verifier, wv, wl.drafter, wd, k_max=K_BLOCK, max_batch=B, max_src=max_src,
                          max_tgt=max_tgt, bf16=True, device=f"cuda:{local}")
     del wv, wd
-    if args.poll_lag is not None:
-        sd.set_option("poll_lag", args.poll_lag)
-    for kv in args.opt:
-        name, _, val = kv.partition("=")
-        sd.set_option(name, int(val))
+    if poll_lag is not None:
+        sd.set_option("poll_lag", poll_lag)
+    for kv in opts:
+        opt_name, _, val = kv.partition("=")
+        sd.set_option(opt_name, int(val))
 
     # the step stream: rank r takes batches r, r + world, ... (replicas; no data-path collective)
-    n_total = args.warmup + args.steps
+    n_total = W_ + K_
     n_batches = max(len(wl.src) // B, 1)
 
     def batch_of(step):
@@ -227,132 +221,225 @@ def run_ours(args):
         out, n, _ = sd.generate(src, lens, mts, K_BLOCK, 1, 0.0)
         out, n = out.cpu().numpy(), n.cpu().numpy()
         script = np.stack([make_script(out[b], int(n[b]), rng, wl.verifier.vocab, max_tgt + K_BLOCK) for b in range(B)])
-        steps_in.append((src, lens, mts, script, out, n))
-
-    def dev_inputs(s):
-        src, lens, mts, script, _, _ = steps_in[s]
-        return (torch.from_numpy(src).to(dev), torch.from_numpy(lens).to(dev), torch.from_numpy(mts).to(dev), script)
+        dv = (torch.from_numpy(src).to(dev), torch.from_numpy(lens).to(dev), torch.from_numpy(mts).to(dev))
+        hv = tuple(torch.from_numpy(a).pin_memory() for a in (src, lens, mts))
+        steps_in.append((dv, hv, script, out, n))
+    ho = torch.zeros((B, max_tgt), dtype=torch.int32).pin_memory()
+    hn = torch.zeros(B, dtype=torch.int32).pin_memory()
 
     def barrier():
+        import torch.distributed as dist
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
     diverged = [0]
 
-    def timed_pass(first, count, host: bool, scripted: bool = True, k: int = K_BLOCK):
-        """Runs steps [first, first+count); returns (tokens, ms, stats list)."""
+    def one_pass(first, count, host, scripted, k, check):
         toks, ms, stats = 0, 0.0, []
         for s in range(first, first + count):
-            src, lens, mts, script, ref_out, ref_n = steps_in[s]
+            dv, hv, script, ref_out, ref_n = steps_in[s]
             sd.set_draft_script(script if scripted else None)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            if host:
-                hs, hl, hm = (torch.from_numpy(a).pin_memory() for a in (src, lens, mts))
-                ho = torch.zeros((B, max_tgt), dtype=torch.int32).pin_memory()
-                hn = torch.zeros(B, dtype=torch.int32).pin_memory()
-                torch.cuda.synchronize()
-                e0.record()
-                st = sd.generate_host(hs, hl, hm, ho, hn, k, BETA, TAU, want_stats=True)
-                e1.record()
-                n = hn.numpy()
-                out = ho.numpy()
-            else:
-                dsrc, dlen, dmt, _ = dev_inputs(s)
-                torch.cuda.synchronize()
-                e0.record()
-                o, nn, st = sd.generate(dsrc, dlen, dmt, k, BETA, TAU)
-                e1.record()
-                out, n = o.cpu().numpy(), nn.cpu().numpy()
             torch.cuda.synchronize()
+            if host:
+                e0.record()
+                st = sd.generate_host(hv[0], hv[1], hv[2], ho, hn, k, BETA, TAU, want_stats=True)
+                e1.record()
+                torch.cuda.synchronize()
+                n, out = hn.numpy(), ho.numpy()
+            else:
+                e0.record()
+                o, nn, st = sd.generate(dv[0], dv[1], dv[2], k, BETA, TAU)
+                e1.record()
+                torch.cuda.synchronize()
+                n = nn.cpu().numpy()
+                out = o.cpu().numpy() if check else None
             ms += e0.elapsed_time(e1)
             toks += int(n.sum())
             stats.append(st)
-            if scripted:       # greedy drafts are always accepted: the result should be the greedy output
+            if check and scripted:      # greedy drafts are always accepted: the result must be the greedy output
                 for b in range(B):
                     if out[b, :n[b]].tolist() != ref_out[b, :ref_n[b]].tolist():
                         diverged[0] += 1
         return toks, ms, stats
 
-    W_, K_ = args.warmup, args.steps
-    timed_pass(0, W_, host=False)                                   # warm-up (untimed)
+    def timed(host=False, scripted=True, k=K_BLOCK, min_ms=MIN_TIMED_MS):
+        """The K-step stream, repeated until the region is at least min_ms long; returns (tokens, ms, stats, repeats)."""
+        toks, ms, stats, reps = 0, 0.0, [], 0
+        while reps == 0 or ms < min_ms:
+            t, m, st = one_pass(W_, K_, host, scripted, k, check=(reps == 0))
+            toks += t; ms += m; stats += st; reps += 1
+            if reps >= 400:
+                break
+        return toks, ms, stats, reps
+
+    one_pass(0, W_, False, True, K_BLOCK, False)                      # warm-up (untimed)
     sampler = ClockSampler(local)
     barrier()
     sampler.start()
     l0 = sd.launch_count()
-    toks, ms, stats = timed_pass(W_, K_, host=False)
+    toks, ms, stats, reps = timed()
     launches = sd.launch_count() - l0
     barrier()
     clocks = sampler.stop()
-    e_toks, e_ms, _ = timed_pass(W_, K_, host=True)                 # end to end, host buffers
-    n_toks, n_ms, n_stats = timed_pass(W_, K_, host=False, scripted=False)   # unscripted drafter
-    timed_pass(0, min(W_, 1), host=False, scripted=False, k=0)               # one untimed step: the k = 0 graphs are captured here
-    a_toks, a_ms, _ = timed_pass(W_, K_, host=False, scripted=False, k=0)    # greedy autoregressive baseline (verifier alone)
-    # dominant kernel: the vocabulary projection with fused row statistics
-    sd.set_option("profile", 1)
-    timed_pass(W_, K_, host=False)
-    vocab_ms, vocab_n = sd.profile_read()
-    sd.set_option("profile", 0)
-    # per-phase times: a pass of its own, because an event after every phase keeps the host from queueing whole
-    # iterations ahead (the timed pass above records none)
-    sd.set_option("stats_timing", 1)
-    _, _, ph_stats = timed_pass(W_, K_, host=False)
-    sd.set_option("stats_timing", 0)
-
+    e_toks, e_ms, _, e_reps = timed(host=True)                        # end to end, host buffers
+    n_toks, n_ms, n_stats, _ = timed(scripted=False, min_ms=MIN_TIMED_MS / 4)     # unscripted drafter
+    one_pass(0, min(W_, 1), False, False, 0, False)                   # the k = 0 graphs are captured here
+    a_toks, a_ms, _, _ = timed(scripted=False, k=0, min_ms=MIN_TIMED_MS / 4)      # greedy autoregressive baseline
+    ph = None
+    if want_breakdown:
+        # per-phase times: a pass of its own, because an event after every phase keeps the host from queueing whole
+        # iterations ahead (the timed pass above records none)
+        sd.set_option("stats_timing", 1)
+        _, _, ph_stats = one_pass(W_, K_, False, True, K_BLOCK, False)
+        sd.set_option("stats_timing", 0)
+        ph = dict({k: sum(s[k] for s in ph_stats) / max(K_, 1) for k in ("ms_encode", "ms_draft", "ms_verify", "ms_commit", "ms_total")},
+                  note="separate untimed pass with an event after every phase (option stats_timing): each iteration "
+                       "then waits for the host, so ms_total here exceeds ms_per_step")
+    sd.close()
     toks_all, ms_max = replicas.reduce_job(toks, ms, dev)
     e_toks_all, e_ms_max = replicas.reduce_job(e_toks, e_ms, dev)
     n_toks_all, n_ms_max = replicas.reduce_job(n_toks, n_ms, dev)
     a_toks_all, a_ms_max = replicas.reduce_job(a_toks, a_ms, dev)
-
-    it = sum(s["iterations"] for s in stats)
     seq_it = sum(s["seq_iterations"] for s in stats)
-    acc = sum(s["accepted"] for s in stats)
-    d, V = wl.verifier.d_model, wl.verifier.vocab
-    rows = B * (K_BLOCK + 1)
-    # column halves per row that the kernel writes 16-byte partial statistics for: one 224-wide tile per SM up to
-    # 128 rows, 128-wide tiles up to 512 rows, 256-wide above (the library's tile rule for this kernel)
-    tile = 224 if rows <= 128 else (128 if rows <= 512 else 256)
-    n_part = 2 * ((V + tile - 1) // tile)
-    alg_bytes = V * d * 2 + rows * d * 2 + rows * n_part * 16 + rows * 8
-    per_launch_ms = vocab_ms / max(vocab_n, 1)
-    achieved = alg_bytes / (per_launch_ms * 1e-3) / 1e9 if per_launch_ms > 0 else 0.0
-    flops = 2.0 * rows * d * V
-    tf = flops / (per_launch_ms * 1e-3) / 1e12 if per_launch_ms > 0 else 0.0
-    bound_hbm = (alg_bytes / (hbm_peak * 1e9)) >= (flops / (tc_peak * 1e12))
-    roof = ({"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak}
-            if bound_hbm else
-            {"bound": "tensor", "achieved": tf, "peak": tc_peak, "unit": "TFLOP/s", "frac": tf / tc_peak})
-    # DRAM bytes of one launch from the ncu capture summarised in profiles/vocab_stats_kernel_b1_ncu.md
-    # (dram__bytes_read.sum + dram__bytes_write.sum at 26 rows); none was taken at other row counts
-    traffic = 33608960 if B == 1 else None
-    roof.update({"traffic": traffic, "kernel": "k_gemm_tc<EPI_STATS> (vocabulary projection + row statistics, verify step)",
-                 "peak_kind": f"of {peak_kind}", "launches_timed": int(vocab_n), "us_per_launch": per_launch_ms * 1e3,
-                 "algorithmic_bytes_per_launch": alg_bytes})
-
-    line = {
-        "metric": "generated tokens/s", "value": toks_all / (ms_max * 1e-3), "unit": "tokens/s",
-        "n_gpus": world, "steps": K_, "warmup": W_, "ms_per_step": ms_max / max(K_, 1),
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": config_of(name, B, world),
+    ar = a_toks_all / (a_ms_max * 1e-3)
+    leg = {
+        "workload": name, "value": toks_all / (ms_max * 1e-3), "unit": "tokens/s",
+        "ms_per_step": ms_max / max(K_ * reps, 1), "timed_ms": ms_max, "repeats": reps,
         "e2e": {"value": e_toks_all / (e_ms_max * 1e-3), "unit": "tokens/s",
                 "h2d_bytes_per_step": int(B * max_src * 4 + B * 8), "d2h_bytes_per_step": int(B * max_tgt * 4 + B * 4)},
-        "gpu_launches": int(launches),
-        "clocks": clocks,
-        "roofline": roof,
-        "tok_per_iteration": {"accepted": acc / max(seq_it, 1), "emitted": toks / max(seq_it, 1)},
-        "iterations": it,
+        "gpu_launches": int(launches), "clocks": clocks,
+        "tok_per_iteration": {"accepted": sum(s["accepted"] for s in stats) / max(seq_it, 1), "emitted": toks / max(seq_it, 1)},
+        "iterations": sum(s["iterations"] for s in stats),
         "scripted_runs_differing_from_greedy": diverged[0],
-        "ms_breakdown": dict({k: sum(s[k] for s in ph_stats) / max(K_, 1) for k in ("ms_encode", "ms_draft", "ms_verify", "ms_commit", "ms_total")},
-                             note="separate untimed pass with an event after every phase (option stats_timing): each iteration "
-                                  "then waits for the host, so ms_total here exceeds ms_per_step"),
         "unscripted": {"value": n_toks_all / (n_ms_max * 1e-3), "unit": "tokens/s",
                        "tok_per_iteration": sum(s["emitted"] for s in n_stats) / max(sum(s["seq_iterations"] for s in n_stats), 1)},
+        "greedy_ar": {"value": ar, "unit": "tokens/s", "specdec_speedup": toks_all / (ms_max * 1e-3) / ar,
+                      "note": "k = 0: the verifier alone, one token per step, same kernels; the paper reports SpecDec at "
+                              "about 4.6x greedy (5.1x / 1.1x over beam-5, Table 1) on a P100 with trained models"},
     }
+    if ph:
+        leg["ms_breakdown"] = ph
+    return leg
 
-    ar = a_toks_all / (a_ms_max * 1e-3)
-    line["greedy_ar"] = {"value": ar, "unit": "tokens/s", "specdec_speedup": line["value"] / ar,
-                         "note": "k = 0: the verifier alone, one token per step, same kernels; the paper reports SpecDec at "
-                                 "about 4.6x greedy (5.1x / 1.1x over beam-5, Table 1) on a P100 with trained models"}
+
+# DRAM bytes of one launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
+# profiles/, keyed by (batch, kernel class); cells that were never captured are absent and reported as null
+NCU_TRAFFIC = {(1, "vocabulary"): 33608960}
+
+
+def verify_step_roofline(torch, binding, B: int, local: int, opts, reps: int = 50):
+    """The metric's second half: one verify step at (B, k = 25, committed prefix 64, source 64), L2 flushed between
+    repetitions, against the HBM roofline (weights + K/V once) or the bf16 tensor roofline (batch 128); with the cost
+    of each kernel class inside the step (every launch of the class issued twice: the step grows by the class's cost)."""
+    from paper_2203_16487_b200 import microbench as MB
+    hbm_peak, tc_peak, peak_kind = load_peaks()
+    peaks_all = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if peak_kind == "measured" else {}
+    k, j, S = K_BLOCK, 64, 64
+    wl = W.config5_microbench(B, S)
+    wv = W.make_weights(wl.verifier, wl.seed_verifier, True)
+    wd = W.make_weights(wl.drafter, wl.seed_drafter, True)
+    sd = binding.SpecDec(wl.verifier, wv, wl.drafter, wd, k_max=k, max_batch=B, max_src=S, max_tgt=j + k + 2, bf16=True,
+                         device=f"cuda:{local}")
+    del wv, wd
+    for kv in opts:
+        opt_name, _, val = kv.partition("=")
+        sd.set_option(opt_name, int(val))
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=f"cuda:{local}")
+    l0 = sd.launch_count()
+    us, us_min, mean_a = MB.measure(sd, wl, B, k, j, S, reps, 5, flush)
+    n_calls = None
+    params, bytes_, flops = MB.algorithmic_work(B, k, j, S, wl.verifier)
+    # launches of one step: count them on one extra call
+    c0 = sd.launch_count()
+    d = torch.zeros((B, k), dtype=torch.int32, device=f"cuda:{local}")
+    acc_t = torch.zeros(B, dtype=torch.int32, device=f"cuda:{local}"); bif_t = torch.zeros_like(acc_t)
+    sd.verify_raw(d, BETA, TAU, acc_t, bif_t)
+    torch.cuda.synchronize()
+    launches_per_step = sd.launch_count() - c0
+    by_kernel = []
+    d_model, V = wl.verifier.d_model, wl.verifier.vocab
+    rows = B * (k + 1)
+    classes = [(1, "attention (self + cross)", 2 * wl.verifier.dec_layers, B * wl.verifier.dec_layers * (j + k + 1 + S) * 2 * d_model * 2),
+               (2, "LayerNorm launches", None, None),
+               (4, "layer GEMMs without residual (QKV, cross-Q, FFN1)", 3 * wl.verifier.dec_layers,
+                wl.verifier.dec_layers * (3 * d_model * d_model + d_model * d_model + wl.verifier.d_ffn * d_model) * 2),
+               (8, "vocabulary projection + row statistics", 1, V * d_model * 2 + rows * d_model * 2)]
+    for bit, label, n_launch, cls_bytes in classes:
+        sd.set_option("diag_repeat", bit)
+        us_c, _, _ = MB.measure(sd, wl, B, k, j, S, max(reps // 2, 10), 3, flush)
+        sd.set_option("diag_repeat", 0)
+        cost = max(us_c - us, 0.0)
+        e = {"class": label, "launches": n_launch, "us_in_step": cost, "share_of_step": cost / us}
+        if cls_bytes:
+            e["algorithmic_bytes"] = int(cls_bytes)
+            e["hbm_frac"] = (cls_bytes / (cost * 1e-6) / 1e9 / hbm_peak) if cost > 0 else None
+        if bit == 8:
+            e["traffic"] = NCU_TRAFFIC.get((B, "vocabulary"))
+        by_kernel.append(e)
+    rest = us - sum(e["us_in_step"] for e in by_kernel)
+    by_kernel.append({"class": "residual GEMMs (attention out x2, FFN2), embedding, accept scan, the rest", "launches": None,
+                      "us_in_step": rest, "share_of_step": rest / us})
+    sd.close()
+    del flush
+    hbm_bound = (bytes_ / (hbm_peak * 1e9)) >= (flops / (tc_peak * 1e12))
+    if hbm_bound:
+        achieved = bytes_ / (us * 1e-6) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s", "frac": achieved / hbm_peak}
+    else:
+        achieved = flops / (us * 1e-6) / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": tc_peak, "unit": "TFLOP/s", "frac": achieved / tc_peak}
+        sus = peaks_all.get("bf16_tflops_sustained")
+        if sus:
+            roof["frac_of_sustained_peak"] = achieved / float(sus)
+    roof.update({
+        "traffic": None, "traffic_note": "no ncu capture of the whole step at this batch; per-class captures are listed under by_kernel",
+        "kernel": f"verify step (all {launches_per_step} launches): B={B}, k={k}, committed prefix {j}, source {S}, L2 flushed between repetitions",
+        "peak_kind": f"of {peak_kind}", "us_per_step_median": us, "us_per_step_min": us_min, "repetitions": reps,
+        "launches_per_step": int(launches_per_step), "algorithmic_bytes_per_launch": int(bytes_), "algorithmic_flops_per_launch": flops,
+        "roofline_us": max(bytes_ / (hbm_peak * 1e9), flops / (tc_peak * 1e12)) * 1e6, "mean_accepted": mean_a, "by_kernel": by_kernel,
+    })
+    return roof
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2203_16487_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    B = args.batch
+    leg = tokens_leg(torch, binding, B, args.steps, args.warmup, rank, world, local, args.opt, args.poll_lag, True)
+    line = {
+        "metric": "generated tokens/s", "value": leg["value"], "unit": "tokens/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": leg["ms_per_step"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": dict(config_of(leg["workload"], B, world), timed_region_ms=leg["timed_ms"],
+                       repeats_of_the_step_stream=leg["repeats"]),
+    }
+    for key in ("e2e", "gpu_launches", "clocks", "tok_per_iteration", "iterations", "scripted_runs_differing_from_greedy",
+                "ms_breakdown", "unscripted", "greedy_ar"):
+        if key in leg:
+            line[key] = leg[key]
+    if rank == 0:
+        # the verify step against its roofline (rank 0: a single-GPU measurement)
+        line["roofline"] = verify_step_roofline(torch, binding, B, local, args.opt)
+    if B == 1 and not args.no_batch128:
+        # the metric's batch-128 half, in the same line: tokens/s on the padded-batch workload and the verify step
+        # against the tensor roofline
+        b128 = tokens_leg(torch, binding, 128, min(args.steps, 6), args.warmup, rank, world, local, args.opt, args.poll_lag, False)
+        if rank == 0:
+            b128["roofline"] = verify_step_roofline(torch, binding, 128, local, args.opt, reps=30)
+        b128["config"] = config_of(b128.pop("workload"), 128, world)
+        line["batch128"] = b128
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         wl1, name1 = workload(1)
         O, mv, md = oracle_models(wl1)
@@ -365,9 +452,20 @@ def run_ours(args):
                                 "sample": f"first {n_s} sentences of {name1}, batch 1, same scripted acceptance; {csecs:.1f} s"}
     if rank == 0:
         print(json.dumps(line))
-    sd.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def spawn_replicas(args) -> int:
+    """`python bench.py --gpus N` without a launcher: start the N ranks here (one process per GPU, NCCL only for the
+    final max / sum) and pass their single JSON line through."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -378,12 +476,15 @@ def main():
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-batch128", action="store_true", help="skip the batch-128 leg of the default (batch 1) run")
     ap.add_argument("--opt", action="append", default=[], help="experiments: name=value passed to specdec_set_option")
     ap.add_argument("--poll-lag", type=int, default=None, help="experiments: iterations the host runs ahead of the finish counter")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(spawn_replicas(args))
     else:
         run_ours(args)
 
