@@ -201,6 +201,12 @@ int specdec_debug_row_stats(specdec_handle* h, float* d_stats, void* stream);
  * 256-entry device array; this copies the first n (<= 256) entries to the host.  Synchronises the device. */
 int specdec_debug_trace(specdec_handle* h, long long* h_out, int n);
 
+/* Diagnostics: the cost of one kernel boundary inside a step.  Replays (from a CUDA graph, on the handle's own stream)
+ * a chain of n_links launches of `grid` CTAs, each of which waits for its predecessor (programmatic dependent
+ * launch, as between the kernels of a step), reads the word it wrote and writes it back; returns the best of ten
+ * replays divided by n_links, in microseconds.  Synchronises. */
+int specdec_debug_link_cost(specdec_handle* h, int n_links, int grid, double* h_us_per_link);
+
 /* Scripted drafts, a benchmark / test hook with no counterpart in the paper: random-init
  * models almost never agree, so a workload's acceptance pattern is imposed instead.  After the
  * drafter pass has run, draft i of a sequence with j committed tokens is replaced by

@@ -24,7 +24,7 @@ EXPORTS = [
     "specdec_commit", "specdec_generate", "specdec_generate_host", "specdec_get_output",
     "specdec_accept_scan", "specdec_debug_logits", "specdec_debug_row_stats", "specdec_set_option",
     "specdec_launch_count", "specdec_last_error", "specdec_set_draft_script", "specdec_profile_read",
-    "specdec_accept_scan_static", "specdec_debug_trace",
+    "specdec_accept_scan_static", "specdec_debug_trace", "specdec_debug_link_cost",
 ]
 
 
@@ -78,6 +78,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.specdec_accept_scan_static.argtypes = [vp, ip, i, i, i, i, f, ip, ip, vp]
     lib.specdec_debug_logits.argtypes = [vp, i, vp, vp]
     lib.specdec_debug_row_stats.argtypes = [vp, vp, vp]
+    lib.specdec_debug_link_cost.argtypes = [vp, i, i, C.POINTER(C.c_double)]
     lib.specdec_debug_trace.argtypes = [vp, C.POINTER(C.c_longlong), i]
     lib.specdec_set_option.argtypes = [vp, C.c_char_p, i]
     lib.specdec_set_draft_script.argtypes = [vp, ip, i, i, vp]
@@ -190,6 +191,12 @@ class SpecDec:
         ms, n = C.c_double(), C.c_longlong()
         self._check(self._lib.specdec_profile_read(self._h, C.byref(ms), C.byref(n)))
         return ms.value, n.value
+
+    def link_cost(self, n_links: int = 64, grid: int = 148) -> float:
+        """Microseconds per kernel boundary in a chain of dependent launches (diagnostics)."""
+        us = C.c_double()
+        self._check(self._lib.specdec_debug_link_cost(self._h, n_links, grid, C.byref(us)))
+        return us.value
 
     def trace(self, n: int):
         buf = (C.c_longlong * n)()

@@ -59,6 +59,15 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
+// One link of a chain of dependent launches (diagnostics: what one kernel boundary costs inside a step): waits for its
+// predecessor, reads the word it wrote, and the first thread writes it back incremented.
+__global__ void k_link(int* word) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int v = *reinterpret_cast<volatile int*>(word);
+    if (blockIdx.x == 0 && threadIdx.x == 0) *word = v + 1;
+}
+
 // Device-resident session state shared by the kernels of one handle.
 struct Session {
     int* len;          // [B] committed target tokens j_b

@@ -40,7 +40,11 @@ struct ModelW {
     float *pos_enc, *pos_dec;
     std::vector<LayerW> enc, dec;
     float *enc_lnf_g, *enc_lnf_b, *dec_lnf_g, *dec_lnf_b;
-    std::vector<void*> ckv;   // per decoder layer: cross K/V of the session [B*S_max, 2d]
+    // cross-attention K | V of the session for every decoder layer: one buffer [B*S_max, dec_layers * 2d] written by a
+    // single projection of the encoder memory (the layers' K/V matrices are stored back to back); ckv[l] = its
+    // column block l, ckv_stride = elements per row
+    std::vector<void*> ckv;
+    int ckv_stride = 0;
 };
 
 struct Arena {
@@ -210,7 +214,6 @@ void layout_model(specdec_handle* h, ModelW& m, const specdec_model_dims& dm) {
         w.ln1_g = vec(d); w.ln1_b = vec(d); w.ln2_g = vec(d); w.ln2_b = vec(d);
         if (dec) {
             w.cq_w = A.take(d * d * e); w.cq_b = vec(d);
-            w.ckv_w = A.take(2 * d * d * e); w.ckv_b = vec(2 * d);
             w.co_w = A.take(d * d * e); w.co_b = vec(d);
             w.lnc_g = vec(d); w.lnc_b = vec(d);
         }
@@ -219,9 +222,21 @@ void layout_model(specdec_handle* h, ModelW& m, const specdec_model_dims& dm) {
     m.dec.resize(dm.dec_layers);
     for (auto& w : m.enc) layer(w, false);
     for (auto& w : m.dec) layer(w, true);
+    {   // the decoder layers' cross K/V projections, contiguous: [dec_layers * 2d, d] and [dec_layers * 2d]
+        char* wall = (char*)A.take((size_t)dm.dec_layers * 2 * d * d * e);
+        float* ball = vec((size_t)dm.dec_layers * 2 * d);
+        for (int l = 0; l < dm.dec_layers; ++l) {
+            m.dec[l].ckv_w = wall ? wall + (size_t)l * 2 * d * d * e : nullptr;
+            m.dec[l].ckv_b = ball ? ball + (size_t)l * 2 * d : nullptr;
+        }
+    }
     m.enc_lnf_g = vec(d); m.enc_lnf_b = vec(d); m.dec_lnf_g = vec(d); m.dec_lnf_b = vec(d);
     m.ckv.resize(dm.dec_layers);
-    for (auto& p : m.ckv) p = A.take((size_t)h->B_cap * h->S_cap * 2 * d * e);
+    m.ckv_stride = dm.dec_layers * 2 * (int)d;
+    {
+        char* all = (char*)A.take((size_t)h->B_cap * h->S_cap * m.ckv_stride * e);
+        for (int l = 0; l < dm.dec_layers; ++l) m.ckv[l] = all ? all + (size_t)l * 2 * d * e : nullptr;
+    }
 }
 
 void layout_rows(Arena& A, Rows& r, int n, int B) {
@@ -715,7 +730,7 @@ int block_cross(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, c
     const LnSpec lc{x, w.lnc_g, w.lnc_b};
     TRY(gemm<T>(h, EPI_STORE, h->y, d, w.cq_w, w.cq_b, d, d, cnt, rows_ub, h->q, d, nullptr, st, nullptr, nullptr, nullptr,
                 nullptr, &lc));
-    TRY(attn<T>(h, false, h->q, d, nullptr, m.ckv[layer], (char*)m.ckv[layer] + (size_t)d * e, 2 * d, r.kv_off_cross,
+    TRY(attn<T>(h, false, h->q, d, nullptr, m.ckv[layer], (char*)m.ckv[layer] + (size_t)d * e, m.ckv_stride, r.kv_off_cross,
                 r, r.nk_cross, cnt, rows_ub, q_ub, h->att, d, H, dh, h->S_max, st, h->ses.src_len));   // encoder K/V: all of it
     h->next_ln = {w.ln2_g, w.ln2_b, h->y};           // the feed-forward sublayer's LayerNorm comes next
     TRY(gemm<T>(h, EPI_RESID, h->att, d, w.co_w, w.co_b, d, d, cnt, rows_ub, nullptr, 0, x, st));
@@ -763,9 +778,9 @@ int encode_model(specdec_handle* h, ModelW& m, cudaStream_t st) {
                          last ? m.enc_lnf_b : m.enc[l + 1].ln1_b, last ? h->mem : nullptr));
     }
     TRY(ln_or_fused<T>(h, h->x, m.enc_lnf_g, m.enc_lnf_b, CNT_ENC, R, h->mem, d, st));
-    for (int l = 0; l < m.dm.dec_layers; ++l)
-        TRY(gemm<T>(h, EPI_STORE, h->mem, d, m.dec[l].ckv_w, m.dec[l].ckv_b, 2 * d, d, CNT_ENC, R, m.ckv[l], 2 * d,
-                    nullptr, st));
+    // cross-attention K / V of every decoder layer in one projection ("the encoder is forwarded only once", Section 3.1.2)
+    TRY(gemm<T>(h, EPI_STORE, h->mem, d, m.dec[0].ckv_w, m.dec[0].ckv_b, m.ckv_stride, d, CNT_ENC, R, m.ckv[0], m.ckv_stride,
+                nullptr, st));
     return 0;
 }
 
@@ -1669,6 +1684,38 @@ int specdec_debug_trace(specdec_handle* h, long long* h_out, int n) {
     if (!h || !h_out || n < 1 || n > 256) return SPECDEC_ERR_INVALID_ARG;
     CUDA_TRY(h, cudaDeviceSynchronize());
     CUDA_TRY(h, cudaMemcpy(h_out, h->trace_buf, (size_t)n * 8, cudaMemcpyDeviceToHost));
+    return SPECDEC_OK;
+}
+
+int specdec_debug_link_cost(specdec_handle* h, int n_links, int grid, double* h_us_per_link) {
+    if (!h || !h_us_per_link || n_links < 1 || n_links > 4096 || grid < 1 || grid > 65535) return SPECDEC_ERR_INVALID_ARG;
+    cudaStream_t st = h->own_stream;
+    int* word = h->ses.counters + 6;                 // (a counter no kernel of the path reads)
+    cudaGraph_t g = nullptr; cudaGraphExec_t ex = nullptr;
+    CUDA_TRY(h, cudaStreamSynchronize(st));
+    CUDA_TRY(h, cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+    cudaError_t e = cudaSuccess;
+    for (int i = 0; i < n_links && e == cudaSuccess; ++i) e = launch_pdl(h, k_link, dim3(grid), dim3(128), 0, st, word);
+    cudaError_t e2 = cudaStreamEndCapture(st, &g);
+    if (e != cudaSuccess || e2 != cudaSuccess || !g) { if (g) cudaGraphDestroy(g); return fail(h, SPECDEC_ERR_CUDA, "link cost: capture failed"); }
+    e = cudaGraphInstantiate(&ex, g, 0);
+    cudaGraphDestroy(g);
+    if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("link cost: ") + cudaGetErrorString(e));
+    cudaEvent_t a, b;
+    cudaEventCreate(&a); cudaEventCreate(&b);
+    float best = 1e30f;
+    for (int rep = 0; rep < 12; ++rep) {
+        cudaEventRecord(a, st);
+        cudaGraphLaunch(ex, st);
+        cudaEventRecord(b, st);
+        cudaStreamSynchronize(st);
+        float ms = 0.f;
+        if (rep >= 2 && cudaEventElapsedTime(&ms, a, b) == cudaSuccess && ms < best) best = ms;
+    }
+    cudaEventDestroy(a); cudaEventDestroy(b);
+    cudaGraphExecDestroy(ex);
+    h->launches += 12LL * n_links;
+    *h_us_per_link = (double)best * 1e3 / n_links;
     return SPECDEC_OK;
 }
 

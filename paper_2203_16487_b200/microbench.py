@@ -89,6 +89,29 @@ def measure(sd, wl, B, k, j, S, reps, warmup, flush, draft=False):
     return float(np.median(times)), float(np.min(times)), mean_a
 
 
+def measure_ttft(sd, wl, k, reps, warmup, flush):
+    """Time to the first committed tokens: specdec_encode (both encoders, cross K/V of every decoder layer), then one
+    draft -> verify -> commit iteration.  Returns median microseconds of (encode, encode + first iteration)."""
+    src, lens = W.pad_batch(wl.src)
+    d_src = torch.from_numpy(src).cuda(); d_len = torch.from_numpy(lens).cuda()
+    enc, tot = [], []
+    for r in range(warmup + reps):
+        if flush is not None:
+            flush.fill_(r & 0xff)
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        e0.record()
+        sd.encode(d_src, d_len, None)
+        e1.record()
+        d = sd.draft(k)
+        sd.verify(d, 3, 1.0)
+        sd.commit(None, None)
+        e2.record()
+        torch.cuda.synchronize()
+        if r >= warmup:
+            enc.append(e0.elapsed_time(e1) * 1e3); tot.append(e0.elapsed_time(e2) * 1e3)
+    return float(np.median(enc)), float(np.median(tot))
+
+
 def peaks():
     p = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -114,7 +137,25 @@ def main():
                     help="Transformer-base pair (default) or the BART-base-shaped pair (GELU, learned positions)")
     ap.add_argument("--opt", action="append", default=[], help="library option name=value (repeatable; experiments)")
     ap.add_argument("--grid", action="store_true", help="the whole k x prefix x batch grid of the verify microbench")
+    ap.add_argument("--ttft", action="store_true", help="time to the first tokens on summarisation-shaped inputs (batch 8, "
+                    "sources of 300-512 ids) or, with --translation, on one translation-shaped sentence")
+    ap.add_argument("--translation", action="store_true")
     args = ap.parse_args()
+    if args.ttft:
+        wl = W.config2_translation(1) if args.translation else W.config4_summarization()
+        wv = W.make_weights(wl.verifier, wl.seed_verifier, True)
+        wd = W.make_weights(wl.drafter, wl.seed_drafter, True)
+        sd = binding.SpecDec(wl.verifier, wv, wl.drafter, wd, k_max=25, max_batch=len(wl.src), max_src=max(len(s) for s in wl.src),
+                             max_tgt=max(wl.max_tgt), bf16=True)
+        for o in args.opt:
+            sd.set_option(o.split("=")[0], int(o.split("=")[1]))
+        flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+        enc, tot = measure_ttft(sd, wl, 25, args.reps, args.warmup, flush)
+        print(json.dumps({"step": "ttft", "workload": wl.name, "batch": len(wl.src), "source_lens": [len(s) for s in wl.src],
+                          "us_encode_median": enc, "us_to_first_tokens_median": tot, "l2_flush": flush is not None,
+                          "link_cost_us": {g: sd.link_cost(64, g) for g in (8, 148, 592)}}))
+        sd.close()
+        return
     S = args.src_len
     hbm, tc, kind = peaks()
     flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
