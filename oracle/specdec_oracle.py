@@ -36,7 +36,9 @@ paper's memory table; a closed-form model with zeroed sublayers; the whole
 encoder / decoder stack against torch.nn's pre-LN Transformer layers in fp64
 (ReLU and GELU); every weight shown to influence the output; the points at
 which mode="bf16" rounds (a recorder in place of bf16_round); decision_margins
-on hand-worked rows.
+on hand-worked rows; the prefix-causal drafter reading against torch.nn layers
+given the same mask, against the plain causal decoder on its prefix rows, cached
+against from scratch.
 Parity unpinned: nothing about translation quality (needs trained weights).
 """
 from __future__ import annotations
@@ -186,24 +188,35 @@ def new_cache(m: Model, mem: np.ndarray) -> DecoderCache:
 
 
 def decoder_rows(m: Model, tokens: Sequence[int], mem: np.ndarray, causal: bool,
-                 cache: Optional[DecoderCache] = None) -> np.ndarray:
+                 cache: Optional[DecoderCache] = None, n_causal: Optional[int] = None) -> np.ndarray:
     """Decoder stack -> logits [len(tokens), V] = LN_f(h) E^T (tied, no bias).
 
     Without a cache the tokens occupy positions 0..T-1 and everything is
-    computed from scratch (the plain definition).  With a cache (causal only)
-    the tokens occupy positions cache.length.. and attend to the cached
-    positions too; the cache is extended in place with the new rows.
+    computed from scratch (the plain definition).  With a cache the tokens
+    occupy positions cache.length.. and attend to the cached positions too; the
+    cache is extended in place with the new rows.
+
+    Self-attention mask: causal (position p sees 0..p), none (causal=False), or
+    -- n_causal given -- "prefix-causal": positions below n_causal are causal,
+    the positions from n_causal on see every position of the pass (the drafter's
+    second reading: committed tokens never look at the [MASK] block, so their
+    rows can be cached like an autoregressive decoder's).  Cached passes need a
+    mask under which cached rows never depend on later ones: causal or
+    prefix-causal with the cache inside the causal part.
     """
     T = len(tokens)
     start = 0 if cache is None else cache.length
     if cache is None:
         cache = new_cache(m, mem)
     else:
-        assert causal, "a non-causal pass cannot reuse cached rows"
+        assert causal or (n_causal is not None and start <= n_causal), "a non-causal pass cannot reuse cached rows"
     x = embed(m, tokens, range(start, start + T), "pos_dec")
     qpos = np.arange(start, start + T)[:, None]
     kpos = np.arange(0, start + T)[None, :]
-    allowed = (kpos <= qpos) if causal else np.ones((T, start + T), dtype=bool)
+    if n_causal is not None:
+        allowed = (kpos <= qpos) | (qpos >= n_causal)
+    else:
+        allowed = (kpos <= qpos) if causal else np.ones((T, start + T), dtype=bool)
     cross_ok = np.ones((T, mem.shape[0]), dtype=bool)
     for l in range(m.dec_layers):
         p = f"dec.{l}"
@@ -247,15 +260,36 @@ def greedy_decode(m: Model, src: Sequence[int], max_tgt: int, bos: int, eos: int
 # Spec-Drafter inference (Section 3.1.3, inference equation)
 # ----------------------------------------------------------------------------
 def draft(md: Model, mem_d: np.ndarray, committed: Sequence[int], k: int,
-          bos: int, mask: int) -> List[int]:
-    """k drafted tokens: argmax at the k [MASK] rows of one non-causal decoder pass.
+          bos: int, mask: int, reading: str = "bidirectional",
+          cache: Optional[DecoderCache] = None) -> List[int]:
+    """k drafted tokens: argmax at the k [MASK] rows of one decoder pass.
 
     Input is [BOS, y_1..y_j, MASK x k] at positions 0..j+k; the row at a mask
     position predicts the token at that position (non-shifted).
+
+    reading = "bidirectional" (default): no self-attention mask at all, every row
+    sees every row ("mask-predict manner", Section 3.1).  reading =
+    "prefix_causal": the committed tokens attend causally among themselves and
+    the [MASK] rows see everything; the drafter decoder can then keep a K/V cache
+    of the committed positions across iterations (Section 3.1.2's latency
+    principle: the decoder is forwarded every iteration, so its work should not
+    grow with the prefix).  With `cache` (positions 0..c-1 of [BOS, y...], c <=
+    j+1) only the rows from c on are computed; the cache is left holding
+    positions 0..j.
     """
     j = len(committed)
-    logits = decoder_rows(md, [bos] + list(committed) + [mask] * k, mem_d, causal=False)
-    return [argmax_lowest(logits[j + 1 + i]) for i in range(k)]
+    tokens = [bos] + list(committed) + [mask] * k
+    if reading == "bidirectional":
+        assert cache is None
+        logits = decoder_rows(md, tokens, mem_d, causal=False)
+        return [argmax_lowest(logits[j + 1 + i]) for i in range(k)]
+    assert reading == "prefix_causal"
+    c = 0 if cache is None else cache.length
+    assert c <= j + 1
+    logits = decoder_rows(md, tokens[c:], mem_d, causal=False, cache=cache, n_causal=j + 1)
+    if cache is not None:
+        cache.truncate(j + 1)                   # the [MASK] rows are not part of the prefix
+    return [argmax_lowest(logits[j + 1 - c + i]) for i in range(k)]
 
 
 # ----------------------------------------------------------------------------
@@ -331,22 +365,24 @@ class GenStats:
 def specdec_generate(mv: Model, md: Model, src: Sequence[int], max_tgt: int, k: int,
                      beta: int, tau: float, bos: int, eos: int, mask: int,
                      use_cache: bool = True, draft_fn=None,
-                     keep_trace: bool = False, script: Optional[Sequence[int]] = None
-                     ) -> Tuple[List[int], GenStats]:
+                     keep_trace: bool = False, script: Optional[Sequence[int]] = None,
+                     drafter_reading: str = "bidirectional") -> Tuple[List[int], GenStats]:
     """Draft -> verify -> commit until EOS or max_tgt, one sequence.
 
     draft_fn(committed, k) may replace the drafter (scripted drafts in tests).
+    drafter_reading: see draft(); "prefix_causal" keeps a drafter K/V cache when use_cache is set.
     script (benchmark hook, no counterpart in the paper): after the drafter has run,
     the draft for target index t is replaced by script[t] wherever script[t] >= 0.
     """
     mem_v = encode(mv, src)
     mem_d = encode(md, src) if draft_fn is None else None
     cache = new_cache(mv, mem_v) if use_cache else None
+    dcache = new_cache(md, mem_d) if (use_cache and draft_fn is None and drafter_reading == "prefix_causal") else None
     out: List[int] = []
     st = GenStats()
     done = max_tgt <= 0
     while not done:
-        d = draft(md, mem_d, out, k, bos, mask) if draft_fn is None else list(draft_fn(list(out), k))
+        d = draft(md, mem_d, out, k, bos, mask, drafter_reading, dcache) if draft_fn is None else list(draft_fn(list(out), k))
         if script is not None:
             j = len(out)
             d = [int(script[j + i]) if j + i < len(script) and script[j + i] >= 0 else d[i] for i in range(k)]

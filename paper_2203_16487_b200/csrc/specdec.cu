@@ -1690,7 +1690,7 @@ int specdec_debug_trace(specdec_handle* h, long long* h_out, int n) {
 int specdec_debug_link_cost(specdec_handle* h, int n_links, int grid, double* h_us_per_link) {
     if (!h || !h_us_per_link || n_links < 1 || n_links > 4096 || grid < 1 || grid > 65535) return SPECDEC_ERR_INVALID_ARG;
     cudaStream_t st = h->own_stream;
-    int* word = h->ses.counters + 6;                 // (a counter no kernel of the path reads)
+    int* word = reinterpret_cast<int*>(h->trace_buf + 255);     // (the last slot of the time-stamp array: no kernel of the path touches it)
     cudaGraph_t g = nullptr; cudaGraphExec_t ex = nullptr;
     CUDA_TRY(h, cudaStreamSynchronize(st));
     CUDA_TRY(h, cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));

@@ -499,3 +499,63 @@ def test_bf16_mode_rounds_exactly_the_contraction_operands(monkeypatch):
     memp = O.encode(mp, src)
     assert np.array_equal(O.encode(m, src), memp)
     assert np.array_equal(O.decoder_rows(m, [1, 4, 5], memp, True), O.decoder_rows(mp, [1, 4, 5], memp, True))
+
+
+# ---------------------------------------------------------------- the drafter's prefix-causal reading
+def test_prefix_causal_mask_equals_torch_layers_and_causal_prefix(tiny):
+    """decoder_rows(..., n_causal = p): positions below p attend causally, positions from p on see everything.
+    (1) fp64 equality with torch.nn decoder layers given that boolean mask; (2) the rows below p equal the plain
+    causal decoder on the prefix alone (they never see the [MASK] block, whatever follows them); (3) a one-layer
+    decoder gives the same [MASK] rows under both readings (first-layer keys and values are functions of token and
+    position only)."""
+    wl, mv, md = tiny
+    m = O.model_from(wl.drafter, md.w, dtype=np.float64)
+    _, dec = _torch_stack(m)
+    t = lambda a: torch.tensor(np.asarray(a, dtype=np.float64))
+    src = wl.src[2]
+    prefix, k = [BOS, 17, 230, 5, 999], 6
+    tokens = prefix + [MASK] * k
+    T, p = len(tokens), len(prefix)
+    mem = O.encode(m, src)
+    blocked = torch.zeros((T, T), dtype=torch.bool)
+    for q in range(p):
+        blocked[q, q + 1:] = True                       # True = not allowed, torch's convention
+    with torch.no_grad():
+        y = (t(m.w["embed"])[torch.tensor(tokens)] * math.sqrt(m.d_model) + t(m.w["pos_dec"])[:T])[None]
+        for L in dec:
+            y = L(y, t(mem)[None], tgt_mask=blocked)
+        y = torch.nn.functional.layer_norm(y, (m.d_model,), t(m.w["dec.ln_f.g"]), t(m.w["dec.ln_f.b"]), 1e-5)
+        ref = (y[0] @ t(m.w["embed"]).T).numpy()
+    got = O.decoder_rows(m, tokens, mem, causal=False, n_causal=p)
+    np.testing.assert_allclose(got, ref, rtol=0, atol=1e-10)
+    np.testing.assert_allclose(got[:p], O.decoder_rows(m, prefix, mem, causal=True), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(got[:p], O.decoder_rows(m, prefix + [MASK] * 2, mem, causal=False, n_causal=p)[:p], rtol=0, atol=1e-12)
+    full = O.decoder_rows(m, tokens, mem, causal=False)
+    assert np.abs(full[p:] - got[p:]).max() > 1e-6 or m.dec_layers == 1     # the readings differ beyond one layer ...
+    one = O.model_from(W.ModelDims(m.d_model, m.n_heads, m.d_ffn, m.vocab, m.enc_layers, 1, 64), m.w, dtype=np.float64)
+    a = O.decoder_rows(one, tokens, mem, causal=False)
+    b = O.decoder_rows(one, tokens, mem, causal=False, n_causal=p)
+    np.testing.assert_allclose(a[p:], b[p:], rtol=0, atol=1e-12)            # ... and coincide on the [MASK] rows of one layer
+    assert np.abs(a[:p] - b[:p]).max() > 1e-6
+
+
+def test_prefix_causal_drafter_cache_equals_from_scratch(tiny):
+    """draft(reading="prefix_causal") with a K/V cache carried across iterations gives the drafts of the uncached
+    pass, for prefixes that grow by 1..k+1 tokens per iteration; the whole loop gives the same output either way, and
+    at beta = 1, tau = 0 it is still greedy decoding (the drafter's reading cannot change a lossless rule's output)."""
+    wl, mv, md = tiny
+    src = wl.src[1]
+    mem_d = O.encode(md, src)
+    cache = O.new_cache(md, mem_d)
+    committed = []
+    rng = np.random.default_rng(5)
+    for step in range(5):
+        d_cached = O.draft(md, mem_d, committed, wl.k, BOS, MASK, "prefix_causal", cache)
+        d_plain = O.draft(md, mem_d, committed, wl.k, BOS, MASK, "prefix_causal")
+        assert d_cached == d_plain and cache.length == len(committed) + 1
+        committed = committed + [int(t) for t in rng.integers(4, 1000, size=int(rng.integers(1, wl.k + 2)))]
+    a, sa = O.specdec_generate(mv, md, src, 32, wl.k, 3, 1.0, BOS, EOS, MASK, drafter_reading="prefix_causal")
+    b, sb = O.specdec_generate(mv, md, src, 32, wl.k, 3, 1.0, BOS, EOS, MASK, drafter_reading="prefix_causal", use_cache=False)
+    assert a == b and sa.accepted == sb.accepted and sa.iterations == sb.iterations
+    g, _ = O.specdec_generate(mv, md, src, 32, wl.k, 1, 0.0, BOS, EOS, MASK, drafter_reading="prefix_causal")
+    assert g == O.greedy_decode(mv, src, 32, BOS, EOS)
