@@ -219,6 +219,14 @@ int specdec_set_draft_script(specdec_handle* h, const int32_t* d_script, int B, 
 int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches);
 
 /* Options (experiments and on-device cross-checks; every combination computes the same result):
+ * "drafter_prefix_causal" 0 (default) / 1: the second reading of the Spec-Drafter's decoder mask.  0: no self-attention
+ *                mask at all (every row of [BOS, committed, MASK x k] sees every row: "mask-predict manner", Section 3.1);
+ *                the whole input is recomputed every iteration.  1: the committed tokens attend causally among
+ *                themselves and only the [MASK] rows see everything; the drafter's decoder then keeps a K/V cache of the
+ *                committed positions and a draft pass computes only the newly committed tokens and the k [MASK] rows
+ *                (Section 3.1.2: the decoder runs every iteration, so its cost should not grow with the prefix).  A
+ *                different function of the same weights: drafts differ, the verified output under beta = 1, tau = 0
+ *                does not.  Takes effect at the next specdec_encode.
  * "gemm"         0 SIMT reference GEMM / 1 tcgen05 tensor-core GEMM (bf16 handles; default 1)
  * "attn"         0 warp-per-row reference attention / 1 tensor-core tile attention (bf16, 64-wide heads; default 1)
  * "skinny"       0/1 weight-streaming GEMM with fused LayerNorm for passes of at most 32 rows (default 1)

@@ -79,6 +79,8 @@ struct Session {
     int* counters;     // [8]: 0 rows of the drafter's full pass, 1 rows of its mask-only pass,
                        //      2 verify rows, 3 encoder rows, 4 unfinished sequences
     unsigned long long* stats;  // [4]: seq_iterations, drafted, accepted, emitted
+    int* dlen;         // [B] prefix-causal drafter: positions of [BOS, committed...] whose K/V its cache already holds
+    int* dticket;      // [1] block ticket of the drafter's row preparation
 };
 enum { CNT_DRAFT_ALL = 0, CNT_DRAFT_MASK = 1, CNT_VERIFY = 2, CNT_ENC = 3, CNT_ACTIVE = 4, CNT_TICKET = 5, CNT_SEQ = 6 };
 
@@ -179,6 +181,74 @@ __global__ void k_draft_prep(Session s, int B, int k, int S_max, int bos, int ma
         msk.nk_cross[row] = sl;
         msk.src_row[row] = off + j + 1 + i;
         msk.slot[row] = b * k + i;
+    }
+}
+
+// Drafter, prefix-causal reading (the committed tokens attend causally among themselves and never see the [MASK]
+// block, so their keys and values are cached like an autoregressive decoder's; Section 3.1.2: the drafter's decoder runs
+// every iteration, so its work should not grow with the prefix).  Rows of sequence b: the positions the cache does not
+// hold yet, c..j of [BOS, committed...], then k [MASK] rows at positions j+1..j+k.  Position p sees keys 0..p when it is
+// a prefix row and every key 0..j+k when it is a [MASK] row.  The last block to finish records the new cache length.
+__global__ void k_draft_prep_pc(Session s, int B, int k, int S_max, int bos, int mask, Rows all, Rows msk) {
+    __shared__ int red_a[32], red_m[32], tot_a[32], tot_l[32];
+    __shared__ int last_s;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
+    int a = 0, m = 0, ta = 0, tl = 0;
+    for (int o = tid; o < B; o += blockDim.x) {
+        const int n = s.finished[o] ? 0 : (s.len[o] + 1 - min(s.dlen[o], s.len[o] + 1)) + k;
+        ta += n; tl += n ? 1 : 0;
+        if (o < b) { a += n; m += n ? k : 0; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        a += __shfl_xor_sync(0xffffffffu, a, o); m += __shfl_xor_sync(0xffffffffu, m, o);
+        ta += __shfl_xor_sync(0xffffffffu, ta, o); tl += __shfl_xor_sync(0xffffffffu, tl, o);
+    }
+    if (lane == 0) { red_a[warp] = a; red_m[warp] = m; tot_a[warp] = ta; tot_l[warp] = tl; }
+    __syncthreads();
+    int off = 0, moff = 0, total = 0, live = 0;
+    for (int w = 0; w < nw; ++w) { off += red_a[w]; moff += red_m[w]; total += tot_a[w]; live += tot_l[w]; }
+    const bool fin = s.finished[b] != 0;
+    const int j = s.len[b], c = min(s.dlen[b], j + 1), n_new = j + 1 - c, n = fin ? 0 : n_new + k, sl = s.src_len[b];
+    if (tid == 0) {
+        all.kv_off[b] = off; all.kv_off_cross[b] = b * S_max;
+        msk.kv_off[b] = off; msk.kv_off_cross[b] = b * S_max;
+        all.q_off[b] = off; all.q_cnt[b] = n;
+        msk.q_off[b] = moff; msk.q_cnt[b] = fin ? 0 : k;
+        if (b == 0) {
+            s.counters[CNT_DRAFT_ALL] = total;
+            s.counters[CNT_DRAFT_MASK] = live * k;
+        }
+    }
+    if (!fin) {
+        for (int t = tid; t < n; t += blockDim.x) {
+            const int row = off + t, p = c + t;
+            all.tok[row] = (t >= n_new) ? mask : (p == 0 ? bos : s.out[(size_t)b * s.out_stride + p - 1]);
+            all.pos[row] = p;
+            all.seq[row] = b;
+            all.nk_self[row] = (t >= n_new) ? j + 1 + k : p + 1;
+            all.nk_cross[row] = sl;
+        }
+        for (int i = tid; i < k; i += blockDim.x) {
+            const int row = moff + i;
+            msk.seq[row] = b;
+            msk.nk_self[row] = j + 1 + k;
+            msk.nk_cross[row] = sl;
+            msk.src_row[row] = off + n_new + i;
+            msk.slot[row] = b * k + i;
+        }
+    }
+    // every block has read the old cache lengths before any is overwritten
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        last_s = (atomicAdd(s.dticket, 1) == (int)gridDim.x - 1) ? 1 : 0;
+    }
+    __syncthreads();
+    if (last_s) {
+        for (int o = tid; o < B; o += blockDim.x)
+            if (!s.finished[o]) s.dlen[o] = s.len[o] + 1;
+        if (tid == 0) *s.dticket = 0;
     }
 }
 
@@ -781,6 +851,8 @@ __global__ void k_session_init(Session s, const int* __restrict__ src_len, const
     if (b >= B) return;
     int mt = max_tgt ? min(max(max_tgt[b], 0), max_tgt_cap) : max_tgt_cap;
     s.len[b] = 0;
+    s.dlen[b] = 0;
+    if (b == 0) *s.dticket = 0;
     s.max_tgt[b] = mt;
     s.finished[b] = (mt <= 0) ? 1 : 0;
     s.src_len[b] = min(max(src_len[b], 1), S_max);

@@ -76,6 +76,11 @@ struct specdec_handle {
     cudaEvent_t enc_fork = nullptr, enc_join = nullptr;
     // verifier KV cache
     std::vector<void*> kc, vc;
+    // drafter KV cache of its decoder layers (prefix-causal reading only; same page geometry as the verifier's)
+    std::vector<void*> dkc, dvc;
+    int drafter_pc = 0;             // option "drafter_prefix_causal", as set
+    int drafter_pc_session = 0;     // ... as in force for the running session (latched by specdec_encode)
+    int dnew_ub = 1;                // upper bound on the prefix positions the next draft pass has to add to that cache
     int* page_table;
     // rows
     Rows rows, mrows;
@@ -273,6 +278,10 @@ void layout_all(specdec_handle* h) {
     h->vc.resize(h->cfg.verifier.dec_layers);
     for (auto& p : h->kc) p = A.take(cache_rows * h->cfg.verifier.d_model * e);
     for (auto& p : h->vc) p = A.take(cache_rows * h->cfg.verifier.d_model * e);
+    h->dkc.resize(h->cfg.drafter.dec_layers);
+    h->dvc.resize(h->cfg.drafter.dec_layers);
+    for (auto& p : h->dkc) p = A.take(cache_rows * h->cfg.drafter.d_model * e);
+    for (auto& p : h->dvc) p = A.take(cache_rows * h->cfg.drafter.d_model * e);
     h->page_table = (int*)A.take((size_t)h->B_cap * h->pages_per_seq * 4);
     layout_rows(A, h->rows, h->R_cap, h->B_cap);
     layout_rows(A, h->mrows, h->R2_cap > 0 ? h->R2_cap : 1, h->B_cap);
@@ -297,6 +306,8 @@ void layout_all(specdec_handle* h) {
     s.src_len = (int*)A.take((size_t)h->B_cap * 4);
     s.out_stride = h->T_cap > 0 ? h->T_cap : 1;
     s.out = (int*)A.take((size_t)h->B_cap * s.out_stride * 4);
+    s.dlen = (int*)A.take((size_t)h->B_cap * 4);
+    s.dticket = (int*)A.take(4);
     s.counters = (int*)A.take(8 * 4);
     s.stats = (unsigned long long*)A.take(4 * 8);
 }
@@ -688,16 +699,19 @@ void prof_collect(specdec_handle* h) {
 // One pre-LN block on `rows_ub` rows of the residual stream x (encoder: no cross-attention).
 // Self-attention keys come from the block's own QKV rows (contiguous) or, for the verifier,
 // from the paged cache after the block's K/V were scattered into it.
+// kc / vc: the paged cache the block's K / V go to and its attention reads (verifier; prefix-causal drafter), or null:
+// keys and values are the block's own rows.  pre_keys: per sequence, cache positions that predate the step.
 template <typename T>
 int block_self(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, const Rows& r, int cnt, int rows_ub,
-               int q_ub, int layer, bool verify, int max_keys, cudaStream_t st, const float* next_g = nullptr,
+               int q_ub, void* kc, void* vc, const int* pre_keys, int max_keys, cudaStream_t st, const float* next_g = nullptr,
                const float* next_b = nullptr) {
     const int d = m.dm.d_model, H = m.dm.n_heads, dh = d / H;
     const size_t e = h->esz;
+    const bool verify = kc != nullptr;
     const LnSpec l1{x, w.ln1_g, w.ln1_b};
     if (verify && tc_usable<T>(h, 3 * d, d) && d % 32 == 0) {
         // K and V columns leave the GEMM epilogue straight into the paged cache
-        KvDest kv{r.seq, r.pos, h->kc[layer], h->vc[layer], d};
+        KvDest kv{r.seq, r.pos, kc, vc, d};
         TRY(gemm<T>(h, EPI_QKV, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, cnt, rows_ub, h->qkv, 3 * d, nullptr, st, nullptr,
                     nullptr, nullptr, &kv, &l1));
     } else {
@@ -706,13 +720,13 @@ int block_self(specdec_handle* h, const ModelW& m, const LayerW& w, float* x, co
         if (verify) {
             Paged pg{h->page_table, h->cfg.page_tokens, h->pages_per_seq};
             k_kv_scatter<T><<<rows_ub, 128, 0, st>>>((const T*)h->qkv, r.seq, r.pos, h->ses.counters + cnt, pg,
-                                                     (T*)h->kc[layer], (T*)h->vc[layer], d);
+                                                     (T*)kc, (T*)vc, d);
             KCHECK(h);
         }
     }
     if (verify) {
-        TRY(attn<T>(h, true, h->qkv, 3 * d, nullptr, h->kc[layer], h->vc[layer], d, nullptr, r, r.nk_self, cnt,
-                    rows_ub, q_ub, h->att, d, H, dh, max_keys, st, h->ses.len));      // cached prefix: positions < len
+        TRY(attn<T>(h, true, h->qkv, 3 * d, nullptr, kc, vc, d, nullptr, r, r.nk_self, cnt,
+                    rows_ub, q_ub, h->att, d, H, dh, max_keys, st, pre_keys));
     } else {
         TRY(attn<T>(h, false, h->qkv, 3 * d, nullptr, (char*)h->qkv + (size_t)d * e, (char*)h->qkv + (size_t)2 * d * e,
                     3 * d, r.kv_off, r, r.nk_self, cnt, rows_ub, q_ub, h->att, d, H, dh, max_keys, st));
@@ -773,7 +787,7 @@ int encode_model(specdec_handle* h, ModelW& m, cudaStream_t st) {
     TRY(embed<T>(h, m, h->rows, m.pos_enc, CNT_ENC, R, st));
     for (int l = 0; l < m.dm.enc_layers; ++l) {
         const bool last = l + 1 == m.dm.enc_layers;
-        TRY(block_self<T>(h, m, m.enc[l], h->x, h->rows, CNT_ENC, R, h->S_max, l, false, h->S_max, st, m.enc[l].ln2_g, m.enc[l].ln2_b));
+        TRY(block_self<T>(h, m, m.enc[l], h->x, h->rows, CNT_ENC, R, h->S_max, nullptr, nullptr, nullptr, h->S_max, st, m.enc[l].ln2_g, m.enc[l].ln2_b));
         TRY(block_ffn<T>(h, m, m.enc[l], h->x, CNT_ENC, R, st, last ? m.enc_lnf_g : m.enc[l + 1].ln1_g,
                          last ? m.enc_lnf_b : m.enc[l + 1].ln1_b, last ? h->mem : nullptr));
     }
@@ -788,6 +802,7 @@ template <typename T>
 int encode_impl(specdec_handle* h, const int* d_src, const int* d_src_len, const int* d_max_tgt, int B, int S_max,
                 cudaStream_t st) {
     h->B = B; h->S_max = S_max; h->len_ub = 0;
+    h->dnew_ub = 1; h->drafter_pc_session = h->drafter_pc;
     h->encoded = false; h->verified = false; h->drafted = false;
     k_session_init<<<cdiv(B, 128), 128, 0, st>>>(h->ses, d_src_len, d_max_tgt, B, h->T_cap, S_max);
     KCHECK(h);
@@ -827,25 +842,48 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
     const int B = h->B, d = m.dm.d_model, H = m.dm.n_heads, dh = d / H, L = m.dm.dec_layers;
     const size_t e = h->esz;
     const int len_ub = std::min(h->len_ub, h->T_cap);
-    const int R1 = B * (len_ub + 1 + k), R2 = B * k, max_keys = len_ub + 1 + k;
-    k_draft_prep<<<B, 128, 0, st>>>(h->ses, B, k, h->S_max, h->cfg.bos_id, h->cfg.mask_id, h->rows, h->mrows);
+    const bool pc = h->drafter_pc_session != 0;
+    // rows of the full pass per sequence: the whole [BOS, committed, MASK x k] input, or (prefix-causal reading) only the
+    // prefix positions its K/V cache does not hold yet plus the k [MASK] rows
+    const int per_seq = pc ? std::min(h->dnew_ub, len_ub + 1) + k : len_ub + 1 + k;
+    const int R1 = B * per_seq, R2 = B * k, max_keys = len_ub + 1 + k;
+    if (pc) k_draft_prep_pc<<<B, 128, 0, st>>>(h->ses, B, k, h->S_max, h->cfg.bos_id, h->cfg.mask_id, h->rows, h->mrows);
+    else k_draft_prep<<<B, 128, 0, st>>>(h->ses, B, k, h->S_max, h->cfg.bos_id, h->cfg.mask_id, h->rows, h->mrows);
     KCHECK(h);
     TRY(embed<T>(h, m, h->rows, m.pos_dec, CNT_DRAFT_ALL, R1, st));
     for (int l = 0; l + 1 < L; ++l) {
-        TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_DRAFT_ALL, R1, max_keys, l, false, max_keys, st, m.dec[l].lnc_g, m.dec[l].lnc_b));
-        TRY(block_cross<T>(h, m, m.dec[l], h->x, h->rows, CNT_DRAFT_ALL, R1, max_keys, l, st));
+        TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_DRAFT_ALL, R1, per_seq, pc ? h->dkc[l] : nullptr, pc ? h->dvc[l] : nullptr, nullptr,
+                          max_keys, st, m.dec[l].lnc_g, m.dec[l].lnc_b));
+        TRY(block_cross<T>(h, m, m.dec[l], h->x, h->rows, CNT_DRAFT_ALL, R1, per_seq, l, st));
         TRY(block_ffn<T>(h, m, m.dec[l], h->x, CNT_DRAFT_ALL, R1, st, m.dec[l + 1].ln1_g, m.dec[l + 1].ln1_b));
     }
     // last layer: K/V from every row, queries and everything after them from the k mask rows only
     const LayerW& w = m.dec[L - 1];
     const LnSpec l1{h->x, w.ln1_g, w.ln1_b};
-    TRY(gemm<T>(h, EPI_STORE, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, CNT_DRAFT_ALL, R1, h->qkv, 3 * d, nullptr, st, nullptr,
-                nullptr, nullptr, nullptr, &l1));
+    const bool scatter_in_gemm = pc && tc_usable<T>(h, 3 * d, d) && d % 32 == 0;
+    if (scatter_in_gemm) {
+        KvDest kv{h->rows.seq, h->rows.pos, h->dkc[L - 1], h->dvc[L - 1], d};
+        TRY(gemm<T>(h, EPI_QKV, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, CNT_DRAFT_ALL, R1, h->qkv, 3 * d, nullptr, st, nullptr,
+                    nullptr, nullptr, &kv, &l1));
+    } else {
+        TRY(gemm<T>(h, EPI_STORE, h->y, d, w.qkv_w, w.qkv_b, 3 * d, d, CNT_DRAFT_ALL, R1, h->qkv, 3 * d, nullptr, st, nullptr,
+                    nullptr, nullptr, nullptr, &l1));
+        if (pc) {
+            Paged pg{h->page_table, h->cfg.page_tokens, h->pages_per_seq};
+            k_kv_scatter<T><<<R1, 128, 0, st>>>((const T*)h->qkv, h->rows.seq, h->rows.pos, h->ses.counters + CNT_DRAFT_ALL, pg,
+                                                (T*)h->dkc[L - 1], (T*)h->dvc[L - 1], d);
+            KCHECK(h);
+        }
+    }
     CUDA_TRY(h, launch_pdl(h, k_gather_rows, dim3(R2), dim3(128), 0, st, (const float*)h->x, (const int*)h->mrows.src_row, (const int*)(h->ses.counters + CNT_DRAFT_MASK), h->x2, d));
     KCHECK(h);
-    TRY(attn<T>(h, false, h->qkv, 3 * d, h->mrows.src_row, (char*)h->qkv + (size_t)d * e,
-                (char*)h->qkv + (size_t)2 * d * e, 3 * d, h->mrows.kv_off, h->mrows, h->mrows.nk_self,
-                CNT_DRAFT_MASK, R2, k, h->att, d, H, dh, max_keys, st));
+    if (pc)
+        TRY(attn<T>(h, true, h->qkv, 3 * d, h->mrows.src_row, h->dkc[L - 1], h->dvc[L - 1], d, nullptr, h->mrows, h->mrows.nk_self,
+                    CNT_DRAFT_MASK, R2, k, h->att, d, H, dh, max_keys, st));
+    else
+        TRY(attn<T>(h, false, h->qkv, 3 * d, h->mrows.src_row, (char*)h->qkv + (size_t)d * e,
+                    (char*)h->qkv + (size_t)2 * d * e, 3 * d, h->mrows.kv_off, h->mrows, h->mrows.nk_self,
+                    CNT_DRAFT_MASK, R2, k, h->att, d, H, dh, max_keys, st));
     TRY(gemm<T>(h, EPI_RESID, h->att, d, w.o_w, w.o_b, d, d, CNT_DRAFT_MASK, R2, nullptr, 0, h->x2, st));
     TRY(block_cross<T>(h, m, w, h->x2, h->mrows, CNT_DRAFT_MASK, R2, k, L - 1, st));
     TRY(block_ffn<T>(h, m, w, h->x2, CNT_DRAFT_MASK, R2, st, m.dec_lnf_g, m.dec_lnf_b));
@@ -862,6 +900,7 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
     }
     h->drafted = true; h->verified = false;
     h->last_draft_rows_ub = R2;
+    h->dnew_ub = 0;                                  // the cache now holds every committed position
     return 0;
 }
 
@@ -879,7 +918,8 @@ int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float ta
     TRY(embed<T>(h, m, h->rows, m.pos_dec, CNT_VERIFY, M, st));
     for (int l = 0; l < L; ++l) {
         const bool last = l + 1 == L;
-        TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, k + 1, l, true, max_keys, st, m.dec[l].lnc_g, m.dec[l].lnc_b));
+        TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, k + 1, h->kc[l], h->vc[l], h->ses.len /* cached prefix: positions < len */,
+                          max_keys, st, m.dec[l].lnc_g, m.dec[l].lnc_b));
         TRY(block_cross<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, k + 1, l, st));
         TRY(block_ffn<T>(h, m, m.dec[l], h->x, CNT_VERIFY, M, st, last ? m.dec_lnf_g : m.dec[l + 1].ln1_g,
                          last ? m.dec_lnf_b : m.dec[l + 1].ln1_b));
@@ -908,6 +948,7 @@ int commit_impl(specdec_handle* h, const int* d_keep, const int* d_next, cudaStr
                            (const int*)(d_keep ? d_keep : h->accepted), (const int*)(d_next ? d_next : h->bif), h->B, k, h->cfg.eos_id, h->h_post));
     KCHECK(h);
     h->len_ub = std::min(h->len_ub + k + 1, h->T_cap);
+    h->dnew_ub = std::min(h->dnew_ub + k + 1, h->T_cap + 1);
     h->verified = false;
     return 0;
 }
@@ -943,7 +984,7 @@ inline void graph_key_tail(const specdec_handle* h, std::vector<long long>& key)
                         (long long)h->use_pdl, (long long)h->use_ln_fuse, (long long)h->use_sk_cluster,
                         (long long)h->use_pair, (long long)h->diag_repeat, (long long)h->use_splitk, (long long)h->attn_stream, (long long)h->attn_stream_keys, (long long)h->attn_warps, (long long)h->attn_rs,
                         (long long)h->skinny_groups, (long long)h->want_trace,
-                        (long long)(h->script_on ? 1 : 0), (long long)h->B, (long long)h->S_max})
+                        (long long)(h->script_on ? 1 : 0), (long long)h->B, (long long)h->S_max, (long long)h->drafter_pc_session})
         key.push_back(v);
 }
 
@@ -1034,9 +1075,11 @@ int encode_staged(specdec_handle* h, const int* d_src, const int* d_src_len, con
     if (d_src_len != h->stage_len) CUDA_TRY(h, cudaMemcpyAsync(h->stage_len, d_src_len, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
     if (d_max_tgt && d_max_tgt != h->stage_mt) CUDA_TRY(h, cudaMemcpyAsync(h->stage_mt, d_max_tgt, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
     h->B = B; h->S_max = S_max;
+    h->drafter_pc_session = h->drafter_pc;
     TRY(graph_call(h, {5, d_max_tgt ? 1 : 0}, st, [&]() {
         return encode_impl<T>(h, h->stage_src, h->stage_len, d_max_tgt ? h->stage_mt : nullptr, B, S_max, st); }));
     h->len_ub = 0; h->encoded = true; h->verified = false; h->drafted = false;
+    h->dnew_ub = 1;
     return 0;
 }
 
@@ -1075,11 +1118,13 @@ int generate_loop(specdec_handle* h, const int* d_src, const int* d_src_len, con
         if (graphs) {
             // the launches depend on the host-side length bound only through its 32-token bucket
             const int true_ub = h->len_ub, lb = len_bucket(h, true_ub);
+            // (prefix-causal drafter: the pass is also sized by how many prefix positions its cache still lacks)
+            const int dn = h->dnew_ub, dkey = (h->drafter_pc_session && k > 0) ? dn : -1;
             bool done = false;
             if (gated) {
                 h->len_ub = lb;
                 long long nk = 0;
-                int rc = graph_call_gated(h, {3, k, lb, beta, tau_bits}, st, [&]() {
+                int rc = graph_call_gated(h, {3, k, lb, beta, tau_bits, dkey}, st, [&]() {
                     int r = k > 0 ? draft_impl<T>(h, k, h->v_draft, st) : 0;
                     h->len_ub = lb;
                     if (!r) r = verify_impl<T>(h, h->v_draft, k, beta, tau, nullptr, nullptr, st);
@@ -1092,7 +1137,8 @@ int generate_loop(specdec_handle* h, const int* d_src, const int* d_src_len, con
             if (!done && !phases) {
                 // one graph per iteration: no graph-to-graph gap between the drafter and the verifier
                 h->len_ub = lb;
-                TRY(graph_call(h, {4, k, lb, beta, tau_bits}, st, [&]() {
+                h->dnew_ub = dn;
+                TRY(graph_call(h, {4, k, lb, beta, tau_bits, dkey}, st, [&]() {
                     int r = k > 0 ? draft_impl<T>(h, k, h->v_draft, st) : 0;
                     h->len_ub = lb;
                     if (!r) r = verify_impl<T>(h, h->v_draft, k, beta, tau, nullptr, nullptr, st);
@@ -1103,7 +1149,8 @@ int generate_loop(specdec_handle* h, const int* d_src, const int* d_src_len, con
             }
             if (!done) {
                 h->len_ub = lb;
-                if (k > 0) TRY(graph_call(h, {1, k, lb}, st, [&]() { return draft_impl<T>(h, k, h->v_draft, st); }));
+                h->dnew_ub = dn;
+                if (k > 0) TRY(graph_call(h, {1, k, lb, dkey}, st, [&]() { return draft_impl<T>(h, k, h->v_draft, st); }));
                 mark();
                 h->len_ub = lb;
                 TRY(graph_call(h, {2, k, lb, beta, tau_bits}, st, [&]() {
@@ -1114,6 +1161,7 @@ int generate_loop(specdec_handle* h, const int* d_src, const int* d_src_len, con
                 it_kernels.push_back(0);
             }
             h->len_ub = std::min(true_ub + k + 1, h->T_cap);
+            h->dnew_ub = std::min((k > 0 ? 0 : dn) + k + 1, h->T_cap + 1);      // (a replayed graph does not run the host code that counts)
             h->last_k = k; h->verified = false; h->drafted = false;
         } else {
             if (k > 0) TRY(draft_impl<T>(h, k, h->v_draft, st));
@@ -1424,6 +1472,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
         h->h_poll[ERRW_SLOT] = value; h->errw_pending = false;
         return SPECDEC_OK;
     }
+    if (!strcmp(name, "drafter_prefix_causal")) { h->drafter_pc = value ? 1 : 0; return SPECDEC_OK; }   // latched by the next specdec_encode
     if (!strcmp(name, "poll_lag")) { h->poll_lag = value; return SPECDEC_OK; }
     if (!strcmp(name, "stats_timing")) { h->stats_timing = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "poll_flag")) { h->poll_flag = value ? 1 : 0; return SPECDEC_OK; }
@@ -1478,9 +1527,11 @@ int specdec_draft(specdec_handle* h, int k, int32_t* d_draft, void* stream) {
     if (h->use_graphs && !h->profile) {
         const int true_ub = h->len_ub, lb = len_bucket(h, true_ub);
         h->len_ub = lb;
-        int rc = graph_call(h, {3, k, lb, (long long)(intptr_t)d_draft}, st, [&]() {
+        const int dn = h->dnew_ub;
+        int rc = graph_call(h, {3, k, lb, (long long)(intptr_t)d_draft, h->drafter_pc_session ? dn : -1}, st, [&]() {
             return DISPATCH(h, draft_impl<bf16>(h, k, d_draft, st), draft_impl<float>(h, k, d_draft, st)); });
         h->len_ub = true_ub;
+        h->dnew_ub = 0;
         h->drafted = true; h->verified = false; h->last_draft_rows_ub = h->B * k;
         return rc;
     }

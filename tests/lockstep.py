@@ -42,10 +42,12 @@ class Report:
 
 def run(sd, mv: O.Model, md: O.Model, srcs, max_tgt, k, beta, tau, margin: float,
         eos: int = W.EOS_ID, max_iters: Optional[int] = None, check_logits_every: int = 0,
-        logit_tol: float = 1e-4, draft_fn=None, pad_to: Optional[int] = None) -> Report:
+        logit_tol: float = 1e-4, draft_fn=None, pad_to: Optional[int] = None,
+        drafter_reading: str = "bidirectional") -> Report:
     rep = Report()
     B = len(srcs)
     sd.set_option("row_lse", 1)
+    sd.set_option("drafter_prefix_causal", 1 if drafter_reading == "prefix_causal" else 0)
     src, lens = W.pad_batch(srcs, pad_to)
     sd.encode(src, lens, np.asarray(max_tgt, np.int32))
     mem_v = [O.encode(mv, s) for s in srcs]
@@ -65,7 +67,8 @@ def run(sd, mv: O.Model, md: O.Model, srcs, max_tgt, k, beta, tau, margin: float
                 o_draft[b] = draft_fn(b, list(out[b]), k)
                 continue
             j = len(out[b])
-            logits = O.decoder_rows(md, [W.BOS_ID] + out[b] + [W.MASK_ID] * k, mem_d[b], causal=False)[j + 1:]
+            logits = O.decoder_rows(md, [W.BOS_ID] + out[b] + [W.MASK_ID] * k, mem_d[b], causal=False,
+                                    n_causal=(j + 1 if drafter_reading == "prefix_causal" else None))[j + 1:]
             o_draft[b] = logits.argmax(axis=1)
             for i in range(k):
                 rep.draft_positions += 1

@@ -453,3 +453,107 @@ def test_generate_with_every_budget_zero(tiny, gate):
         ref, _ = O.specdec_generate(mv, md, srcs[i], mt, wl.k, 3, 1.0, BOS, EOS, MASK)
         assert out[i, :int(n[i])].cpu().tolist() == ref
     sd.close()
+
+
+# ---------------------------------------------------------------- the drafter's prefix-causal reading (cached drafter)
+def test_prefix_causal_drafter_tiny_and_designed_pair(tiny):
+    """Option "drafter_prefix_causal": fp32, every draft and decision in lock-step with the oracle's prefix-causal
+    drafter, then whole generations.  The designed pair accepts several drafts per iteration, so the drafter's cache
+    grows by more than one position at a time; the tiny pair grows it one by one."""
+    wl, wv, wd, mv, md = tiny
+    sd = _handle(wl.verifier, wv, wl.drafter, wd, False)
+    rep = lockstep.run(sd, mv, md, wl.src, wl.max_tgt, wl.k, 3, 1.0, margin=0.0, check_logits_every=3,
+                       drafter_reading="prefix_causal")
+    assert rep.ok and rep.draft_near_ties == 0 and rep.verify_near_ties == 0, rep.notes
+    src, lens = W.pad_batch(wl.src)
+    for graphs in (1, 0):
+        sd.set_option("graphs", graphs)
+        out, n, st = sd.generate(src, lens, wl.max_tgt, wl.k, 3, 1.0)
+        for b, s in enumerate(wl.src):
+            ref, _ = O.specdec_generate(mv, md, s, 32, wl.k, 3, 1.0, BOS, EOS, MASK, drafter_reading="prefix_causal")
+            assert out[b, :int(n[b])].cpu().tolist() == ref
+    sd.close()
+    dv, dwv, dd, dwd, T, D, dsrc = designed.case_study_pair()
+    mv2, md2 = O.model_from(dv, dwv), O.model_from(dd, dwd)
+    sd = _handle(dv, dwv, dd, dwd, False, k_max=10, max_batch=2, max_src=16, max_tgt=40)
+    sd.set_option("drafter_prefix_causal", 1)
+    ref, ost = O.specdec_generate(mv2, md2, dsrc, 40, 10, 3, 1.0, BOS, EOS, MASK, drafter_reading="prefix_causal")
+    for rep_i in range(2):
+        out, n, st = sd.generate(np.stack([dsrc, dsrc]), [len(dsrc)] * 2, [40, 7], 10, 3, 1.0)
+        assert out[0, :int(n[0])].cpu().tolist() == ref and out[1, :int(n[1])].cpu().tolist() == ref[:7]
+    assert ost.accepted >= 8                                  # several drafts accepted per iteration
+    sd.close()
+
+
+def test_prefix_causal_drafter_bf16_lockstep():
+    """The same reading on the bf16 tensor-core path: mid-sized models, five sequences of different lengths, the
+    oracle's decisions committed on both sides (prefixes grow by 1 .. k + 1 tokens per iteration)."""
+    wv, wd = W.make_weights(MID_V, 21, True), W.make_weights(MID_D, 22, True)
+    mv, md = O.model_from(MID_V, wv, mode="bf16"), O.model_from(MID_D, wd, mode="bf16")
+    rng = np.random.default_rng(6)
+    srcs = [W.zipf_ids(rng, n, 2000) for n in (20, 7, 33, 12, 25)]
+    sd = _handle(MID_V, wv, MID_D, wd, True, k_max=12, max_batch=8, max_src=40, max_tgt=40)
+    # drafts that the verifier partly accepts: its own greedy continuation with a wrong token every few positions
+    greedy = [O.greedy_decode(mv, s, 40, BOS, EOS) for s in srcs]
+
+    def draft_fn(b, committed, k):
+        g = greedy[b][len(committed):len(committed) + k]
+        g = g + [7] * (k - len(g))
+        if len(g) > 4:
+            g[4] = 9
+        return g
+    rep = lockstep.run(sd, mv, md, srcs, [30, 18, 40, 5, 33], 12, 3, 1.0, margin=1e-3, check_logits_every=2, pad_to=40,
+                       drafter_reading="prefix_causal")
+    print(rep.iterations, rep.draft_near_ties, rep.verify_near_ties, rep.max_logit_err, rep.max_stat_err)
+    assert rep.ok, rep.notes
+    assert rep.max_logit_err < 2e-2 and rep.draft_near_ties <= 0.05 * rep.draft_positions
+    # with accepted drafts (the GPU drafter still runs and is compared; the committed prefix jumps by up to 5)
+    sd.set_option("drafter_prefix_causal", 1)
+    src, lens = W.pad_batch(srcs, 40)
+    sd.encode(src, lens, np.asarray([30, 18, 40, 5, 33], np.int32))
+    out = [[] for _ in srcs]
+    mem_d = [O.encode(md, s) for s in srcs]
+    for it in range(6):
+        g_draft = sd.draft(12).cpu().numpy()
+        keep, nxt = np.zeros(5, np.int32), np.zeros(5, np.int32)
+        for b in range(5):
+            j = len(out[b])
+            if j >= [30, 18, 40, 5, 33][b]:
+                continue
+            logits = O.decoder_rows(md, [BOS] + out[b] + [MASK] * 12, mem_d[b], causal=False, n_causal=j + 1)[j + 1:]
+            o_draft = logits.argmax(axis=1)
+            for i in range(12):
+                if g_draft[b, i] != o_draft[i]:
+                    assert float(logits[i, o_draft[i]] - logits[i, g_draft[b, i]]) < 1e-3, (it, b, i)
+            d = draft_fn(b, out[b], 12)
+            keep[b] = min(4, [30, 18, 40, 5, 33][b] - j - 1) if [30, 18, 40, 5, 33][b] - j - 1 > 0 else 0
+            nxt[b] = d[keep[b]] if keep[b] < len(d) else 7
+        blk = np.stack([draft_fn(b, out[b], 12) for b in range(5)]).astype(np.int32)
+        sd.verify(blk, 3, 1.0)
+        sd.commit(keep, nxt)
+        for b in range(5):
+            mt = [30, 18, 40, 5, 33][b]
+            if len(out[b]) < mt:
+                O.commit(out[b], blk[b].tolist(), int(keep[b]), int(nxt[b]), mt, EOS)
+    sd.close()
+
+
+def test_prefix_causal_drafter_base_shapes_generate():
+    """Transformer-base shapes, bf16, batch 4 with default options: whole generations with the cached drafter equal the
+    oracle's prefix-causal generations (the output of a random-init pair is the verifier's greedy continuation either
+    way, so the drafts themselves are compared in lock-step on one sentence first)."""
+    wl = W.config2_translation(4)
+    wv = W.make_weights(wl.verifier, wl.seed_verifier, True)
+    wd = W.make_weights(wl.drafter, wl.seed_drafter, True)
+    mv, md = O.model_from(wl.verifier, wv, mode="bf16"), O.model_from(wl.drafter, wd, mode="bf16")
+    sd = _handle(wl.verifier, wv, wl.drafter, wd, True, k_max=25, max_batch=4, max_src=40, max_tgt=64)
+    rep = lockstep.run(sd, mv, md, wl.src[:2], wl.max_tgt[:2], 25, 3, 1.0, margin=1e-3, check_logits_every=4, max_iters=6,
+                       drafter_reading="prefix_causal")
+    print(rep.iterations, rep.draft_positions, rep.draft_near_ties, rep.verify_near_ties, rep.max_logit_err, rep.notes[:3])
+    assert rep.ok, rep.notes
+    src, lens = W.pad_batch(wl.src, 40)
+    out, n, st = sd.generate(src, lens, wl.max_tgt, 25, 3, 1.0)
+    for b in (0, 3):
+        ref, _ = O.specdec_generate(mv, md, wl.src[b], wl.max_tgt[b], 25, 3, 1.0, BOS, EOS, MASK, drafter_reading="prefix_causal")
+        assert out[b, :int(n[b])].cpu().tolist() == ref
+    sd.close()
