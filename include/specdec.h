@@ -207,6 +207,13 @@ int specdec_debug_trace(specdec_handle* h, long long* h_out, int n);
  * replays divided by n_links, in microseconds.  Synchronises. */
 int specdec_debug_link_cost(specdec_handle* h, int n_links, int grid, double* h_us_per_link);
 
+/* Diagnostics: clocks per tcgen05.mma (M = 128 x N = bn x K = 16, bf16) when the operands already sit in shared memory:
+ * one CTA per SM issues n_mma of them back to back with no loads in the loop.  two_sm = 1: the cta_group::2 form
+ * (M = 256 over two SMs).  *h_issue_clocks = clocks until the issuing thread is done, *h_done_clocks = until the last
+ * MMA has completed, both per MMA.  Tells a main loop that waits for operands from one the tensor pipe limits.
+ * bf16 handles only.  Synchronises. */
+int specdec_debug_mma_rate(specdec_handle* h, int bn, int two_sm, int n_mma, double* h_issue_clocks, double* h_done_clocks);
+
 /* Scripted drafts, a benchmark / test hook with no counterpart in the paper: random-init
  * models almost never agree, so a workload's acceptance pattern is imposed instead.  After the
  * drafter pass has run, draft i of a sequence with j committed tokens is replaced by

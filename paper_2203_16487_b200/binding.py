@@ -24,7 +24,7 @@ EXPORTS = [
     "specdec_commit", "specdec_generate", "specdec_generate_host", "specdec_get_output",
     "specdec_accept_scan", "specdec_debug_logits", "specdec_debug_row_stats", "specdec_set_option",
     "specdec_launch_count", "specdec_last_error", "specdec_set_draft_script", "specdec_profile_read",
-    "specdec_accept_scan_static", "specdec_debug_trace", "specdec_debug_link_cost",
+    "specdec_accept_scan_static", "specdec_debug_trace", "specdec_debug_link_cost", "specdec_debug_mma_rate",
 ]
 
 
@@ -79,6 +79,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.specdec_debug_logits.argtypes = [vp, i, vp, vp]
     lib.specdec_debug_row_stats.argtypes = [vp, vp, vp]
     lib.specdec_debug_link_cost.argtypes = [vp, i, i, C.POINTER(C.c_double)]
+    lib.specdec_debug_mma_rate.argtypes = [vp, i, i, i, C.POINTER(C.c_double), C.POINTER(C.c_double)]
     lib.specdec_debug_trace.argtypes = [vp, C.POINTER(C.c_longlong), i]
     lib.specdec_set_option.argtypes = [vp, C.c_char_p, i]
     lib.specdec_set_draft_script.argtypes = [vp, ip, i, i, vp]
@@ -197,6 +198,12 @@ class SpecDec:
         us = C.c_double()
         self._check(self._lib.specdec_debug_link_cost(self._h, n_links, grid, C.byref(us)))
         return us.value
+
+    def mma_rate(self, bn: int, two_sm: bool = False, n_mma: int = 4096):
+        """(issue, completion) clocks per tcgen05.mma with shared-memory-resident operands (diagnostics)."""
+        a, b = C.c_double(), C.c_double()
+        self._check(self._lib.specdec_debug_mma_rate(self._h, bn, 1 if two_sm else 0, n_mma, C.byref(a), C.byref(b)))
+        return a.value, b.value
 
     def trace(self, n: int):
         buf = (C.c_longlong * n)()

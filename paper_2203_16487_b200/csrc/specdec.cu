@@ -21,6 +21,7 @@
 #include "gemm_tc_pair.cuh"
 #include "gemm_tc_splitk.cuh"
 #include "kernels.cuh"
+#include "mma_rate.cuh"
 #include "skinny_gemm.cuh"
 
 using namespace sd;
@@ -1767,6 +1768,28 @@ int specdec_debug_link_cost(specdec_handle* h, int n_links, int grid, double* h_
     cudaGraphExecDestroy(ex);
     h->launches += 12LL * n_links;
     *h_us_per_link = (double)best * 1e3 / n_links;
+    return SPECDEC_OK;
+}
+
+int specdec_debug_mma_rate(specdec_handle* h, int bn, int two_sm, int n_mma, double* h_issue_clocks, double* h_done_clocks) {
+    if (!h || !h_issue_clocks || !h_done_clocks || n_mma < 16 || n_mma > (1 << 20)) return SPECDEC_ERR_INVALID_ARG;
+    if (h->dtype != SPECDEC_DTYPE_BF16 || !h->tma.ready) return fail(h, SPECDEC_ERR_UNSUPPORTED, "mma rate: needs a bf16 handle on an sm_100 device");
+    cudaStream_t st = h->own_stream;
+    long long* scratch = reinterpret_cast<long long*>(h->part);          // (the vocabulary partials: at least 2 x 148 words)
+    int* errw = h->ses.counters + 7;
+    cudaError_t e;
+    if (two_sm) {
+        if (bn == 128) e = sd::mma_rate_run<128, true>(h->tma.n_sm, n_mma, scratch, errw, st, h_issue_clocks, h_done_clocks);
+        else if (bn == 256) e = sd::mma_rate_run<256, true>(h->tma.n_sm, n_mma, scratch, errw, st, h_issue_clocks, h_done_clocks);
+        else return fail(h, SPECDEC_ERR_INVALID_ARG, "mma rate: two-SM tiles are 128 or 256 columns wide");
+    } else {
+        if (bn == 64) e = sd::mma_rate_run<64, false>(h->tma.n_sm, n_mma, scratch, errw, st, h_issue_clocks, h_done_clocks);
+        else if (bn == 128) e = sd::mma_rate_run<128, false>(h->tma.n_sm, n_mma, scratch, errw, st, h_issue_clocks, h_done_clocks);
+        else if (bn == 256) e = sd::mma_rate_run<256, false>(h->tma.n_sm, n_mma, scratch, errw, st, h_issue_clocks, h_done_clocks);
+        else return fail(h, SPECDEC_ERR_INVALID_ARG, "mma rate: tiles are 64, 128 or 256 columns wide");
+    }
+    if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("mma rate: ") + cudaGetErrorString(e));
+    h->launches += 2;
     return SPECDEC_OK;
 }
 

@@ -140,7 +140,24 @@ def main():
     ap.add_argument("--ttft", action="store_true", help="time to the first tokens on summarisation-shaped inputs (batch 8, "
                     "sources of 300-512 ids) or, with --translation, on one translation-shaped sentence")
     ap.add_argument("--translation", action="store_true")
+    ap.add_argument("--mma-rate", action="store_true", help="clocks per tcgen05.mma with operands resident in shared memory, "
+                    "and the cost of a kernel boundary (library diagnostics)")
     args = ap.parse_args()
+    if args.mma_rate:
+        wl = W.config1_tiny()
+        dims = W.ModelDims(128, 2, 512, 2000, 1, 1, 64)
+        wv, wd = W.make_weights(dims, 1, True), W.make_weights(dims, 2, True)
+        sd = binding.SpecDec(dims, wv, dims, wd, k_max=8, max_batch=32, max_src=16, max_tgt=16, bf16=True)
+        rows = []
+        for bn, two in ((64, False), (128, False), (256, False), (128, True), (256, True)):
+            issue, done = sd.mma_rate(bn, two, 8192)
+            m = 256 if two else 128
+            ideal = m * bn * 16 * 2 / (2250e12 / 148 / 1.965e9) / (2 if two else 1)     # clocks per MMA at the nominal dense bf16 rate of the SMs involved
+            rows.append({"M": m, "N": bn, "two_sm": two, "issue_clocks": issue, "completion_clocks": done, "nominal_clocks": ideal,
+                         "fraction_of_nominal": ideal / done})
+        print(json.dumps({"step": "mma_rate", "rows": rows, "link_cost_us": {g: sd.link_cost(64, g) for g in (8, 148, 592)}}))
+        sd.close()
+        return
     if args.ttft:
         wl = W.config2_translation(1) if args.translation else W.config4_summarization()
         wv = W.make_weights(wl.verifier, wl.seed_verifier, True)

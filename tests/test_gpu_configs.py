@@ -287,3 +287,21 @@ def test_bart_base_shaped_pair_gelu_learned_positions():
     ref, _ = O.specdec_generate(mv, md, wl.src[2], 10, 25, 3, 1.0, BOS, EOS, MASK)
     assert out[2, :10].cpu().tolist() == ref
     sd.close()
+
+
+@pytest.mark.parametrize("d,f,enc,dec", [(256, 1024, 12, 2), (512, 2048, 6, 6)])
+def test_drafter_ablation_shapes(d, f, enc, dec):
+    """The drafter-ablation table's other drafters (Section 4.1): model / FFN width 256 / 1024 ("w/o Principle I") and a
+    balanced 6 + 6 drafter ("w/o Principle II"), each paired with the Transformer-base verifier: lock-step against the
+    oracle on two sentences (drafts, accepted lengths, bifurcation tokens, logits)."""
+    from paper_2203_16487_b200 import binding
+    dd = W.ModelDims(d, 8 if d == 512 else 4, f, 32768, enc, dec, 1024)
+    wv, wd = W.make_weights(W.BASE_V, 1001, True), W.make_weights(dd, 4002, True)
+    mv, md = O.model_from(W.BASE_V, wv, mode="bf16"), O.model_from(dd, wd, mode="bf16")
+    wl = W.config2_translation(2)
+    sd = binding.SpecDec(W.BASE_V, wv, dd, wd, k_max=25, max_batch=2, max_src=40, max_tgt=48, bf16=True)
+    rep = lockstep.run(sd, mv, md, wl.src, [16, 16], 25, 3, 1.0, margin=1e-3, check_logits_every=2, max_iters=4)
+    print(rep.iterations, rep.draft_positions, rep.draft_near_ties, rep.verify_near_ties, rep.max_logit_err, rep.notes[:3])
+    assert rep.ok, rep.notes
+    assert rep.max_logit_err < 2e-2
+    sd.close()
