@@ -264,9 +264,10 @@ def tokens_leg(torch, binding, B: int, K_: int, W_: int, rank: int, world: int, 
                         diverged[0] += 1
         return toks, ms, stats
 
-    def timed(host=False, scripted=True, k=K_BLOCK, min_ms=MIN_TIMED_MS):
+    def timed(host=False, scripted=True, k=K_BLOCK, min_ms=None):
         """The K-step stream, repeated until the region is at least min_ms long; returns (tokens, ms, stats, repeats)."""
         toks, ms, stats, reps = 0, 0.0, [], 0
+        min_ms = MIN_TIMED_MS if min_ms is None else min_ms
         while reps == 0 or ms < min_ms:
             t, m, st = one_pass(W_, K_, host, scripted, k, check=(reps == 0))
             toks += t; ms += m; stats += st; reps += 1
@@ -429,14 +430,14 @@ def run_ours(args):
                 "ms_breakdown", "unscripted", "greedy_ar"):
         if key in leg:
             line[key] = leg[key]
-    if rank == 0:
+    if rank == 0 and not args.no_roofline:
         # the verify step against its roofline (rank 0: a single-GPU measurement)
         line["roofline"] = verify_step_roofline(torch, binding, B, local, args.opt)
     if B == 1 and not args.no_batch128:
         # the metric's batch-128 half, in the same line: tokens/s on the padded-batch workload and the verify step
         # against the tensor roofline
         b128 = tokens_leg(torch, binding, 128, min(args.steps, 6), args.warmup, rank, world, local, args.opt, args.poll_lag, False)
-        if rank == 0:
+        if rank == 0 and not args.no_roofline:
             b128["roofline"] = verify_step_roofline(torch, binding, 128, local, args.opt, reps=30)
         b128["config"] = config_of(b128.pop("workload"), 128, world)
         line["batch128"] = b128
@@ -477,9 +478,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-batch128", action="store_true", help="skip the batch-128 leg of the default (batch 1) run")
+    ap.add_argument("--no-roofline", action="store_true", help="skip the verify-step roofline legs (profiling runs)")
+    ap.add_argument("--min-timed-ms", type=float, default=None, help="length of the timed region that the K-step stream is repeated to "
+                    "reach (default 2000; 0 = the K steps once, for profiling runs)")
     ap.add_argument("--opt", action="append", default=[], help="experiments: name=value passed to specdec_set_option")
     ap.add_argument("--poll-lag", type=int, default=None, help="experiments: iterations the host runs ahead of the finish counter")
     args = ap.parse_args()
+    if args.min_timed_ms is not None:
+        global MIN_TIMED_MS
+        MIN_TIMED_MS = args.min_timed_ms
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)

@@ -131,6 +131,35 @@ __global__ void k_verify_prep(Session s, const int* __restrict__ draft, int B, i
     r.nk_cross[i] = s.src_len[b];
 }
 
+// The same, together with the embedding of the block's rows (x = sqrt(d) E[tok] + P[pos]): one block per row.  The row
+// metadata is complete before the block lets its successors start, because kernels further down the chain read it
+// ahead of their own dependency waits.
+template <typename T>
+__global__ void k_verify_prep_embed(Session s, const int* __restrict__ draft, int B, int k, int S_max, int bos, Rows r,
+                                    const T* __restrict__ E, const float* __restrict__ P, float* __restrict__ x, int d,
+                                    float scale, int vocab, int max_pos) {
+    const int i = blockIdx.x;                      // row b * (k + 1) + c
+    pdl_wait();                                    // session state comes from the previous step's commit
+    const int b = i / (k + 1), c = i % (k + 1);
+    const int j = s.len[b];
+    const int tok = (c == 0) ? (j == 0 ? bos : s.out[(size_t)b * s.out_stride + j - 1]) : draft[b * k + c - 1];
+    if (threadIdx.x == 0) {
+        if (i == 0) s.counters[CNT_VERIFY] = B * (k + 1);
+        if (c == 0) { r.kv_off_cross[b] = b * S_max; r.q_off[b] = b * (k + 1); r.q_cnt[b] = k + 1; }
+        r.tok[i] = tok;
+        r.pos[i] = j + c;
+        r.seq[i] = b;
+        r.nk_self[i] = j + c + 1;     // causal: positions 0..j+c
+        r.nk_cross[i] = s.src_len[b];
+        __threadfence();
+    }
+    __syncthreads();
+    pdl_launch_dependents();
+    const int t = min(max(tok, 0), vocab - 1), p = min(max(j + c, 0), max_pos - 1);
+    for (int e = threadIdx.x; e < d; e += blockDim.x)
+        x[(size_t)i * d + e] = scale * to_f(E[(size_t)t * d + e]) + P[(size_t)p * d + e];
+}
+
 // Drafter: packed rows [BOS, committed, MASK x k] of every unfinished sequence.
 // `all` describes the full pass, `msk` the mask-only continuation of the last layer.
 // One block per sequence: it sums the row counts of the sequences before it (B loads spread over its threads: the
@@ -345,6 +374,66 @@ __global__ void k_layernorm(const float* __restrict__ x, const float* __restrict
     for (int e = lane; e < d; e += 32) { float c = xr[e] - mu; v += c * c; }
     float rstd = 1.0f / sqrtf(warp_sum(v) / d + eps);
     for (int e = lane; e < d; e += 32) y[(size_t)row * d + e] = from_f<T>((xr[e] - mu) * rstd * g[e] + b[e]);
+}
+
+// Final LayerNorm of the verify rows together with the pre-pass logit of each row's draft (the dot product of the
+// normalised, operand-rounded row with the draft's embedding row): one warp per row, rows of d = 128 NC elements in registers.
+template <typename T, int NC>
+__global__ void k_layernorm_ld(const float* __restrict__ x, const float* __restrict__ g, const float* __restrict__ b,
+                               T* __restrict__ y, int d, float eps, const T* __restrict__ E, const int* __restrict__ draft,
+                               int B, int k, int vocab, float* __restrict__ ld, int* __restrict__ ld_id) {
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    float4 gm[NC], bt[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const int e = lane * 4 + c * 128;
+        gm[c] = __ldg(reinterpret_cast<const float4*>(g + e));
+        bt[c] = __ldg(reinterpret_cast<const float4*>(b + e));
+    }
+    const bool in_range = row < B * (k + 1);
+    const int bs = in_range ? row / (k + 1) : 0, c0 = in_range ? row % (k + 1) : k;
+    const int tok = (in_range && c0 < k) ? draft[bs * k + c0] : -1;       // drafts predate the step's kernel chain
+    const bool ok = tok >= 0 && tok < vocab;
+    pdl_launch_dependents();
+    pdl_wait();
+    if (!in_range) return;
+    const float* xr = x + (size_t)row * d;
+    float4 v[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) v[c] = *reinterpret_cast<const float4*>(xr + lane * 4 + c * 128);
+    float sm = 0.f;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) sm += v[c].x + v[c].y + v[c].z + v[c].w;
+    const float mu = warp_sum(sm) / d;
+    float q = 0.f;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const float a0 = v[c].x - mu, a1 = v[c].y - mu, a2 = v[c].z - mu, a3 = v[c].w - mu;
+        q += a0 * a0 + a1 * a1 + a2 * a2 + a3 * a3;
+    }
+    const float rstd = 1.0f / sqrtf(warp_sum(q) / d + eps);
+    float dot = 0.f;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const int e = lane * 4 + c * 128;
+        T o[4];
+        o[0] = from_f<T>((v[c].x - mu) * rstd * gm[c].x + bt[c].x);
+        o[1] = from_f<T>((v[c].y - mu) * rstd * gm[c].y + bt[c].y);
+        o[2] = from_f<T>((v[c].z - mu) * rstd * gm[c].z + bt[c].z);
+        o[3] = from_f<T>((v[c].w - mu) * rstd * gm[c].w + bt[c].w);
+        T* yo = y + (size_t)row * d + e;
+        yo[0] = o[0]; yo[1] = o[1]; yo[2] = o[2]; yo[3] = o[3];
+        if (ok) {
+            const T* ep = E + (size_t)tok * d + e;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) dot = fmaf(to_f(o[i]), to_f(ep[i]), dot);
+        }
+    }
+    dot = warp_sum(dot);
+    if (lane == 0) {
+        if (c0 == k) { ld[row] = CUDART_INF_F; ld_id[row] = -1; }
+        else { ld[row] = ok ? dot : -CUDART_INF_F; ld_id[row] = ok ? tok : -2; }
+    }
 }
 
 // ------------------------------------------------------------------ paged KV cache
@@ -611,12 +700,55 @@ __global__ void k_draft_logit(const T* __restrict__ y, const T* __restrict__ E, 
     if (lane == 0) { ld[row] = ok ? s : -CUDART_INF_F; ld_id[row] = ok ? tok : -2; }
 }
 
+// ------------------------------------------------------------------ commit / rollback (Eq. 3)
+// Appends drafts[0..keep) and the next token to sequence b, cuts after the first EOS and at max_tgt.
+// Cache rows beyond the new length are simply dead: the next block overwrites them.
+__device__ __forceinline__ void commit_sequence(const Session& s, int b, const int* __restrict__ draft, int keep, int next,
+                                                int k, int eos) {
+    if (s.finished[b]) return;
+    int j = s.len[b];
+    const int mt = s.max_tgt[b];
+    const int a = min(max(keep, 0), k);
+    bool fin = false;
+    const int n0 = j;
+    for (int c = 0; c <= a && !fin; ++c) {
+        if (j >= mt) { fin = true; break; }
+        const int tok = (c < a) ? draft[b * k + c] : next;
+        s.out[(size_t)b * s.out_stride + j] = tok;
+        ++j;
+        if (tok == eos) fin = true;
+    }
+    if (j >= mt) fin = true;
+    s.len[b] = j;
+    atomicAdd(&s.stats[0], 1ull);
+    atomicAdd(&s.stats[1], (unsigned long long)k);
+    atomicAdd(&s.stats[2], (unsigned long long)a);
+    atomicAdd(&s.stats[3], (unsigned long long)(j - n0));
+    if (fin) { s.finished[b] = 1; atomicSub(&s.counters[CNT_ACTIVE], 1); }
+}
+// The last block of the grid to get here posts (commits of this handle so far) << 32 | (sequences still decoding) to the
+// host-mapped word the generation loop polls: no copy, no event between the iterations.  Call after __syncthreads().
+__device__ __forceinline__ void commit_post(const Session& s, unsigned long long* post) {
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(&s.counters[CNT_TICKET], 1) == (int)gridDim.x - 1) {
+            s.counters[CNT_TICKET] = 0;
+            const int seq = ++s.counters[CNT_SEQ];
+            const int active = atomicAdd(&s.counters[CNT_ACTIVE], 0);
+            *reinterpret_cast<volatile unsigned long long*>(post) = ((unsigned long long)(unsigned)seq << 32) | (unsigned)active;
+            __threadfence_system();
+        }
+    }
+}
+// What the acceptance scan needs to commit its own decision (the generation loop): on = 0 leaves the commit to k_commit.
+struct FusedCommit { Session s; const int* draft; int eos; unsigned long long* post; int on; };
+
 // ------------------------------------------------------------------ acceptance scan (Eq. 7-9)
 // One block per sequence: warps merge the per-tile statistics of the k+1 rows, thread 0
 // finds the first rejected draft.  row_stats (optional) receives 6 floats per row.
 __global__ void k_accept(const RowPart* __restrict__ part, int n_tiles, const float* __restrict__ ld,
                          const int* __restrict__ ld_id, int k, int beta, float tau, int* __restrict__ accepted,
-                         int* __restrict__ bif, float* __restrict__ row_stats, int want_sum) {
+                         int* __restrict__ bif, float* __restrict__ row_stats, int want_sum, FusedCommit fc) {
     extern __shared__ unsigned char sm_acc[];
     RowPart* rs = reinterpret_cast<RowPart*>(sm_acc);       // [k+1]
     __shared__ unsigned char ok_s[256];                     // row c passes both tests (k <= 255 rows take this path)
@@ -671,6 +803,7 @@ __global__ void k_accept(const RowPart* __restrict__ part, int n_tiles, const fl
         }
         accepted[b] = a;
         bif[b] = rs[a].arg;
+        if (fc.on) commit_sequence(fc.s, b, fc.draft, a, rs[a].arg, k, fc.eos);
     }
     if (row_stats)
         for (int c = threadIdx.x; c <= k; c += blockDim.x) {
@@ -678,6 +811,7 @@ __global__ void k_accept(const RowPart* __restrict__ part, int n_tiles, const fl
             o[0] = rs[c].mx; o[1] = (float)rs[c].arg; o[2] = want_sum ? rs[c].mx + logf(rs[c].sum) : 0.f;
             o[3] = (float)rs[c].cnt; o[4] = ld[b * (k + 1) + c]; o[5] = (float)ld_id[b * (k + 1) + c];
         }
+    if (fc.on) { __syncthreads(); commit_post(fc.s, fc.post); }
 }
 
 // The same rule on caller-provided logits [B, k+1, V]: one block per sequence walks the rows
@@ -799,47 +933,14 @@ __global__ void k_apply_script(Session s, const int* __restrict__ script, int st
     if (p < stride) { int t = script[(size_t)b * stride + p]; if (t >= 0) draft[i] = t; }
 }
 
-// ------------------------------------------------------------------ commit / rollback (Eq. 3)
-// Appends drafts[0..keep) and the next token, cuts after the first EOS and at max_tgt.
-// Cache rows beyond the new length are simply dead: the next block overwrites them.
+// Commit as a kernel of its own (specdec_commit; explicit keep / next).
 __global__ void k_commit(Session s, const int* __restrict__ draft, const int* __restrict__ keep,
                          const int* __restrict__ next, int B, int k, int eos, unsigned long long* post) {
     int b = blockIdx.x * blockDim.x + threadIdx.x;
     pdl_wait();                                    // no early trigger: the lengths written here are read by later kernels BEFORE their waits
-    if (b < B && !s.finished[b]) {
-        int j = s.len[b];
-        const int mt = s.max_tgt[b];
-        const int a = min(max(keep[b], 0), k);
-        bool fin = false;
-        int n0 = j;
-        for (int c = 0; c <= a && !fin; ++c) {
-            if (j >= mt) { fin = true; break; }
-            int tok = (c < a) ? draft[b * k + c] : next[b];
-            s.out[(size_t)b * s.out_stride + j] = tok;
-            ++j;
-            if (tok == eos) fin = true;
-        }
-        if (j >= mt) fin = true;
-        s.len[b] = j;
-        atomicAdd(&s.stats[0], 1ull);
-        atomicAdd(&s.stats[1], (unsigned long long)k);
-        atomicAdd(&s.stats[2], (unsigned long long)a);
-        atomicAdd(&s.stats[3], (unsigned long long)(j - n0));
-        if (fin) { s.finished[b] = 1; atomicSub(&s.counters[CNT_ACTIVE], 1); }
-    }
-    // the last block to get here posts (commits of this handle so far) << 32 | (sequences still decoding) to the
-    // host-mapped word the generation loop polls: no copy, no event between the iterations
+    if (b < B) commit_sequence(s, b, draft, keep[b], next[b], k, eos);
     __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        if (atomicAdd(&s.counters[CNT_TICKET], 1) == (int)gridDim.x - 1) {
-            s.counters[CNT_TICKET] = 0;
-            const int seq = ++s.counters[CNT_SEQ];
-            const int active = atomicAdd(&s.counters[CNT_ACTIVE], 0);
-            *reinterpret_cast<volatile unsigned long long*>(post) = ((unsigned long long)(unsigned)seq << 32) | (unsigned)active;
-            __threadfence_system();
-        }
-    }
+    commit_post(s, post);
 }
 
 __global__ void k_session_init(Session s, const int* __restrict__ src_len, const int* __restrict__ max_tgt, int B,

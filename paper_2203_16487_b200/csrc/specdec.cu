@@ -81,6 +81,8 @@ struct specdec_handle {
     std::vector<void*> dkc, dvc;
     int drafter_pc = 0;             // option "drafter_prefix_causal", as set
     int drafter_pc_session = 0;     // ... as in force for the running session (latched by specdec_encode)
+    bool fuse_commit = false;       // the generation loop: the acceptance scan commits its own decision (no commit kernel)
+    bool commit_done = false;       // ... and did so in the verify pass just issued
     int dnew_ub = 1;                // upper bound on the prefix positions the next draft pass has to add to that cache
     int* page_table;
     // rows
@@ -914,9 +916,11 @@ int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float ta
     const int max_keys = std::min(h->len_ub, h->T_cap) + k + 1;
     if (d_draft != h->v_draft && k > 0)
         CUDA_TRY(h, cudaMemcpyAsync(h->v_draft, d_draft, (size_t)B * k * 4, cudaMemcpyDeviceToDevice, st));
-    k_verify_prep<<<cdiv(M, 256), 256, 0, st>>>(h->ses, h->v_draft, B, k, h->S_max, h->cfg.bos_id, h->rows);
+    // row metadata and embedding of the block in one kernel
+    h->fused_x = nullptr;
+    CUDA_TRY(h, launch_pdl(h, k_verify_prep_embed<T>, dim3(M), dim3(128), 0, st, h->ses, (const int*)h->v_draft, B, k, h->S_max, h->cfg.bos_id,
+                           h->rows, (const T*)m.embed, (const float*)m.pos_dec, h->x, d, sqrtf((float)d), m.dm.vocab, m.dm.max_pos));
     KCHECK(h);
-    TRY(embed<T>(h, m, h->rows, m.pos_dec, CNT_VERIFY, M, st));
     for (int l = 0; l < L; ++l) {
         const bool last = l + 1 == L;
         TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_VERIFY, M, k + 1, h->kc[l], h->vc[l], h->ses.len /* cached prefix: positions < len */,
@@ -925,18 +929,36 @@ int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float ta
         TRY(block_ffn<T>(h, m, m.dec[l], h->x, CNT_VERIFY, M, st, last ? m.dec_lnf_g : m.dec[l + 1].ln1_g,
                          last ? m.dec_lnf_b : m.dec[l + 1].ln1_b));
     }
-    TRY(ln_or_fused<T>(h, h->x, m.dec_lnf_g, m.dec_lnf_b, CNT_VERIFY, M, h->y, d, st));
-    CUDA_TRY(h, launch_pdl(h, k_draft_logit<T>, dim3(cdiv(M, 4)), dim3(128), 0, st, (const T*)h->y, (const T*)m.embed,
-                           (const int*)h->v_draft, B, k, d, m.dm.vocab, h->ld, h->ld_id));
-    KCHECK(h);
+    const bool ln_pending = !(h->x == h->fused_x && m.dec_lnf_g == h->fused_g && h->y == h->fused_out);
+    if (ln_pending && d % 128 == 0 && d <= 1024 && !(h->diag_repeat & 2)) {
+        // final LayerNorm and the pre-pass logit of every row's draft in one kernel
+        cudaError_t e = cudaSuccess;
+        const dim3 grid(cdiv(M, 8)), block(256);
+#define LN_LD(NC) e = launch_pdl(h, k_layernorm_ld<T, NC>, grid, block, 0, st, (const float*)h->x, (const float*)m.dec_lnf_g, (const float*)m.dec_lnf_b, (T*)h->y, d, 1e-5f, \
+                                 (const T*)m.embed, (const int*)h->v_draft, B, k, m.dm.vocab, h->ld, h->ld_id)
+        switch (d / 128) {
+            case 1: LN_LD(1); break; case 2: LN_LD(2); break; case 3: LN_LD(3); break; case 4: LN_LD(4); break;
+            case 5: LN_LD(5); break; case 6: LN_LD(6); break; case 7: LN_LD(7); break; default: LN_LD(8); break;
+        }
+#undef LN_LD
+        if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("final layer norm launch: ") + cudaGetErrorString(e));
+        KCHECK(h);
+    } else {
+        TRY(ln_or_fused<T>(h, h->x, m.dec_lnf_g, m.dec_lnf_b, CNT_VERIFY, M, h->y, d, st));
+        CUDA_TRY(h, launch_pdl(h, k_draft_logit<T>, dim3(cdiv(M, 4)), dim3(128), 0, st, (const T*)h->y, (const T*)m.embed,
+                               (const int*)h->v_draft, B, k, d, m.dm.vocab, h->ld, h->ld_id));
+        KCHECK(h);
+    }
     int n_tiles = 0;
     prof_mark(h, st);
     TRY(gemm<T>(h, EPI_STATS, h->y, d, m.embed, nullptr, m.dm.vocab, d, CNT_VERIFY, M, nullptr, 0, nullptr, st, h->ld,
                 h->ld_id, &n_tiles));
     prof_mark(h, st);
+    FusedCommit fc{h->ses, h->v_draft, h->cfg.eos_id, h->h_post, h->fuse_commit ? 1 : 0};
     CUDA_TRY(h, launch_pdl(h, k_accept, dim3(B), dim3(1024), (size_t)(k + 1) * sizeof(RowPart), st, (const RowPart*)h->part, n_tiles,
-                           (const float*)h->ld, (const int*)h->ld_id, k, beta, tau, h->accepted, h->bif, h->row_stats, h->want_lse));
+                           (const float*)h->ld, (const int*)h->ld_id, k, beta, tau, h->accepted, h->bif, h->row_stats, h->want_lse, fc));
     KCHECK(h);
+    h->commit_done = h->fuse_commit;
     if (d_accepted) CUDA_TRY(h, cudaMemcpyAsync(d_accepted, h->accepted, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
     if (d_bif) CUDA_TRY(h, cudaMemcpyAsync(d_bif, h->bif, (size_t)B * 4, cudaMemcpyDeviceToDevice, st));
     h->last_k = k; h->verified = true; h->drafted = false;
@@ -945,9 +967,13 @@ int verify_impl(specdec_handle* h, const int* d_draft, int k, int beta, float ta
 
 int commit_impl(specdec_handle* h, const int* d_keep, const int* d_next, cudaStream_t st) {
     const int k = h->last_k;
-    CUDA_TRY(h, launch_pdl(h, k_commit, dim3(cdiv(h->B, 128)), dim3(128), 0, st, h->ses, (const int*)h->v_draft,
-                           (const int*)(d_keep ? d_keep : h->accepted), (const int*)(d_next ? d_next : h->bif), h->B, k, h->cfg.eos_id, h->h_post));
-    KCHECK(h);
+    if (h->commit_done && !d_keep && !d_next) {
+        h->commit_done = false;                    // the acceptance scan of this verify pass has committed already
+    } else {
+        CUDA_TRY(h, launch_pdl(h, k_commit, dim3(cdiv(h->B, 128)), dim3(128), 0, st, h->ses, (const int*)h->v_draft,
+                               (const int*)(d_keep ? d_keep : h->accepted), (const int*)(d_next ? d_next : h->bif), h->B, k, h->cfg.eos_id, h->h_post));
+        KCHECK(h);
+    }
     h->len_ub = std::min(h->len_ub + k + 1, h->T_cap);
     h->dnew_ub = std::min(h->dnew_ub + k + 1, h->T_cap + 1);
     h->verified = false;
@@ -985,7 +1011,7 @@ inline void graph_key_tail(const specdec_handle* h, std::vector<long long>& key)
                         (long long)h->use_pdl, (long long)h->use_ln_fuse, (long long)h->use_sk_cluster,
                         (long long)h->use_pair, (long long)h->diag_repeat, (long long)h->use_splitk, (long long)h->attn_stream, (long long)h->attn_stream_keys, (long long)h->attn_warps, (long long)h->attn_rs,
                         (long long)h->skinny_groups, (long long)h->want_trace,
-                        (long long)(h->script_on ? 1 : 0), (long long)h->B, (long long)h->S_max, (long long)h->drafter_pc_session})
+                        (long long)(h->script_on ? 1 : 0), (long long)h->B, (long long)h->S_max, (long long)h->drafter_pc_session, (long long)(h->fuse_commit ? 1 : 0)})
         key.push_back(v);
 }
 
@@ -1091,6 +1117,9 @@ int generate_loop(specdec_handle* h, const int* d_src, const int* d_src_len, con
                   int k, int beta, float tau, int* d_out, int out_stride, int* d_out_len, specdec_stats* hs,
                   cudaStream_t st) {
     const bool timed = hs != nullptr, phases = timed && h->stats_timing;
+    // the acceptance scan commits its own decision (one kernel less per iteration) unless the phases are timed apart
+    struct FuseGuard { specdec_handle* h; ~FuseGuard() { h->fuse_commit = false; h->commit_done = false; } } fuse_guard{h};
+    h->fuse_commit = !phases;
     size_t ev = 0;
     auto mark_always = [&]() { if (timed && ev < h->time_ev.size()) cudaEventRecord(h->time_ev[ev++], st); };
     auto mark = [&]() { if (phases) mark_always(); };
@@ -1711,8 +1740,9 @@ int specdec_accept_scan_static(const float* d_logits, const int32_t* d_draft, in
     cudaStream_t st = (cudaStream_t)stream;
     // every slot the second stage reads is rewritten by the first, so nothing has to start at zero
     k_logit_tile_stats<<<dim3(n_tiles, (unsigned)rows), 256, 0, st>>>(d_logits, d_draft, k, V, NA_TILE, n_tiles, part, ld, ld_id);
+    FusedCommit no_commit{};
     k_accept<<<B, 256, (size_t)(k + 1) * sizeof(RowPart), st>>>(part, n_tiles, ld, ld_id, k, beta, tau, d_accepted, d_bif,
-                                                                nullptr, 0);
+                                                                nullptr, 0, no_commit);
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(nullptr, SPECDEC_ERR_CUDA, std::string("accept_scan_static: ") + cudaGetErrorString(e));
     return SPECDEC_OK;
