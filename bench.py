@@ -382,6 +382,8 @@ def verify_step_roofline(torch, binding, B: int, local: int, opts, reps: int = 5
     rest = us - sum(e["us_in_step"] for e in by_kernel)
     by_kernel.append({"class": "residual GEMMs (attention out x2, FFN2), embedding, accept scan, the rest", "launches": None,
                       "us_in_step": rest, "share_of_step": rest / us})
+    link_us = sd.link_cost(64, 148)
+    round_ns = sd.cluster_round(16, 2048, 64)
     sd.close()
     del flush
     hbm_bound = (bytes_ / (hbm_peak * 1e9)) >= (flops / (tc_peak * 1e12))
@@ -400,6 +402,12 @@ def verify_step_roofline(torch, binding, B: int, local: int, opts, reps: int = 5
         "peak_kind": f"of {peak_kind}", "us_per_step_median": us, "us_per_step_min": us_min, "repetitions": reps,
         "launches_per_step": int(launches_per_step), "algorithmic_bytes_per_launch": int(bytes_), "algorithmic_flops_per_launch": flops,
         "roofline_us": max(bytes_ / (hbm_peak * 1e9), flops / (tc_peak * 1e12)) * 1e6, "mean_accepted": mean_a, "by_kernel": by_kernel,
+        # the step is a chain of dependent launches: what the chain alone costs, from the library's own probes
+        "latency_floor": {"launches_per_step": int(launches_per_step), "us_per_kernel_boundary": link_us,
+                          "us": launches_per_step * link_us, "step_over_floor": us / (launches_per_step * link_us),
+                          "us_per_16cta_cluster_exchange_of_32KB": round_ns / 1e3,
+                          "note": "kernel boundary = one link of a chain of dependent 148-CTA launches (programmatic dependent launch, "
+                                  "replayed from a graph); the cluster exchange is what a fused cluster kernel would pay instead of a boundary"},
     })
     return roof
 

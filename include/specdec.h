@@ -207,6 +207,12 @@ int specdec_debug_trace(specdec_handle* h, long long* h_out, int n);
  * replays divided by n_links, in microseconds.  Synchronises. */
 int specdec_debug_link_cost(specdec_handle* h, int n_links, int grid, double* h_us_per_link);
 
+/* Diagnostics: nanoseconds per exchange round between the CTAs of one thread-block cluster (8 or 16 CTAs of 256
+ * threads) through distributed shared memory: every CTA stores bytes_per_peer (0 .. 8192, a multiple of 16) bytes into each
+ * peer's shared memory, arrives on every peer's barrier and waits for all arrivals; `rounds` rounds back to back.
+ * What a fused cluster kernel pays where separate kernels pay a kernel boundary.  Synchronises. */
+int specdec_debug_cluster_round(specdec_handle* h, int cluster_size, int bytes_per_peer, int rounds, double* h_ns_per_round);
+
 /* Diagnostics: clocks per tcgen05.mma (M = 128 x N = bn x K = 16, bf16) when the operands already sit in shared memory:
  * one CTA per SM issues n_mma of them back to back with no loads in the loop.  two_sm = 1: the cta_group::2 form
  * (M = 256 over two SMs).  *h_issue_clocks = clocks until the issuing thread is done, *h_done_clocks = until the last

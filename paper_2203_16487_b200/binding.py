@@ -24,7 +24,7 @@ EXPORTS = [
     "specdec_commit", "specdec_generate", "specdec_generate_host", "specdec_get_output",
     "specdec_accept_scan", "specdec_debug_logits", "specdec_debug_row_stats", "specdec_set_option",
     "specdec_launch_count", "specdec_last_error", "specdec_set_draft_script", "specdec_profile_read",
-    "specdec_accept_scan_static", "specdec_debug_trace", "specdec_debug_link_cost", "specdec_debug_mma_rate",
+    "specdec_accept_scan_static", "specdec_debug_trace", "specdec_debug_link_cost", "specdec_debug_mma_rate", "specdec_debug_cluster_round",
 ]
 
 
@@ -80,6 +80,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.specdec_debug_row_stats.argtypes = [vp, vp, vp]
     lib.specdec_debug_link_cost.argtypes = [vp, i, i, C.POINTER(C.c_double)]
     lib.specdec_debug_mma_rate.argtypes = [vp, i, i, i, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    lib.specdec_debug_cluster_round.argtypes = [vp, i, i, i, C.POINTER(C.c_double)]
     lib.specdec_debug_trace.argtypes = [vp, C.POINTER(C.c_longlong), i]
     lib.specdec_set_option.argtypes = [vp, C.c_char_p, i]
     lib.specdec_set_draft_script.argtypes = [vp, ip, i, i, vp]
@@ -204,6 +205,12 @@ class SpecDec:
         a, b = C.c_double(), C.c_double()
         self._check(self._lib.specdec_debug_mma_rate(self._h, bn, 1 if two_sm else 0, n_mma, C.byref(a), C.byref(b)))
         return a.value, b.value
+
+    def cluster_round(self, cluster_size: int = 16, bytes_per_peer: int = 0, rounds: int = 64) -> float:
+        """Nanoseconds per all-to-all exchange round inside one thread-block cluster (diagnostics)."""
+        ns = C.c_double()
+        self._check(self._lib.specdec_debug_cluster_round(self._h, cluster_size, bytes_per_peer, rounds, C.byref(ns)))
+        return ns.value
 
     def trace(self, n: int):
         buf = (C.c_longlong * n)()

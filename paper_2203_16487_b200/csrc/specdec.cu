@@ -17,6 +17,7 @@
 #include "../../include/specdec.h"
 #include "attention_stream.cuh"
 #include "attention_tc.cuh"
+#include "cluster_round.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_tc_pair.cuh"
 #include "gemm_tc_splitk.cuh"
@@ -1798,6 +1799,20 @@ int specdec_debug_link_cost(specdec_handle* h, int n_links, int grid, double* h_
     cudaGraphExecDestroy(ex);
     h->launches += 12LL * n_links;
     *h_us_per_link = (double)best * 1e3 / n_links;
+    return SPECDEC_OK;
+}
+
+int specdec_debug_cluster_round(specdec_handle* h, int cluster_size, int bytes_per_peer, int rounds, double* h_ns_per_round) {
+    if (!h || !h_ns_per_round || rounds < 1 || rounds > 4096 || bytes_per_peer < 0 || bytes_per_peer > 8192 || bytes_per_peer % 16)
+        return SPECDEC_ERR_INVALID_ARG;
+    cudaStream_t st = h->own_stream;
+    long long* scratch = reinterpret_cast<long long*>(h->trace_buf + 128);
+    cudaError_t e;
+    if (cluster_size == 8) e = sd::cluster_round_run<8>(rounds, bytes_per_peer, scratch, h->ses.counters + 7, st, h_ns_per_round);
+    else if (cluster_size == 16) e = sd::cluster_round_run<16>(rounds, bytes_per_peer, scratch, h->ses.counters + 7, st, h_ns_per_round);
+    else return fail(h, SPECDEC_ERR_INVALID_ARG, "cluster round: clusters of 8 or 16 CTAs");
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(h, SPECDEC_ERR_CUDA, std::string("cluster round: ") + cudaGetErrorString(e)); }
+    h->launches += 2;
     return SPECDEC_OK;
 }
 

@@ -155,7 +155,9 @@ def main():
             ideal = m * bn * 16 * 2 / (2250e12 / 148 / 1.965e9) / (2 if two else 1)     # clocks per MMA at the nominal dense bf16 rate of the SMs involved
             rows.append({"M": m, "N": bn, "two_sm": two, "issue_clocks": issue, "completion_clocks": done, "nominal_clocks": ideal,
                          "fraction_of_nominal": ideal / done})
-        print(json.dumps({"step": "mma_rate", "rows": rows, "link_cost_us": {g: sd.link_cost(64, g) for g in (8, 148, 592)}}))
+        rounds = {f"{cs} CTAs, {b} B per peer": sd.cluster_round(cs, b, 64) for cs in (8, 16) for b in (0, 2048, 4096)}
+        print(json.dumps({"step": "mma_rate", "rows": rows, "link_cost_us": {g: sd.link_cost(64, g) for g in (8, 148, 592)},
+                          "cluster_round_ns": rounds}))
         sd.close()
         return
     if args.ttft:

@@ -17,6 +17,8 @@ def test_link_cost_and_mma_rate():
     assert 16 <= done <= 1024 and issue <= done + 1           # a 128 x 128 x 16 MMA takes tens of clocks
     issue2, done2 = sd.mma_rate(256, True, 2048)
     assert done2 > 0.9 * done                                 # twice the columns over twice the SMs: not faster per instruction
+    ns0, ns1 = sd.cluster_round(16, 0, 32), sd.cluster_round(16, 4096, 32)
+    assert 50 < ns0 < 50000 and ns1 > ns0                     # an exchange round costs hundreds of nanoseconds, more with data
     # and the handle still works afterwards
     import numpy as np
     src = np.arange(4, 12, dtype=np.int32)[None]
