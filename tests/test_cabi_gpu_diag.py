@@ -1,4 +1,4 @@
-"""The library's diagnostics entry points answer with plausible numbers (they back statements in the design notes)."""
+"""The library's diagnostics entry points answer with plausible numbers."""
 import pytest
 
 from paper_2203_16487_b200 import workloads as W
