@@ -160,13 +160,36 @@ __global__ void k_verify_prep_embed(Session s, const int* __restrict__ draft, in
         x[(size_t)i * d + e] = scale * to_f(E[(size_t)t * d + e]) + P[(size_t)p * d + e];
 }
 
+// Embedding of the rows [r0, r0 + n) of the draft pass by the block that prepared them.
+template <typename T>
+__device__ __forceinline__ void embed_rows(const Rows& all, int r0, int n, const T* __restrict__ E, const float* __restrict__ P,
+                                           float* __restrict__ x, int d, float scale, int vocab, int max_pos) {
+    const int per_row = d / 4;                     // float4 pieces per row (d is a multiple of 16)
+    for (int i = threadIdx.x; i < n * per_row; i += blockDim.x) {
+        const int row = r0 + i / per_row, e = (i % per_row) * 4;
+        const int t = min(max(all.tok[row], 0), vocab - 1), p = min(max(all.pos[row], 0), max_pos - 1);
+        const T* ep = E + (size_t)t * d + e;
+        const float4 pv = *reinterpret_cast<const float4*>(P + (size_t)p * d + e);
+        float4 o;
+        o.x = scale * to_f(ep[0]) + pv.x; o.y = scale * to_f(ep[1]) + pv.y; o.z = scale * to_f(ep[2]) + pv.z; o.w = scale * to_f(ep[3]) + pv.w;
+        *reinterpret_cast<float4*>(x + (size_t)row * d + e) = o;
+    }
+}
+
 // Drafter: packed rows [BOS, committed, MASK x k] of every unfinished sequence.
 // `all` describes the full pass, `msk` the mask-only continuation of the last layer.
-// One block per sequence: it sums the row counts of the sequences before it (B loads spread over its threads: the
-// one-block version walked the batch serially, 106 us at 128 sequences), then fills its own rows.
-__global__ void k_draft_prep(Session s, int B, int k, int S_max, int bos, int mask, Rows all, Rows msk) {
+// gridDim.y blocks per sequence: each sums the row counts of the sequences before its own (B loads spread over its
+// threads: the one-block version walked the batch serially, 106 us at 128 sequences), then fills an equal slice of the
+// sequence's rows and embeds that slice (x = sqrt(d) E[tok] + P[pos]; one block per sequence made the embedding of a
+// 90-row pass a 26 us serial walk).  Every block completes its metadata before it lets the successors start, because
+// kernels further down the chain read it ahead of their dependency waits.
+template <typename T>
+__global__ void k_draft_prep(Session s, int B, int k, int S_max, int bos, int mask, Rows all, Rows msk,
+                             const T* __restrict__ E, const float* __restrict__ P, float* __restrict__ x, int d, float scale,
+                             int vocab, int max_pos) {
     __shared__ int red_a[32], red_m[32], tot_a[32], tot_l[32];
-    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
+    const int b = blockIdx.x, part = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
+    pdl_wait();                                    // session state comes from the previous step's commit
     int a = 0, m = 0, ta = 0, tl = 0;               // rows / mask rows of the sequences before b; rows / live sequences of the batch
     for (int o = tid; o < B; o += blockDim.x) {
         const int n = s.finished[o] ? 0 : s.len[o] + 1 + k;
@@ -184,7 +207,8 @@ __global__ void k_draft_prep(Session s, int B, int k, int S_max, int bos, int ma
     for (int w = 0; w < nw; ++w) { off += red_a[w]; moff += red_m[w]; total += tot_a[w]; live += tot_l[w]; }
     const bool fin = s.finished[b] != 0;
     const int j = s.len[b], n = fin ? 0 : j + 1 + k, sl = s.src_len[b];
-    if (tid == 0) {
+    const int chunk = (n + (int)gridDim.y - 1) / (int)gridDim.y, t0 = min(n, part * chunk), t1 = min(n, t0 + chunk);
+    if (tid == 0 && part == 0) {
         all.kv_off[b] = off; all.kv_off_cross[b] = b * S_max;
         msk.kv_off[b] = off; msk.kv_off_cross[b] = b * S_max;
         all.q_off[b] = off; all.q_cnt[b] = n;
@@ -194,8 +218,7 @@ __global__ void k_draft_prep(Session s, int B, int k, int S_max, int bos, int ma
             s.counters[CNT_DRAFT_MASK] = live * k;  // k mask rows per unfinished sequence
         }
     }
-    if (fin) return;
-    for (int t = tid; t < n; t += blockDim.x) {
+    for (int t = t0 + tid; t < t1; t += blockDim.x) {
         const int row = off + t;
         all.tok[row] = (t == 0) ? bos : (t <= j ? s.out[(size_t)b * s.out_stride + t - 1] : mask);
         all.pos[row] = t;
@@ -203,7 +226,7 @@ __global__ void k_draft_prep(Session s, int B, int k, int S_max, int bos, int ma
         all.nk_self[row] = n;            // no causal mask: every valid position
         all.nk_cross[row] = sl;
     }
-    for (int i = tid; i < k; i += blockDim.x) {
+    for (int i = tid; i < ((fin || part) ? 0 : k); i += blockDim.x) {
         const int row = moff + i;
         msk.seq[row] = b;
         msk.nk_self[row] = n;
@@ -211,6 +234,10 @@ __global__ void k_draft_prep(Session s, int B, int k, int S_max, int bos, int ma
         msk.src_row[row] = off + j + 1 + i;
         msk.slot[row] = b * k + i;
     }
+    __threadfence();
+    __syncthreads();
+    pdl_launch_dependents();
+    embed_rows<T>(all, off + t0, t1 - t0, E, P, x, d, scale, vocab, max_pos);
 }
 
 // Drafter, prefix-causal reading (the committed tokens attend causally among themselves and never see the [MASK]
@@ -218,10 +245,14 @@ __global__ void k_draft_prep(Session s, int B, int k, int S_max, int bos, int ma
 // every iteration, so its work should not grow with the prefix).  Rows of sequence b: the positions the cache does not
 // hold yet, c..j of [BOS, committed...], then k [MASK] rows at positions j+1..j+k.  Position p sees keys 0..p when it is
 // a prefix row and every key 0..j+k when it is a [MASK] row.  The last block to finish records the new cache length.
-__global__ void k_draft_prep_pc(Session s, int B, int k, int S_max, int bos, int mask, Rows all, Rows msk) {
+template <typename T>
+__global__ void k_draft_prep_pc(Session s, int B, int k, int S_max, int bos, int mask, Rows all, Rows msk,
+                                const T* __restrict__ E, const float* __restrict__ P, float* __restrict__ x, int d, float scale,
+                                int vocab, int max_pos) {
     __shared__ int red_a[32], red_m[32], tot_a[32], tot_l[32];
     __shared__ int last_s;
-    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
+    const int b = blockIdx.x, part = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
+    pdl_wait();                                    // session state comes from the previous step's commit
     int a = 0, m = 0, ta = 0, tl = 0;
     for (int o = tid; o < B; o += blockDim.x) {
         const int n = s.finished[o] ? 0 : (s.len[o] + 1 - min(s.dlen[o], s.len[o] + 1)) + k;
@@ -239,7 +270,8 @@ __global__ void k_draft_prep_pc(Session s, int B, int k, int S_max, int bos, int
     for (int w = 0; w < nw; ++w) { off += red_a[w]; moff += red_m[w]; total += tot_a[w]; live += tot_l[w]; }
     const bool fin = s.finished[b] != 0;
     const int j = s.len[b], c = min(s.dlen[b], j + 1), n_new = j + 1 - c, n = fin ? 0 : n_new + k, sl = s.src_len[b];
-    if (tid == 0) {
+    const int chunk = (n + (int)gridDim.y - 1) / (int)gridDim.y, t0 = min(n, part * chunk), t1 = min(n, t0 + chunk);
+    if (tid == 0 && part == 0) {
         all.kv_off[b] = off; all.kv_off_cross[b] = b * S_max;
         msk.kv_off[b] = off; msk.kv_off_cross[b] = b * S_max;
         all.q_off[b] = off; all.q_cnt[b] = n;
@@ -250,7 +282,7 @@ __global__ void k_draft_prep_pc(Session s, int B, int k, int S_max, int bos, int
         }
     }
     if (!fin) {
-        for (int t = tid; t < n; t += blockDim.x) {
+        for (int t = t0 + tid; t < t1; t += blockDim.x) {
             const int row = off + t, p = c + t;
             all.tok[row] = (t >= n_new) ? mask : (p == 0 ? bos : s.out[(size_t)b * s.out_stride + p - 1]);
             all.pos[row] = p;
@@ -258,7 +290,7 @@ __global__ void k_draft_prep_pc(Session s, int B, int k, int S_max, int bos, int
             all.nk_self[row] = (t >= n_new) ? j + 1 + k : p + 1;
             all.nk_cross[row] = sl;
         }
-        for (int i = tid; i < k; i += blockDim.x) {
+        for (int i = tid; i < (part ? 0 : k); i += blockDim.x) {
             const int row = moff + i;
             msk.seq[row] = b;
             msk.nk_self[row] = j + 1 + k;
@@ -271,7 +303,7 @@ __global__ void k_draft_prep_pc(Session s, int B, int k, int S_max, int bos, int
     __syncthreads();
     if (tid == 0) {
         __threadfence();
-        last_s = (atomicAdd(s.dticket, 1) == (int)gridDim.x - 1) ? 1 : 0;
+        last_s = (atomicAdd(s.dticket, 1) == (int)(gridDim.x * gridDim.y) - 1) ? 1 : 0;
     }
     __syncthreads();
     if (last_s) {
@@ -279,6 +311,10 @@ __global__ void k_draft_prep_pc(Session s, int B, int k, int S_max, int bos, int
             if (!s.finished[o]) s.dlen[o] = s.len[o] + 1;
         if (tid == 0) *s.dticket = 0;
     }
+    __threadfence();
+    __syncthreads();
+    pdl_launch_dependents();
+    embed_rows<T>(all, off + t0, t1 - t0, E, P, x, d, scale, vocab, max_pos);
 }
 
 // ------------------------------------------------------------------ embedding, gather, layer norm
@@ -888,8 +924,11 @@ __global__ void k_logit_tile_stats(const float* __restrict__ logits, const int* 
 }
 
 // ------------------------------------------------------------------ drafter argmax
+// script (optional; benchmark / test hook): draft i of a sequence with j committed tokens is replaced by
+// script[b * stride + j + i] wherever that entry is >= 0 (len = the committed lengths, k = drafts per sequence).
 __global__ void k_draft_argmax(const RowPart* __restrict__ part, int n_tiles, const int* __restrict__ n_rows,
-                               const int* __restrict__ slot, int* __restrict__ draft) {
+                               const int* __restrict__ slot, int* __restrict__ draft, const int* __restrict__ script,
+                               int stride, const int* __restrict__ len, int k) {
     int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     int lane = threadIdx.x & 31;
     pdl_launch_dependents();
@@ -917,7 +956,13 @@ __global__ void k_draft_argmax(const RowPart* __restrict__ part, int n_tiles, co
         int oa = __shfl_xor_sync(0xffffffffu, arg, o);
         if (om > mx || (om == mx && oa < arg)) { mx = om; arg = oa; }
     }
-    if (lane == 0) draft[slot_of_row] = arg;
+    if (lane == 0) {
+        if (script) {
+            const int b = slot_of_row / k, pos = len[b] + slot_of_row % k;
+            if (pos < stride) { const int t2 = script[(size_t)b * stride + pos]; if (t2 >= 0) arg = t2; }
+        }
+        draft[slot_of_row] = arg;
+    }
 }
 
 // Scripted drafts (benchmark / test hook): draft i of a sequence with j committed tokens is

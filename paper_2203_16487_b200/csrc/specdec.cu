@@ -851,10 +851,15 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
     // prefix positions its K/V cache does not hold yet plus the k [MASK] rows
     const int per_seq = pc ? std::min(h->dnew_ub, len_ub + 1) + k : len_ub + 1 + k;
     const int R1 = B * per_seq, R2 = B * k, max_keys = len_ub + 1 + k;
-    if (pc) k_draft_prep_pc<<<B, 128, 0, st>>>(h->ses, B, k, h->S_max, h->cfg.bos_id, h->cfg.mask_id, h->rows, h->mrows);
-    else k_draft_prep<<<B, 128, 0, st>>>(h->ses, B, k, h->S_max, h->cfg.bos_id, h->cfg.mask_id, h->rows, h->mrows);
+    // row metadata of the pass and the embedding of its rows in one kernel (one block per sequence)
+    h->fused_x = nullptr;
+    // blocks per sequence: enough to fill the machine at small batches, never fewer than two rows a block
+    const int parts = std::max(1, std::min(cdiv(592, B), cdiv(h->T_cap + k + 1, 2)));
+    if (pc) CUDA_TRY(h, launch_pdl(h, k_draft_prep_pc<T>, dim3(B, parts), dim3(128), 0, st, h->ses, B, k, h->S_max, h->cfg.bos_id, h->cfg.mask_id, h->rows, h->mrows,
+                                   (const T*)m.embed, (const float*)m.pos_dec, h->x, d, sqrtf((float)d), m.dm.vocab, m.dm.max_pos));
+    else CUDA_TRY(h, launch_pdl(h, k_draft_prep<T>, dim3(B, parts), dim3(128), 0, st, h->ses, B, k, h->S_max, h->cfg.bos_id, h->cfg.mask_id, h->rows, h->mrows,
+                                (const T*)m.embed, (const float*)m.pos_dec, h->x, d, sqrtf((float)d), m.dm.vocab, m.dm.max_pos));
     KCHECK(h);
-    TRY(embed<T>(h, m, h->rows, m.pos_dec, CNT_DRAFT_ALL, R1, st));
     for (int l = 0; l + 1 < L; ++l) {
         TRY(block_self<T>(h, m, m.dec[l], h->x, h->rows, CNT_DRAFT_ALL, R1, per_seq, pc ? h->dkc[l] : nullptr, pc ? h->dvc[l] : nullptr, nullptr,
                           max_keys, st, m.dec[l].lnc_g, m.dec[l].lnc_b));
@@ -896,12 +901,9 @@ int draft_impl(specdec_handle* h, int k, int* d_draft, cudaStream_t st) {
     TRY(gemm<T>(h, EPI_STATS, h->y, d, m.embed, nullptr, m.dm.vocab, d, CNT_DRAFT_MASK, R2, nullptr, 0, nullptr, st,
                 nullptr, nullptr, &n_tiles));
     CUDA_TRY(h, launch_pdl(h, k_draft_argmax, dim3(cdiv(R2, 4)), dim3(128), 0, st, (const RowPart*)h->part, n_tiles,
-                           (const int*)(h->ses.counters + CNT_DRAFT_MASK), (const int*)h->mrows.slot, d_draft));
+                           (const int*)(h->ses.counters + CNT_DRAFT_MASK), (const int*)h->mrows.slot, d_draft,
+                           (const int*)(h->script_on ? h->script : nullptr), h->T_cap + h->k_cap, (const int*)h->ses.len, k));
     KCHECK(h);
-    if (h->script_on) {
-        CUDA_TRY(h, launch_pdl(h, k_apply_script, dim3(cdiv(B * k, 256)), dim3(256), 0, st, h->ses, (const int*)h->script, h->T_cap + h->k_cap, B, k, d_draft));
-        KCHECK(h);
-    }
     h->drafted = true; h->verified = false;
     h->last_draft_rows_ub = R2;
     h->dnew_ub = 0;                                  // the cache now holds every committed position
