@@ -44,6 +44,8 @@ extern "C" {
                                           handle that finds it set returns this code and clears it.  The handle stays
                                           usable: start over with specdec_encode                                      */
 #define SPECDEC_ERR_UNSUPPORTED   -7
+#define SPECDEC_ERR_CORRUPT       -8   /* an integrity check (option "debug_checks") found a damaged red zone behind an
+                                          arena block or a non-finite activation; specdec_last_error names it        */
 
 #define SPECDEC_DTYPE_F32   0
 #define SPECDEC_DTYPE_BF16  1
@@ -201,6 +203,24 @@ int specdec_debug_row_stats(specdec_handle* h, float* d_stats, void* stream);
  * 256-entry device array; this copies the first n (<= 256) entries to the host.  Synchronises the device. */
 int specdec_debug_trace(specdec_handle* h, long long* h_out, int n);
 
+/* Integrity check (debugging aid; the paper has no counterpart).  The handle's device arena places a 256-byte red
+ * zone with a fixed pattern behind every block it hands out (weights, activations, caches, row metadata, session
+ * state), so a kernel that writes past the end of its buffer damages one.  This call checks every red zone and scans
+ * the activation buffers, the encoder memories and the K/V caches for NaN / Inf, on `stream`, and synchronises it.
+ * It returns SPECDEC_OK whenever the check itself ran; the findings are in *out (first_* are -1 when the count is 0;
+ * buffers are numbered in the order: residual rows, mask rows, normalised rows, QKV rows, attention output, cross
+ * query rows, feed-forward rows, encoder memory, the second encoder's six buffers, K caches, V caches, the drafter's
+ * caches, cross K/V of the verifier and of the drafter).  With option "debug_checks" = 1 every encode / draft / verify /
+ * commit / generate call runs it before returning and fails with SPECDEC_ERR_CORRUPT on a finding. */
+typedef struct specdec_integrity {
+    int32_t zones;                   /* red zones checked                                  */
+    int32_t damaged_zones;
+    int32_t first_damaged_zone;      /* index (allocation order) of the first damaged one  */
+    int32_t first_nonfinite_buffer;
+    int64_t nonfinite;               /* NaN / Inf values found                             */
+} specdec_integrity;
+int specdec_debug_integrity(specdec_handle* h, specdec_integrity* out, void* stream);
+
 /* Diagnostics: the cost of one kernel boundary inside a step.  Replays (from a CUDA graph, on the handle's own stream)
  * a chain of n_links launches of `grid` CTAs, each of which waits for its predecessor (programmatic dependent
  * launch, as between the kernels of a step), reads the word it wrote and writes it back; returns the best of ten
@@ -265,6 +285,9 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
  * "diag_repeat"  bit mask: launch every attention (1), LayerNorm (2), non-residual GEMM (4), vocabulary kernel (8)
  *                twice in a row (same result), so the step time rises by that class's cost inside the pipeline
  * "trace"        see specdec_debug_trace
+ * "debug_checks" 0/1 see specdec_debug_integrity (default 0: the check synchronises)
+ * "poke_zone" i / "heal_zones" / "poke_nan" 0|1: test hooks for that check -- damage red zone i from the host, restore
+ *                every red zone, put a NaN (or a zero) into the last element of the attention-output buffer
  * "inject_error" code: test hook -- the next specdec_verify / specdec_generate finds this code in the device error
  *                word, as if a bounded device-side wait had given up (no kernel waits, nothing faults) */
 int specdec_set_option(specdec_handle* h, const char* name, int value);

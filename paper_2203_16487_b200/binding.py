@@ -25,6 +25,7 @@ EXPORTS = [
     "specdec_accept_scan", "specdec_debug_logits", "specdec_debug_row_stats", "specdec_set_option",
     "specdec_launch_count", "specdec_last_error", "specdec_set_draft_script", "specdec_profile_read",
     "specdec_accept_scan_static", "specdec_debug_trace", "specdec_debug_link_cost", "specdec_debug_mma_rate", "specdec_debug_cluster_round",
+    "specdec_debug_integrity",
 ]
 
 
@@ -37,6 +38,11 @@ class Config(C.Structure):
     _fields_ = [("verifier", ModelDims), ("drafter", ModelDims)] + [(n, C.c_int) for n in (
         "k_max", "max_batch", "max_src", "max_tgt", "page_tokens",
         "pad_id", "bos_id", "eos_id", "mask_id", "compute_dtype", "ffn_activation")]
+
+
+class Integrity(C.Structure):
+    _fields_ = [("zones", C.c_int32), ("damaged_zones", C.c_int32), ("first_damaged_zone", C.c_int32),
+                ("first_nonfinite_buffer", C.c_int32), ("nonfinite", C.c_int64)]
 
 
 class Tensor(C.Structure):
@@ -154,6 +160,8 @@ class SpecDec:
         self._h = h
         del keep
         self.B = 0
+        if os.environ.get("SPECDEC_DEBUG_CHECKS") == "1":        # every step call ends with the integrity check
+            self.set_option("debug_checks", 1)
         self._bufs = {}
 
     # ------------------------------------------------------------------ helpers
@@ -211,6 +219,12 @@ class SpecDec:
         ns = C.c_double()
         self._check(self._lib.specdec_debug_cluster_round(self._h, cluster_size, bytes_per_peer, rounds, C.byref(ns)))
         return ns.value
+
+    def integrity(self) -> dict:
+        """Red zones behind every arena block and a NaN / Inf scan of activations and caches (synchronises)."""
+        rep = Integrity()
+        self._check(self._lib.specdec_debug_integrity(self._h, C.byref(rep), _stream()))
+        return {n: int(getattr(rep, n)) for n, _ in Integrity._fields_}
 
     def trace(self, n: int):
         buf = (C.c_longlong * n)()

@@ -1025,6 +1025,48 @@ __global__ void k_copy_out(Session s, int B, int* __restrict__ out, int out_stri
     if (threadIdx.x == 0) { if (out_len) out_len[b] = n; if (fin) fin[b] = s.finished[b]; }
 }
 
+// ------------------------------------------------------------------ integrity checks (debugging aid)
+// Every arena allocation is followed by a 256-byte red zone holding a fixed pattern; a kernel that writes past the end
+// of its buffer damages one.  One warp per zone: report[0] += damaged zones, report[1] = lowest damaged zone index.
+constexpr unsigned long long RED_PATTERN = 0xC5A5C5A5C5A5C5A5ull;
+__global__ void k_red_fill(unsigned char* base, const unsigned long long* __restrict__ zone_off, int n_zones) {
+    const int z = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (z < n_zones) reinterpret_cast<unsigned long long*>(base + zone_off[z])[lane] = RED_PATTERN;
+}
+__global__ void k_red_check(const unsigned char* base, const unsigned long long* __restrict__ zone_off, int n_zones,
+                            unsigned long long* report) {
+    const int z = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (z >= n_zones) return;
+    const bool bad = reinterpret_cast<const unsigned long long*>(base + zone_off[z])[lane] != RED_PATTERN;
+    if (__any_sync(0xffffffffu, bad) && lane == 0) {
+        atomicAdd(report, 1ull);
+        atomicMin(report + 1, (unsigned long long)z);
+    }
+}
+// Non-finite values (NaN, +-Inf) in activation buffers and caches: blockIdx.y = buffer, blockIdx.x strides over its
+// 16-byte pieces.  report[2] += count, report[3] = lowest buffer index holding one.
+struct ScanBuf { const void* p; unsigned long long n16; int f32; int pad; };   // n16 = whole 16-byte pieces
+__global__ void k_nonfinite_scan(const ScanBuf* __restrict__ bufs, unsigned long long* report) {
+    const ScanBuf b = bufs[blockIdx.y];
+    const uint4* p = reinterpret_cast<const uint4*>(b.p);
+    int cnt = 0;
+    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < b.n16; i += (unsigned long long)gridDim.x * blockDim.x) {
+        const uint4 v = p[i];
+        const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (b.f32) cnt += ((w[j] & 0x7F800000u) == 0x7F800000u) ? 1 : 0;
+            else cnt += (((w[j] & 0x7F80u) == 0x7F80u) ? 1 : 0) + (((w[j] & 0x7F800000u) == 0x7F800000u) ? 1 : 0);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    if ((threadIdx.x & 31) == 0 && cnt) {
+        atomicAdd(report + 2, (unsigned long long)cnt);
+        atomicMin(report + 3, (unsigned long long)blockIdx.y);
+    }
+}
+
 // ------------------------------------------------------------------ weight repacking
 template <typename T>
 __global__ void k_convert(const float* __restrict__ in, T* __restrict__ out, size_t n) {

@@ -49,13 +49,17 @@ struct ModelW {
     int ckv_stride = 0;
 };
 
+// Bump allocator over one device allocation.  Every block is followed by a 256-byte red zone (see k_red_check).
 struct Arena {
     char* base = nullptr;
     size_t off = 0;
+    std::vector<unsigned long long> zones;         // byte offsets of the red zones, in allocation order
     void* take(size_t n) {
         off = (off + 255) & ~size_t(255);
         void* p = base ? base + off : nullptr;
-        off += n;
+        off = (off + n + 255) & ~size_t(255);
+        zones.push_back(off);
+        off += 256;
         return p;
     }
 };
@@ -113,6 +117,11 @@ struct specdec_handle {
     struct NextLn { const float* g; const float* b; void* out; };
     NextLn next_ln = {nullptr, nullptr, nullptr};
     const float* fused_x = nullptr; const float* fused_g = nullptr; const void* fused_out = nullptr;
+    // integrity checks (option "debug_checks", specdec_debug_integrity)
+    unsigned long long* integ_report = nullptr; ScanBuf* integ_bufs = nullptr; unsigned long long* zone_tab = nullptr;
+    int zone_cap = 0, n_zones = 0, n_scan = 0;
+    std::vector<std::string> scan_names;
+    int debug_checks = 0;
     int use_ln_fuse = 0;            // option "ln_fuse": measured slower than the separate LayerNorm launch, kept for comparison
     int use_sk_cluster = 1;         // option "sk_cluster": 1 = LayerNorm-fused weight-streaming GEMMs share the normalised rows in clusters of 8; 2 = the plain ones too (measured slower)
     bool splitk_ready = false;
@@ -258,6 +267,7 @@ void layout_rows(Arena& A, Rows& r, int n, int B) {
 void layout_all(specdec_handle* h) {
     Arena& A = h->arena;
     A.off = 0;
+    A.zones.clear();
     const size_t e = h->esz;
     layout_model(h, h->ver, h->cfg.verifier);
     layout_model(h, h->dra, h->cfg.drafter);
@@ -314,6 +324,10 @@ void layout_all(specdec_handle* h) {
     s.dticket = (int*)A.take(4);
     s.counters = (int*)A.take(8 * 4);
     s.stats = (unsigned long long*)A.take(4 * 8);
+    // integrity checks: report words, the table of scanned buffers, the table of red-zone offsets (sized by the dry run)
+    h->integ_report = (unsigned long long*)A.take(4 * 8);
+    h->integ_bufs = (ScanBuf*)A.take(128 * sizeof(ScanBuf));
+    h->zone_tab = (unsigned long long*)A.take((size_t)h->zone_cap * 8);
 }
 
 // ---------------------------------------------------------------- weight loading
@@ -568,6 +582,7 @@ int gemm_once(specdec_handle* h, int epi, const void* A, int lda, const void* W,
                          ? sd::gemm_tc_pair_launch(h->tma, epi, g, rows_ub, st, n_tiles_out)
                          : sd::gemm_tc_launch(h->tma, epi, g, rows_ub, st, n_tiles_out);
             if (rc != 0) return fail(h, SPECDEC_ERR_CUDA, "tensor-core GEMM launch failed: " + h->tma.err);
+            if (epi == EPI_STATS && g.n_tiles > h->n_tiles_cap) return fail(h, SPECDEC_ERR_CAPACITY, "row statistics: more vocabulary tiles than the table holds");
             ++h->launches;
             return 0;
         }
@@ -1313,6 +1328,38 @@ int check_model(const specdec_model_dims& m, const char* who, std::string& why) 
 }  // namespace
 
 // ================================================================== C ABI
+// Red zones and non-finite scan on `st`; synchronises.  Returns SPECDEC_OK with the report filled in.
+int integrity_run(specdec_handle* h, cudaStream_t st, specdec_integrity* rep) {
+    const unsigned long long init[4] = {0ull, ~0ull, 0ull, ~0ull};
+    CUDA_TRY(h, cudaMemcpyAsync(h->integ_report, init, sizeof(init), cudaMemcpyHostToDevice, st));
+    k_red_check<<<cdiv(h->n_zones, 8), 256, 0, st>>>((const unsigned char*)h->arena.base, h->zone_tab, h->n_zones, h->integ_report);
+    if (h->n_scan > 0) k_nonfinite_scan<<<dim3(2 * h->tma.n_sm, h->n_scan), 256, 0, st>>>(h->integ_bufs, h->integ_report);
+    KCHECK(h);
+    unsigned long long out[4];
+    CUDA_TRY(h, cudaMemcpyAsync(out, h->integ_report, sizeof(out), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(h, cudaStreamSynchronize(st));
+    rep->zones = h->n_zones;
+    rep->damaged_zones = (int)out[0];
+    rep->first_damaged_zone = out[0] ? (int)out[1] : -1;
+    rep->nonfinite = (long long)out[2];
+    rep->first_nonfinite_buffer = out[2] ? (int)out[3] : -1;
+    return SPECDEC_OK;
+}
+
+// With option "debug_checks" every step call ends with the integrity check and fails when it finds something.
+int post_check(specdec_handle* h, int rc, void* stream) {
+    if (rc != SPECDEC_OK || !h || !h->debug_checks) return rc;
+    specdec_integrity rep;
+    TRY(integrity_run(h, (cudaStream_t)stream, &rep));
+    if (rep.damaged_zones)
+        return fail(h, SPECDEC_ERR_CORRUPT, "integrity: " + std::to_string(rep.damaged_zones) + " damaged red zone(s), first behind arena block " +
+                                                std::to_string(rep.first_damaged_zone));
+    if (rep.nonfinite)
+        return fail(h, SPECDEC_ERR_CORRUPT, "integrity: " + std::to_string(rep.nonfinite) + " non-finite value(s), first in " +
+                                                h->scan_names[rep.first_nonfinite_buffer]);
+    return SPECDEC_OK;
+}
+
 extern "C" {
 
 const char* specdec_last_error(const specdec_handle* h) { return h ? h->err.c_str() : g_create_error.c_str(); }
@@ -1356,8 +1403,12 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
     h->R2_cap = h->B_cap * h->k_cap;
     h->R_cap = std::max(std::max(h->B_cap * h->S_cap, h->B_cap * (h->T_cap + 1 + h->k_cap)), h->M_cap);
     h->pages_per_seq = cdiv(h->T_cap + h->k_cap + 1, cfg->page_tokens);
-    h->n_tiles_cap = cdiv(h->v_max, 64);
-    layout_all(h);                       // dry run: sizes only
+    // partial row statistics per vocabulary tile: 64-column tiles on the SIMT path, two column halves per 128- to 256-wide
+    // tile on the tensor-core path (2 * ceil(V / 128) exceeds ceil(V / 64) when V mod 128 is in 1..64)
+    h->n_tiles_cap = std::max(cdiv(h->v_max, 64), 2 * cdiv(h->v_max, 128));
+    layout_all(h);                       // dry runs: the number of red zones, then the sizes
+    h->zone_cap = (int)h->arena.zones.size();
+    layout_all(h);
     const size_t total = h->arena.off + 256;
     char* base = nullptr;
     cudaError_t ce = cudaMalloc((void**)&base, total);
@@ -1369,6 +1420,36 @@ int specdec_create(const specdec_config* cfg, const specdec_tensor* weights, int
     h->arena.base = base;
     layout_all(h);
     cudaMemsetAsync(base, 0, total, st);          // dead rows of every buffer read as zeros, never as NaN patterns
+    {   // red zones behind every block, and the table of buffers the non-finite scan walks
+        h->n_zones = (int)h->arena.zones.size();
+        cudaMemcpyAsync(h->zone_tab, h->arena.zones.data(), (size_t)h->n_zones * 8, cudaMemcpyHostToDevice, st);
+        k_red_fill<<<cdiv(h->n_zones, 8), 256, 0, st>>>((unsigned char*)base, h->zone_tab, h->n_zones);
+        std::vector<ScanBuf> sb;
+        auto add = [&](const char* name, const void* p, size_t bytes, bool f32) {
+            if (!p || bytes < 16 || sb.size() >= 128) return;
+            sb.push_back(ScanBuf{p, (unsigned long long)(bytes / 16), f32 ? 1 : 0, 0});
+            h->scan_names.push_back(name);
+        };
+        const size_t e = h->esz, R = h->R_cap, d = h->d_max, f = h->f_max, Re = (size_t)h->B_cap * h->S_cap;
+        const bool f32 = h->dtype != SPECDEC_DTYPE_BF16;
+        add("residual rows x", h->ws[0].x, R * d * 4, true); add("mask rows x2", h->x2, (size_t)h->R2_cap * d * 4, true);
+        add("normalised rows y", h->ws[0].y, R * d * e, f32); add("qkv rows", h->ws[0].qkv, R * 3 * d * e, f32);
+        add("attention output", h->ws[0].att, R * d * e, f32); add("cross query rows", h->ws[0].q, R * d * e, f32);
+        add("feed-forward rows", h->ws[0].hbuf, R * f * e, f32); add("encoder memory", h->ws[0].mem, Re * d * e, f32);
+        add("second encoder x", h->ws[1].x, Re * d * 4, true); add("second encoder y", h->ws[1].y, Re * d * e, f32);
+        add("second encoder qkv", h->ws[1].qkv, Re * 3 * d * e, f32); add("second encoder attention output", h->ws[1].att, Re * d * e, f32);
+        add("second encoder feed-forward rows", h->ws[1].hbuf, Re * f * e, f32); add("second encoder memory", h->ws[1].mem, Re * d * e, f32);
+        const size_t cache_rows = (size_t)h->B_cap * h->pages_per_seq * h->cfg.page_tokens;
+        for (auto p : h->kc) add("verifier K cache", p, cache_rows * h->cfg.verifier.d_model * e, f32);
+        for (auto p : h->vc) add("verifier V cache", p, cache_rows * h->cfg.verifier.d_model * e, f32);
+        for (auto p : h->dkc) add("drafter K cache", p, cache_rows * h->cfg.drafter.d_model * e, f32);
+        for (auto p : h->dvc) add("drafter V cache", p, cache_rows * h->cfg.drafter.d_model * e, f32);
+        add("verifier cross K/V", h->ver.ckv.empty() ? nullptr : h->ver.ckv[0], Re * h->ver.ckv_stride * e, f32);
+        add("drafter cross K/V", h->dra.ckv.empty() ? nullptr : h->dra.ckv[0], Re * h->dra.ckv_stride * e, f32);
+        h->n_scan = (int)sb.size();
+        cudaMemcpyAsync(h->integ_bufs, sb.data(), sb.size() * sizeof(ScanBuf), cudaMemcpyHostToDevice, st);
+        cudaStreamSynchronize(st);               // the host vectors go out of scope
+    }
     auto bail = [&](int code, const std::string& msg) { cudaFree(base); delete h; return fail(nullptr, code, msg); };
     Manifest mf;
     for (int i = 0; i < n_weights; ++i)
@@ -1513,6 +1594,24 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "sk_cluster")) { h->use_sk_cluster = value < 0 ? 0 : value; return SPECDEC_OK; }   // 0 off, 1 LayerNorm-fused kernels, 2 + plain ones with K <= 512, 3 all
     if (!strcmp(name, "ln_fuse")) { h->use_ln_fuse = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "debug_checks")) { h->debug_checks = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "poke_zone")) {                 // test hook: damage red zone `value` (an in-arena write from the host)
+        if (value < 0 || value >= h->n_zones) return fail(h, SPECDEC_ERR_INVALID_ARG, "poke_zone: no such red zone");
+        const unsigned int junk = 0xDEADBEEFu;
+        CUDA_TRY(h, cudaMemcpy(h->arena.base + h->arena.zones[value] + 100, &junk, 4, cudaMemcpyHostToDevice));
+        return SPECDEC_OK;
+    }
+    if (!strcmp(name, "heal_zones")) {                // test hook: restore every red zone
+        k_red_fill<<<cdiv(h->n_zones, 8), 256>>>((unsigned char*)h->arena.base, h->zone_tab, h->n_zones);
+        CUDA_TRY(h, cudaDeviceSynchronize());
+        return SPECDEC_OK;
+    }
+    if (!strcmp(name, "poke_nan")) {                  // test hook: a NaN (1) or a zero (0) in the last element of the attention-output buffer (a row no pass reaches)
+        const unsigned int word = value ? 0x7FC00000u : 0u;      // bf16: the upper half is the last element
+        char* end = (char*)h->ws[0].att + (size_t)h->R_cap * h->d_max * h->esz;
+        CUDA_TRY(h, cudaMemcpy(end - 4, &word, 4, cudaMemcpyHostToDevice));
+        return SPECDEC_OK;
+    }
     if (!strcmp(name, "pair")) {
         if (value && !h->pair_ready) return fail(h, SPECDEC_ERR_UNSUPPORTED, "two-SM GEMM tiles are not available on this handle");
         h->use_pair = value ? 1 : 0; return SPECDEC_OK;
@@ -1537,8 +1636,8 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
 
 #define DISPATCH(h, call_bf16, call_f32) ((h)->dtype == SPECDEC_DTYPE_BF16 ? (call_bf16) : (call_f32))
 
-int specdec_encode(specdec_handle* h, const int32_t* d_src, const int32_t* d_src_len, const int32_t* d_max_tgt, int B,
-                   int S_max, void* stream) {
+static int encode_entry(specdec_handle* h, const int32_t* d_src, const int32_t* d_src_len, const int32_t* d_max_tgt, int B,
+                        int S_max, void* stream) {
     if (!h) return SPECDEC_ERR_INVALID_ARG;
     if (!d_src || !d_src_len || B < 1 || S_max < 1) return fail(h, SPECDEC_ERR_INVALID_ARG, "encode: bad argument");
     if (B > h->B_cap || S_max > h->S_cap) return fail(h, SPECDEC_ERR_CAPACITY, "encode: B or S_max beyond capacity");
@@ -1549,7 +1648,7 @@ int specdec_encode(specdec_handle* h, const int32_t* d_src, const int32_t* d_src
                     encode_staged<float>(h, d_src, d_src_len, d_max_tgt, B, S_max, st));
 }
 
-int specdec_draft(specdec_handle* h, int k, int32_t* d_draft, void* stream) {
+static int draft_entry(specdec_handle* h, int k, int32_t* d_draft, void* stream) {
     if (!h) return SPECDEC_ERR_INVALID_ARG;
     if (!h->encoded) return fail(h, SPECDEC_ERR_NOT_ENCODED, "draft: no session (call specdec_encode)");
     if (!d_draft) return fail(h, SPECDEC_ERR_INVALID_ARG, "draft: null output");
@@ -1571,7 +1670,7 @@ int specdec_draft(specdec_handle* h, int k, int32_t* d_draft, void* stream) {
     return DISPATCH(h, draft_impl<bf16>(h, k, d_draft, st), draft_impl<float>(h, k, d_draft, st));
 }
 
-int specdec_verify(specdec_handle* h, const int32_t* d_draft, int k, int beta, float tau, int32_t* d_accepted,
+static int verify_entry(specdec_handle* h, const int32_t* d_draft, int k, int beta, float tau, int32_t* d_accepted,
                    int32_t* d_bif, void* stream) {
     if (!h) return SPECDEC_ERR_INVALID_ARG;
     if (!h->encoded) return fail(h, SPECDEC_ERR_NOT_ENCODED, "verify: no session (call specdec_encode)");
@@ -1597,7 +1696,7 @@ int specdec_verify(specdec_handle* h, const int32_t* d_draft, int k, int beta, f
                     verify_impl<float>(h, d_draft, k, beta, tau, d_accepted, d_bif, st));
 }
 
-int specdec_commit(specdec_handle* h, const int32_t* d_keep, const int32_t* d_next, void* stream) {
+static int commit_entry(specdec_handle* h, const int32_t* d_keep, const int32_t* d_next, void* stream) {
     if (!h) return SPECDEC_ERR_INVALID_ARG;
     if (!h->encoded) return fail(h, SPECDEC_ERR_NOT_ENCODED, "commit: no session (call specdec_encode)");
     if (!h->verified) return fail(h, SPECDEC_ERR_INVALID_ARG, "commit: must follow specdec_verify");
@@ -1621,7 +1720,7 @@ int specdec_get_output(specdec_handle* h, int32_t* d_out, int out_stride, int32_
     return SPECDEC_OK;
 }
 
-int specdec_generate(specdec_handle* h, const int32_t* d_src, const int32_t* d_src_len, const int32_t* d_max_tgt, int B,
+static int generate_entry(specdec_handle* h, const int32_t* d_src, const int32_t* d_src_len, const int32_t* d_max_tgt, int B,
                      int S_max, int k, int beta, float tau, int32_t* d_out, int out_stride, int32_t* d_out_len,
                      specdec_stats* h_stats, void* stream) {
     if (!h) return SPECDEC_ERR_INVALID_ARG;
@@ -1638,7 +1737,7 @@ int specdec_generate(specdec_handle* h, const int32_t* d_src, const int32_t* d_s
     return rc;
 }
 
-int specdec_generate_host(specdec_handle* h, const int32_t* h_src, const int32_t* h_src_len, const int32_t* h_max_tgt,
+static int generate_host_entry(specdec_handle* h, const int32_t* h_src, const int32_t* h_src_len, const int32_t* h_max_tgt,
                           int B, int S_max, int k, int beta, float tau, int32_t* h_out, int out_stride,
                           int32_t* h_out_len, specdec_stats* h_stats, void* stream) {
     if (!h) return SPECDEC_ERR_INVALID_ARG;
@@ -1847,6 +1946,35 @@ int specdec_debug_row_stats(specdec_handle* h, float* d_stats, void* stream) {
     CUDA_TRY(h, cudaMemcpyAsync(d_stats, h->row_stats, (size_t)h->B * (h->last_k + 1) * 6 * 4, cudaMemcpyDeviceToDevice,
                                 scope.st));
     return SPECDEC_OK;
+}
+
+// Public step calls: the entry proper, then (option "debug_checks") the integrity check.
+int specdec_encode(specdec_handle* h, const int32_t* d_src, const int32_t* d_src_len, const int32_t* d_max_tgt, int B,
+                   int S_max, void* stream) {
+    return post_check(h, encode_entry(h, d_src, d_src_len, d_max_tgt, B, S_max, stream), stream);
+}
+int specdec_draft(specdec_handle* h, int k, int32_t* d_draft, void* stream) { return post_check(h, draft_entry(h, k, d_draft, stream), stream); }
+int specdec_verify(specdec_handle* h, const int32_t* d_draft, int k, int beta, float tau, int32_t* d_accepted,
+                   int32_t* d_bif, void* stream) {
+    return post_check(h, verify_entry(h, d_draft, k, beta, tau, d_accepted, d_bif, stream), stream);
+}
+int specdec_commit(specdec_handle* h, const int32_t* d_keep, const int32_t* d_next, void* stream) {
+    return post_check(h, commit_entry(h, d_keep, d_next, stream), stream);
+}
+int specdec_generate(specdec_handle* h, const int32_t* d_src, const int32_t* d_src_len, const int32_t* d_max_tgt, int B,
+                     int S_max, int k, int beta, float tau, int32_t* d_out, int out_stride, int32_t* d_out_len,
+                     specdec_stats* h_stats, void* stream) {
+    return post_check(h, generate_entry(h, d_src, d_src_len, d_max_tgt, B, S_max, k, beta, tau, d_out, out_stride, d_out_len, h_stats, stream), stream);
+}
+int specdec_generate_host(specdec_handle* h, const int32_t* h_src, const int32_t* h_src_len, const int32_t* h_max_tgt,
+                          int B, int S_max, int k, int beta, float tau, int32_t* h_out, int out_stride,
+                          int32_t* h_out_len, specdec_stats* h_stats, void* stream) {
+    return post_check(h, generate_host_entry(h, h_src, h_src_len, h_max_tgt, B, S_max, k, beta, tau, h_out, out_stride, h_out_len, h_stats, stream), stream);
+}
+
+int specdec_debug_integrity(specdec_handle* h, specdec_integrity* out, void* stream) {
+    if (!h || !out) return SPECDEC_ERR_INVALID_ARG;
+    return integrity_run(h, (cudaStream_t)stream, out);
 }
 
 }  // extern "C"

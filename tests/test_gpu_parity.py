@@ -557,3 +557,40 @@ def test_prefix_causal_drafter_base_shapes_generate():
         ref, _ = O.specdec_generate(mv, md, wl.src[b], wl.max_tgt[b], 25, 3, 1.0, BOS, EOS, MASK, drafter_reading="prefix_causal")
         assert out[b, :int(n[b])].cpu().tolist() == ref
     sd.close()
+
+
+def test_integrity_checks_find_a_damaged_red_zone_and_a_nan(tiny):
+    """The arena's red zones and the non-finite scan: clean after real work; a red zone damaged from the host (an
+    in-arena write: nothing faults) and a NaN placed in an activation buffer are found, named, and -- with option
+    debug_checks -- fail the next step call with SPECDEC_ERR_CORRUPT; the handle works again once they are repaired."""
+    wl, wv, wd, mv, md = tiny
+    sd = _handle(wl.verifier, wv, wl.drafter, wd, False, k_max=wl.k)
+    src, lens = W.pad_batch(wl.src)
+    want = sd.generate(src, lens, np.array(wl.max_tgt, np.int32), wl.k, wl.beta, wl.tau)[0].cpu().numpy()
+    rep = sd.integrity()
+    assert rep["zones"] > 100 and rep["damaged_zones"] == 0 and rep["first_damaged_zone"] == -1, rep
+    assert rep["nonfinite"] == 0 and rep["first_nonfinite_buffer"] == -1, rep
+    sd.set_option("debug_checks", 1)
+    got = sd.generate(src, lens, np.array(wl.max_tgt, np.int32), wl.k, wl.beta, wl.tau)[0].cpu().numpy()
+    assert (got == want).all()
+    # a damaged red zone
+    sd.set_option("poke_zone", 7)
+    rep = sd.integrity()
+    assert rep["damaged_zones"] == 1 and rep["first_damaged_zone"] == 7, rep
+    b = _binding()
+    with pytest.raises(b.SpecDecError) as ei:
+        sd.generate(src, lens, np.array(wl.max_tgt, np.int32), wl.k, wl.beta, wl.tau)
+    assert ei.value.code == -8 and "red zone" in str(ei.value) and "block 7" in str(ei.value), str(ei.value)
+    sd.set_option("heal_zones", 1)
+    assert sd.integrity()["damaged_zones"] == 0
+    # a NaN in the attention-output buffer (buffer 4 of the scan), in a row no pass of this test reaches
+    sd.set_option("poke_nan", 1)
+    rep = sd.integrity()
+    assert rep["nonfinite"] == 1 and rep["first_nonfinite_buffer"] == 4, rep
+    with pytest.raises(b.SpecDecError) as ei:
+        sd.generate(src, lens, np.array(wl.max_tgt, np.int32), wl.k, wl.beta, wl.tau)
+    assert ei.value.code == -8 and "attention output" in str(ei.value), str(ei.value)
+    sd.set_option("poke_nan", 0)
+    got = sd.generate(src, lens, np.array(wl.max_tgt, np.int32), wl.k, wl.beta, wl.tau)[0].cpu().numpy()
+    assert (got == want).all()
+    sd.close()
