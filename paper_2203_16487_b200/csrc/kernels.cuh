@@ -346,7 +346,7 @@ __global__ void k_gather_rows(const float* __restrict__ x, const int* __restrict
 // fetched by the caller before the dependency wait (they are weights).
 template <typename T, int NC>
 __device__ __forceinline__ void ln_row_regs(const float* __restrict__ xr, const float4* gm, const float4* bt,
-                                            T* __restrict__ y, int row, int d, float eps, int lane) {
+                                            T* __restrict__ y, int row, int d, float eps, int lane, bool store = true) {
     float4 v[NC];
 #pragma unroll
     for (int c = 0; c < NC; ++c) {
@@ -368,12 +368,16 @@ __device__ __forceinline__ void ln_row_regs(const float* __restrict__ xr, const 
 #pragma unroll
     for (int c = 0; c < NC; ++c) {
         const int e = lane * 4 + c * 128;
-        if (e < d) {
+        if (e < d && store) {
             T* o = y + (size_t)row * d + e;
-            o[0] = from_f<T>((v[c].x - mu) * rstd * gm[c].x + bt[c].x);
-            o[1] = from_f<T>((v[c].y - mu) * rstd * gm[c].y + bt[c].y);
-            o[2] = from_f<T>((v[c].z - mu) * rstd * gm[c].z + bt[c].z);
-            o[3] = from_f<T>((v[c].w - mu) * rstd * gm[c].w + bt[c].w);
+            const float r0 = (v[c].x - mu) * rstd * gm[c].x + bt[c].x, r1 = (v[c].y - mu) * rstd * gm[c].y + bt[c].y;
+            const float r2 = (v[c].z - mu) * rstd * gm[c].z + bt[c].z, r3 = (v[c].w - mu) * rstd * gm[c].w + bt[c].w;
+            if constexpr (sizeof(T) == 2) {          // bf16: one 8-byte store per lane and chunk
+                __nv_bfloat162 p0 = __floats2bfloat162_rn(r0, r1), p1 = __floats2bfloat162_rn(r2, r3);
+                *reinterpret_cast<uint2*>(o) = make_uint2(*reinterpret_cast<uint32_t*>(&p0), *reinterpret_cast<uint32_t*>(&p1));
+            } else {
+                *reinterpret_cast<float4*>(o) = make_float4(r0, r1, r2, r3);
+            }
         }
     }
 }
@@ -382,7 +386,8 @@ __device__ __forceinline__ void ln_row_regs(const float* __restrict__ xr, const 
 // (a multiple of 128) are held in registers, so the row is read from memory once.
 template <typename T>
 __global__ void k_layernorm(const float* __restrict__ x, const float* __restrict__ g, const float* __restrict__ b,
-                            const int* __restrict__ n_rows, T* __restrict__ y, int d, float eps) {
+                            const int* __restrict__ n_rows, T* __restrict__ y, int d, float eps, int rows_static) {
+    // rows_static >= 0: the row count is known on the host (saves the dependent load of n_rows in front of the row's own)
     int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     int lane = threadIdx.x & 31;
     const bool regs4 = d % 128 == 0 && d <= 512, regs8 = d % 128 == 0 && d <= 1024;
@@ -399,7 +404,7 @@ __global__ void k_layernorm(const float* __restrict__ x, const float* __restrict
     }
     pdl_launch_dependents();
     pdl_wait();
-    if (row >= *n_rows) return;
+    if (row >= (rows_static >= 0 ? rows_static : *n_rows)) return;
     const float* xr = x + (size_t)row * d;
     if (regs4) { ln_row_regs<T, 4>(xr, gm, bt, y, row, d, eps, lane); return; }
     if (regs8) { ln_row_regs<T, 8>(xr, gm, bt, y, row, d, eps, lane); return; }

@@ -414,7 +414,8 @@ int ln(specdec_handle* h, const float* x, const float* g, const float* b, int cn
     if (rows_ub <= 0) return 0;
     {
         cudaError_t e = launch_pdl(h, k_layernorm<T>, dim3(cdiv(rows_ub, 8)), dim3(256), 0, st, x, g, b,
-                                   (const int*)(h->ses.counters + cnt), (T*)y, d, 1e-5f);
+                                   (const int*)(h->ses.counters + cnt), (T*)y, d, 1e-5f,
+                                   (cnt == CNT_VERIFY || cnt == CNT_ENC) ? rows_ub : -1);
         if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("layer norm launch: ") + cudaGetErrorString(e));
     }
     KCHECK(h);
