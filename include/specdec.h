@@ -239,6 +239,14 @@ int specdec_debug_cluster_round(specdec_handle* h, int cluster_size, int bytes_p
  * MMA has completed, both per MMA.  Tells a main loop that waits for operands from one the tensor pipe limits.
  * bf16 handles only.  Synchronises. */
 int specdec_debug_mma_rate(specdec_handle* h, int bn, int two_sm, int n_mma, double* h_issue_clocks, double* h_done_clocks);
+/* The same with what a real main loop adds.  bg_stages (0..6): while the MMAs are issued, another thread of every CTA
+ * keeps that many bulk copies of 16 KB in flight from global memory (the verifier's embedding table, at least 8 MB) into
+ * a separate region of the CTA's shared memory, as a TMA producer would; *h_bg_bytes_per_clock = bytes it landed per SM
+ * clock and CTA.  commit_every (0 = never, else): a tcgen05.commit after every k-block of four MMAs to a barrier nobody
+ * waits on (the multicast form for two-SM tiles), as a main loop issues one.  Tells whether the producer's writes or
+ * the commits slow the tensor pipe down.  Synchronises. */
+int specdec_debug_mma_rate_bg(specdec_handle* h, int bn, int two_sm, int n_mma, int bg_stages, int commit_every,
+                              double* h_issue_clocks, double* h_done_clocks, double* h_bg_bytes_per_clock);
 
 /* Scripted drafts, a benchmark / test hook with no counterpart in the paper: random-init
  * models almost never agree, so a workload's acceptance pattern is imposed instead.  After the

@@ -25,7 +25,7 @@ EXPORTS = [
     "specdec_accept_scan", "specdec_debug_logits", "specdec_debug_row_stats", "specdec_set_option",
     "specdec_launch_count", "specdec_last_error", "specdec_set_draft_script", "specdec_profile_read",
     "specdec_accept_scan_static", "specdec_debug_trace", "specdec_debug_link_cost", "specdec_debug_mma_rate", "specdec_debug_cluster_round",
-    "specdec_debug_integrity",
+    "specdec_debug_integrity", "specdec_debug_mma_rate_bg",
 ]
 
 
@@ -213,6 +213,14 @@ class SpecDec:
         a, b = C.c_double(), C.c_double()
         self._check(self._lib.specdec_debug_mma_rate(self._h, bn, 1 if two_sm else 0, n_mma, C.byref(a), C.byref(b)))
         return a.value, b.value
+
+    def mma_rate_bg(self, bn: int, two_sm: bool, n_mma: int, bg_stages: int, commit_every: int = 0):
+        """(issue clocks, completion clocks) per tcgen05.mma and the bytes per clock a background bulk-copy stream
+        landed in shared memory meanwhile; commit_every > 0 adds a tcgen05.commit after that many MMAs (diagnostics)."""
+        a, b, c = C.c_double(), C.c_double(), C.c_double()
+        self._check(self._lib.specdec_debug_mma_rate_bg(self._h, bn, 1 if two_sm else 0, n_mma, bg_stages, commit_every,
+                                                        C.byref(a), C.byref(b), C.byref(c)))
+        return a.value, b.value, c.value
 
     def cluster_round(self, cluster_size: int = 16, bytes_per_peer: int = 0, rounds: int = 64) -> float:
         """Nanoseconds per all-to-all exchange round inside one thread-block cluster (diagnostics)."""

@@ -489,34 +489,39 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(TC_BM, BN);
             int kbi = 0, i = 0;
+            int s = 0; uint32_t par = 0;                     // ring position of k-block kbi: stage and phase parity, kept incrementally
+            const bool stamps = g.trace != nullptr && blockIdx.x == 0;
             for (int t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++i) {
                 const int ab = i & 1;
                 if (i >= 2) mbar_wait(smem_u32(&bar_acc_empty[ab]), ((i >> 1) - 1) & 1, abort_flag, err_word, 4);
                 tc_fence_after();
                 const uint32_t acc = tmem_d + ab * BN;
-                // The tensor pipe accepts one MMA at a time from this thread, so whatever the thread does between
-                // two k-blocks is time the pipe idles: the barrier of the NEXT stage is tested before the MMAs of
-                // this one are issued (its latency hides behind them), and the loop carries nothing else.
-                bool ok = mbar_wait(smem_u32(&bar_full[kbi % STAGES]), (kbi / STAGES) & 1, abort_flag, err_word, 2);
-                if (kbi == 0) tc_stamp(g.trace, 4);
+                // The tensor pipe takes one MMA at a time from this thread and the thread stalls in each issue until the
+                // pipe accepts it, so whatever the thread does BETWEEN two issues is free while whatever it does between
+                // the last MMA of a k-block and the first of the next leaves the pipe idle (measured: ~300 clocks of
+                // bookkeeping per MMA throttle the pipe to exactly that).  All bookkeeping for the next k-block -- its
+                // ring position, descriptors and the test of its barrier -- therefore sits between this k-block's issues.
+                bool ok = mbar_wait(smem_u32(&bar_full[s]), par, abort_flag, err_word, 2);
+                if (stamps && kbi == 0) tc_stamp(g.trace, 4);
                 for (int kb = 0; kb < nkb && ok; ++kb, ++kbi) {
-                    const int s = kbi % STAGES;
-                    const int sn = (kbi + 1) % STAGES;
-                    const uint32_t next_bar = smem_u32(&bar_full[sn]), next_par = ((kbi + 1) / STAGES) & 1;
-                    const bool more = kb + 1 < nkb;
-                    const uint32_t early_ok = more ? mbar_try_wait(next_bar, next_par) : 1u;
-                    if (kbi < 16) tc_stamp(g.trace, 40 + kbi);          // landing cadence of the first k-blocks
                     const uint32_t a_src = tiles + s * Cfg::STAGE_BYTES, w_src = a_src + A_BYTES;
                     const uint64_t ad = umma_desc_k_sw128(a_src), wd = umma_desc_k_sw128(w_src);
-#pragma unroll
-                    for (int k4 = 0; k4 < TC_BK / 16; ++k4)      // +32 bytes along K per instruction: 2 address units
-                        umma_bf16(acc, ad + (uint64_t)(k4 * 2), wd + (uint64_t)(k4 * 2), idesc, (kb | k4) ? 1u : 0u);
+                    umma_bf16(acc, ad, wd, idesc, kb ? 1u : 0u);
+                    int sn = s + 1; uint32_t parn = par;
+                    if (sn == STAGES) { sn = 0; parn ^= 1u; }
+                    const uint32_t next_bar = smem_u32(&bar_full[sn]);
+                    umma_bf16(acc, ad + 2, wd + 2, idesc, 1u);       // +32 bytes along K per instruction: 2 address units
+                    const uint32_t early_ok = (kb + 1 < nkb) ? mbar_try_wait(next_bar, parn) : 1u;
+                    umma_bf16(acc, ad + 4, wd + 4, idesc, 1u);
+                    if (stamps && kbi < 16) tc_stamp(g.trace, 40 + kbi);          // landing cadence of the first k-blocks
+                    umma_bf16(acc, ad + 6, wd + 6, idesc, 1u);
                     umma_commit(smem_u32(&bar_empty[s]));        // stage reusable once these MMAs have read it
-                    if (!early_ok) ok = mbar_wait(next_bar, next_par, abort_flag, err_word, 2);
+                    if (!early_ok) ok = mbar_wait(next_bar, parn, abort_flag, err_word, 2);
+                    s = sn; par = parn;
                 }
                 if (!ok) break;
                 umma_commit(smem_u32(&bar_acc_full[ab]));        // accumulator of this tile complete
-                tc_stamp(g.trace, 5 + (i > 0));
+                if (stamps) tc_stamp(g.trace, 5 + (i > 0));
             }
         }
     } else {

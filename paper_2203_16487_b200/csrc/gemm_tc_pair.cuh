@@ -155,28 +155,34 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0 && leader) {
             constexpr uint32_t idesc = umma_idesc_bf16(2 * TC_BM, BN);
             int kbi = 0, i = 0;
+            int s = 0; uint32_t par = 0;                      // ring position kept incrementally; bookkeeping between the issues (see k_gemm_tc)
+            const bool stamps = g.trace != nullptr && blockIdx.x == 0;
             for (int t = pair; t < total && !*abort_flag; t += pairs, ++i) {
                 const int ab = i & 1;
                 if (i >= 2) mbar_wait(smem_u32(&bar_acc_empty[ab]), ((i >> 1) - 1) & 1, abort_flag, err_word, 4);
                 tc_fence_after();
                 const uint32_t acc = tmem_d + ab * BN;
-                bool ok = mbar_wait(smem_u32(&bar_full[kbi % STAGES]), (kbi / STAGES) & 1, abort_flag, err_word, 2);
-                if (kbi == 0) tc_stamp(g.trace, 4);
-                for (int kb = 0; kb < nkb && ok; ++kb, ++kbi) {   // next stage's barrier is tested before this stage's MMAs
-                    const int s = kbi % STAGES, sn = (kbi + 1) % STAGES;
-                    const uint32_t next_bar = smem_u32(&bar_full[sn]), next_par = ((kbi + 1) / STAGES) & 1;
-                    const uint32_t early_ok = (kb + 1 < nkb) ? mbar_try_wait(next_bar, next_par) : 1u;
+                bool ok = mbar_wait(smem_u32(&bar_full[s]), par, abort_flag, err_word, 2);
+                if (stamps && kbi == 0) tc_stamp(g.trace, 4);
+                for (int kb = 0; kb < nkb && ok; ++kb, ++kbi) {
                     const uint32_t a_src = tiles + s * Cfg::STAGE_BYTES, w_src = a_src + A_BYTES;
                     const uint64_t ad = umma_desc_k_sw128(a_src), wd = umma_desc_k_sw128(w_src);
-#pragma unroll
-                    for (int k4 = 0; k4 < TC_BK / 16; ++k4)
-                        umma_bf16_pair(acc, ad + (uint64_t)(k4 * 2), wd + (uint64_t)(k4 * 2), idesc, (kb | k4) ? 1u : 0u);
+                    umma_bf16_pair(acc, ad, wd, idesc, kb ? 1u : 0u);
+                    int sn = s + 1; uint32_t parn = par;
+                    if (sn == STAGES) { sn = 0; parn ^= 1u; }
+                    const uint32_t next_bar = smem_u32(&bar_full[sn]);
+                    umma_bf16_pair(acc, ad + 2, wd + 2, idesc, 1u);
+                    const uint32_t early_ok = (kb + 1 < nkb) ? mbar_try_wait(next_bar, parn) : 1u;
+                    umma_bf16_pair(acc, ad + 4, wd + 4, idesc, 1u);
+                    if (stamps && kbi < 16) tc_stamp(g.trace, 40 + kbi);
+                    umma_bf16_pair(acc, ad + 6, wd + 6, idesc, 1u);
                     umma_commit_pair(smem_u32(&bar_empty[s]));       // both CTAs may refill the stage
-                    if (!early_ok) ok = mbar_wait(next_bar, next_par, abort_flag, err_word, 2);
+                    if (!early_ok) ok = mbar_wait(next_bar, parn, abort_flag, err_word, 2);
+                    s = sn; par = parn;
                 }
                 if (!ok) break;
                 umma_commit_pair(smem_u32(&bar_acc_full[ab]));       // both CTAs' halves of the accumulator are complete
-                tc_stamp(g.trace, 5 + (i > 0));
+                if (stamps) tc_stamp(g.trace, 5 + (i > 0));
             }
         }
     } else {
@@ -295,6 +301,8 @@ k_vocab_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         if (lane == 0 && leader) {
             constexpr uint32_t idesc = umma_idesc_bf16(2 * TC_BM, VP_BN);
             int kbi = 0, i = 0, a_uses = 0, cur_m = -1;
+            int s = 0; uint32_t par = 0;                      // ring position kept incrementally; bookkeeping between the issues (see k_gemm_tc)
+            const bool stamps = g.trace != nullptr && blockIdx.x == 0;
             for (int t = t_begin; t < t_end && !*abort_flag; ++t, ++i) {
                 const int ab = i & 1, m_pair = t / n_tiles;
                 if (i >= 2) mbar_wait(smem_u32(&bar_acc_empty[ab]), ((i >> 1) - 1) & 1, abort_flag, err_word, 4);
@@ -305,24 +313,27 @@ k_vocab_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 if (*abort_flag) break;
                 tc_fence_after();
                 const uint32_t acc = tmem_d + ab * VP_BN;
-                bool ok = mbar_wait(smem_u32(&bar_w_full[kbi % stages]), (kbi / stages) & 1, abort_flag, err_word, 2);
-                if (kbi == 0) tc_stamp(g.trace, 4);
-                for (int kb = 0; kb < nkb && ok; ++kb, ++kbi) {   // next stage's barrier is tested before this stage's MMAs
-                    const int s = kbi % stages, sn = (kbi + 1) % stages;
-                    const uint32_t next_bar = smem_u32(&bar_w_full[sn]), next_par = ((kbi + 1) / stages) & 1;
-                    const uint32_t early_ok = (kb + 1 < nkb) ? mbar_try_wait(next_bar, next_par) : 1u;
-                    if (kbi < 16) tc_stamp(g.trace, 40 + kbi);
+                bool ok = mbar_wait(smem_u32(&bar_w_full[s]), par, abort_flag, err_word, 2);
+                if (stamps && kbi == 0) tc_stamp(g.trace, 4);
+                for (int kb = 0; kb < nkb && ok; ++kb, ++kbi) {
                     const uint64_t ad = umma_desc_k_sw128(a_base + kb * VP_KB_BYTES), wd = umma_desc_k_sw128(w_base + s * VP_KB_BYTES);
-#pragma unroll
-                    for (int k4 = 0; k4 < TC_BK / 16; ++k4)
-                        umma_bf16_pair(acc, ad + (uint64_t)(k4 * 2), wd + (uint64_t)(k4 * 2), idesc, (kb | k4) ? 1u : 0u);
+                    umma_bf16_pair(acc, ad, wd, idesc, kb ? 1u : 0u);
+                    int sn = s + 1; uint32_t parn = par;
+                    if (sn == stages) { sn = 0; parn ^= 1u; }
+                    const uint32_t next_bar = smem_u32(&bar_w_full[sn]);
+                    umma_bf16_pair(acc, ad + 2, wd + 2, idesc, 1u);
+                    const uint32_t early_ok = (kb + 1 < nkb) ? mbar_try_wait(next_bar, parn) : 1u;
+                    umma_bf16_pair(acc, ad + 4, wd + 4, idesc, 1u);
+                    if (stamps && kbi < 16) tc_stamp(g.trace, 40 + kbi);
+                    umma_bf16_pair(acc, ad + 6, wd + 6, idesc, 1u);
                     umma_commit_pair(smem_u32(&bar_w_empty[s]));
-                    if (!early_ok) ok = mbar_wait(next_bar, next_par, abort_flag, err_word, 2);
+                    if (!early_ok) ok = mbar_wait(next_bar, parn, abort_flag, err_word, 2);
+                    s = sn; par = parn;
                 }
                 if (!ok) break;
                 if (t + 1 == t_end || (t + 1) / n_tiles != m_pair) umma_commit_pair(smem_u32(&bar_a_empty));   // rows may be replaced
                 umma_commit_pair(smem_u32(&bar_acc_full[ab]));
-                tc_stamp(g.trace, 5 + (i > 0));
+                if (stamps) tc_stamp(g.trace, 5 + (i > 0));
             }
         }
     } else {

@@ -1918,26 +1918,39 @@ int specdec_debug_cluster_round(specdec_handle* h, int cluster_size, int bytes_p
     return SPECDEC_OK;
 }
 
-int specdec_debug_mma_rate(specdec_handle* h, int bn, int two_sm, int n_mma, double* h_issue_clocks, double* h_done_clocks) {
-    if (!h || !h_issue_clocks || !h_done_clocks || n_mma < 16 || n_mma > (1 << 20)) return SPECDEC_ERR_INVALID_ARG;
+int specdec_debug_mma_rate_bg(specdec_handle* h, int bn, int two_sm, int n_mma, int bg_stages, int commit_every, double* h_issue_clocks,
+                              double* h_done_clocks, double* h_bg_bytes_per_clock) {
+    if (!h || !h_issue_clocks || !h_done_clocks || n_mma < 16 || n_mma > (1 << 20) || bg_stages < 0 || bg_stages > 6 || commit_every < 0) return SPECDEC_ERR_INVALID_ARG;
     if (h->dtype != SPECDEC_DTYPE_BF16 || !h->tma.ready) return fail(h, SPECDEC_ERR_UNSUPPORTED, "mma rate: needs a bf16 handle on an sm_100 device");
     cudaStream_t st = h->own_stream;
-    long long* scratch = reinterpret_cast<long long*>(h->part);          // (the vocabulary partials: at least 2 x 148 words)
+    long long* scratch = reinterpret_cast<long long*>(h->part);          // (the vocabulary partials: at least 4 x 148 words)
     int* errw = h->ses.counters + 7;
+    // the background stream reads the verifier's embedding table (any resident bytes will do)
+    const void* src = h->ver.embed;
+    const long long window = (long long)h->cfg.verifier.vocab * h->cfg.verifier.d_model * 2 / 16384 * 16384;
+    if (bg_stages > 0 && window < (8ll << 20)) return fail(h, SPECDEC_ERR_UNSUPPORTED, "mma rate: the background stream needs an embedding table of at least 8 MB");
+    double bg = 0.0;
     cudaError_t e;
+#define RATE(BN_, PAIR_) e = sd::mma_rate_run<BN_, PAIR_>(h->tma.n_sm, n_mma, scratch, errw, st, h_issue_clocks, h_done_clocks, src, bg_stages, window, &bg, commit_every)
     if (two_sm) {
-        if (bn == 128) e = sd::mma_rate_run<128, true>(h->tma.n_sm, n_mma, scratch, errw, st, h_issue_clocks, h_done_clocks);
-        else if (bn == 256) e = sd::mma_rate_run<256, true>(h->tma.n_sm, n_mma, scratch, errw, st, h_issue_clocks, h_done_clocks);
+        if (bn == 128) RATE(128, true);
+        else if (bn == 256) RATE(256, true);
         else return fail(h, SPECDEC_ERR_INVALID_ARG, "mma rate: two-SM tiles are 128 or 256 columns wide");
     } else {
-        if (bn == 64) e = sd::mma_rate_run<64, false>(h->tma.n_sm, n_mma, scratch, errw, st, h_issue_clocks, h_done_clocks);
-        else if (bn == 128) e = sd::mma_rate_run<128, false>(h->tma.n_sm, n_mma, scratch, errw, st, h_issue_clocks, h_done_clocks);
-        else if (bn == 256) e = sd::mma_rate_run<256, false>(h->tma.n_sm, n_mma, scratch, errw, st, h_issue_clocks, h_done_clocks);
+        if (bn == 64) RATE(64, false);
+        else if (bn == 128) RATE(128, false);
+        else if (bn == 256) RATE(256, false);
         else return fail(h, SPECDEC_ERR_INVALID_ARG, "mma rate: tiles are 64, 128 or 256 columns wide");
     }
+#undef RATE
     if (e != cudaSuccess) return fail(h, SPECDEC_ERR_CUDA, std::string("mma rate: ") + cudaGetErrorString(e));
+    if (h_bg_bytes_per_clock) *h_bg_bytes_per_clock = bg;
     h->launches += 2;
     return SPECDEC_OK;
+}
+
+int specdec_debug_mma_rate(specdec_handle* h, int bn, int two_sm, int n_mma, double* h_issue_clocks, double* h_done_clocks) {
+    return specdec_debug_mma_rate_bg(h, bn, two_sm, n_mma, 0, 0, h_issue_clocks, h_done_clocks, nullptr);
 }
 
 int specdec_debug_row_stats(specdec_handle* h, float* d_stats, void* stream) {

@@ -145,10 +145,16 @@ def main():
     args = ap.parse_args()
     if args.mma_rate:
         wl = W.config1_tiny()
-        dims = W.ModelDims(128, 2, 512, 2000, 1, 1, 64)
+        dims = W.ModelDims(128, 2, 512, 32768, 1, 1, 64)       # (an 8 MB embedding table: the source of the background stream)
         wv, wd = W.make_weights(dims, 1, True), W.make_weights(dims, 2, True)
         sd = binding.SpecDec(dims, wv, dims, wd, k_max=8, max_batch=32, max_src=16, max_tgt=16, bf16=True)
         rows = []
+        loaded = []       # the same MMAs with what a main loop adds: a commit per k-block, a producer's writes into shared memory
+        for bn, two in ((128, False), (256, False), (256, True)):
+            for bg in (0, 1, 2, 3, 4, 6):
+                issue, done, bpc = sd.mma_rate_bg(bn, two, 8192, bg, 1)
+                loaded.append({"M": 256 if two else 128, "N": bn, "two_sm": two, "commit_per_k_block": True, "bulk_copies_in_flight": bg,
+                               "completion_clocks": done, "landed_bytes_per_clock": bpc, "landed_GBs_per_sm": bpc * 1.965})
         for bn, two in ((64, False), (128, False), (256, False), (128, True), (256, True)):
             issue, done = sd.mma_rate(bn, two, 8192)
             m = 256 if two else 128
@@ -156,7 +162,7 @@ def main():
             rows.append({"M": m, "N": bn, "two_sm": two, "issue_clocks": issue, "completion_clocks": done, "nominal_clocks": ideal,
                          "fraction_of_nominal": ideal / done})
         rounds = {f"{cs} CTAs, {b} B per peer": sd.cluster_round(cs, b, 64) for cs in (8, 16) for b in (0, 2048, 4096)}
-        print(json.dumps({"step": "mma_rate", "rows": rows, "link_cost_us": {g: sd.link_cost(64, g) for g in (8, 148, 592)},
+        print(json.dumps({"step": "mma_rate", "rows": rows, "with_commits_and_background_stream": loaded, "link_cost_us": {g: sd.link_cost(64, g) for g in (8, 148, 592)},
                           "cluster_round_ns": rounds}))
         sd.close()
         return
