@@ -467,20 +467,21 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     if (warp == 0) {
         if (lane == 0) {
             int kbi = 0;                               // k-blocks issued so far, over all tiles
-            for (int t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
+            // ring position kept incrementally and the abort flag read only when a wait gave up: this thread's own
+            // instructions are part of every stage's turnaround (freed -> requested again)
+            int ps = 0; uint32_t ppar = 0; bool wrapped = false, dead = false;
+            for (int t = blockIdx.x; t < total && !dead && !*abort_flag; t += gridDim.x) {
                 const int m0 = (LNF ? t / n_tiles : t % m_tiles) * TC_BM, n0 = (LNF ? t % n_tiles : t / m_tiles) * BN;
                 for (int kb = 0; kb < nkb; ++kb, ++kbi) {
-                    const int s = kbi % STAGES;
-                    if (kbi >= STAGES) mbar_wait(smem_u32(&bar_empty[s]), ((kbi / STAGES) - 1) & 1, abort_flag, err_word, 1);
-                    if (*abort_flag) break;
-                    const uint32_t a_dst = tiles + s * Cfg::STAGE_BYTES, w_dst = a_dst + A_BYTES;
-                    const uint32_t bar = smem_u32(&bar_full[s]);
+                    if (wrapped && !mbar_wait(smem_u32(&bar_empty[ps]), ppar, abort_flag, err_word, 1)) { dead = true; break; }
+                    const uint32_t a_dst = tiles + ps * Cfg::STAGE_BYTES, w_dst = a_dst + A_BYTES;
+                    const uint32_t bar = smem_u32(&bar_full[ps]);
                     if (kbi >= pre) {
                         mbar_expect_tx(bar, Cfg::STAGE_BYTES);
                         tma_load_2d(w_dst, &tmW, kb * TC_BK, n0, bar);
                     }
                     tma_load_2d(a_dst, &tmA, kb * TC_BK, m0, bar);
-                    if (kbi == 0) tc_stamp(g.trace, 2);
+                    if (++ps == STAGES) { ps = 0; if (wrapped) ppar ^= 1u; wrapped = true; }
                 }
             }
             tc_stamp(g.trace, 3);

@@ -133,20 +133,19 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 0) {
         if (lane == 0) {
             int kbi = 0;
-            for (int t = pair; t < total && !*abort_flag; t += pairs) {
+            int ps = 0; uint32_t ppar = 0; bool wrapped = false, dead = false;   // producer's ring position (incremental: see k_vocab_pair)
+            for (int t = pair; t < total && !dead && !*abort_flag; t += pairs) {
                 const int m0 = (t % m_pairs) * 2 * TC_BM + (int)rank * TC_BM, n0 = (t / m_pairs) * BN + (int)rank * BNH;
                 for (int kb = 0; kb < nkb; ++kb, ++kbi) {
-                    const int s = kbi % STAGES;
-                    if (kbi >= STAGES) mbar_wait(smem_u32(&bar_empty[s]), ((kbi / STAGES) - 1) & 1, abort_flag, err_word, 1);
-                    if (*abort_flag) break;
-                    const uint32_t a_dst = tiles + s * Cfg::STAGE_BYTES, w_dst = a_dst + A_BYTES;
-                    const uint32_t bar = pair_map(smem_u32(&bar_full[s]), 0);
+                    if (wrapped && !mbar_wait(smem_u32(&bar_empty[ps]), ppar, abort_flag, err_word, 1)) { dead = true; break; }
+                    const uint32_t a_dst = tiles + ps * Cfg::STAGE_BYTES, w_dst = a_dst + A_BYTES;
+                    const uint32_t bar = pair_map(smem_u32(&bar_full[ps]), 0);
                     if (kbi >= pre) {
-                        if (leader) mbar_expect_tx(smem_u32(&bar_full[s]), 2 * Cfg::STAGE_BYTES);
+                        if (leader) mbar_expect_tx(smem_u32(&bar_full[ps]), 2 * Cfg::STAGE_BYTES);
                         tma_load_2d_pair(w_dst, &tmW, kb * TC_BK, n0, bar);
                     }
                     tma_load_2d_pair(a_dst, &tmA, kb * TC_BK, m0, bar);
-                    if (kbi == 0) tc_stamp(g.trace, 2);
+                    if (++ps == STAGES) { ps = 0; if (wrapped) ppar ^= 1u; wrapped = true; }
                 }
             }
             tc_stamp(g.trace, 3);
@@ -273,6 +272,7 @@ k_vocab_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     if (warp == 0) {
         if (lane == 0) {
             int kbi = 0, a_loads = 0, cur_m = -1;
+            int ps = 0; uint32_t ppar = 0; bool wrapped = false, dead = false;   // producer's ring position; ppar = parity of the empty phase awaited
             for (int t = t_begin; t < t_end && !*abort_flag; ++t) {
                 const int m_pair = t / n_tiles, n0 = (t % n_tiles) * VP_BN + (int)rank * VP_BNH;
                 if (m_pair != cur_m) {               // new row pair: replace the resident activation rows
@@ -285,15 +285,17 @@ k_vocab_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     cur_m = m_pair; ++a_loads;
                     if (a_loads == 1) tc_stamp(g.trace, 2);
                 }
+                // (ring position kept incrementally, the abort flag read only when a wait gave up: this thread's own
+                // instructions were what paced the ring -- 0.25 us per k-block with a division by the runtime stage count)
                 for (int kb = 0; kb < nkb; ++kb, ++kbi) {
-                    const int s = kbi % stages;
-                    if (kbi >= stages) mbar_wait(smem_u32(&bar_w_empty[s]), ((kbi / stages) - 1) & 1, abort_flag, err_word, 1);
-                    if (*abort_flag) break;
+                    if (wrapped && !mbar_wait(smem_u32(&bar_w_empty[ps]), ppar, abort_flag, err_word, 1)) { dead = true; break; }
                     if (kbi >= pre) {
-                        if (leader) mbar_expect_tx(smem_u32(&bar_w_full[s]), 2 * VP_KB_BYTES);
-                        tma_load_2d_pair(w_base + s * VP_KB_BYTES, &tmW, kb * TC_BK, n0, pair_map(smem_u32(&bar_w_full[s]), 0));
+                        if (leader) mbar_expect_tx(smem_u32(&bar_w_full[ps]), 2 * VP_KB_BYTES);
+                        tma_load_2d_pair(w_base + ps * VP_KB_BYTES, &tmW, kb * TC_BK, n0, pair_map(smem_u32(&bar_w_full[ps]), 0));
                     }
+                    if (++ps == stages) { ps = 0; if (wrapped) ppar ^= 1u; wrapped = true; }
                 }
+                if (dead) break;
             }
             tc_stamp(g.trace, 3);
         }
