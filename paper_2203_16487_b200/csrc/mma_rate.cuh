@@ -7,7 +7,9 @@
 // bg_stages > 0: meanwhile another thread keeps bg_stages bulk copies of 16 KB each in flight from global memory into a
 // separate region of shared memory -- what a TMA producer does to the shared memory the MMAs read from -- and the
 // bytes it landed per clock are reported beside the MMA rate.  commit_every > 0: a tcgen05.commit (to a barrier nobody
-// waits on; the multicast form for PAIR) after every k-block of four MMAs, as a main loop issues one.
+// waits on; the multicast form for PAIR) after every k-block of four MMAs, as a main loop issues one.  op_stages: how many
+// distinct resident operand stages the k-blocks walk (four without the background stream, two with it; walking two to six
+// stages measured the same rate: the pipe keeps no operands across MMAs).
 #pragma once
 #include "gemm_tc_pair.cuh"
 
@@ -15,7 +17,7 @@ namespace sd {
 
 template <int BN, bool PAIR>
 __global__ void __launch_bounds__(128, 1) k_mma_rate(int n_mma, long long* __restrict__ out_clocks, int* err_word,
-                                                     const uint8_t* __restrict__ bg_src, int bg_stages, long long bg_window, int commit_every) {
+                                                     const uint8_t* __restrict__ bg_src, int bg_stages, long long bg_window, int commit_every, int op_stages) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_done, bar_bg, bar_dummy;   // bar_dummy: target of the in-loop commits (commit_every > 0), never waited on
     __shared__ uint32_t tmem_base_s;
@@ -28,7 +30,7 @@ __global__ void __launch_bounds__(128, 1) k_mma_rate(int n_mma, long long* __res
     uint32_t rank = 0;
     if (PAIR) rank = pair_cta_rank();
     // operands: any finite bit pattern will do for timing
-    for (int i = threadIdx.x; i < 2 * STAGE / 16; i += blockDim.x)
+    for (int i = threadIdx.x; i < op_stages * STAGE / 16; i += blockDim.x)
         *reinterpret_cast<uint4*>(smem_raw + (tiles - smem_u32(smem_raw)) + (size_t)i * 16) = make_uint4(0x3c003c00u, 0x3c003c00u, 0x3c003c00u, 0x3c003c00u);
     if (threadIdx.x == 0) {
         abort_s = 0; stop_s = 0;
@@ -48,8 +50,10 @@ __global__ void __launch_bounds__(128, 1) k_mma_rate(int n_mma, long long* __res
         constexpr uint32_t idesc = umma_idesc_bf16(PAIR ? 2 * TC_BM : TC_BM, BN);
         const long long t0 = clock64();
         // k-blocks of four MMAs (64 K-elements), as the GEMM main loops issue them; optionally one commit per k-block
+        int st = 0;                                   // the k-blocks walk op_stages resident operand stages round robin
         for (int kb = 0; kb < n_mma / 4; ++kb) {
-            const uint32_t a_src = tiles + (kb & 1) * STAGE, w_src = a_src + A_BYTES;
+            const uint32_t a_src = tiles + st * STAGE, w_src = a_src + A_BYTES;
+            if (++st == op_stages) st = 0;
             const uint64_t ad = umma_desc_k_sw128(a_src), wd = umma_desc_k_sw128(w_src);
             const uint32_t acc = tmem_d + ((kb >> 1) & 1) * BN;
 #pragma unroll
@@ -73,7 +77,7 @@ __global__ void __launch_bounds__(128, 1) k_mma_rate(int n_mma, long long* __res
         stop_s = 1;
     } else if (threadIdx.x == 64 && bg_stages > 0) {
         // background stream into shared memory: batches of bg_stages x 16 KB, the next batch once this one has landed
-        const uint32_t dst0 = tiles + 2 * STAGE, bar = smem_u32(&bar_bg);
+        const uint32_t dst0 = tiles + op_stages * STAGE, bar = smem_u32(&bar_bg);
         long long off = ((long long)blockIdx.x << 20) % bg_window, batches = 0;
         if (off + (long long)bg_stages * 16384 > bg_window) off = 0;
         uint32_t ph = 0;
@@ -103,10 +107,12 @@ __global__ void __launch_bounds__(128, 1) k_mma_rate(int n_mma, long long* __res
 template <int BN, bool PAIR>
 inline cudaError_t mma_rate_run(int n_sm, int n_mma, long long* d_scratch, int* err_word, cudaStream_t st, double* issue, double* done,
                                 const void* bg_src = nullptr, int bg_stages = 0, long long bg_window = 0, double* bg_bytes_per_clock = nullptr,
-                                int commit_every = 0) {
+                                int commit_every = 0, int op_stages = 2) {
     constexpr int BNL = PAIR ? BN / 2 : BN;
     if (bg_stages < 0 || bg_stages > 6 || (bg_stages > 0 && (!bg_src || bg_window < (8ll << 20)))) return cudaErrorInvalidValue;
-    const int smem = 2 * (TC_BM * TC_BK * 2 + BNL * TC_BK * 2) + bg_stages * 16384 + 1024;
+    if (op_stages < 1) return cudaErrorInvalidValue;
+    const int smem = op_stages * (TC_BM * TC_BK * 2 + BNL * TC_BK * 2) + bg_stages * 16384 + 1024;
+    if (smem > 232448 - 1024) return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(k_mma_rate<BN, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     const int ctas = PAIR ? (n_sm / 2) * 2 : n_sm, groups = PAIR ? ctas / 2 : ctas;
@@ -117,7 +123,7 @@ inline cudaError_t mma_rate_run(int n_sm, int n_mma, long long* d_scratch, int* 
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = PAIR ? 1 : 0;
     for (int rep = 0; rep < 2; ++rep) {                           // the second run is the one that is read
-        e = cudaLaunchKernelEx(&cfg, k_mma_rate<BN, PAIR>, n_mma, d_scratch, err_word, (const uint8_t*)bg_src, bg_stages, bg_window, commit_every);
+        e = cudaLaunchKernelEx(&cfg, k_mma_rate<BN, PAIR>, n_mma, d_scratch, err_word, (const uint8_t*)bg_src, bg_stages, bg_window, commit_every, op_stages);
         if (e != cudaSuccess) return e;
     }
     std::vector<long long> hbuf(4 * groups);

@@ -1931,7 +1931,7 @@ int specdec_debug_mma_rate_bg(specdec_handle* h, int bn, int two_sm, int n_mma, 
     if (bg_stages > 0 && window < (8ll << 20)) return fail(h, SPECDEC_ERR_UNSUPPORTED, "mma rate: the background stream needs an embedding table of at least 8 MB");
     double bg = 0.0;
     cudaError_t e;
-#define RATE(BN_, PAIR_) e = sd::mma_rate_run<BN_, PAIR_>(h->tma.n_sm, n_mma, scratch, errw, st, h_issue_clocks, h_done_clocks, src, bg_stages, window, &bg, commit_every)
+#define RATE(BN_, PAIR_) e = sd::mma_rate_run<BN_, PAIR_>(h->tma.n_sm, n_mma, scratch, errw, st, h_issue_clocks, h_done_clocks, src, bg_stages, window, &bg, commit_every > 0 ? 1 : 0, bg_stages > 0 ? 2 : 4)
     if (two_sm) {
         if (bn == 128) RATE(128, true);
         else if (bn == 256) RATE(256, true);
