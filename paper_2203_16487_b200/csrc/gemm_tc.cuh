@@ -155,6 +155,47 @@ __device__ __forceinline__ void tmem_ld(uint32_t taddr, float* v) {
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// The same loads split in two, so that the next chunk's load runs under this chunk's arithmetic: tmem_ld_issue starts the
+// load, tmem_ld_done waits for every load issued so far (tcgen05.wait::ld) and names the registers as in/out operands, so no
+// use of them can be scheduled ahead of the wait.
+template <int CW>
+__device__ __forceinline__ void tmem_ld_issue(uint32_t taddr, uint32_t* r) {
+    if constexpr (CW == 32) {
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+            "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+            "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+            : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+              "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+              "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+              "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+            : "r"(taddr) : "memory");
+    } else {
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+            "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+            : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+              "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+            : "r"(taddr) : "memory");
+    }
+}
+template <int CW>
+__device__ __forceinline__ void tmem_ld_done(uint32_t* r) {
+    if constexpr (CW == 32) {
+        asm volatile("tcgen05.wait::ld.sync.aligned;"
+            : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+              "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+              "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+              "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+            : : "memory");
+    } else {
+        asm volatile("tcgen05.wait::ld.sync.aligned;"
+            : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+              "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+            : : "memory");
+    }
+}
+
 __device__ __forceinline__ void tc_cluster_sync() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
@@ -241,14 +282,30 @@ __device__ __forceinline__ void tc_epilogue_tile(const GemmArgs<bf16>& g, int R,
         float mx[4]; int arg[4]; int cnt = 0;
 #pragma unroll
         for (int u = 0; u < 4; ++u) { mx[u] = -CUDART_INF_F; arg[u] = 0x7fffffff; }
-        for (int c = 0; c < HALF / CW; ++c) {
-            tmem_ld<CW>(trow + c * CW, v);
+        // the next chunk's tensor-memory load runs under this chunk's comparisons (two register buffers)
+        uint32_t vr[2][CW];
+        tmem_ld_issue<CW>(trow, vr[0]);
 #pragma unroll
-            for (int j = 0; j < CW; ++j) {
-                const int n = n0 + c * CW + j;
-                const float x = (n >= g.N) ? -CUDART_INF_F : ((n == id) ? ld : v[j]);   // draft column: pre-pass value
-                if (x > mx[j & 3]) { mx[j & 3] = x; arg[j & 3] = n; }
-                cnt += (x > ld) ? 1 : 0;
+        for (int c = 0; c < HALF / CW; ++c) {
+            tmem_ld_done<CW>(vr[c & 1]);
+            if (c + 1 < HALF / CW) tmem_ld_issue<CW>(trow + (c + 1) * CW, vr[(c + 1) & 1]);
+            const int nb = n0 + c * CW;
+            if (nb + CW <= g.N && (unsigned)(id - nb) >= (unsigned)CW) {
+                // whole chunk inside the vocabulary and without the row's draft column: no per-element checks
+#pragma unroll
+                for (int j = 0; j < CW; ++j) {
+                    const float x = __uint_as_float(vr[c & 1][j]);
+                    if (x > mx[j & 3]) { mx[j & 3] = x; arg[j & 3] = nb + j; }
+                    cnt += (x > ld) ? 1 : 0;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < CW; ++j) {
+                    const int n = nb + j;
+                    const float x = (n >= g.N) ? -CUDART_INF_F : ((n == id) ? ld : __uint_as_float(vr[c & 1][j]));   // draft column: pre-pass value
+                    if (x > mx[j & 3]) { mx[j & 3] = x; arg[j & 3] = n; }
+                    cnt += (x > ld) ? 1 : 0;
+                }
             }
         }
         RowPart p; p.mx = mx[0]; p.arg = arg[0]; p.sum = 0.f; p.cnt = cnt;
