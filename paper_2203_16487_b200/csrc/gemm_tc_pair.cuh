@@ -216,6 +216,21 @@ inline int vp_stages(int K) {
 }
 inline size_t vp_smem(int K) { return (size_t)(K / TC_BK + vp_stages(K)) * VP_KB_BYTES + 1024; }
 
+// Work units: a unit is (row pair m, segment sg of the column tiles); pair p takes units p, p + pairs, ... with m fastest,
+// so the pairs that run together walk the SAME column tiles in the same order for different row pairs: a weight tile is
+// then fetched by many SMs of a die within a short time and served by the near half of the L2 (with one private run of
+// column tiles per pair, 23 % of the kernel's L2 traffic came from the far half and the ring landed 40 GB/s per CTA).
+__device__ __forceinline__ int vp_pick_segs(int m_pairs, int n_tiles, int pairs) {
+    int best = 1; long long best_cost = -1;
+    for (int k = 1; k <= 4; ++k) {
+        int sg = (k * pairs) / m_pairs;
+        sg = sg < 1 ? 1 : (sg > n_tiles ? n_tiles : sg);
+        const long long cost = (long long)((m_pairs * sg + pairs - 1) / pairs) * ((n_tiles + sg - 1) / sg);   // rounds x tiles per unit
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = sg; }
+    }
+    return best;
+}
+
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 k_vocab_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, GemmArgs<bf16> g,
              int* err_word, int stages) {
@@ -224,11 +239,12 @@ k_vocab_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     if (!early) pdl_wait();
     const int R = early ? g.rows_static : *g.n_rows;
     const int m_pairs = (R + 2 * TC_BM - 1) / (2 * TC_BM), n_tiles = (g.N + VP_BN - 1) / VP_BN;
-    const int total = m_pairs * n_tiles;
     const int pair = (int)blockIdx.x >> 1, pairs = (int)gridDim.x >> 1;
-    const int per = (total + pairs - 1) / pairs;     // contiguous run of tiles per pair, column tile fastest
-    const int t_begin = pair * per, t_end = min(total, t_begin + per);
-    if (t_begin >= t_end) return;                    // both CTAs of the pair leave together, before any cluster barrier
+    const int segs = m_pairs > 0 ? vp_pick_segs(m_pairs, n_tiles, pairs) : 1;
+    const int units = m_pairs * segs;
+    if (pair >= units) return;                       // both CTAs of the pair leave together, before any cluster barrier
+    // unit u: row pair u % m_pairs, column tiles [nb, ne) of segment u / m_pairs
+#define VP_UNIT(u, m, nb, ne) const int m = (u) % m_pairs, nb = (((u) / m_pairs) * n_tiles) / segs, ne = (((u) / m_pairs + 1) * n_tiles) / segs
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_w_full[VP_MAX_STAGES], bar_w_empty[VP_MAX_STAGES], bar_a_full, bar_a_empty,
@@ -259,7 +275,9 @@ k_vocab_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     int pre = 0;                                     // ring stages requested before the wait (weights only)
     if (early) {
         if (threadIdx.x == 0) {
-            const int n0 = (t_begin % n_tiles) * VP_BN + (int)rank * VP_BNH;
+            VP_UNIT(pair, m_first, nb_first, ne_first);
+            (void)m_first; (void)ne_first;
+            const int n0 = nb_first * VP_BN + (int)rank * VP_BNH;
             for (; pre < stages && pre < nkb; ++pre) {
                 if (leader) mbar_expect_tx(smem_u32(&bar_w_full[pre]), 2 * VP_KB_BYTES);
                 tma_load_2d_pair(w_base + pre * VP_KB_BYTES, &tmW, pre * TC_BK, n0, pair_map(smem_u32(&bar_w_full[pre]), 0));
@@ -271,86 +289,91 @@ k_vocab_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
     if (warp == 0) {
         if (lane == 0) {
-            int kbi = 0, a_loads = 0, cur_m = -1;
+            int kbi = 0, a_loads = 0;
             int ps = 0; uint32_t ppar = 0; bool wrapped = false, dead = false;   // producer's ring position; ppar = parity of the empty phase awaited
-            for (int t = t_begin; t < t_end && !*abort_flag; ++t) {
-                const int m_pair = t / n_tiles, n0 = (t % n_tiles) * VP_BN + (int)rank * VP_BNH;
-                if (m_pair != cur_m) {               // new row pair: replace the resident activation rows
-                    if (a_loads > 0) mbar_wait(smem_u32(&bar_a_empty), (a_loads - 1) & 1, abort_flag, err_word, 5);
-                    if (*abort_flag) break;
-                    if (leader) mbar_expect_tx(smem_u32(&bar_a_full), 2 * nkb * VP_KB_BYTES);
-                    const uint32_t abar = pair_map(smem_u32(&bar_a_full), 0);
-                    for (int kb = 0; kb < nkb; ++kb)
-                        tma_load_2d_pair(a_base + kb * VP_KB_BYTES, &tmA, kb * TC_BK, m_pair * 2 * TC_BM + (int)rank * TC_BM, abar);
-                    cur_m = m_pair; ++a_loads;
-                    if (a_loads == 1) tc_stamp(g.trace, 2);
-                }
-                // (ring position kept incrementally, the abort flag read only when a wait gave up: this thread's own
-                // instructions were what paced the ring -- 0.25 us per k-block with a division by the runtime stage count)
-                for (int kb = 0; kb < nkb; ++kb, ++kbi) {
-                    if (wrapped && !mbar_wait(smem_u32(&bar_w_empty[ps]), ppar, abort_flag, err_word, 1)) { dead = true; break; }
-                    if (kbi >= pre) {
-                        if (leader) mbar_expect_tx(smem_u32(&bar_w_full[ps]), 2 * VP_KB_BYTES);
-                        tma_load_2d_pair(w_base + ps * VP_KB_BYTES, &tmW, kb * TC_BK, n0, pair_map(smem_u32(&bar_w_full[ps]), 0));
+            for (int u = pair; u < units && !dead && !*abort_flag; u += pairs) {
+                VP_UNIT(u, m_pair, nb, ne);
+                // this unit's activation rows replace the resident ones
+                if (a_loads > 0 && !mbar_wait(smem_u32(&bar_a_empty), (a_loads - 1) & 1, abort_flag, err_word, 5)) break;
+                if (leader) mbar_expect_tx(smem_u32(&bar_a_full), 2 * nkb * VP_KB_BYTES);
+                const uint32_t abar = pair_map(smem_u32(&bar_a_full), 0);
+                for (int kb = 0; kb < nkb; ++kb)
+                    tma_load_2d_pair(a_base + kb * VP_KB_BYTES, &tmA, kb * TC_BK, m_pair * 2 * TC_BM + (int)rank * TC_BM, abar);
+                ++a_loads;
+                if (a_loads == 1) tc_stamp(g.trace, 2);
+                for (int n = nb; n < ne && !dead; ++n) {
+                    const int n0 = n * VP_BN + (int)rank * VP_BNH;
+                    for (int kb = 0; kb < nkb; ++kb, ++kbi) {
+                        if (wrapped && !mbar_wait(smem_u32(&bar_w_empty[ps]), ppar, abort_flag, err_word, 1)) { dead = true; break; }
+                        if (kbi >= pre) {
+                            if (leader) mbar_expect_tx(smem_u32(&bar_w_full[ps]), 2 * VP_KB_BYTES);
+                            tma_load_2d_pair(w_base + ps * VP_KB_BYTES, &tmW, kb * TC_BK, n0, pair_map(smem_u32(&bar_w_full[ps]), 0));
+                        }
+                        if (++ps == stages) { ps = 0; if (wrapped) ppar ^= 1u; wrapped = true; }
                     }
-                    if (++ps == stages) { ps = 0; if (wrapped) ppar ^= 1u; wrapped = true; }
                 }
-                if (dead) break;
             }
             tc_stamp(g.trace, 3);
         }
     } else if (warp == 1) {
         if (lane == 0 && leader) {
             constexpr uint32_t idesc = umma_idesc_bf16(2 * TC_BM, VP_BN);
-            int kbi = 0, i = 0, a_uses = 0, cur_m = -1;
+            int kbi = 0, i = 0, a_uses = 0;
             int s = 0; uint32_t par = 0;                      // ring position kept incrementally; bookkeeping between the issues (see k_gemm_tc)
             const bool stamps = g.trace != nullptr && blockIdx.x == 0;
-            for (int t = t_begin; t < t_end && !*abort_flag; ++t, ++i) {
-                const int ab = i & 1, m_pair = t / n_tiles;
-                if (i >= 2) mbar_wait(smem_u32(&bar_acc_empty[ab]), ((i >> 1) - 1) & 1, abort_flag, err_word, 4);
-                if (m_pair != cur_m) {
-                    mbar_wait(smem_u32(&bar_a_full), a_uses & 1, abort_flag, err_word, 6);
-                    cur_m = m_pair; ++a_uses;
+            bool ok = true;
+            for (int u = pair; u < units && ok && !*abort_flag; u += pairs) {
+                VP_UNIT(u, m_pair, nb, ne);
+                (void)m_pair;
+                ok = mbar_wait(smem_u32(&bar_a_full), a_uses & 1, abort_flag, err_word, 6);
+                ++a_uses;
+                for (int n = nb; n < ne && ok; ++n, ++i) {
+                    const int ab = i & 1;
+                    if (i >= 2) ok = mbar_wait(smem_u32(&bar_acc_empty[ab]), ((i >> 1) - 1) & 1, abort_flag, err_word, 4);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t acc = tmem_d + ab * VP_BN;
+                    ok = mbar_wait(smem_u32(&bar_w_full[s]), par, abort_flag, err_word, 2);
+                    if (stamps && kbi == 0) tc_stamp(g.trace, 4);
+                    for (int kb = 0; kb < nkb && ok; ++kb, ++kbi) {
+                        const uint64_t ad = umma_desc_k_sw128(a_base + kb * VP_KB_BYTES), wd = umma_desc_k_sw128(w_base + s * VP_KB_BYTES);
+                        umma_bf16_pair(acc, ad, wd, idesc, kb ? 1u : 0u);
+                        int sn = s + 1; uint32_t parn = par;
+                        if (sn == stages) { sn = 0; parn ^= 1u; }
+                        const uint32_t next_bar = smem_u32(&bar_w_full[sn]);
+                        umma_bf16_pair(acc, ad + 2, wd + 2, idesc, 1u);
+                        const uint32_t early_ok = (kb + 1 < nkb) ? mbar_try_wait(next_bar, parn) : 1u;
+                        umma_bf16_pair(acc, ad + 4, wd + 4, idesc, 1u);
+                        if (stamps && kbi < 16) tc_stamp(g.trace, 40 + kbi);
+                        umma_bf16_pair(acc, ad + 6, wd + 6, idesc, 1u);
+                        umma_commit_pair(smem_u32(&bar_w_empty[s]));
+                        if (!early_ok) ok = mbar_wait(next_bar, parn, abort_flag, err_word, 2);
+                        s = sn; par = parn;
+                    }
+                    if (!ok) break;
+                    if (n + 1 == ne) umma_commit_pair(smem_u32(&bar_a_empty));   // the unit's rows may be replaced
+                    umma_commit_pair(smem_u32(&bar_acc_full[ab]));
+                    if (stamps) tc_stamp(g.trace, 5 + (i > 0));
                 }
-                if (*abort_flag) break;
-                tc_fence_after();
-                const uint32_t acc = tmem_d + ab * VP_BN;
-                bool ok = mbar_wait(smem_u32(&bar_w_full[s]), par, abort_flag, err_word, 2);
-                if (stamps && kbi == 0) tc_stamp(g.trace, 4);
-                for (int kb = 0; kb < nkb && ok; ++kb, ++kbi) {
-                    const uint64_t ad = umma_desc_k_sw128(a_base + kb * VP_KB_BYTES), wd = umma_desc_k_sw128(w_base + s * VP_KB_BYTES);
-                    umma_bf16_pair(acc, ad, wd, idesc, kb ? 1u : 0u);
-                    int sn = s + 1; uint32_t parn = par;
-                    if (sn == stages) { sn = 0; parn ^= 1u; }
-                    const uint32_t next_bar = smem_u32(&bar_w_full[sn]);
-                    umma_bf16_pair(acc, ad + 2, wd + 2, idesc, 1u);
-                    const uint32_t early_ok = (kb + 1 < nkb) ? mbar_try_wait(next_bar, parn) : 1u;
-                    umma_bf16_pair(acc, ad + 4, wd + 4, idesc, 1u);
-                    if (stamps && kbi < 16) tc_stamp(g.trace, 40 + kbi);
-                    umma_bf16_pair(acc, ad + 6, wd + 6, idesc, 1u);
-                    umma_commit_pair(smem_u32(&bar_w_empty[s]));
-                    if (!early_ok) ok = mbar_wait(next_bar, parn, abort_flag, err_word, 2);
-                    s = sn; par = parn;
-                }
-                if (!ok) break;
-                if (t + 1 == t_end || (t + 1) / n_tiles != m_pair) umma_commit_pair(smem_u32(&bar_a_empty));   // rows may be replaced
-                umma_commit_pair(smem_u32(&bar_acc_full[ab]));
-                if (stamps) tc_stamp(g.trace, 5 + (i > 0));
             }
         }
     } else {
         const int q = warp & 3;
         const int half = (warp - 2) >> 2;
         int i = 0;
-        for (int t = t_begin; t < t_end; ++t, ++i) {
-            const int ab = i & 1;
-            const int m0 = (t / n_tiles) * 2 * TC_BM + (int)rank * TC_BM, n_tile = t % n_tiles;
-            tc_epilogue_tile<EPI_STATS, VP_BN>(g, R, m0, n_tile, q, half, lane, tmem_d + ab * VP_BN, nullptr,
-                                               smem_u32(&bar_acc_full[ab]), (i >> 1) & 1, abort_flag, err_word, i > 0);
-            if (lane == 0) mbar_arrive_cluster(pair_map(smem_u32(&bar_acc_empty[ab]), 0));
-            if (threadIdx.x == 64) tc_stamp(g.trace, 8 + 2 * (i > 0));
+        for (int u = pair; u < units; u += pairs) {
+            VP_UNIT(u, m_pair, nb, ne);
+            for (int n = nb; n < ne; ++n, ++i) {
+                const int ab = i & 1;
+                const int m0 = m_pair * 2 * TC_BM + (int)rank * TC_BM;
+                tc_epilogue_tile<EPI_STATS, VP_BN>(g, R, m0, n, q, half, lane, tmem_d + ab * VP_BN, nullptr,
+                                                   smem_u32(&bar_acc_full[ab]), (i >> 1) & 1, abort_flag, err_word, i > 0);
+                if (lane == 0) mbar_arrive_cluster(pair_map(smem_u32(&bar_acc_empty[ab]), 0));
+                if (threadIdx.x == 64) tc_stamp(g.trace, 8 + 2 * (i > 0));
+            }
         }
     }
+#undef VP_UNIT
     tc_fence_before();
     pair_sync();
     if (warp == 1) tmem_dealloc_pair(tmem_d, 512);
