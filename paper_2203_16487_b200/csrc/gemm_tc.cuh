@@ -459,15 +459,17 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     constexpr int STAGES = Cfg::STAGES;
     constexpr int A_BYTES = AR * TC_BK * 2;          // activation part of a stage
     if (threadIdx.x == 0) tc_stamp(g.trace, 0);
-    // With a row count known on the host the kernel can set itself up and start streaming weight tiles before
-    // its predecessor has finished (programmatic dependent launch); a device-side count must be waited for.
-    // So can a launch whose rows fit one row tile whatever their count (one_m_tile): the count is read later.
+    // The kernel sets itself up (barriers, tensor memory) and lets its successors start before its predecessor has
+    // finished (programmatic dependent launch).  With a row count known on the host, or rows that fit one row tile
+    // whatever their count (one_m_tile), it also knows its first tile and starts streaming that tile's weights; a
+    // device-side count is read after the wait.  (Requesting the first tile's weights before the wait for those
+    // launches too -- tiles numbered column tile fastest, a drain path for CTAs left without a tile -- measured no gain.)
     const bool early = g.rows_static >= 0 || g.one_m_tile;
-    if (!early) pdl_wait();
-    int R = g.rows_static >= 0 ? g.rows_static : (early ? 0 : *g.n_rows);
-    const int m_tiles = g.one_m_tile ? 1 : (R + TC_BM - 1) / TC_BM, n_tiles = (g.N + BN - 1) / BN;
-    const int total = m_tiles * n_tiles;
-    if ((int)blockIdx.x >= total) return;            // whole CTA leaves before touching barriers or tensor memory
+    int R = g.rows_static >= 0 ? g.rows_static : 0;
+    int m_tiles = g.one_m_tile ? 1 : (R + TC_BM - 1) / TC_BM;
+    const int n_tiles = (g.N + BN - 1) / BN;
+    int total = m_tiles * n_tiles;
+    if (g.rows_static >= 0 && (int)blockIdx.x >= total) return;   // (static count) whole CTA leaves before touching barriers or tensor memory
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[STAGES], bar_empty[STAGES], bar_acc_full[2], bar_acc_empty[2];
@@ -516,9 +518,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 tma_load_2d(tiles + pre * Cfg::STAGE_BYTES + A_BYTES, &tmW, pre * TC_BK, n0, bar);
             }
         }
-        pdl_launch_dependents();
-        pdl_wait();                                    // activations, residual and outputs belong to the predecessors until here
-        if (g.rows_static < 0) R = *g.n_rows;
+    }
+    pdl_launch_dependents();
+    pdl_wait();                                        // activations, residual and outputs belong to the predecessors until here
+    if (g.rows_static < 0) {
+        R = *g.n_rows;
+        if (!g.one_m_tile) m_tiles = (R + TC_BM - 1) / TC_BM;
+        total = m_tiles * n_tiles;                     // a CTA without a tile walks through its empty loops to the common exit
     }
 
     if (warp == 0) {
@@ -597,7 +603,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         }
     }
     if constexpr (LNF) {
-        if (warp >= 2) {
+        if (warp >= 2 && (int)blockIdx.x < total) {  // (a cluster without a tile exchanged nothing)
             const int q = warp & 3, half = (warp - 2) >> 2;
             const int m0 = ((int)blockIdx.x / n_tiles) * TC_BM, n_tile = (int)blockIdx.x % n_tiles;
             if (half == 0) {                         // one thread per row: the whole row's statistics, slots in a fixed order
