@@ -14,6 +14,8 @@
 #include <unordered_map>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/specdec.h"
 #include "attention_stream.cuh"
 #include "attention_tc.cuh"
@@ -1347,6 +1349,12 @@ int integrity_run(specdec_handle* h, cudaStream_t st, specdec_integrity* rep) {
     return SPECDEC_OK;
 }
 
+// A named range around every public step call, for timeline tools (header-only NVTX: no cost without a tool attached).
+struct NvtxRange {
+    explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+};
+
 // With option "debug_checks" every step call ends with the integrity check and fails when it finds something.
 int post_check(specdec_handle* h, int rc, void* stream) {
     if (rc != SPECDEC_OK || !h || !h->debug_checks) return rc;
@@ -1965,24 +1973,32 @@ int specdec_debug_row_stats(specdec_handle* h, float* d_stats, void* stream) {
 // Public step calls: the entry proper, then (option "debug_checks") the integrity check.
 int specdec_encode(specdec_handle* h, const int32_t* d_src, const int32_t* d_src_len, const int32_t* d_max_tgt, int B,
                    int S_max, void* stream) {
+    NvtxRange r("specdec_encode");
     return post_check(h, encode_entry(h, d_src, d_src_len, d_max_tgt, B, S_max, stream), stream);
 }
-int specdec_draft(specdec_handle* h, int k, int32_t* d_draft, void* stream) { return post_check(h, draft_entry(h, k, d_draft, stream), stream); }
+int specdec_draft(specdec_handle* h, int k, int32_t* d_draft, void* stream) {
+    NvtxRange r("specdec_draft");
+    return post_check(h, draft_entry(h, k, d_draft, stream), stream);
+}
 int specdec_verify(specdec_handle* h, const int32_t* d_draft, int k, int beta, float tau, int32_t* d_accepted,
                    int32_t* d_bif, void* stream) {
+    NvtxRange r("specdec_verify");
     return post_check(h, verify_entry(h, d_draft, k, beta, tau, d_accepted, d_bif, stream), stream);
 }
 int specdec_commit(specdec_handle* h, const int32_t* d_keep, const int32_t* d_next, void* stream) {
+    NvtxRange r("specdec_commit");
     return post_check(h, commit_entry(h, d_keep, d_next, stream), stream);
 }
 int specdec_generate(specdec_handle* h, const int32_t* d_src, const int32_t* d_src_len, const int32_t* d_max_tgt, int B,
                      int S_max, int k, int beta, float tau, int32_t* d_out, int out_stride, int32_t* d_out_len,
                      specdec_stats* h_stats, void* stream) {
+    NvtxRange r("specdec_generate");
     return post_check(h, generate_entry(h, d_src, d_src_len, d_max_tgt, B, S_max, k, beta, tau, d_out, out_stride, d_out_len, h_stats, stream), stream);
 }
 int specdec_generate_host(specdec_handle* h, const int32_t* h_src, const int32_t* h_src_len, const int32_t* h_max_tgt,
                           int B, int S_max, int k, int beta, float tau, int32_t* h_out, int out_stride,
                           int32_t* h_out_len, specdec_stats* h_stats, void* stream) {
+    NvtxRange r("specdec_generate_host");
     return post_check(h, generate_host_entry(h, h_src, h_src_len, h_max_tgt, B, S_max, k, beta, tau, h_out, out_stride, h_out_len, h_stats, stream), stream);
 }
 
