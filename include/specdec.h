@@ -274,6 +274,8 @@ int specdec_profile_read(specdec_handle* h, double* h_ms, long long* h_launches)
  * "sk_cluster"   0 off / 1 (default): those GEMMs run in clusters of 8 CTAs that share the normalised input rows
  *                through distributed shared memory; 2 / 3 also the GEMMs without a LayerNorm (K <= 512 / all)
  * "pair"         0/1 two-SM tensor-core tiles (cta_group::2) for GEMMs with >= 1024 rows and columns (default 0)
+ * "enc_skinny"   0 / 1 (default) / 2: the weight-streaming GEMM also serves neither / the drafter's / both encoders when a
+ *                source has at most 32 positions
  * "ln_fuse"      0/1 the LayerNorm that reads the residual stream next runs inside the residual GEMM (default 0)
  * "splitk"       0/1 residual GEMMs with K >= 1024 over few row tiles split K across a cluster (default 1)
  * "attn_rs"      0 never / 1 by rule (default) / 2 whenever the keys allow: scores stay in the MMA accumulators

@@ -124,6 +124,8 @@ struct specdec_handle {
     int zone_cap = 0, n_zones = 0, n_scan = 0;
     std::vector<std::string> scan_names;
     int debug_checks = 0;
+    int enc_skinny = 1;             // option "enc_skinny": 1 = the drafter's encoder (the longer of the two side-by-side chains) uses the weight-streaming GEMM for sources of at most 32 positions (default: 360 -> 340 us for a 29-token source), 2 = both encoders (no better: they get in each other's way), 0 = neither
+    bool enc_skinny_now = false;
     int use_ln_fuse = 0;            // option "ln_fuse": measured slower than the separate LayerNorm launch, kept for comparison
     int use_sk_cluster = 1;         // option "sk_cluster": 1 = LayerNorm-fused weight-streaming GEMMs share the normalised rows in clusters of 8; 2 = the plain ones too (measured slower)
     bool splitk_ready = false;
@@ -538,7 +540,7 @@ int gemm_once(specdec_handle* h, int epi, const void* A, int lda, const void* W,
     if (rows_ub <= 0) return 0;
     // (not in the encoders: the two encoders run side by side on two streams, and the weight-streaming kernels' 64-256
     // CTAs per launch get in each other's way there -- 440 us against 386 us with 8-32-CTA tile GEMMs for a 32-token source)
-    const bool skinny = cnt != CNT_ENC && skinny_ok<T>(h, epi, rows_ub, N, K, lnp != nullptr);
+    const bool skinny = (cnt != CNT_ENC || h->enc_skinny_now) && skinny_ok<T>(h, epi, rows_ub, N, K, lnp != nullptr);
     if (lnp && !skinny) {           // separate normalisation launch, then a plain GEMM on its output
         TRY(ln_or_fused<T>(h, lnp->x, lnp->g, lnp->b, cnt, rows_ub, h->y, K, st));
         A = h->y; lda = K;
@@ -806,6 +808,8 @@ void use_workset(specdec_handle* h, int i) {
 template <typename T>
 int encode_model(specdec_handle* h, ModelW& m, cudaStream_t st) {
     const int R = h->B * h->S_max, d = m.dm.d_model;
+    h->enc_skinny_now = h->enc_skinny == 2 || (h->enc_skinny == 1 && &m == &h->dra);
+    struct Off { specdec_handle* h; ~Off() { h->enc_skinny_now = false; } } off{h};
     TRY(embed<T>(h, m, h->rows, m.pos_enc, CNT_ENC, R, st));
     for (int l = 0; l < m.dm.enc_layers; ++l) {
         const bool last = l + 1 == m.dm.enc_layers;
@@ -1032,7 +1036,7 @@ inline void graph_key_tail(const specdec_handle* h, std::vector<long long>& key)
                         (long long)h->use_pdl, (long long)h->use_ln_fuse, (long long)h->use_sk_cluster,
                         (long long)h->use_pair, (long long)h->diag_repeat, (long long)h->use_splitk, (long long)h->attn_stream, (long long)h->attn_stream_keys, (long long)h->attn_warps, (long long)h->attn_rs,
                         (long long)h->skinny_groups, (long long)h->want_trace,
-                        (long long)(h->script_on ? 1 : 0), (long long)h->B, (long long)h->S_max, (long long)h->drafter_pc_session, (long long)(h->fuse_commit ? 1 : 0)})
+                        (long long)(h->script_on ? 1 : 0), (long long)h->B, (long long)h->S_max, (long long)h->drafter_pc_session, (long long)(h->fuse_commit ? 1 : 0), (long long)h->enc_skinny})
         key.push_back(v);
 }
 
@@ -1603,6 +1607,7 @@ int specdec_set_option(specdec_handle* h, const char* name, int value) {
     if (!strcmp(name, "tc_bn")) { h->tma.force_bn = value; return SPECDEC_OK; }
     if (!strcmp(name, "sk_cluster")) { h->use_sk_cluster = value < 0 ? 0 : value; return SPECDEC_OK; }   // 0 off, 1 LayerNorm-fused kernels, 2 + plain ones with K <= 512, 3 all
     if (!strcmp(name, "ln_fuse")) { h->use_ln_fuse = value ? 1 : 0; return SPECDEC_OK; }
+    if (!strcmp(name, "enc_skinny")) { h->enc_skinny = value < 0 ? 0 : (value > 2 ? 2 : value); return SPECDEC_OK; }
     if (!strcmp(name, "debug_checks")) { h->debug_checks = value ? 1 : 0; return SPECDEC_OK; }
     if (!strcmp(name, "poke_zone")) {                 // test hook: damage red zone `value` (an in-arena write from the host)
         if (value < 0 || value >= h->n_zones) return fail(h, SPECDEC_ERR_INVALID_ARG, "poke_zone: no such red zone");
